@@ -1,0 +1,406 @@
+/*
+ * tfe_oracle.c -- plain CPU oracle for the Engram lookup-and-inject step.
+ *
+ * TEST INFRASTRUCTURE, NOT PRODUCT CODE.  Only the tests, the smoke check and
+ * the benchmark's CPU-baseline / reference legs may build, load or call this
+ * file.  It shares no code, header, table or constant with the CUDA library
+ * and includes nothing from it.  It is written for the eye, not for speed:
+ * every function is the definition it cites, written out as loops over plain
+ * arrays, floating point in double.  The only parallelism is one optional
+ * OpenMP "parallel for" over independent query positions.
+ *
+ * What it computes (paper sections in brackets):
+ *   - trailing n-gram phrase keys of a token stream          [Sec. 2.2, Sec. 4.2]
+ *   - exact phrase match against a table of token tuples     [Sec. 4.2, two-level index]
+ *   - longest-match selection / all-match retention          [Sec. 4.2, selection policy]
+ *   - tier walk GPU / host DRAM / SSD                         [Sec. 4.3, memory hierarchy]
+ *   - aggregation  m_t = sum_i alpha_i e_i                    [Sec. 2.2 aggregation eq.; Sec. 4.2 e_phi eq.]
+ *   - gated residual injection  h'_t = h_t + g_t * m_t        [Sec. 2.2 injection eq.]
+ *   - list of matched-but-not-GPU-resident phrases            [Sec. 4.3, staged / asynchronous reads]
+ *   - insertion of fetched entries into the GPU tier          [Sec. 4.3, "inserts the entry into a faster tier"]
+ *
+ * Parity pins: every function here is pinned by tests that do not call it to
+ * produce their expected values (hand-made cases, closed forms, a library
+ * conversion routine, brute force) EXCEPT the COSINE gate away from its
+ * special cases (m = h, m = -h, m orthogonal to h, m = 0): the paper only says
+ * the gate "may be a scalar, a vector, or a learned function", so the formula
+ * g = lambda * sigmoid(cos(h, m)) is this build's own reading --
+ * COSINE gate: parity unpinned.
+ *
+ * Conventions shared by all functions
+ *   tokens        int32 [B][T] row-major.  Ids outside [0, vocab) are padding:
+ *                 an n-gram containing one matches nothing.
+ *   query index   q = b * (T - q_start) + (t - q_start), t in [q_start, T).
+ *   phrase table  phrase_tokens int32 [N][4] (unused trailing entries = -1),
+ *                 phrase_len uint8 [N]; tuples are pairwise distinct.
+ *   residency     slot_state int32 [N]: >= 0 GPU-tier slot, -1 host DRAM, -2 SSD.
+ *   rows          bf16 bit patterns (uint16) [C][d] row-major, the GPU tier.
+ *   flags         0 absent, 1 GPU hit (injected), 2 host miss, 3 SSD miss.
+ *   sel_slot      slot for a GPU hit, -1 / -2 for a miss, -3 for absent.
+ *   sel_phrase    phrase id, 0xFFFFFFFF for absent.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORC_ABSENT_PHRASE 0xFFFFFFFFu
+#define ORC_MAX_ORDERS 4
+
+enum { ORC_POLICY_LONGEST = 0, ORC_POLICY_ALL = 1 };
+enum { ORC_GATE_CONST = 0, ORC_GATE_COSINE = 1 };
+enum { ORC_HIDDEN_BF16 = 0, ORC_HIDDEN_F32 = 1 };
+
+int orc_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ------------------------------------------------------------------ bf16 */
+
+/* bf16 -> real number: a bf16 is the upper half of an IEEE binary32. */
+double orc_bf16_to_double(uint16_t b)
+{
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* real number -> nearest bf16, ties to the even significand.  bf16 has an
+ * 8-bit significand (1 implicit + 7 stored) and binary32's exponent range, so
+ * the spacing of representable values around x is 2^(e-7) with
+ * e = max(floor(log2|x|), -126). */
+uint16_t orc_bf16_from_double(double x)
+{
+    uint16_t sign = (uint16_t)(signbit(x) ? 0x8000u : 0u);
+    if (isnan(x)) return (uint16_t)(sign | 0x7FC0u);
+    double a = fabs(x);
+    if (isinf(a)) return (uint16_t)(sign | 0x7F80u);
+    if (a == 0.0) return sign;
+    int e;
+    (void)frexp(a, &e);          /* a = f * 2^e, f in [0.5, 1)  =>  floor(log2 a) = e - 1 */
+    e -= 1;
+    if (e < -126) e = -126;
+    double ulp = ldexp(1.0, e - 7);
+    double r = nearbyint(a / ulp) * ulp;   /* default rounding mode: to nearest, ties to even; a/ulp is exact */
+    if (r >= ldexp(1.0, 128)) return (uint16_t)(sign | 0x7F80u);
+    float f = (float)r;                    /* exact: r has at most 8 significant bits */
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    return (uint16_t)(sign | (uint16_t)(u >> 16));
+}
+
+/* ------------------------------------------------------- n-gram helpers */
+
+/* The trailing n-gram ending at position t of sequence b: x[b][t-n+1 .. t].
+ * Returns 0 when it would start before the sequence or contains a padding id. */
+static int trailing_ngram(const int32_t *tokens, int32_t T, int32_t b, int32_t t,
+                          int32_t n, int32_t vocab, int32_t gram[ORC_MAX_ORDERS])
+{
+    if (t - n + 1 < 0) return 0;
+    for (int32_t k = 0; k < n; ++k) {
+        int32_t x = tokens[(int64_t)b * T + (t - n + 1 + k)];
+        if (x < 0 || x >= vocab) return 0;
+        gram[k] = x;
+    }
+    return 1;
+}
+
+static int phrase_equals(const int32_t *phrase_tokens, const uint8_t *phrase_len,
+                         int64_t i, const int32_t *gram, int32_t n)
+{
+    if ((int32_t)phrase_len[i] != n) return 0;
+    for (int32_t k = 0; k < n; ++k)
+        if (phrase_tokens[i * 4 + k] != gram[k]) return 0;
+    return 1;
+}
+
+/* ------------------------------------------------ exact match, matcher O1 */
+
+/* Brute force: for every query position and every order scan all N phrases.
+ * match[q][oi] = phrase id whose tuple equals the trailing orders[oi]-gram, or -1.
+ * [Sec. 4.2: the tokenised form tau_i is what inference-time matching uses.] */
+void orc_match_brute(int64_t N, const int32_t *phrase_tokens, const uint8_t *phrase_len,
+                     const int32_t *tokens, int32_t B, int32_t T, int32_t q_start,
+                     int32_t vocab, int32_t n_orders, const int32_t *orders,
+                     int64_t *match)
+{
+    int32_t Tq = T - q_start;
+    for (int32_t b = 0; b < B; ++b)
+        for (int32_t t = q_start; t < T; ++t) {
+            int64_t q = (int64_t)b * Tq + (t - q_start);
+            for (int32_t oi = 0; oi < n_orders; ++oi) {
+                int32_t gram[ORC_MAX_ORDERS];
+                int64_t found = -1;
+                if (trailing_ngram(tokens, T, b, t, orders[oi], vocab, gram))
+                    for (int64_t i = 0; i < N; ++i)
+                        if (phrase_equals(phrase_tokens, phrase_len, i, gram, orders[oi])) {
+                            found = i;
+                            break;
+                        }
+                match[q * n_orders + oi] = found;
+            }
+        }
+}
+
+/* ------------------------------------------------ exact match, matcher O2 */
+
+/* Total order on (length, tokens): shorter first, then lexicographic. */
+static int tuple_cmp(int32_t na, const int32_t *a, int32_t nb, const int32_t *b)
+{
+    if (na != nb) return na < nb ? -1 : 1;
+    for (int32_t k = 0; k < na; ++k)
+        if (a[k] != b[k]) return a[k] < b[k] ? -1 : 1;
+    return 0;
+}
+
+typedef struct {
+    const int32_t *phrase_tokens;
+    const uint8_t *phrase_len;
+} sort_ctx;
+
+static int perm_cmp(const void *pa, const void *pb, void *vctx)
+{
+    const sort_ctx *c = (const sort_ctx *)vctx;
+    int64_t a = *(const int64_t *)pa, b = *(const int64_t *)pb;
+    return tuple_cmp(c->phrase_len[a], c->phrase_tokens + a * 4,
+                     c->phrase_len[b], c->phrase_tokens + b * 4);
+}
+
+/* perm[0..N) <- phrase ids in ascending (length, tokens) order.
+ * Returns the number of adjacent equal tuples (0 for a valid table). */
+int64_t orc_sort_phrases(int64_t N, const int32_t *phrase_tokens, const uint8_t *phrase_len,
+                         int64_t *perm)
+{
+    sort_ctx c = { phrase_tokens, phrase_len };
+    for (int64_t i = 0; i < N; ++i) perm[i] = i;
+    qsort_r(perm, (size_t)N, sizeof(int64_t), perm_cmp, &c);
+    int64_t dup = 0;
+    for (int64_t i = 1; i < N; ++i)
+        if (perm_cmp(&perm[i - 1], &perm[i], &c) == 0) ++dup;
+    return dup;
+}
+
+/* Sorted search: binary search (lower bound) for the trailing n-gram in the
+ * sorted phrase order.  Same output contract as orc_match_brute. */
+void orc_match_sorted(int64_t N, const int32_t *phrase_tokens, const uint8_t *phrase_len,
+                      const int64_t *perm,
+                      const int32_t *tokens, int32_t B, int32_t T, int32_t q_start,
+                      int32_t vocab, int32_t n_orders, const int32_t *orders,
+                      int64_t *match)
+{
+    int32_t Tq = T - q_start;
+    int64_t Q = (int64_t)B * Tq;
+#pragma omp parallel for schedule(static)
+    for (int64_t q = 0; q < Q; ++q) {
+        int32_t b = (int32_t)(q / Tq), t = (int32_t)(q % Tq) + q_start;
+        for (int32_t oi = 0; oi < n_orders; ++oi) {
+            int32_t gram[ORC_MAX_ORDERS];
+            int64_t found = -1;
+            if (trailing_ngram(tokens, T, b, t, orders[oi], vocab, gram)) {
+                int64_t lo = 0, hi = N;            /* first position whose tuple is >= gram */
+                while (lo < hi) {
+                    int64_t mid = lo + (hi - lo) / 2;
+                    int64_t i = perm[mid];
+                    if (tuple_cmp(phrase_len[i], phrase_tokens + i * 4, orders[oi], gram) < 0)
+                        lo = mid + 1;
+                    else
+                        hi = mid;
+                }
+                if (lo < N && phrase_equals(phrase_tokens, phrase_len, perm[lo], gram, orders[oi]))
+                    found = perm[lo];
+            }
+            match[q * n_orders + oi] = found;
+        }
+    }
+}
+
+/* ------------------------------------- selection, tier walk, miss hand-off */
+
+static uint8_t tier_flag(int32_t slot_state)
+{
+    if (slot_state >= 0) return 1;       /* value already in the GPU cache: usable now      */
+    if (slot_state == -1) return 2;      /* in host DRAM: must be staged to the GPU first   */
+    return 3;                            /* only on SSD: asynchronous read, insert on arrival */
+}
+
+/* From the per-order matches decide, for every query, which phrase(s) are
+ * retained [Sec. 4.2: deterministic policy, longer phrases preferred; or all
+ * matches retained] and walk the hierarchy for each [Sec. 4.3].
+ *
+ * LONGEST: outputs are [Q].  The retained phrase is the matched one of
+ *          greatest order; orders are ascending, so it is the last match.
+ * ALL:     outputs are [Q][n_orders], column oi <-> orders[oi].
+ *
+ * Every retained phrase that is not in the GPU tier is appended to the miss
+ * list (query index, phrase id, tier flag 2 or 3) in ascending (q, order);
+ * duplicates are kept.  Returns the miss count. */
+int64_t orc_select(int32_t policy, int64_t Q, int32_t n_orders, const int64_t *match,
+                   const int32_t *slot_state,
+                   uint32_t *sel_phrase, int32_t *sel_slot, uint8_t *flags,
+                   uint32_t *miss_q, uint32_t *miss_phrase, uint8_t *miss_tier)
+{
+    int64_t n_miss = 0;
+    for (int64_t q = 0; q < Q; ++q) {
+        if (policy == ORC_POLICY_LONGEST) {
+            int64_t best = -1;
+            for (int32_t oi = 0; oi < n_orders; ++oi)
+                if (match[q * n_orders + oi] >= 0) best = match[q * n_orders + oi];
+            if (best < 0) {
+                sel_phrase[q] = ORC_ABSENT_PHRASE; sel_slot[q] = -3; flags[q] = 0;
+                continue;
+            }
+            int32_t s = slot_state[best];
+            sel_phrase[q] = (uint32_t)best;
+            sel_slot[q] = s >= 0 ? s : (s == -1 ? -1 : -2);
+            flags[q] = tier_flag(s);
+            if (flags[q] != 1) {
+                miss_q[n_miss] = (uint32_t)q; miss_phrase[n_miss] = (uint32_t)best;
+                miss_tier[n_miss] = flags[q]; ++n_miss;
+            }
+        } else {
+            for (int32_t oi = 0; oi < n_orders; ++oi) {
+                int64_t k = q * n_orders + oi, i = match[k];
+                if (i < 0) {
+                    sel_phrase[k] = ORC_ABSENT_PHRASE; sel_slot[k] = -3; flags[k] = 0;
+                    continue;
+                }
+                int32_t s = slot_state[i];
+                sel_phrase[k] = (uint32_t)i;
+                sel_slot[k] = s >= 0 ? s : (s == -1 ? -1 : -2);
+                flags[k] = tier_flag(s);
+                if (flags[k] != 1) {
+                    miss_q[n_miss] = (uint32_t)q; miss_phrase[n_miss] = (uint32_t)i;
+                    miss_tier[n_miss] = flags[k]; ++n_miss;
+                }
+            }
+        }
+    }
+    return n_miss;
+}
+
+/* ------------------------------------------------ aggregation + injection */
+
+static double hidden_at(const void *h, int32_t hidden_dtype, int64_t idx)
+{
+    if (hidden_dtype == ORC_HIDDEN_F32) return (double)((const float *)h)[idx];
+    return orc_bf16_to_double(((const uint16_t *)h)[idx]);
+}
+
+/* h'_t = h_t + g_t * m_t  [Sec. 2.2 injection eq.] for every query whose
+ * retained phrase(s) include a GPU-resident one; every other query keeps h_t
+ * unchanged.
+ *
+ *   m_t  LONGEST: the row of the selected phrase.
+ *        ALL:     sum over the matched phrases that are GPU-resident of
+ *                 alpha_i * row_i, alpha_i = n_i / (sum of n_j over ALL matched
+ *                 phrases of this query, resident or not)  [Sec. 4.2 e_phi eq.;
+ *                 alpha "determined by phrase length"].
+ *   g_t  CONST:   lambda.
+ *        COSINE:  lambda * sigmoid( <h,m> / sqrt(<h,h><m,m> + 1e-12) ).
+ *
+ * sel_slot / flags are orc_select's outputs for the same policy.  out_exact
+ * (double [Q][d]) receives the unrounded value; out_rounded receives it in the
+ * hidden dtype (bf16 bits or float), rounded to nearest even.  For untouched
+ * queries out_rounded is a bitwise copy of h.  Either output may be NULL. */
+void orc_inject(int32_t policy, int32_t gate, double lambda, int64_t Q, int32_t d,
+                int32_t n_orders, const int32_t *orders,
+                const int32_t *sel_slot, const uint8_t *flags,
+                const uint16_t *rows, const void *h, int32_t hidden_dtype,
+                double *out_exact, void *out_rounded)
+{
+#pragma omp parallel
+    {
+        double *m = (double *)malloc(sizeof(double) * (size_t)d);
+#pragma omp for schedule(static)
+        for (int64_t q = 0; q < Q; ++q) {
+            int have_m = 0;
+            if (policy == ORC_POLICY_LONGEST) {
+                if (flags[q] == 1) {
+                    have_m = 1;
+                    for (int32_t j = 0; j < d; ++j)
+                        m[j] = orc_bf16_to_double(rows[(int64_t)sel_slot[q] * d + j]);
+                }
+            } else {
+                double n_sum = 0.0;
+                for (int32_t oi = 0; oi < n_orders; ++oi)
+                    if (flags[q * n_orders + oi] != 0) n_sum += (double)orders[oi];
+                for (int32_t j = 0; j < d; ++j) m[j] = 0.0;
+                for (int32_t oi = 0; oi < n_orders; ++oi) {
+                    if (flags[q * n_orders + oi] != 1) continue;
+                    have_m = 1;
+                    double alpha = (double)orders[oi] / n_sum;
+                    const uint16_t *row = rows + (int64_t)sel_slot[q * n_orders + oi] * d;
+                    for (int32_t j = 0; j < d; ++j) m[j] += alpha * orc_bf16_to_double(row[j]);
+                }
+            }
+            double g = lambda;
+            if (have_m && gate == ORC_GATE_COSINE) {
+                double s = 0.0, a = 0.0, c = 0.0;
+                for (int32_t j = 0; j < d; ++j) {
+                    double hj = hidden_at(h, hidden_dtype, q * d + j);
+                    s += hj * m[j]; a += hj * hj; c += m[j] * m[j];
+                }
+                g = lambda / (1.0 + exp(-s / sqrt(a * c + 1e-12)));
+            }
+            for (int32_t j = 0; j < d; ++j) {
+                int64_t idx = q * d + j;
+                double hj = hidden_at(h, hidden_dtype, idx);
+                double v = have_m ? hj + g * m[j] : hj;
+                if (out_exact) out_exact[idx] = v;
+                if (!out_rounded) continue;
+                if (hidden_dtype == ORC_HIDDEN_F32)
+                    ((float *)out_rounded)[idx] = have_m ? (float)v : ((const float *)h)[idx];
+                else
+                    ((uint16_t *)out_rounded)[idx] =
+                        have_m ? orc_bf16_from_double(v) : ((const uint16_t *)h)[idx];
+            }
+        }
+        free(m);
+    }
+}
+
+/* --------------------------------------------------- GPU-tier installation */
+
+/* Insert n fetched entries into the GPU tier [Sec. 4.3].  Entry k = phrase
+ * ids[k] with row src[k][0..d) goes to slot dst[k].  Preconditions (checked;
+ * on violation nothing changes and the 1-based index of the first offending
+ * check is returned as a negative number):
+ *   -1 an id is not a phrase;       -2 a phrase is already GPU-resident;
+ *   -3 a slot is outside [0, C);    -4 ids not pairwise distinct;
+ *   -5 slots not pairwise distinct.
+ * Effects, for k in order: the phrase that owned dst[k], if any, falls back to
+ * the host-DRAM tier (eviction); rows[dst[k]] <- src[k]; the phrase becomes
+ * GPU-resident at dst[k].  slot_owner int64 [C]: phrase id or -1.  Returns 0. */
+int32_t orc_cache_install(int64_t N, int64_t C, int32_t d,
+                          int32_t *slot_state, int64_t *slot_owner, uint16_t *rows,
+                          int32_t n, const uint32_t *ids, const uint16_t *src, const int32_t *dst)
+{
+    for (int32_t k = 0; k < n; ++k) {
+        if ((int64_t)ids[k] >= N) return -1;
+        if (slot_state[ids[k]] >= 0) return -2;
+        if (dst[k] < 0 || (int64_t)dst[k] >= C) return -3;
+    }
+    for (int32_t k = 0; k < n; ++k)
+        for (int32_t l = 0; l < k; ++l) {
+            if (ids[k] == ids[l]) return -4;
+            if (dst[k] == dst[l]) return -5;
+        }
+    for (int32_t k = 0; k < n; ++k) {
+        int64_t prev = slot_owner[dst[k]];
+        if (prev >= 0) slot_state[prev] = -1;
+        if (rows && src)
+            memcpy(rows + (int64_t)dst[k] * d, src + (int64_t)k * d, sizeof(uint16_t) * (size_t)d);
+        slot_state[ids[k]] = dst[k];
+        slot_owner[dst[k]] = (int64_t)ids[k];
+    }
+    return 0;
+}

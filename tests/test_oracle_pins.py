@@ -1,0 +1,455 @@
+"""Pins for the CPU oracle: every expected value here comes from the paper's
+definitions worked by hand, a closed form, a library routine, or an independent
+brute-force written in this file -- never from the oracle itself."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_07388_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bf(x):
+    """float(s) -> bf16 bit patterns via torch's float32->bfloat16 conversion (library routine)."""
+    t = torch.tensor(np.asarray(x, dtype=np.float32)).to(torch.bfloat16)
+    return t.view(torch.int16).numpy().view(np.uint16).copy()
+
+
+def unbf(b):
+    t = torch.from_numpy(np.asarray(b, dtype=np.uint16).view(np.int16).copy()).view(torch.bfloat16)
+    return t.to(torch.float64).numpy()
+
+
+def mk_oracle(orc, phrases, slots, rows, d, vocab, orders, C):
+    pt = np.full((len(phrases), 4), -1, np.int32)
+    pl = np.zeros(len(phrases), np.uint8)
+    for i, p in enumerate(phrases):
+        pt[i, :len(p)] = p
+        pl[i] = len(p)
+    return orc.Oracle(pt, pl, np.asarray(slots, np.int32), rows, d=d, vocab=vocab, orders=orders,
+                      gpu_slots=C)
+
+
+# ---------------------------------------------------------------- bf16 codec
+
+
+def test_bf16_decode_matches_library(oracle_mod):
+    bits = np.concatenate([np.arange(0, 0x7F80, 37, dtype=np.uint16),
+                           np.arange(0x8000, 0xFF80, 41, dtype=np.uint16),
+                           np.array([0, 1, 0x007F, 0x0080, 0x7F7F, 0x8000, 0x3F80], np.uint16)])
+    np.testing.assert_array_equal(oracle_mod.bf16_to_double(bits), unbf(bits))
+
+
+def test_bf16_encode_matches_library_on_float32_inputs(oracle_mod):
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.standard_normal(4000).astype(np.float32) * 3,
+                        (rng.standard_normal(500) * 1e-3).astype(np.float32),
+                        np.array([0.0, -0.0, 1.0, -1.0, 1e38, -1e38, 1e-40, 3.3895e38], np.float32)])
+    # exact ties between two bf16 neighbours: odd and even significands
+    ties = np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -(2.0 + 2.0 ** -7), 0.75 + 2.0 ** -9], np.float32)
+    x = np.concatenate([x, ties])
+    np.testing.assert_array_equal(oracle_mod.bf16_from_double(x.astype(np.float64)), bf(x))
+
+
+def test_bf16_encode_rounds_the_real_number_not_its_float32(oracle_mod):
+    # 1 + 2^-8 is a tie (-> 1.0, even); a hair above it must go up, a hair below it down,
+    # even though float32 cannot tell them from the tie.
+    up = oracle_mod.bf16_from_double(np.array([1.0 + 2.0 ** -8 + 2.0 ** -40]))
+    dn = oracle_mod.bf16_from_double(np.array([1.0 + 2.0 ** -8 - 2.0 ** -40]))
+    assert unbf(up)[0] == 1.0 + 2.0 ** -7
+    assert unbf(dn)[0] == 1.0
+    # overflow, subnormals, signed zero
+    assert oracle_mod.bf16_from_double(np.array([1e39]))[0] == 0x7F80
+    assert oracle_mod.bf16_from_double(np.array([-1e39]))[0] == 0xFF80
+    assert oracle_mod.bf16_from_double(np.array([2.0 ** -133]))[0] == 0x0001
+    assert oracle_mod.bf16_from_double(np.array([2.0 ** -135]))[0] == 0x0000
+    assert oracle_mod.bf16_from_double(np.array([-0.0]))[0] == 0x8000
+
+
+# ------------------------------------------------- exact match and selection
+
+
+def _load_worked():
+    rows = []
+    with open(os.path.join(GOLDEN, "worked_lookup.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            rows.append([int(v) for v in line.split()])
+    return np.array(rows)
+
+
+WORKED_PHRASES = [(11, 12), (10, 11, 12), (12, 13), (13, 14), (12, 13, 14), (14, 14)]
+WORKED_SLOTS = [3, 0, -1, -2, 2, 1]
+WORKED_STREAM = [[10, 11, 12, 13, 14, 14, 99, 14, 14]]
+
+
+@pytest.mark.parametrize("matcher", ["brute", "sorted"])
+def test_worked_lookup_longest_and_all(oracle_mod, matcher):
+    g = _load_worked()
+    o = mk_oracle(oracle_mod, WORKED_PHRASES, WORKED_SLOTS, np.zeros((4, 8), np.uint16), 8, 100,
+                  [2, 3], 4)
+    tok = np.array(WORKED_STREAM, np.int32)
+    r = o.lookup(tok, 0, oracle_mod.POLICY_LONGEST, matcher)
+    np.testing.assert_array_equal(r.match, g[:, 1:3])
+    np.testing.assert_array_equal(r.sel_phrase.astype(np.int64),
+                                  np.where(g[:, 3] < 0, 0xFFFFFFFF, g[:, 3]))
+    np.testing.assert_array_equal(r.sel_slot, g[:, 4])
+    np.testing.assert_array_equal(r.flags, g[:, 5])
+    assert list(zip(r.miss_q, r.miss_phrase, r.miss_tier)) == [(3, 2, 2)]
+    ra = o.lookup(tok, 0, oracle_mod.POLICY_ALL, matcher)
+    assert list(zip(ra.miss_q, ra.miss_phrase, ra.miss_tier)) == [(3, 2, 2), (4, 3, 3)]
+    assert ra.flags.tolist()[4] == [3, 1] and ra.sel_slot.tolist()[4] == [-2, 2]
+    assert ra.flags.tolist()[2] == [1, 1] and ra.sel_phrase.tolist()[2] == [0, 1]
+
+
+def test_q_start_sequence_start_and_padding(oracle_mod):
+    # two sequences; an n-gram never crosses the start of its own sequence, ids outside
+    # [0, vocab) break every n-gram that contains them; ids 0 and vocab-1 are ordinary tokens.
+    V = 50
+    phrases = [(0, 49), (49, 0, 49), (7, 7), (7, 7, 7), (49, 7)]
+    o = mk_oracle(oracle_mod, phrases, [0, 1, 2, 3, 4], np.zeros((5, 8), np.uint16), 8, V, [2, 3], 5)
+    tok = np.array([[49, 0, 49, 7, 7, 7, 7],
+                    [7, 7, -1, 7, 7, 50, 49]], np.int32)
+    r = o.lookup(tok, 0)
+    # seq 0: t0 none | t1 (49,0) none | t2 (0,49)->0,(49,0,49)->1 | t3 (49,7)->4 | t4 (7,7)->2 |
+    #        t5 (7,7)->2,(7,7,7)->3 | t6 same
+    # seq 1: t0 none (the 49 7 of the previous row must not leak) | t1 (7,7)->2 | t2 pad | t3 pad in gram |
+    #        t4 (7,7)->2 ; 3-gram holds the pad | t5 pad(50) | t6 pad in gram
+    exp = [-1, -1, 1, 4, 2, 3, 3, -1, 2, -1, -1, 2, -1, -1]
+    np.testing.assert_array_equal(r.sel_phrase.astype(np.int64), np.where(np.array(exp) < 0, 0xFFFFFFFF, exp))
+    # q_start = 4 keeps only t in [4, 7) of each sequence, numbered b*3 + (t-4)
+    r2 = o.lookup(tok, 4)
+    np.testing.assert_array_equal(r2.sel_phrase.astype(np.int64),
+                                  np.where(np.array(exp[4:7] + exp[11:14]) < 0, 0xFFFFFFFF,
+                                           exp[4:7] + exp[11:14]))
+
+
+def _dict_matcher(phrases, tok, q_start, vocab, orders):
+    """Independent matcher: python dict keyed by the token tuple."""
+    table = {tuple(int(x) for x in p): i for i, p in enumerate(phrases)}
+    B, T = tok.shape
+    out = []
+    for b in range(B):
+        for t in range(q_start, T):
+            row = []
+            for n in orders:
+                g = tuple(int(x) for x in tok[b, t - n + 1:t + 1]) if t - n + 1 >= 0 else ()
+                ok = len(g) == n and all(0 <= x < vocab for x in g)
+                row.append(table.get(g, -1) if ok else -1)
+            out.append(row)
+    return np.array(out, np.int64)
+
+
+@pytest.mark.parametrize("seed,orders", [(1, [2, 3]), (2, [1, 2, 3, 4]), (3, [2, 4]), (4, [3])])
+def test_matchers_agree_with_dict_brute_force(oracle_mod, seed, orders):
+    # tiny alphabet so that phrases share prefixes/suffixes, nest inside each other and
+    # differ from stream n-grams in exactly one token all the time
+    rng = np.random.default_rng(seed)
+    V = 6
+    phrases = set()
+    target = min(300, sum(V ** n for n in orders) // 2)
+    while len(phrases) < target:
+        n = int(rng.choice(orders))
+        phrases.add(tuple(int(x) for x in rng.integers(0, V, n)))
+    phrases = sorted(phrases, key=lambda p: rng.random())
+    slots = rng.permutation(len(phrases)).astype(np.int32)
+    o = mk_oracle(oracle_mod, phrases, slots, np.zeros((len(phrases), 8), np.uint16), 8, V, orders,
+                  len(phrases))
+    tok = rng.integers(-1, V + 1, size=(5, 40)).astype(np.int32)
+    for q_start in (0, 3, 39):
+        exp = _dict_matcher(phrases, tok, q_start, V, orders)
+        np.testing.assert_array_equal(o.match(tok, q_start, "brute"), exp)
+        np.testing.assert_array_equal(o.match(tok, q_start, "sorted"), exp)
+
+
+def test_duplicate_tuple_is_refused(oracle_mod):
+    o = mk_oracle(oracle_mod, [(1, 2), (3, 4, 5), (1, 2)], [0, 1, 2], np.zeros((3, 8), np.uint16), 8,
+                  10, [2, 3], 3)
+    with pytest.raises(ValueError):
+        o.sorted_perm()
+
+
+# ----------------------------------------------------------------- injection
+
+
+def _one_hit_oracle(oracle_mod, row_vals, d=8, slot=1, C=3, state=None):
+    rows = np.zeros((C, d), np.uint16)
+    rows[slot] = bf(row_vals)
+    o = mk_oracle(oracle_mod, [(1, 2)], [slot if state is None else state], rows, d, 10, [2], C)
+    tok = np.array([[1, 2, 3]], np.int32)      # q0 absent (no 2-gram), q1 hit, q2 absent
+    return o, tok
+
+
+def test_injection_equation_by_hand(oracle_mod):
+    d = 8
+    row = [0.5, -0.25, 2.0, 0.0, 1.0, 2.0 ** -8, 3 * 2.0 ** -8, -1.5]
+    o, tok = _one_hit_oracle(oracle_mod, row)
+    hval = np.array([[9, 9, 9, 9, 9, 9, 9, 9],
+                     [1.0, 1.0, -4.0, 0.75, -1.0, 1.0, 1.0, 0.5],
+                     [7, 7, 7, 7, 7, 7, 7, 7]], np.float32)
+    h = bf(hval)
+    r = o.lookup(tok)
+    assert r.flags.tolist() == [0, 1, 0]
+    exact, rounded = o.inject(r, h, lam=1.0)
+    # h + 1.0 * row, real numbers
+    np.testing.assert_array_equal(exact[1], [1.5, 0.75, -2.0, 0.75, 0.0, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -1.0])
+    # bf16: 1+2^-8 is a tie -> even (1.0); 1+3*2^-8 is a tie -> even (1+2^-6)
+    np.testing.assert_array_equal(unbf(rounded[1]), [1.5, 0.75, -2.0, 0.75, 0.0, 1.0, 1.0 + 2.0 ** -6, -1.0])
+    # rows 0 and 2: absent -> bitwise h
+    np.testing.assert_array_equal(rounded[[0, 2]], h[[0, 2]])
+    np.testing.assert_array_equal(exact[[0, 2]], hval[[0, 2]].astype(np.float64))
+    # lambda = 0.25
+    exact, rounded = o.inject(r, h, lam=0.25)
+    np.testing.assert_array_equal(exact[1, :5], [1.125, 0.9375, -3.5, 0.75, -0.75])
+
+
+def test_injection_closed_forms(oracle_mod):
+    rng = np.random.default_rng(5)
+    d = 64
+    m = rng.standard_normal(d).astype(np.float32)
+    o, tok = _one_hit_oracle(oracle_mod, m, d=d)
+    r = o.lookup(tok)
+    h = bf(rng.standard_normal((3, d)))
+    # lambda = 0: identity, bitwise
+    _, out = o.inject(r, h, lam=0.0)
+    np.testing.assert_array_equal(out, h)
+    # h = 0, lambda = 2^k: out = 2^k * m exactly (a power-of-two scaling of a bf16 is a bf16)
+    z = np.zeros_like(h)
+    for k in (-3, 0, 4):
+        _, out = o.inject(r, z, lam=2.0 ** k)
+        np.testing.assert_array_equal(unbf(out[1]), unbf(bf(m)) * 2.0 ** k)
+    # m = h, lambda = 1: out = 2h exactly
+    hh = np.stack([h[0], bf(m), h[2]])
+    _, out = o.inject(r, hh, lam=1.0)
+    np.testing.assert_array_equal(unbf(out[1]), 2 * unbf(bf(m)))
+    # all-zero rows: identity
+    o0, _ = _one_hit_oracle(oracle_mod, np.zeros(d), d=d)
+    _, out = o0.inject(o0.lookup(tok), h, lam=3.0)
+    np.testing.assert_array_equal(unbf(out), unbf(h))
+    # matched but not GPU-resident: identity, bitwise, and listed as a miss
+    for state, tier in ((-1, 2), (-2, 3)):
+        om, _ = _one_hit_oracle(oracle_mod, m, d=d, state=state)
+        rm = om.lookup(tok)
+        _, out = om.inject(rm, h, lam=1.0)
+        np.testing.assert_array_equal(out, h)
+        assert list(zip(rm.miss_q, rm.miss_phrase, rm.miss_tier)) == [(1, 0, tier)]
+        assert rm.sel_slot.tolist() == [-3, state, -3]
+
+
+def test_injection_fp32_hidden(oracle_mod):
+    d = 8
+    row = [0.5, -0.25, 2.0, 0.0, 1.0, 0.1, 0.2, -1.5]
+    o, tok = _one_hit_oracle(oracle_mod, row)
+    h = np.linspace(-1, 1, 3 * d).astype(np.float32).reshape(3, d)
+    r = o.lookup(tok)
+    exact, out = o.inject(r, h, lam=0.3, hidden_dtype=oracle_mod.HIDDEN_F32)
+    want = h[1].astype(np.float64) + 0.3 * unbf(bf(row))
+    np.testing.assert_allclose(exact[1], want, rtol=0, atol=1e-15)
+    np.testing.assert_array_equal(out[1], want.astype(np.float32))
+    np.testing.assert_array_equal(out[[0, 2]], h[[0, 2]])
+
+
+# --------------------------------------------------------------- aggregation
+
+
+def _two_match_oracle(oracle_mod, r2, r3, s2=0, s3=1, d=4):
+    rows = np.zeros((2, d), np.uint16)
+    if s2 >= 0:
+        rows[s2] = bf(r2)
+    if s3 >= 0:
+        rows[s3] = bf(r3)
+    o = mk_oracle(oracle_mod, [(2, 3), (1, 2, 3)], [s2, s3], rows, d, 10, [2, 3], 2)
+    return o, np.array([[1, 2, 3]], np.int32)
+
+
+def test_all_policy_weights_by_length(oracle_mod):
+    A = oracle_mod.POLICY_ALL
+    o, tok = _two_match_oracle(oracle_mod, [5.0, 0.0, -10.0, 2.5], [10.0, 5.0, 0.0, -2.5])
+    h = bf(np.array([[0, 0, 0, 0], [0, 0, 0, 0], [1.0, 1.0, 1.0, 1.0]], np.float32))
+    r = o.lookup(tok, 0, A)
+    exact, out = o.inject(r, h, policy=A, lam=0.5)
+    # alpha = 2/5 and 3/5:  m = (2+6, 0+3, -4+0, 1-1.5) = (8, 3, -4, -0.5);  out = 1 + 0.5 m
+    np.testing.assert_allclose(exact[2], [5.0, 2.5, -1.0, 0.75], rtol=0, atol=1e-12)
+    np.testing.assert_array_equal(unbf(out[2]), [5.0, 2.5, -1.0, 0.75])
+    np.testing.assert_array_equal(out[:2], h[:2])
+    # identical vectors: the weights sum to one, m = e
+    o, tok = _two_match_oracle(oracle_mod, [1.0, 2.0, 3.0, 4.0], [1.0, 2.0, 3.0, 4.0])
+    exact, _ = o.inject(o.lookup(tok, 0, A), h, policy=A, lam=1.0)
+    np.testing.assert_allclose(exact[2], [2.0, 3.0, 4.0, 5.0], rtol=0, atol=1e-12)
+    # a matched but non-resident member keeps its weight share and is listed as a miss
+    o, tok = _two_match_oracle(oracle_mod, [5.0, 0.0, -10.0, 2.5], None, s2=0, s3=-1)
+    r = o.lookup(tok, 0, A)
+    exact, _ = o.inject(r, h, policy=A, lam=0.5)
+    np.testing.assert_allclose(exact[2], [2.0, 1.0, -1.0, 1.5], rtol=0, atol=1e-12)
+    assert list(zip(r.miss_q, r.miss_phrase, r.miss_tier)) == [(2, 1, 2)]
+    # LONGEST on the same table selects the host-resident 3-gram: no injection at all
+    rl = o.lookup(tok, 0)
+    _, out = o.inject(rl, h, lam=0.5)
+    np.testing.assert_array_equal(out, h)
+
+
+def test_all_policy_single_match_reduces_to_longest(oracle_mod):
+    rng = np.random.default_rng(11)
+    d = 16
+    rows = bf(rng.standard_normal((1, d)))
+    o = mk_oracle(oracle_mod, [(4, 5)], [0], rows, d, 10, [2, 3], 1)
+    tok = np.array([[3, 4, 5, 4, 5]], np.int32)
+    h = bf(rng.standard_normal((5, d)))
+    rl, ra = o.lookup(tok), o.lookup(tok, 0, oracle_mod.POLICY_ALL)
+    el, ol = o.inject(rl, h, lam=0.7)
+    ea, oa = o.inject(ra, h, policy=oracle_mod.POLICY_ALL, lam=0.7)
+    np.testing.assert_array_equal(ol, oa)
+    np.testing.assert_allclose(el, ea, rtol=0, atol=1e-15)
+
+
+# --------------------------------------------------------------- cosine gate
+
+
+def test_cosine_gate_special_cases(oracle_mod):
+    d = 8
+    G = oracle_mod.GATE_COSINE
+    hv = np.array([1.0, -2.0, 0.5, 0.25, 0.0, 1.5, -1.0, 2.0], np.float32)
+    sig = lambda x: 1.0 / (1.0 + np.exp(-x))
+    lam = 0.8
+    cases = {
+        "m=h": (hv, lam * sig(1.0)),
+        "m=-h": (-hv, lam * sig(-1.0)),
+        "m orthogonal": (np.array([2.0, 1.0, 0, 0, 5.0, 0, 0, 0], np.float32), lam * 0.5),
+    }
+    for name, (mv, g) in cases.items():
+        o, tok = _one_hit_oracle(oracle_mod, mv, d=d)
+        h = bf(np.stack([hv, hv, hv]))
+        exact, _ = o.inject(o.lookup(tok), h, gate=G, lam=lam)
+        np.testing.assert_allclose(exact[1], hv.astype(np.float64) + g * mv.astype(np.float64),
+                                   rtol=0, atol=1e-9, err_msg=name)
+    o, tok = _one_hit_oracle(oracle_mod, np.zeros(d), d=d)
+    h = bf(np.stack([hv, hv, hv]))
+    _, out = o.inject(o.lookup(tok), h, gate=G, lam=lam)
+    np.testing.assert_array_equal(unbf(out), unbf(h))
+
+
+# ------------------------------------------------ tiers, miss list, install
+
+
+def _small_workload(oracle_mod, residency="hot_host_ssd", seed=9, N=1500, C=600, policy_orders=(2, 3)):
+    w = synth.config(1, seed=seed, n_phrases=N, gpu_slots=C, residency=residency, d=32, B=6, T=40,
+                     p=0.45, orders=tuple(policy_orders))
+    tb = synth.make_table(w)
+    rows = synth.make_rows_np(w, tb)
+    o = oracle_mod.Oracle(tb.phrase_tokens, tb.phrase_len, tb.init_slot, rows, d=w.d, vocab=w.vocab,
+                          orders=w.orders, gpu_slots=w.gpu_slots)
+    return w, tb, o
+
+
+@pytest.mark.parametrize("policy", [0, 1])
+def test_tier_and_miss_list_invariants(oracle_mod, policy):
+    w, tb, o = _small_workload(oracle_mod)
+    tok = synth.make_queries(w, tb)
+    r = o.lookup(tok, 0, policy)
+    f = r.flags.ravel()
+    assert np.bincount(f, minlength=4).sum() == f.size
+    assert len(r.miss_q) == np.count_nonzero(f >= 2) > 0
+    assert np.count_nonzero(f == 1) > 0
+    # listed phrases are exactly the non-resident retained ones, in ascending (q, order)
+    assert np.all(o.slot_state[r.miss_phrase] < 0)
+    np.testing.assert_array_equal(r.miss_tier, np.where(o.slot_state[r.miss_phrase] == -1, 2, 3))
+    if policy == 0:
+        assert np.all(np.diff(r.miss_q.astype(np.int64)) > 0)
+        np.testing.assert_array_equal(r.miss_q, np.nonzero(f >= 2)[0])
+        np.testing.assert_array_equal(r.miss_phrase, r.sel_phrase[f >= 2])
+    else:
+        qq, oo = np.nonzero(r.flags >= 2)
+        np.testing.assert_array_equal(r.miss_q, qq)
+        np.testing.assert_array_equal(r.miss_phrase, r.sel_phrase[qq, oo])
+    # GPU hits point at the slot that holds that phrase
+    hit = f == 1
+    np.testing.assert_array_equal(o.slot_owner[r.sel_slot.ravel()[hit]], r.sel_phrase.ravel()[hit])
+
+
+def test_install_converges_to_the_all_resident_result(oracle_mod):
+    w, tb, o = _small_workload(oracle_mod, N=1200, C=1200, residency="hot_host_ssd")
+    # start with only 400 resident: rebuild residency by hand
+    w2 = synth.config(1, seed=9, n_phrases=1200, gpu_slots=1200, residency="hot_host_ssd",
+                      reserve_free=800, d=32, B=6, T=40, p=0.45)
+    tb2 = synth.make_table(w2)
+    rows2 = synth.make_rows_np(w2, tb2)
+    o2 = oracle_mod.Oracle(tb2.phrase_tokens, tb2.phrase_len, tb2.init_slot, rows2, d=32,
+                           vocab=w2.vocab, orders=w2.orders, gpu_slots=1200)
+    tok = synth.make_queries(w2, tb2)
+    h = synth.make_hidden_np(w2)
+    r = o2.lookup(tok)
+    assert len(r.miss_q) > 0
+    ids = np.unique(r.miss_phrase)
+    free = np.nonzero(o2.slot_owner < 0)[0][:len(ids)].astype(np.int32)
+    assert o2.cache_install(ids, synth.phrase_rows_np(w2, ids), free) == 0
+    r2 = o2.lookup(tok)
+    assert len(r2.miss_q) == 0
+    np.testing.assert_array_equal(r2.sel_phrase, r.sel_phrase)
+    # reference: the same table with every phrase resident from the start (other slots)
+    wall = synth.config(1, seed=9, n_phrases=1200, gpu_slots=1200, residency="all", d=32, B=6, T=40,
+                        p=0.45)
+    tball = synth.make_table(wall)
+    oall = oracle_mod.Oracle(tball.phrase_tokens, tball.phrase_len, tball.init_slot,
+                             synth.make_rows_np(wall, tball), d=32, vocab=wall.vocab,
+                             orders=wall.orders, gpu_slots=1200)
+    rall = oall.lookup(tok)
+    np.testing.assert_array_equal(rall.sel_phrase, r2.sel_phrase)     # slot permutation changes slots only
+    np.testing.assert_array_equal(rall.flags, r2.flags)
+    _, out_a = oall.inject(rall, h, lam=1.0)
+    _, out_b = o2.inject(r2, h, lam=1.0)
+    np.testing.assert_array_equal(out_a, out_b)
+
+
+def test_cache_install_state_machine(oracle_mod):
+    d = 4
+    rows = np.zeros((3, d), np.uint16)
+    rows[0] = bf([1, 1, 1, 1])
+    rows[1] = bf([2, 2, 2, 2])
+    phrases = [(1, 2), (2, 3), (3, 4), (4, 5)]
+    o = mk_oracle(oracle_mod, phrases, [0, 1, -1, -2], rows, d, 10, [2], 3)
+    before = (o.slot_state.copy(), o.slot_owner.copy(), o.rows.copy())
+    src = bf(np.array([[7, 7, 7, 7], [8, 8, 8, 8]], np.float32))
+    # refusals leave everything untouched
+    assert o.cache_install([9, 2], src, [2, 1]) == -1      # unknown phrase
+    assert o.cache_install([0, 2], src, [2, 1]) == -2      # already resident
+    assert o.cache_install([2, 3], src, [2, 3]) == -3      # slot out of range
+    assert o.cache_install([2, 2], src, [2, 1]) == -4      # repeated id
+    assert o.cache_install([2, 3], src, [2, 2]) == -5      # repeated slot
+    for a, b in zip(before, (o.slot_state, o.slot_owner, o.rows)):
+        np.testing.assert_array_equal(a, b)
+    # phrase 2 -> free slot 2; phrase 3 -> slot 1, evicting phrase 1 to the host tier
+    assert o.cache_install([2, 3], src, [2, 1]) == 0
+    assert o.slot_state.tolist() == [0, -1, 2, 1]
+    assert o.slot_owner.tolist() == [0, 3, 2]
+    np.testing.assert_array_equal(o.rows[2], src[0])
+    np.testing.assert_array_equal(o.rows[1], src[1])
+    tok = np.array([[1, 2, 3, 4, 5]], np.int32)
+    r = o.lookup(tok)
+    assert r.flags.tolist() == [0, 1, 2, 1, 1]
+    assert r.sel_slot.tolist() == [-3, 0, -1, 2, 1]
+    assert list(zip(r.miss_q, r.miss_phrase, r.miss_tier)) == [(2, 1, 2)]
+
+
+# ------------------------------------------------------ the paper's Table 1
+
+
+def test_paper_table_hash_occupancy_fixture():
+    rows = []
+    with open(os.path.join(GOLDEN, "hash_occupancy.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            M, B, avg = line.split()
+            rows.append((int(M), int(B), float(avg)))
+    assert len(rows) == 3
+    for M, B, avg in rows:
+        assert M / B == avg
+        occupied = B * (1.0 - (1.0 - 1.0 / B) ** M)
+        assert 0 < occupied <= B
+    # M = B: a fraction 1 - 1/e of the slots is occupied
+    M, B, _ = rows[0]
+    assert abs(B * (1.0 - (1.0 - 1.0 / B) ** M) / B - (1 - np.exp(-1))) < 1e-6
