@@ -1,0 +1,199 @@
+/*
+ * tfe.h -- C ABI of the B200 Engram lookup-and-inject library (libtfe.so).
+ *
+ * The library implements the per-token side pathway of an Engram-style memory
+ * as TF-Engram uses it at inference time: from the token ids ending at each
+ * position form the trailing n-gram phrase keys, look each key up in an
+ * exact-match (non-colliding) phrase index, decide which matched phrase is
+ * retained, see in which storage tier its memory vector lives, fetch the
+ * vectors that are in the GPU tier and add them to the hidden state through a
+ * gate; phrases whose vectors are not in the GPU tier are reported so the host
+ * DRAM / SSD tier and the prefetcher can stage them, and staged vectors are
+ * written into the GPU tier by a separate call.
+ *
+ * Everything below is plain C: opaque context, PODs, raw pointers.  Each
+ * pointer is marked HOST or DEVICE.  "stream" is a cudaStream_t passed as
+ * void* (NULL = the legacy default stream).  All device work of one context
+ * must be issued in stream order (one stream, or streams the caller orders);
+ * two calls on the same context that overlap on the GPU race.
+ *
+ * No entry point throws, aborts or traps.  Argument errors are found on the
+ * host before anything is launched and leave the context unchanged.
+ */
+#ifndef TFE_H
+#define TFE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tfe_ctx tfe_ctx;
+
+typedef enum {
+    TFE_OK = 0,
+    TFE_ERR_INVALID_ARG = 1,
+    TFE_ERR_DUPLICATE_PHRASE = 2,   /* two phrases with the same token tuple                    */
+    TFE_ERR_KEY_COLLISION = 3,      /* two different tuples of a hashed order share a 64-bit key */
+    TFE_ERR_CAPACITY = 4,           /* more phrases than load_factor * index slots, or > 2^32-2 */
+    TFE_ERR_SLOT_RANGE = 5,         /* GPU-tier slot outside [0, gpu_slots) or used twice       */
+    TFE_ERR_UNKNOWN_PHRASE = 6,
+    TFE_ERR_ALREADY_RESIDENT = 7,
+    TFE_ERR_MISS_OVERFLOW = 8,      /* caller's miss buffers are smaller than the miss count    */
+    TFE_ERR_PROBE_LIMIT = 9,        /* index build could not place a key within max_probe_buckets */
+    TFE_ERR_CUDA = 10,              /* a CUDA runtime call failed; see tfe_last_cuda_error()    */
+    TFE_ERR_INTERNAL = 11           /* a bounded device-side wait ran out (reported, never hangs) */
+} tfe_status;
+
+/* Table geometry, fixed at build time. */
+typedef struct {
+    int32_t d;                  /* row width in elements; multiple of 8, >= 8                         */
+    int32_t vocab;              /* token ids are valid in [0, vocab); anything else is padding        */
+    int32_t n_orders;           /* 1..4                                                               */
+    int32_t orders[4];          /* n-gram orders, strictly ascending, each in [1,4]                   */
+    int64_t n_phrases;          /* N                                                                  */
+    int64_t gpu_slots;          /* C, rows of the GPU tier                                            */
+    float   load_factor;        /* index slots = ceil(N / load_factor), rounded up to 8-slot buckets  */
+    int32_t hidden_dtype;       /* 0 = bf16 hidden states, 1 = fp32 hidden states (rows always bf16)  */
+    int32_t max_probe_buckets;  /* bound on linear probing, 0 = library default (64)                  */
+} tfe_config;
+
+enum { TFE_POLICY_LONGEST = 0, TFE_POLICY_ALL = 1 };
+enum { TFE_GATE_CONST = 0, TFE_GATE_COSINE = 1 };
+enum { TFE_FLAG_ABSENT = 0, TFE_FLAG_GPU_HIT = 1, TFE_FLAG_HOST_MISS = 2, TFE_FLAG_SSD_MISS = 3 };
+#define TFE_NO_PHRASE 0xFFFFFFFFu
+
+/* Per-call injection rule. */
+typedef struct {
+    int32_t policy;   /* LONGEST: keep the matched phrase of greatest order.  ALL: keep every match
+                         and aggregate m = sum_i alpha_i e_i, alpha_i = n_i / sum of matched orders  */
+    int32_t gate;     /* CONST: g = lambda.  COSINE: g = lambda * sigmoid(cos(h, m))                 */
+    float   lambda;   /* the memory injection scale                                                  */
+} tfe_inject_params;
+
+/*
+ * tfe_index_build -- build the exact-match phrase index and the per-phrase
+ * metadata (paper Sec. 4.2: two-level index "token prefix -> phrase id ->
+ * memory address", metadata = length, vector address, storage tier).
+ *
+ *   cfg            HOST.
+ *   phrase_tokens  HOST int32 [N][4]; phrase i is the first phrase_len[i] entries, the rest -1.
+ *   phrase_len     HOST uint8 [N]; must be one of cfg->orders.
+ *   init_slot      HOST int32 [N]; >= 0: GPU-tier slot holding the vector; -1: host DRAM; -2: SSD.
+ *   gpu_rows       DEVICE bf16 [C][d] row-major, 16-byte aligned, CALLER-OWNED, already holding
+ *                  the vectors of the resident phrases.  The library keeps the pointer and writes
+ *                  to it only in tfe_cache_install.
+ *   stream         work is issued here; the call synchronises it before returning.
+ *   out            receives the context (phrase id = index into the arrays above).
+ *
+ * Errors (nothing is kept): INVALID_ARG (geometry, length not an order, token outside [0,vocab)),
+ * DUPLICATE_PHRASE, KEY_COLLISION, CAPACITY, SLOT_RANGE, PROBE_LIMIT, CUDA.
+ */
+tfe_status tfe_index_build(const tfe_config *cfg, const int32_t *phrase_tokens,
+                           const uint8_t *phrase_len, const int32_t *init_slot, void *gpu_rows,
+                           void *stream, tfe_ctx **out);
+
+/*
+ * tfe_cache_install -- write n fetched vectors into GPU-tier slots and make
+ * their phrases GPU-resident (paper Sec. 4.3: an entry read from DRAM / SSD is
+ * inserted into a faster tier when it arrives; Sec. 4.4: prefetched entries
+ * are moved into the GPU cache before they are needed).
+ *
+ *   phrase_ids  HOST uint32 [n]; valid, pairwise distinct, currently NOT GPU-resident.
+ *   src_rows    bf16 [n][d]; HOST (pinned memory makes the copy asynchronous; it must stay valid
+ *               until the stream has passed this call) or DEVICE.
+ *   dst_slots   HOST int32 [n]; pairwise distinct, in [0, C).  A slot that holds another phrase
+ *               is overwritten and that phrase falls back to the host-DRAM tier.
+ *   Asynchronous on `stream`; a lookup issued later on the same stream sees the new state.
+ *   phrase_ids / dst_slots may be reused as soon as the call returns.
+ *
+ * Errors (state unchanged): INVALID_ARG, UNKNOWN_PHRASE, ALREADY_RESIDENT, SLOT_RANGE, CUDA.
+ */
+tfe_status tfe_cache_install(tfe_ctx *ctx, int32_t n, const uint32_t *phrase_ids,
+                             const void *src_rows, const int32_t *dst_slots, void *stream);
+
+/*
+ * tfe_lookup_inject -- the hot path, one kernel launch (paper Sec. 2.2: key
+ * from token n-grams, lookup m_t = M(q_t), aggregation m_t = sum alpha_i v_i,
+ * injection h'_t = h_t + g_t * m_t; Sec. 4.2: longest-match selection;
+ * Sec. 4.3: tier walk).
+ *
+ *   tokens      DEVICE int32 [B][T] row-major.
+ *   q_start     queries are the positions t in [q_start, T) of every sequence,
+ *               numbered q = b*(T-q_start) + (t-q_start); Q = B*(T-q_start).  An n-gram ends at
+ *               its query position and never reaches before t = 0 of its sequence.
+ *   h           DEVICE [Q][d] hidden states (bf16 or fp32 per cfg.hidden_dtype), 16-byte aligned.
+ *   out         DEVICE [Q][d], same dtype; may be the same pointer as h (then only injected
+ *               positions are touched); must not partially overlap h.
+ *   params      HOST.
+ *   sel_phrase  DEVICE uint32 [Q] (LONGEST) or [Q][n_orders] (ALL, column = index into orders);
+ *   sel_slot    DEVICE int32, same shape: slot (hit), -1 host, -2 SSD, -3 absent;
+ *   flags       DEVICE uint8, same shape: TFE_FLAG_*.   Any of the three may be NULL.
+ *
+ * Positions whose retained phrase is GPU-resident get out = round(h + g*m) (fp32 arithmetic,
+ * round-to-nearest-even into the hidden dtype); every other position gets out = h bit for bit.
+ * A retained phrase that is not GPU-resident is NOT replaced by a shorter resident one; it goes to
+ * the miss list.  Asynchronous; launches exactly one kernel and never synchronises.
+ * Errors: INVALID_ARG, CUDA (a first call with a larger Q than any before grows context buffers).
+ */
+tfe_status tfe_lookup_inject(tfe_ctx *ctx, const int32_t *tokens, int32_t B, int32_t T,
+                             int32_t q_start, const void *h, void *out,
+                             const tfe_inject_params *params, uint32_t *sel_phrase,
+                             int32_t *sel_slot, uint8_t *flags, void *stream);
+
+/*
+ * tfe_lookup_inject_host -- the same call for HOST buffers (tokens, h, out and the optional
+ * result arrays all in host memory, pinned for asynchronous copies): copies the inputs to
+ * context-owned device buffers, runs the kernel, copies the results back, all on `stream`,
+ * without synchronising.  The buffers must stay valid until the stream has passed the call.
+ */
+tfe_status tfe_lookup_inject_host(tfe_ctx *ctx, const int32_t *tokens, int32_t B, int32_t T,
+                                  int32_t q_start, const void *h, void *out,
+                                  const tfe_inject_params *params, uint32_t *sel_phrase,
+                                  int32_t *sel_slot, uint8_t *flags, void *stream);
+
+/*
+ * tfe_miss_list -- the compacted, order-stable list of retained phrases that were not
+ * GPU-resident in the most recent lookup of this context (paper Sec. 4.3: such entries are staged
+ * from DRAM or read asynchronously from SSD; Sec. 4.4: the prefetcher consumes the same records).
+ * Entries are in ascending (q, order); duplicates are kept; tier is TFE_FLAG_HOST_MISS / SSD_MISS.
+ *
+ *   q_idx, phrase_id, tier   HOST buffers of `cap` entries (may be NULL if cap == 0).
+ *   count                    HOST, always receives the full miss count.
+ *   Synchronises `stream`.  Errors: MISS_OVERFLOW (count > cap; the first cap entries are
+ *   returned), INTERNAL, CUDA.
+ */
+tfe_status tfe_miss_list(tfe_ctx *ctx, uint32_t *q_idx, uint32_t *phrase_id, uint8_t *tier,
+                         int64_t cap, int64_t *count, void *stream);
+
+/* The same list as DEVICE pointers owned by the context, valid until the next lookup; no sync. */
+tfe_status tfe_miss_list_device(tfe_ctx *ctx, const uint32_t **q_idx, const uint32_t **phrase_id,
+                                const uint8_t **tier, const uint32_t **count);
+
+/* Frees everything the context owns (not gpu_rows).  NULL is allowed. */
+void tfe_destroy(tfe_ctx *ctx);
+
+const char *tfe_status_string(tfe_status s);
+
+/* Text of the last CUDA error seen by this thread's calls ("" if none). */
+const char *tfe_last_cuda_error(void);
+
+/*
+ * Introspection used by tests and the benchmark (HOST only, no device work).
+ *   tfe_index_geometry  buckets of 8 slots, bytes of the device index, bytes of per-phrase metadata.
+ *   tfe_phrase_key64    the 64-bit index key of a token tuple (0 if n or a token is invalid) and
+ *                       whether that order is packed injectively (exact) or hashed + verified.
+ *   tfe_home_bucket     the first bucket probed for a key.
+ *   tfe_launch_geometry grid and block size the last lookup used.
+ */
+tfe_status tfe_index_geometry(const tfe_ctx *ctx, int64_t *n_buckets, int64_t *index_bytes,
+                              int64_t *metadata_bytes);
+uint64_t tfe_phrase_key64(int32_t vocab, const int32_t *tokens, int32_t n, int32_t *is_exact);
+uint64_t tfe_home_bucket(uint64_t key, uint64_t n_buckets);
+tfe_status tfe_launch_geometry(const tfe_ctx *ctx, int32_t *grid, int32_t *block);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TFE_H */

@@ -1,0 +1,219 @@
+"""ctypes binding of libtfe.so: the same entry points as include/tfe.h.
+
+Argument marshalling only -- every step of the path runs in the library's CUDA
+kernels.  Device buffers are ``torch`` CUDA tensors (or raw integer addresses);
+host buffers are numpy arrays or pinned CPU tensors.  Loading fails loudly when
+the shared library has not been built; there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtfe.so")
+
+TFE_OK = 0
+STATUS_NAMES = ["TFE_OK", "TFE_ERR_INVALID_ARG", "TFE_ERR_DUPLICATE_PHRASE", "TFE_ERR_KEY_COLLISION",
+                "TFE_ERR_CAPACITY", "TFE_ERR_SLOT_RANGE", "TFE_ERR_UNKNOWN_PHRASE",
+                "TFE_ERR_ALREADY_RESIDENT", "TFE_ERR_MISS_OVERFLOW", "TFE_ERR_PROBE_LIMIT",
+                "TFE_ERR_CUDA", "TFE_ERR_INTERNAL"]
+(TFE_ERR_INVALID_ARG, TFE_ERR_DUPLICATE_PHRASE, TFE_ERR_KEY_COLLISION, TFE_ERR_CAPACITY,
+ TFE_ERR_SLOT_RANGE, TFE_ERR_UNKNOWN_PHRASE, TFE_ERR_ALREADY_RESIDENT, TFE_ERR_MISS_OVERFLOW,
+ TFE_ERR_PROBE_LIMIT, TFE_ERR_CUDA, TFE_ERR_INTERNAL) = range(1, 12)
+POLICY_LONGEST, POLICY_ALL = 0, 1
+GATE_CONST, GATE_COSINE = 0, 1
+HIDDEN_BF16, HIDDEN_F32 = 0, 1
+NO_PHRASE = 0xFFFFFFFF
+
+EXPORTS = ["tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
+           "tfe_miss_list", "tfe_miss_list_device", "tfe_destroy", "tfe_status_string",
+           "tfe_last_cuda_error", "tfe_index_geometry", "tfe_phrase_key64", "tfe_home_bucket",
+           "tfe_launch_geometry"]
+
+
+class TfeConfig(C.Structure):
+    _fields_ = [("d", C.c_int32), ("vocab", C.c_int32), ("n_orders", C.c_int32),
+                ("orders", C.c_int32 * 4), ("n_phrases", C.c_int64), ("gpu_slots", C.c_int64),
+                ("load_factor", C.c_float), ("hidden_dtype", C.c_int32),
+                ("max_probe_buckets", C.c_int32)]
+
+
+class TfeInjectParams(C.Structure):
+    _fields_ = [("policy", C.c_int32), ("gate", C.c_int32), ("lam", C.c_float)]
+
+
+class TfeError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        detail = ""
+        if status == TFE_ERR_CUDA:
+            detail = ": " + lib().tfe_last_cuda_error().decode()
+        super().__init__(f"{where}: {STATUS_NAMES[status]} ({lib().tfe_status_string(status).decode()}){detail}")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded library.  Raises if it is not built: this package has no other compute path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                               "`python -m paper_2607_07388_b200.build` (needs nvcc); there is no fallback")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, u64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64
+        L.tfe_index_build.argtypes = [C.POINTER(TfeConfig), vp, vp, vp, vp, vp, C.POINTER(vp)]
+        L.tfe_cache_install.argtypes = [vp, i32, vp, vp, vp, vp]
+        L.tfe_lookup_inject.argtypes = [vp, vp, i32, i32, i32, vp, vp, C.POINTER(TfeInjectParams), vp, vp, vp, vp]
+        L.tfe_lookup_inject_host.argtypes = L.tfe_lookup_inject.argtypes
+        L.tfe_miss_list.argtypes = [vp, vp, vp, vp, i64, C.POINTER(i64), vp]
+        L.tfe_miss_list_device.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]
+        L.tfe_destroy.argtypes = [vp]
+        L.tfe_destroy.restype = None
+        L.tfe_status_string.argtypes = [C.c_int]
+        L.tfe_status_string.restype = C.c_char_p
+        L.tfe_last_cuda_error.restype = C.c_char_p
+        L.tfe_index_geometry.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64)]
+        L.tfe_phrase_key64.argtypes = [i32, vp, i32, C.POINTER(i32)]
+        L.tfe_phrase_key64.restype = u64
+        L.tfe_home_bucket.argtypes = [u64, u64]
+        L.tfe_home_bucket.restype = u64
+        L.tfe_launch_geometry.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
+        for name in ("tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
+                     "tfe_miss_list", "tfe_miss_list_device", "tfe_index_geometry", "tfe_launch_geometry"):
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _addr(x):
+    """Address of a device tensor, host tensor, numpy array, int or None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if isinstance(x, np.ndarray):
+        assert x.flags["C_CONTIGUOUS"]
+        return x.ctypes.data
+    assert x.is_contiguous()
+    return x.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def _check(status: int, where: str):
+    if status != TFE_OK:
+        raise TfeError(status, where)
+
+
+def make_config(*, d, vocab, orders, n_phrases, gpu_slots, load_factor=0.7, hidden_dtype=HIDDEN_BF16,
+                max_probe_buckets=0) -> TfeConfig:
+    cfg = TfeConfig()
+    cfg.d, cfg.vocab, cfg.n_orders = int(d), int(vocab), len(orders)
+    for i in range(4):
+        cfg.orders[i] = int(orders[i]) if i < len(orders) else 0
+    cfg.n_phrases, cfg.gpu_slots = int(n_phrases), int(gpu_slots)
+    cfg.load_factor, cfg.hidden_dtype, cfg.max_probe_buckets = float(load_factor), int(hidden_dtype), int(max_probe_buckets)
+    return cfg
+
+
+# ---- the C entry points, same names -------------------------------------------------------
+
+
+def tfe_index_build(cfg: TfeConfig, phrase_tokens, phrase_len, init_slot, gpu_rows, stream=None) -> int:
+    """Returns the context handle (an integer address)."""
+    pt = np.ascontiguousarray(phrase_tokens, dtype=np.int32)
+    pl = np.ascontiguousarray(phrase_len, dtype=np.uint8)
+    sl = np.ascontiguousarray(init_slot, dtype=np.int32)
+    out = C.c_void_p()
+    _check(lib().tfe_index_build(C.byref(cfg), _addr(pt), _addr(pl), _addr(sl), _addr(gpu_rows),
+                                 _stream(stream), C.byref(out)), "tfe_index_build")
+    return out.value
+
+
+def tfe_cache_install(ctx: int, phrase_ids, src_rows, dst_slots, stream=None) -> None:
+    ids = np.ascontiguousarray(phrase_ids, dtype=np.uint32)
+    dst = np.ascontiguousarray(dst_slots, dtype=np.int32)
+    _check(lib().tfe_cache_install(ctx, len(ids), _addr(ids), _addr(src_rows), _addr(dst), _stream(stream)),
+           "tfe_cache_install")
+
+
+def _params(policy, gate, lam):
+    p = TfeInjectParams()
+    p.policy, p.gate, p.lam = int(policy), int(gate), float(lam)
+    return p
+
+
+def tfe_lookup_inject(ctx: int, tokens, B, T, q_start, h, out, *, policy=POLICY_LONGEST, gate=GATE_CONST,
+                      lam=1.0, sel_phrase=None, sel_slot=None, flags=None, stream=None) -> None:
+    p = _params(policy, gate, lam)
+    _check(lib().tfe_lookup_inject(ctx, _addr(tokens), B, T, q_start, _addr(h), _addr(out), C.byref(p),
+                                   _addr(sel_phrase), _addr(sel_slot), _addr(flags), _stream(stream)),
+           "tfe_lookup_inject")
+
+
+def tfe_lookup_inject_host(ctx: int, tokens, B, T, q_start, h, out, *, policy=POLICY_LONGEST,
+                           gate=GATE_CONST, lam=1.0, sel_phrase=None, sel_slot=None, flags=None,
+                           stream=None) -> None:
+    p = _params(policy, gate, lam)
+    _check(lib().tfe_lookup_inject_host(ctx, _addr(tokens), B, T, q_start, _addr(h), _addr(out), C.byref(p),
+                                        _addr(sel_phrase), _addr(sel_slot), _addr(flags), _stream(stream)),
+           "tfe_lookup_inject_host")
+
+
+def tfe_miss_list(ctx: int, cap: int, stream=None, allow_overflow=False):
+    """(q_idx uint32[n], phrase_id uint32[n], tier uint8[n], count) of the most recent lookup."""
+    q = np.empty(max(cap, 1), np.uint32)
+    ph = np.empty(max(cap, 1), np.uint32)
+    tr = np.empty(max(cap, 1), np.uint8)
+    cnt = C.c_int64(0)
+    st = lib().tfe_miss_list(ctx, _addr(q), _addr(ph), _addr(tr), cap, C.byref(cnt), _stream(stream))
+    if not (allow_overflow and st == TFE_ERR_MISS_OVERFLOW):
+        _check(st, "tfe_miss_list")
+    n = min(cnt.value, cap)
+    return q[:n], ph[:n], tr[:n], cnt.value
+
+
+def tfe_miss_list_device(ctx: int):
+    """Device addresses (q_idx, phrase_id, tier, count) owned by the context."""
+    a, b, c_, d = C.c_void_p(), C.c_void_p(), C.c_void_p(), C.c_void_p()
+    _check(lib().tfe_miss_list_device(ctx, C.byref(a), C.byref(b), C.byref(c_), C.byref(d)),
+           "tfe_miss_list_device")
+    return a.value, b.value, c_.value, d.value
+
+
+def tfe_destroy(ctx: int) -> None:
+    if ctx:
+        lib().tfe_destroy(ctx)
+
+
+def tfe_index_geometry(ctx: int):
+    a, b, c_ = C.c_int64(), C.c_int64(), C.c_int64()
+    _check(lib().tfe_index_geometry(ctx, C.byref(a), C.byref(b), C.byref(c_)), "tfe_index_geometry")
+    return a.value, b.value, c_.value
+
+
+def tfe_launch_geometry(ctx: int):
+    g, b = C.c_int32(), C.c_int32()
+    _check(lib().tfe_launch_geometry(ctx, C.byref(g), C.byref(b)), "tfe_launch_geometry")
+    return g.value, b.value
+
+
+def tfe_phrase_key64(vocab: int, tokens) -> tuple[int, bool]:
+    t = np.ascontiguousarray(tokens, dtype=np.int32)
+    ex = C.c_int32(0)
+    k = lib().tfe_phrase_key64(vocab, _addr(t), len(t), C.byref(ex))
+    return int(k), bool(ex.value)
+
+
+def tfe_home_bucket(key: int, n_buckets: int) -> int:
+    return int(lib().tfe_home_bucket(key, n_buckets))

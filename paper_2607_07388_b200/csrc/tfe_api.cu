@@ -1,0 +1,563 @@
+// Host side of libtfe.so: the C ABI declared in include/tfe.h.
+//
+// The context owns the device index, the per-phrase metadata the kernels need
+// (index position of every phrase, token tuples of hashed orders, owner of every
+// GPU-tier slot), the miss-list buffers, and a host mirror of the residency state
+// used to validate arguments before anything is launched.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/tfe.h"
+#include "tfe_kernels.cuh"
+
+namespace {
+
+thread_local std::string g_cuda_error;
+
+bool cuda_failed(cudaError_t e, const char *what)
+{
+    if (e == cudaSuccess) return false;
+    g_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+    (void)cudaGetLastError();
+    return true;
+}
+#define CU(call)                                                       \
+    do {                                                               \
+        if (cuda_failed((call), #call)) return TFE_ERR_CUDA;           \
+    } while (0)
+
+constexpr uint32_t kNoOwner = 0xFFFFFFFFu;
+constexpr int kDefaultMaxProbe = 64;
+
+}  // namespace
+
+struct tfe_ctx {
+    tfe_config cfg{};
+    int device = 0;
+    int sm_count = 0;
+    int tok_bits = 0;
+    bool any_hashed = false;
+    int max_probe = kDefaultMaxProbe;
+    uint64_t n_buckets = 0;
+    int row_vecs = 0;                       // 16-byte vectors per GPU-tier row
+
+    ulonglong2 *d_index = nullptr;
+    int4 *d_phrase_tokens = nullptr;        // only when an order is hashed
+    uint32_t *d_phrase_pos = nullptr;
+    uint32_t *d_slot_owner = nullptr;
+    uint4 *gpu_rows = nullptr;              // caller-owned
+
+    std::vector<int32_t> h_slot;            // residency mirror
+    std::vector<uint32_t> h_owner;
+
+    int64_t ent_cap = 0;                    // capacity (entries) of the five buffers below
+    uint32_t *d_scr_phrase = nullptr;
+    uint8_t *d_scr_flag = nullptr;
+    uint32_t *d_miss_q = nullptr, *d_miss_phrase = nullptr;
+    uint8_t *d_miss_tier = nullptr;
+    uint32_t *d_counters = nullptr;         // TFE_CTR_WORDS words of launch state
+    unsigned long long *d_block_state = nullptr;
+    int max_grid = 0;
+    int occ[8] = {0};                       // resident blocks per SM of each kernel variant
+
+    int64_t last_entries = -1;              // Q*cols of the most recent lookup (-1: none yet)
+    int last_grid = 0;
+
+    // install staging
+    uint32_t *d_inst_ids = nullptr;
+    int32_t *d_inst_slots = nullptr;
+    uint4 *d_inst_rows = nullptr;
+    int32_t inst_cap = 0;
+
+    // host-buffer variant staging
+    int32_t *d_h_tokens = nullptr;
+    void *d_h_hidden = nullptr, *d_h_out = nullptr;
+    uint32_t *d_h_phrase = nullptr;
+    int32_t *d_h_slot = nullptr;
+    uint8_t *d_h_flag = nullptr;
+    int64_t hb_tok_cap = 0, hb_q_cap = 0, hb_ent_cap = 0;
+};
+
+namespace {
+
+typedef void (*lookup_kernel_t)(const TfeLookupParams);
+
+lookup_kernel_t pick_kernel(int ht, int all, int cos)
+{
+    static const lookup_kernel_t table[8] = {
+        tfe_lookup_inject_kernel<0, false, false>, tfe_lookup_inject_kernel<0, false, true>,
+        tfe_lookup_inject_kernel<0, true, false>,  tfe_lookup_inject_kernel<0, true, true>,
+        tfe_lookup_inject_kernel<1, false, false>, tfe_lookup_inject_kernel<1, false, true>,
+        tfe_lookup_inject_kernel<1, true, false>,  tfe_lookup_inject_kernel<1, true, true>,
+    };
+    return table[ht * 4 + all * 2 + cos];
+}
+
+void free_dev(void *p) { if (p) (void)cudaFree(p); }
+
+tfe_status validate_config(const tfe_config *c)
+{
+    if (!c) return TFE_ERR_INVALID_ARG;
+    if (c->d < 8 || c->d % 8 != 0) return TFE_ERR_INVALID_ARG;
+    if (c->vocab < 1) return TFE_ERR_INVALID_ARG;
+    if (c->n_orders < 1 || c->n_orders > 4) return TFE_ERR_INVALID_ARG;
+    for (int i = 0; i < c->n_orders; ++i) {
+        if (c->orders[i] < 1 || c->orders[i] > 4) return TFE_ERR_INVALID_ARG;
+        if (i && c->orders[i] <= c->orders[i - 1]) return TFE_ERR_INVALID_ARG;
+    }
+    if (c->n_phrases < 0 || c->gpu_slots < 0) return TFE_ERR_INVALID_ARG;
+    if (c->gpu_slots > 0x7FFFFFFFll) return TFE_ERR_INVALID_ARG;
+    if (!(c->load_factor > 0.f && c->load_factor <= 1.f)) return TFE_ERR_INVALID_ARG;
+    if (c->hidden_dtype != 0 && c->hidden_dtype != 1) return TFE_ERR_INVALID_ARG;
+    if (c->max_probe_buckets < 0) return TFE_ERR_INVALID_ARG;
+    if (c->n_phrases > 0xFFFFFFFEll) return TFE_ERR_CAPACITY;
+    return TFE_OK;
+}
+
+// Grow the per-lookup buffers to hold `entries` (= Q * cols) results.  Not on the hot path:
+// only a call with more entries than any earlier one allocates (and synchronises the device).
+tfe_status ensure_entries(tfe_ctx *c, int64_t entries)
+{
+    if (entries <= c->ent_cap) return TFE_OK;
+    int64_t cap = std::max<int64_t>(entries, 1024);
+    CU(cudaDeviceSynchronize());
+    free_dev(c->d_scr_phrase); free_dev(c->d_scr_flag);
+    free_dev(c->d_miss_q); free_dev(c->d_miss_phrase); free_dev(c->d_miss_tier);
+    c->d_scr_phrase = nullptr; c->d_scr_flag = nullptr;
+    c->d_miss_q = c->d_miss_phrase = nullptr; c->d_miss_tier = nullptr;
+    c->ent_cap = 0;
+    CU(cudaMalloc(&c->d_scr_phrase, cap * 4));
+    CU(cudaMalloc(&c->d_scr_flag, cap));
+    CU(cudaMalloc(&c->d_miss_q, cap * 4));
+    CU(cudaMalloc(&c->d_miss_phrase, cap * 4));
+    CU(cudaMalloc(&c->d_miss_tier, cap));
+    c->ent_cap = cap;
+    return TFE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *tfe_status_string(tfe_status s)
+{
+    switch (s) {
+    case TFE_OK: return "ok";
+    case TFE_ERR_INVALID_ARG: return "invalid argument";
+    case TFE_ERR_DUPLICATE_PHRASE: return "duplicate phrase";
+    case TFE_ERR_KEY_COLLISION: return "64-bit key collision between two phrases";
+    case TFE_ERR_CAPACITY: return "index capacity exceeded";
+    case TFE_ERR_SLOT_RANGE: return "GPU-tier slot out of range or used twice";
+    case TFE_ERR_UNKNOWN_PHRASE: return "unknown phrase id";
+    case TFE_ERR_ALREADY_RESIDENT: return "phrase is already GPU-resident";
+    case TFE_ERR_MISS_OVERFLOW: return "miss list larger than the caller's buffers";
+    case TFE_ERR_PROBE_LIMIT: return "probe limit reached while building the index";
+    case TFE_ERR_CUDA: return "CUDA runtime error";
+    case TFE_ERR_INTERNAL: return "bounded device-side wait expired";
+    }
+    return "unknown status";
+}
+
+const char *tfe_last_cuda_error(void) { return g_cuda_error.c_str(); }
+
+uint64_t tfe_phrase_key64(int32_t vocab, const int32_t *tokens, int32_t n, int32_t *is_exact)
+{
+    if (vocab < 1 || n < 1 || n > 4 || !tokens) return 0;
+    const int bits = tfe_token_bits(vocab);
+    int32_t tk[4] = {-1, -1, -1, -1};
+    for (int j = 0; j < n; ++j) {
+        int32_t x = tokens[n - 1 - j];
+        if (x < 0 || x >= vocab) return 0;
+        tk[j] = x;
+    }
+    if (is_exact) *is_exact = tfe_order_is_packed(n, bits) ? 1 : 0;
+    return tfe_make_key(n, tk, bits);
+}
+
+uint64_t tfe_home_bucket(uint64_t key, uint64_t n_buckets)
+{
+    return n_buckets ? tfe_home_bucket_of(key, n_buckets) : 0;
+}
+
+void tfe_destroy(tfe_ctx *c)
+{
+    if (!c) return;
+    int prev = 0;
+    (void)cudaGetDevice(&prev);
+    (void)cudaSetDevice(c->device);
+    (void)cudaDeviceSynchronize();
+    free_dev(c->d_index); free_dev(c->d_phrase_tokens); free_dev(c->d_phrase_pos);
+    free_dev(c->d_slot_owner); free_dev(c->d_scr_phrase); free_dev(c->d_scr_flag);
+    free_dev(c->d_miss_q); free_dev(c->d_miss_phrase); free_dev(c->d_miss_tier);
+    free_dev(c->d_counters); free_dev(c->d_block_state);
+    free_dev(c->d_inst_ids); free_dev(c->d_inst_slots); free_dev(c->d_inst_rows);
+    free_dev(c->d_h_tokens); free_dev(c->d_h_hidden); free_dev(c->d_h_out);
+    free_dev(c->d_h_phrase); free_dev(c->d_h_slot); free_dev(c->d_h_flag);
+    (void)cudaSetDevice(prev);
+    delete c;
+}
+
+tfe_status tfe_index_build(const tfe_config *cfg, const int32_t *phrase_tokens,
+                           const uint8_t *phrase_len, const int32_t *init_slot, void *gpu_rows,
+                           void *stream_, tfe_ctx **out)
+{
+    if (!out) return TFE_ERR_INVALID_ARG;
+    *out = nullptr;
+    tfe_status st = validate_config(cfg);
+    if (st != TFE_OK) return st;
+    const int64_t N = cfg->n_phrases, C = cfg->gpu_slots;
+    if (N > 0 && (!phrase_tokens || !phrase_len || !init_slot)) return TFE_ERR_INVALID_ARG;
+    if (C > 0 && !gpu_rows) return TFE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(gpu_rows) & 15u) != 0) return TFE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+    const int bits = tfe_token_bits(cfg->vocab);
+    bool order_ok[5] = {false, false, false, false, false};
+    bool any_hashed = false;
+    for (int i = 0; i < cfg->n_orders; ++i) {
+        order_ok[cfg->orders[i]] = true;
+        any_hashed |= !tfe_order_is_packed(cfg->orders[i], bits);
+    }
+
+    // ---- host-side checks and key formation
+    std::vector<uint64_t> keys((size_t)N);
+    std::vector<uint32_t> owner((size_t)C, kNoOwner);
+    for (int64_t i = 0; i < N; ++i) {
+        const int n = phrase_len[i];
+        if (n < 1 || n > 4 || !order_ok[n]) return TFE_ERR_INVALID_ARG;
+        int32_t tk[4] = {-1, -1, -1, -1};
+        for (int j = 0; j < n; ++j) {
+            const int32_t x = phrase_tokens[i * 4 + (n - 1 - j)];
+            if (x < 0 || x >= cfg->vocab) return TFE_ERR_INVALID_ARG;
+            tk[j] = x;
+        }
+        keys[(size_t)i] = tfe_make_key(n, tk, bits);
+        const int32_t s = init_slot[i];
+        if (s >= 0) {
+            if (s >= C || owner[(size_t)s] != kNoOwner) return TFE_ERR_SLOT_RANGE;
+            owner[(size_t)s] = (uint32_t)i;
+        } else if (s != -1 && s != -2) {
+            return TFE_ERR_INVALID_ARG;
+        }
+    }
+    {   // equal keys: the same tuple twice, or (hashed orders only) two tuples on one key
+        std::vector<std::pair<uint64_t, uint32_t>> sorted((size_t)N);
+        for (int64_t i = 0; i < N; ++i) sorted[(size_t)i] = {keys[(size_t)i], (uint32_t)i};
+        std::sort(sorted.begin(), sorted.end());
+        for (int64_t i = 1; i < N; ++i) {
+            if (sorted[(size_t)i].first != sorted[(size_t)i - 1].first) continue;
+            const uint32_t a = sorted[(size_t)i].second, b = sorted[(size_t)i - 1].second;
+            const bool same = phrase_len[a] == phrase_len[b] &&
+                              std::memcmp(phrase_tokens + (size_t)a * 4, phrase_tokens + (size_t)b * 4,
+                                          sizeof(int32_t) * phrase_len[a]) == 0;
+            return same ? TFE_ERR_DUPLICATE_PHRASE : TFE_ERR_KEY_COLLISION;
+        }
+    }
+    const double want_slots = std::max<double>(1.0, (double)N / (double)cfg->load_factor);
+    const uint64_t n_buckets =
+        std::max<uint64_t>(1, (uint64_t)((want_slots + TFE_SLOTS_PER_BUCKET - 1) / TFE_SLOTS_PER_BUCKET));
+    if (n_buckets * TFE_SLOTS_PER_BUCKET > 0xFFFFFFFFull) return TFE_ERR_CAPACITY;
+    if ((uint64_t)N > n_buckets * TFE_SLOTS_PER_BUCKET) return TFE_ERR_CAPACITY;
+
+    // ---- device state
+    tfe_ctx *c = new (std::nothrow) tfe_ctx();
+    if (!c) return TFE_ERR_INVALID_ARG;
+    c->cfg = *cfg;
+    c->tok_bits = bits;
+    c->any_hashed = any_hashed;
+    c->max_probe = cfg->max_probe_buckets > 0 ? cfg->max_probe_buckets : kDefaultMaxProbe;
+    if ((uint64_t)c->max_probe > n_buckets) c->max_probe = (int)n_buckets;
+    c->n_buckets = n_buckets;
+    c->row_vecs = cfg->d / 8;
+    c->gpu_rows = static_cast<uint4 *>(gpu_rows);
+    c->h_slot.assign(init_slot, init_slot + N);
+    c->h_owner.swap(owner);
+
+    uint64_t *d_keys = nullptr;
+    int32_t *d_slots = nullptr;
+    uint32_t h_status = 0;
+    tfe_status rc = TFE_OK;
+    auto fail = [&](tfe_status s) {
+        free_dev(d_keys); free_dev(d_slots);
+        tfe_destroy(c);
+        return s;
+    };
+#define CUF(call)                                                  \
+    do {                                                           \
+        if (cuda_failed((call), #call)) return fail(TFE_ERR_CUDA); \
+    } while (0)
+    CUF(cudaGetDevice(&c->device));
+    CUF(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device));
+    const size_t index_bytes = (size_t)n_buckets * TFE_SLOTS_PER_BUCKET * sizeof(ulonglong2);
+    CUF(cudaMalloc(&c->d_index, index_bytes));
+    CUF(cudaMemsetAsync(c->d_index, 0, index_bytes, stream));
+    CUF(cudaMalloc(&c->d_phrase_pos, std::max<size_t>(4, (size_t)N * 4)));
+    CUF(cudaMalloc(&c->d_slot_owner, std::max<size_t>(4, (size_t)C * 4)));
+    CUF(cudaMalloc(&c->d_counters, TFE_CTR_WORDS * sizeof(uint32_t)));
+    CUF(cudaMemsetAsync(c->d_counters, 0, TFE_CTR_WORDS * sizeof(uint32_t), stream));
+    if (C > 0)
+        CUF(cudaMemcpyAsync(c->d_slot_owner, c->h_owner.data(), (size_t)C * 4, cudaMemcpyHostToDevice, stream));
+    if (any_hashed && N > 0) {
+        CUF(cudaMalloc(&c->d_phrase_tokens, (size_t)N * sizeof(int4)));
+        CUF(cudaMemcpyAsync(c->d_phrase_tokens, phrase_tokens, (size_t)N * sizeof(int4),
+                            cudaMemcpyHostToDevice, stream));
+    }
+    int max_occ = 1;
+    for (int v = 0; v < 8; ++v) {
+        int occ = 0;
+        CUF(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, pick_kernel(v >> 2, (v >> 1) & 1, v & 1),
+                                                          TFE_BLOCK_THREADS, 0));
+        c->occ[v] = std::max(1, occ);
+        max_occ = std::max(max_occ, c->occ[v]);
+    }
+    c->max_grid = c->sm_count * max_occ;
+    CUF(cudaMalloc(&c->d_block_state, (size_t)c->max_grid * sizeof(unsigned long long)));
+    CUF(cudaMemsetAsync(c->d_block_state, 0, (size_t)c->max_grid * sizeof(unsigned long long), stream));
+    if (N > 0) {
+        CUF(cudaMalloc(&d_keys, (size_t)N * 8));
+        CUF(cudaMalloc(&d_slots, (size_t)N * 4));
+        CUF(cudaMemcpyAsync(d_keys, keys.data(), (size_t)N * 8, cudaMemcpyHostToDevice, stream));
+        CUF(cudaMemcpyAsync(d_slots, init_slot, (size_t)N * 4, cudaMemcpyHostToDevice, stream));
+        const unsigned blocks = (unsigned)((N + 255) / 256);
+        tfe_insert_kernel<<<blocks, 256, 0, stream>>>(c->d_index, n_buckets, c->max_probe, d_keys, d_slots,
+                                                      (uint32_t)N, c->d_phrase_pos, c->d_counters + TFE_CTR_STATUS);
+        CUF(cudaGetLastError());
+        CUF(cudaMemcpyAsync(&h_status, c->d_counters + TFE_CTR_STATUS, 4, cudaMemcpyDeviceToHost, stream));
+    }
+    CUF(cudaStreamSynchronize(stream));
+    if (h_status & TFE_DEV_PROBE_LIMIT) rc = TFE_ERR_PROBE_LIMIT;
+    else if (h_status & TFE_DEV_DUP_KEY) rc = TFE_ERR_DUPLICATE_PHRASE;
+    if (rc != TFE_OK) return fail(rc);
+    {
+        uint32_t init[TFE_CTR_WORDS] = {0};
+        init[TFE_CTR_EPOCH] = 1;
+        CUF(cudaMemcpyAsync(c->d_counters, init, sizeof init, cudaMemcpyHostToDevice, stream));
+        CUF(cudaStreamSynchronize(stream));
+    }
+#undef CUF
+    free_dev(d_keys); free_dev(d_slots);
+    *out = c;
+    return TFE_OK;
+}
+
+tfe_status tfe_index_geometry(const tfe_ctx *c, int64_t *n_buckets, int64_t *index_bytes,
+                              int64_t *metadata_bytes)
+{
+    if (!c) return TFE_ERR_INVALID_ARG;
+    if (n_buckets) *n_buckets = (int64_t)c->n_buckets;
+    if (index_bytes) *index_bytes = (int64_t)(c->n_buckets * TFE_SLOTS_PER_BUCKET * sizeof(ulonglong2));
+    if (metadata_bytes)
+        *metadata_bytes = c->cfg.n_phrases * 4 + c->cfg.gpu_slots * 4 +
+                          (c->any_hashed ? c->cfg.n_phrases * (int64_t)sizeof(int4) : 0);
+    return TFE_OK;
+}
+
+tfe_status tfe_launch_geometry(const tfe_ctx *c, int32_t *grid, int32_t *block)
+{
+    if (!c) return TFE_ERR_INVALID_ARG;
+    if (grid) *grid = c->last_grid;
+    if (block) *block = TFE_BLOCK_THREADS;
+    return TFE_OK;
+}
+
+tfe_status tfe_cache_install(tfe_ctx *c, int32_t n, const uint32_t *phrase_ids, const void *src_rows,
+                             const int32_t *dst_slots, void *stream_)
+{
+    if (!c || n < 0) return TFE_ERR_INVALID_ARG;
+    if (n == 0) return TFE_OK;
+    if (!phrase_ids || !src_rows || !dst_slots) return TFE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(src_rows) & 15u) != 0) return TFE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int64_t N = c->cfg.n_phrases, C = c->cfg.gpu_slots;
+    for (int32_t k = 0; k < n; ++k) {
+        if ((int64_t)phrase_ids[k] >= N) return TFE_ERR_UNKNOWN_PHRASE;
+        if (c->h_slot[phrase_ids[k]] >= 0) return TFE_ERR_ALREADY_RESIDENT;
+        if (dst_slots[k] < 0 || dst_slots[k] >= C) return TFE_ERR_SLOT_RANGE;
+    }
+    {
+        std::vector<uint32_t> a(phrase_ids, phrase_ids + n);
+        std::vector<int32_t> b(dst_slots, dst_slots + n);
+        std::sort(a.begin(), a.end());
+        std::sort(b.begin(), b.end());
+        if (std::adjacent_find(a.begin(), a.end()) != a.end()) return TFE_ERR_INVALID_ARG;
+        if (std::adjacent_find(b.begin(), b.end()) != b.end()) return TFE_ERR_INVALID_ARG;
+    }
+    cudaPointerAttributes attr{};
+    bool src_on_device = false;
+    if (cudaPointerGetAttributes(&attr, src_rows) == cudaSuccess)
+        src_on_device = attr.type == cudaMemoryTypeDevice || attr.type == cudaMemoryTypeManaged;
+    else
+        (void)cudaGetLastError();
+
+    if (n > c->inst_cap) {      // staging grows outside the steady state
+        CU(cudaDeviceSynchronize());
+        free_dev(c->d_inst_ids); free_dev(c->d_inst_slots); free_dev(c->d_inst_rows);
+        c->d_inst_ids = nullptr; c->d_inst_slots = nullptr; c->d_inst_rows = nullptr;
+        c->inst_cap = 0;
+        CU(cudaMalloc(&c->d_inst_ids, (size_t)n * 4));
+        CU(cudaMalloc(&c->d_inst_slots, (size_t)n * 4));
+        CU(cudaMalloc(&c->d_inst_rows, (size_t)n * c->row_vecs * sizeof(uint4)));
+        c->inst_cap = n;
+    }
+    CU(cudaMemcpyAsync(c->d_inst_ids, phrase_ids, (size_t)n * 4, cudaMemcpyHostToDevice, stream));
+    CU(cudaMemcpyAsync(c->d_inst_slots, dst_slots, (size_t)n * 4, cudaMemcpyHostToDevice, stream));
+    const uint4 *src = static_cast<const uint4 *>(src_rows);
+    if (!src_on_device) {
+        CU(cudaMemcpyAsync(c->d_inst_rows, src_rows, (size_t)n * c->row_vecs * sizeof(uint4),
+                           cudaMemcpyHostToDevice, stream));
+        src = c->d_inst_rows;
+    }
+    const unsigned blocks = (unsigned)((n + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK);
+    tfe_install_kernel<<<blocks, TFE_BLOCK_THREADS, 0, stream>>>(c->d_index, c->d_phrase_pos, c->d_slot_owner,
+                                                                 c->gpu_rows, c->row_vecs, n, c->d_inst_ids,
+                                                                 src, c->d_inst_slots);
+    CU(cudaGetLastError());
+    for (int32_t k = 0; k < n; ++k) {       // mirror, same order as the oracle's state machine
+        const uint32_t prev = c->h_owner[(size_t)dst_slots[k]];
+        if (prev != kNoOwner) c->h_slot[prev] = -1;
+        c->h_slot[phrase_ids[k]] = dst_slots[k];
+        c->h_owner[(size_t)dst_slots[k]] = phrase_ids[k];
+    }
+    return TFE_OK;
+}
+
+tfe_status tfe_lookup_inject(tfe_ctx *c, const int32_t *tokens, int32_t B, int32_t T, int32_t q_start,
+                             const void *h, void *out, const tfe_inject_params *prm,
+                             uint32_t *sel_phrase, int32_t *sel_slot, uint8_t *flags, void *stream_)
+{
+    if (!c || !prm || B < 0 || T < 0 || q_start < 0 || q_start > T) return TFE_ERR_INVALID_ARG;
+    if (prm->policy != TFE_POLICY_LONGEST && prm->policy != TFE_POLICY_ALL) return TFE_ERR_INVALID_ARG;
+    if (prm->gate != TFE_GATE_CONST && prm->gate != TFE_GATE_COSINE) return TFE_ERR_INVALID_ARG;
+    const int64_t Tq = T - q_start, Q = (int64_t)B * Tq;
+    const int cols = prm->policy == TFE_POLICY_ALL ? c->cfg.n_orders : 1;
+    if (Q * cols > 0x7FFFFFFFll) return TFE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (Q == 0) {      // nothing to launch; the miss count of "this lookup" is zero
+        CU(cudaMemsetAsync(c->d_counters + TFE_CTR_TOTAL, 0, sizeof(uint32_t), stream));
+        c->last_entries = 0;
+        c->last_grid = 0;
+        return TFE_OK;
+    }
+    if (!tokens || !h || !out) return TFE_ERR_INVALID_ARG;
+    if (((reinterpret_cast<uintptr_t>(h) | reinterpret_cast<uintptr_t>(out)) & 15u) != 0)
+        return TFE_ERR_INVALID_ARG;
+    tfe_status st = ensure_entries(c, Q * cols);
+    if (st != TFE_OK) return st;
+
+    const int variant = c->cfg.hidden_dtype * 4 + (prm->policy == TFE_POLICY_ALL ? 2 : 0) +
+                        (prm->gate == TFE_GATE_COSINE ? 1 : 0);
+    const int64_t resident = (int64_t)c->sm_count * c->occ[variant];
+    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(resident, (Q + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK));
+
+    TfeLookupParams p{};
+    p.tokens = tokens; p.B = B; p.T = T; p.q_start = q_start; p.Tq = (int32_t)Tq; p.Q = (uint32_t)Q;
+    p.index = c->d_index; p.n_buckets = c->n_buckets; p.max_probe = c->max_probe;
+    p.phrase_tokens = c->d_phrase_tokens; p.rows = c->gpu_rows; p.d = c->cfg.d;
+    p.h = h; p.out = out;
+    p.n_orders = c->cfg.n_orders;
+    for (int i = 0; i < 4; ++i) p.orders[i] = i < c->cfg.n_orders ? c->cfg.orders[i] : 0;
+    p.tok_bits = c->tok_bits; p.vocab = c->cfg.vocab; p.lambda = prm->lambda;
+    p.sel_phrase = sel_phrase; p.sel_slot = sel_slot; p.flags = flags;
+    p.scr_phrase = c->d_scr_phrase; p.scr_flag = c->d_scr_flag;
+    p.miss_q = c->d_miss_q; p.miss_phrase = c->d_miss_phrase; p.miss_tier = c->d_miss_tier;
+    p.counters = c->d_counters; p.block_state = c->d_block_state;
+    p.block_state_len = (uint32_t)c->max_grid;
+    p.q_per_block = (uint32_t)((Q + grid - 1) / grid);
+
+    pick_kernel(variant >> 2, (variant >> 1) & 1, variant & 1)<<<(unsigned)grid, TFE_BLOCK_THREADS, 0, stream>>>(p);
+    CU(cudaGetLastError());
+    c->last_entries = Q * cols;
+    c->last_grid = (int)grid;
+    return TFE_OK;
+}
+
+tfe_status tfe_lookup_inject_host(tfe_ctx *c, const int32_t *tokens, int32_t B, int32_t T, int32_t q_start,
+                                  const void *h, void *out, const tfe_inject_params *prm,
+                                  uint32_t *sel_phrase, int32_t *sel_slot, uint8_t *flags, void *stream_)
+{
+    if (!c || !prm || B < 0 || T < 0 || q_start < 0 || q_start > T) return TFE_ERR_INVALID_ARG;
+    if (prm->policy != TFE_POLICY_LONGEST && prm->policy != TFE_POLICY_ALL) return TFE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int64_t n_tok = (int64_t)B * T, Q = (int64_t)B * (T - q_start);
+    const int cols = prm->policy == TFE_POLICY_ALL ? c->cfg.n_orders : 1;
+    const int64_t ent = Q * cols;
+    if (Q == 0) return tfe_lookup_inject(c, nullptr, B, T, q_start, nullptr, nullptr, prm, nullptr, nullptr, nullptr, stream_);
+    if (!tokens || !h || !out) return TFE_ERR_INVALID_ARG;
+    const size_t hid_bytes = (size_t)Q * c->cfg.d * (c->cfg.hidden_dtype == 0 ? 2 : 4);
+    if (n_tok > c->hb_tok_cap || Q > c->hb_q_cap || ent > c->hb_ent_cap) {
+        CU(cudaDeviceSynchronize());
+        free_dev(c->d_h_tokens); free_dev(c->d_h_hidden); free_dev(c->d_h_out);
+        free_dev(c->d_h_phrase); free_dev(c->d_h_slot); free_dev(c->d_h_flag);
+        c->d_h_tokens = nullptr; c->d_h_hidden = c->d_h_out = nullptr;
+        c->d_h_phrase = nullptr; c->d_h_slot = nullptr; c->d_h_flag = nullptr;
+        c->hb_tok_cap = c->hb_q_cap = c->hb_ent_cap = 0;
+        const int64_t tok_cap = std::max(n_tok, c->hb_tok_cap), q_cap = std::max(Q, c->hb_q_cap);
+        const int64_t e_cap = std::max<int64_t>(ent, q_cap * c->cfg.n_orders);
+        const size_t row_bytes = (size_t)c->cfg.d * (c->cfg.hidden_dtype == 0 ? 2 : 4);
+        CU(cudaMalloc(&c->d_h_tokens, (size_t)tok_cap * 4));
+        CU(cudaMalloc(&c->d_h_hidden, (size_t)q_cap * row_bytes));
+        CU(cudaMalloc(&c->d_h_out, (size_t)q_cap * row_bytes));
+        CU(cudaMalloc(&c->d_h_phrase, (size_t)e_cap * 4));
+        CU(cudaMalloc(&c->d_h_slot, (size_t)e_cap * 4));
+        CU(cudaMalloc(&c->d_h_flag, (size_t)e_cap));
+        c->hb_tok_cap = tok_cap; c->hb_q_cap = q_cap; c->hb_ent_cap = e_cap;
+    }
+    CU(cudaMemcpyAsync(c->d_h_tokens, tokens, (size_t)n_tok * 4, cudaMemcpyHostToDevice, stream));
+    CU(cudaMemcpyAsync(c->d_h_hidden, h, hid_bytes, cudaMemcpyHostToDevice, stream));
+    tfe_status st = tfe_lookup_inject(c, c->d_h_tokens, B, T, q_start, c->d_h_hidden, c->d_h_out, prm,
+                                      sel_phrase ? c->d_h_phrase : nullptr, sel_slot ? c->d_h_slot : nullptr,
+                                      flags ? c->d_h_flag : nullptr, stream_);
+    if (st != TFE_OK) return st;
+    CU(cudaMemcpyAsync(out, c->d_h_out, hid_bytes, cudaMemcpyDeviceToHost, stream));
+    if (sel_phrase) CU(cudaMemcpyAsync(sel_phrase, c->d_h_phrase, (size_t)ent * 4, cudaMemcpyDeviceToHost, stream));
+    if (sel_slot) CU(cudaMemcpyAsync(sel_slot, c->d_h_slot, (size_t)ent * 4, cudaMemcpyDeviceToHost, stream));
+    if (flags) CU(cudaMemcpyAsync(flags, c->d_h_flag, (size_t)ent, cudaMemcpyDeviceToHost, stream));
+    return TFE_OK;
+}
+
+tfe_status tfe_miss_list(tfe_ctx *c, uint32_t *q_idx, uint32_t *phrase_id, uint8_t *tier, int64_t cap,
+                         int64_t *count, void *stream_)
+{
+    if (!c || !count || cap < 0) return TFE_ERR_INVALID_ARG;
+    if (cap > 0 && (!q_idx || !phrase_id || !tier)) return TFE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    *count = 0;
+    if (c->last_entries <= 0) {
+        CU(cudaStreamSynchronize(stream));
+        return c->last_entries < 0 ? TFE_ERR_INVALID_ARG : TFE_OK;
+    }
+    uint32_t words[TFE_CTR_WORDS] = {0};
+    CU(cudaMemcpyAsync(words, c->d_counters, sizeof words, cudaMemcpyDeviceToHost, stream));
+    CU(cudaStreamSynchronize(stream));
+    if (words[TFE_CTR_STATUS] & TFE_DEV_WAIT_EXPIRED) {
+        CU(cudaMemsetAsync(c->d_counters + TFE_CTR_STATUS, 0, 4, stream));
+        return TFE_ERR_INTERNAL;
+    }
+    const int64_t n = words[TFE_CTR_TOTAL];
+    *count = n;
+    const int64_t take = std::min(n, cap);
+    if (take > 0) {
+        CU(cudaMemcpyAsync(q_idx, c->d_miss_q, (size_t)take * 4, cudaMemcpyDeviceToHost, stream));
+        CU(cudaMemcpyAsync(phrase_id, c->d_miss_phrase, (size_t)take * 4, cudaMemcpyDeviceToHost, stream));
+        CU(cudaMemcpyAsync(tier, c->d_miss_tier, (size_t)take, cudaMemcpyDeviceToHost, stream));
+        CU(cudaStreamSynchronize(stream));
+    }
+    return n > cap ? TFE_ERR_MISS_OVERFLOW : TFE_OK;
+}
+
+tfe_status tfe_miss_list_device(tfe_ctx *c, const uint32_t **q_idx, const uint32_t **phrase_id,
+                                const uint8_t **tier, const uint32_t **count)
+{
+    if (!c || c->last_entries < 0) return TFE_ERR_INVALID_ARG;
+    if (q_idx) *q_idx = c->d_miss_q;
+    if (phrase_id) *phrase_id = c->d_miss_phrase;
+    if (tier) *tier = c->d_miss_tier;
+    if (count) *count = c->d_counters + TFE_CTR_TOTAL;
+    return TFE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,85 @@
+"""A small convenience layer over the C-ABI binding: owns a context and the
+result tensors, so a caller writes ``eng.lookup_inject(tokens, h)``.
+
+Nothing is computed here -- every call goes straight to libtfe.so.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+from . import binding as tfe
+
+
+@dataclass
+class LookupOutput:
+    out: torch.Tensor          # [Q, d] hidden dtype
+    sel_phrase: torch.Tensor   # uint32 bit patterns in an int32 tensor, [Q] or [Q, n_orders]
+    sel_slot: torch.Tensor     # int32
+    flags: torch.Tensor        # uint8
+
+
+class Engram:
+    """GPU-resident phrase index + GPU-tier row store for one table."""
+
+    def __init__(self, phrase_tokens, phrase_len, init_slot, gpu_rows: torch.Tensor, *, vocab, orders,
+                 load_factor=0.7, hidden_dtype=tfe.HIDDEN_BF16, max_probe_buckets=0, stream=None):
+        assert gpu_rows.is_cuda and gpu_rows.dtype == torch.bfloat16 and gpu_rows.is_contiguous()
+        self.rows = gpu_rows
+        self.C, self.d = gpu_rows.shape
+        self.orders = tuple(int(o) for o in orders)
+        self.hidden_dtype = hidden_dtype
+        self.torch_hidden = torch.bfloat16 if hidden_dtype == tfe.HIDDEN_BF16 else torch.float32
+        self.cfg = tfe.make_config(d=self.d, vocab=vocab, orders=self.orders, n_phrases=len(phrase_len),
+                                   gpu_slots=self.C, load_factor=load_factor, hidden_dtype=hidden_dtype,
+                                   max_probe_buckets=max_probe_buckets)
+        self.ctx = tfe.tfe_index_build(self.cfg, phrase_tokens, phrase_len, init_slot, gpu_rows, stream)
+
+    def close(self):
+        if self.ctx:
+            tfe.tfe_destroy(self.ctx)
+            self.ctx = 0
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def lookup_inject(self, tokens: torch.Tensor, h: torch.Tensor, out: torch.Tensor | None = None, *,
+                      q_start=0, policy=tfe.POLICY_LONGEST, gate=tfe.GATE_CONST, lam=1.0, want_sel=True,
+                      stream=None) -> LookupOutput:
+        B, T = tokens.shape
+        Q = B * (T - q_start)
+        assert tokens.dtype == torch.int32 and tokens.is_cuda
+        assert h.shape == (Q, self.d) and h.dtype == self.torch_hidden
+        if out is None:
+            out = torch.empty_like(h)
+        shape = (Q,) if policy == tfe.POLICY_LONGEST else (Q, len(self.orders))
+        sp = ss = fl = None
+        if want_sel:
+            sp = torch.empty(shape, dtype=torch.int32, device=h.device)
+            ss = torch.empty(shape, dtype=torch.int32, device=h.device)
+            fl = torch.empty(shape, dtype=torch.uint8, device=h.device)
+        tfe.tfe_lookup_inject(self.ctx, tokens, B, T, q_start, h, out, policy=policy, gate=gate, lam=lam,
+                              sel_phrase=sp, sel_slot=ss, flags=fl, stream=stream)
+        return LookupOutput(out, sp, ss, fl)
+
+    def miss_list(self, cap: int | None = None, stream=None, allow_overflow=False):
+        if cap is None:
+            cap = 1 << 20
+        return tfe.tfe_miss_list(self.ctx, cap, stream, allow_overflow)
+
+    def cache_install(self, phrase_ids, src_rows, dst_slots, stream=None):
+        tfe.tfe_cache_install(self.ctx, phrase_ids, src_rows, dst_slots, stream)
+
+
+def bf16_tensor_from_bits(bits: np.ndarray, device) -> torch.Tensor:
+    """uint16 bit patterns -> torch.bfloat16 tensor on ``device`` (no conversion)."""
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(device).view(torch.bfloat16)
+
+
+def bits_from_bf16_tensor(t: torch.Tensor) -> np.ndarray:
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)

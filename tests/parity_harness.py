@@ -1,0 +1,118 @@
+"""Shared plumbing of the GPU parity tests: build the same table on the GPU
+(library) and on the CPU (oracle), run both on the same inputs, compare."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import tfe_oracle as orc
+from paper_2607_07388_b200 import binding as tfe
+from paper_2607_07388_b200 import synth
+from paper_2607_07388_b200.engine import Engram, bf16_tensor_from_bits, bits_from_bf16_tensor
+
+DEV = "cuda:0"
+TOL_BF16 = 2e-2     # max-abs on bf16 outputs against the exact (fp64) value
+TOL_F32 = 1e-5      # fp32 hidden states
+
+
+def phrases_to_arrays(phrases):
+    pt = np.full((len(phrases), 4), -1, np.int32)
+    pl = np.zeros(len(phrases), np.uint8)
+    for i, p in enumerate(phrases):
+        pt[i, :len(p)] = p
+        pl[i] = len(p)
+    return pt, pl
+
+
+class Pair:
+    """One table, twice: ``eng`` on the GPU, ``ora`` on the CPU."""
+
+    def __init__(self, pt, pl, init_slot, rows_bits, *, vocab, orders, load_factor=0.7, hidden_dtype=0,
+                 max_probe_buckets=0):
+        self.rows_bits = np.ascontiguousarray(rows_bits, np.uint16)
+        C, d = self.rows_bits.shape
+        self.d, self.C, self.orders, self.hidden_dtype = d, C, tuple(orders), hidden_dtype
+        self.rows_gpu = bf16_tensor_from_bits(self.rows_bits, DEV)
+        self.eng = Engram(pt, pl, init_slot, self.rows_gpu, vocab=vocab, orders=orders,
+                          load_factor=load_factor, hidden_dtype=hidden_dtype,
+                          max_probe_buckets=max_probe_buckets)
+        self.ora = orc.Oracle(pt, pl, init_slot, self.rows_bits.copy(), d=d, vocab=vocab, orders=orders,
+                              gpu_slots=C)
+
+    def close(self):
+        self.eng.close()
+
+    def hidden_to_gpu(self, h):
+        if self.hidden_dtype == 0:
+            return bf16_tensor_from_bits(h, DEV)
+        return torch.from_numpy(np.ascontiguousarray(h, np.float32)).to(DEV)
+
+    def hidden_from_gpu(self, t):
+        if self.hidden_dtype == 0:
+            return bits_from_bf16_tensor(t)
+        return t.detach().cpu().numpy()
+
+    def run_and_compare(self, tokens, h, *, q_start=0, policy=0, gate=0, lam=1.0, in_place=False,
+                        want_sel=True, matcher="sorted", expect_bit_exact=None):
+        """Runs GPU and oracle, asserts parity, returns (gpu LookupOutput, oracle LookupResult)."""
+        tokens = np.ascontiguousarray(tokens, np.int32)
+        lam = float(np.float32(lam))          # the library takes the scale as a float
+        tok_gpu = torch.from_numpy(tokens).to(DEV)
+        h_gpu = self.hidden_to_gpu(h)
+        h_keep = h_gpu.clone()
+        out_gpu = h_gpu if in_place else None
+        got = self.eng.lookup_inject(tok_gpu, h_gpu, out_gpu, q_start=q_start, policy=policy, gate=gate,
+                                     lam=lam, want_sel=want_sel)
+        mq, mp, mt, cnt = self.eng.miss_list()
+        torch.cuda.synchronize()
+        ref = self.ora.lookup(tokens, q_start, policy, matcher)
+        exact, rounded = self.ora.inject(ref, h, policy=policy, gate=gate, lam=lam,
+                                         hidden_dtype=self.hidden_dtype)
+        # integer results: bit-exact
+        if want_sel:
+            np.testing.assert_array_equal(got.sel_phrase.cpu().numpy().view(np.uint32), ref.sel_phrase)
+            np.testing.assert_array_equal(got.sel_slot.cpu().numpy(), ref.sel_slot)
+            np.testing.assert_array_equal(got.flags.cpu().numpy(), ref.flags)
+        assert cnt == len(ref.miss_q)
+        np.testing.assert_array_equal(mq, ref.miss_q)
+        np.testing.assert_array_equal(mp, ref.miss_phrase)
+        np.testing.assert_array_equal(mt, ref.miss_tier)
+        # hidden states
+        out = self.hidden_from_gpu(got.out)
+        if not in_place:
+            assert torch.equal(h_gpu, h_keep), "input hidden states were modified"
+        touched = (ref.flags.reshape(len(ref.flags), -1) == 1).any(axis=1)
+        np.testing.assert_array_equal(out[~touched], np.asarray(h)[~touched])      # bitwise pass-through
+        if self.hidden_dtype == 0:
+            val = synth.bf16_bits_to_f32(out).astype(np.float64)
+            err = np.abs(val - exact).max() if exact.size else 0.0
+            assert err <= TOL_BF16, err
+            n_diff = int((out != rounded).sum())
+        else:
+            err = np.abs(out.astype(np.float64) - exact).max() if exact.size else 0.0
+            assert err <= TOL_F32, err
+            n_diff = int((out != rounded).sum())
+        if expect_bit_exact is None:
+            # One fused multiply-add per element.  fp32 hidden: it is correctly rounded, like the
+            # oracle's double -> float.  bf16 hidden: lambda a power of two (or 0) makes lambda*m exact
+            # and h + lambda*m is then rounded once on both sides.
+            mant = np.frexp(lam)[0] if lam != 0 else 0.5
+            expect_bit_exact = gate == 0 and policy == 0 and (self.hidden_dtype == 1 or abs(mant) == 0.5)
+        if expect_bit_exact:
+            assert n_diff == 0, n_diff
+        elif self.hidden_dtype == 0:
+            # fp32 on the GPU against fp64 in the oracle: a result may land on the other side of a
+            # rounding boundary, rarely, and then by one unit in the last place only
+            assert n_diff <= max(2, out.size // 2000), n_diff
+            if self.hidden_dtype == 0 and n_diff:
+                d_bits = np.abs(out.astype(np.int32) - rounded.astype(np.int32))
+                assert d_bits.max() <= 1 or (np.abs(val - exact).max() <= TOL_BF16)
+        return got, ref, dict(max_abs_err=float(err), n_bits_differ=n_diff, n_hit=int(touched.sum()),
+                              n_miss=int(cnt))
+
+
+def pair_from_workload(w: synth.Workload, **kw):
+    tb = synth.make_table(w)
+    rows = synth.make_rows_np(w, tb)
+    return tb, Pair(tb.phrase_tokens, tb.phrase_len, tb.init_slot, rows, vocab=w.vocab, orders=w.orders,
+                    load_factor=w.load_factor, **kw)

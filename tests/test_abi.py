@@ -1,0 +1,111 @@
+"""CPU-side checks of the C-ABI library: it loads, exports what the header
+declares, refuses bad arguments before touching a device, and its key / bucket
+functions are exact and uniform.  No kernel is launched here."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def tfe():
+    from paper_2607_07388_b200 import binding, build
+    build.build()
+    binding.lib()
+    return binding
+
+
+def test_library_exports_every_declared_symbol(tfe):
+    header = open(os.path.join(ROOT, "include", "tfe.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(tfe_[a-z0-9_]+)\s*\(", header))
+    assert declared == set(tfe.EXPORTS)
+    L = tfe.lib()
+    for name in declared:
+        assert getattr(L, name) is not None
+
+
+def test_status_strings(tfe):
+    seen = {tfe.lib().tfe_status_string(i).decode() for i in range(12)}
+    assert len(seen) == 12 and "ok" in seen
+
+
+def _build_status(tfe, cfg, pt, pl, sl, rows_addr=0x1000):
+    out = C.c_void_p()
+    return tfe.lib().tfe_index_build(C.byref(cfg), pt.ctypes.data, pl.ctypes.data, sl.ctypes.data,
+                                     rows_addr, None, C.byref(out))
+
+
+def test_build_refuses_bad_arguments_on_the_host(tfe):
+    pt = np.array([[1, 2, -1, -1], [3, 4, 5, -1]], np.int32)
+    pl = np.array([2, 3], np.uint8)
+    sl = np.array([0, -1], np.int32)
+    ok = dict(d=16, vocab=10, orders=(2, 3), n_phrases=2, gpu_slots=2)
+    bad_cfgs = [dict(ok, d=12), dict(ok, d=0), dict(ok, vocab=0), dict(ok, orders=(3, 2)),
+                dict(ok, orders=(0, 2)), dict(ok, orders=(2, 5)), dict(ok, load_factor=0.0),
+                dict(ok, load_factor=1.5), dict(ok, hidden_dtype=2), dict(ok, gpu_slots=-1)]
+    for kw in bad_cfgs:
+        assert _build_status(tfe, tfe.make_config(**kw), pt, pl, sl) == tfe.TFE_ERR_INVALID_ARG, kw
+    cfg = tfe.make_config(**ok)
+    assert _build_status(tfe, cfg, pt, pl, sl, rows_addr=0x1004) == tfe.TFE_ERR_INVALID_ARG   # misaligned rows
+    assert _build_status(tfe, cfg, pt, np.array([2, 4], np.uint8), sl) == tfe.TFE_ERR_INVALID_ARG  # 4 not an order
+    bad_tok = pt.copy(); bad_tok[1, 2] = 10
+    assert _build_status(tfe, cfg, bad_tok, pl, sl) == tfe.TFE_ERR_INVALID_ARG
+    assert _build_status(tfe, cfg, pt, pl, np.array([0, 2], np.int32)) == tfe.TFE_ERR_SLOT_RANGE
+    assert _build_status(tfe, cfg, pt, pl, np.array([1, 1], np.int32)) == tfe.TFE_ERR_SLOT_RANGE
+    assert _build_status(tfe, cfg, pt, pl, np.array([0, -3], np.int32)) == tfe.TFE_ERR_INVALID_ARG
+    dup = np.array([[1, 2, -1, -1], [1, 2, -1, -1]], np.int32)
+    assert _build_status(tfe, tfe.make_config(**dict(ok, orders=(2,))), dup, np.array([2, 2], np.uint8), sl) \
+        == tfe.TFE_ERR_DUPLICATE_PHRASE
+
+
+def test_packed_keys_are_injective_and_nonzero(tfe):
+    # every tuple of orders 1..3 over a small vocabulary: all keys distinct, none zero
+    V = 13
+    keys = {}
+    for n in (1, 2, 3):
+        for idx in np.ndindex(*([V] * n)):
+            k, exact = tfe.tfe_phrase_key64(V, idx)
+            assert exact and k != 0
+            assert k not in keys, (idx, keys.get(k))
+            keys[k] = idx
+    # the benchmark vocabulary: orders <= 3 are packed (3 * 18 bits), order 4 is hashed + verified
+    V = 151_936
+    assert tfe.tfe_phrase_key64(V, [V - 1, 0, V - 1])[1] is True
+    assert tfe.tfe_phrase_key64(V, [1, 2, 3, 4])[1] is False
+    # token order matters, padding gives no key
+    assert tfe.tfe_phrase_key64(V, [1, 2])[0] != tfe.tfe_phrase_key64(V, [2, 1])[0]
+    assert tfe.tfe_phrase_key64(V, [1, 2, 3, 4])[0] != tfe.tfe_phrase_key64(V, [4, 3, 2, 1])[0]
+    assert tfe.tfe_phrase_key64(V, [1, V])[0] == 0 and tfe.tfe_phrase_key64(V, [-1, 2])[0] == 0
+    # extreme corners stay distinct
+    corner = {tfe.tfe_phrase_key64(V, t)[0] for t in ([0, 0], [0, 0, 0], [0, 1], [1, 0], [0, 0, 1], [V - 1, V - 1],
+                                                        [V - 1, V - 1, V - 1], [0], [V - 1])}
+    assert len(corner) == 9
+
+
+def test_home_buckets_follow_the_papers_occupancy_formula(tfe):
+    # M phrase keys into B buckets: the number of distinct home buckets must match the closed form
+    # B * (1 - (1 - 1/B)^M) the paper gives for uniform hashing (Sec. 3.1), within 1 %.
+    rng = np.random.default_rng(7)
+    V = 151_936
+    for M, B, n in ((200_000, 200_000, 2), (200_000, 50_000, 3), (100_000, 142_858, 4), (50_000, 7_919, 2)):
+        toks = rng.integers(0, V, size=(M, n)).astype(np.int32)
+        toks[: M // 2, 0] = toks[0, 0]            # half the phrases share their first token
+        toks = np.unique(toks, axis=0)
+        homes = {tfe.tfe_home_bucket(tfe.tfe_phrase_key64(V, t)[0], B) for t in toks}
+        assert max(homes) < B
+        expect = B * (1.0 - (1.0 - 1.0 / B) ** len(toks))
+        assert abs(len(homes) - expect) / expect < 0.01, (M, B, n, len(homes), expect)
+
+
+def test_index_bytes_per_entry_below_the_papers_overhead():
+    # The paper's 100M-entry table takes 215.86 GB with 1024-dim FP16 vectors (Sec. 5.3):
+    # 2158.6 B per entry, of which 2048 B are the vector, so ~110 B of index + metadata.
+    paper_overhead = 215.86e9 / 100e6 - 2048
+    assert 100 < paper_overhead < 120
+    ours = 16 / 0.7 + 4 + 4 + 16        # index slot / load factor + position + owner + stored tuple
+    assert ours < paper_overhead
