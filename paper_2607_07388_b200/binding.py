@@ -13,7 +13,7 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libtfe.so")
+LIB_PATH = os.environ.get("TFE_LIB") or os.path.join(_HERE, "libtfe.so")   # TFE_LIB: a tuning build
 
 TFE_OK = 0
 STATUS_NAMES = ["TFE_OK", "TFE_ERR_INVALID_ARG", "TFE_ERR_DUPLICATE_PHRASE", "TFE_ERR_KEY_COLLISION",
@@ -31,7 +31,7 @@ NO_PHRASE = 0xFFFFFFFF
 EXPORTS = ["tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
            "tfe_miss_list", "tfe_miss_list_device", "tfe_destroy", "tfe_status_string",
            "tfe_last_cuda_error", "tfe_index_geometry", "tfe_phrase_key64", "tfe_home_bucket",
-           "tfe_launch_geometry"]
+           "tfe_launch_geometry", "tfe_set_tuning"]
 
 
 class TfeConfig(C.Structure):
@@ -82,9 +82,11 @@ def lib() -> C.CDLL:
         L.tfe_phrase_key64.restype = u64
         L.tfe_home_bucket.argtypes = [u64, u64]
         L.tfe_home_bucket.restype = u64
-        L.tfe_launch_geometry.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
+        L.tfe_launch_geometry.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
+        L.tfe_set_tuning.argtypes = [vp, i32, i32]
         for name in ("tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
-                     "tfe_miss_list", "tfe_miss_list_device", "tfe_index_geometry", "tfe_launch_geometry"):
+                     "tfe_miss_list", "tfe_miss_list_device", "tfe_index_geometry", "tfe_launch_geometry",
+                     "tfe_set_tuning"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -203,9 +205,17 @@ def tfe_index_geometry(ctx: int):
 
 
 def tfe_launch_geometry(ctx: int):
-    g, b = C.c_int32(), C.c_int32()
-    _check(lib().tfe_launch_geometry(ctx, C.byref(g), C.byref(b)), "tfe_launch_geometry")
-    return g.value, b.value
+    """(grid, block, queries per warp batch, bulk-copy staged?) of the most recent lookup."""
+    g, b, t, s = C.c_int32(), C.c_int32(), C.c_int32(), C.c_int32()
+    _check(lib().tfe_launch_geometry(ctx, C.byref(g), C.byref(b), C.byref(t), C.byref(s)), "tfe_launch_geometry")
+    return g.value, b.value, t.value, s.value
+
+
+KERNEL_AUTO, KERNEL_REGISTER, KERNEL_STAGED = 0, 1, 2
+
+
+def tfe_set_tuning(ctx: int, batch_queries: int = 0, kernel: int = KERNEL_AUTO) -> None:
+    _check(lib().tfe_set_tuning(ctx, int(batch_queries), int(kernel)), "tfe_set_tuning")
 
 
 def tfe_phrase_key64(vocab: int, tokens) -> tuple[int, bool]:

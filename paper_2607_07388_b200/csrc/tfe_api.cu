@@ -5,6 +5,8 @@
 // GPU-tier slot), the miss-list buffers, and a host mirror of the residency state
 // used to validate arguments before anything is launched.
 #include <algorithm>
+#include <climits>
+#include <cstdint>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -32,6 +34,7 @@ bool cuda_failed(cudaError_t e, const char *what)
 
 constexpr uint32_t kNoOwner = 0xFFFFFFFFu;
 constexpr int kDefaultMaxProbe = 64;
+constexpr int kVarSlots = 16;
 
 }  // namespace
 
@@ -60,12 +63,16 @@ struct tfe_ctx {
     uint32_t *d_miss_q = nullptr, *d_miss_phrase = nullptr;
     uint8_t *d_miss_tier = nullptr;
     uint32_t *d_counters = nullptr;         // TFE_CTR_WORDS words of launch state
-    unsigned long long *d_block_state = nullptr;
-    int max_grid = 0;
-    int occ[8] = {0};                       // resident blocks per SM of each kernel variant
+    int occ[kVarSlots] = {0};
+    int occ_tma[3] = {0};                   // the bulk-copy staged kernels: bf16 fp32-math, bf16 packed, fp32 hidden                      // resident blocks per SM of each kernel variant
 
     int64_t last_entries = -1;              // Q*cols of the most recent lookup (-1: none yet)
-    int last_grid = 0;
+#ifdef TFE_DBG_TIMELINE
+    long long *dbg = nullptr;
+#endif
+    int last_grid = 0, last_block = 0, last_qb = 0, last_staged = 0;
+    int qb_override = 0;                    // 0: choose per call
+    int kernel_override = 0;                // 0: choose per call, 1: register-staged, 2: bulk-copy staged
 
     // install staging
     uint32_t *d_inst_ids = nullptr;
@@ -86,15 +93,55 @@ namespace {
 
 typedef void (*lookup_kernel_t)(const TfeLookupParams);
 
-lookup_kernel_t pick_kernel(int ht, int all, int cos)
+// Kernel variants.  0..7: hidden dtype x policy x gate in fp32 arithmetic;
+// 8: bf16 hidden, LONGEST / CONST with the packed bf16 fused multiply-add (lambda a bf16 number).
+enum { kVarPacked = 8, kVarCount = 9 };
+
+lookup_kernel_t pick_kernel(int variant)
 {
-    static const lookup_kernel_t table[8] = {
-        tfe_lookup_inject_kernel<0, false, false>, tfe_lookup_inject_kernel<0, false, true>,
-        tfe_lookup_inject_kernel<0, true, false>,  tfe_lookup_inject_kernel<0, true, true>,
-        tfe_lookup_inject_kernel<1, false, false>, tfe_lookup_inject_kernel<1, false, true>,
-        tfe_lookup_inject_kernel<1, true, false>,  tfe_lookup_inject_kernel<1, true, true>,
+    static const lookup_kernel_t table[kVarCount] = {
+        tfe_lookup_inject_kernel<0, false, false, false>, tfe_lookup_inject_kernel<0, false, true, false>,
+        tfe_lookup_inject_kernel<0, true, false, false>,  tfe_lookup_inject_kernel<0, true, true, false>,
+        tfe_lookup_inject_kernel<1, false, false, false>, tfe_lookup_inject_kernel<1, false, true, false>,
+        tfe_lookup_inject_kernel<1, true, false, false>,  tfe_lookup_inject_kernel<1, true, true, false>,
+        tfe_lookup_inject_kernel<0, false, false, true>,
     };
-    return table[ht * 4 + all * 2 + cos];
+    return table[variant];
+}
+
+// Bulk-copy staged kernels for large out-of-place LONGEST / CONST calls.
+typedef void (*tma_kernel_t)(const TfeLookupParams, uint32_t);
+
+tma_kernel_t pick_tma_kernel(int ht, bool packed)
+{
+    if (ht == 1) return tfe_lookup_inject_tma_kernel<1, false>;
+    return packed ? tfe_lookup_inject_tma_kernel<0, true> : tfe_lookup_inject_tma_kernel<0, false>;
+}
+
+// Queries per warp batch (1..8) for a call of Q queries on `warps` resident warps: the split into
+// r rounds of ceil(Q / (warps*r)) queries that leaves the busiest warp the least work.
+int pick_batch(int64_t Q, int64_t warps)
+{
+    if (Q <= warps) return 1;
+    int best_qb = 8;
+    int64_t best_load = INT64_MAX;
+    for (int64_t r = 1; r <= 64; ++r) {
+        const int64_t qb = (Q + warps * r - 1) / (warps * r);
+        if (qb > 8) continue;
+        if (r * qb < best_load) { best_load = r * qb; best_qb = (int)qb; }
+        if (qb == 1) break;
+    }
+    return best_qb;
+}
+
+TfeFastDiv make_fastdiv(uint32_t d)
+{
+    uint32_t s = 0;
+    while ((1ull << s) < d) ++s;
+    TfeFastDiv f;
+    f.shr = 31 + s;
+    f.mul = (uint32_t)((1ull << f.shr) / d + 1);
+    return f;
 }
 
 void free_dev(void *p) { if (p) (void)cudaFree(p); }
@@ -193,7 +240,7 @@ void tfe_destroy(tfe_ctx *c)
     free_dev(c->d_index); free_dev(c->d_phrase_tokens); free_dev(c->d_phrase_pos);
     free_dev(c->d_slot_owner); free_dev(c->d_scr_phrase); free_dev(c->d_scr_flag);
     free_dev(c->d_miss_q); free_dev(c->d_miss_phrase); free_dev(c->d_miss_tier);
-    free_dev(c->d_counters); free_dev(c->d_block_state);
+    free_dev(c->d_counters);
     free_dev(c->d_inst_ids); free_dev(c->d_inst_slots); free_dev(c->d_inst_rows);
     free_dev(c->d_h_tokens); free_dev(c->d_h_hidden); free_dev(c->d_h_out);
     free_dev(c->d_h_phrase); free_dev(c->d_h_slot); free_dev(c->d_h_flag);
@@ -306,17 +353,19 @@ tfe_status tfe_index_build(const tfe_config *cfg, const int32_t *phrase_tokens,
         CUF(cudaMemcpyAsync(c->d_phrase_tokens, phrase_tokens, (size_t)N * sizeof(int4),
                             cudaMemcpyHostToDevice, stream));
     }
-    int max_occ = 1;
-    for (int v = 0; v < 8; ++v) {
+    for (int v = 0; v < kVarCount; ++v) {
         int occ = 0;
-        CUF(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, pick_kernel(v >> 2, (v >> 1) & 1, v & 1),
-                                                          TFE_BLOCK_THREADS, 0));
+        CUF(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, pick_kernel(v), TFE_BLOCK_THREADS, 0));
         c->occ[v] = std::max(1, occ);
-        max_occ = std::max(max_occ, c->occ[v]);
     }
-    c->max_grid = c->sm_count * max_occ;
-    CUF(cudaMalloc(&c->d_block_state, (size_t)c->max_grid * sizeof(unsigned long long)));
-    CUF(cudaMemsetAsync(c->d_block_state, 0, (size_t)c->max_grid * sizeof(unsigned long long), stream));
+    for (int v = 0; v < 3; ++v) {
+        int occ = 0;
+        CUF(cudaFuncSetAttribute(pick_tma_kernel(v == 2, v == 1), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 TFE_TMA_SMEM));
+        CUF(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, pick_tma_kernel(v == 2, v == 1), TFE_TMA_THREADS,
+                                                          TFE_TMA_SMEM));
+        c->occ_tma[v] = std::max(1, occ);
+    }
     if (N > 0) {
         CUF(cudaMalloc(&d_keys, (size_t)N * 8));
         CUF(cudaMalloc(&d_slots, (size_t)N * 4));
@@ -332,12 +381,8 @@ tfe_status tfe_index_build(const tfe_config *cfg, const int32_t *phrase_tokens,
     if (h_status & TFE_DEV_PROBE_LIMIT) rc = TFE_ERR_PROBE_LIMIT;
     else if (h_status & TFE_DEV_DUP_KEY) rc = TFE_ERR_DUPLICATE_PHRASE;
     if (rc != TFE_OK) return fail(rc);
-    {
-        uint32_t init[TFE_CTR_WORDS] = {0};
-        init[TFE_CTR_EPOCH] = 1;
-        CUF(cudaMemcpyAsync(c->d_counters, init, sizeof init, cudaMemcpyHostToDevice, stream));
-        CUF(cudaStreamSynchronize(stream));
-    }
+    CUF(cudaMemsetAsync(c->d_counters, 0, TFE_CTR_WORDS * sizeof(uint32_t), stream));
+    CUF(cudaStreamSynchronize(stream));
 #undef CUF
     free_dev(d_keys); free_dev(d_slots);
     *out = c;
@@ -356,11 +401,30 @@ tfe_status tfe_index_geometry(const tfe_ctx *c, int64_t *n_buckets, int64_t *ind
     return TFE_OK;
 }
 
-tfe_status tfe_launch_geometry(const tfe_ctx *c, int32_t *grid, int32_t *block)
+#ifdef TFE_DBG_TIMELINE
+tfe_status tfe_debug_timeline(tfe_ctx *c, void *device_buffer)
+{
+    c->dbg = static_cast<long long *>(device_buffer);
+    return TFE_OK;
+}
+#endif
+
+tfe_status tfe_set_tuning(tfe_ctx *c, int32_t batch_queries, int32_t kernel)
+{
+    if (!c || batch_queries < 0 || batch_queries > 8 || kernel < 0 || kernel > 2) return TFE_ERR_INVALID_ARG;
+    c->qb_override = batch_queries;
+    c->kernel_override = kernel;
+    return TFE_OK;
+}
+
+tfe_status tfe_launch_geometry(const tfe_ctx *c, int32_t *grid, int32_t *block, int32_t *batch_queries,
+                               int32_t *staged)
 {
     if (!c) return TFE_ERR_INVALID_ARG;
     if (grid) *grid = c->last_grid;
-    if (block) *block = TFE_BLOCK_THREADS;
+    if (block) *block = c->last_block;
+    if (batch_queries) *batch_queries = c->last_qb;
+    if (staged) *staged = c->last_staged;
     return TFE_OK;
 }
 
@@ -448,30 +512,58 @@ tfe_status tfe_lookup_inject(tfe_ctx *c, const int32_t *tokens, int32_t B, int32
     tfe_status st = ensure_entries(c, Q * cols);
     if (st != TFE_OK) return st;
 
-    const int variant = c->cfg.hidden_dtype * 4 + (prm->policy == TFE_POLICY_ALL ? 2 : 0) +
-                        (prm->gate == TFE_GATE_COSINE ? 1 : 0);
-    const int64_t resident = (int64_t)c->sm_count * c->occ[variant];
-    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(resident, (Q + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK));
-
+    const bool all = prm->policy == TFE_POLICY_ALL, cos = prm->gate == TFE_GATE_COSINE;
+    uint32_t lam_bits;
+    std::memcpy(&lam_bits, &prm->lambda, sizeof lam_bits);
+    const bool lam_is_bf16 = (lam_bits & 0xFFFFu) == 0 && (lam_bits & 0x7F800000u) != 0x7F800000u;
+    const int ht = c->cfg.hidden_dtype;
+    const int variant = (all || cos) ? ht * 4 + (all ? 2 : 0) + (cos ? 1 : 0)
+                                     : ((ht == 0 && lam_is_bf16) ? kVarPacked : ht * 4);
+    // Large out-of-place LONGEST / CONST calls go through the bulk-copy staged kernel (h rows are
+    // requested before the probe and wait in shared memory); everything else -- small calls where
+    // latency counts, in-place calls, ALL / COSINE -- through the register-staged one.
+    const uint32_t row_bytes = (uint32_t)c->cfg.d * (ht == 0 ? 2u : 4u);
+    const int tma_idx = ht == 1 ? 2 : (lam_is_bf16 ? 1 : 0);
+    const int64_t tma_warps = (int64_t)c->sm_count * c->occ_tma[tma_idx] * TFE_TMA_WARPS;
+    bool use_tma = !all && !cos && h != out && row_bytes <= TFE_TMA_STAGE_BYTES;
+    if (c->kernel_override == 1) use_tma = false;
+    else if (c->kernel_override != 2) use_tma = use_tma && Q >= 2 * tma_warps;
+    const int64_t resident = use_tma ? (int64_t)c->sm_count * c->occ_tma[tma_idx]
+                                     : (int64_t)c->sm_count * c->occ[variant];
+    const int warps_per_block = use_tma ? TFE_TMA_WARPS : TFE_WARPS_PER_BLOCK;
+    const int64_t qb = c->qb_override ? c->qb_override : pick_batch(Q, resident * warps_per_block);
+    const int64_t n_batches = (Q + qb - 1) / qb;
+    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(resident, (n_batches + warps_per_block - 1) / warps_per_block));
     TfeLookupParams p{};
     p.tokens = tokens; p.B = B; p.T = T; p.q_start = q_start; p.Tq = (int32_t)Tq; p.Q = (uint32_t)Q;
+    p.div_tq = make_fastdiv((uint32_t)Tq); p.qb = (uint32_t)qb;
     p.index = c->d_index; p.n_buckets = c->n_buckets; p.max_probe = c->max_probe;
     p.phrase_tokens = c->d_phrase_tokens; p.rows = c->gpu_rows; p.d = c->cfg.d;
     p.h = h; p.out = out;
     p.n_orders = c->cfg.n_orders;
     for (int i = 0; i < 4; ++i) p.orders[i] = i < c->cfg.n_orders ? c->cfg.orders[i] : 0;
     p.tok_bits = c->tok_bits; p.vocab = c->cfg.vocab; p.lambda = prm->lambda;
+    p.lambda_bf16x2 = (lam_bits >> 16) | (lam_bits & 0xFFFF0000u);
     p.sel_phrase = sel_phrase; p.sel_slot = sel_slot; p.flags = flags;
     p.scr_phrase = c->d_scr_phrase; p.scr_flag = c->d_scr_flag;
     p.miss_q = c->d_miss_q; p.miss_phrase = c->d_miss_phrase; p.miss_tier = c->d_miss_tier;
-    p.counters = c->d_counters; p.block_state = c->d_block_state;
-    p.block_state_len = (uint32_t)c->max_grid;
-    p.q_per_block = (uint32_t)((Q + grid - 1) / grid);
+    p.counters = c->d_counters;
+#ifdef TFE_DBG_TIMELINE
+    p.dbg = c->dbg;
+#endif
 
-    pick_kernel(variant >> 2, (variant >> 1) & 1, variant & 1)<<<(unsigned)grid, TFE_BLOCK_THREADS, 0, stream>>>(p);
+    if (use_tma) {
+        const uint32_t stages = std::min<uint32_t>(TFE_TMA_MAX_STAGES, TFE_TMA_STAGE_BYTES / row_bytes);
+        pick_tma_kernel(ht, lam_is_bf16)<<<(unsigned)grid, TFE_TMA_THREADS, TFE_TMA_SMEM, stream>>>(p, stages);
+    } else {
+        pick_kernel(variant)<<<(unsigned)grid, TFE_BLOCK_THREADS, 0, stream>>>(p);
+    }
     CU(cudaGetLastError());
     c->last_entries = Q * cols;
     c->last_grid = (int)grid;
+    c->last_block = use_tma ? TFE_TMA_THREADS : TFE_BLOCK_THREADS;
+    c->last_staged = use_tma ? 1 : 0;
+    c->last_qb = (int)qb;
     return TFE_OK;
 }
 
@@ -533,7 +625,7 @@ tfe_status tfe_miss_list(tfe_ctx *c, uint32_t *q_idx, uint32_t *phrase_id, uint8
     uint32_t words[TFE_CTR_WORDS] = {0};
     CU(cudaMemcpyAsync(words, c->d_counters, sizeof words, cudaMemcpyDeviceToHost, stream));
     CU(cudaStreamSynchronize(stream));
-    if (words[TFE_CTR_STATUS] & TFE_DEV_WAIT_EXPIRED) {
+    if (words[TFE_CTR_STATUS] & TFE_DEV_COPY_TIMEOUT) {
         CU(cudaMemsetAsync(c->d_counters + TFE_CTR_STATUS, 0, 4, stream));
         return TFE_ERR_INTERNAL;
     }

@@ -20,17 +20,22 @@
 #define TFE_BLOCK_THREADS 256
 #define TFE_WARPS_PER_BLOCK (TFE_BLOCK_THREADS / 32)
 #define TFE_NONE64 0xFFFFFFFFFFFFFFFFull
-#define TFE_WAIT_LIMIT (8u << 20)      // polls of ~0.25 us each before a wait gives up
 
 // device status bits (counters[TFE_CTR_STATUS])
-#define TFE_DEV_WAIT_EXPIRED 1u
+#define TFE_DEV_COPY_TIMEOUT 1u
 #define TFE_DEV_PROBE_LIMIT 2u
 #define TFE_DEV_DUP_KEY 4u
+
+// Division by a divisor fixed per call: q = (n * mul) >> shr, exact for every n < 2^31
+// (mul = floor(2^shr / d) + 1, shr = 31 + ceil(log2 d); the host computes both).
+struct TfeFastDiv { uint32_t mul, shr; };
 
 struct TfeLookupParams {
     const int32_t *tokens;
     int32_t B, T, q_start, Tq;
     uint32_t Q;
+    TfeFastDiv div_tq;              // division by Tq
+    uint32_t qb;                    // queries per warp batch: 1, 2, 4 or 8
     const ulonglong2 *index;
     uint64_t n_buckets;
     int32_t max_probe;
@@ -44,6 +49,7 @@ struct TfeLookupParams {
     int32_t tok_bits;
     int32_t vocab;
     float lambda;
+    uint32_t lambda_bf16x2;         // lambda twice as bf16, valid when it is exactly a bf16 number
     uint32_t *sel_phrase;           // optional outputs
     int32_t *sel_slot;
     uint8_t *flags;
@@ -52,15 +58,16 @@ struct TfeLookupParams {
     uint32_t *miss_q, *miss_phrase; // context miss list, [Q*cols]
     uint8_t *miss_tier;
     uint32_t *counters;             // TFE_CTR_* words
-    unsigned long long *block_state;// [block_state_len] (epoch << 32) | misses of that block
-    uint32_t block_state_len, q_per_block;
+#ifdef TFE_DBG_TIMELINE
+    long long *dbg;                 // [warps][8] clock stamps
+#endif
 };
 
-// Device-resident launch state (uint32 words).  A lookup launch numbers its blocks with TICKET,
-// tags what it publishes with EPOCH, and its last block to finish resets TICKET / DONE, moves
-// RUNNING to TOTAL and advances EPOCH.  EPOCH starts at 1; tag 0 means "never written".
-enum { TFE_CTR_RUNNING = 0, TFE_CTR_TOTAL = 1, TFE_CTR_STATUS = 2, TFE_CTR_TICKET = 3, TFE_CTR_DONE = 4,
-       TFE_CTR_EPOCH = 5, TFE_CTR_WORDS = 8 };
+// Device-resident launch state (uint32 words).  Blocks of a lookup add their miss counts to
+// RUNNING and tick DONE when they finish; the block that finishes last compacts the miss list,
+// moves RUNNING to TOTAL and zeroes RUNNING / DONE for the next launch.  Because nothing of this
+// lives in kernel parameters, a launch can be replayed unchanged.
+enum { TFE_CTR_RUNNING = 0, TFE_CTR_TOTAL = 1, TFE_CTR_STATUS = 2, TFE_CTR_DONE = 3, TFE_CTR_WORDS = 4 };
 
 // ------------------------------------------------------------------ index build
 
@@ -117,18 +124,18 @@ __device__ __forceinline__ uint2 ld_row2(const uint2 *p)
     asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
     return v;
 }
-__device__ __forceinline__ ulonglong2 ld_slot(const ulonglong2 *p)
-{
-    ulonglong2 v;
-    asm volatile("ld.global.nc.v2.u64 {%0,%1}, [%2];" : "=l"(v.x), "=l"(v.y) : "l"(p));
-    return v;
-}
 __device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
 __device__ __forceinline__ uint32_t pack_bf2(float lo, float hi)   // round to nearest even
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
+}
+__device__ __forceinline__ uint32_t fma_bf16x2(uint32_t a, uint32_t b, uint32_t c)   // a*b + c per half
+{
+    uint32_t d;
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
 }
 __device__ __forceinline__ float warp_sum(float v)
 {
@@ -148,12 +155,17 @@ __device__ __forceinline__ bool tuple_matches(const int4 st, const int32_t (&tk)
     }
 }
 
-// The retained GPU-resident rows of one query and their aggregation weights.
-struct TfeRowSet {
-    const uint4 *ptr[4];
-    float alpha[4];
-    int n;
-};
+__device__ __forceinline__ ulonglong4 ld_bucket32(const ulonglong4 *p)    // 32 bytes = two index slots
+{
+    ulonglong4 v;
+    asm volatile("ld.global.nc.v4.u64 {%0,%1,%2,%3}, [%4];" : "=l"(v.x), "=l"(v.y), "=l"(v.z), "=l"(v.w) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ uint32_t tfe_div(uint32_t n, TfeFastDiv d)
+{
+    return (uint32_t)(((unsigned long long)n * d.mul) >> d.shr);
+}
 
 // Elements handled by one lane in one step: 8 (bf16 hidden: one 16-byte vector of h,
 // of the row and of out) or 4 (fp32 hidden: 16 bytes of h / out, 8 bytes of the row).
@@ -215,363 +227,583 @@ __device__ __forceinline__ void store_hidden(void *orow, int step_idx, const flo
     st_stream(reinterpret_cast<uint4 *>(orow) + step_idx, v);
 }
 
-// m = sum_r alpha_r * row_r for this lane's elements of one step (fp32, ascending order).
+// m = sum_r alpha_r * row_r for this lane's elements of one step (fp32, ascending order);
+// LONGEST keeps one row with weight 1, which this reproduces exactly.
 template <int HT, bool ALL>
-__device__ __forceinline__ void load_memory(const TfeRowSet &rs, int step_idx, float (&m)[TfeVec<HT>::N])
+__device__ __forceinline__ void load_memory(const uint4 *const (&rowp)[ALL ? 4 : 1], const float (&alpha)[ALL ? 4 : 1],
+                                            int step_idx, float (&m)[TfeVec<HT>::N])
 {
     if constexpr (!ALL) {
-        load_row<HT>(rs.ptr[0], step_idx, m);
+        load_row<HT>(rowp[0], step_idx, m);
     } else {
 #pragma unroll
         for (int k = 0; k < TfeVec<HT>::N; ++k) m[k] = 0.f;
-        for (int r = 0; r < rs.n; ++r) {
-            float e[TfeVec<HT>::N];
-            load_row<HT>(rs.ptr[r], step_idx, e);
 #pragma unroll
-            for (int k = 0; k < TfeVec<HT>::N; ++k) m[k] = fmaf(rs.alpha[r], e[k], m[k]);
+        for (int r = 0; r < 4; ++r) {
+            if (rowp[r] == nullptr) continue;
+            float e[TfeVec<HT>::N];
+            load_row<HT>(rowp[r], step_idx, e);
+#pragma unroll
+            for (int k = 0; k < TfeVec<HT>::N; ++k) m[k] = fmaf(alpha[r], e[k], m[k]);
         }
     }
 }
 
+// End of a lookup block.  Every thread has recorded flag bytes (and phrase ids of misses) in the
+// context scratch arrays; `my_miss` is warp-uniform.  Blocks add their miss counts to RUNNING and
+// tick DONE; the block that finishes last turns the flag bytes into the ordered miss list
+// (ascending entry index = ascending (q, order)), publishes TOTAL and re-arms the counters.
+__device__ __forceinline__ void tfe_finish_block(const TfeLookupParams &p, uint32_t my_miss, int cols)
+{
+    __shared__ uint32_t s_miss, s_last, s_total, s_scan;
+    __shared__ uint32_t s_warp[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n_warps_blk = (blockDim.x + 31) >> 5;
+    if (threadIdx.x == 0) s_miss = 0;
+    __syncthreads();
+    // ---- hand the block's miss count in; the block that finishes last builds the list
+    __threadfence();                       // this thread's flag / phrase records, device-wide
+    if (lane == 0 && my_miss) atomicAdd(&s_miss, my_miss);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (s_miss) atomicAdd(&p.counters[TFE_CTR_RUNNING], s_miss);
+        __threadfence();
+        s_last = atomicAdd(&p.counters[TFE_CTR_DONE], 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (threadIdx.x == 0) {
+        s_total = *(volatile uint32_t *)&p.counters[TFE_CTR_RUNNING];
+        s_scan = 0;
+    }
+    __syncthreads();
+    const uint32_t total = s_total;
+    if (total != 0) {
+        // order-stable compaction: every thread takes 16 consecutive flag bytes per round
+        const uint32_t n_ent = p.Q * (uint32_t)cols;
+        const uint32_t per_round = blockDim.x * 16;
+        for (uint32_t e0 = 0; e0 < n_ent; e0 += per_round) {
+            const uint32_t mine = e0 + threadIdx.x * 16;
+            uint32_t w[4] = {0, 0, 0, 0};
+            if (mine + 16 <= n_ent) {
+                const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(p.scr_flag + mine));
+                w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+            } else if (mine < n_ent) {
+                for (uint32_t k = 0; mine + k < n_ent; ++k)
+                    w[k >> 2] |= (uint32_t)__ldcg(p.scr_flag + mine + k) << (8 * (k & 3));
+            }
+            uint32_t cnt = 0;                    // flags 2 and 3 have bit 1 set
+#pragma unroll
+            for (int k = 0; k < 4; ++k) cnt += __popc(w[k] & 0x02020202u);
+            uint32_t incl = cnt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += n;
+            }
+            if (lane == 31) s_warp[warp] = incl;
+            __syncthreads();
+            uint32_t off = s_scan + incl - cnt;
+            for (int k = 0; k < warp; ++k) off += s_warp[k];
+            if (cnt) {
+#pragma unroll
+                for (int k = 0; k < 16; ++k) {
+                    const uint32_t flag = (w[k >> 2] >> (8 * (k & 3))) & 0xFFu;
+                    if (flag >= 2) {
+                        const uint32_t e = mine + k;
+                        p.miss_q[off] = e / (uint32_t)cols;
+                        p.miss_phrase[off] = __ldcg(p.scr_phrase + e);
+                        p.miss_tier[off] = (uint8_t)flag;
+                        ++off;
+                    }
+                }
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                uint32_t t = 0;
+                for (int k = 0; k < n_warps_blk; ++k) t += s_warp[k];
+                s_scan += t;
+            }
+            __syncthreads();
+        }
+    }
+    if (threadIdx.x == 0) {
+        p.counters[TFE_CTR_TOTAL] = total;
+        p.counters[TFE_CTR_RUNNING] = 0;
+        p.counters[TFE_CTR_DONE] = 0;
+    }
+}
+
+// One lane's probe: the trailing n-gram of query q (n = this lane's order) -> key -> index.
+// Returns the index value {phrase id, residency} or TFE_NONE64 (no such phrase, n-gram reaches
+// before the sequence start, or it holds an id outside [0, vocab)).
+__device__ __forceinline__ unsigned long long tfe_probe_lane(const TfeLookupParams &p, uint32_t q, bool mine,
+                                                             int my_order, bool my_hashed)
+{
+    unsigned long long found = TFE_NONE64;
+#ifndef TFE_DBG_NO_PROBE
+    if (mine && my_order > 0) {
+        const uint32_t b = tfe_div(q, p.div_tq);
+        const int32_t t = p.q_start + (int32_t)(q - b * (uint32_t)p.Tq);
+        int32_t tk[4] = {-1, -1, -1, -1};
+        bool ok = t - (my_order - 1) >= 0;
+        if (ok) {
+            const int32_t *tp = p.tokens + (size_t)b * p.T + t;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (j < my_order) {
+                    tk[j] = __ldg(tp - j);
+                    if ((uint32_t)tk[j] >= (uint32_t)p.vocab) ok = false;
+                }
+        }
+        if (ok) {
+            const uint64_t key = tfe_make_key(my_order, tk, p.tok_bits);
+            uint64_t bucket = tfe_home_bucket_of(key, p.n_buckets);
+            for (int probe = 0; probe < p.max_probe; ++probe) {
+                const ulonglong4 *bp = reinterpret_cast<const ulonglong4 *>(p.index + bucket * TFE_SLOTS_PER_BUCKET);
+                ulonglong4 w[4];                 // 8 slots of {key, value}
+#pragma unroll
+                for (int k = 0; k < 4; ++k) w[k] = ld_bucket32(bp + k);
+                bool any_empty = false;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    if (w[k].x == key) found = w[k].y;
+                    if (w[k].z == key) found = w[k].w;
+                    any_empty |= (w[k].x == 0ull) | (w[k].z == 0ull);
+                }
+                if (found != TFE_NONE64 || any_empty) break;
+                bucket = bucket + 1 == p.n_buckets ? 0 : bucket + 1;           // full of other keys: go on
+            }
+            // hashed orders: a key match is confirmed against the stored token tuple
+            if (my_hashed && found != TFE_NONE64) {
+                const int4 st = __ldg(p.phrase_tokens + (uint32_t)(found >> 32));
+                if (!tuple_matches(st, tk, my_order)) found = TFE_NONE64;
+            }
+        }
+    }
+#endif
+    return found;
+}
+
+// LONGEST policy for the quad of lanes that probed one query: the match of greatest order is
+// retained, its tier decides hit / miss, lane 4*ql records the result.  Returns (on that lane) the
+// GPU-tier slot to add, or -1.
+__device__ __forceinline__ int32_t tfe_select_longest(const TfeLookupParams &p, unsigned long long found, uint32_t q,
+                                                      bool mine, int lane, uint32_t &my_miss)
+{
+    const uint32_t quad_found = (__ballot_sync(0xFFFFFFFFu, found != TFE_NONE64) >> (lane & ~3)) & 0xFu;
+    const int top = quad_found ? 31 - __clz(quad_found) : 0;                   // greatest order that matched
+    const unsigned long long sel = __shfl_sync(0xFFFFFFFFu, found, (lane & ~3) + top);
+    int32_t my_slot = -1;
+    if ((lane & 3) == 0 && mine) {
+        uint32_t phrase = 0xFFFFFFFFu;
+        int32_t st_ = -3;
+        uint32_t flag = 0;
+        if (quad_found) {
+            phrase = (uint32_t)(sel >> 32);
+            st_ = (int32_t)(uint32_t)sel;
+            flag = st_ >= 0 ? 1 : (st_ == -1 ? 2 : 3);
+        }
+        if (flag == 1) my_slot = st_;
+        p.scr_flag[q] = (uint8_t)flag;
+        if (flag >= 2) { p.scr_phrase[q] = phrase; ++my_miss; }
+        if (p.flags) p.flags[q] = (uint8_t)flag;
+        if (p.sel_phrase) p.sel_phrase[q] = phrase;
+        if (p.sel_slot) p.sel_slot[q] = st_;
+    }
+    return my_slot;
+}
+
 // --------------------------------------------------------------- the hot path
 //
-// Work split: block `rank` (ticket order) owns the contiguous query range
-// [rank*q_per_block, ...); its warps take queries from that range one at a time
-// through a shared counter.  One warp per query:
-//   * four 8-lane groups, one per configured order, form their key and scan one
-//     128-byte index bucket per load (one coalesced request per group);
-//   * the warp picks the retained phrase(s), classifies the tier, records the
-//     result, then streams h -> out for the row, adding g*m for GPU hits.
-// Misses are compacted at the end of the block: blocks publish their miss count,
-// a block that has misses adds up the counts of all lower-ranked blocks (they were
-// started earlier and never wait on it) and writes its entries behind them, so the
-// list comes out in ascending (q, order) without a second launch.
-template <int HT, bool ALL, bool COS>
-__global__ void __launch_bounds__(TFE_BLOCK_THREADS, (!ALL && !COS) ? 4 : 2)
+// One launch does everything, and every warp works on its own: it takes batches of `qb`
+// consecutive queries (qb = 1, 2, 4 or 8) in a grid-strided order and runs two phases per batch.
+//
+//   Probe   one THREAD per (query, order): lane 4*ql + oi forms the key of the trailing
+//           orders[oi]-gram of the batch's query ql, fetches the whole 128-byte home bucket with
+//           four 32-byte loads and scans it in registers; a full bucket without the key sends it
+//           on to the next one.  A match of a hashed order is confirmed against the stored tuple.
+//           The four lanes of a query then agree on the retained phrase (LONGEST) or each keeps
+//           its own (ALL); lane 4*ql records the result.
+//   Gather  the whole warp per query: h streams to out in 16-byte vectors, GPU hits fetch their
+//           row alongside and add g*m.
+//
+// Why a thread and not a group of lanes per probe: the probe is a few dozen instructions plus one
+// dependent load.  A warp that spends its instruction slots on 4 probes at a time (8 lanes
+// scanning one bucket, ballots and shuffles to combine) executed ~780 instructions per query and
+// the call was issue-bound at 45 us; per-thread probing needs ~200.
+// Why no block-wide phases: the longest probe chain among 256 threads (a run of full buckets) is
+// several dependent DRAM round trips, and a barrier makes 8 warps wait for it (measured: 12.8 us
+// of probing before any byte streamed).  Autonomous warps wait only for their own 32 lanes while
+// the other warps of the SM keep the memory pipes busy.
+#ifndef TFE_MIN_BLOCKS
+#define TFE_MIN_BLOCKS 3
+#endif
+
+template <int HT, bool ALL, bool COS, bool PACKED>
+__global__ void __launch_bounds__(TFE_BLOCK_THREADS, (ALL || COS) ? 2 : TFE_MIN_BLOCKS)
 tfe_lookup_inject_kernel(const TfeLookupParams p)
 {
     constexpr int VN = TfeVec<HT>::N;
-    constexpr int UNROLL = ALL ? 2 : 4;
-    __shared__ uint32_t s_rank, s_epoch, s_next, s_any_miss;
-    __shared__ uint32_t s_red[TFE_WARPS_PER_BLOCK];
-    __shared__ uint32_t s_scan_base;
+    constexpr int UNROLL = 4;
+    static_assert(!PACKED || (HT == 0 && !ALL && !COS), "packed bf16 path is LONGEST/CONST on bf16 only");
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int grp = lane >> 3, sub = lane & 7;
-    if (threadIdx.x == 0) {
-        s_rank = atomicAdd(&p.counters[TFE_CTR_TICKET], 1u);
-        s_epoch = *(volatile uint32_t *)&p.counters[TFE_CTR_EPOCH];
-        s_next = 0;
-        s_any_miss = 0;
-    }
-    __syncthreads();
-    const uint32_t rank = s_rank, epoch = s_epoch;
-    const uint32_t q_begin = min(p.Q, rank * p.q_per_block);
-    const uint32_t q_end = min(p.Q, q_begin + p.q_per_block);
     const int cols = ALL ? p.n_orders : 1;
     const int steps = p.d / VN;                  // 16-byte steps of h per row
     const size_t hid_row_bytes = (size_t)p.d * (HT == 0 ? 2 : 4);
     const bool in_place = p.out == p.h;
-
-    const int my_order = grp < p.n_orders ? p.orders[grp] : 0;
+    const int ql = lane >> 2, oi = lane & 3;
+    const int my_order = oi < p.n_orders ? p.orders[oi] : 0;
     const bool my_hashed = my_order > 0 && !tfe_order_is_packed(my_order, p.tok_bits);
+    const uint32_t qb = p.qb;
+    const uint32_t n_batches = (p.Q + qb - 1) / qb;
+    const uint32_t n_warps = gridDim.x * TFE_WARPS_PER_BLOCK;
+    uint32_t my_miss = 0;                        // per thread here; summed per warp below
 
-    for (;;) {
-        uint32_t lq = 0;
-        if (lane == 0) lq = atomicAdd(&s_next, 1u);
-        lq = __shfl_sync(0xFFFFFFFFu, lq, 0);
-        if (lq >= q_end - q_begin) break;
-        const uint32_t q = q_begin + lq;
-        const uint32_t b = q / (uint32_t)p.Tq;
-        const int32_t t = p.q_start + (int32_t)(q - b * (uint32_t)p.Tq);
+    for (uint32_t batch = blockIdx.x * TFE_WARPS_PER_BLOCK + warp; batch < n_batches; batch += n_warps) {
+        const uint32_t q0 = batch * qb;
 
-        // ---- trailing n-gram keys: lane `sub` of every group fetches the token at t - sub
-        int32_t tk_mine = -1;
-        if (sub < 4 && t - sub >= 0) {
-            tk_mine = __ldg(p.tokens + (size_t)b * p.T + (t - sub));
-            if ((uint32_t)tk_mine >= (uint32_t)p.vocab) tk_mine = -1;
-        }
-        int32_t tk[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) tk[j] = __shfl_sync(0xFFFFFFFFu, tk_mine, (lane & ~7) + j);
-        bool active = my_order > 0;
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (j < my_order && tk[j] < 0) active = false;
-        const uint64_t key = active ? tfe_make_key(my_order, tk, p.tok_bits) : 0ull;
-
-        // ---- exact-match probe: 8 lanes scan one bucket per iteration
-        uint64_t bucket = active ? tfe_home_bucket_of(key, p.n_buckets) : 0ull;
-        unsigned long long found = TFE_NONE64;
-        for (int probe = 0; probe < p.max_probe; ++probe) {
-            if (!__any_sync(0xFFFFFFFFu, active)) break;
-            ulonglong2 s = make_ulonglong2(0ull, 0ull);
-            if (active) s = ld_slot(p.index + bucket * TFE_SLOTS_PER_BUCKET + sub);
-            const uint32_t hit = __ballot_sync(0xFFFFFFFFu, active && s.x == key);
-            const uint32_t emp = __ballot_sync(0xFFFFFFFFu, active && s.x == 0ull);
-            const uint32_t ghit = (hit >> (grp * 8)) & 0xFFu, gemp = (emp >> (grp * 8)) & 0xFFu;
-            const int src = (lane & ~7) + (ghit ? __ffs(ghit) - 1 : 0);
-            const unsigned long long v = __shfl_sync(0xFFFFFFFFu, s.y, src);
-            if (active) {
-                if (ghit) { found = v; active = false; }
-                else if (gemp) active = false;
-                else bucket = bucket + 1 == p.n_buckets ? 0 : bucket + 1;
-            }
-        }
-        // hashed orders: a key match is confirmed against the stored token tuple
-        if (my_hashed && found != TFE_NONE64) {
-            const int4 st = __ldg(p.phrase_tokens + (uint32_t)(found >> 32));
-            if (!tuple_matches(st, tk, my_order)) found = TFE_NONE64;
-        }
-
-        // ---- selection policy + tier walk (all lanes hold all four group results)
-        unsigned long long res[4];
-#pragma unroll
-        for (int g = 0; g < 4; ++g) res[g] = __shfl_sync(0xFFFFFFFFu, found, g * 8);
-
-        TfeRowSet rs;
-        rs.n = 0;
-        if (!ALL) {
-            unsigned long long sel = TFE_NONE64;
-#pragma unroll
-            for (int g = 0; g < 4; ++g)
-                if (g < p.n_orders && res[g] != TFE_NONE64) sel = res[g];
-            uint32_t phrase = TFE_NONE64 & 0xFFFFFFFFu;
-            int32_t slot = -3;
-            uint8_t flag = 0;
-            if (sel != TFE_NONE64) {
-                phrase = (uint32_t)(sel >> 32);
-                slot = (int32_t)(uint32_t)sel;
-                flag = slot >= 0 ? 1 : (slot == -1 ? 2 : 3);
-                if (slot < -2) slot = -2;
-            }
-            if (lane == 0) {
-                p.scr_flag[q] = flag;
-                p.scr_phrase[q] = phrase;
-                if (p.flags) p.flags[q] = flag;
-                if (p.sel_phrase) p.sel_phrase[q] = phrase;
-                if (p.sel_slot) p.sel_slot[q] = slot;
-                if (flag >= 2) s_any_miss = 1;
-            }
-            if (flag == 1) {
-                rs.n = 1;
-                rs.ptr[0] = p.rows + (size_t)slot * (size_t)(p.d / 8);
-                rs.alpha[0] = 1.f;
-            }
-        } else {
-            int n_sum = 0;
-#pragma unroll
-            for (int g = 0; g < 4; ++g)
-                if (g < p.n_orders && res[g] != TFE_NONE64) n_sum += p.orders[g];
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-                if (g >= p.n_orders) continue;
-                uint32_t phrase = TFE_NONE64 & 0xFFFFFFFFu;
-                int32_t slot = -3;
-                uint8_t flag = 0;
-                if (res[g] != TFE_NONE64) {
-                    phrase = (uint32_t)(res[g] >> 32);
-                    slot = (int32_t)(uint32_t)res[g];
-                    flag = slot >= 0 ? 1 : (slot == -1 ? 2 : 3);
-                    if (slot < -2) slot = -2;
-                }
-                if (lane == g) {
-                    const size_t k = (size_t)q * cols + g;
-                    p.scr_flag[k] = flag;
-                    p.scr_phrase[k] = phrase;
-                    if (p.flags) p.flags[k] = flag;
-                    if (p.sel_phrase) p.sel_phrase[k] = phrase;
-                    if (p.sel_slot) p.sel_slot[k] = slot;
-                    if (flag >= 2) s_any_miss = 1;
-                }
-                if (flag == 1) {
-                    rs.ptr[rs.n] = p.rows + (size_t)slot * (size_t)(p.d / 8);
-                    rs.alpha[rs.n] = (float)p.orders[g] / (float)n_sum;
-                    ++rs.n;
-                }
-            }
-        }
-
-        // ---- gather + gated residual injection: out = h + g * m
-        const char *hrow = reinterpret_cast<const char *>(p.h) + (size_t)q * hid_row_bytes;
-        char *orow = reinterpret_cast<char *>(p.out) + (size_t)q * hid_row_bytes;
-        if (rs.n == 0) {
-            if (!in_place) {
-                for (int s0 = 0; s0 < steps; s0 += 32 * 4) {
-                    uint4 v[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int i = s0 + u * 32 + lane;
-                        if (i < steps) v[u] = ld_stream(reinterpret_cast<const uint4 *>(hrow) + i);
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int i = s0 + u * 32 + lane;
-                        if (i < steps) st_stream(reinterpret_cast<uint4 *>(orow) + i, v[u]);
-                    }
-                }
-            }
-            continue;
-        }
-        float gate = p.lambda;
-        if (COS) {
-            float sa = 0.f, sb = 0.f, sc = 0.f;      // <h,m>, <h,h>, <m,m>
-            for (int i = lane; i < steps; i += 32) {
-                float x[VN], m[VN];
-                load_hidden<HT>(hrow, i, x);
-                load_memory<HT, ALL>(rs, i, m);
-#pragma unroll
-                for (int k = 0; k < VN; ++k) {
-                    sa = fmaf(x[k], m[k], sa); sb = fmaf(x[k], x[k], sb); sc = fmaf(m[k], m[k], sc);
-                }
-            }
-            sa = warp_sum(sa); sb = warp_sum(sb); sc = warp_sum(sc);
-            gate = p.lambda / (1.f + __expf(-sa * rsqrtf(fmaf(sb, sc, 1e-12f))));
-        }
+        // ================================ probe phase ================================
+        const uint32_t q = q0 + ql;
+        const bool mine = ql < (int)qb && q < p.Q;
+        const unsigned long long found = tfe_probe_lane(p, q, mine, my_order, my_hashed);
+        // ---- selection policy + tier walk; the 4 lanes of a query form one aligned quad
+        __syncwarp();
+        int32_t my_slot = -1;                    // GPU-tier slot this lane contributes, or -1
+        float my_alpha = 0.f;
         if constexpr (!ALL) {
-            // one row: keep the raw 16-byte vectors in flight, unpack when they are consumed
-            for (int s0 = 0; s0 < steps; s0 += 32 * UNROLL) {
-                uint4 hv[UNROLL];
-                typename TfeVec<HT>::RowRaw rv[UNROLL];
-#pragma unroll
-                for (int u = 0; u < UNROLL; ++u) {
-                    const int i = s0 + u * 32 + lane;
-                    if (i < steps) {
-                        hv[u] = ld_stream(reinterpret_cast<const uint4 *>(hrow) + i);
-                        rv[u] = ld_row_raw<HT>(rs.ptr[0], i);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < UNROLL; ++u) {
-                    const int i = s0 + u * 32 + lane;
-                    if (i < steps) {
-                        float x[VN], m[VN], y[VN];
-                        unpack_hidden<HT>(hv[u], x);
-                        unpack_row<HT>(rv[u], m);
-#pragma unroll
-                        for (int k = 0; k < VN; ++k) y[k] = fmaf(gate, m[k], x[k]);
-                        store_hidden<HT>(orow, i, y);
-                    }
-                }
-            }
+            my_slot = tfe_select_longest(p, found, q, mine, lane, my_miss);
         } else {
-            for (int s0 = 0; s0 < steps; s0 += 32 * UNROLL) {
-                float x[UNROLL][VN], m[UNROLL][VN];
+            const uint32_t quad_found = (__ballot_sync(0xFFFFFFFFu, found != TFE_NONE64) >> (lane & ~3)) & 0xFu;
+            int n_sum = 0;                       // sum of the matched orders of this query
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u) {
-                    const int i = s0 + u * 32 + lane;
-                    if (i < steps) {
-                        load_hidden<HT>(hrow, i, x[u]);
-                        load_memory<HT, ALL>(rs, i, m[u]);
+            for (int g = 0; g < 4; ++g)
+                if ((quad_found >> g) & 1u) n_sum += p.orders[g];
+            if (oi < p.n_orders && mine) {
+                uint32_t phrase = 0xFFFFFFFFu;
+                int32_t st_ = -3;
+                uint32_t flag = 0;
+                if (found != TFE_NONE64) {
+                    phrase = (uint32_t)(found >> 32);
+                    st_ = (int32_t)(uint32_t)found;
+                    flag = st_ >= 0 ? 1 : (st_ == -1 ? 2 : 3);
+                }
+                if (flag == 1) { my_slot = st_; my_alpha = (float)my_order / (float)n_sum; }
+                const size_t k = (size_t)q * cols + oi;
+                p.scr_flag[k] = (uint8_t)flag;
+                if (flag >= 2) { p.scr_phrase[k] = phrase; ++my_miss; }
+                if (p.flags) p.flags[k] = (uint8_t)flag;
+                if (p.sel_phrase) p.sel_phrase[k] = phrase;
+                if (p.sel_slot) p.sel_slot[k] = st_;
+            }
+        }
+
+        // ================================ gather phase ===============================
+        for (uint32_t lq = 0; lq < qb; ++lq) {
+            const uint32_t gq = q0 + lq;
+            if (gq >= p.Q) break;
+#ifdef TFE_DBG_NO_GATHER
+            break;
+#endif
+            const char *hrow = reinterpret_cast<const char *>(p.h) + (size_t)gq * hid_row_bytes;
+            char *orow = reinterpret_cast<char *>(p.out) + (size_t)gq * hid_row_bytes;
+            // rows to add: held by the lanes of quad lq
+            const uint4 *rowp[ALL ? 4 : 1];
+            float alpha[ALL ? 4 : 1];
+            int n_rows = 0;
+#pragma unroll
+            for (int g = 0; g < (ALL ? 4 : 1); ++g) {
+                const int32_t sl = __shfl_sync(0xFFFFFFFFu, my_slot, 4 * lq + g);
+                alpha[g] = ALL ? __shfl_sync(0xFFFFFFFFu, my_alpha, 4 * lq + g) : 1.f;
+                rowp[g] = sl >= 0 ? p.rows + (size_t)sl * (size_t)(p.d / 8) : nullptr;
+                n_rows += sl >= 0;
+            }
+            if (n_rows == 0) {                   // nothing to add: out = h bit for bit
+                if (!in_place) {
+                    for (int s0 = 0; s0 < steps; s0 += 32 * UNROLL) {
+                        uint4 v[UNROLL];
+#pragma unroll
+                        for (int u = 0; u < UNROLL; ++u) {
+                            const int k = s0 + u * 32 + lane;
+                            if (k < steps) v[u] = ld_stream(reinterpret_cast<const uint4 *>(hrow) + k);
+                        }
+#pragma unroll
+                        for (int u = 0; u < UNROLL; ++u) {
+                            const int k = s0 + u * 32 + lane;
+                            if (k < steps) st_stream(reinterpret_cast<uint4 *>(orow) + k, v[u]);
+                        }
                     }
                 }
+                continue;
+            }
+            float gate = p.lambda;
+            if constexpr (COS) {
+                float sa = 0.f, sb = 0.f, sc = 0.f;      // <h,m>, <h,h>, <m,m>
+                for (int k = lane; k < steps; k += 32) {
+                    float x[VN], m[VN];
+                    load_hidden<HT>(hrow, k, x);
+                    load_memory<HT, ALL>(rowp, alpha, k, m);
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u) {
-                    const int i = s0 + u * 32 + lane;
-                    if (i < steps) {
-                        float y[VN];
-#pragma unroll
-                        for (int k = 0; k < VN; ++k) y[k] = fmaf(gate, m[u][k], x[u][k]);
-                        store_hidden<HT>(orow, i, y);
+                    for (int e = 0; e < VN; ++e) {
+                        sa = fmaf(x[e], m[e], sa); sb = fmaf(x[e], x[e], sb); sc = fmaf(m[e], m[e], sc);
                     }
+                }
+                sa = warp_sum(sa); sb = warp_sum(sb); sc = warp_sum(sc);
+                gate = p.lambda / (1.f + __expf(-sa * rsqrtf(fmaf(sb, sc, 1e-12f))));
+            }
+            if constexpr (!ALL) {
+                // one row: keep the raw 16-byte vectors in flight, convert when they are consumed
+                for (int s0 = 0; s0 < steps; s0 += 32 * UNROLL) {
+                    uint4 hv[UNROLL];
+                    typename TfeVec<HT>::RowRaw rv[UNROLL];
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u) {
+                        const int k = s0 + u * 32 + lane;
+                        if (k < steps) {
+                            hv[u] = ld_stream(reinterpret_cast<const uint4 *>(hrow) + k);
+                            rv[u] = ld_row_raw<HT>(rowp[0], k);
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u) {
+                        const int k = s0 + u * 32 + lane;
+                        if (k >= steps) continue;
+                        if constexpr (PACKED) {
+                            // lambda is a bf16 number: one fused multiply-add per bf16 pair, rounded
+                            // once from the exact h + lambda*m
+                            const uint32_t lam2 = p.lambda_bf16x2;
+                            uint4 o;
+                            o.x = fma_bf16x2(lam2, rv[u].x, hv[u].x); o.y = fma_bf16x2(lam2, rv[u].y, hv[u].y);
+                            o.z = fma_bf16x2(lam2, rv[u].z, hv[u].z); o.w = fma_bf16x2(lam2, rv[u].w, hv[u].w);
+                            st_stream(reinterpret_cast<uint4 *>(orow) + k, o);
+                        } else {
+                            float x[VN], m[VN], y[VN];
+                            unpack_hidden<HT>(hv[u], x);
+                            unpack_row<HT>(rv[u], m);
+#pragma unroll
+                            for (int e = 0; e < VN; ++e) y[e] = fmaf(gate, m[e], x[e]);
+                            store_hidden<HT>(orow, k, y);
+                        }
+                    }
+                }
+            } else {
+                for (int k = lane; k < steps; k += 32) {
+                    float x[VN], m[VN], y[VN];
+                    load_hidden<HT>(hrow, k, x);
+                    load_memory<HT, ALL>(rowp, alpha, k, m);
+#pragma unroll
+                    for (int e = 0; e < VN; ++e) y[e] = fmaf(gate, m[e], x[e]);
+                    store_hidden<HT>(orow, k, y);
                 }
             }
         }
     }
 
-    // ---- order-stable miss compaction for this block's query range
-    __syncthreads();
-    const uint32_t n_ent = (q_end - q_begin) * (uint32_t)cols;
-    const size_t ent0 = (size_t)q_begin * cols;
-    uint32_t cnt = 0;
-    if (s_any_miss) {
-        for (uint32_t i = threadIdx.x; i < n_ent; i += TFE_BLOCK_THREADS) cnt += p.scr_flag[ent0 + i] >= 2;
-        cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
-        if (lane == 0) s_red[warp] = cnt;
-        __syncthreads();
-        cnt = 0;
-#pragma unroll
-        for (int w = 0; w < TFE_WARPS_PER_BLOCK; ++w) cnt += s_red[w];
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) {
-        if (cnt) atomicAdd(&p.counters[TFE_CTR_RUNNING], cnt);
-        __threadfence();
-        atomicExch(&p.block_state[rank], ((unsigned long long)epoch << 32) | cnt);
-    }
-    if (cnt != 0) {     // block-uniform
-        // misses of all lower-ranked blocks (bounded wait; they publish when they finish)
-        uint32_t before = 0;
-        bool expired = false;
-        for (uint32_t j = threadIdx.x; j < rank; j += TFE_BLOCK_THREADS) {
-            unsigned long long v = 0;
-            uint32_t polls = 0;
-            for (;;) {
-                v = *(volatile unsigned long long *)&p.block_state[j];
-                if ((uint32_t)(v >> 32) == epoch) break;
-                if (++polls > TFE_WAIT_LIMIT) { expired = true; break; }
-                __nanosleep(200);
-            }
-            if (!expired) before += (uint32_t)v;
-        }
-        const int any_expired = __syncthreads_or(expired);
-        before = __reduce_add_sync(0xFFFFFFFFu, before);
-        if (lane == 0) s_red[warp] = before;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t tot = 0;
-            for (int w = 0; w < TFE_WARPS_PER_BLOCK; ++w) tot += s_red[w];
-            s_scan_base = tot;
-            if (any_expired) atomicOr(&p.counters[TFE_CTR_STATUS], TFE_DEV_WAIT_EXPIRED);
-        }
-        __syncthreads();
-        if (!any_expired) {
-            for (uint32_t i0 = 0; i0 < n_ent; i0 += TFE_BLOCK_THREADS) {
-                const uint32_t i = i0 + threadIdx.x;
-                uint8_t flag = 0;
-                if (i < n_ent) flag = p.scr_flag[ent0 + i];
-                const bool is_miss = flag >= 2;
-                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, is_miss);
-                if (lane == 0) s_red[warp] = __popc(bal);
-                __syncthreads();
-                uint32_t off = s_scan_base;
-                for (int w = 0; w < warp; ++w) off += s_red[w];
-                off += __popc(bal & ((1u << lane) - 1u));
-                if (is_miss) {
-                    p.miss_q[off] = q_begin + i / (uint32_t)cols;
-                    p.miss_phrase[off] = p.scr_phrase[ent0 + i];
-                    p.miss_tier[off] = flag;
-                }
-                __syncthreads();
-                if (threadIdx.x == 0) {
-                    uint32_t tot = 0;
-                    for (int w = 0; w < TFE_WARPS_PER_BLOCK; ++w) tot += s_red[w];
-                    s_scan_base += tot;
-                }
-                __syncthreads();
-            }
-        }
-    }
+    my_miss = __reduce_add_sync(0xFFFFFFFFu, my_miss);
+    tfe_finish_block(p, my_miss, cols);
+}
 
-    // ---- the block that finishes last closes the call: it publishes the miss total and re-arms
-    // the ticket / done counters and the epoch for the next launch (all state lives on the device,
-    // so a launch can be replayed with unchanged parameters)
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        if (atomicAdd(&p.counters[TFE_CTR_DONE], 1u) == gridDim.x - 1) {
-            __threadfence();
-            p.counters[TFE_CTR_TOTAL] = atomicExch(&p.counters[TFE_CTR_RUNNING], 0u);
-            p.counters[TFE_CTR_TICKET] = 0;
-            p.counters[TFE_CTR_DONE] = 0;
-            uint32_t next = epoch + 1;
-            if (next == 0) {      // the tag wrapped: forget every stale tag before reusing values
-                for (uint32_t j = 0; j < p.block_state_len; ++j) p.block_state[j] = 0ull;
-                next = 1;
-            }
-            p.counters[TFE_CTR_EPOCH] = next;
+// ----------------------------------- the hot path, bulk-copy staged version
+//
+// Same computation as tfe_lookup_inject_kernel for the LONGEST / CONST policy, out-of-place,
+// for calls large enough to be bandwidth-bound.  The difference is where the hidden-state rows
+// wait: a warp asks the bulk-copy engine (cp.async.bulk, completion on an mbarrier) for the h
+// rows of its batch BEFORE it starts probing, into its own 8 KiB of shared memory.  The probe
+// chain (token ids -> bucket -> next bucket -> stored tuple: several dependent DRAM round trips)
+// then runs while HBM is already streaming, and a row that needs no update leaves again with a
+// single bulk store -- no register, no load/store instruction touches it.  Rows to add are fetched
+// with ordinary vector loads once the probe has named them.
+//
+// Per warp: TFE_TMA_STAGE_BYTES of staging, split into `stages` slots of one h row each
+// (stages = min(4, staging / row bytes) >= 1); slot s serves queries s, s + stages, ... of the
+// batch in turn.  Every wait is bounded: if a copy never completes the warp records
+// TFE_DEV_COPY_TIMEOUT and stops consuming, and the host reports TFE_ERR_INTERNAL.
+#ifndef TFE_TMA_WARPS
+#define TFE_TMA_WARPS 7
+#endif
+#ifndef TFE_TMA_MIN_BLOCKS
+#define TFE_TMA_MIN_BLOCKS 4
+#endif
+#define TFE_TMA_THREADS (TFE_TMA_WARPS * 32)
+#define TFE_TMA_STAGE_BYTES 8192
+#define TFE_TMA_MAX_STAGES 4
+#define TFE_TMA_SMEM (TFE_TMA_WARPS * (TFE_TMA_STAGE_BYTES + TFE_TMA_MAX_STAGES * 8))
+#define TFE_TMA_WAIT_LIMIT (1u << 20)
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void *gmem_src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_dst), "l"(gmem_src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_store(void *gmem_dst, uint32_t smem_src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 :: "l"(gmem_dst), "r"(smem_src), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+template <int HT, bool PACKED>
+__global__ void __launch_bounds__(TFE_TMA_THREADS, TFE_TMA_MIN_BLOCKS)
+tfe_lookup_inject_tma_kernel(const TfeLookupParams p, const uint32_t stages)
+{
+    constexpr int VN = TfeVec<HT>::N;
+    static_assert(!PACKED || HT == 0, "packed bf16 path needs bf16 hidden states");
+    extern __shared__ __align__(128) unsigned char tfe_tma_smem[];
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int ql = lane >> 2, oi = lane & 3;
+    const int my_order = oi < p.n_orders ? p.orders[oi] : 0;
+    const bool my_hashed = my_order > 0 && !tfe_order_is_packed(my_order, p.tok_bits);
+    const int steps = p.d / VN;
+    const uint32_t row_bytes = (uint32_t)p.d * (HT == 0 ? 2 : 4);
+    const uint32_t qb = p.qb;
+    const uint32_t n_batches = (p.Q + qb - 1) / qb;
+    const uint32_t n_warps = gridDim.x * TFE_TMA_WARPS;
+
+    unsigned char *const stage_mem = tfe_tma_smem + (size_t)warp * TFE_TMA_STAGE_BYTES;
+    const uint32_t stage0 = smem_addr(stage_mem);
+    const uint32_t bar0 = smem_addr(tfe_tma_smem + (size_t)TFE_TMA_WARPS * TFE_TMA_STAGE_BYTES +
+                                    (size_t)warp * TFE_TMA_MAX_STAGES * 8);
+    if (lane < TFE_TMA_MAX_STAGES) mbar_init(bar0 + lane * 8, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+
+    uint32_t phase = 0;                          // bit s: parity the next wait on slot s expects
+    uint32_t my_miss = 0;
+    bool failed = false;
+#ifdef TFE_DBG_TIMELINE
+    long long *dbg = p.dbg + (size_t)(blockIdx.x * TFE_TMA_WARPS + warp) * 16;
+    if (lane == 0) { dbg[0] = clock64(); unsigned sm; asm("mov.u32 %0, %%smid;" : "=r"(sm)); dbg[15] = sm;
+        unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); dbg[14] = (long long)gt; }
+#endif
+
+    for (uint32_t batch = blockIdx.x * TFE_TMA_WARPS + warp; batch < n_batches && !failed; batch += n_warps) {
+        const uint32_t q0 = batch * qb;
+        const uint32_t nq = min(qb, p.Q - q0);
+
+        // ---- ask for the first h rows of the batch: lane s fills slot s
+        if (lane < (int)min(stages, nq)) {
+            mbar_expect_tx(bar0 + lane * 8, row_bytes);
+            bulk_load(stage0 + lane * row_bytes, reinterpret_cast<const char *>(p.h) + (size_t)(q0 + lane) * row_bytes,
+                      row_bytes, bar0 + lane * 8);
         }
+
+        // ---- probe + select while the rows are on their way
+        const uint32_t q = q0 + ql;
+        const bool mine = ql < (int)qb && q < p.Q;
+        const unsigned long long found = tfe_probe_lane(p, q, mine, my_order, my_hashed);
+        __syncwarp();
+        const int32_t my_slot = tfe_select_longest(p, found, q, mine, lane, my_miss);
+#ifdef TFE_DBG_TIMELINE
+        if (lane == 0 && batch < n_warps) dbg[1] = clock64();
+#endif
+
+        // ---- consume the batch in order
+        for (uint32_t lq = 0; lq < nq; ++lq) {
+            const uint32_t s = lq % stages;
+            const uint32_t gq = q0 + lq;
+            const int32_t sl = __shfl_sync(0xFFFFFFFFu, my_slot, 4 * lq);
+            typename TfeVec<HT>::RowRaw rv[4];
+            const uint4 *rowp = sl >= 0 ? p.rows + (size_t)sl * (size_t)(p.d / 8) : nullptr;
+            if (rowp != nullptr) {               // first vectors of the row: in flight during the wait
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int k = u * 32 + lane;
+                    if (k < steps) rv[u] = ld_row_raw<HT>(rowp, k);
+                }
+            }
+            {   // the h row of this query has landed in slot s?
+                uint32_t polls = 0;
+                while (!mbar_try_wait(bar0 + s * 8, (phase >> s) & 1u)) {
+                    if (++polls > TFE_TMA_WAIT_LIMIT) { failed = true; break; }
+                }
+                failed = __any_sync(0xFFFFFFFFu, failed);
+                if (failed) break;
+                phase ^= 1u << s;
+            }
+            unsigned char *const hs = stage_mem + (size_t)s * row_bytes;
+            char *orow = reinterpret_cast<char *>(p.out) + (size_t)gq * row_bytes;
+            if (rowp == nullptr) {
+                // nothing to add: the row leaves as it came, bit for bit
+                if (lane == 0) {
+                    bulk_store(orow, stage0 + s * row_bytes, row_bytes);
+                    if (lq + stages < nq) bulk_store_wait_read();       // slot is about to be refilled
+                }
+            } else {
+                for (int s0 = 0; s0 < steps; s0 += 32 * 4) {
+                    if (s0 > 0) {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int k = s0 + u * 32 + lane;
+                            if (k < steps) rv[u] = ld_row_raw<HT>(rowp, k);
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int k = s0 + u * 32 + lane;
+                        if (k >= steps) continue;
+                        const uint4 hv = reinterpret_cast<const uint4 *>(hs)[k];
+                        if constexpr (PACKED) {
+                            const uint32_t lam2 = p.lambda_bf16x2;
+                            uint4 o;
+                            o.x = fma_bf16x2(lam2, rv[u].x, hv.x); o.y = fma_bf16x2(lam2, rv[u].y, hv.y);
+                            o.z = fma_bf16x2(lam2, rv[u].z, hv.z); o.w = fma_bf16x2(lam2, rv[u].w, hv.w);
+                            st_stream(reinterpret_cast<uint4 *>(orow) + k, o);
+                        } else {
+                            float x[VN], m[VN], y[VN];
+                            unpack_hidden<HT>(hv, x);
+                            unpack_row<HT>(rv[u], m);
+#pragma unroll
+                            for (int e = 0; e < VN; ++e) y[e] = fmaf(p.lambda, m[e], x[e]);
+                            store_hidden<HT>(orow, k, y);
+                        }
+                    }
+                }
+            }
+            __syncwarp();                        // every lane is done with slot s
+#ifdef TFE_DBG_TIMELINE
+            if (lane == 0 && batch < n_warps && lq < 8) dbg[2 + lq] = clock64();
+#endif
+            // ---- refill slot s with the h row of query lq + stages
+            if (lq + stages < nq && lane == 0) {
+                mbar_expect_tx(bar0 + s * 8, row_bytes);
+                bulk_load(stage0 + s * row_bytes,
+                          reinterpret_cast<const char *>(p.h) + (size_t)(gq + stages) * row_bytes, row_bytes,
+                          bar0 + s * 8);
+            }
+        }
+        if (lane == 0) bulk_store_wait_read();   // the next batch reuses the slots
+        __syncwarp();
     }
+    if (lane == 0) bulk_store_wait_all();
+#ifdef TFE_DBG_TIMELINE
+    if (lane == 0) dbg[10] = clock64();
+#endif
+    if (failed && lane == 0) atomicOr(&p.counters[TFE_CTR_STATUS], TFE_DEV_COPY_TIMEOUT);
+
+    my_miss = __reduce_add_sync(0xFFFFFFFFu, my_miss);
+    tfe_finish_block(p, my_miss, 1);
 }
 
 // ------------------------------------------------------------- cache install

@@ -94,19 +94,31 @@ class Pair:
             n_diff = int((out != rounded).sum())
         if expect_bit_exact is None:
             # One fused multiply-add per element.  fp32 hidden: it is correctly rounded, like the
-            # oracle's double -> float.  bf16 hidden: lambda a power of two (or 0) makes lambda*m exact
-            # and h + lambda*m is then rounded once on both sides.
-            mant = np.frexp(lam)[0] if lam != 0 else 0.5
-            expect_bit_exact = gate == 0 and policy == 0 and (self.hidden_dtype == 1 or abs(mant) == 0.5)
+            # oracle's double -> float.  bf16 hidden with lambda exactly a bf16 number: the kernel uses
+            # the packed bf16 fused multiply-add, which rounds the exact h + lambda*m once, as the
+            # oracle does.
+            lam_is_bf16 = (np.float32(lam).view(np.uint32) & np.uint32(0xFFFF)) == 0
+            expect_bit_exact = gate == 0 and policy == 0 and (self.hidden_dtype == 1 or bool(lam_is_bf16))
         if expect_bit_exact:
             assert n_diff == 0, n_diff
         elif self.hidden_dtype == 0:
-            # fp32 on the GPU against fp64 in the oracle: a result may land on the other side of a
-            # rounding boundary, rarely, and then by one unit in the last place only
-            assert n_diff <= max(2, out.size // 2000), n_diff
-            if self.hidden_dtype == 0 and n_diff:
-                d_bits = np.abs(out.astype(np.int32) - rounded.astype(np.int32))
-                assert d_bits.max() <= 1 or (np.abs(val - exact).max() <= TOL_BF16)
+            if gate == 0 and policy == 0:
+                # any lambda: the kernel rounds h + lambda*m to fp32 first (one fused multiply-add) and
+                # then to bf16.  Taking the oracle's exact value through the same two roundings
+                # (numpy double -> float32, torch float32 -> bfloat16) must give the same bits.
+                two_step = torch.from_numpy(exact.astype(np.float32)).to(torch.bfloat16)
+                two_step = two_step.view(torch.int16).numpy().view(np.uint16)
+                np.testing.assert_array_equal(out[touched], two_step[touched])
+                # against the oracle's single rounding of the exact value such a result may sit on the
+                # other side of a rounding boundary -- by one bf16 step, never more
+                a = synth.bf16_bits_to_f32(out).astype(np.float64)
+                b = synth.bf16_bits_to_f32(rounded).astype(np.float64)
+                mag = np.maximum(np.maximum(np.abs(a), np.abs(b)), 2.0 ** -126)
+                ulp = np.ldexp(1.0, np.floor(np.log2(mag)).astype(np.int64) - 7)
+                assert (np.abs(a - b) <= ulp).all(), float((np.abs(a - b) / ulp).max())
+            # aggregation / cosine gate run in fp32 on the GPU and fp64 in the oracle: the absolute
+            # tolerance above is the contract; most elements still round to the same bf16
+            assert n_diff <= max(2, out.size // 20), n_diff
         return got, ref, dict(max_abs_err=float(err), n_bits_differ=n_diff, n_hit=int(touched.sum()),
                               n_miss=int(cnt))
 

@@ -178,9 +178,56 @@ def test_empty_table(H):
 @pytest.mark.parametrize("load", [0.5, 0.7, 0.95])
 def test_results_do_not_depend_on_load_factor(H, load):
     w = synth.config(1, load_factor=load, residency="hot_host_ssd", gpu_slots=9000)
-    tb, pr = H.pair_from_workload(w)
+    tb, pr = H.pair_from_workload(w, max_probe_buckets=4096)      # crowded tables need long probe chains
     tok = synth.make_queries(w, tb)
     pr.run_and_compare(tok, synth.make_hidden_np(w))
+    pr.close()
+
+
+def test_crowded_index_is_refused_under_the_default_probe_bound(H):
+    from paper_2607_07388_b200 import binding as tfe
+    w = synth.config(1, load_factor=1.0)
+    with pytest.raises(tfe.TfeError) as ei:
+        H.pair_from_workload(w, max_probe_buckets=2)
+    assert ei.value.status == tfe.TFE_ERR_PROBE_LIMIT
+
+
+# ------------------------------------------------ large calls, every batch size
+
+
+@pytest.mark.parametrize("d,hidden,lam,orders", [
+    (1024, 0, 1.0, (2, 3, 4)),      # packed bf16 fused multiply-add
+    (1024, 0, 0.3, (2, 3)),         # fp32 arithmetic
+    (1000, 0, 1.0, (2, 3, 4)),      # ragged vector tail
+    (2048, 0, 0.5, (2, 3)),         # two chunks per row
+    (2560, 1, 0.3, (2, 3, 4)),      # fp32 hidden states, five chunks per row
+    (64, 0, 2.0, (2, 3)),           # short rows
+])
+def test_large_calls_both_kernels_all_batch_sizes(H, d, hidden, lam, orders):
+    from paper_2607_07388_b200 import binding as tfe
+    w = synth.config(3, n_phrases=30_000, gpu_slots=24_000, residency="hot_host_ssd", B=3, T=2731, d=d,
+                     orders=orders, p=0.4, rows="procedural")
+    tb = synth.make_table(w)
+    pr = H.Pair(tb.phrase_tokens, tb.phrase_len, tb.init_slot, synth.make_rows_np(w, tb), vocab=w.vocab,
+                orders=w.orders, hidden_dtype=hidden)
+    tok = synth.make_queries(w, tb)
+    h = synth.make_hidden_np(w)
+    if hidden:
+        h = synth.bf16_bits_to_f32(h) * np.float32(1.0009765625)
+    seen = set()
+    for kernel in (tfe.KERNEL_REGISTER, tfe.KERNEL_STAGED):
+        for qb in (0, 1, 3, 5, 8):      # 0: the library's own choice
+            tfe.tfe_set_tuning(pr.eng.ctx, qb, kernel)
+            _, ref, info = pr.run_and_compare(tok, h, lam=lam)
+            g = tfe.tfe_launch_geometry(pr.eng.ctx)
+            seen.add((g[3], g[2]))
+            assert info["n_hit"] > 500 and info["n_miss"] > 50
+            pr.run_and_compare(tok, h, lam=lam, in_place=True)
+            pr.run_and_compare(tok, h[: w.B * (w.T - 2000)], lam=lam, q_start=2000, want_sel=False)
+            pr.run_and_compare(tok, h, lam=lam, policy=1, gate=1)
+    fits = d * (4 if hidden else 2) <= 8192        # rows above 8 KiB always take the register-staged kernel
+    want = {(0, 1), (0, 3), (0, 5), (0, 8)} | ({(1, 1), (1, 3), (1, 5), (1, 8)} if fits else set())
+    assert want <= seen
     pr.close()
 
 
@@ -207,7 +254,7 @@ def test_miss_list_overflow_and_device_view(H):
 
     class Raw:          # view context-owned device memory as a tensor
         def __init__(self, ptr, n, typestr):
-            self.__cuda_array_interface__ = {"shape": (n,), "typestr": typestr, "data": (ptr, True), "version": 2}
+            self.__cuda_array_interface__ = {"shape": (n,), "typestr": typestr, "data": (ptr, False), "version": 2}
 
     assert int(torch.as_tensor(Raw(dc, 1, "<i4"), device=H.DEV).cpu()[0]) == n
     np.testing.assert_array_equal(torch.as_tensor(Raw(dq, n, "<i4"), device=H.DEV).cpu().numpy().view(np.uint32),
