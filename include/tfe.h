@@ -41,7 +41,7 @@ typedef enum {
     TFE_ERR_UNKNOWN_PHRASE = 6,
     TFE_ERR_ALREADY_RESIDENT = 7,
     TFE_ERR_MISS_OVERFLOW = 8,      /* caller's miss buffers are smaller than the miss count    */
-    TFE_ERR_PROBE_LIMIT = 9,        /* index build could not place a key within max_probe_buckets */
+    TFE_ERR_PROBE_LIMIT = 9,        /* index build could not place a key within max_kicks moves   */
     TFE_ERR_CUDA = 10,              /* a CUDA runtime call failed; see tfe_last_cuda_error()    */
     TFE_ERR_INTERNAL = 11           /* a bounded device-side wait ran out (reported, never hangs) */
 } tfe_status;
@@ -54,9 +54,9 @@ typedef struct {
     int32_t orders[4];          /* n-gram orders, strictly ascending, each in [1,4]                   */
     int64_t n_phrases;          /* N                                                                  */
     int64_t gpu_slots;          /* C, rows of the GPU tier                                            */
-    float   load_factor;        /* index slots = ceil(N / load_factor), rounded up to 8-slot buckets  */
+    float   load_factor;        /* index slots = ceil(N / load_factor), rounded up to 4-slot buckets  */
     int32_t hidden_dtype;       /* 0 = bf16 hidden states, 1 = fp32 hidden states (rows always bf16)  */
-    int32_t max_probe_buckets;  /* bound on linear probing, 0 = library default (64)                  */
+    int32_t max_kicks;          /* cuckoo moves allowed per insertion at build, 0 = default (2000)    */
 } tfe_config;
 
 enum { TFE_POLICY_LONGEST = 0, TFE_POLICY_ALL = 1 };

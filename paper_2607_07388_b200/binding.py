@@ -38,7 +38,7 @@ class TfeConfig(C.Structure):
     _fields_ = [("d", C.c_int32), ("vocab", C.c_int32), ("n_orders", C.c_int32),
                 ("orders", C.c_int32 * 4), ("n_phrases", C.c_int64), ("gpu_slots", C.c_int64),
                 ("load_factor", C.c_float), ("hidden_dtype", C.c_int32),
-                ("max_probe_buckets", C.c_int32)]
+                ("max_kicks", C.c_int32)]
 
 
 class TfeInjectParams(C.Structure):
@@ -118,13 +118,13 @@ def _check(status: int, where: str):
 
 
 def make_config(*, d, vocab, orders, n_phrases, gpu_slots, load_factor=0.7, hidden_dtype=HIDDEN_BF16,
-                max_probe_buckets=0) -> TfeConfig:
+                max_kicks=0) -> TfeConfig:
     cfg = TfeConfig()
     cfg.d, cfg.vocab, cfg.n_orders = int(d), int(vocab), len(orders)
     for i in range(4):
         cfg.orders[i] = int(orders[i]) if i < len(orders) else 0
     cfg.n_phrases, cfg.gpu_slots = int(n_phrases), int(gpu_slots)
-    cfg.load_factor, cfg.hidden_dtype, cfg.max_probe_buckets = float(load_factor), int(hidden_dtype), int(max_probe_buckets)
+    cfg.load_factor, cfg.hidden_dtype, cfg.max_kicks = float(load_factor), int(hidden_dtype), int(max_kicks)
     return cfg
 
 

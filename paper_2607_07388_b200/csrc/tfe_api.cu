@@ -33,7 +33,7 @@ bool cuda_failed(cudaError_t e, const char *what)
     } while (0)
 
 constexpr uint32_t kNoOwner = 0xFFFFFFFFu;
-constexpr int kDefaultMaxProbe = 64;
+constexpr int kDefaultMaxKicks = 2000;
 constexpr int kVarSlots = 16;
 
 }  // namespace
@@ -44,7 +44,6 @@ struct tfe_ctx {
     int sm_count = 0;
     int tok_bits = 0;
     bool any_hashed = false;
-    int max_probe = kDefaultMaxProbe;
     uint64_t n_buckets = 0;
     int row_vecs = 0;                       // 16-byte vectors per GPU-tier row
 
@@ -160,9 +159,56 @@ tfe_status validate_config(const tfe_config *c)
     if (c->gpu_slots > 0x7FFFFFFFll) return TFE_ERR_INVALID_ARG;
     if (!(c->load_factor > 0.f && c->load_factor <= 1.f)) return TFE_ERR_INVALID_ARG;
     if (c->hidden_dtype != 0 && c->hidden_dtype != 1) return TFE_ERR_INVALID_ARG;
-    if (c->max_probe_buckets < 0) return TFE_ERR_INVALID_ARG;
+    if (c->max_kicks < 0) return TFE_ERR_INVALID_ARG;
     if (c->n_phrases > 0xFFFFFFFEll) return TFE_ERR_CAPACITY;
     return TFE_OK;
+}
+
+// Two-choice cuckoo placement of N keys into buckets of 4 slots (host, sequential, deterministic).
+// slots[] receives {key, value}; pos[i] the slot index of phrase i.  A key goes to a free slot of
+// either of its buckets; when both are full a resident key is moved to its other bucket, up to
+// max_kicks moves per insertion.  Returns false if a key could not be placed.
+struct HostSlot { uint64_t key, val; };
+
+bool cuckoo_build(const std::vector<uint64_t> &keys, const int32_t *init_slot, uint64_t n_buckets, int max_kicks,
+                  std::vector<HostSlot> &slots, std::vector<uint32_t> &pos)
+{
+    const size_t N = keys.size();
+    slots.assign((size_t)n_buckets * TFE_SLOTS_PER_BUCKET, HostSlot{0, 0});
+    pos.assign(std::max<size_t>(N, 1), 0);
+    uint64_t rng = 0x853C49E6748FEA9Bull;
+    auto try_place = [&](uint64_t bucket, uint64_t key, uint64_t val) -> bool {
+        HostSlot *b = &slots[(size_t)bucket * TFE_SLOTS_PER_BUCKET];
+        for (int s = 0; s < TFE_SLOTS_PER_BUCKET; ++s)
+            if (b[s].key == 0) {
+                b[s] = HostSlot{key, val};
+                pos[(size_t)(val >> 32)] = (uint32_t)(bucket * TFE_SLOTS_PER_BUCKET + s);
+                return true;
+            }
+        return false;
+    };
+    for (size_t i = 0; i < N; ++i) {
+        uint64_t key = keys[i];
+        uint64_t val = ((uint64_t)i << 32) | (uint32_t)init_slot[i];
+        uint64_t avoid = UINT64_MAX;           // the bucket the key in hand was just taken from
+        bool placed = false;
+        for (int kick = 0; kick <= max_kicks; ++kick) {
+            const uint64_t b1 = tfe_home_bucket_of(key, n_buckets);
+            const uint64_t b2 = tfe_second_bucket_of(key, b1, n_buckets);
+            if (try_place(b1, key, val) || try_place(b2, key, val)) { placed = true; break; }
+            // both full: take a victim from the bucket we did not just come from
+            const uint64_t from = b1 == avoid ? b2 : (b2 == avoid ? b1 : ((rng >> 40) & 1 ? b1 : b2));
+            rng = rng * 6364136223846793005ull + 1442695040888963407ull;
+            const int s = (int)((rng >> 33) % TFE_SLOTS_PER_BUCKET);
+            HostSlot &victim = slots[(size_t)from * TFE_SLOTS_PER_BUCKET + s];
+            std::swap(key, victim.key);
+            std::swap(val, victim.val);
+            pos[(size_t)(victim.val >> 32)] = (uint32_t)(from * TFE_SLOTS_PER_BUCKET + s);
+            avoid = from;
+        }
+        if (!placed) return false;
+    }
+    return true;
 }
 
 // Grow the per-lookup buffers to hold `entries` (= Q * cols) results.  Not on the hot path:
@@ -316,20 +362,14 @@ tfe_status tfe_index_build(const tfe_config *cfg, const int32_t *phrase_tokens,
     c->cfg = *cfg;
     c->tok_bits = bits;
     c->any_hashed = any_hashed;
-    c->max_probe = cfg->max_probe_buckets > 0 ? cfg->max_probe_buckets : kDefaultMaxProbe;
-    if ((uint64_t)c->max_probe > n_buckets) c->max_probe = (int)n_buckets;
     c->n_buckets = n_buckets;
     c->row_vecs = cfg->d / 8;
     c->gpu_rows = static_cast<uint4 *>(gpu_rows);
     c->h_slot.assign(init_slot, init_slot + N);
     c->h_owner.swap(owner);
 
-    uint64_t *d_keys = nullptr;
-    int32_t *d_slots = nullptr;
-    uint32_t h_status = 0;
     tfe_status rc = TFE_OK;
     auto fail = [&](tfe_status s) {
-        free_dev(d_keys); free_dev(d_slots);
         tfe_destroy(c);
         return s;
     };
@@ -337,12 +377,17 @@ tfe_status tfe_index_build(const tfe_config *cfg, const int32_t *phrase_tokens,
     do {                                                           \
         if (cuda_failed((call), #call)) return fail(TFE_ERR_CUDA); \
     } while (0)
+    std::vector<HostSlot> slots;
+    std::vector<uint32_t> pos;
+    if (!cuckoo_build(keys, init_slot, n_buckets, cfg->max_kicks > 0 ? cfg->max_kicks : kDefaultMaxKicks, slots, pos))
+        return fail(TFE_ERR_PROBE_LIMIT);
     CUF(cudaGetDevice(&c->device));
     CUF(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device));
     const size_t index_bytes = (size_t)n_buckets * TFE_SLOTS_PER_BUCKET * sizeof(ulonglong2);
     CUF(cudaMalloc(&c->d_index, index_bytes));
-    CUF(cudaMemsetAsync(c->d_index, 0, index_bytes, stream));
+    CUF(cudaMemcpyAsync(c->d_index, slots.data(), index_bytes, cudaMemcpyHostToDevice, stream));
     CUF(cudaMalloc(&c->d_phrase_pos, std::max<size_t>(4, (size_t)N * 4)));
+    if (N > 0) CUF(cudaMemcpyAsync(c->d_phrase_pos, pos.data(), (size_t)N * 4, cudaMemcpyHostToDevice, stream));
     CUF(cudaMalloc(&c->d_slot_owner, std::max<size_t>(4, (size_t)C * 4)));
     CUF(cudaMalloc(&c->d_counters, TFE_CTR_WORDS * sizeof(uint32_t)));
     CUF(cudaMemsetAsync(c->d_counters, 0, TFE_CTR_WORDS * sizeof(uint32_t), stream));
@@ -366,25 +411,11 @@ tfe_status tfe_index_build(const tfe_config *cfg, const int32_t *phrase_tokens,
                                                           TFE_TMA_SMEM));
         c->occ_tma[v] = std::max(1, occ);
     }
-    if (N > 0) {
-        CUF(cudaMalloc(&d_keys, (size_t)N * 8));
-        CUF(cudaMalloc(&d_slots, (size_t)N * 4));
-        CUF(cudaMemcpyAsync(d_keys, keys.data(), (size_t)N * 8, cudaMemcpyHostToDevice, stream));
-        CUF(cudaMemcpyAsync(d_slots, init_slot, (size_t)N * 4, cudaMemcpyHostToDevice, stream));
-        const unsigned blocks = (unsigned)((N + 255) / 256);
-        tfe_insert_kernel<<<blocks, 256, 0, stream>>>(c->d_index, n_buckets, c->max_probe, d_keys, d_slots,
-                                                      (uint32_t)N, c->d_phrase_pos, c->d_counters + TFE_CTR_STATUS);
-        CUF(cudaGetLastError());
-        CUF(cudaMemcpyAsync(&h_status, c->d_counters + TFE_CTR_STATUS, 4, cudaMemcpyDeviceToHost, stream));
-    }
     CUF(cudaStreamSynchronize(stream));
-    if (h_status & TFE_DEV_PROBE_LIMIT) rc = TFE_ERR_PROBE_LIMIT;
-    else if (h_status & TFE_DEV_DUP_KEY) rc = TFE_ERR_DUPLICATE_PHRASE;
     if (rc != TFE_OK) return fail(rc);
     CUF(cudaMemsetAsync(c->d_counters, 0, TFE_CTR_WORDS * sizeof(uint32_t), stream));
     CUF(cudaStreamSynchronize(stream));
 #undef CUF
-    free_dev(d_keys); free_dev(d_slots);
     *out = c;
     return TFE_OK;
 }
@@ -537,7 +568,7 @@ tfe_status tfe_lookup_inject(tfe_ctx *c, const int32_t *tokens, int32_t B, int32
     TfeLookupParams p{};
     p.tokens = tokens; p.B = B; p.T = T; p.q_start = q_start; p.Tq = (int32_t)Tq; p.Q = (uint32_t)Q;
     p.div_tq = make_fastdiv((uint32_t)Tq); p.qb = (uint32_t)qb;
-    p.index = c->d_index; p.n_buckets = c->n_buckets; p.max_probe = c->max_probe;
+    p.index = c->d_index; p.n_buckets = c->n_buckets;
     p.phrase_tokens = c->d_phrase_tokens; p.rows = c->gpu_rows; p.d = c->cfg.d;
     p.h = h; p.out = out;
     p.n_orders = c->cfg.n_orders;

@@ -1,15 +1,14 @@
 // Device kernels of the Engram lookup-and-inject library (sm_100a).
 //
-//   tfe_insert_kernel          index build: place (key -> phrase id, residency) by atomicCAS
 //   tfe_lookup_inject_kernel   the hot path: keys -> probe -> select -> tier -> gather -> inject
 //                              -> order-stable miss compaction, one launch
 //   tfe_install_kernel         write fetched rows into GPU-tier slots, update residency
 //
-// Index layout: an array of 128-byte buckets, 8 slots of {key64, val64} each.
+// Index layout: an array of 64-byte buckets, 4 slots of {key64, val64} each, filled by
+// two-choice cuckoo hashing on the host: a key lives in one of its two buckets, so a
+// lookup is exactly two independent 64-byte reads and never a dependent chain.
 // val64 = phrase id (high 32 bits) | residency (low 32 bits as int32: >= 0 GPU-tier
-// slot, -1 host DRAM, -2 SSD).  Linear probing over buckets; keys are never
-// removed, so a bucket with an empty slot ends the probe sequence of every key
-// that would have passed through it.
+// slot, -1 host DRAM, -2 SSD).
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -38,7 +37,6 @@ struct TfeLookupParams {
     uint32_t qb;                    // queries per warp batch: 1, 2, 4 or 8
     const ulonglong2 *index;
     uint64_t n_buckets;
-    int32_t max_probe;
     const int4 *phrase_tokens;      // [N] token tuples, only read for hashed orders
     const uint4 *rows;              // GPU tier, [C][d] bf16
     int32_t d;
@@ -68,34 +66,6 @@ struct TfeLookupParams {
 // moves RUNNING to TOTAL and zeroes RUNNING / DONE for the next launch.  Because nothing of this
 // lives in kernel parameters, a launch can be replayed unchanged.
 enum { TFE_CTR_RUNNING = 0, TFE_CTR_TOTAL = 1, TFE_CTR_STATUS = 2, TFE_CTR_DONE = 3, TFE_CTR_WORDS = 4 };
-
-// ------------------------------------------------------------------ index build
-
-__global__ void tfe_insert_kernel(ulonglong2 *index, uint64_t n_buckets, int max_probe,
-                                  const uint64_t *keys, const int32_t *slot_state, uint32_t n,
-                                  uint32_t *phrase_pos, uint32_t *status)
-{
-    uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    const uint64_t key = keys[i];
-    const uint64_t val = ((uint64_t)i << 32) | (uint32_t)slot_state[i];
-    uint64_t bucket = tfe_home_bucket_of(key, n_buckets);
-    for (int probe = 0; probe < max_probe; ++probe) {
-        for (int s = 0; s < TFE_SLOTS_PER_BUCKET; ++s) {
-            ulonglong2 *slot = index + bucket * TFE_SLOTS_PER_BUCKET + s;
-            unsigned long long seen = *(volatile unsigned long long *)&slot->x;
-            if (seen == 0ull) seen = atomicCAS(&slot->x, 0ull, (unsigned long long)key);
-            if (seen == 0ull) {
-                slot->y = val;
-                phrase_pos[i] = (uint32_t)(bucket * TFE_SLOTS_PER_BUCKET + s);
-                return;
-            }
-            if (seen == key) { atomicOr(status, TFE_DEV_DUP_KEY); return; }
-        }
-        bucket = bucket + 1 == n_buckets ? 0 : bucket + 1;
-    }
-    atomicOr(status, TFE_DEV_PROBE_LIMIT);
-}
 
 // -------------------------------------------------------------- small helpers
 
@@ -359,21 +329,17 @@ __device__ __forceinline__ unsigned long long tfe_probe_lane(const TfeLookupPara
         }
         if (ok) {
             const uint64_t key = tfe_make_key(my_order, tk, p.tok_bits);
-            uint64_t bucket = tfe_home_bucket_of(key, p.n_buckets);
-            for (int probe = 0; probe < p.max_probe; ++probe) {
-                const ulonglong4 *bp = reinterpret_cast<const ulonglong4 *>(p.index + bucket * TFE_SLOTS_PER_BUCKET);
-                ulonglong4 w[4];                 // 8 slots of {key, value}
+            const uint64_t b1 = tfe_home_bucket_of(key, p.n_buckets);
+            const uint64_t b2 = tfe_second_bucket_of(key, b1, p.n_buckets);
+            const ulonglong4 *p1 = reinterpret_cast<const ulonglong4 *>(p.index + b1 * TFE_SLOTS_PER_BUCKET);
+            const ulonglong4 *p2 = reinterpret_cast<const ulonglong4 *>(p.index + b2 * TFE_SLOTS_PER_BUCKET);
+            ulonglong4 w[4];                     // 2 buckets x 4 slots of {key, value}, all four loads in flight
+            w[0] = ld_bucket32(p1); w[1] = ld_bucket32(p1 + 1);
+            w[2] = ld_bucket32(p2); w[3] = ld_bucket32(p2 + 1);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) w[k] = ld_bucket32(bp + k);
-                bool any_empty = false;
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    if (w[k].x == key) found = w[k].y;
-                    if (w[k].z == key) found = w[k].w;
-                    any_empty |= (w[k].x == 0ull) | (w[k].z == 0ull);
-                }
-                if (found != TFE_NONE64 || any_empty) break;
-                bucket = bucket + 1 == p.n_buckets ? 0 : bucket + 1;           // full of other keys: go on
+            for (int k = 0; k < 4; ++k) {
+                if (w[k].x == key) found = w[k].y;
+                if (w[k].z == key) found = w[k].w;
             }
             // hashed orders: a key match is confirmed against the stored token tuple
             if (my_hashed && found != TFE_NONE64) {

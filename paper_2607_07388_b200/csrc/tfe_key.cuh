@@ -20,7 +20,7 @@
 #define TFE_HD inline
 #endif
 
-#define TFE_SLOTS_PER_BUCKET 8
+#define TFE_SLOTS_PER_BUCKET 4
 #define TFE_TAG_SHIFT 61
 
 TFE_HD uint64_t tfe_mix64(uint64_t z)
@@ -60,14 +60,26 @@ TFE_HD uint64_t tfe_make_key(int n, const int32_t tk[4], int tok_bits)
     return ((uint64_t)n << TFE_TAG_SHIFT) | acc;
 }
 
-// First bucket probed for a key: a multiply-high range reduction of the mixed
-// key, so any bucket count (not only powers of two) is covered evenly.
+// The two buckets a key may live in (bucketed cuckoo hashing, 4 slots of 16 bytes per bucket).
+// Each is a multiply-high range reduction of a mixed key, so any bucket count (not only powers
+// of two) is covered evenly; the second is forced to differ from the first.
+TFE_HD uint64_t tfe_mulhi64(uint64_t a, uint64_t b)
+{
+#if defined(__CUDA_ARCH__)
+    return __umul64hi(a, b);
+#else
+    return (uint64_t)(((unsigned __int128)a * b) >> 64);
+#endif
+}
+
 TFE_HD uint64_t tfe_home_bucket_of(uint64_t key, uint64_t n_buckets)
 {
-    uint64_t h = tfe_mix64(key);
-#if defined(__CUDA_ARCH__)
-    return __umul64hi(h, n_buckets);
-#else
-    return (uint64_t)(((unsigned __int128)h * n_buckets) >> 64);
-#endif
+    return tfe_mulhi64(tfe_mix64(key), n_buckets);
+}
+
+TFE_HD uint64_t tfe_second_bucket_of(uint64_t key, uint64_t first, uint64_t n_buckets)
+{
+    uint64_t b = tfe_mulhi64(tfe_mix64(key ^ 0xD6E8FEB86659FD93ull), n_buckets);
+    if (b == first) b = b + 1 == n_buckets ? 0 : b + 1;
+    return b;
 }

@@ -25,7 +25,7 @@ class Engram:
     """GPU-resident phrase index + GPU-tier row store for one table."""
 
     def __init__(self, phrase_tokens, phrase_len, init_slot, gpu_rows: torch.Tensor, *, vocab, orders,
-                 load_factor=0.7, hidden_dtype=tfe.HIDDEN_BF16, max_probe_buckets=0, stream=None):
+                 load_factor=0.7, hidden_dtype=tfe.HIDDEN_BF16, max_kicks=0, stream=None):
         assert gpu_rows.is_cuda and gpu_rows.dtype == torch.bfloat16 and gpu_rows.is_contiguous()
         self.rows = gpu_rows
         self.C, self.d = gpu_rows.shape
@@ -34,7 +34,7 @@ class Engram:
         self.torch_hidden = torch.bfloat16 if hidden_dtype == tfe.HIDDEN_BF16 else torch.float32
         self.cfg = tfe.make_config(d=self.d, vocab=vocab, orders=self.orders, n_phrases=len(phrase_len),
                                    gpu_slots=self.C, load_factor=load_factor, hidden_dtype=hidden_dtype,
-                                   max_probe_buckets=max_probe_buckets)
+                                   max_kicks=max_kicks)
         self.ctx = tfe.tfe_index_build(self.cfg, phrase_tokens, phrase_len, init_slot, gpu_rows, stream)
 
     def close(self):
