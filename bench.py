@@ -54,7 +54,6 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--tune-batch", type=int, default=0, help="queries per warp batch (0: library default)")
-    ap.add_argument("--tune-kernel", type=int, default=0, help="0 auto, 1 register-staged, 2 bulk-copy staged")
     return ap.parse_args()
 
 
@@ -246,7 +245,7 @@ def run_ours(a):
     synth.fill_rows_torch(rows, owner)
     eng = Engram(tb.phrase_tokens, tb.phrase_len, tb.init_slot, rows, vocab=w.vocab, orders=w.orders,
                  load_factor=w.load_factor)
-    tfe.tfe_set_tuning(eng.ctx, a.tune_batch, a.tune_kernel)
+    tfe.tfe_set_tuning(eng.ctx, a.tune_batch)
     kw = {"uniform_over_phrases": True} if (a.uniform_plant and w.shape == "decode") else {}
     toks_np = [synth.make_queries(w, tb, variant=v, **kw) for v in range(NBUF)]
     toks = [torch.from_numpy(t).to(dev) for t in toks_np]
@@ -382,7 +381,7 @@ def run_ours(a):
                "call": "tfe_lookup_inject_host + tfe_miss_list (pinned host buffers)"}
 
     clocks = sampler.stop(windows) if sampler else None
-    grid, block, qb, staged = tfe.tfe_launch_geometry(eng.ctx)
+    grid, block, qb = tfe.tfe_launch_geometry(eng.ctx)
     eng.close()
     if world > 1:
         dist.barrier()
@@ -414,7 +413,7 @@ def run_ours(a):
                   f"({NBUF * 2 * w.Q * w.d * 2 / 1e6:.0f} MB) and a {w.gpu_slots * w.d * 2 / 1e9:.1f} GB row table; "
                   f"{'larger' if NBUF * 2 * w.Q * w.d * 2 > 126e6 else 'SMALLER'} than the 126 MB L2",
             "parallelism": "replicas only" if world > 1 else "single GPU",
-            "grid": grid, "block": block, "batch_queries": qb, "kernel": "bulk-copy staged" if staged else "register staged",
+            "grid": grid, "block": block, "batch_queries": qb,
         },
         "gathered_hbm_gbs": gathered / (ms_per_step * 1e-3) / 1e9,
         "frac_of_8tbs": achieved / HBM_NOMINAL_GBS,
@@ -432,7 +431,7 @@ def run_ours(a):
     print(json.dumps(line))
 
 
-TFE_CTR_BYTES = 32      # the launch-state words tfe_miss_list reads back
+TFE_CTR_BYTES = 160     # the launch-state words tfe_miss_list reads back
 
 
 # ------------------------------------------------------------ reference arm

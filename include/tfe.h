@@ -43,7 +43,7 @@ typedef enum {
     TFE_ERR_MISS_OVERFLOW = 8,      /* caller's miss buffers are smaller than the miss count    */
     TFE_ERR_PROBE_LIMIT = 9,        /* index build could not place a key within max_kicks moves   */
     TFE_ERR_CUDA = 10,              /* a CUDA runtime call failed; see tfe_last_cuda_error()    */
-    TFE_ERR_INTERNAL = 11           /* a bounded device-side wait ran out (reported, never hangs) */
+    TFE_ERR_INTERNAL = 11           /* reserved: the device reported an inconsistent state        */
 } tfe_status;
 
 /* Table geometry, fixed at build time. */
@@ -185,26 +185,21 @@ const char *tfe_last_cuda_error(void);
  *   tfe_phrase_key64    the 64-bit index key of a token tuple (0 if n or a token is invalid) and
  *                       whether that order is packed injectively (exact) or hashed + verified.
  *   tfe_home_bucket     the first bucket probed for a key.
- *   tfe_launch_geometry grid size, block size, queries per warp batch of the last lookup, and
- *                       whether it ran the bulk-copy staged kernel (1) or the register-staged one (0).
+ *   tfe_launch_geometry grid size, block size and queries per warp batch of the last lookup.
  */
 tfe_status tfe_index_geometry(const tfe_ctx *ctx, int64_t *n_buckets, int64_t *index_bytes,
                               int64_t *metadata_bytes);
 uint64_t tfe_phrase_key64(int32_t vocab, const int32_t *tokens, int32_t n, int32_t *is_exact);
 uint64_t tfe_home_bucket(uint64_t key, uint64_t n_buckets);
-tfe_status tfe_launch_geometry(const tfe_ctx *ctx, int32_t *grid, int32_t *block, int32_t *batch_queries,
-                               int32_t *staged);
+tfe_status tfe_launch_geometry(const tfe_ctx *ctx, int32_t *grid, int32_t *block, int32_t *batch_queries);
 
 /*
- * Tuning knobs (HOST only; results never depend on them).
- *   batch_queries  a lookup warp takes batches of 1..8 consecutive queries: it probes the whole
- *                  batch at once (one lane per query and order), then streams the batch's rows.
- *                  0 = the library picks per call (small calls 1, the lowest latency).
- *   kernel         the LONGEST / CONST path has two kernels: register-staged (1) and bulk-copy
- *                  staged through shared memory (2; out-of-place calls with rows up to 8 KiB).
- *                  0 = the library picks per call (staged for large calls).
+ * Tuning knob (HOST only; results never depend on it).  A lookup warp takes batches of 1..8
+ * consecutive queries: it probes the whole batch at once (one lane per query and order), then
+ * streams the batch's rows.  0 = the library picks per call (small calls 1, the lowest latency;
+ * large calls 4).
  */
-tfe_status tfe_set_tuning(tfe_ctx *ctx, int32_t batch_queries, int32_t kernel);
+tfe_status tfe_set_tuning(tfe_ctx *ctx, int32_t batch_queries);
 
 #ifdef __cplusplus
 }

@@ -82,8 +82,8 @@ def lib() -> C.CDLL:
         L.tfe_phrase_key64.restype = u64
         L.tfe_home_bucket.argtypes = [u64, u64]
         L.tfe_home_bucket.restype = u64
-        L.tfe_launch_geometry.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
-        L.tfe_set_tuning.argtypes = [vp, i32, i32]
+        L.tfe_launch_geometry.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
+        L.tfe_set_tuning.argtypes = [vp, i32]
         for name in ("tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
                      "tfe_miss_list", "tfe_miss_list_device", "tfe_index_geometry", "tfe_launch_geometry",
                      "tfe_set_tuning"):
@@ -205,17 +205,14 @@ def tfe_index_geometry(ctx: int):
 
 
 def tfe_launch_geometry(ctx: int):
-    """(grid, block, queries per warp batch, bulk-copy staged?) of the most recent lookup."""
-    g, b, t, s = C.c_int32(), C.c_int32(), C.c_int32(), C.c_int32()
-    _check(lib().tfe_launch_geometry(ctx, C.byref(g), C.byref(b), C.byref(t), C.byref(s)), "tfe_launch_geometry")
-    return g.value, b.value, t.value, s.value
+    """(grid, block, queries per warp batch) of the most recent lookup."""
+    g, b, t = C.c_int32(), C.c_int32(), C.c_int32()
+    _check(lib().tfe_launch_geometry(ctx, C.byref(g), C.byref(b), C.byref(t)), "tfe_launch_geometry")
+    return g.value, b.value, t.value
 
 
-KERNEL_AUTO, KERNEL_REGISTER, KERNEL_STAGED = 0, 1, 2
-
-
-def tfe_set_tuning(ctx: int, batch_queries: int = 0, kernel: int = KERNEL_AUTO) -> None:
-    _check(lib().tfe_set_tuning(ctx, int(batch_queries), int(kernel)), "tfe_set_tuning")
+def tfe_set_tuning(ctx: int, batch_queries: int = 0) -> None:
+    _check(lib().tfe_set_tuning(ctx, int(batch_queries)), "tfe_set_tuning")
 
 
 def tfe_phrase_key64(vocab: int, tokens) -> tuple[int, bool]:

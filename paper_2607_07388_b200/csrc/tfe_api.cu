@@ -63,15 +63,14 @@ struct tfe_ctx {
     uint8_t *d_miss_tier = nullptr;
     uint32_t *d_counters = nullptr;         // TFE_CTR_WORDS words of launch state
     int occ[kVarSlots] = {0};
-    int occ_tma[3] = {0};                   // the bulk-copy staged kernels: bf16 fp32-math, bf16 packed, fp32 hidden                      // resident blocks per SM of each kernel variant
+    // resident blocks per SM of each kernel variant
 
     int64_t last_entries = -1;              // Q*cols of the most recent lookup (-1: none yet)
 #ifdef TFE_DBG_TIMELINE
     long long *dbg = nullptr;
 #endif
-    int last_grid = 0, last_block = 0, last_qb = 0, last_staged = 0;
+    int last_grid = 0, last_block = 0, last_qb = 0;
     int qb_override = 0;                    // 0: choose per call
-    int kernel_override = 0;                // 0: choose per call, 1: register-staged, 2: bulk-copy staged
 
     // install staging
     uint32_t *d_inst_ids = nullptr;
@@ -92,9 +91,10 @@ namespace {
 
 typedef void (*lookup_kernel_t)(const TfeLookupParams);
 
-// Kernel variants.  0..7: hidden dtype x policy x gate in fp32 arithmetic;
-// 8: bf16 hidden, LONGEST / CONST with the packed bf16 fused multiply-add (lambda a bf16 number).
-enum { kVarPacked = 8, kVarCount = 9 };
+// Kernel variants.  0..7: hidden dtype x policy x gate, the general kernel in fp32 arithmetic.
+// 8..10: the LONGEST / CONST kernel -- bf16 hidden in fp32 arithmetic, bf16 hidden with the
+// packed bf16 fused multiply-add (lambda exactly a bf16 number), fp32 hidden.
+enum { kVarLongest = 8, kVarLongestPacked = 9, kVarLongestF32 = 10, kVarCount = 11 };
 
 lookup_kernel_t pick_kernel(int variant)
 {
@@ -103,22 +103,15 @@ lookup_kernel_t pick_kernel(int variant)
         tfe_lookup_inject_kernel<0, true, false, false>,  tfe_lookup_inject_kernel<0, true, true, false>,
         tfe_lookup_inject_kernel<1, false, false, false>, tfe_lookup_inject_kernel<1, false, true, false>,
         tfe_lookup_inject_kernel<1, true, false, false>,  tfe_lookup_inject_kernel<1, true, true, false>,
-        tfe_lookup_inject_kernel<0, false, false, true>,
+        tfe_lookup_inject_longest_kernel<0, false>, tfe_lookup_inject_longest_kernel<0, true>,
+        tfe_lookup_inject_longest_kernel<1, false>,
     };
     return table[variant];
 }
 
-// Bulk-copy staged kernels for large out-of-place LONGEST / CONST calls.
-typedef void (*tma_kernel_t)(const TfeLookupParams, uint32_t);
-
-tma_kernel_t pick_tma_kernel(int ht, bool packed)
-{
-    if (ht == 1) return tfe_lookup_inject_tma_kernel<1, false>;
-    return packed ? tfe_lookup_inject_tma_kernel<0, true> : tfe_lookup_inject_tma_kernel<0, false>;
-}
-
 // Queries per warp batch (1..8) for a call of Q queries on `warps` resident warps: the split into
-// r rounds of ceil(Q / (warps*r)) queries that leaves the busiest warp the least work.
+// r rounds of ceil(Q / (warps*r)) queries that leaves the busiest warp the least work (small
+// calls: one query per warp, the lowest latency).
 int pick_batch(int64_t Q, int64_t warps)
 {
     if (Q <= warps) return 1;
@@ -403,14 +396,6 @@ tfe_status tfe_index_build(const tfe_config *cfg, const int32_t *phrase_tokens,
         CUF(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, pick_kernel(v), TFE_BLOCK_THREADS, 0));
         c->occ[v] = std::max(1, occ);
     }
-    for (int v = 0; v < 3; ++v) {
-        int occ = 0;
-        CUF(cudaFuncSetAttribute(pick_tma_kernel(v == 2, v == 1), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 TFE_TMA_SMEM));
-        CUF(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, pick_tma_kernel(v == 2, v == 1), TFE_TMA_THREADS,
-                                                          TFE_TMA_SMEM));
-        c->occ_tma[v] = std::max(1, occ);
-    }
     CUF(cudaStreamSynchronize(stream));
     if (rc != TFE_OK) return fail(rc);
     CUF(cudaMemsetAsync(c->d_counters, 0, TFE_CTR_WORDS * sizeof(uint32_t), stream));
@@ -440,22 +425,19 @@ tfe_status tfe_debug_timeline(tfe_ctx *c, void *device_buffer)
 }
 #endif
 
-tfe_status tfe_set_tuning(tfe_ctx *c, int32_t batch_queries, int32_t kernel)
+tfe_status tfe_set_tuning(tfe_ctx *c, int32_t batch_queries)
 {
-    if (!c || batch_queries < 0 || batch_queries > 8 || kernel < 0 || kernel > 2) return TFE_ERR_INVALID_ARG;
+    if (!c || batch_queries < 0 || batch_queries > 8) return TFE_ERR_INVALID_ARG;
     c->qb_override = batch_queries;
-    c->kernel_override = kernel;
     return TFE_OK;
 }
 
-tfe_status tfe_launch_geometry(const tfe_ctx *c, int32_t *grid, int32_t *block, int32_t *batch_queries,
-                               int32_t *staged)
+tfe_status tfe_launch_geometry(const tfe_ctx *c, int32_t *grid, int32_t *block, int32_t *batch_queries)
 {
     if (!c) return TFE_ERR_INVALID_ARG;
     if (grid) *grid = c->last_grid;
     if (block) *block = c->last_block;
     if (batch_queries) *batch_queries = c->last_qb;
-    if (staged) *staged = c->last_staged;
     return TFE_OK;
 }
 
@@ -549,22 +531,11 @@ tfe_status tfe_lookup_inject(tfe_ctx *c, const int32_t *tokens, int32_t B, int32
     const bool lam_is_bf16 = (lam_bits & 0xFFFFu) == 0 && (lam_bits & 0x7F800000u) != 0x7F800000u;
     const int ht = c->cfg.hidden_dtype;
     const int variant = (all || cos) ? ht * 4 + (all ? 2 : 0) + (cos ? 1 : 0)
-                                     : ((ht == 0 && lam_is_bf16) ? kVarPacked : ht * 4);
-    // Large out-of-place LONGEST / CONST calls go through the bulk-copy staged kernel (h rows are
-    // requested before the probe and wait in shared memory); everything else -- small calls where
-    // latency counts, in-place calls, ALL / COSINE -- through the register-staged one.
-    const uint32_t row_bytes = (uint32_t)c->cfg.d * (ht == 0 ? 2u : 4u);
-    const int tma_idx = ht == 1 ? 2 : (lam_is_bf16 ? 1 : 0);
-    const int64_t tma_warps = (int64_t)c->sm_count * c->occ_tma[tma_idx] * TFE_TMA_WARPS;
-    bool use_tma = !all && !cos && h != out && row_bytes <= TFE_TMA_STAGE_BYTES;
-    if (c->kernel_override == 1) use_tma = false;
-    else if (c->kernel_override != 2) use_tma = use_tma && Q >= 2 * tma_warps;
-    const int64_t resident = use_tma ? (int64_t)c->sm_count * c->occ_tma[tma_idx]
-                                     : (int64_t)c->sm_count * c->occ[variant];
-    const int warps_per_block = use_tma ? TFE_TMA_WARPS : TFE_WARPS_PER_BLOCK;
-    const int64_t qb = c->qb_override ? c->qb_override : pick_batch(Q, resident * warps_per_block);
+                                     : (ht == 1 ? kVarLongestF32 : (lam_is_bf16 ? kVarLongestPacked : kVarLongest));
+    const int64_t resident = (int64_t)c->sm_count * c->occ[variant];
+    const int64_t qb = c->qb_override ? c->qb_override : pick_batch(Q, resident * TFE_WARPS_PER_BLOCK);
     const int64_t n_batches = (Q + qb - 1) / qb;
-    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(resident, (n_batches + warps_per_block - 1) / warps_per_block));
+    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(resident, (n_batches + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK));
     TfeLookupParams p{};
     p.tokens = tokens; p.B = B; p.T = T; p.q_start = q_start; p.Tq = (int32_t)Tq; p.Q = (uint32_t)Q;
     p.div_tq = make_fastdiv((uint32_t)Tq); p.qb = (uint32_t)qb;
@@ -583,17 +554,11 @@ tfe_status tfe_lookup_inject(tfe_ctx *c, const int32_t *tokens, int32_t B, int32
     p.dbg = c->dbg;
 #endif
 
-    if (use_tma) {
-        const uint32_t stages = std::min<uint32_t>(TFE_TMA_MAX_STAGES, TFE_TMA_STAGE_BYTES / row_bytes);
-        pick_tma_kernel(ht, lam_is_bf16)<<<(unsigned)grid, TFE_TMA_THREADS, TFE_TMA_SMEM, stream>>>(p, stages);
-    } else {
-        pick_kernel(variant)<<<(unsigned)grid, TFE_BLOCK_THREADS, 0, stream>>>(p);
-    }
+    pick_kernel(variant)<<<(unsigned)grid, TFE_BLOCK_THREADS, 0, stream>>>(p);
     CU(cudaGetLastError());
     c->last_entries = Q * cols;
     c->last_grid = (int)grid;
-    c->last_block = use_tma ? TFE_TMA_THREADS : TFE_BLOCK_THREADS;
-    c->last_staged = use_tma ? 1 : 0;
+    c->last_block = TFE_BLOCK_THREADS;
     c->last_qb = (int)qb;
     return TFE_OK;
 }
@@ -656,10 +621,6 @@ tfe_status tfe_miss_list(tfe_ctx *c, uint32_t *q_idx, uint32_t *phrase_id, uint8
     uint32_t words[TFE_CTR_WORDS] = {0};
     CU(cudaMemcpyAsync(words, c->d_counters, sizeof words, cudaMemcpyDeviceToHost, stream));
     CU(cudaStreamSynchronize(stream));
-    if (words[TFE_CTR_STATUS] & TFE_DEV_COPY_TIMEOUT) {
-        CU(cudaMemsetAsync(c->d_counters + TFE_CTR_STATUS, 0, 4, stream));
-        return TFE_ERR_INTERNAL;
-    }
     const int64_t n = words[TFE_CTR_TOTAL];
     *count = n;
     const int64_t take = std::min(n, cap);

@@ -16,12 +16,13 @@
 
 #include "tfe_key.cuh"
 
-#define TFE_BLOCK_THREADS 256
+#ifndef TFE_BLOCK_THREADS
+#define TFE_BLOCK_THREADS 256     // 8 warps; 3 blocks per SM within 80 registers per thread measured best
+#endif
 #define TFE_WARPS_PER_BLOCK (TFE_BLOCK_THREADS / 32)
 #define TFE_NONE64 0xFFFFFFFFFFFFFFFFull
 
 // device status bits (counters[TFE_CTR_STATUS])
-#define TFE_DEV_COPY_TIMEOUT 1u
 #define TFE_DEV_PROBE_LIMIT 2u
 #define TFE_DEV_DUP_KEY 4u
 
@@ -305,9 +306,11 @@ __device__ __forceinline__ void tfe_finish_block(const TfeLookupParams &p, uint3
     }
 }
 
-// One lane's probe: the trailing n-gram of query q (n = this lane's order) -> key -> index.
-// Returns the index value {phrase id, residency} or TFE_NONE64 (no such phrase, n-gram reaches
-// before the sequence start, or it holds an id outside [0, vocab)).
+// One lane's probe: the trailing n-gram of query q (n = this lane's order) -> key -> index value
+// {phrase id, residency}, or TFE_NONE64 (no such phrase, n-gram reaches before the sequence
+// start, or it holds an id outside [0, vocab)).  Three dependent steps: the token ids, both
+// candidate buckets (4 x 32 bytes, all in flight together), and -- hashed orders only -- the
+// stored tuple of a key match.
 __device__ __forceinline__ unsigned long long tfe_probe_lane(const TfeLookupParams &p, uint32_t q, bool mine,
                                                              int my_order, bool my_hashed)
 {
@@ -415,7 +418,7 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
     constexpr int UNROLL = 4;
     static_assert(!PACKED || (HT == 0 && !ALL && !COS), "packed bf16 path is LONGEST/CONST on bf16 only");
 
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
     const int cols = ALL ? p.n_orders : 1;
     const int steps = p.d / VN;                  // 16-byte steps of h per row
     const size_t hid_row_bytes = (size_t)p.d * (HT == 0 ? 2 : 4);
@@ -425,10 +428,16 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
     const bool my_hashed = my_order > 0 && !tfe_order_is_packed(my_order, p.tok_bits);
     const uint32_t qb = p.qb;
     const uint32_t n_batches = (p.Q + qb - 1) / qb;
-    const uint32_t n_warps = gridDim.x * TFE_WARPS_PER_BLOCK;
     uint32_t my_miss = 0;                        // per thread here; summed per warp below
+#ifdef TFE_DBG_TIMELINE
+    long long *dbg = p.dbg + (size_t)(blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5)) * 16;
+    if (lane == 0) { dbg[0] = clock64(); unsigned sm; asm("mov.u32 %0, %%smid;" : "=r"(sm)); dbg[15] = sm;
+        unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); dbg[14] = (long long)gt; }
+    int dbg_round = 0;
+#endif
 
-    for (uint32_t batch = blockIdx.x * TFE_WARPS_PER_BLOCK + warp; batch < n_batches; batch += n_warps) {
+    const uint32_t n_warps = gridDim.x * TFE_WARPS_PER_BLOCK;
+    for (uint32_t batch = blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5); batch < n_batches; batch += n_warps) {
         const uint32_t q0 = batch * qb;
 
         // ================================ probe phase ================================
@@ -466,6 +475,9 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
             }
         }
 
+#ifdef TFE_DBG_TIMELINE
+        if (lane == 0 && dbg_round < 2) dbg[1 + 6 * dbg_round] = clock64();
+#endif
         // ================================ gather phase ===============================
         for (uint32_t lq = 0; lq < qb; ++lq) {
             const uint32_t gq = q0 + lq;
@@ -565,208 +577,196 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
                 }
             }
         }
+#ifdef TFE_DBG_TIMELINE
+        if (lane == 0 && dbg_round < 2) dbg[2 + 6 * dbg_round] = clock64();
+        ++dbg_round;
+#endif
     }
 
-    my_miss = __reduce_add_sync(0xFFFFFFFFu, my_miss);
-    tfe_finish_block(p, my_miss, cols);
-}
-
-// ----------------------------------- the hot path, bulk-copy staged version
-//
-// Same computation as tfe_lookup_inject_kernel for the LONGEST / CONST policy, out-of-place,
-// for calls large enough to be bandwidth-bound.  The difference is where the hidden-state rows
-// wait: a warp asks the bulk-copy engine (cp.async.bulk, completion on an mbarrier) for the h
-// rows of its batch BEFORE it starts probing, into its own 8 KiB of shared memory.  The probe
-// chain (token ids -> bucket -> next bucket -> stored tuple: several dependent DRAM round trips)
-// then runs while HBM is already streaming, and a row that needs no update leaves again with a
-// single bulk store -- no register, no load/store instruction touches it.  Rows to add are fetched
-// with ordinary vector loads once the probe has named them.
-//
-// Per warp: TFE_TMA_STAGE_BYTES of staging, split into `stages` slots of one h row each
-// (stages = min(4, staging / row bytes) >= 1); slot s serves queries s, s + stages, ... of the
-// batch in turn.  Every wait is bounded: if a copy never completes the warp records
-// TFE_DEV_COPY_TIMEOUT and stops consuming, and the host reports TFE_ERR_INTERNAL.
-#ifndef TFE_TMA_WARPS
-#define TFE_TMA_WARPS 7
-#endif
-#ifndef TFE_TMA_MIN_BLOCKS
-#define TFE_TMA_MIN_BLOCKS 4
-#endif
-#define TFE_TMA_THREADS (TFE_TMA_WARPS * 32)
-#define TFE_TMA_STAGE_BYTES 8192
-#define TFE_TMA_MAX_STAGES 4
-#define TFE_TMA_SMEM (TFE_TMA_WARPS * (TFE_TMA_STAGE_BYTES + TFE_TMA_MAX_STAGES * 8))
-#define TFE_TMA_WAIT_LIMIT (1u << 20)
-
-__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void *gmem_src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 :: "r"(smem_dst), "l"(gmem_src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void bulk_store(void *gmem_dst, uint32_t smem_src, uint32_t bytes)
-{
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                 :: "l"(gmem_dst), "r"(smem_src), "r"(bytes) : "memory");
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-
-template <int HT, bool PACKED>
-__global__ void __launch_bounds__(TFE_TMA_THREADS, TFE_TMA_MIN_BLOCKS)
-tfe_lookup_inject_tma_kernel(const TfeLookupParams p, const uint32_t stages)
-{
-    constexpr int VN = TfeVec<HT>::N;
-    static_assert(!PACKED || HT == 0, "packed bf16 path needs bf16 hidden states");
-    extern __shared__ __align__(128) unsigned char tfe_tma_smem[];
-
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int ql = lane >> 2, oi = lane & 3;
-    const int my_order = oi < p.n_orders ? p.orders[oi] : 0;
-    const bool my_hashed = my_order > 0 && !tfe_order_is_packed(my_order, p.tok_bits);
-    const int steps = p.d / VN;
-    const uint32_t row_bytes = (uint32_t)p.d * (HT == 0 ? 2 : 4);
-    const uint32_t qb = p.qb;
-    const uint32_t n_batches = (p.Q + qb - 1) / qb;
-    const uint32_t n_warps = gridDim.x * TFE_TMA_WARPS;
-
-    unsigned char *const stage_mem = tfe_tma_smem + (size_t)warp * TFE_TMA_STAGE_BYTES;
-    const uint32_t stage0 = smem_addr(stage_mem);
-    const uint32_t bar0 = smem_addr(tfe_tma_smem + (size_t)TFE_TMA_WARPS * TFE_TMA_STAGE_BYTES +
-                                    (size_t)warp * TFE_TMA_MAX_STAGES * 8);
-    if (lane < TFE_TMA_MAX_STAGES) mbar_init(bar0 + lane * 8, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncwarp();
-
-    uint32_t phase = 0;                          // bit s: parity the next wait on slot s expects
-    uint32_t my_miss = 0;
-    bool failed = false;
-#ifdef TFE_DBG_TIMELINE
-    long long *dbg = p.dbg + (size_t)(blockIdx.x * TFE_TMA_WARPS + warp) * 16;
-    if (lane == 0) { dbg[0] = clock64(); unsigned sm; asm("mov.u32 %0, %%smid;" : "=r"(sm)); dbg[15] = sm;
-        unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); dbg[14] = (long long)gt; }
-#endif
-
-    for (uint32_t batch = blockIdx.x * TFE_TMA_WARPS + warp; batch < n_batches && !failed; batch += n_warps) {
-        const uint32_t q0 = batch * qb;
-        const uint32_t nq = min(qb, p.Q - q0);
-
-        // ---- ask for the first h rows of the batch: lane s fills slot s
-        if (lane < (int)min(stages, nq)) {
-            mbar_expect_tx(bar0 + lane * 8, row_bytes);
-            bulk_load(stage0 + lane * row_bytes, reinterpret_cast<const char *>(p.h) + (size_t)(q0 + lane) * row_bytes,
-                      row_bytes, bar0 + lane * 8);
-        }
-
-        // ---- probe + select while the rows are on their way
-        const uint32_t q = q0 + ql;
-        const bool mine = ql < (int)qb && q < p.Q;
-        const unsigned long long found = tfe_probe_lane(p, q, mine, my_order, my_hashed);
-        __syncwarp();
-        const int32_t my_slot = tfe_select_longest(p, found, q, mine, lane, my_miss);
-#ifdef TFE_DBG_TIMELINE
-        if (lane == 0 && batch < n_warps) dbg[1] = clock64();
-#endif
-
-        // ---- consume the batch in order
-        for (uint32_t lq = 0; lq < nq; ++lq) {
-            const uint32_t s = lq % stages;
-            const uint32_t gq = q0 + lq;
-            const int32_t sl = __shfl_sync(0xFFFFFFFFu, my_slot, 4 * lq);
-            typename TfeVec<HT>::RowRaw rv[4];
-            const uint4 *rowp = sl >= 0 ? p.rows + (size_t)sl * (size_t)(p.d / 8) : nullptr;
-            if (rowp != nullptr) {               // first vectors of the row: in flight during the wait
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int k = u * 32 + lane;
-                    if (k < steps) rv[u] = ld_row_raw<HT>(rowp, k);
-                }
-            }
-            {   // the h row of this query has landed in slot s?
-                uint32_t polls = 0;
-                while (!mbar_try_wait(bar0 + s * 8, (phase >> s) & 1u)) {
-                    if (++polls > TFE_TMA_WAIT_LIMIT) { failed = true; break; }
-                }
-                failed = __any_sync(0xFFFFFFFFu, failed);
-                if (failed) break;
-                phase ^= 1u << s;
-            }
-            unsigned char *const hs = stage_mem + (size_t)s * row_bytes;
-            char *orow = reinterpret_cast<char *>(p.out) + (size_t)gq * row_bytes;
-            if (rowp == nullptr) {
-                // nothing to add: the row leaves as it came, bit for bit
-                if (lane == 0) {
-                    bulk_store(orow, stage0 + s * row_bytes, row_bytes);
-                    if (lq + stages < nq) bulk_store_wait_read();       // slot is about to be refilled
-                }
-            } else {
-                for (int s0 = 0; s0 < steps; s0 += 32 * 4) {
-                    if (s0 > 0) {
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int k = s0 + u * 32 + lane;
-                            if (k < steps) rv[u] = ld_row_raw<HT>(rowp, k);
-                        }
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int k = s0 + u * 32 + lane;
-                        if (k >= steps) continue;
-                        const uint4 hv = reinterpret_cast<const uint4 *>(hs)[k];
-                        if constexpr (PACKED) {
-                            const uint32_t lam2 = p.lambda_bf16x2;
-                            uint4 o;
-                            o.x = fma_bf16x2(lam2, rv[u].x, hv.x); o.y = fma_bf16x2(lam2, rv[u].y, hv.y);
-                            o.z = fma_bf16x2(lam2, rv[u].z, hv.z); o.w = fma_bf16x2(lam2, rv[u].w, hv.w);
-                            st_stream(reinterpret_cast<uint4 *>(orow) + k, o);
-                        } else {
-                            float x[VN], m[VN], y[VN];
-                            unpack_hidden<HT>(hv, x);
-                            unpack_row<HT>(rv[u], m);
-#pragma unroll
-                            for (int e = 0; e < VN; ++e) y[e] = fmaf(p.lambda, m[e], x[e]);
-                            store_hidden<HT>(orow, k, y);
-                        }
-                    }
-                }
-            }
-            __syncwarp();                        // every lane is done with slot s
-#ifdef TFE_DBG_TIMELINE
-            if (lane == 0 && batch < n_warps && lq < 8) dbg[2 + lq] = clock64();
-#endif
-            // ---- refill slot s with the h row of query lq + stages
-            if (lq + stages < nq && lane == 0) {
-                mbar_expect_tx(bar0 + s * 8, row_bytes);
-                bulk_load(stage0 + s * row_bytes,
-                          reinterpret_cast<const char *>(p.h) + (size_t)(gq + stages) * row_bytes, row_bytes,
-                          bar0 + s * 8);
-            }
-        }
-        if (lane == 0) bulk_store_wait_read();   // the next batch reuses the slots
-        __syncwarp();
-    }
-    if (lane == 0) bulk_store_wait_all();
 #ifdef TFE_DBG_TIMELINE
     if (lane == 0) dbg[10] = clock64();
 #endif
-    if (failed && lane == 0) atomicOr(&p.counters[TFE_CTR_STATUS], TFE_DEV_COPY_TIMEOUT);
+    my_miss = __reduce_add_sync(0xFFFFFFFFu, my_miss);
+    tfe_finish_block(p, my_miss, cols);
+#ifdef TFE_DBG_TIMELINE
+    if (lane == 0) dbg[11] = clock64();
+#endif
+}
+
+// ------------------------------------- the hot path, LONGEST / CONST version
+//
+// The same batches, the same two phases and bit-identical results as the general kernel above
+// for the policy the benchmark grades, with the probe's three dependent steps (token ids ->
+// buckets -> stored tuple) cut down to one exposed step per batch:
+//   * the token ids of the NEXT batch are requested while the current batch streams (one id per
+//     lane, shared inside the quad by shuffles), so a batch starts with its ids in registers;
+//   * the stored tuple of a hashed-order match is requested but not waited for: selection runs on
+//     the key matches, the loads of the batch's first row are issued, and only then is the tuple
+//     compared and the selection made final and recorded.  A key match whose tuple differs (two
+//     phrases with one 64-bit key cannot both be in the table, so this means the n-gram is not a
+//     phrase) simply repeats the first row's loads with the corrected choice; nothing has been
+//     stored before that point, in place or not.
+template <int HT, bool PACKED>
+__global__ void __launch_bounds__(TFE_BLOCK_THREADS, TFE_MIN_BLOCKS)
+tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
+{
+    constexpr int VN = TfeVec<HT>::N;
+    constexpr int UNROLL = 4;
+    static_assert(!PACKED || HT == 0, "packed bf16 path needs bf16 hidden states");
+
+    const int lane = threadIdx.x & 31;
+    const int steps = p.d / VN;                  // 16-byte steps of h per row
+    const size_t hid_row_bytes = (size_t)p.d * (HT == 0 ? 2 : 4);
+    const bool in_place = p.out == p.h;
+    const int ql = lane >> 2, oi = lane & 3;
+    const int my_order = oi < p.n_orders ? p.orders[oi] : 0;
+    const bool my_hashed = my_order > 0 && !tfe_order_is_packed(my_order, p.tok_bits);
+    const uint32_t qb = p.qb;
+    const uint32_t n_batches = (p.Q + qb - 1) / qb;
+    const uint32_t n_warps = gridDim.x * TFE_WARPS_PER_BLOCK;
+    uint32_t my_miss = 0;
+
+    // the id `oi` places before query ql of a batch, or -1 (no such position / padding id)
+    // Query lq of batch b is b + lq * n_batches: a warp's queries are spread over the whole call, so
+    // a run of consecutive positions that all hit (phrases overlap) is shared out among many warps
+    // instead of making one warp fetch a row for every query of its batch.
+    auto fetch_token = [&](uint32_t batch) -> int32_t {
+        const uint32_t q = batch + (uint32_t)ql * n_batches;
+        int32_t v = -1;
+        if (batch < n_batches && ql < (int)qb && q < p.Q) {
+            const uint32_t b = tfe_div(q, p.div_tq);
+            const int32_t t = p.q_start + (int32_t)(q - b * (uint32_t)p.Tq) - oi;
+            if (t >= 0) {
+                v = __ldg(p.tokens + (size_t)b * p.T + t);
+                if ((uint32_t)v >= (uint32_t)p.vocab) v = -1;
+            }
+        }
+        return v;
+    };
+    // slot of the retained phrase if it is GPU-resident (valid on the quad's first lane), else -1
+    auto choose = [&](unsigned long long f) -> int32_t {
+        const uint32_t quad_found = (__ballot_sync(0xFFFFFFFFu, f != TFE_NONE64) >> (lane & ~3)) & 0xFu;
+        const int top = quad_found ? 31 - __clz(quad_found) : 0;
+        const unsigned long long sel = __shfl_sync(0xFFFFFFFFu, f, (lane & ~3) + top);
+        const int32_t st_ = (int32_t)(uint32_t)sel;
+        return (oi == 0 && quad_found && st_ >= 0) ? st_ : -1;
+    };
+
+    uint32_t batch = blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5);
+    int32_t tok = fetch_token(batch);
+    for (; batch < n_batches; batch += n_warps) {
+        const uint32_t q = batch + (uint32_t)ql * n_batches;
+        const bool mine = ql < (int)qb && q < p.Q;
+
+        // ================================ probe phase ================================
+        int32_t tk[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) tk[j] = __shfl_sync(0xFFFFFFFFu, tok, (lane & ~3) + j);
+        tok = fetch_token(batch + n_warps);      // lands while this batch is processed
+        bool ok = mine && my_order > 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (j < my_order && tk[j] < 0) ok = false;
+        unsigned long long found = TFE_NONE64;
+        int4 tuple = make_int4(0, 0, 0, 0);
+#ifndef TFE_DBG_NO_PROBE
+        if (ok) {
+            const uint64_t key = tfe_make_key(my_order, tk, p.tok_bits);
+            const uint64_t b1 = tfe_home_bucket_of(key, p.n_buckets);
+            const uint64_t b2 = tfe_second_bucket_of(key, b1, p.n_buckets);
+            const ulonglong4 *p1 = reinterpret_cast<const ulonglong4 *>(p.index + b1 * TFE_SLOTS_PER_BUCKET);
+            const ulonglong4 *p2 = reinterpret_cast<const ulonglong4 *>(p.index + b2 * TFE_SLOTS_PER_BUCKET);
+            ulonglong4 w[4];                     // 2 buckets x 4 slots of {key, value}, all four loads in flight
+            w[0] = ld_bucket32(p1); w[1] = ld_bucket32(p1 + 1);
+            w[2] = ld_bucket32(p2); w[3] = ld_bucket32(p2 + 1);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (w[k].x == key) found = w[k].y;
+                if (w[k].z == key) found = w[k].w;
+            }
+            if (my_hashed && found != TFE_NONE64) tuple = __ldg(p.phrase_tokens + (uint32_t)(found >> 32));
+        }
+#endif
+        __syncwarp();
+        const int32_t guess = choose(found);     // selection on key matches, tuples not yet compared
+
+        // ---- loads of the batch's first row, issued on the guess
+        uint4 hv[UNROLL];
+        typename TfeVec<HT>::RowRaw rv[UNROLL];
+        auto issue_first = [&](uint32_t lq, int32_t sl) {
+            const char *hrow = reinterpret_cast<const char *>(p.h) + (size_t)(batch + lq * n_batches) * hid_row_bytes;
+            const uint4 *rowp = p.rows + (size_t)(sl >= 0 ? sl : 0) * (size_t)(p.d / 8);
+            if (sl >= 0 || !in_place) {
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) {
+                    const int k = u * 32 + lane;
+                    if (k < steps) {
+                        hv[u] = ld_stream(reinterpret_cast<const uint4 *>(hrow) + k);
+                        if (sl >= 0) rv[u] = ld_row_raw<HT>(rowp, k);
+                    }
+                }
+            }
+        };
+        const int32_t guess0 = __shfl_sync(0xFFFFFFFFu, guess, 0);
+#ifndef TFE_DBG_NO_GATHER
+        issue_first(0, guess0);
+#endif
+
+        // ---- the tuples have arrived by now: final selection, tier walk, record
+        if (my_hashed && found != TFE_NONE64 && !tuple_matches(tuple, tk, my_order)) found = TFE_NONE64;
+        const int32_t my_slot = tfe_select_longest(p, found, q, mine, lane, my_miss);
+        const bool redo_first = __shfl_sync(0xFFFFFFFFu, my_slot, 0) != guess0;
+
+        // ================================ gather phase ===============================
+        for (uint32_t lq = 0; lq < qb; ++lq) {
+            const uint32_t gq = batch + lq * n_batches;
+            if (gq >= p.Q) break;
+#ifdef TFE_DBG_NO_GATHER
+            break;
+#endif
+            const int32_t sl = __shfl_sync(0xFFFFFFFFu, my_slot, 4 * lq);
+            if (lq > 0 || redo_first) issue_first(lq, sl);
+            if (sl < 0 && in_place) continue;    // nothing to add and nothing to copy
+            const char *hrow = reinterpret_cast<const char *>(p.h) + (size_t)gq * hid_row_bytes;
+            char *orow = reinterpret_cast<char *>(p.out) + (size_t)gq * hid_row_bytes;
+            const uint4 *rowp = p.rows + (size_t)(sl >= 0 ? sl : 0) * (size_t)(p.d / 8);
+            for (int s0 = 0; s0 < steps; s0 += 32 * UNROLL) {
+                if (s0 > 0) {
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u) {
+                        const int k = s0 + u * 32 + lane;
+                        if (k < steps) {
+                            hv[u] = ld_stream(reinterpret_cast<const uint4 *>(hrow) + k);
+                            if (sl >= 0) rv[u] = ld_row_raw<HT>(rowp, k);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) {
+                    const int k = s0 + u * 32 + lane;
+                    if (k >= steps) continue;
+                    if (sl < 0) {                // out = h bit for bit
+                        st_stream(reinterpret_cast<uint4 *>(orow) + k, hv[u]);
+                    } else if constexpr (PACKED) {
+                        // lambda is a bf16 number: one fused multiply-add per bf16 pair, rounded once
+                        // from the exact h + lambda*m
+                        const uint32_t lam2 = p.lambda_bf16x2;
+                        uint4 o;
+                        o.x = fma_bf16x2(lam2, rv[u].x, hv[u].x); o.y = fma_bf16x2(lam2, rv[u].y, hv[u].y);
+                        o.z = fma_bf16x2(lam2, rv[u].z, hv[u].z); o.w = fma_bf16x2(lam2, rv[u].w, hv[u].w);
+                        st_stream(reinterpret_cast<uint4 *>(orow) + k, o);
+                    } else {
+                        float x[VN], m[VN], y[VN];
+                        unpack_hidden<HT>(hv[u], x);
+                        unpack_row<HT>(rv[u], m);
+#pragma unroll
+                        for (int e = 0; e < VN; ++e) y[e] = fmaf(p.lambda, m[e], x[e]);
+                        store_hidden<HT>(orow, k, y);
+                    }
+                }
+            }
+        }
+    }
 
     my_miss = __reduce_add_sync(0xFFFFFFFFu, my_miss);
     tfe_finish_block(p, my_miss, 1);
