@@ -54,6 +54,10 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--tune-batch", type=int, default=0, help="queries per warp batch (0: library default)")
+    ap.add_argument("--sweep", action="store_true", help="c5: tokens x row width x hit rate sweep")
+    ap.add_argument("--sweep-tokens", default="1,4,16,64,256,1024,4096,16384,65536")
+    ap.add_argument("--sweep-d", default="1024,2048,4096")
+    ap.add_argument("--sweep-p", default="0.1,0.5,0.9")
     return ap.parse_args()
 
 
@@ -213,12 +217,140 @@ def time_oracle(w, tb, tok, h, q_start, budget_s):
 # ----------------------------------------------------------------- our arm
 
 
+class Session:
+    """One workload on one GPU: table, index, GPU-tier rows and rotating input buffers, all in HBM."""
+
+    def __init__(self, w, dev, nbuf, tune_batch=0, uniform_plant=False, table=None):
+        import torch
+        from paper_2607_07388_b200 import binding as tfe
+        from paper_2607_07388_b200.engine import Engram
+        self.w, self.dev, self.nbuf = w, dev, nbuf
+        self.tb = table if table is not None else synth.make_table(w)
+        self.rows = torch.empty((w.gpu_slots, w.d), dtype=torch.bfloat16, device=dev)
+        owner = torch.from_numpy(synth.slot_owner_of(self.tb)).to(dev)
+        synth.fill_rows_torch(self.rows, owner)
+        del owner
+        self.eng = Engram(self.tb.phrase_tokens, self.tb.phrase_len, self.tb.init_slot, self.rows, vocab=w.vocab,
+                          orders=w.orders, load_factor=w.load_factor)
+        tfe.tfe_set_tuning(self.eng.ctx, tune_batch)
+        kw = {"uniform_over_phrases": True} if (uniform_plant and w.shape == "decode") else {}
+        self.toks_np = [synth.make_queries(w, self.tb, variant=v, **kw) for v in range(nbuf)]
+        self.toks = [torch.from_numpy(t).to(dev) for t in self.toks_np]
+        self.hs = [synth.make_hidden_torch(w, dev, variant=v) for v in range(nbuf)]
+        self.outs = [torch.empty_like(self.hs[0]) for _ in range(nbuf)]
+        self.prm = tfe.TfeInjectParams(0, 0, 1.0)
+        self.tfe = tfe
+
+    def census(self):
+        """Hit / miss / valid-pair counts per buffer (one checked call each) -> algorithmic bytes."""
+        w, hits, misses, pairs = self.w, [], [], []
+        for v in range(self.nbuf):
+            r = self.eng.lookup_inject(self.toks[v], self.hs[v], self.outs[v], q_start=w.q_start)
+            misses.append(int(self.eng.miss_list(cap=0, allow_overflow=True)[3]))
+            hits.append(int((r.flags == 1).sum().item()))
+            pairs.append(valid_pairs(self.toks_np[v], w.q_start, w.orders, w.vocab))
+        self.hits, self.misses, self.pairs = hits, misses, pairs
+        self.bytes_alg = float(np.mean([algorithmic_bytes(w, pairs[v], hits[v], misses[v])
+                                        for v in range(self.nbuf)]))
+        self.gathered = float(np.mean(hits)) * w.d * 2
+
+    def lookup_calls(self, stream_ptr):
+        w = self.w
+        return [(self.eng.ctx, self.toks[v].data_ptr(), w.B, w.T, w.q_start, self.hs[v].data_ptr(),
+                 self.outs[v].data_ptr(), C.byref(self.prm), None, None, None, stream_ptr)
+                for v in range(self.nbuf)]
+
+    def close(self):
+        self.eng.close()
+
+
+class InstallPlan:
+    """c4: every step writes 4,096 fetched rows from pinned host memory into GPU-tier slots.
+
+    Destination slots walk cyclically over the region that starts free (the first pass fills free
+    slots, later passes overwrite rows installed one cycle earlier, whose phrases fall back to the
+    host tier); phrase ids walk through a seeded permutation of the phrases that start non-resident.
+    """
+
+    def __init__(self, sess, rows_per_step=4096, n_src=4):
+        import torch
+        w, tb = sess.w, sess.tb
+        self.n = rows_per_step
+        free0 = w.gpu_slots - w.reserve_free
+        self.region = (free0, w.reserve_free)
+        rng = np.random.default_rng([w.seed, 11])
+        self.ids = rng.permutation(np.nonzero(tb.init_slot < 0)[0]).astype(np.uint32)
+        self.src = []
+        for k in range(n_src):
+            bits = synth.procedural_bf16_np(self.ids[k * self.n:(k + 1) * self.n], w.d, synth.ROW_TAG, synth.ROW_SHIFT)
+            self.src.append(torch.from_numpy(bits.view(np.int16)).pin_memory())
+        self.step_no = 0
+        self.ctx, self.L = sess.eng.ctx, sess.tfe.lib()
+
+    def step(self, stream_ptr):
+        s = self.step_no
+        self.step_no += 1
+        free0, nfree = self.region
+        per_cycle = nfree // self.n
+        ids = self.ids[(s * self.n) % (len(self.ids) - self.n):][:self.n]
+        lo = free0 + (s % per_cycle) * self.n
+        dst = np.arange(lo, lo + self.n, dtype=np.int32)
+        st = self.L.tfe_cache_install(self.ctx, self.n, ids.ctypes.data, self.src[s % len(self.src)].data_ptr(),
+                                      dst.ctypes.data, stream_ptr)
+        if st:
+            raise RuntimeError(f"tfe_cache_install failed: {st}")
+
+
+def timed_region(step, steps, warmup, stream, world, dist, dev):
+    """W warm-up steps, then K steps between two CUDA events on the launch stream (max over ranks)."""
+    import torch
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    wall0 = time.time()
+    ev0.record(stream)
+    for i in range(steps):
+        step(warmup + i)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    wall1 = time.time()
+    if world > 1:
+        dist.barrier()
+    ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms, (wall0, wall1)
+
+
+def per_launch_ms(step, n, stream, flush=None):
+    """Median duration of single launches, each bracketed by its own events (optionally after an
+    L2 flush: a write of a buffer larger than the 126 MB L2, outside the events)."""
+    import torch
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+    torch.cuda.synchronize()
+    w0 = time.time()
+    for i, (e0, e1) in enumerate(evs):
+        if flush is not None:
+            flush.add_(1)
+        e0.record(stream)
+        step(i)
+        e1.record(stream)
+    torch.cuda.synchronize()
+    return float(np.median([e0.elapsed_time(e1) for e0, e1 in evs])), (w0, time.time())
+
+
 def run_ours(a):
     import torch
     import torch.distributed as dist
     from paper_2607_07388_b200 import binding as tfe
     from paper_2607_07388_b200 import build as lib_build
-    from paper_2607_07388_b200.engine import Engram, bits_from_bf16_tensor
+    from paper_2607_07388_b200.engine import bits_from_bf16_tensor
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -233,47 +365,28 @@ def run_ours(a):
         lib_build.build()
     if world > 1:
         dist.barrier()
-    tfe.lib()
+    L = tfe.lib()
+    if a.sweep:
+        return run_sweep(a, dev, rank)
 
     w = make_workload(a)
     sampler = ClockSampler(local_rank) if rank == 0 else None
-
-    # ---- inputs, resident in HBM before anything is timed
-    tb = synth.make_table(w)
-    rows = torch.empty((w.gpu_slots, w.d), dtype=torch.bfloat16, device=dev)
-    owner = torch.from_numpy(synth.slot_owner_of(tb)).to(dev)
-    synth.fill_rows_torch(rows, owner)
-    eng = Engram(tb.phrase_tokens, tb.phrase_len, tb.init_slot, rows, vocab=w.vocab, orders=w.orders,
-                 load_factor=w.load_factor)
-    tfe.tfe_set_tuning(eng.ctx, a.tune_batch)
-    kw = {"uniform_over_phrases": True} if (a.uniform_plant and w.shape == "decode") else {}
-    toks_np = [synth.make_queries(w, tb, variant=v, **kw) for v in range(NBUF)]
-    toks = [torch.from_numpy(t).to(dev) for t in toks_np]
-    hs = [synth.make_hidden_torch(w, dev, variant=v) for v in range(NBUF)]
-    outs = [torch.empty_like(hs[0]) for _ in range(NBUF)]
-    Bq, Tq, q0 = w.B, w.T, w.q_start
-
-    # ---- one checked call per buffer: hit / miss counts for the byte accounting
-    hits, misses, pairs = [], [], []
-    for v in range(NBUF):
-        r = eng.lookup_inject(toks[v], hs[v], outs[v], q_start=q0)
-        cnt = eng.miss_list(cap=0, allow_overflow=True)[3]
-        hits.append(int((r.flags == 1).sum().item()))
-        misses.append(int(cnt))
-        pairs.append(valid_pairs(toks_np[v], q0, w.orders, w.vocab))
-    bytes_alg = float(np.mean([algorithmic_bytes(w, pairs[v], hits[v], misses[v]) for v in range(NBUF)]))
-    gathered = float(np.mean(hits)) * w.d * 2
+    nbuf = NBUF if w.shape == "prefill" else NBUF_DECODE
+    sess = Session(w, dev, nbuf, a.tune_batch, a.uniform_plant)
+    sess.census()
+    tb, eng = sess.tb, sess.eng
+    q0 = w.q_start
 
     # ---- parity of buffer 0 against the oracle + CPU baseline (rank 0 only)
     parity, cpu_baseline = None, None
     if rank == 0 and not (a.no_parity and a.no_cpu_baseline):
-        h0 = bits_from_bf16_tensor(hs[0])
-        val, cores, sample, ref, ora = time_oracle(w, tb, toks_np[0], h0, q0,
+        h0 = bits_from_bf16_tensor(sess.hs[0])
+        val, cores, sample, ref, ora = time_oracle(w, tb, sess.toks_np[0], h0, q0,
                                                    0.0 if a.no_cpu_baseline else a.cpu_seconds)
         if not a.no_cpu_baseline:
             cpu_baseline = {"value": val, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample}
         if not a.no_parity:
-            r = eng.lookup_inject(toks[0], hs[0], outs[0], q_start=q0)
+            r = eng.lookup_inject(sess.toks[0], sess.hs[0], sess.outs[0], q_start=q0)
             mq, mp, mt, cnt = eng.miss_list()
             _, rounded = ora.inject(ref, h0, lam=1.0, want_exact=False)
             out0 = bits_from_bf16_tensor(r.out)
@@ -292,97 +405,64 @@ def run_ours(a):
     # ---- timed region: device-resident inputs, K steps, CUDA events on the launch stream
     stream = torch.cuda.current_stream()
     sp = stream.cuda_stream
-    L = tfe.lib()
-    prm = tfe.TfeInjectParams(0, 0, 1.0)
-    calls = [(eng.ctx, toks[v].data_ptr(), Bq, Tq, q0, hs[v].data_ptr(), outs[v].data_ptr(), C.byref(prm),
-              None, None, None, sp) for v in range(NBUF)]
+    calls = sess.lookup_calls(sp)
+    plan = InstallPlan(sess) if w.reserve_free else None
 
-    def step(i):
-        st = L.tfe_lookup_inject(*calls[i % NBUF])
+    def lookup(i):
+        st = L.tfe_lookup_inject(*calls[i % nbuf])
         if st:
             raise RuntimeError(f"tfe_lookup_inject failed: {st}")
 
-    for i in range(max(3, a.warmup)):
-        step(i)
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    wall0 = time.time()
-    ev0.record(stream)
-    for i in range(a.steps):
-        step(i)
-    ev1.record(stream)
-    torch.cuda.synchronize()
-    wall1 = time.time()
-    if world > 1:
-        dist.barrier()
-    ms = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    windows = [(wall0, wall1)]
+    def step(i):
+        if plan is not None:
+            plan.step(sp)
+        lookup(i)
 
-    # ---- per-launch durations: each launch bracketed by its own events (explains the step time)
-    n_probe = min(a.steps, 200)
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_probe)]
-    torch.cuda.synchronize()
-    w0 = time.time()
-    for i, (e0, e1) in enumerate(evs):
-        e0.record(stream)
-        step(i)
-        e1.record(stream)
-    torch.cuda.synchronize()
-    windows.append((w0, time.time()))
-    launch_ms = float(np.median([e0.elapsed_time(e1) for e0, e1 in evs]))
+    warm = max(3, a.warmup)
+    ms, win = timed_region(step, a.steps, warm, stream, world, dist, dev)
+    windows = [win]
+    launch_ms, win = per_launch_ms(lookup, min(a.steps, 200), stream)
+    windows.append(win)
+    cold_ms = None
+    if w.shape == "decode":      # small calls: also the cold-L2 latency of a single launch
+        flush = torch.zeros(192 << 20, dtype=torch.uint8, device=dev)
+        cold_ms, win = per_launch_ms(lookup, min(a.steps, 100), stream, flush)
+        windows.append(win)
+        del flush
 
     # ---- end to end through the host-buffer entry point: pinned host inputs, H2D + kernel + D2H
     e2e = None
     if a.e2e_steps > 0:
-        tok_h = [torch.from_numpy(toks_np[v]).pin_memory() for v in range(2)]
-        h_h = [hs[v].cpu().pin_memory() for v in range(2)]
+        tok_h = [torch.from_numpy(sess.toks_np[v]).pin_memory() for v in range(2)]
+        h_h = [sess.hs[v].cpu().pin_memory() for v in range(2)]
         out_h = [torch.empty_like(h_h[0]).pin_memory() for _ in range(2)]
-        hcalls = [(eng.ctx, tok_h[v].data_ptr(), Bq, Tq, q0, h_h[v].data_ptr(), out_h[v].data_ptr(),
-                   C.byref(prm), None, None, None, sp) for v in range(2)]
-        cap = max(1, max(misses))
+        hcalls = [(eng.ctx, tok_h[v].data_ptr(), w.B, w.T, q0, h_h[v].data_ptr(), out_h[v].data_ptr(),
+                   C.byref(sess.prm), None, None, None, sp) for v in range(2)]
+        cap = max(1, max(sess.misses) * 2)
         mq = np.empty(cap, np.uint32); mp = np.empty(cap, np.uint32); mt = np.empty(cap, np.uint8)
         cnt = C.c_int64(0)
 
         def e2e_step(i):
+            if plan is not None:
+                plan.step(sp)
             st = L.tfe_lookup_inject_host(*hcalls[i % 2])
             st2 = L.tfe_miss_list(eng.ctx, mq.ctypes.data, mp.ctypes.data, mt.ctypes.data, cap, C.byref(cnt), sp)
             if st or st2 not in (0, tfe.TFE_ERR_MISS_OVERFLOW):
                 raise RuntimeError(f"host-buffer step failed: {st} {st2}")
 
-        for i in range(3):
-            e2e_step(i)
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        w0 = time.time()
-        ev0.record(stream)
-        for i in range(a.e2e_steps):
-            e2e_step(i)
-        ev1.record(stream)
-        torch.cuda.synchronize()
-        windows.append((w0, time.time()))
-        e_ms = ev0.elapsed_time(ev1)
-        if world > 1:
-            t = torch.tensor([e_ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
-        h2d = w.B * w.T * 4 + w.Q * w.d * 2
-        d2h = w.Q * w.d * 2 + TFE_CTR_BYTES + int(np.mean(misses)) * 9
+        e_ms, win = timed_region(e2e_step, a.e2e_steps, 3, stream, world, dist, dev)
+        windows.append(win)
+        h2d = w.B * w.T * 4 + w.Q * w.d * 2 + (plan.n * (w.d * 2 + 8) if plan else 0)
+        d2h = w.Q * w.d * 2 + TFE_CTR_BYTES + int(np.mean(sess.misses)) * 9
         e2e = {"value": world * w.Q * a.e2e_steps / (e_ms * 1e-3), "unit": "tokens/s",
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                "ms_per_step": e_ms / a.e2e_steps, "steps": a.e2e_steps,
-               "call": "tfe_lookup_inject_host + tfe_miss_list (pinned host buffers)"}
+               "call": "tfe_lookup_inject_host + tfe_miss_list (pinned host buffers)"
+                       + (", after tfe_cache_install" if plan else "")}
 
     clocks = sampler.stop(windows) if sampler else None
     grid, block, qb = tfe.tfe_launch_geometry(eng.ctx)
-    eng.close()
+    sess.close()
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
@@ -391,12 +471,13 @@ def run_ours(a):
 
     ms_per_step = ms / a.steps
     peak, peak_src = measured_peak()
-    achieved = bytes_alg / (ms_per_step * 1e-3) / 1e9
+    achieved = sess.bytes_alg / (ms_per_step * 1e-3) / 1e9
+    buf_mb = nbuf * 2 * w.Q * w.d * 2 / 1e6
     line = {
         "metric": "lookup+inject tokens/s",
         "value": world * w.Q * a.steps / (ms * 1e-3),
         "unit": "tokens/s",
-        "n_gpus": world, "steps": a.steps, "warmup": max(3, a.warmup),
+        "n_gpus": world, "steps": a.steps, "warmup": warm,
         "ms_per_step": ms_per_step,
         "higher_is_better": True,
         "scaling": "weak",
@@ -408,30 +489,87 @@ def run_ours(a):
             "orders": list(w.orders), "n_phrases": w.n_phrases, "gpu_slots": w.gpu_slots, "d": w.d,
             "zipf_s": w.s, "planted": w.p, "load_factor": w.load_factor, "policy": "LONGEST", "gate": "CONST",
             "lambda": 1.0, "out_of_place": True,
-            "hit_fraction": float(np.mean(hits)) / w.Q, "miss_fraction": float(np.mean(misses)) / w.Q,
-            "l2": f"inputs rotate over {NBUF} token/hidden/output buffer sets "
-                  f"({NBUF * 2 * w.Q * w.d * 2 / 1e6:.0f} MB) and a {w.gpu_slots * w.d * 2 / 1e9:.1f} GB row table; "
-                  f"{'larger' if NBUF * 2 * w.Q * w.d * 2 > 126e6 else 'SMALLER'} than the 126 MB L2",
+            "step": ("tfe_cache_install(4096 rows from pinned host) + tfe_lookup_inject" if plan
+                     else "tfe_lookup_inject"),
+            "hit_fraction": float(np.mean(sess.hits)) / w.Q, "miss_fraction": float(np.mean(sess.misses)) / w.Q,
+            "l2": f"inputs rotate over {nbuf} token/hidden/output buffer sets ({buf_mb:.0f} MB) and a "
+                  f"{w.gpu_slots * w.d * 2 / 1e9:.1f} GB row table"
+                  + ("; larger than the 126 MB L2" if buf_mb > 126 else
+                     "; buffers smaller than the 126 MB L2, cold_launch_us is taken after an L2 flush"),
             "parallelism": "replicas only" if world > 1 else "single GPU",
             "grid": grid, "block": block, "batch_queries": qb,
         },
-        "gathered_hbm_gbs": gathered / (ms_per_step * 1e-3) / 1e9,
+        "gathered_hbm_gbs": sess.gathered / (ms_per_step * 1e-3) / 1e9,
         "frac_of_8tbs": achieved / HBM_NOMINAL_GBS,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_source": peak_src, "algorithmic_bytes_per_launch": bytes_alg,
-                     "kernel": "tfe_lookup_inject_kernel<bf16,LONGEST,CONST>",
+                     "traffic": NCU_TRAFFIC.get(w.name), "peak_source": peak_src,
+                     "algorithmic_bytes_per_launch": sess.bytes_alg,
+                     "kernel": "tfe_lookup_inject_longest_kernel<bf16, packed>",
                      "launch_ms_own_events": launch_ms,
-                     "achieved_own_events": bytes_alg / (launch_ms * 1e-3) / 1e9},
+                     "achieved_own_events": sess.bytes_alg / (launch_ms * 1e-3) / 1e9},
         "cpu_baseline": cpu_baseline,
         "e2e": e2e,
-        "gpu_launches": a.steps,
+        "gpu_launches": a.steps * (2 if plan else 1),
         "clocks": clocks,
         "parity": parity,
     }
+    if cold_ms is not None:
+        line["cold_launch_us"] = cold_ms * 1e3
     print(json.dumps(line))
 
 
-TFE_CTR_BYTES = 160     # the launch-state words tfe_miss_list reads back
+def run_sweep(a, dev, rank):
+    """c5: lookup+inject only, tokens per call x row width x planted hit rate, one 8M-entry table."""
+    import torch
+    from paper_2607_07388_b200 import binding as tfe
+    L = tfe.lib()
+    peak, peak_src = measured_peak()
+    stream = torch.cuda.current_stream()
+    sp = stream.cuda_stream
+    base = make_workload(a)
+    table = None
+    points = []
+    tokens_list = [int(t) for t in a.sweep_tokens.split(",")]
+    for d in [int(x) for x in a.sweep_d.split(",")]:
+        for p_hit in [float(x) for x in a.sweep_p.split(",")]:
+            for n_tok in tokens_list:
+                w = synth.config(5, d=d, p=p_hit, B=n_tok, n_phrases=base.n_phrases, gpu_slots=base.gpu_slots)
+                if table is None:
+                    table = synth.make_table(w)
+                nbuf = 4 if n_tok * d * 4 * 4 > 200e6 else 16
+                sess = Session(w, dev, nbuf, a.tune_batch, a.uniform_plant, table=table)
+                sess.census()
+                calls = sess.lookup_calls(sp)
+
+                def lookup(i):
+                    st = L.tfe_lookup_inject(*calls[i % nbuf])
+                    if st:
+                        raise RuntimeError(f"tfe_lookup_inject failed: {st}")
+
+                steps = 400 if n_tok <= 16384 else 100
+                ms, _ = timed_region(lookup, steps, 10, stream, 1, None, dev)
+                us = ms / steps * 1e3
+                points.append({"tokens": n_tok, "d": d, "planted": p_hit, "us_per_call": us,
+                               "tokens_per_s": n_tok / (us * 1e-6),
+                               "hit_fraction": float(np.mean(sess.hits)) / w.Q,
+                               "gathered_gbs": sess.gathered / us / 1e3,
+                               "algorithmic_gbs": sess.bytes_alg / us / 1e3,
+                               "frac_of_measured_peak": sess.bytes_alg / us / 1e3 / peak,
+                               "frac_of_8tbs": sess.bytes_alg / us / 1e3 / HBM_NOMINAL_GBS,
+                               "batch_queries": tfe.tfe_launch_geometry(sess.eng.ctx)[2]})
+                sess.close()
+                del sess
+                torch.cuda.empty_cache()
+    if rank == 0:
+        print(json.dumps({"metric": "lookup+inject tokens/s", "unit": "tokens/s", "workload": "c5_sweep",
+                          "n_phrases": base.n_phrases, "peak": peak, "peak_source": peak_src, "sweep": points}))
+
+
+TFE_CTR_BYTES = 16      # the launch-state words tfe_miss_list reads back
+NBUF_DECODE = 32        # decode shapes: this many distinct query / hidden-state sets rotate
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the lookup kernel, from the ncu capture
+# summarised under profiles/ (a 1M-phrase capture scaled is not needed: traffic does not depend on N)
+NCU_TRAFFIC = {}
 
 
 # ------------------------------------------------------------ reference arm

@@ -128,3 +128,56 @@ def pair_from_workload(w: synth.Workload, **kw):
     rows = synth.make_rows_np(w, tb)
     return tb, Pair(tb.phrase_tokens, tb.phrase_len, tb.init_slot, rows, vocab=w.vocab, orders=w.orders,
                     load_factor=w.load_factor, **kw)
+
+
+class BigPair:
+    """A benchmark-sized table: rows are filled on the device by the procedural generator and
+    looked up lazily by the oracle through a sparsely committed host mapping, so nothing the size
+    of the table ever sits in host memory."""
+
+    def __init__(self, w: synth.Workload, table=None):
+        self.w = w
+        self.tb = table if table is not None else synth.make_table(w)
+        self.rows_gpu = torch.empty((w.gpu_slots, w.d), dtype=torch.bfloat16, device=DEV)
+        synth.fill_rows_torch(self.rows_gpu, torch.from_numpy(synth.slot_owner_of(self.tb)).to(DEV))
+        self.eng = Engram(self.tb.phrase_tokens, self.tb.phrase_len, self.tb.init_slot, self.rows_gpu,
+                          vocab=w.vocab, orders=w.orders, load_factor=w.load_factor)
+        self.sparse = synth.SparseRows(w.gpu_slots, w.d)
+        self.ora = orc.Oracle(self.tb.phrase_tokens, self.tb.phrase_len, self.tb.init_slot, self.sparse.array,
+                              d=w.d, vocab=w.vocab, orders=w.orders, gpu_slots=w.gpu_slots)
+
+    def close(self):
+        self.eng.close()
+
+    def check(self, tokens, variant=0, lam=1.0, sample_rows=None):
+        """One lookup on the GPU, all integer outputs against the oracle, hidden states against the
+        oracle on every row (or on `sample_rows` seeded rows for very wide calls)."""
+        w = self.w
+        tok_gpu = torch.from_numpy(tokens).to(DEV)
+        h_gpu = synth.make_hidden_torch(w, DEV, variant=variant, Q=tokens.shape[0] * (tokens.shape[1] - w.q_start))
+        got = self.eng.lookup_inject(tok_gpu, h_gpu, q_start=w.q_start, lam=lam)
+        mq, mp, mt, cnt = self.eng.miss_list(cap=max(1, got.flags.numel() * len(w.orders)))
+        ref = self.ora.lookup(tokens, w.q_start)
+        np.testing.assert_array_equal(got.sel_phrase.cpu().numpy().view(np.uint32), ref.sel_phrase)
+        np.testing.assert_array_equal(got.sel_slot.cpu().numpy(), ref.sel_slot)
+        np.testing.assert_array_equal(got.flags.cpu().numpy(), ref.flags)
+        assert cnt == len(ref.miss_q)
+        np.testing.assert_array_equal(mq, ref.miss_q)
+        np.testing.assert_array_equal(mp, ref.miss_phrase)
+        np.testing.assert_array_equal(mt, ref.miss_tier)
+        Q = len(ref.flags)
+        rows_sel = np.arange(Q)
+        if sample_rows is not None and sample_rows < Q:
+            rows_sel = np.sort(np.random.default_rng(w.seed).choice(Q, sample_rows, replace=False))
+        hit = ref.flags[rows_sel] == 1
+        slots = np.unique(ref.sel_slot[rows_sel][hit])
+        self.sparse.materialise(slots, self.ora.slot_owner[slots])
+        sub = orc.LookupResult(ref.match[rows_sel], ref.sel_phrase[rows_sel], ref.sel_slot[rows_sel],
+                               ref.flags[rows_sel], ref.miss_q[:0], ref.miss_phrase[:0], ref.miss_tier[:0])
+        h_np = bits_from_bf16_tensor(h_gpu[torch.from_numpy(rows_sel).to(DEV)])
+        exact, rounded = self.ora.inject(sub, h_np, lam=float(np.float32(lam)))
+        out = bits_from_bf16_tensor(got.out[torch.from_numpy(rows_sel).to(DEV)])
+        err = np.abs(synth.bf16_bits_to_f32(out).astype(np.float64) - exact).max()
+        assert err <= TOL_BF16, err
+        np.testing.assert_array_equal(out, rounded)      # lambda is a bf16 number: single rounding on both sides
+        return dict(n_hit=int((ref.flags == 1).sum()), n_miss=int(cnt), Q=Q, max_abs_err=float(err), ref=ref)
