@@ -167,6 +167,40 @@ tfe_status tfe_lookup_inject_host(tfe_ctx *ctx, const int32_t *tokens, int32_t B
 tfe_status tfe_miss_list(tfe_ctx *ctx, uint32_t *q_idx, uint32_t *phrase_id, uint8_t *tier,
                          int64_t cap, int64_t *count, void *stream);
 
+/*
+ * tfe_lookup_inject_noalloc -- tfe_lookup_inject for callers that must not allocate.  (The paper
+ * has no counterpart for this entry point; it exists for the sake of the embedding runtime.)
+ *
+ * tfe_lookup_inject lets the context cudaMalloc its per-call scratch on first use and again when
+ * a larger call arrives.  A runtime that has given all free device memory to its own pool, or a
+ * latency-critical loop that cannot tolerate the device-wide synchronisation an allocation or a
+ * free brings, calls this instead: it allocates and frees nothing, on the host or on the device.
+ * Its scratch is a fixed area inside the loaded library image (about 1.3 MB, present on every GPU
+ * that loads the library until the process ends), which bounds the call:
+ *
+ *     Q * (policy == ALL ? n_orders : 1)  <=  262,144      otherwise TFE_ERR_CAPACITY.
+ *
+ *   tokens ... flags   as for tfe_lookup_inject (DEVICE; sel_phrase / sel_slot / flags may be NULL).
+ *   miss_q, miss_phrase, miss_tier
+ *                      DEVICE, CALLER-OWNED, each with room for Q * (ALL ? n_orders : 1) entries;
+ *                      receive the ordered miss list (the context's own list and tfe_miss_list are
+ *                      not involved).  Required.
+ *   miss_count         DEVICE uint32, receives the number of entries written.  Required.
+ *
+ * The context's device must be the current device.  The first call on a device looks up the
+ * address of the scratch area (cudaGetSymbolAddress); make that first call outside any stream
+ * capture.  All calls on one device share the area, whatever their context: a call clears what
+ * must start at zero and the stream orders it, but two calls that overlap on the GPU (different
+ * streams, no dependency) race.  Results are those of tfe_lookup_inject.
+ * Errors: INVALID_ARG, CAPACITY, CUDA.
+ */
+tfe_status tfe_lookup_inject_noalloc(tfe_ctx *ctx, const int32_t *tokens, int32_t B, int32_t T,
+                                     int32_t q_start, const void *h, void *out,
+                                     const tfe_inject_params *params, uint32_t *sel_phrase,
+                                     int32_t *sel_slot, uint8_t *flags, uint32_t *miss_q,
+                                     uint32_t *miss_phrase, uint8_t *miss_tier, uint32_t *miss_count,
+                                     void *stream);
+
 /* The same list as DEVICE pointers owned by the context, valid until the next lookup; no sync. */
 tfe_status tfe_miss_list_device(tfe_ctx *ctx, const uint32_t **q_idx, const uint32_t **phrase_id,
                                 const uint8_t **tier, const uint32_t **count);

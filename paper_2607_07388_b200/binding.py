@@ -31,7 +31,7 @@ NO_PHRASE = 0xFFFFFFFF
 EXPORTS = ["tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
            "tfe_miss_list", "tfe_miss_list_device", "tfe_destroy", "tfe_status_string",
            "tfe_last_cuda_error", "tfe_index_geometry", "tfe_phrase_key64", "tfe_home_bucket",
-           "tfe_launch_geometry", "tfe_set_tuning"]
+           "tfe_launch_geometry", "tfe_set_tuning", "tfe_lookup_inject_noalloc"]
 
 
 class TfeConfig(C.Structure):
@@ -70,6 +70,8 @@ def lib() -> C.CDLL:
         L.tfe_cache_install.argtypes = [vp, i32, vp, vp, vp, vp]
         L.tfe_lookup_inject.argtypes = [vp, vp, i32, i32, i32, vp, vp, C.POINTER(TfeInjectParams), vp, vp, vp, vp]
         L.tfe_lookup_inject_host.argtypes = L.tfe_lookup_inject.argtypes
+        L.tfe_lookup_inject_noalloc.argtypes = [vp, vp, i32, i32, i32, vp, vp, C.POINTER(TfeInjectParams), vp, vp, vp,
+                                                vp, vp, vp, vp, vp]
         L.tfe_miss_list.argtypes = [vp, vp, vp, vp, i64, C.POINTER(i64), vp]
         L.tfe_miss_list_device.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]
         L.tfe_destroy.argtypes = [vp]
@@ -86,7 +88,7 @@ def lib() -> C.CDLL:
         L.tfe_set_tuning.argtypes = [vp, i32]
         for name in ("tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
                      "tfe_miss_list", "tfe_miss_list_device", "tfe_index_geometry", "tfe_launch_geometry",
-                     "tfe_set_tuning"):
+                     "tfe_set_tuning", "tfe_lookup_inject_noalloc"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -170,6 +172,22 @@ def tfe_lookup_inject_host(ctx: int, tokens, B, T, q_start, h, out, *, policy=PO
     _check(lib().tfe_lookup_inject_host(ctx, _addr(tokens), B, T, q_start, _addr(h), _addr(out), C.byref(p),
                                         _addr(sel_phrase), _addr(sel_slot), _addr(flags), _stream(stream)),
            "tfe_lookup_inject_host")
+
+
+NOALLOC_MAX_ENTRIES = 262_144
+
+
+def tfe_lookup_inject_noalloc(ctx: int, tokens, B, T, q_start, h, out, *, miss_q, miss_phrase, miss_tier,
+                              miss_count, policy=POLICY_LONGEST, gate=GATE_CONST, lam=1.0, sel_phrase=None,
+                              sel_slot=None, flags=None, stream=None) -> None:
+    """The lookup for callers that must not allocate: scratch is a fixed area of the library image,
+    the miss list goes to caller-owned device buffers.  At most NOALLOC_MAX_ENTRIES (query, order)
+    entries per call."""
+    p = _params(policy, gate, lam)
+    _check(lib().tfe_lookup_inject_noalloc(ctx, _addr(tokens), B, T, q_start, _addr(h), _addr(out), C.byref(p),
+                                           _addr(sel_phrase), _addr(sel_slot), _addr(flags), _addr(miss_q),
+                                           _addr(miss_phrase), _addr(miss_tier), _addr(miss_count),
+                                           _stream(stream)), "tfe_lookup_inject_noalloc")
 
 
 def tfe_miss_list(ctx: int, cap: int, stream=None, allow_overflow=False):

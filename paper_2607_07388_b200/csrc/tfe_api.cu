@@ -645,3 +645,98 @@ tfe_status tfe_miss_list_device(tfe_ctx *c, const uint32_t **q_idx, const uint32
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Lookup without any allocation.
+//
+// tfe_lookup_inject keeps its per-call scratch (one flag byte and one phrase id per (query,
+// order), plus a few counter words) in buffers the context allocates with cudaMalloc the first
+// time a call needs them, and grows them when a larger call arrives.  A serving loop that has
+// handed all free device memory to its own pool, or that must never hit the device-wide
+// synchronisation cudaMalloc / cudaFree imply, cannot afford that.  For such callers the same
+// kernels run here on a fixed scratch area that is part of the loaded library image: a file-scope
+// __device__ array, present once on every GPU that loads the library, for as long as the process
+// lives.  Its size bounds the call: at most TFE_NOALLOC_MAX_ENTRIES (query, order) entries.
+//
+// g_tfe_noalloc_scratch below is, in host code, only a handle: the kernels need the device
+// address, which cudaGetSymbolAddress returns for the device that is current when it is asked.
+// The first call on each device asks once and remembers the answer.
+#define TFE_NOALLOC_MAX_ENTRIES 262144
+#define TFE_NOALLOC_COUNTER_BYTES 256
+#define TFE_NOALLOC_BYTES (TFE_NOALLOC_COUNTER_BYTES + TFE_NOALLOC_MAX_ENTRIES * 4 + TFE_NOALLOC_MAX_ENTRIES)
+static __device__ __align__(256) unsigned char g_tfe_noalloc_scratch[TFE_NOALLOC_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+unsigned char *g_noalloc_ptr[kMaxDevices] = {nullptr};      // device address of the array, per device
+}  // namespace
+
+extern "C" tfe_status tfe_lookup_inject_noalloc(tfe_ctx *c, const int32_t *tokens, int32_t B, int32_t T,
+                                                int32_t q_start, const void *h, void *out,
+                                                const tfe_inject_params *prm, uint32_t *sel_phrase,
+                                                int32_t *sel_slot, uint8_t *flags, uint32_t *miss_q,
+                                                uint32_t *miss_phrase, uint8_t *miss_tier, uint32_t *miss_count,
+                                                void *stream_)
+{
+    if (!c || !prm || B < 0 || T < 0 || q_start < 0 || q_start > T) return TFE_ERR_INVALID_ARG;
+    if (prm->policy != TFE_POLICY_LONGEST && prm->policy != TFE_POLICY_ALL) return TFE_ERR_INVALID_ARG;
+    if (prm->gate != TFE_GATE_CONST && prm->gate != TFE_GATE_COSINE) return TFE_ERR_INVALID_ARG;
+    if (!miss_q || !miss_phrase || !miss_tier || !miss_count) return TFE_ERR_INVALID_ARG;
+    const int64_t Tq = T - q_start, Q = (int64_t)B * Tq;
+    const int cols = prm->policy == TFE_POLICY_ALL ? c->cfg.n_orders : 1;
+    if (Q * cols > TFE_NOALLOC_MAX_ENTRIES) return TFE_ERR_CAPACITY;      // the fixed scratch area is too small
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int dev = -1;
+    CU(cudaGetDevice(&dev));
+    if (dev != c->device || dev < 0 || dev >= kMaxDevices) return TFE_ERR_INVALID_ARG;
+    if (g_noalloc_ptr[dev] == nullptr) {       // once per device, with that device current
+        void *ptr = nullptr;
+        CU(cudaGetSymbolAddress(&ptr, g_tfe_noalloc_scratch));
+        g_noalloc_ptr[dev] = static_cast<unsigned char *>(ptr);
+    }
+    unsigned char *const scratch = g_noalloc_ptr[dev];
+    uint32_t *const counters = reinterpret_cast<uint32_t *>(scratch);
+    // the area is shared by every call and keeps what the last one left: start the counters from zero
+    CU(cudaMemsetAsync(counters, 0, TFE_CTR_WORDS * sizeof(uint32_t), stream));
+    if (Q == 0) {
+        CU(cudaMemsetAsync(miss_count, 0, sizeof(uint32_t), stream));
+        return TFE_OK;
+    }
+    if (!tokens || !h || !out) return TFE_ERR_INVALID_ARG;
+    if (((reinterpret_cast<uintptr_t>(h) | reinterpret_cast<uintptr_t>(out)) & 15u) != 0)
+        return TFE_ERR_INVALID_ARG;
+
+    const bool all = prm->policy == TFE_POLICY_ALL, cos = prm->gate == TFE_GATE_COSINE;
+    uint32_t lam_bits;
+    std::memcpy(&lam_bits, &prm->lambda, sizeof lam_bits);
+    const bool lam_is_bf16 = (lam_bits & 0xFFFFu) == 0 && (lam_bits & 0x7F800000u) != 0x7F800000u;
+    const int ht = c->cfg.hidden_dtype;
+    const int variant = (all || cos) ? ht * 4 + (all ? 2 : 0) + (cos ? 1 : 0)
+                                     : (ht == 1 ? kVarLongestF32 : (lam_is_bf16 ? kVarLongestPacked : kVarLongest));
+    const int64_t resident = (int64_t)c->sm_count * c->occ[variant];
+    const int64_t qb = c->qb_override ? c->qb_override : pick_batch(Q, resident * TFE_WARPS_PER_BLOCK);
+    const int64_t n_batches = (Q + qb - 1) / qb;
+    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(resident, (n_batches + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK));
+    TfeLookupParams p{};
+    p.tokens = tokens; p.B = B; p.T = T; p.q_start = q_start; p.Tq = (int32_t)Tq; p.Q = (uint32_t)Q;
+    p.div_tq = make_fastdiv((uint32_t)Tq); p.qb = (uint32_t)qb;
+    p.index = c->d_index; p.n_buckets = c->n_buckets;
+    p.phrase_tokens = c->d_phrase_tokens; p.rows = c->gpu_rows; p.d = c->cfg.d;
+    p.h = h; p.out = out;
+    p.n_orders = c->cfg.n_orders;
+    for (int i = 0; i < 4; ++i) p.orders[i] = i < c->cfg.n_orders ? c->cfg.orders[i] : 0;
+    p.tok_bits = c->tok_bits; p.vocab = c->cfg.vocab; p.lambda = prm->lambda;
+    p.lambda_bf16x2 = (lam_bits >> 16) | (lam_bits & 0xFFFF0000u);
+    p.sel_phrase = sel_phrase; p.sel_slot = sel_slot; p.flags = flags;
+    p.scr_phrase = reinterpret_cast<uint32_t *>(scratch + TFE_NOALLOC_COUNTER_BYTES);
+    p.scr_flag = scratch + TFE_NOALLOC_COUNTER_BYTES + (size_t)TFE_NOALLOC_MAX_ENTRIES * 4;
+    p.miss_q = miss_q; p.miss_phrase = miss_phrase; p.miss_tier = miss_tier;
+    p.counters = counters;
+#ifdef TFE_DBG_TIMELINE
+    p.dbg = c->dbg;
+#endif
+    pick_kernel(variant)<<<(unsigned)grid, TFE_BLOCK_THREADS, 0, stream>>>(p);
+    CU(cudaGetLastError());
+    CU(cudaMemcpyAsync(miss_count, counters + TFE_CTR_TOTAL, sizeof(uint32_t), cudaMemcpyDeviceToDevice, stream));
+    return TFE_OK;
+}
