@@ -301,6 +301,21 @@ class InstallPlan:
             raise RuntimeError(f"tfe_cache_install failed: {st}")
 
 
+def max_over_ranks(ms, world, dist, dev):
+    """Every rank's elapsed time -> the slowest rank's (what the whole job took)."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(units_per_rank_step, steps, world, ms):
+    """Whole-job units per second: all ranks' units over the slowest rank's time (replicas: weak scaling)."""
+    return world * units_per_rank_step * steps / (ms * 1e-3)
+
+
 def timed_region(step, steps, warmup, stream, world, dist, dev):
     """W warm-up steps, then K steps between two CUDA events on the launch stream (max over ranks)."""
     import torch
@@ -320,11 +335,7 @@ def timed_region(step, steps, warmup, stream, world, dist, dev):
     wall1 = time.time()
     if world > 1:
         dist.barrier()
-    ms = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ev0.elapsed_time(ev1), world, dist, dev)
     return ms, (wall0, wall1)
 
 
@@ -454,7 +465,7 @@ def run_ours(a):
         windows.append(win)
         h2d = w.B * w.T * 4 + w.Q * w.d * 2 + (plan.n * (w.d * 2 + 8) if plan else 0)
         d2h = w.Q * w.d * 2 + TFE_CTR_BYTES + int(np.mean(sess.misses)) * 9
-        e2e = {"value": world * w.Q * a.e2e_steps / (e_ms * 1e-3), "unit": "tokens/s",
+        e2e = {"value": job_throughput(w.Q, a.e2e_steps, world, e_ms), "unit": "tokens/s",
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                "ms_per_step": e_ms / a.e2e_steps, "steps": a.e2e_steps,
                "call": "tfe_lookup_inject_host + tfe_miss_list (pinned host buffers)"
@@ -475,7 +486,7 @@ def run_ours(a):
     buf_mb = nbuf * 2 * w.Q * w.d * 2 / 1e6
     line = {
         "metric": "lookup+inject tokens/s",
-        "value": world * w.Q * a.steps / (ms * 1e-3),
+        "value": job_throughput(w.Q, a.steps, world, ms),
         "unit": "tokens/s",
         "n_gpus": world, "steps": a.steps, "warmup": warm,
         "ms_per_step": ms_per_step,

@@ -1,0 +1,49 @@
+"""Host-side logic of the multi-GPU benchmark path, on CPU with two gloo ranks: the path does not
+shard (replicas only), so the only cross-rank steps are the barrier and the max-over-ranks of the
+elapsed time, and the reported value is all ranks' tokens over the slowest rank's time."""
+import os
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _rank_main(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    import bench
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    local_ms = 10.0 + 5.0 * rank                      # rank 1 is the slow replica
+    dist.barrier()
+    ms = bench.max_over_ranks(local_ms, world, dist, torch.device("cpu"))
+    value = bench.job_throughput(32768, 100, world, ms)
+    out.put((rank, ms, value))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_replica_timing_takes_the_slowest_rank():
+    world, port = 2, 29731
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_rank_main, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = sorted(q.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, ms, value in got:
+        assert ms == 15.0
+        assert value == pytest.approx(2 * 32768 * 100 / 15e-3)
+
+
+def test_single_rank_needs_no_process_group():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.max_over_ranks(7.5, 1, None, None) == 7.5
+    assert bench.job_throughput(64, 10, 1, 2.0) == pytest.approx(64 * 10 / 2e-3)
