@@ -233,13 +233,22 @@ class Session:
         self.eng = Engram(self.tb.phrase_tokens, self.tb.phrase_len, self.tb.init_slot, self.rows, vocab=w.vocab,
                           orders=w.orders, load_factor=w.load_factor)
         tfe.tfe_set_tuning(self.eng.ctx, tune_batch)
-        kw = {"uniform_over_phrases": True} if (uniform_plant and w.shape == "decode") else {}
-        self.toks_np = [synth.make_queries(w, self.tb, variant=v, **kw) for v in range(nbuf)]
-        self.toks = [torch.from_numpy(t).to(dev) for t in self.toks_np]
-        self.hs = [synth.make_hidden_torch(w, dev, variant=v) for v in range(nbuf)]
-        self.outs = [torch.empty_like(self.hs[0]) for _ in range(nbuf)]
+        self.uniform_plant = uniform_plant
         self.prm = tfe.TfeInjectParams(0, 0, 1.0)
         self.tfe = tfe
+        self.set_inputs(w, nbuf)
+
+    def set_inputs(self, w, nbuf):
+        """(Re)make the rotating query / hidden / output buffers; `w` may differ from the table's
+        workload in batch size and planted rate only."""
+        import torch
+        self.w, self.nbuf = w, nbuf
+        self.toks = self.hs = self.outs = None
+        kw = {"uniform_over_phrases": True} if (self.uniform_plant and w.shape == "decode") else {}
+        self.toks_np = [synth.make_queries(w, self.tb, variant=v, **kw) for v in range(nbuf)]
+        self.toks = [torch.from_numpy(t).to(self.dev) for t in self.toks_np]
+        self.hs = [synth.make_hidden_torch(w, self.dev, variant=v) for v in range(nbuf)]
+        self.outs = [torch.empty_like(self.hs[0]) for _ in range(nbuf)]
 
     def census(self):
         """Hit / miss / valid-pair counts per buffer (one checked call each) -> algorithmic bytes."""
@@ -542,13 +551,15 @@ def run_sweep(a, dev, rank):
     points = []
     tokens_list = [int(t) for t in a.sweep_tokens.split(",")]
     for d in [int(x) for x in a.sweep_d.split(",")]:
+        w0 = synth.config(5, d=d, B=1, n_phrases=base.n_phrases, gpu_slots=base.gpu_slots)
+        if table is None:
+            table = synth.make_table(w0)
+        sess = Session(w0, dev, 1, a.tune_batch, a.uniform_plant, table=table)     # rows + index once per width
         for p_hit in [float(x) for x in a.sweep_p.split(",")]:
             for n_tok in tokens_list:
                 w = synth.config(5, d=d, p=p_hit, B=n_tok, n_phrases=base.n_phrases, gpu_slots=base.gpu_slots)
-                if table is None:
-                    table = synth.make_table(w)
                 nbuf = 4 if n_tok * d * 4 * 4 > 200e6 else 16
-                sess = Session(w, dev, nbuf, a.tune_batch, a.uniform_plant, table=table)
+                sess.set_inputs(w, nbuf)
                 sess.census()
                 calls = sess.lookup_calls(sp)
 
@@ -568,9 +579,9 @@ def run_sweep(a, dev, rank):
                                "frac_of_measured_peak": sess.bytes_alg / us / 1e3 / peak,
                                "frac_of_8tbs": sess.bytes_alg / us / 1e3 / HBM_NOMINAL_GBS,
                                "batch_queries": tfe.tfe_launch_geometry(sess.eng.ctx)[2]})
-                sess.close()
-                del sess
-                torch.cuda.empty_cache()
+        sess.close()
+        del sess
+        torch.cuda.empty_cache()
     if rank == 0:
         print(json.dumps({"metric": "lookup+inject tokens/s", "unit": "tokens/s", "workload": "c5_sweep",
                           "n_phrases": base.n_phrases, "peak": peak, "peak_source": peak_src, "sweep": points}))
@@ -580,7 +591,7 @@ TFE_CTR_BYTES = 16      # the launch-state words tfe_miss_list reads back
 NBUF_DECODE = 32        # decode shapes: this many distinct query / hidden-state sets rotate
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the lookup kernel, from the ncu capture
 # summarised under profiles/ (a 1M-phrase capture scaled is not needed: traffic does not depend on N)
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {"c3_prefill8x4096": 124_960_000}
 
 
 # ------------------------------------------------------------ reference arm

@@ -109,21 +109,23 @@ lookup_kernel_t pick_kernel(int variant)
     return table[variant];
 }
 
-// Queries per warp batch (1..8) for a call of Q queries on `warps` resident warps: the split into
-// r rounds of ceil(Q / (warps*r)) queries that leaves the busiest warp the least work (small
-// calls: one query per warp, the lowest latency).
+// Queries per warp batch (1..8) for a call of Q queries on `warps` resident warps.  A split into r
+// rounds of qb = ceil(Q / (warps*r)) queries gives the busiest warp r*qb queries; among the splits
+// within 8 % of the least such load the largest batch wins (fewer probe phases per warp).  Small
+// calls: one query per warp, the lowest latency.
 int pick_batch(int64_t Q, int64_t warps)
 {
     if (Q <= warps) return 1;
-    int best_qb = 8;
-    int64_t best_load = INT64_MAX;
-    for (int64_t r = 1; r <= 64; ++r) {
-        const int64_t qb = (Q + warps * r - 1) / (warps * r);
-        if (qb > 8) continue;
-        if (r * qb < best_load) { best_load = r * qb; best_qb = (int)qb; }
-        if (qb == 1) break;
+    int64_t load[9];
+    int64_t best = INT64_MAX;
+    for (int qb = 1; qb <= 8; ++qb) {
+        const int64_t r = (Q + warps * qb - 1) / (warps * qb);      // rounds needed with this batch size
+        load[qb] = r * qb;
+        best = std::min(best, load[qb]);
     }
-    return best_qb;
+    for (int qb = 8; qb >= 1; --qb)
+        if (load[qb] * 100 <= best * 108) return qb;
+    return 1;
 }
 
 TfeFastDiv make_fastdiv(uint32_t d)
