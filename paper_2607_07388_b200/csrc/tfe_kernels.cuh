@@ -62,11 +62,11 @@ struct TfeLookupParams {
 #endif
 };
 
-// Device-resident launch state (uint32 words).  Blocks of a lookup add their miss counts to
-// RUNNING and tick DONE when they finish; the block that finishes last compacts the miss list,
+// Device-resident launch state (uint32 words; DONE and RUNNING form one 8-byte word that a single
+// atomic updates).  Blocks of a lookup add their miss counts to RUNNING and tick DONE when they finish; the block that finishes last compacts the miss list,
 // moves RUNNING to TOTAL and zeroes RUNNING / DONE for the next launch.  Because nothing of this
 // lives in kernel parameters, a launch can be replayed unchanged.
-enum { TFE_CTR_RUNNING = 0, TFE_CTR_TOTAL = 1, TFE_CTR_STATUS = 2, TFE_CTR_DONE = 3, TFE_CTR_WORDS = 4 };
+enum { TFE_CTR_DONE = 0, TFE_CTR_RUNNING = 1, TFE_CTR_TOTAL = 2, TFE_CTR_STATUS = 3, TFE_CTR_WORDS = 4 };
 
 // -------------------------------------------------------------- small helpers
 
@@ -222,7 +222,7 @@ __device__ __forceinline__ void load_memory(const uint4 *const (&rowp)[ALL ? 4 :
 
 // End of a lookup block.  Every thread has recorded flag bytes (and phrase ids of misses) in the
 // context scratch arrays; `my_miss` is warp-uniform.  Blocks add their miss counts to RUNNING and
-// tick DONE; the block that finishes last turns the flag bytes into the ordered miss list
+// tick DONE (one 64-bit atomic); the block that finishes last turns the flag bytes into the ordered miss list
 // (ascending entry index = ascending (q, order)), publishes TOTAL and re-arms the counters.
 __device__ __forceinline__ void tfe_finish_block(const TfeLookupParams &p, uint32_t my_miss, int cols)
 {
@@ -237,18 +237,16 @@ __device__ __forceinline__ void tfe_finish_block(const TfeLookupParams &p, uint3
     if (lane == 0 && my_miss) atomicAdd(&s_miss, my_miss);
     __syncthreads();
     if (threadIdx.x == 0) {
-        if (s_miss) atomicAdd(&p.counters[TFE_CTR_RUNNING], s_miss);
-        __threadfence();
-        s_last = atomicAdd(&p.counters[TFE_CTR_DONE], 1u) == gridDim.x - 1;
+        // one atomic carries both: blocks done (low word) and misses so far (high word)
+        const unsigned long long before = atomicAdd(
+            reinterpret_cast<unsigned long long *>(&p.counters[TFE_CTR_DONE]), ((unsigned long long)s_miss << 32) | 1ull);
+        s_last = (uint32_t)before == gridDim.x - 1;
+        s_total = (uint32_t)(before >> 32) + s_miss;
+        s_scan = 0;
     }
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    if (threadIdx.x == 0) {
-        s_total = *(volatile uint32_t *)&p.counters[TFE_CTR_RUNNING];
-        s_scan = 0;
-    }
-    __syncthreads();
     const uint32_t total = s_total;
     if (total != 0) {
         // order-stable compaction: every thread takes 16 consecutive flag bytes per round
@@ -301,8 +299,8 @@ __device__ __forceinline__ void tfe_finish_block(const TfeLookupParams &p, uint3
     }
     if (threadIdx.x == 0) {
         p.counters[TFE_CTR_TOTAL] = total;
-        p.counters[TFE_CTR_RUNNING] = 0;
         p.counters[TFE_CTR_DONE] = 0;
+        p.counters[TFE_CTR_RUNNING] = 0;
     }
 }
 
