@@ -18,6 +18,7 @@
  *   - gated residual injection  h'_t = h_t + g_t * m_t        [Sec. 2.2 injection eq.]
  *   - list of matched-but-not-GPU-resident phrases            [Sec. 4.3, staged / asynchronous reads]
  *   - insertion of fetched entries into the GPU tier          [Sec. 4.3, "inserts the entry into a faster tier"]
+ *   - prefetch candidates from predicted tokens + priority     [Sec. 4.4, candidate set Q_t, score s = p r c]
  *
  * Parity pins: every function here is pinned by tests that do not call it to
  * produce their expected values (hand-made cases, closed forms, a library
@@ -403,4 +404,79 @@ int32_t orc_cache_install(int64_t N, int64_t C, int32_t d,
         slot_owner[dst[k]] = (int64_t)ids[k];
     }
     return 0;
+}
+
+/* ------------------------------------------- prefetch candidates + priority */
+
+/* Early-exit guided prefetching, the part after the top-K tokens are known [Sec. 4.4]: each
+ * predicted next token cand[b][k] (probability prob[b][k]) is combined with the recent history of
+ * its sequence into the n-grams it would complete -- (history[b][H-n+1 .. H-1], cand[b][k]) for
+ * every configured order n -- and looked up in the phrase table [Sec. 4.4, candidate set Q_t].  A
+ * phrase that is found and is not in the GPU tier is a prefetch candidate with priority
+ *     s = p * r * c          [Sec. 4.4, priority score]
+ * p = prob[b][k], r = usefulness[phrase] (1 if usefulness is NULL), c = benefit of fetching it
+ * from its tier (benefit_host or benefit_ssd; entries already in the GPU tier have no benefit and
+ * are not candidates).  The product is taken in single precision, left to right, because the
+ * ranking is decided by it and the GPU ranks in single precision.  Candidates with s <= 0 are
+ * dropped.  The `budget` candidates of highest priority are returned in descending priority; equal
+ * priorities keep ascending (b, k, order).  Duplicates (one phrase reached from several tokens)
+ * are kept.
+ *
+ * out_src = b*K + k.  Returns the number of candidates before the budget cut; the first
+ * min(budget, that number) output entries are valid.  Uses the sorted phrase order `perm`. */
+typedef struct { float score; uint32_t idx, phrase, src; uint8_t tier; } orc_cand;
+
+static int cand_cmp(const void *pa, const void *pb)
+{
+    const orc_cand *a = (const orc_cand *)pa, *b = (const orc_cand *)pb;
+    if (a->score != b->score) return a->score > b->score ? -1 : 1;
+    return a->idx < b->idx ? -1 : (a->idx > b->idx ? 1 : 0);
+}
+
+int64_t orc_prefetch_candidates(int64_t N, const int32_t *phrase_tokens, const uint8_t *phrase_len,
+                                const int64_t *perm, const int32_t *slot_state,
+                                const int32_t *history, int32_t B, int32_t H,
+                                const int32_t *cand, const float *prob, int32_t K,
+                                int32_t vocab, int32_t n_orders, const int32_t *orders,
+                                const float *usefulness, float benefit_host, float benefit_ssd, int32_t budget,
+                                uint32_t *out_phrase, uint8_t *out_tier, float *out_score, uint32_t *out_src)
+{
+    int64_t cap = (int64_t)B * K * n_orders, n = 0;
+    orc_cand *list = (orc_cand *)malloc(sizeof(orc_cand) * (size_t)(cap > 0 ? cap : 1));
+    for (int32_t b = 0; b < B; ++b)
+        for (int32_t k = 0; k < K; ++k)
+            for (int32_t oi = 0; oi < n_orders; ++oi) {
+                int32_t no = orders[oi], gram[ORC_MAX_ORDERS], ok = no - 1 <= H;
+                for (int32_t j = 0; ok && j < no - 1; ++j) {
+                    gram[j] = history[(int64_t)b * H + (H - (no - 1) + j)];
+                    if (gram[j] < 0 || gram[j] >= vocab) ok = 0;
+                }
+                if (!ok) continue;
+                gram[no - 1] = cand[(int64_t)b * K + k];
+                if (gram[no - 1] < 0 || gram[no - 1] >= vocab) continue;
+                int64_t lo = 0, hi = N;
+                while (lo < hi) {
+                    int64_t mid = lo + (hi - lo) / 2, i = perm[mid];
+                    if (tuple_cmp(phrase_len[i], phrase_tokens + i * 4, no, gram) < 0) lo = mid + 1; else hi = mid;
+                }
+                if (lo >= N || !phrase_equals(phrase_tokens, phrase_len, perm[lo], gram, no)) continue;
+                int64_t id = perm[lo];
+                if (slot_state[id] >= 0) continue;                 /* already in the GPU tier */
+                float c = slot_state[id] == -1 ? benefit_host : benefit_ssd;
+                float r = usefulness ? usefulness[id] : 1.0f;
+                float pr = prob[(int64_t)b * K + k] * r;
+                float s = pr * c;
+                if (!(s > 0.0f)) continue;
+                list[n].score = s; list[n].idx = (uint32_t)(((int64_t)b * K + k) * n_orders + oi);
+                list[n].phrase = (uint32_t)id; list[n].src = (uint32_t)((int64_t)b * K + k);
+                list[n].tier = (uint8_t)(slot_state[id] == -1 ? 2 : 3);
+                ++n;
+            }
+    qsort(list, (size_t)n, sizeof(orc_cand), cand_cmp);
+    for (int64_t i = 0; i < n && i < budget; ++i) {
+        out_phrase[i] = list[i].phrase; out_tier[i] = list[i].tier;
+        out_score[i] = list[i].score; out_src[i] = list[i].src;
+    }
+    free(list);
+    return n;
 }

@@ -59,6 +59,7 @@ def lib() -> C.CDLL:
         _lib.orc_sort_phrases.restype = C.c_int64
         _lib.orc_select.restype = C.c_int64
         _lib.orc_cache_install.restype = C.c_int32
+        _lib.orc_prefetch_candidates.restype = C.c_int64
     return _lib
 
 
@@ -182,3 +183,23 @@ class Oracle:
         return int(lib().orc_cache_install(
             C.c_int64(self.N), C.c_int64(self.C), C.c_int32(self.d), _p(self.slot_state),
             _p(self.slot_owner), _p(self.rows), C.c_int32(len(ids)), _p(ids), _p(src), _p(dst)))
+
+    # -- prefetch candidates + priority ------------------------------------------
+    def prefetch_candidates(self, history, cand, prob, *, usefulness=None, benefit_host=1.0, benefit_ssd=2.0,
+                            budget=4096):
+        """(phrase uint32[n], tier uint8[n], score float32[n], src uint32[n], total candidates)."""
+        history = _c(history, np.int32)
+        cand = _c(cand, np.int32)
+        prob = _c(prob, np.float32)
+        B, H = history.shape
+        K = cand.shape[1]
+        use = None if usefulness is None else _c(usefulness, np.float32)
+        op, ot = np.empty(max(budget, 1), np.uint32), np.empty(max(budget, 1), np.uint8)
+        osc, osr = np.empty(max(budget, 1), np.float32), np.empty(max(budget, 1), np.uint32)
+        total = lib().orc_prefetch_candidates(
+            C.c_int64(self.N), _p(self.phrase_tokens), _p(self.phrase_len), _p(self.sorted_perm()),
+            _p(self.slot_state), _p(history), C.c_int32(B), C.c_int32(H), _p(cand), _p(prob), C.c_int32(K),
+            C.c_int32(self.vocab), C.c_int32(len(self.orders)), _p(self.orders), _p(use),
+            C.c_float(benefit_host), C.c_float(benefit_ssd), C.c_int32(budget), _p(op), _p(ot), _p(osc), _p(osr))
+        n = int(min(total, budget))
+        return op[:n].copy(), ot[:n].copy(), osc[:n].copy(), osr[:n].copy(), int(total)

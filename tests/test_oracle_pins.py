@@ -453,3 +453,92 @@ def test_paper_table_hash_occupancy_fixture():
     # M = B: a fraction 1 - 1/e of the slots is occupied
     M, B, _ = rows[0]
     assert abs(B * (1.0 - (1.0 - 1.0 / B) ** M) / B - (1 - np.exp(-1))) < 1e-6
+
+
+# ------------------------------------------- prefetch candidates + priority
+
+
+def _py_prefetch(phrases, state, history, cand, prob, vocab, orders, use, c_host, c_ssd, budget):
+    """Independent restatement: dict matcher, float32 products, python sort."""
+    table = {tuple(int(x) for x in p): i for i, p in enumerate(phrases)}
+    B, H = history.shape
+    K = cand.shape[1]
+    out = []
+    for b in range(B):
+        for k in range(K):
+            for oi, n in enumerate(orders):
+                if n - 1 > H:
+                    continue
+                g = tuple(int(x) for x in history[b, H - (n - 1):]) + (int(cand[b, k]),) if n > 1 else (int(cand[b, k]),)
+                if not all(0 <= x < vocab for x in g) or g not in table:
+                    continue
+                i = table[g]
+                if state[i] >= 0:
+                    continue
+                c = np.float32(c_host if state[i] == -1 else c_ssd)
+                r = np.float32(1.0 if use is None else use[i])
+                s = np.float32(np.float32(np.float32(prob[b, k]) * r) * c)
+                if not s > 0:
+                    continue
+                out.append((-float(s), (b * K + k) * len(orders) + oi, i, 2 if state[i] == -1 else 3, b * K + k))
+    out.sort()
+    return out[:budget], len(out)
+
+
+def test_prefetch_candidates_by_hand(oracle_mod):
+    # history "... 10 11", predicted next tokens 12 (p=.5), 13 (p=.3), 14 (p=.2)
+    phrases = [(11, 12), (10, 11, 12), (11, 13), (11, 14), (10, 11, 14), (12,)]
+    state = [-2, -1, 0, -1, -2, -1]           # SSD, host, GPU-resident, host, SSD, host
+    o = mk_oracle(oracle_mod, phrases, state, np.zeros((1, 8), np.uint16), 8, 100, [2, 3], 1)
+    hist = np.array([[10, 11]], np.int32)
+    cand = np.array([[12, 13, 14]], np.int32)
+    prob = np.array([[0.5, 0.3, 0.2]], np.float32)
+    use = np.array([1.0, 2.0, 1.0, 4.0, 1.0, 1.0], np.float32)
+    ph, tr, sc, src, total = o.prefetch_candidates(hist, cand, prob, usefulness=use, benefit_host=1.0, benefit_ssd=2.0,
+                                                   budget=10)
+    # (11,12) SSD: .5*1*2 = 1.0 ; (10,11,12) host: .5*2*1 = 1.0 (same priority, later order) ; (11,13) is
+    # GPU-resident: no candidate ; (11,14) host: .2*4*1 = .8 ; (10,11,14) SSD: .2*1*2 = .4 ; (12,) is an
+    # order-1 phrase but order 1 is not configured
+    assert total == 4
+    assert ph.tolist() == [0, 1, 3, 4] and tr.tolist() == [3, 2, 2, 3] and src.tolist() == [0, 0, 2, 2]
+    np.testing.assert_array_equal(sc, np.array([1.0, 1.0, np.float32(0.2) * np.float32(4.0), np.float32(np.float32(0.2) * 1) * 2],
+                                               np.float32))
+    # budget cut keeps the best
+    ph2, _, _, _, total2 = o.prefetch_candidates(hist, cand, prob, usefulness=use, budget=2)
+    assert total2 == 4 and ph2.tolist() == [0, 1]
+    # no usefulness table: r = 1
+    ph3, _, sc3, _, _ = o.prefetch_candidates(hist, cand, prob, budget=10)
+    assert ph3.tolist() == [0, 1, 4, 3]       # 1.0, 0.5, 0.4, 0.2
+    # zero benefit for the host tier drops host-resident candidates
+    ph4, tr4, _, _, total4 = o.prefetch_candidates(hist, cand, prob, benefit_host=0.0, budget=10)
+    assert total4 == 2 and set(tr4.tolist()) == {3}
+
+
+@pytest.mark.parametrize("seed,orders", [(1, [2, 3]), (2, [1, 2, 3, 4]), (3, [3])])
+def test_prefetch_candidates_against_python_restatement(oracle_mod, seed, orders):
+    rng = np.random.default_rng(seed)
+    V = 7
+    phrases = set()
+    target = min(250, sum(V ** n for n in orders) // 2)
+    while len(phrases) < target:
+        n = int(rng.choice(orders))
+        phrases.add(tuple(int(x) for x in rng.integers(0, V, n)))
+    phrases = sorted(phrases, key=lambda p: rng.random())
+    state = rng.choice([-2, -1, 5], size=len(phrases)).astype(np.int32)
+    state[state == 5] = np.arange((state == 5).sum())
+    o = mk_oracle(oracle_mod, phrases, state, np.zeros((len(phrases), 8), np.uint16), 8, V, orders, len(phrases))
+    B, H, K = 6, 3, 9
+    hist = rng.integers(-1, V + 1, size=(B, H)).astype(np.int32)
+    cand = rng.integers(-1, V + 1, size=(B, K)).astype(np.int32)
+    prob = rng.random((B, K)).astype(np.float32)
+    prob[rng.random((B, K)) < 0.2] = np.float32(0.25)       # ties
+    use = rng.choice([0.5, 1.0, 2.0, 0.0], size=len(phrases)).astype(np.float32)
+    for budget in (5, 10_000):
+        ph, tr, sc, src, total = o.prefetch_candidates(hist, cand, prob, usefulness=use, benefit_host=1.0,
+                                                       benefit_ssd=1.5, budget=budget)
+        exp, exp_total = _py_prefetch(phrases, state, hist, cand, prob, V, orders, use, 1.0, 1.5, budget)
+        assert total == exp_total > 5
+        assert ph.tolist() == [e[2] for e in exp]
+        assert tr.tolist() == [e[3] for e in exp]
+        assert src.tolist() == [e[4] for e in exp]
+        np.testing.assert_array_equal(sc, np.array([-e[0] for e in exp], np.float32))
