@@ -56,6 +56,9 @@ def parse_args():
     ap.add_argument("--tune-batch", type=int, default=0, help="queries per warp batch (0: library default)")
     ap.add_argument("--graph-steps", type=int, default=32,
                     help="also time the steps replayed from one CUDA graph of this many launches (0: skip)")
+    ap.add_argument("--prefetch", action="store_true",
+                    help="time tfe_prefetch_candidates (B sequences x top-K tokens) on the workload's table")
+    ap.add_argument("--top-k", type=int, default=64)
     ap.add_argument("--sweep", action="store_true", help="c5: tokens x row width x hit rate sweep")
     ap.add_argument("--sweep-tokens", default="1,4,16,64,256,1024,4096,16384,65536")
     ap.add_argument("--sweep-d", default="1024,2048,4096")
@@ -390,6 +393,8 @@ def run_ours(a):
     L = tfe.lib()
     if a.sweep:
         return run_sweep(a, dev, rank)
+    if a.prefetch:
+        return run_prefetch(a, dev, rank)
 
     w = make_workload(a)
     sampler = ClockSampler(local_rank) if rank == 0 else None
@@ -569,6 +574,72 @@ def run_ours(a):
     if cold_ms is not None:
         line["cold_launch_us"] = cold_ms * 1e3
     print(json.dumps(line))
+
+
+def run_prefetch(a, dev, rank):
+    """Candidate expansion + priority (the step after the early-exit head's top-K) on a decode workload."""
+    import torch
+    from paper_2607_07388_b200 import binding as tfe
+    from oracle import tfe_oracle as orc
+    w = make_workload(a)
+    assert w.shape == "decode", "--prefetch needs a decode workload (c2, c4, c5)"
+    sess = Session(w, dev, 1, a.tune_batch)
+    tb, eng = sess.tb, sess.eng
+    K, B, Hh = a.top_k, w.B, max(w.orders) - 1
+    nbuf = 16
+    rng = np.random.default_rng([w.seed, 31])
+    hists, cands, probs = [], [], []
+    for v in range(nbuf):        # histories copied from the table stream; candidates: the true next token + Zipf filler
+        src = rng.integers(0, tb.safe_len - Hh - 1, size=B)
+        hist = np.stack([tb.stream[s0:s0 + Hh] for s0 in src]).astype(np.int32)
+        cand = synth.zipf_tokens(rng, B * K, synth.zipf_cdf(w.vocab, w.s),
+                                 np.random.default_rng([w.seed, 2]).permutation(w.vocab)).reshape(B, K).astype(np.int32)
+        cand[:, 0] = tb.stream[src + Hh]
+        pr = rng.random((B, K)).astype(np.float32)
+        pr /= pr.sum(axis=1, keepdims=True)
+        hists.append(hist); cands.append(cand); probs.append(pr)
+    t = lambda x: torch.from_numpy(x).to(dev)
+    d_h, d_c, d_p = [t(x) for x in hists], [t(x) for x in cands], [t(x) for x in probs]
+    budget = 4096
+    outs = (torch.empty(budget, dtype=torch.int32, device=dev), torch.empty(budget, dtype=torch.uint8, device=dev),
+            torch.empty(budget, dtype=torch.float32, device=dev), torch.empty(budget, dtype=torch.int32, device=dev),
+            torch.zeros(2, dtype=torch.int32, device=dev))
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        v = i % nbuf
+        tfe.tfe_prefetch_candidates(eng.ctx, d_h[v], B, Hh, d_c[v], d_p[v], K, out_phrase=outs[0], out_tier=outs[1],
+                                    out_score=outs[2], out_src=outs[3], out_count=outs[4], budget=budget,
+                                    benefit_host=1.0, benefit_ssd=2.0, stream=stream)
+
+    step(0)
+    torch.cuda.synchronize()
+    n, total = int(outs[4][0].item()), int(outs[4][1].item())
+    # parity of buffer 0 and the oracle's time
+    orc.build()
+    ora = orc.Oracle(tb.phrase_tokens, tb.phrase_len, tb.init_slot, np.zeros((1, 8), np.uint16), d=8, vocab=w.vocab,
+                     orders=w.orders, gpu_slots=w.gpu_slots)       # rows are not used by this operation
+    ora.sorted_perm()
+    t0 = time.perf_counter()
+    eph, etr, esc, esr, etotal = ora.prefetch_candidates(hists[0], cands[0], probs[0], benefit_host=1.0, benefit_ssd=2.0,
+                                                         budget=budget)
+    cpu_s = time.perf_counter() - t0
+    parity = bool(etotal == total and n == len(eph)
+                  and np.array_equal(outs[0][:n].cpu().numpy().view(np.uint32), eph)
+                  and np.array_equal(outs[2][:n].cpu().numpy().view(np.uint32), esc.view(np.uint32)))
+    ms, _ = timed_region(step, a.steps, max(3, a.warmup), stream, 1, None, dev)
+    us = ms / a.steps * 1e3
+    E = B * K * len(w.orders)
+    if rank == 0:
+        print(json.dumps({"metric": "prefetch candidate expansion probes/s", "value": E / (us * 1e-6), "unit": "probes/s",
+                          "us_per_call": us, "steps": a.steps,
+                          "config": {"workload": w.name, "B": B, "top_k": K, "orders": list(w.orders), "probes": E,
+                                     "n_phrases": w.n_phrases, "budget": budget, "candidates": total, "returned": n},
+                          "index_bytes_per_call": E * 128, "index_gbs": E * 128 / us / 1e3,
+                          "cpu_baseline": {"value": E / cpu_s, "unit": "probes/s", "cores": 1, "kind": "oracle",
+                                           "sample": "one call, single thread"},
+                          "parity": parity}))
+    sess.close()
 
 
 def run_sweep(a, dev, rank):

@@ -205,6 +205,42 @@ tfe_status tfe_lookup_inject_noalloc(tfe_ctx *ctx, const int32_t *tokens, int32_
 tfe_status tfe_miss_list_device(tfe_ctx *ctx, const uint32_t **q_idx, const uint32_t **phrase_id,
                                 const uint8_t **tier, const uint32_t **count);
 
+/* Scoring of prefetch candidates. */
+typedef struct {
+    float   benefit_host;   /* c_i of an entry that sits in host DRAM (>= 0)                           */
+    float   benefit_ssd;    /* c_i of an entry that sits only on SSD (>= 0); GPU-resident entries: 0   */
+    int32_t budget;         /* at most this many candidates are returned, 0..4096                      */
+} tfe_prefetch_params;
+
+/*
+ * tfe_prefetch_candidates -- candidate phrase expansion and priority for early-exit guided
+ * prefetching (paper Sec. 4.4: the top-K predicted tokens "are combined with the recent token
+ * history to infer possible future phrases", mapped through the token-to-phrase index to the
+ * candidate set Q_t; each candidate gets the priority s_i = p_i * r_i * c_i and "high-priority
+ * candidates are prefetched first, while low-priority candidates are dropped when the I/O budget
+ * or queue capacity is exhausted").  The early-exit head itself (projection + top-K) is not part
+ * of this library: its top-K tokens and probabilities are inputs.
+ *
+ *   history      DEVICE int32 [B][H]: the last H tokens of every sequence (H >= n_max - 1 to let
+ *                every order contribute; an order n with n - 1 > H contributes nothing).
+ *   cand_tokens  DEVICE int32 [B][K]: predicted next tokens;  cand_prob DEVICE float [B][K]: p.
+ *   usefulness   DEVICE float [N]: r of every phrase, or NULL for r = 1.
+ *   params       HOST.
+ * For every sequence b, token k and configured order n the n-gram (history[b][H-n+1..H-1],
+ * cand_tokens[b][k]) is looked up; a phrase found outside the GPU tier is a candidate with
+ * s = (p * r) * c in fp32, dropped if s <= 0.  Outputs (DEVICE, `budget` entries each): phrase id,
+ * tier (TFE_FLAG_HOST_MISS / TFE_FLAG_SSD_MISS), s, and source b*K + k of the `budget` best, in
+ * descending s, equal s in ascending (b, k, order); duplicates of one phrase are kept.
+ * out_count DEVICE uint32 [2]: entries written, candidates found before the cut.
+ * Asynchronous on `stream`, two kernel launches; a first call with more entries than any before
+ * grows context buffers.  Errors: INVALID_ARG, CUDA.
+ */
+tfe_status tfe_prefetch_candidates(tfe_ctx *ctx, const int32_t *history, int32_t B, int32_t H,
+                                   const int32_t *cand_tokens, const float *cand_prob, int32_t K,
+                                   const float *usefulness, const tfe_prefetch_params *params,
+                                   uint32_t *out_phrase, uint8_t *out_tier, float *out_score,
+                                   uint32_t *out_src, uint32_t *out_count, void *stream);
+
 /* Frees everything the context owns (not gpu_rows).  NULL is allowed. */
 void tfe_destroy(tfe_ctx *ctx);
 

@@ -31,7 +31,7 @@ NO_PHRASE = 0xFFFFFFFF
 EXPORTS = ["tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
            "tfe_miss_list", "tfe_miss_list_device", "tfe_destroy", "tfe_status_string",
            "tfe_last_cuda_error", "tfe_index_geometry", "tfe_phrase_key64", "tfe_home_bucket",
-           "tfe_launch_geometry", "tfe_set_tuning", "tfe_lookup_inject_noalloc"]
+           "tfe_launch_geometry", "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates"]
 
 
 class TfeConfig(C.Structure):
@@ -43,6 +43,10 @@ class TfeConfig(C.Structure):
 
 class TfeInjectParams(C.Structure):
     _fields_ = [("policy", C.c_int32), ("gate", C.c_int32), ("lam", C.c_float)]
+
+
+class TfePrefetchParams(C.Structure):
+    _fields_ = [("benefit_host", C.c_float), ("benefit_ssd", C.c_float), ("budget", C.c_int32)]
 
 
 class TfeError(RuntimeError):
@@ -73,6 +77,8 @@ def lib() -> C.CDLL:
         L.tfe_lookup_inject_noalloc.argtypes = [vp, vp, i32, i32, i32, vp, vp, C.POINTER(TfeInjectParams), vp, vp, vp,
                                                 vp, vp, vp, vp, vp]
         L.tfe_miss_list.argtypes = [vp, vp, vp, vp, i64, C.POINTER(i64), vp]
+        L.tfe_prefetch_candidates.argtypes = [vp, vp, i32, i32, vp, vp, i32, vp, C.POINTER(TfePrefetchParams),
+                                              vp, vp, vp, vp, vp, vp]
         L.tfe_miss_list_device.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]
         L.tfe_destroy.argtypes = [vp]
         L.tfe_destroy.restype = None
@@ -88,7 +94,7 @@ def lib() -> C.CDLL:
         L.tfe_set_tuning.argtypes = [vp, i32]
         for name in ("tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
                      "tfe_miss_list", "tfe_miss_list_device", "tfe_index_geometry", "tfe_launch_geometry",
-                     "tfe_set_tuning", "tfe_lookup_inject_noalloc"):
+                     "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -188,6 +194,19 @@ def tfe_lookup_inject_noalloc(ctx: int, tokens, B, T, q_start, h, out, *, miss_q
                                            _addr(sel_phrase), _addr(sel_slot), _addr(flags), _addr(miss_q),
                                            _addr(miss_phrase), _addr(miss_tier), _addr(miss_count),
                                            _stream(stream)), "tfe_lookup_inject_noalloc")
+
+
+PREFETCH_MAX_BUDGET = 4096
+
+
+def tfe_prefetch_candidates(ctx: int, history, B, H, cand_tokens, cand_prob, K, *, out_phrase, out_tier, out_score,
+                            out_src, out_count, usefulness=None, benefit_host=1.0, benefit_ssd=2.0, budget=4096,
+                            stream=None) -> None:
+    p = TfePrefetchParams(float(benefit_host), float(benefit_ssd), int(budget))
+    _check(lib().tfe_prefetch_candidates(ctx, _addr(history), B, H, _addr(cand_tokens), _addr(cand_prob), K,
+                                         _addr(usefulness), C.byref(p), _addr(out_phrase), _addr(out_tier),
+                                         _addr(out_score), _addr(out_src), _addr(out_count), _stream(stream)),
+           "tfe_prefetch_candidates")
 
 
 def tfe_miss_list(ctx: int, cap: int, stream=None, allow_overflow=False):

@@ -66,9 +66,6 @@ struct tfe_ctx {
     // resident blocks per SM of each kernel variant
 
     int64_t last_entries = -1;              // Q*cols of the most recent lookup (-1: none yet)
-#ifdef TFE_DBG_TIMELINE
-    long long *dbg = nullptr;
-#endif
     int last_grid = 0, last_block = 0, last_qb = 0;
     int qb_override = 0;                    // 0: choose per call
 
@@ -77,6 +74,13 @@ struct tfe_ctx {
     int32_t *d_inst_slots = nullptr;
     uint4 *d_inst_rows = nullptr;
     int32_t inst_cap = 0;
+
+    // prefetch-candidate scratch
+    unsigned long long *d_pf_keys = nullptr;
+    uint32_t *d_pf_phrase = nullptr;
+    uint8_t *d_pf_tier = nullptr;
+    uint32_t *d_pf_counter = nullptr;
+    int64_t pf_cap = 0;
 
     // host-buffer variant staging
     int32_t *d_h_tokens = nullptr;
@@ -285,6 +289,7 @@ void tfe_destroy(tfe_ctx *c)
     free_dev(c->d_inst_ids); free_dev(c->d_inst_slots); free_dev(c->d_inst_rows);
     free_dev(c->d_h_tokens); free_dev(c->d_h_hidden); free_dev(c->d_h_out);
     free_dev(c->d_h_phrase); free_dev(c->d_h_slot); free_dev(c->d_h_flag);
+    free_dev(c->d_pf_keys); free_dev(c->d_pf_phrase); free_dev(c->d_pf_tier); free_dev(c->d_pf_counter);
     (void)cudaSetDevice(prev);
     delete c;
 }
@@ -419,13 +424,6 @@ tfe_status tfe_index_geometry(const tfe_ctx *c, int64_t *n_buckets, int64_t *ind
     return TFE_OK;
 }
 
-#ifdef TFE_DBG_TIMELINE
-tfe_status tfe_debug_timeline(tfe_ctx *c, void *device_buffer)
-{
-    c->dbg = static_cast<long long *>(device_buffer);
-    return TFE_OK;
-}
-#endif
 
 tfe_status tfe_set_tuning(tfe_ctx *c, int32_t batch_queries)
 {
@@ -552,9 +550,6 @@ tfe_status tfe_lookup_inject(tfe_ctx *c, const int32_t *tokens, int32_t B, int32
     p.scr_phrase = c->d_scr_phrase; p.scr_flag = c->d_scr_flag;
     p.miss_q = c->d_miss_q; p.miss_phrase = c->d_miss_phrase; p.miss_tier = c->d_miss_tier;
     p.counters = c->d_counters;
-#ifdef TFE_DBG_TIMELINE
-    p.dbg = c->dbg;
-#endif
 
     pick_kernel(variant)<<<(unsigned)grid, TFE_BLOCK_THREADS, 0, stream>>>(p);
     CU(cudaGetLastError());
@@ -646,6 +641,59 @@ tfe_status tfe_miss_list_device(tfe_ctx *c, const uint32_t **q_idx, const uint32
     return TFE_OK;
 }
 
+tfe_status tfe_prefetch_candidates(tfe_ctx *c, const int32_t *history, int32_t B, int32_t H,
+                                   const int32_t *cand_tokens, const float *cand_prob, int32_t K,
+                                   const float *usefulness, const tfe_prefetch_params *prm,
+                                   uint32_t *out_phrase, uint8_t *out_tier, float *out_score, uint32_t *out_src,
+                                   uint32_t *out_count, void *stream_)
+{
+    if (!c || !prm || B < 0 || H < 0 || K < 0) return TFE_ERR_INVALID_ARG;
+    if (prm->budget < 0 || prm->budget > TFE_PREFETCH_MAX_BUDGET) return TFE_ERR_INVALID_ARG;
+    if (!(prm->benefit_host >= 0.f) || !(prm->benefit_ssd >= 0.f)) return TFE_ERR_INVALID_ARG;
+    if (!out_count || (prm->budget > 0 && (!out_phrase || !out_tier || !out_score || !out_src)))
+        return TFE_ERR_INVALID_ARG;
+    const int64_t E = (int64_t)B * K * c->cfg.n_orders;
+    if (E > 0x7FFFFFFFll) return TFE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (E == 0) {
+        CU(cudaMemsetAsync(out_count, 0, 2 * sizeof(uint32_t), stream));
+        return TFE_OK;
+    }
+    if (!cand_tokens || !cand_prob || (H > 0 && !history)) return TFE_ERR_INVALID_ARG;
+    if (E > c->pf_cap) {        // grows outside the steady state
+        CU(cudaDeviceSynchronize());
+        free_dev(c->d_pf_keys); free_dev(c->d_pf_phrase); free_dev(c->d_pf_tier);
+        c->d_pf_keys = nullptr; c->d_pf_phrase = nullptr; c->d_pf_tier = nullptr;
+        c->pf_cap = 0;
+        const int64_t cap = std::max<int64_t>(E, 4096);
+        CU(cudaMalloc(&c->d_pf_keys, (size_t)cap * 8));
+        CU(cudaMalloc(&c->d_pf_phrase, (size_t)cap * 4));
+        CU(cudaMalloc(&c->d_pf_tier, (size_t)cap));
+        if (!c->d_pf_counter) {
+            CU(cudaMalloc(&c->d_pf_counter, sizeof(uint32_t)));
+            CU(cudaMemset(c->d_pf_counter, 0, sizeof(uint32_t)));
+        }
+        c->pf_cap = cap;
+    }
+    TfePrefetchParams p{};
+    p.history = history; p.cand = cand_tokens; p.prob = cand_prob; p.usefulness = usefulness;
+    p.B = B; p.H = H; p.K = K; p.n_entries = (uint32_t)E;
+    p.div_orders = make_fastdiv((uint32_t)c->cfg.n_orders); p.div_k = make_fastdiv((uint32_t)K);
+    p.index = c->d_index; p.n_buckets = c->n_buckets; p.phrase_tokens = c->d_phrase_tokens;
+    p.n_orders = c->cfg.n_orders;
+    for (int i = 0; i < 4; ++i) p.orders[i] = i < c->cfg.n_orders ? c->cfg.orders[i] : 0;
+    p.tok_bits = c->tok_bits; p.vocab = c->cfg.vocab;
+    p.benefit_host = prm->benefit_host; p.benefit_ssd = prm->benefit_ssd;
+    p.keys = c->d_pf_keys; p.entry_phrase = c->d_pf_phrase; p.entry_tier = c->d_pf_tier; p.counter = c->d_pf_counter;
+    tfe_prefetch_probe_kernel<<<(unsigned)((E + 255) / 256), 256, 0, stream>>>(p);
+    CU(cudaGetLastError());
+    tfe_prefetch_select_kernel<<<1, 1024, 0, stream>>>(c->d_pf_keys, c->d_pf_phrase, c->d_pf_tier, c->d_pf_counter,
+                                                       (uint32_t)prm->budget, p.div_orders, (uint32_t)c->cfg.n_orders,
+                                                       out_phrase, out_tier, out_score, out_src, out_count);
+    CU(cudaGetLastError());
+    return TFE_OK;
+}
+
 }  // extern "C"
 
 // ---------------------------------------------------------------------------------------------
@@ -734,9 +782,6 @@ extern "C" tfe_status tfe_lookup_inject_noalloc(tfe_ctx *c, const int32_t *token
     p.scr_flag = scratch + TFE_NOALLOC_COUNTER_BYTES + (size_t)TFE_NOALLOC_MAX_ENTRIES * 4;
     p.miss_q = miss_q; p.miss_phrase = miss_phrase; p.miss_tier = miss_tier;
     p.counters = counters;
-#ifdef TFE_DBG_TIMELINE
-    p.dbg = c->dbg;
-#endif
     pick_kernel(variant)<<<(unsigned)grid, TFE_BLOCK_THREADS, 0, stream>>>(p);
     CU(cudaGetLastError());
     CU(cudaMemcpyAsync(miss_count, counters + TFE_CTR_TOTAL, sizeof(uint32_t), cudaMemcpyDeviceToDevice, stream));

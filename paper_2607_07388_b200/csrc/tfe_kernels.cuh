@@ -57,9 +57,6 @@ struct TfeLookupParams {
     uint32_t *miss_q, *miss_phrase; // context miss list, [Q*cols]
     uint8_t *miss_tier;
     uint32_t *counters;             // TFE_CTR_* words
-#ifdef TFE_DBG_TIMELINE
-    long long *dbg;                 // [warps][8] clock stamps
-#endif
 };
 
 // Device-resident launch state (uint32 words; DONE and RUNNING form one 8-byte word that a single
@@ -313,7 +310,6 @@ __device__ __forceinline__ unsigned long long tfe_probe_lane(const TfeLookupPara
                                                              int my_order, bool my_hashed)
 {
     unsigned long long found = TFE_NONE64;
-#ifndef TFE_DBG_NO_PROBE
     if (mine && my_order > 0) {
         const uint32_t b = tfe_div(q, p.div_tq);
         const int32_t t = p.q_start + (int32_t)(q - b * (uint32_t)p.Tq);
@@ -349,7 +345,6 @@ __device__ __forceinline__ unsigned long long tfe_probe_lane(const TfeLookupPara
             }
         }
     }
-#endif
     return found;
 }
 
@@ -427,12 +422,6 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
     const uint32_t qb = p.qb;
     const uint32_t n_batches = (p.Q + qb - 1) / qb;
     uint32_t my_miss = 0;                        // per thread here; summed per warp below
-#ifdef TFE_DBG_TIMELINE
-    long long *dbg = p.dbg + (size_t)(blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5)) * 16;
-    if (lane == 0) { dbg[0] = clock64(); unsigned sm; asm("mov.u32 %0, %%smid;" : "=r"(sm)); dbg[15] = sm;
-        unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); dbg[14] = (long long)gt; }
-    int dbg_round = 0;
-#endif
 
     const uint32_t n_warps = gridDim.x * TFE_WARPS_PER_BLOCK;
     for (uint32_t batch = blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5); batch < n_batches; batch += n_warps) {
@@ -473,16 +462,10 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
             }
         }
 
-#ifdef TFE_DBG_TIMELINE
-        if (lane == 0 && dbg_round < 2) dbg[1 + 6 * dbg_round] = clock64();
-#endif
         // ================================ gather phase ===============================
         for (uint32_t lq = 0; lq < qb; ++lq) {
             const uint32_t gq = q0 + lq;
             if (gq >= p.Q) break;
-#ifdef TFE_DBG_NO_GATHER
-            break;
-#endif
             const char *hrow = reinterpret_cast<const char *>(p.h) + (size_t)gq * hid_row_bytes;
             char *orow = reinterpret_cast<char *>(p.out) + (size_t)gq * hid_row_bytes;
             // rows to add: held by the lanes of quad lq
@@ -575,20 +558,10 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
                 }
             }
         }
-#ifdef TFE_DBG_TIMELINE
-        if (lane == 0 && dbg_round < 2) dbg[2 + 6 * dbg_round] = clock64();
-        ++dbg_round;
-#endif
     }
 
-#ifdef TFE_DBG_TIMELINE
-    if (lane == 0) dbg[10] = clock64();
-#endif
     my_miss = __reduce_add_sync(0xFFFFFFFFu, my_miss);
     tfe_finish_block(p, my_miss, cols);
-#ifdef TFE_DBG_TIMELINE
-    if (lane == 0) dbg[11] = clock64();
-#endif
 }
 
 // ------------------------------------- the hot path, LONGEST / CONST version
@@ -667,7 +640,6 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
             if (j < my_order && tk[j] < 0) ok = false;
         unsigned long long found = TFE_NONE64;
         int4 tuple = make_int4(0, 0, 0, 0);
-#ifndef TFE_DBG_NO_PROBE
         if (ok) {
             const uint64_t key = tfe_make_key(my_order, tk, p.tok_bits);
             const uint64_t b1 = tfe_home_bucket_of(key, p.n_buckets);
@@ -684,7 +656,6 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
             }
             if (my_hashed && found != TFE_NONE64) tuple = __ldg(p.phrase_tokens + (uint32_t)(found >> 32));
         }
-#endif
         __syncwarp();
         const int32_t guess = choose(found);     // selection on key matches, tuples not yet compared
 
@@ -706,9 +677,7 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
             }
         };
         const int32_t guess0 = __shfl_sync(0xFFFFFFFFu, guess, 0);
-#ifndef TFE_DBG_NO_GATHER
         issue_first(0, guess0);
-#endif
 
         // ---- the tuples have arrived by now: final selection, tier walk, record
         if (my_hashed && found != TFE_NONE64 && !tuple_matches(tuple, tk, my_order)) found = TFE_NONE64;
@@ -719,9 +688,6 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
         for (uint32_t lq = 0; lq < qb; ++lq) {
             const uint32_t gq = batch + lq * n_batches;
             if (gq >= p.Q) break;
-#ifdef TFE_DBG_NO_GATHER
-            break;
-#endif
             const int32_t sl = __shfl_sync(0xFFFFFFFFu, my_slot, 4 * lq);
             if (lq > 0 || redo_first) issue_first(lq, sl);
             if (sl < 0 && in_place) continue;    // nothing to add and nothing to copy
@@ -795,3 +761,185 @@ tfe_install_kernel(ulonglong2 *index, const uint32_t *phrase_pos, uint32_t *slot
     uint4 *o = rows + (size_t)dst * row_vecs;
     for (int i = lane; i < row_vecs; i += 32) o[i] = ld_stream(s + i);
 }
+
+// ------------------------------------------- prefetch candidates + priority
+//
+// Early-exit guided prefetching after the top-K tokens are known: every predicted next token is
+// combined with the recent history of its sequence into the n-grams it would complete, those are
+// looked up with the same probe as above, and every phrase found outside the GPU tier becomes a
+// candidate with priority s = p * r * c (token probability, usefulness of the entry, benefit of
+// fetching it from its tier).  The `budget` best are returned in descending priority.
+//
+//   tfe_prefetch_probe_kernel   one thread per (sequence, token, order): probe, score, append
+//                               {priority, entry index} as one 64-bit key to a compact list
+//   tfe_prefetch_select_kernel  one block: radix-select the budget-th largest key, gather the keys at
+//                               or above it in shared memory, bitonic sort, write the result
+// The priority is a non-negative fp32 number, so its bit pattern orders like its value; the low
+// word of a key is ~index, so a descending key sort is descending priority with ascending
+// (sequence, token, order) among equals, and keys are unique.
+#define TFE_PREFETCH_MAX_BUDGET 4096
+
+struct TfePrefetchParams {
+    const int32_t *history;         // [B][H]
+    const int32_t *cand;            // [B][K]
+    const float *prob;              // [B][K]
+    const float *usefulness;        // [N] or nullptr (= 1)
+    int32_t B, H, K;
+    uint32_t n_entries;             // B * K * n_orders
+    TfeFastDiv div_orders, div_k;
+    const ulonglong2 *index;
+    uint64_t n_buckets;
+    const int4 *phrase_tokens;
+    int32_t n_orders, orders[4], tok_bits, vocab;
+    float benefit_host, benefit_ssd;
+    unsigned long long *keys;       // [n_entries] compact candidate list
+    uint32_t *entry_phrase;         // [n_entries] by entry index
+    uint8_t *entry_tier;
+    uint32_t *counter;              // number of candidates (reset by the select kernel)
+};
+
+__global__ void __launch_bounds__(256) tfe_prefetch_probe_kernel(const TfePrefetchParams p)
+{
+    const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = threadIdx.x & 31;
+    unsigned long long key64 = 0;
+    if (idx < p.n_entries) {
+        const uint32_t bk = tfe_div(idx, p.div_orders);
+        const int oi = (int)(idx - bk * (uint32_t)p.n_orders);
+        const uint32_t b = tfe_div(bk, p.div_k);
+        const int n = p.orders[oi];
+        int32_t tk[4] = {-1, -1, -1, -1};
+        bool ok = n - 1 <= p.H;
+        if (ok) {
+            tk[0] = __ldg(p.cand + bk);
+#pragma unroll
+            for (int j = 1; j < 4; ++j)
+                if (j < n) tk[j] = __ldg(p.history + (size_t)b * p.H + (p.H - j));
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (j < n && (uint32_t)tk[j] >= (uint32_t)p.vocab) ok = false;
+        }
+        if (ok) {
+            const uint64_t key = tfe_make_key(n, tk, p.tok_bits);
+            const uint64_t b1 = tfe_home_bucket_of(key, p.n_buckets);
+            const uint64_t b2 = tfe_second_bucket_of(key, b1, p.n_buckets);
+            const ulonglong4 *p1 = reinterpret_cast<const ulonglong4 *>(p.index + b1 * TFE_SLOTS_PER_BUCKET);
+            const ulonglong4 *p2 = reinterpret_cast<const ulonglong4 *>(p.index + b2 * TFE_SLOTS_PER_BUCKET);
+            ulonglong4 w[4];
+            w[0] = ld_bucket32(p1); w[1] = ld_bucket32(p1 + 1);
+            w[2] = ld_bucket32(p2); w[3] = ld_bucket32(p2 + 1);
+            unsigned long long found = TFE_NONE64;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (w[k].x == key) found = w[k].y;
+                if (w[k].z == key) found = w[k].w;
+            }
+            if (found != TFE_NONE64 && !tfe_order_is_packed(n, p.tok_bits)) {
+                const int4 st = __ldg(p.phrase_tokens + (uint32_t)(found >> 32));
+                if (!tuple_matches(st, tk, n)) found = TFE_NONE64;
+            }
+            const int32_t state = (int32_t)(uint32_t)found;
+            if (found != TFE_NONE64 && state < 0) {          // a phrase, and not in the GPU tier
+                const uint32_t phrase = (uint32_t)(found >> 32);
+                const float c = state == -1 ? p.benefit_host : p.benefit_ssd;
+                const float r = p.usefulness ? __ldg(p.usefulness + phrase) : 1.f;
+                const float s = __fmul_rn(__fmul_rn(__ldg(p.prob + bk), r), c);
+                if (s > 0.f) {
+                    key64 = ((unsigned long long)__float_as_uint(s) << 32) | (0xFFFFFFFFu - idx);
+                    p.entry_phrase[idx] = phrase;
+                    p.entry_tier[idx] = state == -1 ? 2 : 3;
+                }
+            }
+        }
+    }
+    // append: one atomic per warp
+    const uint32_t has = __ballot_sync(0xFFFFFFFFu, key64 != 0);
+    if (has) {
+        uint32_t base = 0;
+        if (lane == __ffs(has) - 1) base = atomicAdd(p.counter, __popc(has));
+        base = __shfl_sync(0xFFFFFFFFu, base, __ffs(has) - 1);
+        if (key64 != 0) p.keys[base + __popc(has & ((1u << lane) - 1u))] = key64;
+    }
+}
+
+__global__ void __launch_bounds__(1024)
+tfe_prefetch_select_kernel(const unsigned long long *keys, const uint32_t *entry_phrase, const uint8_t *entry_tier,
+                           uint32_t *counter, uint32_t budget, TfeFastDiv div_orders, uint32_t n_orders,
+                           uint32_t *out_phrase, uint8_t *out_tier, float *out_score, uint32_t *out_src,
+                           uint32_t *out_count)
+{
+    __shared__ unsigned long long s_keys[TFE_PREFETCH_MAX_BUDGET];
+    __shared__ uint32_t s_hist[256];
+    __shared__ uint32_t s_fill;
+    __shared__ unsigned long long s_prefix;
+    __shared__ uint32_t s_want;
+    const uint32_t n = *(volatile uint32_t *)counter;
+    const uint32_t take = min(n, budget);
+    // ---- threshold: the take-th largest key, by most-significant-digit-first radix selection
+    unsigned long long thresh = 0;
+    if (n > take) {
+        if (threadIdx.x == 0) { s_prefix = 0; s_want = take; }
+        __syncthreads();
+        for (int shift = 56; shift >= 0; shift -= 8) {
+            if (threadIdx.x < 256) s_hist[threadIdx.x] = 0;
+            __syncthreads();
+            const unsigned long long prefix = s_prefix;
+            const unsigned long long mask = shift == 56 ? 0ull : ~0ull << (shift + 8);
+            for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) {
+                const unsigned long long k = keys[i];
+                if ((k & mask) == prefix) atomicAdd(&s_hist[(k >> shift) & 0xFFu], 1u);
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                uint32_t want = s_want, d = 255;
+                for (;; --d) {               // digits from the top until `want` keys are covered
+                    if (s_hist[d] >= want) break;
+                    want -= s_hist[d];
+                    if (d == 0) break;
+                }
+                s_want = want;
+                s_prefix = prefix | ((unsigned long long)d << shift);
+            }
+            __syncthreads();
+        }
+        thresh = s_prefix;
+    }
+    // ---- gather the keys at or above the threshold (exactly `take`: keys are unique), pad, sort
+    uint32_t pow2 = 1;
+    while (pow2 < take) pow2 <<= 1;
+    if (threadIdx.x == 0) s_fill = 0;
+    for (uint32_t i = threadIdx.x; i < pow2; i += blockDim.x) s_keys[i] = 0;
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) {
+        const unsigned long long k = keys[i];
+        if (k >= thresh) s_keys[atomicAdd(&s_fill, 1u)] = k;
+    }
+    __syncthreads();
+    for (uint32_t size = 2; size <= pow2; size <<= 1)
+        for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
+            for (uint32_t i = threadIdx.x; i < pow2 / 2; i += blockDim.x) {
+                const uint32_t lo = 2 * i - (i & (stride - 1));       // pairs (lo, lo + stride)
+                const uint32_t hi = lo + stride;
+                const bool descending = (lo & size) == 0;
+                const unsigned long long a = s_keys[lo], b = s_keys[hi];
+                if ((a < b) == descending) { s_keys[lo] = b; s_keys[hi] = a; }
+            }
+            __syncthreads();
+        }
+    for (uint32_t i = threadIdx.x; i < take; i += blockDim.x) {
+        const unsigned long long k = s_keys[i];
+        const uint32_t idx = 0xFFFFFFFFu - (uint32_t)k;
+        out_phrase[i] = entry_phrase[idx];
+        out_tier[i] = entry_tier[idx];
+        out_score[i] = __uint_as_float((uint32_t)(k >> 32));
+        out_src[i] = tfe_div(idx, div_orders);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        out_count[0] = take;
+        out_count[1] = n;
+        *counter = 0;                        // ready for the next call
+    }
+    (void)n_orders;
+}
+

@@ -72,6 +72,23 @@ class Engram:
             cap = 1 << 20
         return tfe.tfe_miss_list(self.ctx, cap, stream, allow_overflow)
 
+    def prefetch_candidates(self, history: torch.Tensor, cand_tokens: torch.Tensor, cand_prob: torch.Tensor, *,
+                            usefulness: torch.Tensor | None = None, benefit_host=1.0, benefit_ssd=2.0, budget=4096,
+                            stream=None):
+        """(phrase, tier, score, src, [written, found]) device tensors of the `budget` best candidates."""
+        B, H = history.shape
+        K = cand_tokens.shape[1]
+        dev = cand_tokens.device
+        ph = torch.empty(max(budget, 1), dtype=torch.int32, device=dev)
+        tr = torch.empty(max(budget, 1), dtype=torch.uint8, device=dev)
+        sc = torch.empty(max(budget, 1), dtype=torch.float32, device=dev)
+        sr = torch.empty(max(budget, 1), dtype=torch.int32, device=dev)
+        cnt = torch.zeros(2, dtype=torch.int32, device=dev)
+        tfe.tfe_prefetch_candidates(self.ctx, history, B, H, cand_tokens, cand_prob, K, out_phrase=ph, out_tier=tr,
+                                    out_score=sc, out_src=sr, out_count=cnt, usefulness=usefulness,
+                                    benefit_host=benefit_host, benefit_ssd=benefit_ssd, budget=budget, stream=stream)
+        return ph, tr, sc, sr, cnt
+
     def cache_install(self, phrase_ids, src_rows, dst_slots, stream=None):
         tfe.tfe_cache_install(self.ctx, phrase_ids, src_rows, dst_slots, stream)
 
