@@ -144,9 +144,19 @@ tfe_status tfe_lookup_inject(tfe_ctx *ctx, const int32_t *tokens, int32_t B, int
 
 /*
  * tfe_lookup_inject_host -- the same call for HOST buffers (tokens, h, out and the optional
- * result arrays all in host memory, pinned for asynchronous copies): copies the inputs to
- * context-owned device buffers, runs the kernel, copies the results back, all on `stream`,
- * without synchronising.  The buffers must stay valid until the stream has passed the call.
+ * result arrays all in host memory; pinned memory lets the copies run asynchronously and
+ * overlap): copies the inputs to context-owned device buffers, runs the kernel, copies the
+ * results back, without synchronising the host.  Everything is ordered after the work already
+ * queued on `stream`, and `stream` continues only when the last result byte is in host memory,
+ * so the caller sees the call as one operation on `stream`.  The buffers must stay valid until
+ * the stream has passed the call.
+ *
+ * LONGEST / CONST calls with at least 16 MiB of hidden state are issued in pieces (query ranges;
+ * up to 32, small at both ends, up to 8 MiB in the middle) through two context-owned copy
+ * streams, so that one piece's kernel runs while the next piece comes in and the previous one
+ * goes back; the last piece's launch builds the miss list of the whole call.  Results are the
+ * same as for the single launch.  Other variants copy, launch once and copy back on `stream`.
+ * The first piecewise call on a context creates the two streams and their events.
  */
 tfe_status tfe_lookup_inject_host(tfe_ctx *ctx, const int32_t *tokens, int32_t B, int32_t T,
                                   int32_t q_start, const void *h, void *out,

@@ -89,6 +89,11 @@ struct tfe_ctx {
     int32_t *d_h_slot = nullptr;
     uint8_t *d_h_flag = nullptr;
     int64_t hb_tok_cap = 0, hb_q_cap = 0, hb_ent_cap = 0;
+    // copy streams and events of the host-buffer variant's pipeline (created on its first call)
+    enum { kPipeMaxChunks = 32 };
+    cudaStream_t hb_in = nullptr, hb_out = nullptr;
+    cudaEvent_t hb_ev_start = nullptr, hb_ev_done = nullptr;
+    cudaEvent_t hb_ev_in[kPipeMaxChunks] = {}, hb_ev_k[kPipeMaxChunks] = {};
 };
 
 namespace {
@@ -97,8 +102,9 @@ typedef void (*lookup_kernel_t)(const TfeLookupParams);
 
 // Kernel variants.  0..7: hidden dtype x policy x gate, the general kernel in fp32 arithmetic.
 // 8..10: the LONGEST / CONST kernel -- bf16 hidden in fp32 arithmetic, bf16 hidden with the
-// packed bf16 fused multiply-add (lambda exactly a bf16 number), fp32 hidden.
-enum { kVarLongest = 8, kVarLongestPacked = 9, kVarLongestF32 = 10, kVarCount = 11 };
+// packed bf16 fused multiply-add (lambda exactly a bf16 number), fp32 hidden.  11..13: the same
+// three for a call issued in several launches over query ranges (variant + kVarRanged).
+enum { kVarLongest = 8, kVarLongestPacked = 9, kVarLongestF32 = 10, kVarRanged = 3, kVarCount = 14 };
 
 lookup_kernel_t pick_kernel(int variant)
 {
@@ -107,8 +113,10 @@ lookup_kernel_t pick_kernel(int variant)
         tfe_lookup_inject_kernel<0, true, false, false>,  tfe_lookup_inject_kernel<0, true, true, false>,
         tfe_lookup_inject_kernel<1, false, false, false>, tfe_lookup_inject_kernel<1, false, true, false>,
         tfe_lookup_inject_kernel<1, true, false, false>,  tfe_lookup_inject_kernel<1, true, true, false>,
-        tfe_lookup_inject_longest_kernel<0, false>, tfe_lookup_inject_longest_kernel<0, true>,
-        tfe_lookup_inject_longest_kernel<1, false>,
+        tfe_lookup_inject_longest_kernel<0, false, false>, tfe_lookup_inject_longest_kernel<0, true, false>,
+        tfe_lookup_inject_longest_kernel<1, false, false>,
+        tfe_lookup_inject_longest_kernel<0, false, true>,  tfe_lookup_inject_longest_kernel<0, true, true>,
+        tfe_lookup_inject_longest_kernel<1, false, true>,
     };
     return table[variant];
 }
@@ -290,6 +298,14 @@ void tfe_destroy(tfe_ctx *c)
     free_dev(c->d_h_tokens); free_dev(c->d_h_hidden); free_dev(c->d_h_out);
     free_dev(c->d_h_phrase); free_dev(c->d_h_slot); free_dev(c->d_h_flag);
     free_dev(c->d_pf_keys); free_dev(c->d_pf_phrase); free_dev(c->d_pf_tier); free_dev(c->d_pf_counter);
+    if (c->hb_in) (void)cudaStreamDestroy(c->hb_in);
+    if (c->hb_out) (void)cudaStreamDestroy(c->hb_out);
+    if (c->hb_ev_start) (void)cudaEventDestroy(c->hb_ev_start);
+    if (c->hb_ev_done) (void)cudaEventDestroy(c->hb_ev_done);
+    for (int k = 0; k < tfe_ctx::kPipeMaxChunks; ++k) {
+        if (c->hb_ev_in[k]) (void)cudaEventDestroy(c->hb_ev_in[k]);
+        if (c->hb_ev_k[k]) (void)cudaEventDestroy(c->hb_ev_k[k]);
+    }
     (void)cudaSetDevice(prev);
     delete c;
 }
@@ -502,6 +518,64 @@ tfe_status tfe_cache_install(tfe_ctx *c, int32_t n, const uint32_t *phrase_ids, 
     return TFE_OK;
 }
 
+// Bytes of hidden state per piece of the host-buffer variant's copy / compute pipeline: the
+// largest piece, and the smallest (the last ones).
+#ifndef TFE_HOST_CHUNK_BYTES
+#define TFE_HOST_CHUNK_BYTES ((size_t)8 << 20)
+#endif
+#ifndef TFE_HOST_TAIL_BYTES
+#define TFE_HOST_TAIL_BYTES ((size_t)1 << 20)       // the last two pieces; earlier ones double up to the above
+#endif
+
+namespace {
+
+// Variant of the lookup kernel a call runs: the LONGEST / CONST kernels where they apply.
+int lookup_variant(const tfe_ctx *c, const tfe_inject_params *prm)
+{
+    const bool all = prm->policy == TFE_POLICY_ALL, cos = prm->gate == TFE_GATE_COSINE;
+    uint32_t lam_bits;
+    std::memcpy(&lam_bits, &prm->lambda, sizeof lam_bits);
+    const bool lam_is_bf16 = (lam_bits & 0xFFFFu) == 0 && (lam_bits & 0x7F800000u) != 0x7F800000u;
+    const int ht = c->cfg.hidden_dtype;
+    return (all || cos) ? ht * 4 + (all ? 2 : 0) + (cos ? 1 : 0)
+                        : (ht == 1 ? kVarLongestF32 : (lam_is_bf16 ? kVarLongestPacked : kVarLongest));
+}
+
+tfe_status lookup_inject_range(tfe_ctx *c, const int32_t *tokens, int32_t B, int32_t T, int32_t q_start,
+                               const void *h, void *out, const tfe_inject_params *prm,
+                               uint32_t *sel_phrase, int32_t *sel_slot, uint8_t *flags, cudaStream_t stream,
+                               int64_t q_lo, int64_t q_hi, bool finalize);
+
+// Piece boundaries of the host-buffer pipeline over Q rows: cut[0] = 0 < ... < cut[n] = Q, n returned.
+// The first piece's copy-in and the last piece's kernel and copy-back are the exposed parts, in
+// between both copy engines stay busy; so pieces are small at both ends (tail, tail, 2 tail,
+// 4 tail, ...) and large (few stream hand-overs) in the middle.
+int plan_pieces(int64_t Q, int64_t row_bytes, int64_t *cut)
+{
+    const int max_n = tfe_ctx::kPipeMaxChunks;
+    const int64_t tail = std::max<int64_t>(64, (int64_t)TFE_HOST_TAIL_BYTES / row_bytes / 64 * 64);
+    int64_t big = std::max<int64_t>(tail, (int64_t)TFE_HOST_CHUNK_BYTES / row_bytes / 64 * 64);
+    for (;; big *= 2) {
+        int64_t head[max_n], back[max_n];
+        int nh = 0, nb = 0;
+        int64_t left = Q, next = tail;
+        while (left > 0 && nh + nb < max_n) {
+            const int64_t a = std::min(left, next);
+            head[nh++] = a; left -= a;
+            const int64_t b = std::min(left, next);
+            if (b > 0 && nh + nb < max_n) { back[nb++] = b; left -= b; }
+            if (nh >= 2) next = std::min(big, next * 2);
+        }
+        if (left > 0) continue;         // too many pieces: larger middle pieces
+        for (int k = 0; k < nh; ++k) cut[k + 1] = cut[k] + head[k];
+        for (int k = 0; k < nb; ++k) cut[nh + k + 1] = cut[nh + k] + back[nb - 1 - k];
+        return nh + nb;
+    }
+}
+
+
+}  // namespace
+
 tfe_status tfe_lookup_inject(tfe_ctx *c, const int32_t *tokens, int32_t B, int32_t T, int32_t q_start,
                              const void *h, void *out, const tfe_inject_params *prm,
                              uint32_t *sel_phrase, int32_t *sel_slot, uint8_t *flags, void *stream_)
@@ -524,21 +598,36 @@ tfe_status tfe_lookup_inject(tfe_ctx *c, const int32_t *tokens, int32_t B, int32
         return TFE_ERR_INVALID_ARG;
     tfe_status st = ensure_entries(c, Q * cols);
     if (st != TFE_OK) return st;
+    return lookup_inject_range(c, tokens, B, T, q_start, h, out, prm, sel_phrase, sel_slot, flags, stream, 0, Q, true);
+}
 
-    const bool all = prm->policy == TFE_POLICY_ALL, cos = prm->gate == TFE_GATE_COSINE;
+namespace {
+
+// One launch over queries [q_lo, q_hi) of a call of Q queries.  A call issued in several launches
+// (LONGEST / CONST kernels only) passes finalize on the last one, which builds the miss list of
+// the whole call; the launches must run in order on one stream.
+tfe_status lookup_inject_range(tfe_ctx *c, const int32_t *tokens, int32_t B, int32_t T, int32_t q_start,
+                               const void *h, void *out, const tfe_inject_params *prm,
+                               uint32_t *sel_phrase, int32_t *sel_slot, uint8_t *flags, cudaStream_t stream,
+                               int64_t q_lo, int64_t q_hi, bool finalize)
+{
+    const int64_t Tq = T - q_start, Q = (int64_t)B * Tq;
+    const int cols = prm->policy == TFE_POLICY_ALL ? c->cfg.n_orders : 1;
     uint32_t lam_bits;
     std::memcpy(&lam_bits, &prm->lambda, sizeof lam_bits);
-    const bool lam_is_bf16 = (lam_bits & 0xFFFFu) == 0 && (lam_bits & 0x7F800000u) != 0x7F800000u;
-    const int ht = c->cfg.hidden_dtype;
-    const int variant = (all || cos) ? ht * 4 + (all ? 2 : 0) + (cos ? 1 : 0)
-                                     : (ht == 1 ? kVarLongestF32 : (lam_is_bf16 ? kVarLongestPacked : kVarLongest));
+    const bool ranged = q_lo != 0 || q_hi != Q || !finalize;
+    int variant = lookup_variant(c, prm);
+    if (ranged && variant < kVarLongest) return TFE_ERR_INTERNAL;
+    if (ranged) variant += kVarRanged;
+    const int64_t Qr = q_hi - q_lo;
     const int64_t resident = (int64_t)c->sm_count * c->occ[variant];
-    const int64_t qb = c->qb_override ? c->qb_override : pick_batch(Q, resident * TFE_WARPS_PER_BLOCK);
-    const int64_t n_batches = (Q + qb - 1) / qb;
+    const int64_t qb = c->qb_override ? c->qb_override : pick_batch(Qr, resident * TFE_WARPS_PER_BLOCK);
+    const int64_t n_batches = (Qr + qb - 1) / qb;
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(resident, (n_batches + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK));
     TfeLookupParams p{};
     p.tokens = tokens; p.B = B; p.T = T; p.q_start = q_start; p.Tq = (int32_t)Tq; p.Q = (uint32_t)Q;
     p.div_tq = make_fastdiv((uint32_t)Tq); p.qb = (uint32_t)qb;
+    p.q_lo = (uint32_t)q_lo; p.q_hi = (uint32_t)q_hi; p.finalize = finalize ? 1u : 0u;
     p.index = c->d_index; p.n_buckets = c->n_buckets;
     p.phrase_tokens = c->d_phrase_tokens; p.rows = c->gpu_rows; p.d = c->cfg.d;
     p.h = h; p.out = out;
@@ -560,12 +649,15 @@ tfe_status tfe_lookup_inject(tfe_ctx *c, const int32_t *tokens, int32_t B, int32
     return TFE_OK;
 }
 
+}  // namespace
+
 tfe_status tfe_lookup_inject_host(tfe_ctx *c, const int32_t *tokens, int32_t B, int32_t T, int32_t q_start,
                                   const void *h, void *out, const tfe_inject_params *prm,
                                   uint32_t *sel_phrase, int32_t *sel_slot, uint8_t *flags, void *stream_)
 {
     if (!c || !prm || B < 0 || T < 0 || q_start < 0 || q_start > T) return TFE_ERR_INVALID_ARG;
     if (prm->policy != TFE_POLICY_LONGEST && prm->policy != TFE_POLICY_ALL) return TFE_ERR_INVALID_ARG;
+    if (prm->gate != TFE_GATE_CONST && prm->gate != TFE_GATE_COSINE) return TFE_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const int64_t n_tok = (int64_t)B * T, Q = (int64_t)B * (T - q_start);
     const int cols = prm->policy == TFE_POLICY_ALL ? c->cfg.n_orders : 1;
@@ -591,16 +683,69 @@ tfe_status tfe_lookup_inject_host(tfe_ctx *c, const int32_t *tokens, int32_t B, 
         CU(cudaMalloc(&c->d_h_flag, (size_t)e_cap));
         c->hb_tok_cap = tok_cap; c->hb_q_cap = q_cap; c->hb_ent_cap = e_cap;
     }
-    CU(cudaMemcpyAsync(c->d_h_tokens, tokens, (size_t)n_tok * 4, cudaMemcpyHostToDevice, stream));
-    CU(cudaMemcpyAsync(c->d_h_hidden, h, hid_bytes, cudaMemcpyHostToDevice, stream));
-    tfe_status st = tfe_lookup_inject(c, c->d_h_tokens, B, T, q_start, c->d_h_hidden, c->d_h_out, prm,
-                                      sel_phrase ? c->d_h_phrase : nullptr, sel_slot ? c->d_h_slot : nullptr,
-                                      flags ? c->d_h_flag : nullptr, stream_);
+    const size_t row_bytes = (size_t)c->cfg.d * (c->cfg.hidden_dtype == 0 ? 2 : 4);
+    const int variant = lookup_variant(c, prm);
+    // The LONGEST / CONST kernels can run a call in pieces, so the hidden states go through a
+    // three-stage pipeline: piece k's kernel runs while piece k+1 comes in and piece k-1 goes
+    // back.  Other variants take one launch between the copies.
+    int64_t cut[tfe_ctx::kPipeMaxChunks + 1];
+    int n_chunks = 1;
+    cut[0] = 0; cut[1] = Q;
+    if (variant >= kVarLongest && hid_bytes >= 2 * (size_t)TFE_HOST_CHUNK_BYTES)
+        n_chunks = plan_pieces(Q, (int64_t)row_bytes, cut);
+    if (n_chunks == 1) {
+        CU(cudaMemcpyAsync(c->d_h_tokens, tokens, (size_t)n_tok * 4, cudaMemcpyHostToDevice, stream));
+        CU(cudaMemcpyAsync(c->d_h_hidden, h, hid_bytes, cudaMemcpyHostToDevice, stream));
+        tfe_status st = tfe_lookup_inject(c, c->d_h_tokens, B, T, q_start, c->d_h_hidden, c->d_h_out, prm,
+                                          sel_phrase ? c->d_h_phrase : nullptr, sel_slot ? c->d_h_slot : nullptr,
+                                          flags ? c->d_h_flag : nullptr, stream_);
+        if (st != TFE_OK) return st;
+        CU(cudaMemcpyAsync(out, c->d_h_out, hid_bytes, cudaMemcpyDeviceToHost, stream));
+        if (sel_phrase) CU(cudaMemcpyAsync(sel_phrase, c->d_h_phrase, (size_t)ent * 4, cudaMemcpyDeviceToHost, stream));
+        if (sel_slot) CU(cudaMemcpyAsync(sel_slot, c->d_h_slot, (size_t)ent * 4, cudaMemcpyDeviceToHost, stream));
+        if (flags) CU(cudaMemcpyAsync(flags, c->d_h_flag, (size_t)ent, cudaMemcpyDeviceToHost, stream));
+        return TFE_OK;
+    }
+    if (!c->hb_in) {
+        CU(cudaStreamCreateWithFlags(&c->hb_in, cudaStreamNonBlocking));
+        CU(cudaStreamCreateWithFlags(&c->hb_out, cudaStreamNonBlocking));
+        CU(cudaEventCreateWithFlags(&c->hb_ev_start, cudaEventDisableTiming));
+        CU(cudaEventCreateWithFlags(&c->hb_ev_done, cudaEventDisableTiming));
+        for (int k = 0; k < tfe_ctx::kPipeMaxChunks; ++k) {
+            CU(cudaEventCreateWithFlags(&c->hb_ev_in[k], cudaEventDisableTiming));
+            CU(cudaEventCreateWithFlags(&c->hb_ev_k[k], cudaEventDisableTiming));
+        }
+    }
+    tfe_status st = ensure_entries(c, ent);
     if (st != TFE_OK) return st;
-    CU(cudaMemcpyAsync(out, c->d_h_out, hid_bytes, cudaMemcpyDeviceToHost, stream));
-    if (sel_phrase) CU(cudaMemcpyAsync(sel_phrase, c->d_h_phrase, (size_t)ent * 4, cudaMemcpyDeviceToHost, stream));
-    if (sel_slot) CU(cudaMemcpyAsync(sel_slot, c->d_h_slot, (size_t)ent * 4, cudaMemcpyDeviceToHost, stream));
-    if (flags) CU(cudaMemcpyAsync(flags, c->d_h_flag, (size_t)ent, cudaMemcpyDeviceToHost, stream));
+    // everything the caller queued on its stream comes first (the staging buffers may be in use)
+    CU(cudaEventRecord(c->hb_ev_start, stream));
+    CU(cudaStreamWaitEvent(c->hb_in, c->hb_ev_start, 0));
+    CU(cudaStreamWaitEvent(c->hb_out, c->hb_ev_start, 0));
+    CU(cudaMemcpyAsync(c->d_h_tokens, tokens, (size_t)n_tok * 4, cudaMemcpyHostToDevice, c->hb_in));
+    for (int k = 0; k < n_chunks; ++k) {
+        const int64_t q_lo = cut[k], q_hi = cut[k + 1], nq = q_hi - q_lo;
+        const size_t off = (size_t)q_lo * row_bytes, len = (size_t)nq * row_bytes;
+        CU(cudaMemcpyAsync(static_cast<char *>(c->d_h_hidden) + off, static_cast<const char *>(h) + off, len,
+                           cudaMemcpyHostToDevice, c->hb_in));
+        CU(cudaEventRecord(c->hb_ev_in[k], c->hb_in));
+        CU(cudaStreamWaitEvent(stream, c->hb_ev_in[k], 0));
+        st = lookup_inject_range(c, c->d_h_tokens, B, T, q_start, c->d_h_hidden, c->d_h_out, prm,
+                                 sel_phrase ? c->d_h_phrase : nullptr, sel_slot ? c->d_h_slot : nullptr,
+                                 flags ? c->d_h_flag : nullptr, stream, q_lo, q_hi, q_hi == Q);
+        if (st != TFE_OK) return st;
+        CU(cudaEventRecord(c->hb_ev_k[k], stream));
+        CU(cudaStreamWaitEvent(c->hb_out, c->hb_ev_k[k], 0));
+        CU(cudaMemcpyAsync(static_cast<char *>(out) + off, static_cast<const char *>(c->d_h_out) + off, len,
+                           cudaMemcpyDeviceToHost, c->hb_out));
+        if (sel_phrase) CU(cudaMemcpyAsync(sel_phrase + q_lo, c->d_h_phrase + q_lo, (size_t)nq * 4, cudaMemcpyDeviceToHost, c->hb_out));
+        if (sel_slot) CU(cudaMemcpyAsync(sel_slot + q_lo, c->d_h_slot + q_lo, (size_t)nq * 4, cudaMemcpyDeviceToHost, c->hb_out));
+        if (flags) CU(cudaMemcpyAsync(flags + q_lo, c->d_h_flag + q_lo, (size_t)nq, cudaMemcpyDeviceToHost, c->hb_out));
+    }
+    // the caller's stream resumes once the last piece is back in host memory
+    CU(cudaEventRecord(c->hb_ev_done, c->hb_out));
+    CU(cudaStreamWaitEvent(stream, c->hb_ev_done, 0));
+    c->last_entries = ent;
     return TFE_OK;
 }
 
@@ -770,6 +915,7 @@ extern "C" tfe_status tfe_lookup_inject_noalloc(tfe_ctx *c, const int32_t *token
     TfeLookupParams p{};
     p.tokens = tokens; p.B = B; p.T = T; p.q_start = q_start; p.Tq = (int32_t)Tq; p.Q = (uint32_t)Q;
     p.div_tq = make_fastdiv((uint32_t)Tq); p.qb = (uint32_t)qb;
+    p.q_lo = 0; p.q_hi = (uint32_t)Q; p.finalize = 1;
     p.index = c->d_index; p.n_buckets = c->n_buckets;
     p.phrase_tokens = c->d_phrase_tokens; p.rows = c->gpu_rows; p.d = c->cfg.d;
     p.h = h; p.out = out;

@@ -35,7 +35,9 @@ struct TfeLookupParams {
     int32_t B, T, q_start, Tq;
     uint32_t Q;
     TfeFastDiv div_tq;              // division by Tq
-    uint32_t qb;                    // queries per warp batch: 1, 2, 4 or 8
+    uint32_t qb;                    // queries per warp batch, 1..8
+    uint32_t q_lo, q_hi;            // LONGEST / CONST kernel: this launch handles queries [q_lo, q_hi) of the call
+    uint32_t finalize;              // 1: this launch closes the call (builds the miss list over all Q queries)
     const ulonglong2 *index;
     uint64_t n_buckets;
     const int4 *phrase_tokens;      // [N] token tuples, only read for hashed orders
@@ -221,7 +223,8 @@ __device__ __forceinline__ void load_memory(const uint4 *const (&rowp)[ALL ? 4 :
 // context scratch arrays; `my_miss` is warp-uniform.  Blocks add their miss counts to RUNNING and
 // tick DONE (one 64-bit atomic); the block that finishes last turns the flag bytes into the ordered miss list
 // (ascending entry index = ascending (q, order)), publishes TOTAL and re-arms the counters.
-__device__ __forceinline__ void tfe_finish_block(const TfeLookupParams &p, uint32_t my_miss, int cols)
+__device__ __forceinline__ void tfe_finish_block(const TfeLookupParams &p, uint32_t my_miss, int cols,
+                                                 bool finalize = true)
 {
     __shared__ uint32_t s_miss, s_last, s_total, s_scan;
     __shared__ uint32_t s_warp[32];
@@ -243,6 +246,10 @@ __device__ __forceinline__ void tfe_finish_block(const TfeLookupParams &p, uint3
     }
     __syncthreads();
     if (!s_last) return;
+    if (!finalize) {        // a partial launch of a call issued in pieces: misses keep accumulating
+        if (threadIdx.x == 0) p.counters[TFE_CTR_DONE] = 0;
+        return;
+    }
     __threadfence();
     const uint32_t total = s_total;
     if (total != 0) {
@@ -577,7 +584,7 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
 //     phrases with one 64-bit key cannot both be in the table, so this means the n-gram is not a
 //     phrase) simply repeats the first row's loads with the corrected choice; nothing has been
 //     stored before that point, in place or not.
-template <int HT, bool PACKED>
+template <int HT, bool PACKED, bool RANGED>
 __global__ void __launch_bounds__(TFE_BLOCK_THREADS, TFE_MIN_BLOCKS)
 tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
 {
@@ -593,18 +600,20 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
     const int my_order = oi < p.n_orders ? p.orders[oi] : 0;
     const bool my_hashed = my_order > 0 && !tfe_order_is_packed(my_order, p.tok_bits);
     const uint32_t qb = p.qb;
-    const uint32_t n_batches = (p.Q + qb - 1) / qb;
+    // RANGED: the call is issued in several launches, each over a query range [q_lo, q_hi)
+    const uint32_t q_lo = RANGED ? p.q_lo : 0u, q_hi = RANGED ? p.q_hi : p.Q;
+    const uint32_t n_batches = (q_hi - q_lo + qb - 1) / qb;
     const uint32_t n_warps = gridDim.x * TFE_WARPS_PER_BLOCK;
     uint32_t my_miss = 0;
 
     // the id `oi` places before query ql of a batch, or -1 (no such position / padding id)
-    // Query lq of batch b is b + lq * n_batches: a warp's queries are spread over the whole call, so
+    // Query lq of batch b is q_lo + b + lq * n_batches: a warp's queries are spread over the whole call, so
     // a run of consecutive positions that all hit (phrases overlap) is shared out among many warps
     // instead of making one warp fetch a row for every query of its batch.
     auto fetch_token = [&](uint32_t batch) -> int32_t {
-        const uint32_t q = batch + (uint32_t)ql * n_batches;
+        const uint32_t q = q_lo + batch + (uint32_t)ql * n_batches;
         int32_t v = -1;
-        if (batch < n_batches && ql < (int)qb && q < p.Q) {
+        if (batch < n_batches && ql < (int)qb && q < q_hi) {
             const uint32_t b = tfe_div(q, p.div_tq);
             const int32_t t = p.q_start + (int32_t)(q - b * (uint32_t)p.Tq) - oi;
             if (t >= 0) {
@@ -626,8 +635,8 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
     uint32_t batch = blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5);
     int32_t tok = fetch_token(batch);
     for (; batch < n_batches; batch += n_warps) {
-        const uint32_t q = batch + (uint32_t)ql * n_batches;
-        const bool mine = ql < (int)qb && q < p.Q;
+        const uint32_t q = q_lo + batch + (uint32_t)ql * n_batches;
+        const bool mine = ql < (int)qb && q < q_hi;
 
         // ================================ probe phase ================================
         int32_t tk[4];
@@ -663,7 +672,7 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
         uint4 hv[UNROLL];
         typename TfeVec<HT>::RowRaw rv[UNROLL];
         auto issue_first = [&](uint32_t lq, int32_t sl) {
-            const char *hrow = reinterpret_cast<const char *>(p.h) + (size_t)(batch + lq * n_batches) * hid_row_bytes;
+            const char *hrow = reinterpret_cast<const char *>(p.h) + (size_t)(q_lo + batch + lq * n_batches) * hid_row_bytes;
             const uint4 *rowp = p.rows + (size_t)(sl >= 0 ? sl : 0) * (size_t)(p.d / 8);
             if (sl >= 0 || !in_place) {
 #pragma unroll
@@ -686,8 +695,8 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
 
         // ================================ gather phase ===============================
         for (uint32_t lq = 0; lq < qb; ++lq) {
-            const uint32_t gq = batch + lq * n_batches;
-            if (gq >= p.Q) break;
+            const uint32_t gq = q_lo + batch + lq * n_batches;
+            if (gq >= q_hi) break;
             const int32_t sl = __shfl_sync(0xFFFFFFFFu, my_slot, 4 * lq);
             if (lq > 0 || redo_first) issue_first(lq, sl);
             if (sl < 0 && in_place) continue;    // nothing to add and nothing to copy
@@ -733,7 +742,7 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
     }
 
     my_miss = __reduce_add_sync(0xFFFFFFFFu, my_miss);
-    tfe_finish_block(p, my_miss, 1);
+    tfe_finish_block(p, my_miss, 1, !RANGED || p.finalize != 0);
 }
 
 // ------------------------------------------------------------- cache install

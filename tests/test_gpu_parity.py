@@ -330,3 +330,35 @@ def test_host_buffer_entry_point(H):
     np.testing.assert_array_equal(out, rounded)
     np.testing.assert_array_equal(mq, ref.miss_q)
     pr.close()
+
+
+def test_host_buffer_entry_point_in_pieces(H):
+    """A host-buffer call large enough to be issued as several launches over query ranges
+    (copies and kernels overlapped): every output and the ordered miss list of the whole call
+    must equal the oracle's, call after call, and a plain device call afterwards must be
+    unaffected.  T is odd so the pieces end inside sequences."""
+    from paper_2607_07388_b200 import binding as tfe
+    w = synth.config(1, B=6, T=2731, d=1024, n_phrases=60_000, gpu_slots=40_000, residency="hot_host", p=0.6)
+    assert w.Q * w.d * 2 >= 32 << 20
+    tb, pr = H.pair_from_workload(w)
+    h = synth.make_hidden_np(w)
+    for variant in (0, 1):
+        tok = synth.make_queries(w, tb, variant=variant)
+        out = np.empty_like(h)
+        sp = np.empty(w.Q, np.uint32); ss = np.empty(w.Q, np.int32); fl = np.empty(w.Q, np.uint8)
+        tfe.tfe_lookup_inject_host(pr.eng.ctx, tok, w.B, w.T, 0, h, out, lam=1.0, sel_phrase=sp, sel_slot=ss,
+                                   flags=fl)
+        mq, mp, mt, cnt = pr.eng.miss_list()
+        ref = pr.ora.lookup(tok)
+        _, rounded = pr.ora.inject(ref, h, lam=1.0)
+        np.testing.assert_array_equal(sp, ref.sel_phrase)
+        np.testing.assert_array_equal(ss, ref.sel_slot)
+        np.testing.assert_array_equal(fl, ref.flags)
+        np.testing.assert_array_equal(out, rounded)
+        assert cnt == len(ref.miss_q) and cnt > 1000
+        assert len(np.unique(ref.miss_q // 2048)) > 4        # misses in many pieces
+        np.testing.assert_array_equal(mq, ref.miss_q)
+        np.testing.assert_array_equal(mp, ref.miss_phrase)
+        np.testing.assert_array_equal(mt, ref.miss_tier)
+    pr.run_and_compare(tok, h, lam=1.0)
+    pr.close()
