@@ -206,7 +206,7 @@ def time_oracle(w, tb, tok, h, q_start, budget_s):
     t0 = time.perf_counter()
     oracle_step(orc, ora, tok, h, q_start)
     t1 = time.perf_counter() - t0
-    reps = int(max(1, min(50, budget_s / max(t1, 1e-6))))
+    reps = int(max(1, min(5000, budget_s / max(t1, 1e-6))))
     times = []
     for _ in range(reps):
         t0 = time.perf_counter()

@@ -19,6 +19,7 @@
  *   - list of matched-but-not-GPU-resident phrases            [Sec. 4.3, staged / asynchronous reads]
  *   - insertion of fetched entries into the GPU tier          [Sec. 4.3, "inserts the entry into a faster tier"]
  *   - prefetch candidates from predicted tokens + priority     [Sec. 4.4, candidate set Q_t, score s = p r c]
+ *   - retention ranking of GPU-tier slots (frequency, recency) [Sec. 4.3, cache policy signals]
  *
  * Parity pins: every function here is pinned by tests that do not call it to
  * produce their expected values (hand-made cases, closed forms, a library
@@ -27,6 +28,9 @@
  * the gate "may be a scalar, a vector, or a learned function", so the formula
  * g = lambda * sigmoid(cos(h, m)) is this build's own reading --
  * COSINE gate: parity unpinned.
+ * The same holds for the retention ranking: the paper lists its signals and no formula, so the
+ * key (decayed frequency, then recency) is this build's reading, pinned only where it reduces to
+ * textbook least-recently-used / least-frequently-used order -- retention ranking: parity unpinned.
  *
  * Conventions shared by all functions
  *   tokens        int32 [B][T] row-major.  Ids outside [0, vocab) are padding:
@@ -404,6 +408,82 @@ int32_t orc_cache_install(int64_t N, int64_t C, int32_t d,
         slot_owner[dst[k]] = (int64_t)ids[k];
     }
     return 0;
+}
+
+/* ------------------------------------------------ GPU-tier retention ranking */
+
+/* The paper ranks cached entries by signals -- access frequency and recency first among them --
+ * and prints no formula [Sec. 4.3, cache policy].  PARITY UNPINNED BY THE PAPER: the reading below
+ * is this build's, pinned by its special cases (pure LRU, pure LFU, free slots first).
+ *
+ * State per GPU-tier slot: freq = number of injections served from the slot since its row was
+ * installed, last = epoch of the most recent one.  The epoch counts lookup calls.  A lookup at epoch
+ * e adds 1 to freq and sets last = e for every entry it injects from the GPU tier (flag 1); an
+ * install at epoch e sets freq = 1, last = e (the row counts as used once, now).
+ *
+ * Retention key of a slot at epoch `now` (larger = more worth keeping), all in unsigned 32-bit:
+ *     age     = now - last
+ *     decayed = freq >> min(31, age / half_life)        (half_life <= 0: no decay)
+ *     key     = min(decayed, 65535) << 16  |  (65535 - min(age, 65535))
+ * i.e. frequency halved once per half_life idle epochs, ties broken by recency.  A slot without an
+ * owner has key 0.  Victims are the n slots of smallest (key, slot), in that order. */
+void orc_cache_touch(int64_t n_ent, const uint8_t *flags, const int32_t *sel_slot, uint32_t epoch,
+                     uint32_t *freq, uint32_t *last)
+{
+    for (int64_t e = 0; e < n_ent; ++e)
+        if (flags[e] == 1) {
+            freq[sel_slot[e]] += 1u;
+            last[sel_slot[e]] = epoch;
+        }
+}
+
+void orc_cache_installed(int32_t n, const int32_t *dst_slots, uint32_t epoch, uint32_t *freq, uint32_t *last)
+{
+    for (int32_t k = 0; k < n; ++k) {
+        freq[dst_slots[k]] = 1u;
+        last[dst_slots[k]] = epoch;
+    }
+}
+
+uint32_t orc_retention_key(uint32_t freq, uint32_t last, uint32_t now, int32_t half_life)
+{
+    const uint32_t age = now - last;
+    uint32_t shift = 0;
+    if (half_life > 0) {
+        shift = age / (uint32_t)half_life;
+        if (shift > 31u) shift = 31u;
+    }
+    uint32_t decayed = freq >> shift;
+    if (decayed > 65535u) decayed = 65535u;
+    return (decayed << 16) | (65535u - (age > 65535u ? 65535u : age));
+}
+
+typedef struct { uint32_t key; int32_t slot; } orc_slot_rank;
+
+static int slot_rank_cmp(const void *pa, const void *pb)
+{
+    const orc_slot_rank *a = (const orc_slot_rank *)pa, *b = (const orc_slot_rank *)pb;
+    if (a->key != b->key) return a->key < b->key ? -1 : 1;
+    return a->slot < b->slot ? -1 : (a->slot > b->slot ? 1 : 0);
+}
+
+/* slot_owner[s] < 0: slot s is free.  Writes min(n, C) slots (and their keys) and returns that count. */
+int64_t orc_cache_victims(int64_t C, const int64_t *slot_owner, const uint32_t *freq, const uint32_t *last,
+                          uint32_t now, int32_t half_life, int64_t n, int32_t *out_slots, uint32_t *out_keys)
+{
+    orc_slot_rank *r = (orc_slot_rank *)malloc((size_t)(C > 0 ? C : 1) * sizeof *r);
+    for (int64_t s = 0; s < C; ++s) {
+        r[s].slot = (int32_t)s;
+        r[s].key = slot_owner[s] < 0 ? 0u : orc_retention_key(freq[s], last[s], now, half_life);
+    }
+    qsort(r, (size_t)C, sizeof *r, slot_rank_cmp);
+    const int64_t take = n < C ? n : C;
+    for (int64_t k = 0; k < take; ++k) {
+        out_slots[k] = r[k].slot;
+        if (out_keys) out_keys[k] = r[k].key;
+    }
+    free(r);
+    return take;
 }
 
 /* ------------------------------------------- prefetch candidates + priority */

@@ -60,6 +60,9 @@ def lib() -> C.CDLL:
         _lib.orc_select.restype = C.c_int64
         _lib.orc_cache_install.restype = C.c_int32
         _lib.orc_prefetch_candidates.restype = C.c_int64
+        _lib.orc_cache_victims.restype = C.c_int64
+        _lib.orc_retention_key.restype = C.c_uint32
+        _lib.orc_retention_key.argtypes = [C.c_uint32, C.c_uint32, C.c_uint32, C.c_int32]
     return _lib
 
 
@@ -115,6 +118,10 @@ class Oracle:
         res = np.nonzero(self.slot_state >= 0)[0]
         self.slot_owner[self.slot_state[res]] = res
         self._perm = None
+        # retention state of the GPU tier (frequency, epoch of last use), epoch = lookups so far
+        self.freq = np.zeros(self.C, np.uint32)
+        self.last = np.zeros(self.C, np.uint32)
+        self.epoch = 0
 
     # -- exact match ------------------------------------------------------
     def sorted_perm(self) -> np.ndarray:
@@ -180,9 +187,31 @@ class Oracle:
         ids = _c(ids, np.uint32)
         dst = _c(dst_slots, np.int32)
         src = None if src_rows is None else _c(src_rows, np.uint16)
-        return int(lib().orc_cache_install(
+        rc = int(lib().orc_cache_install(
             C.c_int64(self.N), C.c_int64(self.C), C.c_int32(self.d), _p(self.slot_state),
             _p(self.slot_owner), _p(self.rows), C.c_int32(len(ids)), _p(ids), _p(src), _p(dst)))
+        if rc == 0:
+            lib().orc_cache_installed(C.c_int32(len(ids)), _p(dst), C.c_uint32(self.epoch), _p(self.freq),
+                                      _p(self.last))
+        return rc
+
+    # -- GPU-tier retention ranking ---------------------------------------------
+    def touch(self, res: LookupResult) -> None:
+        """Account one lookup call: bump the slots it injected from, then advance the epoch."""
+        flags = _c(res.flags, np.uint8).ravel()
+        slots = _c(res.sel_slot, np.int32).ravel()
+        lib().orc_cache_touch(C.c_int64(flags.size), _p(flags), _p(slots), C.c_uint32(self.epoch),
+                              _p(self.freq), _p(self.last))
+        self.epoch += 1
+
+    def cache_victims(self, n, half_life=0):
+        """(slots int32[m], keys uint32[m]), m = min(n, C): ascending (retention key, slot)."""
+        m = min(int(n), self.C)
+        slots, keys = np.empty(max(m, 1), np.int32), np.empty(max(m, 1), np.uint32)
+        got = lib().orc_cache_victims(C.c_int64(self.C), _p(self.slot_owner), _p(self.freq), _p(self.last),
+                                      C.c_uint32(self.epoch), C.c_int32(half_life), C.c_int64(n), _p(slots),
+                                      _p(keys))
+        return slots[:got].copy(), keys[:got].copy()
 
     # -- prefetch candidates + priority ------------------------------------------
     def prefetch_candidates(self, history, cand, prob, *, usefulness=None, benefit_host=1.0, benefit_ssd=2.0,

@@ -542,3 +542,107 @@ def test_prefetch_candidates_against_python_restatement(oracle_mod, seed, orders
         assert tr.tolist() == [e[3] for e in exp]
         assert src.tolist() == [e[4] for e in exp]
         np.testing.assert_array_equal(sc, np.array([-e[0] for e in exp], np.float32))
+
+
+# ---------------------------------------------------------------- retention ranking (Sec. 4.3)
+
+def _mini_oracle(orc, C, owners=None):
+    """An oracle over C single-slot phrases (phrase i lives in slot i unless owners says otherwise)."""
+    N = C
+    pt = np.full((N, 4), -1, np.int32)
+    pt[:, 0] = np.arange(N) // 50
+    pt[:, 1] = np.arange(N) % 50
+    pl = np.full(N, 2, np.uint8)
+    init = np.arange(N, dtype=np.int32) if owners is None else np.asarray(owners, np.int32)
+    rows = np.zeros((C, 16), np.uint16)
+    return orc.Oracle(pt, pl, init, rows, d=16, vocab=64, orders=(2,), gpu_slots=C)
+
+
+def test_retention_key_hand_worked(oracle_mod):
+    k = oracle_mod.lib().orc_retention_key
+    # no decay: frequency in the high half, 65535 - age in the low half
+    assert k(3, 10, 12, 0) == (3 << 16) | (65535 - 2)
+    # half-life 4, idle for 9 epochs: two halvings of 13 -> 3
+    assert k(13, 1, 10, 4) == (3 << 16) | (65535 - 9)
+    # saturation of both halves; shift capped at 31
+    assert k(1 << 20, 5, 5, 0) == (65535 << 16) | 65535
+    assert k(7, 0, 100000, 0) == (7 << 16) | 0
+    assert k(0xFFFFFFFF, 0, 1000, 1) == (1 << 16) | (65535 - 1000)
+    # monotone: more hits never lowers the key; longer idle never raises it
+    for f in range(0, 40):
+        assert k(f + 1, 3, 9, 2) >= k(f, 3, 9, 2)
+        assert k(20, 3, 9 + f + 1, 2) <= k(20, 3, 9 + f, 2)
+
+
+def test_retention_reduces_to_lru_and_lfu(oracle_mod):
+    rng = np.random.default_rng(5)
+    C = 64
+    o = _mini_oracle(oracle_mod, C)
+    # equal frequencies, distinct last-use epochs: victims come in least-recently-used order
+    o.freq[:] = 1
+    o.last[:] = rng.permutation(C).astype(np.uint32)
+    o.epoch = C
+    slots, _ = o.cache_victims(10, half_life=0)
+    np.testing.assert_array_equal(slots, np.argsort(o.last, kind="stable")[:10])
+    # equal last use, distinct frequencies: least-frequently-used order
+    o.last[:] = 7
+    o.freq[:] = (rng.permutation(C) + 1).astype(np.uint32)
+    slots, _ = o.cache_victims(C + 5, half_life=0)
+    np.testing.assert_array_equal(slots, np.argsort(o.freq, kind="stable"))
+    # ties keep ascending slot order
+    o.freq[:] = 2
+    slots, keys = o.cache_victims(5)
+    np.testing.assert_array_equal(slots, np.arange(5))
+    assert len(set(keys.tolist())) == 1
+
+
+def test_retention_free_slots_first_and_state_updates(oracle_mod):
+    C = 12
+    owners = np.arange(C, dtype=np.int32)
+    owners[[3, 8]] = -1                      # phrases 3 and 8 start on the host: slots 3 and 8 are free
+    o = _mini_oracle(oracle_mod, C, owners)
+    toks = np.array([[0, 0, 0, 1, 0, 1, 0, 5]], np.int32)     # 2-grams (0,0) (0,0) (0,1) (1,0) (0,1) (1,0) (0,5)
+    res = o.lookup(toks)
+    o.touch(res)                              # epoch 0 -> 1
+    res2 = o.lookup(np.array([[0, 1, 0, 0]], np.int32))
+    o.touch(res2)                             # epoch 1 -> 2
+    # phrase ids: (0,0)=0, (0,1)=1, (0,5)=5, (1,0)=50 (not in this 12-phrase table)
+    expect_freq = np.zeros(C, np.uint32); expect_last = np.zeros(C, np.uint32)
+    expect_freq[0], expect_last[0] = 3, 1     # (0,0): twice in call 0, once in call 1
+    expect_freq[1], expect_last[1] = 3, 1     # (0,1): twice in call 0, once in call 1
+    expect_freq[5], expect_last[5] = 1, 0
+    np.testing.assert_array_equal(o.freq, expect_freq)
+    np.testing.assert_array_equal(o.last, expect_last)
+    assert o.epoch == 2
+    slots, keys = o.cache_victims(4)
+    # free slots (key 0) first in slot order, then never-used owned slots: age 2, freq 0
+    np.testing.assert_array_equal(slots, [3, 8, 2, 4])
+    np.testing.assert_array_equal(keys, [0, 0, 65533, 65533])
+    # installing phrase 3 into slot 8 makes the slot owned, used once, now
+    assert o.cache_install([3], np.ones((1, 16), np.uint16), [8]) == 0
+    assert o.freq[8] == 1 and o.last[8] == 2
+    slots, _ = o.cache_victims(C)
+    assert slots[0] == 3 and list(slots).index(8) > list(slots).index(5) > list(slots).index(4)
+    assert slots[-1] == 1 and slots[-2] == 0
+
+
+def test_retention_against_independent_restatement(oracle_mod):
+    rng = np.random.default_rng(11)
+    C = 5000
+    owners = np.arange(C, dtype=np.int32)
+    owners[rng.choice(C, 37, replace=False)] = -1
+    o = _mini_oracle(oracle_mod, C, owners)
+    o.freq[:] = rng.geometric(0.02, C).astype(np.uint32) * (rng.random(C) < 0.8)
+    o.freq[rng.choice(C, 5)] = 3_000_000
+    o.epoch = 90_000
+    o.last[:] = (o.epoch - np.minimum(o.epoch, rng.geometric(0.0005, C))).astype(np.uint32)
+    for hl in (0, 1, 7, 300, 100_000):
+        age = (np.uint64(o.epoch) - o.last.astype(np.uint64))
+        shift = np.minimum(31, age // hl) if hl > 0 else np.zeros(C, np.uint64)
+        dec = np.minimum(o.freq.astype(np.uint64) >> shift.astype(np.uint64), 65535)
+        key = (dec << np.uint64(16)) | (np.uint64(65535) - np.minimum(age, 65535))
+        key[o.slot_owner < 0] = 0
+        order = np.lexsort((np.arange(C), key))
+        slots, keys = o.cache_victims(700, half_life=hl)
+        np.testing.assert_array_equal(slots, order[:700])
+        np.testing.assert_array_equal(keys, key[order[:700]].astype(np.uint32))
