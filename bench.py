@@ -59,6 +59,8 @@ def parse_args():
     ap.add_argument("--prefetch", action="store_true",
                     help="time tfe_prefetch_candidates (B sequences x top-K tokens) on the workload's table")
     ap.add_argument("--top-k", type=int, default=64)
+    ap.add_argument("--cache-policy", action="store_true",
+                    help="time the retention bookkeeping in the lookup and tfe_cache_select_victims on the workload")
     ap.add_argument("--sweep", action="store_true", help="c5: tokens x row width x hit rate sweep")
     ap.add_argument("--sweep-tokens", default="1,4,16,64,256,1024,4096,16384,65536")
     ap.add_argument("--sweep-d", default="1024,2048,4096")
@@ -395,6 +397,8 @@ def run_ours(a):
         return run_sweep(a, dev, rank)
     if a.prefetch:
         return run_prefetch(a, dev, rank)
+    if a.cache_policy:
+        return run_cache_policy(a, dev, rank)
 
     w = make_workload(a)
     sampler = ClockSampler(local_rank) if rank == 0 else None
@@ -639,6 +643,74 @@ def run_prefetch(a, dev, rank):
                           "cpu_baseline": {"value": E / cpu_s, "unit": "probes/s", "cores": 1, "kind": "oracle",
                                            "sample": "one call, single thread"},
                           "parity": parity}))
+    sess.close()
+
+
+def run_cache_policy(a, dev, rank):
+    """GPU-tier retention ranking: cost of the frequency / recency bookkeeping inside the lookup, and
+    tfe_cache_select_victims over all GPU-tier slots (a stream over 40 bytes per slot)."""
+    import torch
+    from paper_2607_07388_b200 import binding as tfe
+    L = tfe.lib()
+    w = make_workload(a)
+    nbuf = 4 if w.shape == "prefill" else 32
+    sess = Session(w, dev, nbuf, a.tune_batch)
+    eng = sess.eng
+    stream = torch.cuda.current_stream()
+    sp = stream.cuda_stream
+    calls = sess.lookup_calls(sp)
+
+    def lookup(i):
+        st = L.tfe_lookup_inject(*calls[i % nbuf])
+        if st:
+            raise RuntimeError(f"tfe_lookup_inject failed: {st}")
+
+    off_ms, _ = timed_region(lookup, a.steps, max(3, a.warmup), stream, 1, None, dev)
+    eng.cache_policy_enable()
+    on_ms, _ = timed_region(lookup, a.steps, max(3, a.warmup), stream, 1, None, dev)
+    # parity: a fresh state, one lookup per buffer in order, against the oracle's state machine
+    eng.cache_policy_enable()
+    for v in range(nbuf):
+        lookup(v)
+    freq, last, epoch = eng.cache_stats()
+    orc, ora = oracle_for(w, sess.tb)
+    t_cpu = 0.0
+    for v in range(nbuf):
+        ref = ora.lookup(sess.toks_np[v], w.q_start)
+        t0 = time.perf_counter()
+        ora.touch(ref)
+        t_cpu += time.perf_counter() - t0
+    n_vic, half_life = min(4096, w.gpu_slots), 2
+    slots, keys = eng.cache_select_victims(n_vic, half_life)
+    t0 = time.perf_counter()
+    e_slots, e_keys = ora.cache_victims(n_vic, half_life)
+    t_cpu_sel = time.perf_counter() - t0
+    parity = {"epoch": bool(epoch == ora.epoch), "freq": bool(np.array_equal(freq, ora.freq)),
+              "last": bool(np.array_equal(last, ora.last)), "victims": bool(np.array_equal(slots, e_slots)),
+              "keys": bool(np.array_equal(keys, e_keys))}
+
+    def select(i):
+        eng.cache_select_victims(n_vic, half_life)
+
+    reps = max(20, min(200, a.steps))
+    sel_ms, _ = timed_region(select, reps, 3, stream, 1, None, dev)
+    us = sel_ms / reps * 1e3
+    peak, peak_src = measured_peak()
+    bytes_alg = w.gpu_slots * 40 + n_vic * 24
+    if rank == 0:
+        print(json.dumps({
+            "metric": "victim selection slots/s", "value": w.gpu_slots / (us * 1e-6), "unit": "slots/s",
+            "us_per_call": us, "steps": reps,
+            "config": {"workload": w.name, "gpu_slots": w.gpu_slots, "n_victims": n_vic, "half_life": half_life,
+                       "call": "tfe_cache_select_victims: 8 launches + copy of the slots to the host + synchronise"},
+            "roofline": {"bound": "hbm", "achieved": bytes_alg / us / 1e3, "peak": peak, "unit": "GB/s",
+                         "frac": bytes_alg / us / 1e3 / peak, "traffic": None, "peak_source": peak_src,
+                         "algorithmic_bytes_per_call": bytes_alg},
+            "lookup_us": {"bookkeeping_off": off_ms / a.steps * 1e3, "bookkeeping_on": on_ms / a.steps * 1e3,
+                          "launches": "direct, one per step"},
+            "cpu_baseline": {"value": w.gpu_slots / t_cpu_sel, "unit": "slots/s", "cores": 1, "kind": "oracle",
+                             "sample": "one selection over all slots (qsort), single thread"},
+            "parity": parity}))
     sess.close()
 
 

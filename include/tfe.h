@@ -215,6 +215,47 @@ tfe_status tfe_lookup_inject_noalloc(tfe_ctx *ctx, const int32_t *tokens, int32_
 tfe_status tfe_miss_list_device(tfe_ctx *ctx, const uint32_t **q_idx, const uint32_t **phrase_id,
                                 const uint8_t **tier, const uint32_t **count);
 
+/*
+ * GPU-tier retention ranking (paper Sec. 4.3: "TF-Engram can rank memory entries using access
+ * frequency, recency, ..." -- the signals are the paper's, it gives no formula; the ranking below
+ * is this library's reading).
+ *
+ * tfe_cache_policy_enable -- starts the bookkeeping: from now on every lookup of this context
+ * (tfe_lookup_inject, tfe_lookup_inject_host; not tfe_lookup_inject_noalloc) adds 1 to `freq` and
+ * stores the call's epoch in `last` for every GPU-tier slot it injects from, and every
+ * tfe_cache_install sets {freq, last} = {1, epoch} for the slots it fills.  The epoch is a device
+ * counter of completed lookups (a replayed launch advances it like a fresh one).  Calling it
+ * again clears the counters and the epoch.  Allocates 12 bytes per GPU-tier slot; waits for the
+ * device.  Errors: INVALID_ARG, CUDA.
+ */
+tfe_status tfe_cache_policy_enable(tfe_ctx *ctx, void *stream);
+
+/*
+ * tfe_cache_select_victims -- the n slots least worth keeping at the current epoch `now`:
+ *     age     = now - last                                  (unsigned 32-bit)
+ *     decayed = freq >> min(31, age / half_life)            (half_life <= 0: no decay)
+ *     key     = min(decayed, 65535) << 16 | (65535 - min(age, 65535));  key = 0 for a free slot
+ * in ascending (key, slot): free slots first, then by decayed frequency, ties by least recent
+ * use, then by slot.  half_life -> large gives least-frequently-used order, equal frequencies
+ * give least-recently-used order.
+ *
+ *   n        0..4096;  slots HOST int32 [n];  keys HOST uint32 [n] or NULL;
+ *   count    HOST: entries written = min(n, gpu_slots).
+ * Eight kernel launches on `stream`, then synchronises it (the slots feed tfe_cache_install,
+ * which takes host arrays).  tfe_cache_select_victims_device returns the DEVICE copies of the
+ * most recent selection (owned by the context, valid until the next one).
+ * Errors: INVALID_ARG (also: policy not enabled), CUDA.
+ */
+tfe_status tfe_cache_select_victims(tfe_ctx *ctx, int32_t n, int32_t half_life, int32_t *slots,
+                                    uint32_t *keys, int32_t *count, void *stream);
+tfe_status tfe_cache_select_victims_device(tfe_ctx *ctx, const int32_t **slots, const uint32_t **keys);
+
+/*
+ * tfe_cache_stats -- copies the bookkeeping to the host: freq_last HOST uint32 [gpu_slots][2]
+ * ({freq, last} per slot) and/or the epoch (either may be NULL).  Synchronises `stream`.
+ */
+tfe_status tfe_cache_stats(tfe_ctx *ctx, uint32_t *freq_last, uint32_t *epoch, void *stream);
+
 /* Scoring of prefetch candidates. */
 typedef struct {
     float   benefit_host;   /* c_i of an entry that sits in host DRAM (>= 0)                           */

@@ -31,7 +31,9 @@ NO_PHRASE = 0xFFFFFFFF
 EXPORTS = ["tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
            "tfe_miss_list", "tfe_miss_list_device", "tfe_destroy", "tfe_status_string",
            "tfe_last_cuda_error", "tfe_index_geometry", "tfe_phrase_key64", "tfe_home_bucket",
-           "tfe_launch_geometry", "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates"]
+           "tfe_launch_geometry", "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
+           "tfe_cache_policy_enable", "tfe_cache_select_victims", "tfe_cache_select_victims_device",
+           "tfe_cache_stats"]
 
 
 class TfeConfig(C.Structure):
@@ -92,9 +94,15 @@ def lib() -> C.CDLL:
         L.tfe_home_bucket.restype = u64
         L.tfe_launch_geometry.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
         L.tfe_set_tuning.argtypes = [vp, i32]
+        L.tfe_cache_policy_enable.argtypes = [vp, vp]
+        L.tfe_cache_select_victims.argtypes = [vp, i32, i32, vp, vp, C.POINTER(i32), vp]
+        L.tfe_cache_select_victims_device.argtypes = [vp, C.POINTER(vp), C.POINTER(vp)]
+        L.tfe_cache_stats.argtypes = [vp, vp, C.POINTER(C.c_uint32), vp]
         for name in ("tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
                      "tfe_miss_list", "tfe_miss_list_device", "tfe_index_geometry", "tfe_launch_geometry",
-                     "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates"):
+                     "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
+                     "tfe_cache_policy_enable", "tfe_cache_select_victims", "tfe_cache_select_victims_device",
+                     "tfe_cache_stats"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -207,6 +215,36 @@ def tfe_prefetch_candidates(ctx: int, history, B, H, cand_tokens, cand_prob, K, 
                                          _addr(usefulness), C.byref(p), _addr(out_phrase), _addr(out_tier),
                                          _addr(out_score), _addr(out_src), _addr(out_count), _stream(stream)),
            "tfe_prefetch_candidates")
+
+
+VICTIMS_MAX = 4096
+
+
+def tfe_cache_policy_enable(ctx: int, stream=None) -> None:
+    _check(lib().tfe_cache_policy_enable(ctx, _stream(stream)), "tfe_cache_policy_enable")
+
+
+def tfe_cache_select_victims(ctx: int, n: int, half_life: int = 0, stream=None):
+    """(slots int32[m], keys uint32[m]), m = min(n, gpu_slots), ascending (retention key, slot)."""
+    slots, keys = np.empty(max(n, 1), np.int32), np.empty(max(n, 1), np.uint32)
+    cnt = C.c_int32(0)
+    _check(lib().tfe_cache_select_victims(ctx, int(n), int(half_life), _addr(slots), _addr(keys), C.byref(cnt),
+                                          _stream(stream)), "tfe_cache_select_victims")
+    return slots[:cnt.value], keys[:cnt.value]
+
+
+def tfe_cache_select_victims_device(ctx: int):
+    a, b = C.c_void_p(), C.c_void_p()
+    _check(lib().tfe_cache_select_victims_device(ctx, C.byref(a), C.byref(b)), "tfe_cache_select_victims_device")
+    return a.value, b.value
+
+
+def tfe_cache_stats(ctx: int, gpu_slots: int, stream=None):
+    """(freq uint32[C], last uint32[C], epoch)."""
+    fl = np.empty((max(gpu_slots, 1), 2), np.uint32)
+    ep = C.c_uint32(0)
+    _check(lib().tfe_cache_stats(ctx, _addr(fl), C.byref(ep), _stream(stream)), "tfe_cache_stats")
+    return fl[:gpu_slots, 0].copy(), fl[:gpu_slots, 1].copy(), ep.value
 
 
 def tfe_miss_list(ctx: int, cap: int, stream=None, allow_overflow=False):

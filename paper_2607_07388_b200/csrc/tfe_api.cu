@@ -82,6 +82,15 @@ struct tfe_ctx {
     uint32_t *d_pf_counter = nullptr;
     int64_t pf_cap = 0;
 
+    // retention ranking (tfe_cache_policy_enable): per-slot {freq, last}, the lookup count, and
+    // the victim selection's work space
+    uint2 *d_slot_stats = nullptr;
+    uint32_t *d_epoch = nullptr;
+    uint32_t *d_slot_key = nullptr, *d_vs_hist = nullptr, *d_vs_keys = nullptr;
+    TfeVictimState *d_vs_state = nullptr;
+    unsigned long long *d_vs_list = nullptr;
+    int32_t *d_vs_slots = nullptr;
+
     // host-buffer variant staging
     int32_t *d_h_tokens = nullptr;
     void *d_h_hidden = nullptr, *d_h_out = nullptr;
@@ -298,6 +307,8 @@ void tfe_destroy(tfe_ctx *c)
     free_dev(c->d_h_tokens); free_dev(c->d_h_hidden); free_dev(c->d_h_out);
     free_dev(c->d_h_phrase); free_dev(c->d_h_slot); free_dev(c->d_h_flag);
     free_dev(c->d_pf_keys); free_dev(c->d_pf_phrase); free_dev(c->d_pf_tier); free_dev(c->d_pf_counter);
+    free_dev(c->d_slot_stats); free_dev(c->d_epoch); free_dev(c->d_slot_key); free_dev(c->d_vs_hist);
+    free_dev(c->d_vs_keys); free_dev(c->d_vs_state); free_dev(c->d_vs_list); free_dev(c->d_vs_slots);
     if (c->hb_in) (void)cudaStreamDestroy(c->hb_in);
     if (c->hb_out) (void)cudaStreamDestroy(c->hb_out);
     if (c->hb_ev_start) (void)cudaEventDestroy(c->hb_ev_start);
@@ -404,7 +415,7 @@ tfe_status tfe_index_build(const tfe_config *cfg, const int32_t *phrase_tokens,
     CUF(cudaMemcpyAsync(c->d_index, slots.data(), index_bytes, cudaMemcpyHostToDevice, stream));
     CUF(cudaMalloc(&c->d_phrase_pos, std::max<size_t>(4, (size_t)N * 4)));
     if (N > 0) CUF(cudaMemcpyAsync(c->d_phrase_pos, pos.data(), (size_t)N * 4, cudaMemcpyHostToDevice, stream));
-    CUF(cudaMalloc(&c->d_slot_owner, std::max<size_t>(4, (size_t)C * 4)));
+    CUF(cudaMalloc(&c->d_slot_owner, std::max<size_t>(4, (size_t)(C + 3) / 4 * 4) * 4));      // whole 16-byte groups
     CUF(cudaMalloc(&c->d_counters, TFE_CTR_WORDS * sizeof(uint32_t)));
     CUF(cudaMemsetAsync(c->d_counters, 0, TFE_CTR_WORDS * sizeof(uint32_t), stream));
     if (C > 0)
@@ -507,7 +518,7 @@ tfe_status tfe_cache_install(tfe_ctx *c, int32_t n, const uint32_t *phrase_ids, 
     const unsigned blocks = (unsigned)((n + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK);
     tfe_install_kernel<<<blocks, TFE_BLOCK_THREADS, 0, stream>>>(c->d_index, c->d_phrase_pos, c->d_slot_owner,
                                                                  c->gpu_rows, c->row_vecs, n, c->d_inst_ids,
-                                                                 src, c->d_inst_slots);
+                                                                 src, c->d_inst_slots, c->d_slot_stats, c->d_epoch);
     CU(cudaGetLastError());
     for (int32_t k = 0; k < n; ++k) {       // mirror, same order as the oracle's state machine
         const uint32_t prev = c->h_owner[(size_t)dst_slots[k]];
@@ -639,6 +650,7 @@ tfe_status lookup_inject_range(tfe_ctx *c, const int32_t *tokens, int32_t B, int
     p.scr_phrase = c->d_scr_phrase; p.scr_flag = c->d_scr_flag;
     p.miss_q = c->d_miss_q; p.miss_phrase = c->d_miss_phrase; p.miss_tier = c->d_miss_tier;
     p.counters = c->d_counters;
+    p.slot_stats = c->d_slot_stats; p.epoch = c->d_epoch;
 
     pick_kernel(variant)<<<(unsigned)grid, TFE_BLOCK_THREADS, 0, stream>>>(p);
     CU(cudaGetLastError());
@@ -783,6 +795,82 @@ tfe_status tfe_miss_list_device(tfe_ctx *c, const uint32_t **q_idx, const uint32
     if (phrase_id) *phrase_id = c->d_miss_phrase;
     if (tier) *tier = c->d_miss_tier;
     if (count) *count = c->d_counters + TFE_CTR_TOTAL;
+    return TFE_OK;
+}
+
+tfe_status tfe_cache_policy_enable(tfe_ctx *c, void *stream_)
+{
+    if (!c) return TFE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const size_t C = ((size_t)std::max<int64_t>(1, c->cfg.gpu_slots) + 3) / 4 * 4;     // whole 16-byte groups
+    if (!c->d_slot_stats) {
+        CU(cudaDeviceSynchronize());        // no lookup in flight while the kernels' arguments change
+        uint2 *stats = nullptr;
+        CU(cudaMalloc(&stats, C * sizeof(uint2)));
+        CU(cudaMalloc(&c->d_epoch, sizeof(uint32_t)));
+        CU(cudaMalloc(&c->d_slot_key, C * sizeof(uint32_t)));
+        CU(cudaMalloc(&c->d_vs_hist, TFE_VICTIM_BINS * sizeof(uint32_t)));
+        CU(cudaMalloc(&c->d_vs_state, sizeof(TfeVictimState)));
+        CU(cudaMalloc(&c->d_vs_list, TFE_VICTIMS_MAX * sizeof(unsigned long long)));
+        CU(cudaMalloc(&c->d_vs_slots, TFE_VICTIMS_MAX * sizeof(int32_t)));
+        CU(cudaMalloc(&c->d_vs_keys, TFE_VICTIMS_MAX * sizeof(uint32_t)));
+        c->d_slot_stats = stats;
+    }
+    CU(cudaMemsetAsync(c->d_slot_stats, 0, C * sizeof(uint2), stream));
+    CU(cudaMemsetAsync(c->d_epoch, 0, sizeof(uint32_t), stream));
+    CU(cudaMemsetAsync(c->d_vs_hist, 0, TFE_VICTIM_BINS * sizeof(uint32_t), stream));
+    return TFE_OK;
+}
+
+tfe_status tfe_cache_select_victims(tfe_ctx *c, int32_t n, int32_t half_life, int32_t *slots, uint32_t *keys,
+                                    int32_t *count, void *stream_)
+{
+    if (!c || n < 0 || n > TFE_VICTIMS_MAX || !count || (n > 0 && !slots)) return TFE_ERR_INVALID_ARG;
+    if (!c->d_slot_stats) return TFE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int64_t C = c->cfg.gpu_slots;
+    const int32_t take = (int32_t)std::min<int64_t>(n, C);
+    *count = take;
+    if (take == 0) return TFE_OK;
+    CU(cudaMemsetAsync(c->d_vs_state, 0, sizeof(TfeVictimState), stream));
+    const unsigned grid = (unsigned)std::max<int64_t>(
+        1, std::min<int64_t>((int64_t)c->sm_count * 4, (C + 4 * TFE_VICTIM_THREADS - 1) / (4 * TFE_VICTIM_THREADS)));
+    static const int kShift[6] = {53, 42, 31, 20, 9, 0}, kBits[6] = {11, 11, 11, 11, 11, 9};
+    tfe_victim_pass_kernel<true><<<grid, TFE_VICTIM_THREADS, 0, stream>>>(c->d_slot_stats, c->d_slot_owner, c->d_epoch, half_life,
+                                                            c->d_slot_key, (uint32_t)C, (uint32_t)take, kShift[0],
+                                                            kBits[0], c->d_vs_hist, c->d_vs_state);
+    for (int i = 1; i < 6; ++i)
+        tfe_victim_pass_kernel<false><<<grid, TFE_VICTIM_THREADS, 0, stream>>>(c->d_slot_stats, c->d_slot_owner, c->d_epoch, half_life,
+                                                                 c->d_slot_key, (uint32_t)C, 0u, kShift[i], kBits[i],
+                                                                 c->d_vs_hist, c->d_vs_state);
+    tfe_victim_collect_kernel<<<grid, TFE_VICTIM_THREADS, 0, stream>>>(c->d_slot_key, (uint32_t)C, c->d_vs_state, c->d_vs_list,
+                                                        TFE_VICTIMS_MAX);
+    tfe_victim_sort_kernel<<<1, 1024, 0, stream>>>(c->d_vs_list, c->d_vs_state, (uint32_t)take, c->d_vs_slots,
+                                                   c->d_vs_keys);
+    CU(cudaGetLastError());
+    CU(cudaMemcpyAsync(slots, c->d_vs_slots, (size_t)take * 4, cudaMemcpyDeviceToHost, stream));
+    if (keys) CU(cudaMemcpyAsync(keys, c->d_vs_keys, (size_t)take * 4, cudaMemcpyDeviceToHost, stream));
+    CU(cudaStreamSynchronize(stream));
+    return TFE_OK;
+}
+
+tfe_status tfe_cache_select_victims_device(tfe_ctx *c, const int32_t **slots, const uint32_t **keys)
+{
+    if (!c || !c->d_slot_stats) return TFE_ERR_INVALID_ARG;
+    if (slots) *slots = c->d_vs_slots;
+    if (keys) *keys = c->d_vs_keys;
+    return TFE_OK;
+}
+
+tfe_status tfe_cache_stats(tfe_ctx *c, uint32_t *freq_last, uint32_t *epoch, void *stream_)
+{
+    if (!c || !c->d_slot_stats) return TFE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (freq_last && c->cfg.gpu_slots > 0)
+        CU(cudaMemcpyAsync(freq_last, c->d_slot_stats, (size_t)c->cfg.gpu_slots * sizeof(uint2), cudaMemcpyDeviceToHost,
+                           stream));
+    if (epoch) CU(cudaMemcpyAsync(epoch, c->d_epoch, sizeof(uint32_t), cudaMemcpyDeviceToHost, stream));
+    CU(cudaStreamSynchronize(stream));
     return TFE_OK;
 }
 

@@ -59,6 +59,8 @@ struct TfeLookupParams {
     uint32_t *miss_q, *miss_phrase; // context miss list, [Q*cols]
     uint8_t *miss_tier;
     uint32_t *counters;             // TFE_CTR_* words
+    uint2 *slot_stats;              // per GPU-tier slot {injections since install, epoch of the last one}, or nullptr
+    uint32_t *epoch;                // lookups completed so far (device word), with slot_stats
 };
 
 // Device-resident launch state (uint32 words; DONE and RUNNING form one 8-byte word that a single
@@ -305,7 +307,15 @@ __device__ __forceinline__ void tfe_finish_block(const TfeLookupParams &p, uint3
         p.counters[TFE_CTR_TOTAL] = total;
         p.counters[TFE_CTR_DONE] = 0;
         p.counters[TFE_CTR_RUNNING] = 0;
+        if (p.slot_stats != nullptr) *p.epoch = *p.epoch + 1;     // every block has read it by now
     }
+}
+
+// A GPU-tier slot served an injection in the lookup of epoch `epoch`.
+__device__ __forceinline__ void tfe_touch_slot(uint2 *slot_stats, int32_t slot, uint32_t epoch)
+{
+    atomicAdd(&slot_stats[slot].x, 1u);
+    slot_stats[slot].y = epoch;
 }
 
 // One lane's probe: the trailing n-gram of query q (n = this lane's order) -> key -> index value
@@ -469,6 +479,8 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
             }
         }
 
+        if (p.slot_stats != nullptr && my_slot >= 0) tfe_touch_slot(p.slot_stats, my_slot, __ldcg(p.epoch));
+
         // ================================ gather phase ===============================
         for (uint32_t lq = 0; lq < qb; ++lq) {
             const uint32_t gq = q0 + lq;
@@ -604,6 +616,7 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
     const uint32_t q_lo = RANGED ? p.q_lo : 0u, q_hi = RANGED ? p.q_hi : p.Q;
     const uint32_t n_batches = (q_hi - q_lo + qb - 1) / qb;
     const uint32_t n_warps = gridDim.x * TFE_WARPS_PER_BLOCK;
+    const uint32_t epoch = p.slot_stats != nullptr ? __ldcg(p.epoch) : 0u;
     uint32_t my_miss = 0;
 
     // the id `oi` places before query ql of a batch, or -1 (no such position / padding id)
@@ -739,6 +752,8 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
                 }
             }
         }
+        // bookkeeping for the retention ranking, off the path between probe and gather
+        if (p.slot_stats != nullptr && my_slot >= 0) tfe_touch_slot(p.slot_stats, my_slot, epoch);
     }
 
     my_miss = __reduce_add_sync(0xFFFFFFFFu, my_miss);
@@ -752,7 +767,7 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
 __global__ void __launch_bounds__(TFE_BLOCK_THREADS)
 tfe_install_kernel(ulonglong2 *index, const uint32_t *phrase_pos, uint32_t *slot_owner, uint4 *rows,
                    int32_t row_vecs, int32_t n, const uint32_t *ids, const uint4 *src,
-                   const int32_t *dst_slots)
+                   const int32_t *dst_slots, uint2 *slot_stats, const uint32_t *epoch)
 {
     const int lane = threadIdx.x & 31;
     const int k = blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5);
@@ -765,6 +780,7 @@ tfe_install_kernel(ulonglong2 *index, const uint32_t *phrase_pos, uint32_t *slot
             index[phrase_pos[prev]].y = ((unsigned long long)prev << 32) | 0xFFFFFFFFull;   // -1: host tier
         index[phrase_pos[id]].y = ((unsigned long long)id << 32) | (uint32_t)dst;
         slot_owner[dst] = id;
+        if (slot_stats != nullptr) slot_stats[dst] = make_uint2(1u, *epoch);     // used once, now
     }
     const uint4 *s = src + (size_t)k * row_vecs;
     uint4 *o = rows + (size_t)dst * row_vecs;
@@ -952,3 +968,197 @@ tfe_prefetch_select_kernel(const unsigned long long *keys, const uint32_t *entry
     (void)n_orders;
 }
 
+
+
+// ------------------------------------------------ GPU-tier retention ranking
+//
+// Which slots to overwrite next (Sec. 4.3: cached entries are ranked by access frequency and
+// recency, among other signals; the formula is this library's).  Per slot the lookup kernels keep
+// {freq, last}: injections served since the row was installed and the epoch (lookup count) of the
+// most recent one.  At epoch `now`
+//     age = now - last,  decayed = freq >> min(31, age / half_life)   (half_life <= 0: no decay)
+//     key = min(decayed, 65535) << 16 | (65535 - min(age, 65535)),    0 for a slot without owner
+// and the victims are the n slots of smallest (key, slot).  (key << 32 | slot) is a distinct
+// 64-bit number per slot, so this is a selection of the n smallest of C distinct numbers:
+//
+//   tfe_victim_pass_kernel   x6, most significant digit first (11,11,11,11,11,9 bits): histogram of
+//                            the digit over the slots that agree with the digits chosen so far; the
+//                            block that finishes last picks the digit holding the n-th smallest
+//                            and re-arms the histogram.  The first pass computes and stores the keys.
+//   tfe_victim_collect_kernel  appends every number <= the n-th smallest to a list (any order)
+//   tfe_victim_sort_kernel     one block: bitonic sort of the list, writes slots and keys
+#define TFE_VICTIMS_MAX 4096
+#define TFE_VICTIM_BINS 2048
+
+struct TfeVictimState {
+    unsigned long long prefix;      // digits chosen so far, in place
+    uint32_t k_rem;                 // rank (1-based) of the wanted number among those sharing the prefix
+    uint32_t ticket;                // blocks done in the current pass
+    uint32_t n_out;                 // entries appended by the collect kernel
+    uint32_t pad;
+};
+
+__device__ __forceinline__ uint32_t tfe_retention_key(uint2 st, uint32_t owner, uint32_t now, int32_t half_life)
+{
+    if (owner == 0xFFFFFFFFu) return 0u;
+    const uint32_t age = now - st.y;
+    const uint32_t shift = half_life > 0 ? min(31u, age / (uint32_t)half_life) : 0u;
+    return (min(st.x >> shift, 65535u) << 16) | (65535u - min(age, 65535u));
+}
+
+#define TFE_VICTIM_THREADS 512
+
+// slot_stats, slot_owner and slot_key hold a multiple of 4 entries (the tail is padding).
+template <bool FIRST>
+__global__ void __launch_bounds__(TFE_VICTIM_THREADS)
+tfe_victim_pass_kernel(const uint2 *slot_stats, const uint32_t *slot_owner, const uint32_t *epoch, int32_t half_life,
+                       uint32_t *slot_key, uint32_t C, uint32_t n_first, int shift, int bits, uint32_t *hist,
+                       TfeVictimState *state)
+{
+    __shared__ uint32_t s_hist[TFE_VICTIM_BINS];
+    __shared__ uint32_t s_part[256];
+    __shared__ uint32_t s_last;
+    for (int i = threadIdx.x; i < TFE_VICTIM_BINS; i += blockDim.x) s_hist[i] = 0;
+    __syncthreads();
+    const unsigned long long prefix = FIRST ? 0ull : state->prefix;
+    const uint32_t now = FIRST ? *epoch : 0u;
+    const int above = shift + bits;             // bits above this digit are decided
+    const uint32_t mask = (1u << bits) - 1u;
+    const uint32_t n_quads = (C + 3u) >> 2;
+    const uint32_t n_round = (n_quads + 31u) & ~31u;    // whole warps stay together for the match
+    const uint32_t stride = gridDim.x * blockDim.x;
+    uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
+    uint4 nxt = make_uint4(0, 0, 0, 0);         // the keys one iteration ahead (later passes)
+    if (!FIRST && g < n_quads) nxt = reinterpret_cast<const uint4 *>(slot_key)[g];
+    for (; g < n_round; g += stride) {
+        uint32_t key[4] = {0, 0, 0, 0};
+        if (FIRST) {
+            if (g < n_quads) {
+                const uint4 a = __ldcs(reinterpret_cast<const uint4 *>(slot_stats) + 2 * g);
+                const uint4 b = __ldcs(reinterpret_cast<const uint4 *>(slot_stats) + 2 * g + 1);
+                const uint4 o = __ldcs(reinterpret_cast<const uint4 *>(slot_owner) + g);
+                key[0] = tfe_retention_key(make_uint2(a.x, a.y), o.x, now, half_life);
+                key[1] = tfe_retention_key(make_uint2(a.z, a.w), o.y, now, half_life);
+                key[2] = tfe_retention_key(make_uint2(b.x, b.y), o.z, now, half_life);
+                key[3] = tfe_retention_key(make_uint2(b.z, b.w), o.w, now, half_life);
+                reinterpret_cast<uint4 *>(slot_key)[g] = make_uint4(key[0], key[1], key[2], key[3]);
+            }
+        } else {
+            key[0] = nxt.x; key[1] = nxt.y; key[2] = nxt.z; key[3] = nxt.w;
+            if (g + stride < n_quads) nxt = reinterpret_cast<const uint4 *>(slot_key)[g + stride];
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t s0 = 4 * g + j;
+            const unsigned long long comp = ((unsigned long long)key[j] << 32) | s0;
+            const bool live = s0 < C && g < n_quads && (above >= 64 || (comp >> above) == (prefix >> above));
+            const uint32_t digit = (uint32_t)(comp >> shift) & mask;
+            // one shared-memory atomic per distinct digit of the warp
+            const uint32_t vote = __ballot_sync(0xFFFFFFFFu, live);
+            if (live) {
+                const uint32_t peers = __match_any_sync(vote, digit);
+                if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&s_hist[digit], __popc(peers));
+            }
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < TFE_VICTIM_BINS; i += blockDim.x)
+        if (s_hist[i]) atomicAdd(&hist[i], s_hist[i]);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(&state->ticket, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    // ---- last block: the digit whose bin holds the k_rem-th smallest
+    constexpr int PER = TFE_VICTIM_BINS / 256;
+    uint32_t mine[PER], sum = 0;
+    if (threadIdx.x < 256) {
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            mine[j] = __ldcg(hist + threadIdx.x * PER + j);
+            hist[threadIdx.x * PER + j] = 0;
+            sum += mine[j];
+        }
+        s_part[threadIdx.x] = sum;
+    }
+    __syncthreads();
+    // inclusive scan of the 256 partial sums by the first 8 warps, then the thread whose range
+    // holds the k-th smallest announces itself
+    const uint32_t k_want = FIRST ? n_first : state->k_rem;
+    uint32_t incl = 0;
+    if (threadIdx.x < 256) {
+        incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if ((threadIdx.x & 31) >= o) incl += v;
+        }
+        if ((threadIdx.x & 31) == 31) s_hist[threadIdx.x >> 5] = incl;      // warp totals
+    }
+    __syncthreads();
+    if (threadIdx.x < 256) {
+        for (int wq = 0; wq < (int)(threadIdx.x >> 5); ++wq) incl += s_hist[wq];
+        if (incl >= k_want && incl - sum < k_want) {
+            s_part[0] = threadIdx.x;                // owning thread (exactly one)
+            s_hist[8] = k_want - (incl - sum);      // rank within its bins
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < 256 && threadIdx.x == s_part[0]) {
+        uint32_t k = s_hist[8];
+        int j = 0;
+        for (; j < PER - 1 && mine[j] < k; ++j) k -= mine[j];
+        state->prefix = prefix | ((unsigned long long)(threadIdx.x * PER + j) << shift);
+        state->k_rem = k;
+        state->ticket = 0;
+    }
+}
+
+__global__ void __launch_bounds__(TFE_VICTIM_THREADS)
+tfe_victim_collect_kernel(const uint32_t *slot_key, uint32_t C, TfeVictimState *state, unsigned long long *list,
+                          uint32_t cap)
+{
+    const unsigned long long limit = state->prefix;
+    const uint32_t n_quads = (C + 3u) >> 2;
+    for (uint32_t g = blockIdx.x * blockDim.x + threadIdx.x; g < n_quads; g += gridDim.x * blockDim.x) {
+        const uint4 k4 = reinterpret_cast<const uint4 *>(slot_key)[g];
+        const uint32_t key[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t s0 = 4 * g + j;
+            const unsigned long long comp = ((unsigned long long)key[j] << 32) | s0;
+            if (s0 < C && comp <= limit) {
+                const uint32_t at = atomicAdd(&state->n_out, 1u);
+                if (at < cap) list[at] = comp;
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(1024)
+tfe_victim_sort_kernel(const unsigned long long *list, TfeVictimState *state, uint32_t n, int32_t *out_slots,
+                       uint32_t *out_keys)
+{
+    __shared__ unsigned long long s_v[TFE_VICTIMS_MAX];
+    uint32_t pow2 = 1;
+    while (pow2 < n) pow2 <<= 1;
+    for (uint32_t i = threadIdx.x; i < pow2; i += blockDim.x) s_v[i] = i < n ? list[i] : ~0ull;
+    __syncthreads();
+    for (uint32_t k = 2; k <= pow2; k <<= 1)
+        for (uint32_t j = k >> 1; j > 0; j >>= 1) {
+            for (uint32_t t = threadIdx.x; t < pow2 / 2; t += blockDim.x) {
+                const uint32_t i = ((t & ~(j - 1)) << 1) | (t & (j - 1));      // the pair's lower index
+                const uint32_t l = i | j;
+                const unsigned long long a = s_v[i], b = s_v[l];
+                const bool up = (i & k) == 0;
+                if ((a > b) == up) { s_v[i] = b; s_v[l] = a; }
+            }
+            __syncthreads();
+        }
+    for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) {
+        out_slots[i] = (int32_t)(uint32_t)s_v[i];
+        out_keys[i] = (uint32_t)(s_v[i] >> 32);
+    }
+    if (threadIdx.x == 0) state->n_out = 0;      // re-armed for the next selection
+}

@@ -92,6 +92,15 @@ class Engram:
     def cache_install(self, phrase_ids, src_rows, dst_slots, stream=None):
         tfe.tfe_cache_install(self.ctx, phrase_ids, src_rows, dst_slots, stream)
 
+    def cache_policy_enable(self, stream=None):
+        tfe.tfe_cache_policy_enable(self.ctx, stream)
+
+    def cache_select_victims(self, n, half_life=0, stream=None):
+        return tfe.tfe_cache_select_victims(self.ctx, n, half_life, stream)
+
+    def cache_stats(self, stream=None):
+        return tfe.tfe_cache_stats(self.ctx, self.C, stream)
+
 
 def bf16_tensor_from_bits(bits: np.ndarray, device) -> torch.Tensor:
     """uint16 bit patterns -> torch.bfloat16 tensor on ``device`` (no conversion)."""

@@ -1,0 +1,112 @@
+"""GPU-tier retention ranking (frequency / recency bookkeeping in the lookup kernels, victim
+selection) against the oracle's state machine, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_07388_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def H():
+    import parity_harness
+    return parity_harness
+
+
+def _compare_state(pr):
+    freq, last, epoch = pr.eng.cache_stats()
+    assert epoch == pr.ora.epoch
+    np.testing.assert_array_equal(freq, pr.ora.freq)
+    np.testing.assert_array_equal(last, pr.ora.last)
+
+
+def _compare_victims(pr, n, half_life):
+    slots, keys = pr.eng.cache_select_victims(n, half_life)
+    e_slots, e_keys = pr.ora.cache_victims(n, half_life)
+    np.testing.assert_array_equal(slots, e_slots)
+    np.testing.assert_array_equal(keys, e_keys)
+    return slots
+
+
+@pytest.mark.parametrize("policy", [0, 1])
+def test_bookkeeping_and_victims_follow_the_oracle(H, policy):
+    w = synth.config(1, B=6, T=300, n_phrases=30_000, gpu_slots=9_000, residency="hot_host", p=0.7,
+                     reserve_free=500)
+    tb, pr = H.pair_from_workload(w)
+    pr.eng.cache_policy_enable()
+    h = synth.make_hidden_np(w)
+    for step in range(5):
+        tok = synth.make_queries(w, tb, variant=step % 3)      # repeats make some slots hotter
+        g, ref, _ = pr.run_and_compare(tok, h, policy=policy, lam=1.0)
+        pr.ora.touch(ref)
+        _compare_state(pr)
+    assert pr.ora.freq.max() >= 3 and (pr.ora.freq > 0).sum() > 300
+    for n, hl in ((1, 0), (37, 0), (500, 0), (501, 1), (2000, 2), (4096, 0), (4096, 3)):
+        _compare_victims(pr, n, hl)
+    # install over the 64 worst slots (all free here), then over 64 occupied ones; state and ranking follow
+    res = pr.ora.lookup(tok, policy=policy)
+    want = np.unique(res.miss_phrase)[:128].astype(np.uint32)
+    assert len(want) == 128
+    for part in (want[:64], want[64:]):
+        if part is want[64:]:
+            dst = _compare_victims(pr, 700, 2)[-64:].copy()         # occupied, least worth keeping after the free ones
+            assert (pr.ora.slot_owner[dst] >= 0).all()
+        else:
+            dst = _compare_victims(pr, 64, 2).copy()
+            assert (pr.ora.slot_owner[dst] < 0).all()
+        src = synth.phrase_rows_np(w, part)
+        assert pr.ora.cache_install(part, src, dst) == 0
+        pr.eng.cache_install(part, src, dst)
+        _compare_state(pr)
+        g, ref, _ = pr.run_and_compare(tok, h, policy=policy, lam=1.0)
+        pr.ora.touch(ref)
+        _compare_state(pr)
+        _compare_victims(pr, 1000, 2)
+    pr.close()
+
+
+def test_policy_off_and_argument_checks(H):
+    from paper_2607_07388_b200 import binding as tfe
+    w = synth.config(1)
+    tb, pr = H.pair_from_workload(w)
+    with pytest.raises(tfe.TfeError):
+        pr.eng.cache_select_victims(4)             # bookkeeping not enabled
+    pr.eng.cache_policy_enable()
+    with pytest.raises(tfe.TfeError):
+        pr.eng.cache_select_victims(tfe.VICTIMS_MAX + 1)
+    slots, keys = pr.eng.cache_select_victims(0)
+    assert len(slots) == 0
+    # nothing looked up yet: every owned slot has freq 0, age 0 -> key 65535, ascending slot order
+    slots, keys = pr.eng.cache_select_victims(100)
+    np.testing.assert_array_equal(slots, np.arange(100))
+    assert (keys == 65535).all()
+    # enabling again clears the state
+    tok = synth.make_queries(w, tb)
+    g, ref, _ = pr.run_and_compare(tok, synth.make_hidden_np(w), lam=1.0)
+    assert pr.eng.cache_stats()[2] == 1
+    pr.eng.cache_policy_enable()
+    freq, last, epoch = pr.eng.cache_stats()
+    assert epoch == 0 and freq.sum() == 0 and last.sum() == 0
+    pr.close()
+
+
+def test_victims_more_than_slots_and_host_pipeline_epoch(H):
+    # fewer slots than requested: all of them come back, ranked; the piecewise host-buffer call
+    # counts as one lookup (one epoch) and bumps every injected slot once per hit
+    from paper_2607_07388_b200 import binding as tfe
+    w = synth.config(1, B=6, T=2731, d=1024, n_phrases=3_000, gpu_slots=1_500, residency="hot_host", p=0.6)
+    tb, pr = H.pair_from_workload(w)
+    pr.eng.cache_policy_enable()
+    tok = synth.make_queries(w, tb)
+    h = synth.make_hidden_np(w)
+    out = np.empty_like(h)
+    tfe.tfe_lookup_inject_host(pr.eng.ctx, tok, w.B, w.T, 0, h, out, lam=1.0)
+    torch.cuda.synchronize()
+    ref = pr.ora.lookup(tok)
+    pr.ora.touch(ref)
+    _compare_state(pr)
+    slots = _compare_victims(pr, 4096, 0)
+    assert len(slots) == 1500 and len(set(slots.tolist())) == 1500
+    pr.close()
