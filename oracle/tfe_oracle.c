@@ -20,6 +20,7 @@
  *   - insertion of fetched entries into the GPU tier          [Sec. 4.3, "inserts the entry into a faster tier"]
  *   - prefetch candidates from predicted tokens + priority     [Sec. 4.4, candidate set Q_t, score s = p r c]
  *   - retention ranking of GPU-tier slots (frequency, recency) [Sec. 4.3, cache policy signals]
+ *   - early-exit prefetch head: softmax(W_pref h), top-K        [Sec. 4.4, p_early and T_early equations]
  *
  * Parity pins: every function here is pinned by tests that do not call it to
  * produce their expected values (hand-made cases, closed forms, a library
@@ -559,4 +560,63 @@ int64_t orc_prefetch_candidates(int64_t N, const int32_t *phrase_tokens, const u
     }
     free(list);
     return n;
+}
+
+/* ------------------------------------------------ early-exit prefetch head */
+
+/* The auxiliary head at layer L-r turns the intermediate hidden state of every sequence into an
+ * approximate next-token distribution
+ *     p_early = softmax(W_pref h)            [Sec. 4.4, p_early equation]
+ * and keeps its K most likely tokens
+ *     T_early = TopK(p_early)                [Sec. 4.4, T_early equation].
+ * W_pref is [V][d], h is [B][d], both bf16 bit patterns; everything else in double.
+ *
+ * orc_head_logits: z[b][v] = sum_j W[v][j] * h[b][j], summed in ascending j. */
+void orc_head_logits(int32_t V, int32_t d, int32_t B, const uint16_t *W, const uint16_t *h, double *z)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t v = 0; v < V; ++v)
+        for (int32_t b = 0; b < B; ++b) {
+            double acc = 0.0;
+            for (int32_t j = 0; j < d; ++j)
+                acc += orc_bf16_to_double(W[(size_t)v * d + j]) * orc_bf16_to_double(h[(size_t)b * d + j]);
+            z[(size_t)b * V + v] = acc;
+        }
+}
+
+/* orc_head_topk: for every row of z the softmax over all V entries (with the usual subtraction of
+ * the row maximum, which cancels) and the K entries of largest probability, in descending
+ * probability; equal logits keep ascending token id.  tokens [B][K], prob [B][K]; lse[b] receives
+ * log(sum_v exp(z[b][v])) when lse is not NULL.  K <= V. */
+typedef struct { double z; int32_t v; } orc_logit;
+
+static int logit_cmp(const void *pa, const void *pb)
+{
+    const orc_logit *a = (const orc_logit *)pa, *b = (const orc_logit *)pb;
+    if (a->z != b->z) return a->z > b->z ? -1 : 1;
+    return a->v < b->v ? -1 : (a->v > b->v ? 1 : 0);
+}
+
+void orc_head_topk(int32_t V, int32_t B, int32_t K, const double *z, int32_t *tokens, double *prob, double *lse)
+{
+#pragma omp parallel for schedule(static)
+    for (int32_t b = 0; b < B; ++b) {
+        const double *row = z + (size_t)b * V;
+        orc_logit *r = (orc_logit *)malloc((size_t)V * sizeof *r);
+        double top = row[0];
+        for (int32_t v = 0; v < V; ++v) {
+            r[v].z = row[v];
+            r[v].v = v;
+            if (row[v] > top) top = row[v];
+        }
+        double sum = 0.0;
+        for (int32_t v = 0; v < V; ++v) sum += exp(row[v] - top);
+        qsort(r, (size_t)V, sizeof *r, logit_cmp);
+        for (int32_t k = 0; k < K; ++k) {
+            tokens[(size_t)b * K + k] = r[k].v;
+            prob[(size_t)b * K + k] = exp(r[k].z - top) / sum;
+        }
+        if (lse) lse[b] = top + log(sum);
+        free(r);
+    }
 }

@@ -232,3 +232,24 @@ class Oracle:
             C.c_float(benefit_host), C.c_float(benefit_ssd), C.c_int32(budget), _p(op), _p(ot), _p(osc), _p(osr))
         n = int(min(total, budget))
         return op[:n].copy(), ot[:n].copy(), osc[:n].copy(), osr[:n].copy(), int(total)
+
+
+# -- early-exit prefetch head (independent of any phrase table) ---------------------------------
+def head_logits(W, h) -> np.ndarray:
+    """float64 [B, V]: W_pref h for bf16 bit patterns W [V, d], h [B, d]."""
+    W, h = _c(W, np.uint16), _c(h, np.uint16)
+    V, d = W.shape
+    B = h.shape[0]
+    assert h.shape[1] == d
+    z = np.empty((B, V), np.float64)
+    lib().orc_head_logits(C.c_int32(V), C.c_int32(d), C.c_int32(B), _p(W), _p(h), _p(z))
+    return z
+
+
+def head_topk(z, K):
+    """(tokens int32 [B, K], prob float64 [B, K], lse float64 [B]) of softmax over each row of z."""
+    z = _c(z, np.float64)
+    B, V = z.shape
+    tokens, prob, lse = np.empty((B, K), np.int32), np.empty((B, K), np.float64), np.empty(B, np.float64)
+    lib().orc_head_topk(C.c_int32(V), C.c_int32(B), C.c_int32(K), _p(z), _p(tokens), _p(prob), _p(lse))
+    return tokens, prob, lse

@@ -646,3 +646,70 @@ def test_retention_against_independent_restatement(oracle_mod):
         slots, keys = o.cache_victims(700, half_life=hl)
         np.testing.assert_array_equal(slots, order[:700])
         np.testing.assert_array_equal(keys, key[order[:700]].astype(np.uint32))
+
+
+# ---------------------------------------------------------------- early-exit prefetch head (Sec. 4.4)
+
+def test_head_hand_worked(oracle_mod):
+    # W rows pick out single coordinates of h, so the logits are the entries of h: ln 1 .. ln 4 (rounded
+    # to bf16) and the distribution is (almost) 0.1, 0.2, 0.3, 0.4
+    lg = unbf(bf(np.log([1.0, 2.0, 3.0, 4.0])))
+    W = bf(np.eye(4))
+    h = bf(np.log([[1.0, 2.0, 3.0, 4.0]]))
+    z = oracle_mod.head_logits(W, h)
+    np.testing.assert_array_equal(z, lg[None, :])
+    tok, prob, lse = oracle_mod.head_topk(z, 3)
+    np.testing.assert_array_equal(tok, [[3, 2, 1]])
+    expect = np.exp(lg) / np.exp(lg).sum()
+    np.testing.assert_allclose(prob[0], expect[[3, 2, 1]], rtol=1e-14)
+    np.testing.assert_allclose(prob[0], [0.4, 0.3, 0.2], atol=2e-3)       # bf16 rounding of the logs
+    np.testing.assert_allclose(lse[0], np.log(np.exp(lg).sum()), rtol=1e-14)
+
+
+def test_head_against_library_routines(oracle_mod):
+    rng = np.random.default_rng(3)
+    V, d, B, K = 3000, 96, 5, 17
+    W = bf(rng.standard_normal((V, d)) * 0.3)
+    h = bf(rng.standard_normal((B, d)))
+    z = oracle_mod.head_logits(W, h)
+    zt = torch.from_numpy(unbf(h)) @ torch.from_numpy(unbf(W)).T                 # float64 matmul
+    np.testing.assert_allclose(z, zt.numpy(), rtol=0, atol=1e-12)
+    tok, prob, lse = oracle_mod.head_topk(z, K)
+    p = torch.softmax(torch.from_numpy(z), dim=1)
+    pv, pi = torch.topk(p, K, dim=1)
+    np.testing.assert_array_equal(tok, pi.numpy())
+    np.testing.assert_allclose(prob, pv.numpy(), rtol=1e-12)
+    np.testing.assert_allclose(lse, torch.logsumexp(torch.from_numpy(z), dim=1).numpy(), rtol=1e-13)
+    # all of it sums to one
+    _, pall, _ = oracle_mod.head_topk(z, V)
+    np.testing.assert_allclose(pall.sum(axis=1), 1.0, rtol=1e-12)
+
+
+def test_head_invariants(oracle_mod):
+    rng = np.random.default_rng(4)
+    V, d = 500, 32
+    W = bf(rng.standard_normal((V, d)))
+    h = bf(rng.standard_normal((3, d)))
+    z = oracle_mod.head_logits(W, h)
+    tok, prob, _ = oracle_mod.head_topk(z, 8)
+    # h = 0: uniform distribution, ties resolved by ascending token id
+    t0, p0, l0 = oracle_mod.head_topk(oracle_mod.head_logits(W, np.zeros((1, d), np.uint16)), 5)
+    np.testing.assert_array_equal(t0, [[0, 1, 2, 3, 4]])
+    np.testing.assert_allclose(p0, 1.0 / V, rtol=1e-14)
+    np.testing.assert_allclose(l0, np.log(V), rtol=1e-14)
+    # permuting the rows of W permutes the token ids and nothing else
+    perm = rng.permutation(V)
+    tp, pp, _ = oracle_mod.head_topk(oracle_mod.head_logits(W[perm], h), 8)
+    np.testing.assert_array_equal(perm[tp], tok)
+    np.testing.assert_allclose(pp, prob, rtol=1e-12)        # the sum runs in another order
+    # a constant added to every logit changes no probability
+    t2, p2, _ = oracle_mod.head_topk(z + 7.5, 8)
+    np.testing.assert_array_equal(t2, tok)
+    np.testing.assert_allclose(p2, prob, rtol=1e-12)
+    # duplicate rows of W tie exactly: the lower id comes first
+    W2 = W.copy(); W2[10] = W2[400]
+    z2 = oracle_mod.head_logits(W2, h)
+    t3, _, _ = oracle_mod.head_topk(z2, V)
+    for b in range(3):
+        pos = {int(v): i for i, v in enumerate(t3[b])}
+        assert pos[400] == pos[10] + 1
