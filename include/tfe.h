@@ -322,6 +322,43 @@ tfe_status tfe_launch_geometry(const tfe_ctx *ctx, int32_t *grid, int32_t *block
  */
 tfe_status tfe_set_tuning(tfe_ctx *ctx, int32_t batch_queries);
 
+/*
+ * Early-exit prefetch head (paper Sec. 4.4): p_early(x_{t+1} | x_<=t) = softmax(W_pref h_t^{L-r})
+ * and T_early = TopK(p_early) -- the K most likely next tokens of every sequence with their
+ * probabilities, which are the inputs of tfe_prefetch_candidates.  The only dense contraction of
+ * the method; it runs on the tensor cores.  A head is independent of any phrase index.
+ *
+ * tfe_head_create -- w_pref DEVICE bf16 [V][d] row-major, 16-byte aligned, CALLER-OWNED and read
+ * in place by every call (it must outlive the head); d a multiple of 64; max_batch 1..256.
+ * Allocates the logits buffer (max_batch * V * 4 bytes) and small work areas on the current
+ * device.  Errors: INVALID_ARG, CUDA.
+ */
+typedef struct tfe_head tfe_head;
+tfe_status tfe_head_create(const void *w_pref, int32_t V, int32_t d, int32_t max_batch, tfe_head **out);
+void       tfe_head_destroy(tfe_head *head);
+
+/*
+ * tfe_head_topk -- hidden DEVICE bf16 [B][d] (16-byte aligned), 0 <= B <= max_batch, 1 <= K <= 128,
+ * K <= V.  Outputs DEVICE: cand_tokens int32 [B][K], cand_prob float [B][K], per sequence in
+ * descending probability, equal logits in ascending token id.  Logits are bf16 products
+ * accumulated in fp32 (tensor cores); selection and softmax in fp32.  Asynchronous on `stream`,
+ * three kernel launches, never synchronises.  Errors: INVALID_ARG, CUDA, INTERNAL.
+ */
+tfe_status tfe_head_topk(tfe_head *head, const void *hidden, int32_t B, int32_t K, int32_t *cand_tokens,
+                         float *cand_prob, void *stream);
+
+/* DEVICE views of the most recent call: logits fp32 [B][ld] and log-sum-exp fp32 [B]; owned by the head. */
+tfe_status tfe_head_buffers(tfe_head *head, const float **logits, int64_t *ld, const float **lse);
+
+/*
+ * tfe_head_status -- synchronises `stream` and reads the device status word: 0, or a bit set by a
+ * wait inside the kernel that ran out (1 loader, 2 MMA issuer, 4 epilogue); then INTERNAL.
+ */
+tfe_status tfe_head_status(tfe_head *head, uint32_t *device_flags, void *stream);
+
+/* Launch geometry: CTAs, vocabulary rows per CTA, rows of each CTA's short last tile. */
+tfe_status tfe_head_geometry(const tfe_head *head, int32_t *grid, int32_t *rows_per_cta, int32_t *tail_rows);
+
 #ifdef __cplusplus
 }
 #endif

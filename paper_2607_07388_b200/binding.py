@@ -33,7 +33,8 @@ EXPORTS = ["tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_loo
            "tfe_last_cuda_error", "tfe_index_geometry", "tfe_phrase_key64", "tfe_home_bucket",
            "tfe_launch_geometry", "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
            "tfe_cache_policy_enable", "tfe_cache_select_victims", "tfe_cache_select_victims_device",
-           "tfe_cache_stats"]
+           "tfe_cache_stats", "tfe_head_create", "tfe_head_destroy", "tfe_head_topk", "tfe_head_buffers",
+           "tfe_head_status", "tfe_head_geometry"]
 
 
 class TfeConfig(C.Structure):
@@ -98,11 +99,19 @@ def lib() -> C.CDLL:
         L.tfe_cache_select_victims.argtypes = [vp, i32, i32, vp, vp, C.POINTER(i32), vp]
         L.tfe_cache_select_victims_device.argtypes = [vp, C.POINTER(vp), C.POINTER(vp)]
         L.tfe_cache_stats.argtypes = [vp, vp, C.POINTER(C.c_uint32), vp]
+        L.tfe_head_create.argtypes = [vp, i32, i32, i32, C.POINTER(vp)]
+        L.tfe_head_destroy.argtypes = [vp]
+        L.tfe_head_destroy.restype = None
+        L.tfe_head_topk.argtypes = [vp, vp, i32, i32, vp, vp, vp]
+        L.tfe_head_buffers.argtypes = [vp, C.POINTER(vp), C.POINTER(i64), C.POINTER(vp)]
+        L.tfe_head_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+        L.tfe_head_geometry.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
         for name in ("tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
                      "tfe_miss_list", "tfe_miss_list_device", "tfe_index_geometry", "tfe_launch_geometry",
                      "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
                      "tfe_cache_policy_enable", "tfe_cache_select_victims", "tfe_cache_select_victims_device",
-                     "tfe_cache_stats"):
+                     "tfe_cache_stats", "tfe_head_create", "tfe_head_topk", "tfe_head_buffers", "tfe_head_status",
+                     "tfe_head_geometry"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -299,3 +308,45 @@ def tfe_phrase_key64(vocab: int, tokens) -> tuple[int, bool]:
 
 def tfe_home_bucket(key: int, n_buckets: int) -> int:
     return int(lib().tfe_home_bucket(key, n_buckets))
+
+
+# -- early-exit prefetch head -------------------------------------------------------------------
+HEAD_MAX_K = 128
+HEAD_MAX_BATCH = 256
+
+
+def tfe_head_create(w_pref, V: int, d: int, max_batch: int) -> int:
+    out = C.c_void_p()
+    _check(lib().tfe_head_create(_addr(w_pref), int(V), int(d), int(max_batch), C.byref(out)), "tfe_head_create")
+    return out.value
+
+
+def tfe_head_destroy(head: int) -> None:
+    lib().tfe_head_destroy(head)
+
+
+def tfe_head_topk(head: int, hidden, B: int, K: int, cand_tokens, cand_prob, stream=None) -> None:
+    _check(lib().tfe_head_topk(head, _addr(hidden), int(B), int(K), _addr(cand_tokens), _addr(cand_prob),
+                               _stream(stream)), "tfe_head_topk")
+
+
+def tfe_head_buffers(head: int):
+    """Device addresses (logits fp32 [B][ld], ld, lse fp32 [B]) of the most recent call."""
+    a, ld, b = C.c_void_p(), C.c_int64(0), C.c_void_p()
+    _check(lib().tfe_head_buffers(head, C.byref(a), C.byref(ld), C.byref(b)), "tfe_head_buffers")
+    return a.value, ld.value, b.value
+
+
+def tfe_head_status(head: int, stream=None) -> int:
+    """Synchronises; returns the device status word (0 = no wait ran out)."""
+    flags = C.c_uint32(0)
+    st = lib().tfe_head_status(head, C.byref(flags), _stream(stream))
+    if st not in (TFE_OK, TFE_ERR_INTERNAL):
+        _check(st, "tfe_head_status")
+    return flags.value
+
+
+def tfe_head_geometry(head: int):
+    g, r, t = C.c_int32(0), C.c_int32(0), C.c_int32(0)
+    _check(lib().tfe_head_geometry(head, C.byref(g), C.byref(r), C.byref(t)), "tfe_head_geometry")
+    return g.value, r.value, t.value

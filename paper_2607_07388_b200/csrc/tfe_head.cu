@@ -1,0 +1,649 @@
+// Early-exit prefetch head (paper Sec. 4.4): p_early = softmax(W_pref h), T_early = TopK(p_early).
+//
+// The only dense contraction of the method: logits[b][v] = sum_j W_pref[v][j] * h[b][j] with
+// V ~ 150 k vocabulary rows, d ~ 1 k and a decode batch of B <= 256 hidden states.  W_pref (V*d*2
+// bytes, ~311 MB) is read once per call and is what bounds the call (HBM); the arithmetic only
+// keeps up on the tensor cores, so the product runs as tcgen05 MMAs:
+//
+//   tfe_head_gemm_kernel     persistent, one CTA per SM, warp-specialised.  Every CTA owns a
+//                            contiguous range of vocabulary rows and walks it in tiles of 128 rows
+//                            (the MMA's M); the batch is the MMA's N.  Warp 0 streams W tiles and
+//                            the matching k-slice of h through a ring of shared-memory stages with
+//                            TMA (128-byte swizzle), warp 1 issues tcgen05.mma (M=128, N=batch
+//                            padded to 16, K=16 per instruction, fp32 accumulators in tensor
+//                            memory, two accumulators so that a tile's epilogue overlaps the next
+//                            tile's MMAs), warps 2-5 read finished accumulators with tcgen05.ld and
+//                            store fp32 logits [B][V].  All mbarrier waits are bounded.
+//   tfe_head_partial_kernel  grid (segments, B): softmax statistics (max, sum of exponentials) and
+//                            the K largest logits of one segment of one row (radix selection in
+//                            shared memory).
+//   tfe_head_merge_kernel    one block per row: merges the segments' candidates, sorts the best K
+//                            (descending logit, equal logits ascending token id) and turns them
+//                            into probabilities exp(z - logsumexp).
+//
+// The logits make a round trip through global memory (B*V*4 bytes, 39 MB for B = 64); they are
+// written and re-read within microseconds and stay in the 126 MB L2 for the batch sizes of decode.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdint>
+#include <cstring>
+
+#include "../../include/tfe.h"
+
+#define HEAD_TILE_M 128             // vocabulary rows per tile (MMA M)
+#define HEAD_TILE_K 64              // bf16 elements per stage along d: one 128-byte swizzle row
+#define HEAD_UMMA_K 16              // bf16 elements per tcgen05.mma
+#define HEAD_MAX_N 256              // batch columns (MMA N)
+#define HEAD_THREADS 192            // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+#define HEAD_MAX_STAGES 8
+#define HEAD_MAX_K 128              // top-K limit
+#define HEAD_SEGMENTS 8             // segments per row in the selection
+#define HEAD_SEL_THREADS 512
+#define HEAD_WAIT_LIMIT (1u << 22)  // polls of one mbarrier before a wait gives up
+
+// device status bits
+#define HEAD_ST_TIMEOUT_PRODUCER 1u
+#define HEAD_ST_TIMEOUT_MMA 2u
+#define HEAD_ST_TIMEOUT_EPILOGUE 4u
+
+namespace {
+
+// ------------------------------------------------------------------ PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after HEAD_WAIT_LIMIT polls or when another role has given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
+{
+    for (uint32_t i = 0; i < HEAD_WAIT_LIMIT; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 1023u) == 1023u && *abort_flag) return false;
+    }
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int32_t x, int32_t y,
+                                            uint64_t hint)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4}], [%2], %5;"
+        :
+        : "r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y), "l"(hint)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate; issued by one thread.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        :
+        : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The mbarrier receives one arrival when every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 16 consecutive fp32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory operand descriptor, K-major tile whose rows are 128 bytes (64 bf16) and were
+// written by TMA with the 128-byte swizzle: rows 128 B apart, groups of 8 rows 1024 B apart.
+// Fields: start address >> 4 [0,14); leading byte offset >> 4 [16,30) (unused with a swizzle,
+// 1); stride byte offset >> 4 [32,46) = 64; descriptor version [46,48) = 1; swizzle mode
+// [61,64) = 2 (128 bytes).
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr)
+{
+    uint64_t d = (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// Instruction descriptor of kind::f16: D fp32 (bits [4,6) = 1), A and B bf16 ([7,10) = [10,13) = 1),
+// both K-major (bits 15, 16 = 0), N >> 3 at [17,23), M >> 4 at [24,29).
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(uint32_t M, uint32_t N)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+// ------------------------------------------------------------------ GEMM
+
+struct HeadGemmParams {
+    int32_t V, d, B;
+    int32_t N;                      // B rounded up to 16
+    int32_t rows_per_cta;           // multiple of 8
+    int32_t tail_rows;              // rows_per_cta % 128: rows of every CTA's last, short tile (0: none)
+    int32_t stages;
+    uint32_t tmem_cols;             // power of two >= 2 N
+    float *logits;                  // [B][ld]
+    int64_t ld;
+    uint32_t *status;
+};
+
+__global__ void __launch_bounds__(HEAD_THREADS, 1)
+tfe_head_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w_tail,
+                     const __grid_constant__ CUtensorMap map_h, const HeadGemmParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t s_full[HEAD_MAX_STAGES], s_empty[HEAD_MAX_STAGES], s_acc_full[2], s_acc_empty[2];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ volatile uint32_t s_abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t stage_bytes = HEAD_TILE_M * 128u + (uint32_t)p.N * 128u;
+    const uint32_t smem_base = smem_u32(smem);
+
+    // this CTA's vocabulary rows and tiles
+    const int64_t r0 = (int64_t)blockIdx.x * p.rows_per_cta;
+    const int64_t r1 = min((int64_t)p.V, r0 + (int64_t)p.rows_per_cta);
+    const int32_t n_rows = (int32_t)max((int64_t)0, r1 - r0);
+    const int32_t n_tiles = (n_rows + HEAD_TILE_M - 1) / HEAD_TILE_M;
+    const int32_t num_kb = p.d / HEAD_TILE_K;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&s_full[s]), 1); mbar_init(smem_u32(&s_empty[s]), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&s_acc_full[a]), 1); mbar_init(smem_u32(&s_acc_empty[a]), 4); }
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&s_tmem_base), p.tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = s_tmem_base;
+
+    if (warp == 0) {
+        // ============================ TMA producer ============================
+        if (lane == 0) {
+            const uint64_t hint_stream = 0x12F0000000000000ull;     // evict first: W is read once
+            const uint64_t hint_keep = 0x14F0000000000000ull;       // evict last: h is read by every tile
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int32_t t = 0; t < n_tiles && ok; ++t) {
+                const int32_t row0 = (int32_t)r0 + t * HEAD_TILE_M;
+                const int32_t valid = min(HEAD_TILE_M, n_rows - t * HEAD_TILE_M);
+                // a short last tile is fetched with the short box, so no row of the next CTA is read
+                const bool use_tail = valid < HEAD_TILE_M && valid == p.tail_rows;
+                const uint32_t w_bytes = use_tail ? (uint32_t)p.tail_rows * 128u : HEAD_TILE_M * 128u;
+                for (int32_t kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, &s_abort)) {
+                        atomicOr(p.status, HEAD_ST_TIMEOUT_PRODUCER);
+                        s_abort = 1;
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t bar = smem_u32(&s_full[stage]);
+                    const uint32_t dst = smem_base + stage * stage_bytes;
+                    mbar_expect_tx(bar, w_bytes + (uint32_t)p.N * 128u);
+                    tma_load_2d(dst, use_tail ? &map_w_tail : &map_w, bar, kb * HEAD_TILE_K, row0, hint_stream);
+                    tma_load_2d(dst + HEAD_TILE_M * 128u, &map_h, bar, kb * HEAD_TILE_K, 0, hint_keep);
+                    if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ============================ MMA issuer ==============================
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16(HEAD_TILE_M, (uint32_t)p.N);
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int32_t t = 0; t < n_tiles && ok; ++t) {
+                const uint32_t acc = (uint32_t)t & 1u, acc_phase = ((uint32_t)t >> 1) & 1u;
+                if (!mbar_wait(smem_u32(&s_acc_empty[acc]), acc_phase ^ 1u, &s_abort)) {
+                    atomicOr(p.status, HEAD_ST_TIMEOUT_MMA);
+                    s_abort = 1;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)p.N;
+                for (int32_t kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(smem_u32(&s_full[stage]), phase, &s_abort)) {
+                        atomicOr(p.status, HEAD_ST_TIMEOUT_MMA);
+                        s_abort = 1;
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_base + stage * stage_bytes;
+                    const uint64_t a_desc = umma_desc_sw128(a_addr);
+                    const uint64_t b_desc = umma_desc_sw128(a_addr + HEAD_TILE_M * 128u);
+#pragma unroll
+                    for (int k = 0; k < HEAD_TILE_K / HEAD_UMMA_K; ++k) {
+                        // 16 bf16 = 32 bytes further along the swizzled row: +2 in the address field
+                        umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                  (kb > 0 || k > 0) ? 1u : 0u);
+                    }
+                    umma_commit(smem_u32(&s_empty[stage]));         // the stage is free when these MMAs are done
+                    if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(smem_u32(&s_acc_full[acc]));    // the accumulator is complete
+            }
+        }
+    } else {
+        // ============================ epilogue ================================
+        const uint32_t quarter = (uint32_t)warp & 3u;               // tensor-memory lanes 32*quarter .. +31
+        for (int32_t t = 0; t < n_tiles; ++t) {
+            const uint32_t acc = (uint32_t)t & 1u, acc_phase = ((uint32_t)t >> 1) & 1u;
+            if (!mbar_wait(smem_u32(&s_acc_full[acc]), acc_phase, &s_abort)) {
+                if (lane == 0) atomicOr(p.status, HEAD_ST_TIMEOUT_EPILOGUE);
+                s_abort = 1;
+                break;
+            }
+            tc_fence_after();
+            const int32_t valid = min(HEAD_TILE_M, n_rows - t * HEAD_TILE_M);
+            const int32_t row_in_tile = (int32_t)(quarter * 32u) + lane;
+            const int64_t row = r0 + (int64_t)t * HEAD_TILE_M + row_in_tile;
+            const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + acc * (uint32_t)p.N;
+            for (int32_t c0 = 0; c0 < p.N; c0 += 16) {
+                uint32_t v[16];
+                tmem_ld16(taddr + (uint32_t)c0, v);
+                tmem_ld_wait();
+                if (row_in_tile < valid) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (c0 + j < p.B) p.logits[(int64_t)(c0 + j) * p.ld + row] = __uint_as_float(v[j]);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty[acc]));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, p.tmem_cols);
+    }
+}
+
+// ------------------------------------------------------------------ selection
+
+// fp32 -> uint32 whose unsigned order is the float order (NaN sorts above +inf; not produced here)
+__device__ __forceinline__ uint32_t orderable(float x)
+{
+    const uint32_t u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float from_orderable(uint32_t k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
+}
+
+struct HeadSelParams {
+    const float *logits;
+    int64_t ld;
+    int32_t V, B, K;
+    int32_t seg_len;                // multiple of 4
+    float *seg_max, *seg_sum;       // [B][HEAD_SEGMENTS]
+    unsigned long long *seg_cand;   // [B][HEAD_SEGMENTS][K]: orderable(z) << 32 | ~token, 0 = none
+    int32_t *out_tokens;            // [B][K]
+    float *out_prob;                // [B][K]
+    float *out_lse;                 // [B] or nullptr
+};
+
+// One segment of one row: max, sum of exp(z - max), and the K candidates of largest
+// (logit, then smaller token id): distinct 64-bit keys, so a radix selection needs no tie rule.
+__global__ void __launch_bounds__(HEAD_SEL_THREADS)
+tfe_head_partial_kernel(const HeadSelParams p)
+{
+    extern __shared__ float s_z[];                  // seg_len logits
+    __shared__ uint32_t s_hist[256];
+    __shared__ float s_red[HEAD_SEL_THREADS / 32];
+    __shared__ unsigned long long s_prefix;
+    __shared__ uint32_t s_want, s_fill;
+    const int seg = blockIdx.x, b = blockIdx.y;
+    const int32_t v0 = seg * p.seg_len;
+    const int32_t n = max(0, min(p.seg_len, p.V - v0));
+    const float *row = p.logits + (int64_t)b * p.ld + v0;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    float mx = -INFINITY;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const float z = __ldcs(row + i);
+        s_z[i] = z;
+        mx = fmaxf(mx, z);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+    if (lane == 0) s_red[warp] = mx;
+    __syncthreads();
+    mx = s_red[0];
+    for (int w = 1; w < HEAD_SEL_THREADS / 32; ++w) mx = fmaxf(mx, s_red[w]);
+    __syncthreads();
+    float sum = 0.f;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) sum += __expf(s_z[i] - mx);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+    if (lane == 0) s_red[warp] = sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int w = 0; w < HEAD_SEL_THREADS / 32; ++w) t += s_red[w];
+        p.seg_max[b * HEAD_SEGMENTS + seg] = mx;
+        p.seg_sum[b * HEAD_SEGMENTS + seg] = n > 0 ? t : 0.f;
+        s_prefix = 0;
+        s_want = (uint32_t)min(p.K, n);
+        s_fill = 0;
+    }
+    unsigned long long *cand = p.seg_cand + ((int64_t)b * HEAD_SEGMENTS + seg) * p.K;
+    for (int i = threadIdx.x; i < p.K; i += blockDim.x) cand[i] = 0ull;
+    __syncthreads();
+    const uint32_t take = s_want;
+    if (take == 0) return;
+    // ---- the take-th largest key, most significant byte first
+    for (int shift = 56; shift >= 0; shift -= 8) {
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) s_hist[i] = 0;
+        __syncthreads();
+        const unsigned long long prefix = s_prefix;
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            const unsigned long long key = ((unsigned long long)orderable(s_z[i]) << 32) | (uint32_t)~(uint32_t)(v0 + i);
+            if (shift == 56 || (key >> (shift + 8)) == (prefix >> (shift + 8)))
+                atomicAdd(&s_hist[(uint32_t)(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t want = s_want;
+            int dgt = 255;
+            for (; dgt > 0 && s_hist[dgt] < want; --dgt) want -= s_hist[dgt];
+            s_prefix = prefix | ((unsigned long long)dgt << shift);
+            s_want = want;
+        }
+        __syncthreads();
+    }
+    const unsigned long long kth = s_prefix;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const unsigned long long key = ((unsigned long long)orderable(s_z[i]) << 32) | (uint32_t)~(uint32_t)(v0 + i);
+        if (key >= kth) {
+            const uint32_t at = atomicAdd(&s_fill, 1u);
+            if (at < (uint32_t)p.K) cand[at] = key;
+        }
+    }
+}
+
+// One row: sort the segments' candidates, keep the best K, normalise.
+__global__ void __launch_bounds__(HEAD_SEL_THREADS)
+tfe_head_merge_kernel(const HeadSelParams p)
+{
+    __shared__ unsigned long long s_v[HEAD_SEGMENTS * HEAD_MAX_K];
+    __shared__ float s_lse;
+    const int b = blockIdx.x;
+    const uint32_t n = (uint32_t)(HEAD_SEGMENTS * p.K);
+    uint32_t pow2 = 1;
+    while (pow2 < n) pow2 <<= 1;
+    const unsigned long long *cand = p.seg_cand + (int64_t)b * HEAD_SEGMENTS * p.K;
+    for (uint32_t i = threadIdx.x; i < pow2; i += blockDim.x) s_v[i] = i < n ? cand[i] : 0ull;
+    if (threadIdx.x == 0) {
+        float m = -INFINITY;
+        for (int s = 0; s < HEAD_SEGMENTS; ++s)
+            if (p.seg_sum[b * HEAD_SEGMENTS + s] > 0.f) m = fmaxf(m, p.seg_max[b * HEAD_SEGMENTS + s]);
+        float t = 0.f;
+        for (int s = 0; s < HEAD_SEGMENTS; ++s)
+            if (p.seg_sum[b * HEAD_SEGMENTS + s] > 0.f)
+                t += p.seg_sum[b * HEAD_SEGMENTS + s] * __expf(p.seg_max[b * HEAD_SEGMENTS + s] - m);
+        s_lse = m + __logf(t);
+        if (p.out_lse) p.out_lse[b] = s_lse;
+    }
+    __syncthreads();
+    // bitonic sort, descending
+    for (uint32_t k = 2; k <= pow2; k <<= 1)
+        for (uint32_t j = k >> 1; j > 0; j >>= 1) {
+            for (uint32_t t = threadIdx.x; t < pow2 / 2; t += blockDim.x) {
+                const uint32_t i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+                const uint32_t l = i | j;
+                const unsigned long long a = s_v[i], c = s_v[l];
+                const bool down = (i & k) == 0;
+                if ((a < c) == down) { s_v[i] = c; s_v[l] = a; }
+            }
+            __syncthreads();
+        }
+    const float lse = s_lse;
+    for (int i = threadIdx.x; i < p.K; i += blockDim.x) {
+        const unsigned long long key = s_v[i];
+        int32_t tok = -1;
+        float pr = 0.f;
+        if (key != 0ull) {
+            tok = (int32_t)~(uint32_t)key;
+            pr = __expf(from_orderable((uint32_t)(key >> 32)) - lse);
+        }
+        p.out_tokens[(int64_t)b * p.K + i] = tok;
+        p.out_prob[(int64_t)b * p.K + i] = pr;
+    }
+}
+
+// ------------------------------------------------------------------ host side
+
+typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+encode_tiled_fn get_encode_tiled()
+{
+    static encode_tiled_fn fn = nullptr;
+    if (!fn) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<encode_tiled_fn>(sym);
+    }
+    return fn;
+}
+
+// bf16 matrix [rows][cols] row-major, box = 64 columns x box_rows rows, 128-byte swizzle
+bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows)
+{
+    encode_tiled_fn enc = get_encode_tiled();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {HEAD_TILE_K, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+struct tfe_head {
+    const void *w = nullptr;
+    int32_t V = 0, d = 0, max_batch = 0;
+    int device = 0, sm_count = 0;
+    int32_t rows_per_cta = 0, tail_rows = 0, grid = 0;
+    CUtensorMap map_w, map_w_tail;
+    float *d_logits = nullptr;
+    int64_t ld = 0;
+    float *d_seg_max = nullptr, *d_seg_sum = nullptr, *d_lse = nullptr;
+    unsigned long long *d_seg_cand = nullptr;
+    uint32_t *d_status = nullptr;
+    int32_t seg_len = 0;
+};
+
+extern "C" {
+
+tfe_status tfe_head_create(const void *w_pref, int32_t V, int32_t d, int32_t max_batch, tfe_head **out)
+{
+    if (!out) return TFE_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!w_pref || V < 1 || d < HEAD_TILE_K || d % HEAD_TILE_K != 0 || max_batch < 1 || max_batch > HEAD_MAX_N)
+        return TFE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(w_pref) & 15u) != 0) return TFE_ERR_INVALID_ARG;
+    tfe_head *h = new tfe_head();
+    auto fail = [&](tfe_status st) { tfe_head_destroy(h); return st; };
+    h->w = w_pref; h->V = V; h->d = d; h->max_batch = max_batch;
+    if (cudaGetDevice(&h->device) != cudaSuccess) return fail(TFE_ERR_CUDA);
+    if (cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess)
+        return fail(TFE_ERR_CUDA);
+    // contiguous row ranges of equal size (a multiple of 8) per CTA
+    const int32_t ctas = std::max(1, std::min(h->sm_count, (V + HEAD_TILE_M - 1) / HEAD_TILE_M));
+    h->rows_per_cta = (int32_t)((((int64_t)V + ctas - 1) / ctas + 7) / 8 * 8);
+    h->grid = (int32_t)(((int64_t)V + h->rows_per_cta - 1) / h->rows_per_cta);
+    h->tail_rows = h->rows_per_cta % HEAD_TILE_M;
+    if (!make_map(&h->map_w, w_pref, (uint64_t)V, (uint64_t)d, HEAD_TILE_M)) return fail(TFE_ERR_CUDA);
+    if (!make_map(&h->map_w_tail, w_pref, (uint64_t)V, (uint64_t)d, h->tail_rows ? (uint32_t)h->tail_rows : 8u))
+        return fail(TFE_ERR_CUDA);
+    h->ld = ((int64_t)V + 3) / 4 * 4;
+    h->seg_len = (int32_t)((((int64_t)V + HEAD_SEGMENTS - 1) / HEAD_SEGMENTS + 3) / 4 * 4);
+    const size_t nb = (size_t)max_batch;
+    if (cudaMalloc(&h->d_logits, nb * (size_t)h->ld * sizeof(float)) != cudaSuccess) return fail(TFE_ERR_CUDA);
+    if (cudaMalloc(&h->d_seg_max, nb * HEAD_SEGMENTS * sizeof(float)) != cudaSuccess) return fail(TFE_ERR_CUDA);
+    if (cudaMalloc(&h->d_seg_sum, nb * HEAD_SEGMENTS * sizeof(float)) != cudaSuccess) return fail(TFE_ERR_CUDA);
+    if (cudaMalloc(&h->d_lse, nb * sizeof(float)) != cudaSuccess) return fail(TFE_ERR_CUDA);
+    if (cudaMalloc(&h->d_seg_cand, nb * HEAD_SEGMENTS * HEAD_MAX_K * sizeof(unsigned long long)) != cudaSuccess)
+        return fail(TFE_ERR_CUDA);
+    if (cudaMalloc(&h->d_status, sizeof(uint32_t)) != cudaSuccess) return fail(TFE_ERR_CUDA);
+    if (cudaMemset(h->d_status, 0, sizeof(uint32_t)) != cudaSuccess) return fail(TFE_ERR_CUDA);
+    if (cudaFuncSetAttribute(tfe_head_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) !=
+        cudaSuccess)
+        return fail(TFE_ERR_CUDA);
+    if (cudaFuncSetAttribute(tfe_head_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             h->seg_len * (int)sizeof(float)) != cudaSuccess)
+        return fail(TFE_ERR_CUDA);
+    *out = h;
+    return TFE_OK;
+}
+
+void tfe_head_destroy(tfe_head *h)
+{
+    if (!h) return;
+    int prev = 0;
+    (void)cudaGetDevice(&prev);
+    (void)cudaSetDevice(h->device);
+    (void)cudaDeviceSynchronize();
+    if (h->d_logits) (void)cudaFree(h->d_logits);
+    if (h->d_seg_max) (void)cudaFree(h->d_seg_max);
+    if (h->d_seg_sum) (void)cudaFree(h->d_seg_sum);
+    if (h->d_lse) (void)cudaFree(h->d_lse);
+    if (h->d_seg_cand) (void)cudaFree(h->d_seg_cand);
+    if (h->d_status) (void)cudaFree(h->d_status);
+    (void)cudaSetDevice(prev);
+    delete h;
+}
+
+tfe_status tfe_head_topk(tfe_head *h, const void *hidden, int32_t B, int32_t K, int32_t *cand_tokens,
+                         float *cand_prob, void *stream_)
+{
+    if (!h || B < 0 || B > h->max_batch || K < 1 || K > HEAD_MAX_K || K > h->V) return TFE_ERR_INVALID_ARG;
+    if (B == 0) return TFE_OK;
+    if (!hidden || !cand_tokens || !cand_prob) return TFE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(hidden) & 15u) != 0) return TFE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    HeadGemmParams g{};
+    g.V = h->V; g.d = h->d; g.B = B;
+    g.N = (B + 15) / 16 * 16;
+    g.rows_per_cta = h->rows_per_cta; g.tail_rows = h->tail_rows;
+    const uint32_t stage_bytes = HEAD_TILE_M * 128u + (uint32_t)g.N * 128u;
+    const uint32_t budget = 227 * 1024 - 2048 - 1024;          // minus the alignment slack
+    g.stages = (int32_t)std::min<uint32_t>(HEAD_MAX_STAGES, budget / stage_bytes);
+    if (g.stages < 2) return TFE_ERR_INTERNAL;
+    uint32_t cols = 32;
+    while (cols < 2u * (uint32_t)g.N) cols <<= 1;
+    g.tmem_cols = cols;
+    g.logits = h->d_logits; g.ld = h->ld; g.status = h->d_status;
+    CUtensorMap map_h;
+    if (!make_map(&map_h, hidden, (uint64_t)B, (uint64_t)h->d, (uint32_t)g.N)) return TFE_ERR_CUDA;
+    const size_t smem = (size_t)g.stages * stage_bytes + 1024;
+    tfe_head_gemm_kernel<<<h->grid, HEAD_THREADS, smem, stream>>>(h->map_w, h->map_w_tail, map_h, g);
+    if (cudaGetLastError() != cudaSuccess) return TFE_ERR_CUDA;
+
+    HeadSelParams s{};
+    s.logits = h->d_logits; s.ld = h->ld; s.V = h->V; s.B = B; s.K = K; s.seg_len = h->seg_len;
+    s.seg_max = h->d_seg_max; s.seg_sum = h->d_seg_sum; s.seg_cand = h->d_seg_cand;
+    s.out_tokens = cand_tokens; s.out_prob = cand_prob; s.out_lse = h->d_lse;
+    tfe_head_partial_kernel<<<dim3(HEAD_SEGMENTS, (unsigned)B), HEAD_SEL_THREADS, (size_t)h->seg_len * sizeof(float),
+                              stream>>>(s);
+    tfe_head_merge_kernel<<<(unsigned)B, HEAD_SEL_THREADS, 0, stream>>>(s);
+    if (cudaGetLastError() != cudaSuccess) return TFE_ERR_CUDA;
+    return TFE_OK;
+}
+
+tfe_status tfe_head_buffers(tfe_head *h, const float **logits, int64_t *ld, const float **lse)
+{
+    if (!h) return TFE_ERR_INVALID_ARG;
+    if (logits) *logits = h->d_logits;
+    if (ld) *ld = h->ld;
+    if (lse) *lse = h->d_lse;
+    return TFE_OK;
+}
+
+tfe_status tfe_head_status(tfe_head *h, uint32_t *device_flags, void *stream_)
+{
+    if (!h || !device_flags) return TFE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (cudaMemcpyAsync(device_flags, h->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return TFE_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return TFE_ERR_CUDA;
+    return *device_flags ? TFE_ERR_INTERNAL : TFE_OK;
+}
+
+tfe_status tfe_head_geometry(const tfe_head *h, int32_t *grid, int32_t *rows_per_cta, int32_t *tail_rows)
+{
+    if (!h) return TFE_ERR_INVALID_ARG;
+    if (grid) *grid = h->grid;
+    if (rows_per_cta) *rows_per_cta = h->rows_per_cta;
+    if (tail_rows) *tail_rows = h->tail_rows;
+    return TFE_OK;
+}
+
+}  // extern "C"

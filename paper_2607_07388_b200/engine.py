@@ -109,3 +109,55 @@ def bf16_tensor_from_bits(bits: np.ndarray, device) -> torch.Tensor:
 
 def bits_from_bf16_tensor(t: torch.Tensor) -> np.ndarray:
     return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+class EarlyExitHead:
+    """softmax(W_pref h) + top-K on the GPU.  ``w_pref``: bf16 CUDA tensor [V, d], kept alive here."""
+
+    def __init__(self, w_pref: torch.Tensor, max_batch: int = 256):
+        assert w_pref.is_cuda and w_pref.dtype == torch.bfloat16 and w_pref.is_contiguous()
+        self.w = w_pref
+        self.V, self.d = w_pref.shape
+        self.max_batch = max_batch
+        self.handle = tfe.tfe_head_create(w_pref, self.V, self.d, max_batch)
+
+    def close(self):
+        if getattr(self, "handle", 0):
+            tfe.tfe_head_destroy(self.handle)
+            self.handle = 0
+
+    def __del__(self):
+        self.close()
+
+    def topk(self, hidden: torch.Tensor, K: int, stream=None):
+        """(tokens int32 [B, K], prob float32 [B, K]) on the device."""
+        assert hidden.is_cuda and hidden.dtype == torch.bfloat16 and hidden.is_contiguous()
+        B = hidden.shape[0]
+        tokens = torch.empty((B, K), dtype=torch.int32, device=hidden.device)
+        prob = torch.empty((B, K), dtype=torch.float32, device=hidden.device)
+        tfe.tfe_head_topk(self.handle, hidden, B, K, tokens, prob, stream)
+        return tokens, prob
+
+    def logits(self, B: int) -> torch.Tensor:
+        """fp32 [B, V] copy of the logits of the most recent call (synchronises)."""
+        addr, ld, _ = tfe.tfe_head_buffers(self.handle)
+        torch.cuda.synchronize()
+        return _device_view(addr, (B, ld), "<f4", self.w.device)[:, :self.V].clone()
+
+    def lse(self, B: int) -> torch.Tensor:
+        _, _, addr = tfe.tfe_head_buffers(self.handle)
+        torch.cuda.synchronize()
+        return _device_view(addr, (B,), "<f4", self.w.device).clone()
+
+    def status(self) -> int:
+        return tfe.tfe_head_status(self.handle)
+
+
+class _DevicePointer:
+    def __init__(self, ptr, shape, typestr):
+        self.__cuda_array_interface__ = {"shape": tuple(shape), "typestr": typestr, "data": (ptr, False), "version": 2}
+
+
+def _device_view(ptr: int, shape, typestr: str, device) -> torch.Tensor:
+    """A tensor over library-owned device memory (no copy, no ownership)."""
+    return torch.as_tensor(_DevicePointer(ptr, shape, typestr), device=device)

@@ -255,6 +255,8 @@ def procedural_int(idx, tag: int):
 
 ROW_TAG, ROW_SHIFT = 0x0A11CE, 10      # rows:   s * 2^-10, std about 0.036
 HID_TAG, HID_SHIFT = 0x0B0B00, 5       # hidden: s * 2^-5,  std about 1.15
+HEAD_W_TAG, HEAD_W_SHIFT = 0x0EAD00, 10 # early-exit head projection rows: std about 0.036
+HEAD_H_TAG, HEAD_H_SHIFT = 0x0EAD01, 5  # intermediate hidden states: std about 1.15 (logits: std about 1.3 at d = 1024)
 
 
 def procedural_bf16_np(ids: np.ndarray, d: int, tag: int, shift: int) -> np.ndarray:
@@ -410,3 +412,29 @@ def make_hidden_torch(w: Workload, device, variant: int = 0, Q: int | None = Non
         ids = torch.arange(q0, min(Q, q0 + step), dtype=torch.int64, device=device) + variant * (1 << 24)
         out[q0:q0 + len(ids)] = procedural_bf16_torch(ids, w.d, HID_TAG, HID_SHIFT)
     return out
+
+
+# ---------------------------------------------------------------- early-exit head inputs
+
+def head_weights_np(V: int, d: int, rows=None) -> np.ndarray:
+    """uint16 [V, d] (or the given rows) of the synthetic prefetch-head projection W_pref."""
+    ids = np.arange(V, dtype=np.int64) if rows is None else np.asarray(rows, np.int64)
+    return procedural_bf16_np(ids, d, HEAD_W_TAG, HEAD_W_SHIFT)
+
+
+def head_weights_torch(V: int, d: int, device, chunk_rows: int = 1 << 15):
+    import torch
+    W = torch.empty((V, d), dtype=torch.bfloat16, device=device)
+    for r0 in range(0, V, chunk_rows):
+        r1 = min(V, r0 + chunk_rows)
+        W[r0:r1] = procedural_bf16_torch(torch.arange(r0, r1, device=device), d, HEAD_W_TAG, HEAD_W_SHIFT)
+    return W
+
+
+def head_hidden_np(B: int, d: int, variant: int = 0) -> np.ndarray:
+    return procedural_bf16_np(np.arange(B, dtype=np.int64) + variant * 100_003, d, HEAD_H_TAG, HEAD_H_SHIFT)
+
+
+def head_hidden_torch(B: int, d: int, device, variant: int = 0):
+    import torch
+    return procedural_bf16_torch(torch.arange(B, device=device) + variant * 100_003, d, HEAD_H_TAG, HEAD_H_SHIFT)

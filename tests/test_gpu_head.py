@@ -1,0 +1,116 @@
+"""Early-exit prefetch head (tcgen05 GEMM + softmax + top-K) against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_07388_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = torch.device("cuda:0")
+
+
+@pytest.fixture(scope="module")
+def orc():
+    from oracle import tfe_oracle
+    tfe_oracle.build()
+    return tfe_oracle
+
+
+def _bits_to_gpu(bits):
+    from paper_2607_07388_b200.engine import bf16_tensor_from_bits
+    return bf16_tensor_from_bits(bits, DEV)
+
+
+def _inputs(seed, V, d, B, w_scale=0.25):
+    rng = np.random.default_rng(seed)
+    W = synth.f32_to_bf16_bits((rng.standard_normal((V, d)) * w_scale).astype(np.float32))
+    h = synth.f32_to_bf16_bits(rng.standard_normal((B, d)).astype(np.float32))
+    return W, h
+
+
+def check_topk(z64, tokens, prob, K, logit_tol, lse=None):
+    """The K tokens returned for every row must be a valid top-K of the oracle's logits up to
+    `logit_tol` (rows of W whose logits are closer than that may swap), carry the oracle's
+    probabilities, and come in descending order."""
+    B, V = z64.shape
+    m = z64.max(axis=1, keepdims=True)
+    lse64 = (m + np.log(np.exp(z64 - m).sum(axis=1, keepdims=True)))[:, 0]
+    if lse is not None:
+        np.testing.assert_allclose(lse, lse64, rtol=0, atol=5e-4)
+    for b in range(B):
+        t = tokens[b]
+        assert len(set(t.tolist())) == K and t.min() >= 0 and t.max() < V
+        kth = np.partition(z64[b], V - K)[V - K]                 # K-th largest oracle logit
+        assert z64[b, t].min() >= kth - logit_tol, (b, z64[b, t].min(), kth)
+        rest = np.ones(V, bool); rest[t] = False
+        assert z64[b, rest].max() <= z64[b, t].min() + logit_tol
+        p64 = np.exp(z64[b, t] - lse64[b])
+        np.testing.assert_allclose(prob[b], p64, rtol=2e-3, atol=1e-9)
+        assert (np.diff(prob[b]) <= 1e-7 * prob[b][:-1] + 1e-12).all()      # descending
+        # clear winners (further than the tolerance from the cut) must be present, in the oracle's order
+        order = np.argsort(-z64[b], kind="stable")
+        clear = [v for v in order[:K] if z64[b, v] > kth + 2 * logit_tol]
+        assert set(clear) <= set(t.tolist())
+
+
+@pytest.mark.parametrize("V,d,B,K", [(1000, 64, 3, 16), (4096 + 72, 128, 17, 64), (20_000, 256, 64, 128),
+                                     (148 * 128 * 2, 192, 33, 16), (333, 64, 1, 1), (50_000, 1024, 130, 64)])
+def test_head_against_oracle(orc, V, d, B, K):
+    from paper_2607_07388_b200.engine import EarlyExitHead
+    W, h = _inputs(V + d + B, V, d, B)
+    head = EarlyExitHead(_bits_to_gpu(W), max_batch=max(B, 16))
+    tok, prob = head.topk(_bits_to_gpu(h), K)
+    assert head.status() == 0
+    z = head.logits(B).cpu().numpy()
+    z64 = orc.head_logits(W, h)
+    # bf16 products are exact in fp32; the error is the fp32 accumulation over d terms
+    tol = 4e-6 * d * np.abs(z64).max()
+    np.testing.assert_allclose(z, z64, rtol=0, atol=tol)
+    check_topk(z64, tok.cpu().numpy(), prob.cpu().numpy(), K, logit_tol=2 * tol, lse=head.lse(B).cpu().numpy())
+    # a second call with another batch on the same head (buffers and barriers are re-armed)
+    W2, h2 = _inputs(V + 1, 8, d, min(B, 5))
+    tok2, prob2 = head.topk(_bits_to_gpu(h2), min(K, 8))
+    assert head.status() == 0
+    z64b = orc.head_logits(W, h2)
+    check_topk(z64b, tok2.cpu().numpy(), prob2.cpu().numpy(), min(K, 8), logit_tol=2 * tol)
+    head.close()
+
+
+def test_head_exact_cases(orc):
+    """Logits that fp32 accumulates exactly: ties resolve by token id, probabilities are exact softmax."""
+    from paper_2607_07388_b200.engine import EarlyExitHead
+    V, d, B = 2000, 64, 4
+    rng = np.random.default_rng(9)
+    Wf = rng.integers(-4, 5, size=(V, d)).astype(np.float32)          # small integers: every partial sum is exact
+    Wf[700] = Wf[20]; Wf[1500] = Wf[20]                                # three identical rows
+    hf = rng.integers(-3, 4, size=(B, d)).astype(np.float32)
+    hf[3] = 0                                                          # a zero state: uniform distribution
+    W, h = synth.f32_to_bf16_bits(Wf), synth.f32_to_bf16_bits(hf)
+    head = EarlyExitHead(_bits_to_gpu(W), max_batch=16)
+    K = 128
+    tok, prob = head.topk(_bits_to_gpu(h), K)
+    assert head.status() == 0
+    z64 = orc.head_logits(W, h)
+    np.testing.assert_array_equal(head.logits(B).cpu().numpy().astype(np.float64), z64)     # bit-exact logits
+    e_tok, e_prob, _ = orc.head_topk(z64, K)
+    np.testing.assert_array_equal(tok.cpu().numpy(), e_tok)            # identical selection and order, ties by id
+    np.testing.assert_allclose(prob.cpu().numpy(), e_prob, rtol=1e-4, atol=1e-30)      # fp32 underflows below ~1e-38
+    np.testing.assert_array_equal(tok[3].cpu().numpy(), np.arange(K))
+    head.close()
+
+
+def test_head_argument_checks():
+    from paper_2607_07388_b200 import binding as tfe
+    w = torch.zeros((256, 64), dtype=torch.bfloat16, device=DEV)
+    for V, d, mb in ((0, 64, 4), (256, 32, 4), (256, 96, 4), (256, 64, 0), (256, 64, 257)):
+        with pytest.raises(tfe.TfeError):
+            tfe.tfe_head_create(w, V, d, mb)
+    hd = tfe.tfe_head_create(w, 256, 64, 8)
+    h = torch.zeros((8, 64), dtype=torch.bfloat16, device=DEV)
+    t = torch.empty((8, 4), dtype=torch.int32, device=DEV); p = torch.empty((8, 4), dtype=torch.float32, device=DEV)
+    for B, K in ((9, 4), (4, 0), (4, 129), (-1, 4)):
+        with pytest.raises(tfe.TfeError):
+            tfe.tfe_head_topk(hd, h, B, K, t, p)
+    tfe.tfe_head_topk(hd, h, 0, 4, t, p)                               # empty batch: nothing to do
+    assert tfe.tfe_head_status(hd) == 0
+    tfe.tfe_head_destroy(hd)
