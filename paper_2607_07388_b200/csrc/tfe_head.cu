@@ -343,61 +343,130 @@ struct HeadSelParams {
 };
 
 // One segment of one row: max, sum of exp(z - max), and the K candidates of largest
-// (logit, then smaller token id): distinct 64-bit keys, so a radix selection needs no tie rule.
+// (logit, then smaller token id) as 64-bit keys orderable(z) << 32 | ~token (distinct, so
+// "largest K keys" has one answer), written in descending order.
+//
+// One sweep brings the segment into shared memory and gives every thread the maximum and the
+// sum of exponentials of its own elements (online: one exponential per element).  The K-th
+// largest of the 256 maxima of thread pairs bounds the K-th largest element from below -- they are K
+// distinct elements (with fewer than K groups there is no bound) -- so a second sweep keeps only the elements at or above it, a few more than
+// K; each survivor finds its rank by counting the survivors above it and the first K land in
+// order.  More than HEAD_KEEP_CAP survivors (many equal logits) send the block to an exact radix
+// selection over all keys, eight 8-bit digits, slower but indifferent to the distribution.
+#define HEAD_KEEP_CAP 2048
+
+__device__ __forceinline__ unsigned long long head_key(float z, int32_t token)
+{
+    return ((unsigned long long)orderable(z) << 32) | (uint32_t)~(uint32_t)token;
+}
+
 __global__ void __launch_bounds__(HEAD_SEL_THREADS)
 tfe_head_partial_kernel(const HeadSelParams p)
 {
     extern __shared__ float s_z[];                  // seg_len logits
+    __shared__ unsigned long long s_keep[HEAD_KEEP_CAP];
+    __shared__ unsigned long long s_tmax[HEAD_SEL_THREADS / 2];
+    __shared__ float s_red[2 * HEAD_SEL_THREADS / 32];
     __shared__ uint32_t s_hist[256];
-    __shared__ float s_red[HEAD_SEL_THREADS / 32];
-    __shared__ unsigned long long s_prefix;
-    __shared__ uint32_t s_want, s_fill;
+    __shared__ unsigned long long s_prefix, s_theta;
+    __shared__ uint32_t s_want, s_fill, s_nkeep;
     const int seg = blockIdx.x, b = blockIdx.y;
     const int32_t v0 = seg * p.seg_len;
     const int32_t n = max(0, min(p.seg_len, p.V - v0));
     const float *row = p.logits + (int64_t)b * p.ld + v0;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int NW = HEAD_SEL_THREADS / 32;
 
-    float mx = -INFINITY;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        const float z = __ldcs(row + i);
+    // ---- sweep 1: global -> shared, per-thread maximum (as a key) and online sum of exponentials
+    float m = -INFINITY, sum = 0.f;
+    unsigned long long kmax = 0ull;
+    auto take_in = [&](float z, int i) {
         s_z[i] = z;
-        mx = fmaxf(mx, z);
+        if (z > m) {                                // the first of equal values keeps the smaller token id
+            sum = sum * __expf(m - z) + 1.f;
+            m = z;
+            kmax = head_key(z, v0 + i);
+        } else {
+            sum += __expf(z - m);
+        }
+    };
+    // 16-byte loads, several in flight per thread (the row and the segment start are 16-byte aligned)
+    const int n4 = n >> 2;
+    const float4 *row4 = reinterpret_cast<const float4 *>(row);
+    int i4 = threadIdx.x;
+    for (; i4 + 2 * (int)blockDim.x < n4; i4 += 3 * blockDim.x) {
+        const float4 a = __ldcs(row4 + i4), c = __ldcs(row4 + i4 + blockDim.x), e = __ldcs(row4 + i4 + 2 * blockDim.x);
+        take_in(a.x, 4 * i4); take_in(a.y, 4 * i4 + 1); take_in(a.z, 4 * i4 + 2); take_in(a.w, 4 * i4 + 3);
+        const int ic = i4 + blockDim.x, ie = i4 + 2 * blockDim.x;
+        take_in(c.x, 4 * ic); take_in(c.y, 4 * ic + 1); take_in(c.z, 4 * ic + 2); take_in(c.w, 4 * ic + 3);
+        take_in(e.x, 4 * ie); take_in(e.y, 4 * ie + 1); take_in(e.z, 4 * ie + 2); take_in(e.w, 4 * ie + 3);
     }
+    for (; i4 < n4; i4 += blockDim.x) {
+        const float4 a = __ldcs(row4 + i4);
+        take_in(a.x, 4 * i4); take_in(a.y, 4 * i4 + 1); take_in(a.z, 4 * i4 + 2); take_in(a.w, 4 * i4 + 3);
+    }
+    for (int i = 4 * n4 + threadIdx.x; i < n; i += blockDim.x) take_in(__ldcs(row + i), i);
+    // neighbouring threads pool their maxima: 256 groups, still at least K of them
+    kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, 1));
+    if ((lane & 1) == 0) s_tmax[threadIdx.x >> 1] = kmax;
+    if (threadIdx.x == 0) { s_prefix = 0; s_fill = 0; s_nkeep = 0; s_theta = 0ull; }     // no bound: keep everything
+    float bm = m;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-    if (lane == 0) s_red[warp] = mx;
+    for (int o = 16; o > 0; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xFFFFFFFFu, bm, o));
+    if (lane == 0) s_red[warp] = bm;
     __syncthreads();
-    mx = s_red[0];
-    for (int w = 1; w < HEAD_SEL_THREADS / 32; ++w) mx = fmaxf(mx, s_red[w]);
-    __syncthreads();
-    float sum = 0.f;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) sum += __expf(s_z[i] - mx);
+    bm = s_red[0];
+    for (int w = 1; w < NW; ++w) bm = fmaxf(bm, s_red[w]);
+    float part = (sum > 0.f) ? sum * __expf(m - bm) : 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
-    if (lane == 0) s_red[warp] = sum;
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+    if (lane == 0) s_red[NW + warp] = part;
+    unsigned long long *cand = p.seg_cand + ((int64_t)b * HEAD_SEGMENTS + seg) * p.K;
+    const uint32_t take = (uint32_t)min(p.K, n);
+    for (int i = take + threadIdx.x; i < p.K; i += blockDim.x) cand[i] = 0ull;
+    // ---- the take-th largest per-thread maximum: rank by counting (keys are distinct or 0)
+    if (take > 0 && threadIdx.x < HEAD_SEL_THREADS / 2) {
+        const unsigned long long mine = s_tmax[threadIdx.x];
+        uint32_t above = 0;
+        for (int j = 0; j < HEAD_SEL_THREADS / 2; ++j) above += s_tmax[j] > mine;
+        if (mine != 0ull && above == take - 1) s_theta = mine;
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
         float t = 0.f;
-        for (int w = 0; w < HEAD_SEL_THREADS / 32; ++w) t += s_red[w];
-        p.seg_max[b * HEAD_SEGMENTS + seg] = mx;
+        for (int w = 0; w < NW; ++w) t += s_red[NW + w];
+        p.seg_max[b * HEAD_SEGMENTS + seg] = bm;
         p.seg_sum[b * HEAD_SEGMENTS + seg] = n > 0 ? t : 0.f;
-        s_prefix = 0;
-        s_want = (uint32_t)min(p.K, n);
-        s_fill = 0;
+        s_want = take;
     }
-    unsigned long long *cand = p.seg_cand + ((int64_t)b * HEAD_SEGMENTS + seg) * p.K;
-    for (int i = threadIdx.x; i < p.K; i += blockDim.x) cand[i] = 0ull;
-    __syncthreads();
-    const uint32_t take = s_want;
     if (take == 0) return;
-    // ---- the take-th largest key, most significant byte first
+    // ---- sweep 2: keep what is at or above the bound
+    const unsigned long long theta = s_theta;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const unsigned long long key = head_key(s_z[i], v0 + i);
+        if (key >= theta) {
+            const uint32_t at = atomicAdd(&s_nkeep, 1u);
+            if (at < HEAD_KEEP_CAP) s_keep[at] = key;
+        }
+    }
+    __syncthreads();
+    const uint32_t n_keep = s_nkeep;
+    if (n_keep <= HEAD_KEEP_CAP) {
+        for (uint32_t i = threadIdx.x; i < n_keep; i += blockDim.x) {
+            const unsigned long long key = s_keep[i];
+            uint32_t rank = 0;
+            for (uint32_t j = 0; j < n_keep; ++j) rank += s_keep[j] > key;
+            if (rank < take) cand[rank] = key;
+        }
+        return;
+    }
+    // ---- exact radix selection of the take-th largest key, most significant byte first
     for (int shift = 56; shift >= 0; shift -= 8) {
         for (int i = threadIdx.x; i < 256; i += blockDim.x) s_hist[i] = 0;
         __syncthreads();
         const unsigned long long prefix = s_prefix;
         for (int i = threadIdx.x; i < n; i += blockDim.x) {
-            const unsigned long long key = ((unsigned long long)orderable(s_z[i]) << 32) | (uint32_t)~(uint32_t)(v0 + i);
+            const unsigned long long key = head_key(s_z[i], v0 + i);
             if (shift == 56 || (key >> (shift + 8)) == (prefix >> (shift + 8)))
                 atomicAdd(&s_hist[(uint32_t)(key >> shift) & 255u], 1u);
         }
@@ -411,28 +480,34 @@ tfe_head_partial_kernel(const HeadSelParams p)
         }
         __syncthreads();
     }
+    // the keys at or above it are exactly `take`; they fit the keep list (take <= HEAD_MAX_K)
     const unsigned long long kth = s_prefix;
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        const unsigned long long key = ((unsigned long long)orderable(s_z[i]) << 32) | (uint32_t)~(uint32_t)(v0 + i);
-        if (key >= kth) {
-            const uint32_t at = atomicAdd(&s_fill, 1u);
-            if (at < (uint32_t)p.K) cand[at] = key;
-        }
+        const unsigned long long key = head_key(s_z[i], v0 + i);
+        if (key >= kth) s_keep[atomicAdd(&s_fill, 1u)] = key;
+    }
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < take; i += blockDim.x) {
+        const unsigned long long key = s_keep[i];
+        uint32_t rank = 0;
+        for (uint32_t j = 0; j < take; ++j) rank += s_keep[j] > key;
+        cand[rank] = key;
     }
 }
 
-// One row: sort the segments' candidates, keep the best K, normalise.
+// One row: every segment's list is in descending order, so a candidate's place in the merged
+// order is the number of keys above it in every list (binary searches); the first K are
+// written out with their probabilities exp(z - logsumexp).
 __global__ void __launch_bounds__(HEAD_SEL_THREADS)
 tfe_head_merge_kernel(const HeadSelParams p)
 {
     __shared__ unsigned long long s_v[HEAD_SEGMENTS * HEAD_MAX_K];
     __shared__ float s_lse;
     const int b = blockIdx.x;
-    const uint32_t n = (uint32_t)(HEAD_SEGMENTS * p.K);
-    uint32_t pow2 = 1;
-    while (pow2 < n) pow2 <<= 1;
-    const unsigned long long *cand = p.seg_cand + (int64_t)b * HEAD_SEGMENTS * p.K;
-    for (uint32_t i = threadIdx.x; i < pow2; i += blockDim.x) s_v[i] = i < n ? cand[i] : 0ull;
+    const int K = p.K;
+    const uint32_t n = (uint32_t)(HEAD_SEGMENTS * K);
+    const unsigned long long *cand = p.seg_cand + (int64_t)b * HEAD_SEGMENTS * K;
+    for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) s_v[i] = cand[i];
     if (threadIdx.x == 0) {
         float m = -INFINITY;
         for (int s = 0; s < HEAD_SEGMENTS; ++s)
@@ -445,29 +520,24 @@ tfe_head_merge_kernel(const HeadSelParams p)
         if (p.out_lse) p.out_lse[b] = s_lse;
     }
     __syncthreads();
-    // bitonic sort, descending
-    for (uint32_t k = 2; k <= pow2; k <<= 1)
-        for (uint32_t j = k >> 1; j > 0; j >>= 1) {
-            for (uint32_t t = threadIdx.x; t < pow2 / 2; t += blockDim.x) {
-                const uint32_t i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
-                const uint32_t l = i | j;
-                const unsigned long long a = s_v[i], c = s_v[l];
-                const bool down = (i & k) == 0;
-                if ((a < c) == down) { s_v[i] = c; s_v[l] = a; }
-            }
-            __syncthreads();
-        }
     const float lse = s_lse;
-    for (int i = threadIdx.x; i < p.K; i += blockDim.x) {
+    for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) {
         const unsigned long long key = s_v[i];
-        int32_t tok = -1;
-        float pr = 0.f;
-        if (key != 0ull) {
-            tok = (int32_t)~(uint32_t)key;
-            pr = __expf(from_orderable((uint32_t)(key >> 32)) - lse);
+        if (key == 0ull) continue;
+        uint32_t rank = 0;
+        for (int s = 0; s < HEAD_SEGMENTS && rank < (uint32_t)K; ++s) {
+            const unsigned long long *list = s_v + s * K;
+            int lo = 0, hi = K;                     // first position whose key is not above `key`
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (list[mid] > key) lo = mid + 1; else hi = mid;
+            }
+            rank += (uint32_t)lo;
         }
-        p.out_tokens[(int64_t)b * p.K + i] = tok;
-        p.out_prob[(int64_t)b * p.K + i] = pr;
+        if (rank < (uint32_t)K) {
+            p.out_tokens[(int64_t)b * K + rank] = (int32_t)~(uint32_t)key;
+            p.out_prob[(int64_t)b * K + rank] = __expf(from_orderable((uint32_t)(key >> 32)) - lse);
+        }
     }
 }
 
