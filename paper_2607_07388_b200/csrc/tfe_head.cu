@@ -14,12 +14,11 @@
 //                            memory, two accumulators so that a tile's epilogue overlaps the next
 //                            tile's MMAs), warps 2-5 read finished accumulators with tcgen05.ld and
 //                            store fp32 logits [B][V].  All mbarrier waits are bounded.
-//   tfe_head_partial_kernel  grid (segments, B): softmax statistics (max, sum of exponentials) and
-//                            the K largest logits of one segment of one row (radix selection in
-//                            shared memory).
-//   tfe_head_merge_kernel    one block per row: merges the segments' candidates, sorts the best K
-//                            (descending logit, equal logits ascending token id) and turns them
-//                            into probabilities exp(z - logsumexp).
+//   tfe_head_select_kernel   grid (segments, B): softmax statistics (max, sum of exponentials) and
+//                            the K largest logits of one segment of one row, in order; the block
+//                            that finishes a row last merges the segments' candidates (descending
+//                            logit, equal logits ascending token id) and turns the best K into
+//                            probabilities exp(z - logsumexp).
 //
 // The logits make a round trip through global memory (B*V*4 bytes, 39 MB for B = 64); they are
 // written and re-read within microseconds and stay in the 126 MB L2 for the batch sizes of decode.
@@ -340,187 +339,52 @@ struct HeadSelParams {
     int32_t *out_tokens;            // [B][K]
     float *out_prob;                // [B][K]
     float *out_lse;                 // [B] or nullptr
+    uint32_t *row_done;             // [B] segments finished per row, zero between calls
 };
 
-// One segment of one row: max, sum of exp(z - max), and the K candidates of largest
-// (logit, then smaller token id) as 64-bit keys orderable(z) << 32 | ~token (distinct, so
-// "largest K keys" has one answer), written in descending order.
+// Selection, one block per (segment, row): the segment's softmax statistics (max, sum of
+// exp(z - max)) and its K best candidates as 64-bit keys orderable(z) << 32 | ~token -- distinct,
+// so "largest K keys" has one answer: descending logit, equal logits ascending token id -- in
+// descending order.  The block that finishes a row last merges the segments.
 //
-// One sweep brings the segment into shared memory and gives every thread the maximum and the
-// sum of exponentials of its own elements (online: one exponential per element).  The K-th
-// largest of the 256 maxima of thread pairs bounds the K-th largest element from below -- they are K
-// distinct elements (with fewer than K groups there is no bound) -- so a second sweep keeps only the elements at or above it, a few more than
-// K; each survivor finds its rank by counting the survivors above it and the first K land in
+// One sweep over the segment gives every thread the maximum and the sum of exponentials of its
+// own elements (online softmax, one rescale per four elements).  Neighbouring
+// threads pool their maxima into 256 group maxima; the K-th largest of those bounds the K-th
+// largest element from below (they are K different elements; with fewer than K non-empty groups
+// the bound is -inf), so a second sweep (the segment is still in L2) keeps only the elements at or above it, a few more than
+// K.  Each survivor finds its rank by counting the survivors above it, and the first K land in
 // order.  More than HEAD_KEEP_CAP survivors (many equal logits) send the block to an exact radix
 // selection over all keys, eight 8-bit digits, slower but indifferent to the distribution.
 #define HEAD_KEEP_CAP 2048
+#define HEAD_GROUPS (HEAD_SEL_THREADS / 2)
 
 __device__ __forceinline__ unsigned long long head_key(float z, int32_t token)
 {
     return ((unsigned long long)orderable(z) << 32) | (uint32_t)~(uint32_t)token;
 }
 
-__global__ void __launch_bounds__(HEAD_SEL_THREADS)
-tfe_head_partial_kernel(const HeadSelParams p)
+// Merge of one row: every segment's list is in descending order, so a candidate's place in the
+// merged order is the number of keys above it in every list (binary searches); the first K are
+// written out with their probabilities exp(z - logsumexp).  s_v: HEAD_SEGMENTS * K keys.
+__device__ __forceinline__ void head_merge_row(const HeadSelParams &p, int b, unsigned long long *s_v, float *s_lse)
 {
-    extern __shared__ float s_z[];                  // seg_len logits
-    __shared__ unsigned long long s_keep[HEAD_KEEP_CAP];
-    __shared__ unsigned long long s_tmax[HEAD_SEL_THREADS / 2];
-    __shared__ float s_red[2 * HEAD_SEL_THREADS / 32];
-    __shared__ uint32_t s_hist[256];
-    __shared__ unsigned long long s_prefix, s_theta;
-    __shared__ uint32_t s_want, s_fill, s_nkeep;
-    const int seg = blockIdx.x, b = blockIdx.y;
-    const int32_t v0 = seg * p.seg_len;
-    const int32_t n = max(0, min(p.seg_len, p.V - v0));
-    const float *row = p.logits + (int64_t)b * p.ld + v0;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    constexpr int NW = HEAD_SEL_THREADS / 32;
-
-    // ---- sweep 1: global -> shared, per-thread maximum (as a key) and online sum of exponentials
-    float m = -INFINITY, sum = 0.f;
-    unsigned long long kmax = 0ull;
-    auto take_in = [&](float z, int i) {
-        s_z[i] = z;
-        if (z > m) {                                // the first of equal values keeps the smaller token id
-            sum = sum * __expf(m - z) + 1.f;
-            m = z;
-            kmax = head_key(z, v0 + i);
-        } else {
-            sum += __expf(z - m);
-        }
-    };
-    // 16-byte loads, several in flight per thread (the row and the segment start are 16-byte aligned)
-    const int n4 = n >> 2;
-    const float4 *row4 = reinterpret_cast<const float4 *>(row);
-    int i4 = threadIdx.x;
-    for (; i4 + 2 * (int)blockDim.x < n4; i4 += 3 * blockDim.x) {
-        const float4 a = __ldcs(row4 + i4), c = __ldcs(row4 + i4 + blockDim.x), e = __ldcs(row4 + i4 + 2 * blockDim.x);
-        take_in(a.x, 4 * i4); take_in(a.y, 4 * i4 + 1); take_in(a.z, 4 * i4 + 2); take_in(a.w, 4 * i4 + 3);
-        const int ic = i4 + blockDim.x, ie = i4 + 2 * blockDim.x;
-        take_in(c.x, 4 * ic); take_in(c.y, 4 * ic + 1); take_in(c.z, 4 * ic + 2); take_in(c.w, 4 * ic + 3);
-        take_in(e.x, 4 * ie); take_in(e.y, 4 * ie + 1); take_in(e.z, 4 * ie + 2); take_in(e.w, 4 * ie + 3);
-    }
-    for (; i4 < n4; i4 += blockDim.x) {
-        const float4 a = __ldcs(row4 + i4);
-        take_in(a.x, 4 * i4); take_in(a.y, 4 * i4 + 1); take_in(a.z, 4 * i4 + 2); take_in(a.w, 4 * i4 + 3);
-    }
-    for (int i = 4 * n4 + threadIdx.x; i < n; i += blockDim.x) take_in(__ldcs(row + i), i);
-    // neighbouring threads pool their maxima: 256 groups, still at least K of them
-    kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, 1));
-    if ((lane & 1) == 0) s_tmax[threadIdx.x >> 1] = kmax;
-    if (threadIdx.x == 0) { s_prefix = 0; s_fill = 0; s_nkeep = 0; s_theta = 0ull; }     // no bound: keep everything
-    float bm = m;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xFFFFFFFFu, bm, o));
-    if (lane == 0) s_red[warp] = bm;
-    __syncthreads();
-    bm = s_red[0];
-    for (int w = 1; w < NW; ++w) bm = fmaxf(bm, s_red[w]);
-    float part = (sum > 0.f) ? sum * __expf(m - bm) : 0.f;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
-    if (lane == 0) s_red[NW + warp] = part;
-    unsigned long long *cand = p.seg_cand + ((int64_t)b * HEAD_SEGMENTS + seg) * p.K;
-    const uint32_t take = (uint32_t)min(p.K, n);
-    for (int i = take + threadIdx.x; i < p.K; i += blockDim.x) cand[i] = 0ull;
-    // ---- the take-th largest per-thread maximum: rank by counting (keys are distinct or 0)
-    if (take > 0 && threadIdx.x < HEAD_SEL_THREADS / 2) {
-        const unsigned long long mine = s_tmax[threadIdx.x];
-        uint32_t above = 0;
-        for (int j = 0; j < HEAD_SEL_THREADS / 2; ++j) above += s_tmax[j] > mine;
-        if (mine != 0ull && above == take - 1) s_theta = mine;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float t = 0.f;
-        for (int w = 0; w < NW; ++w) t += s_red[NW + w];
-        p.seg_max[b * HEAD_SEGMENTS + seg] = bm;
-        p.seg_sum[b * HEAD_SEGMENTS + seg] = n > 0 ? t : 0.f;
-        s_want = take;
-    }
-    if (take == 0) return;
-    // ---- sweep 2: keep what is at or above the bound
-    const unsigned long long theta = s_theta;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        const unsigned long long key = head_key(s_z[i], v0 + i);
-        if (key >= theta) {
-            const uint32_t at = atomicAdd(&s_nkeep, 1u);
-            if (at < HEAD_KEEP_CAP) s_keep[at] = key;
-        }
-    }
-    __syncthreads();
-    const uint32_t n_keep = s_nkeep;
-    if (n_keep <= HEAD_KEEP_CAP) {
-        for (uint32_t i = threadIdx.x; i < n_keep; i += blockDim.x) {
-            const unsigned long long key = s_keep[i];
-            uint32_t rank = 0;
-            for (uint32_t j = 0; j < n_keep; ++j) rank += s_keep[j] > key;
-            if (rank < take) cand[rank] = key;
-        }
-        return;
-    }
-    // ---- exact radix selection of the take-th largest key, most significant byte first
-    for (int shift = 56; shift >= 0; shift -= 8) {
-        for (int i = threadIdx.x; i < 256; i += blockDim.x) s_hist[i] = 0;
-        __syncthreads();
-        const unsigned long long prefix = s_prefix;
-        for (int i = threadIdx.x; i < n; i += blockDim.x) {
-            const unsigned long long key = head_key(s_z[i], v0 + i);
-            if (shift == 56 || (key >> (shift + 8)) == (prefix >> (shift + 8)))
-                atomicAdd(&s_hist[(uint32_t)(key >> shift) & 255u], 1u);
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t want = s_want;
-            int dgt = 255;
-            for (; dgt > 0 && s_hist[dgt] < want; --dgt) want -= s_hist[dgt];
-            s_prefix = prefix | ((unsigned long long)dgt << shift);
-            s_want = want;
-        }
-        __syncthreads();
-    }
-    // the keys at or above it are exactly `take`; they fit the keep list (take <= HEAD_MAX_K)
-    const unsigned long long kth = s_prefix;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        const unsigned long long key = head_key(s_z[i], v0 + i);
-        if (key >= kth) s_keep[atomicAdd(&s_fill, 1u)] = key;
-    }
-    __syncthreads();
-    for (uint32_t i = threadIdx.x; i < take; i += blockDim.x) {
-        const unsigned long long key = s_keep[i];
-        uint32_t rank = 0;
-        for (uint32_t j = 0; j < take; ++j) rank += s_keep[j] > key;
-        cand[rank] = key;
-    }
-}
-
-// One row: every segment's list is in descending order, so a candidate's place in the merged
-// order is the number of keys above it in every list (binary searches); the first K are
-// written out with their probabilities exp(z - logsumexp).
-__global__ void __launch_bounds__(HEAD_SEL_THREADS)
-tfe_head_merge_kernel(const HeadSelParams p)
-{
-    __shared__ unsigned long long s_v[HEAD_SEGMENTS * HEAD_MAX_K];
-    __shared__ float s_lse;
-    const int b = blockIdx.x;
     const int K = p.K;
     const uint32_t n = (uint32_t)(HEAD_SEGMENTS * K);
     const unsigned long long *cand = p.seg_cand + (int64_t)b * HEAD_SEGMENTS * K;
-    for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) s_v[i] = cand[i];
+    for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) s_v[i] = __ldcg(cand + i);
     if (threadIdx.x == 0) {
-        float m = -INFINITY;
+        float m = -INFINITY, t = 0.f;
         for (int s = 0; s < HEAD_SEGMENTS; ++s)
-            if (p.seg_sum[b * HEAD_SEGMENTS + s] > 0.f) m = fmaxf(m, p.seg_max[b * HEAD_SEGMENTS + s]);
-        float t = 0.f;
-        for (int s = 0; s < HEAD_SEGMENTS; ++s)
-            if (p.seg_sum[b * HEAD_SEGMENTS + s] > 0.f)
-                t += p.seg_sum[b * HEAD_SEGMENTS + s] * __expf(p.seg_max[b * HEAD_SEGMENTS + s] - m);
-        s_lse = m + __logf(t);
-        if (p.out_lse) p.out_lse[b] = s_lse;
+            if (__ldcg(p.seg_sum + b * HEAD_SEGMENTS + s) > 0.f) m = fmaxf(m, __ldcg(p.seg_max + b * HEAD_SEGMENTS + s));
+        for (int s = 0; s < HEAD_SEGMENTS; ++s) {
+            const float ss = __ldcg(p.seg_sum + b * HEAD_SEGMENTS + s);
+            if (ss > 0.f) t += ss * __expf(__ldcg(p.seg_max + b * HEAD_SEGMENTS + s) - m);
+        }
+        *s_lse = m + __logf(t);
+        if (p.out_lse) p.out_lse[b] = *s_lse;
     }
     __syncthreads();
-    const float lse = s_lse;
+    const float lse = *s_lse;
     for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) {
         const unsigned long long key = s_v[i];
         if (key == 0ull) continue;
@@ -539,6 +403,186 @@ tfe_head_merge_kernel(const HeadSelParams p)
             p.out_prob[(int64_t)b * K + rank] = __expf(from_orderable((uint32_t)(key >> 32)) - lse);
         }
     }
+}
+
+__global__ void __launch_bounds__(HEAD_SEL_THREADS)
+tfe_head_select_kernel(const HeadSelParams p)
+{
+    __shared__ unsigned long long s_keep[HEAD_KEEP_CAP];
+    __shared__ float s_gmax[HEAD_GROUPS];
+    __shared__ float s_red[2 * HEAD_SEL_THREADS / 32];
+    __shared__ uint32_t s_hist[256];
+    __shared__ unsigned long long s_prefix;
+    __shared__ float s_theta, s_lse;
+    __shared__ uint32_t s_want, s_fill, s_nkeep, s_last;
+    const int seg = blockIdx.x, b = blockIdx.y;
+    const int32_t v0 = seg * p.seg_len;
+    const int32_t n = max(0, min(p.seg_len, p.V - v0));
+    const float *row = p.logits + (int64_t)b * p.ld + v0;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int NW = HEAD_SEL_THREADS / 32;
+
+    // ---- sweep 1: global -> shared, per-thread maximum and online sum of exponentials
+    float m = -INFINITY, sum = 0.f;
+    auto take_in = [&](float z) {
+        const float nm = fmaxf(m, z);
+        sum = sum * __expf(m - nm) + __expf(z - nm);
+        m = nm;
+    };
+    auto take_in4 = [&](const float4 a) {           // one rescale of the running sum per four elements
+        const float nm = fmaxf(fmaxf(m, fmaxf(a.x, a.y)), fmaxf(a.z, a.w));
+        sum = sum * __expf(m - nm) + ((__expf(a.x - nm) + __expf(a.y - nm)) + (__expf(a.z - nm) + __expf(a.w - nm)));
+        m = nm;
+    };
+    // 16-byte loads, several in flight per thread (the row and the segment start are 16-byte aligned)
+    const int n4 = n >> 2;
+    const float4 *row4 = reinterpret_cast<const float4 *>(row);
+    int i4 = threadIdx.x;
+    for (; i4 + 2 * (int)blockDim.x < n4; i4 += 3 * blockDim.x) {
+        const float4 a = __ldcg(row4 + i4), c = __ldcg(row4 + i4 + blockDim.x), e = __ldcg(row4 + i4 + 2 * blockDim.x);
+        take_in4(a); take_in4(c); take_in4(e);
+    }
+    for (; i4 < n4; i4 += blockDim.x) take_in4(__ldcg(row4 + i4));
+    for (int i = 4 * n4 + threadIdx.x; i < n; i += blockDim.x) take_in(__ldcg(row + i));
+
+    const float pair = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+    if ((lane & 1) == 0) s_gmax[threadIdx.x >> 1] = pair;
+    if (threadIdx.x == 0) { s_prefix = 0; s_fill = 0; s_nkeep = 0; }
+    float bm = pair;
+#pragma unroll
+    for (int o = 16; o > 1; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xFFFFFFFFu, bm, o));
+    if (lane == 0) s_red[warp] = bm;
+    __syncthreads();
+    bm = s_red[0];
+    for (int w = 1; w < NW; ++w) bm = fmaxf(bm, s_red[w]);
+    float part = (sum > 0.f) ? sum * __expf(m - bm) : 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+    if (lane == 0) s_red[NW + warp] = part;
+    unsigned long long *cand = p.seg_cand + ((int64_t)b * HEAD_SEGMENTS + seg) * p.K;
+    const uint32_t take = (uint32_t)min(p.K, n);
+    for (int i = take + threadIdx.x; i < p.K; i += blockDim.x) cand[i] = 0ull;
+    // ---- the take-th largest group maximum (with multiplicity): radix selection over the 256
+    // values, four 8-bit digits of the order-preserving integer image, most significant first
+    {
+        const uint32_t gkey = threadIdx.x < HEAD_GROUPS ? orderable(s_gmax[threadIdx.x]) : 0u;
+        uint32_t prefix = 0, want = take;
+        for (int shift = 24; shift >= 0 && take > 0; shift -= 8) {
+            if (threadIdx.x < 256) s_hist[threadIdx.x] = 0;
+            __syncthreads();
+            if (threadIdx.x < HEAD_GROUPS && (shift == 24 || (gkey >> (shift + 8)) == (prefix >> (shift + 8))))
+                atomicAdd(&s_hist[(gkey >> shift) & 255u], 1u);
+            __syncthreads();
+            // every warp repeats the search: lane l owns digits 255-8l .. 248-8l, largest first
+            uint32_t c[8], local = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { c[j] = s_hist[255 - 8 * lane - j]; local += c[j]; }
+            uint32_t incl = local;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            const bool owner = incl >= want && incl - local < want;
+            uint32_t dgt = 0, rest = 0;
+            if (owner) {
+                uint32_t before = incl - local;
+                int j = 0;
+                for (; j < 7 && before + c[j] < want; ++j) before += c[j];
+                dgt = 255u - 8u * lane - j;
+                rest = want - before;
+            }
+            const uint32_t who = __ffs(__ballot_sync(0xFFFFFFFFu, owner)) - 1;
+            prefix |= __shfl_sync(0xFFFFFFFFu, dgt, who) << shift;
+            want = __shfl_sync(0xFFFFFFFFu, rest, who);
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) s_theta = from_orderable(prefix);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int w = 0; w < NW; ++w) t += s_red[NW + w];
+        p.seg_max[b * HEAD_SEGMENTS + seg] = bm;
+        p.seg_sum[b * HEAD_SEGMENTS + seg] = n > 0 ? t : 0.f;
+        s_want = take;
+    }
+    if (take > 0) {
+        // ---- sweep 2: keep what is at or above the bound
+        const float theta = s_theta;
+        auto keep = [&](float z, int i) {
+            if (z >= theta) {
+                const uint32_t at = atomicAdd(&s_nkeep, 1u);
+                if (at < HEAD_KEEP_CAP) s_keep[at] = head_key(z, v0 + i);
+            }
+        };
+        int j4 = threadIdx.x;                       // the segment again, now from L2
+        for (; j4 + 2 * (int)blockDim.x < n4; j4 += 3 * blockDim.x) {
+            const int jc = j4 + blockDim.x, je = j4 + 2 * blockDim.x;
+            const float4 a = __ldcg(row4 + j4), c = __ldcg(row4 + jc), e = __ldcg(row4 + je);
+            keep(a.x, 4 * j4); keep(a.y, 4 * j4 + 1); keep(a.z, 4 * j4 + 2); keep(a.w, 4 * j4 + 3);
+            keep(c.x, 4 * jc); keep(c.y, 4 * jc + 1); keep(c.z, 4 * jc + 2); keep(c.w, 4 * jc + 3);
+            keep(e.x, 4 * je); keep(e.y, 4 * je + 1); keep(e.z, 4 * je + 2); keep(e.w, 4 * je + 3);
+        }
+        for (; j4 < n4; j4 += blockDim.x) {
+            const float4 a = __ldcg(row4 + j4);
+            keep(a.x, 4 * j4); keep(a.y, 4 * j4 + 1); keep(a.z, 4 * j4 + 2); keep(a.w, 4 * j4 + 3);
+        }
+        for (int i = 4 * n4 + threadIdx.x; i < n; i += blockDim.x) keep(__ldcg(row + i), i);
+        __syncthreads();
+        const uint32_t n_keep = s_nkeep;
+        if (n_keep <= HEAD_KEEP_CAP) {
+            for (uint32_t i = threadIdx.x; i < n_keep; i += blockDim.x) {
+                const unsigned long long key = s_keep[i];
+                uint32_t rank = 0;
+                for (uint32_t j = 0; j < n_keep; ++j) rank += s_keep[j] > key;
+                if (rank < take) cand[rank] = key;
+            }
+        } else {
+            // ---- exact radix selection of the take-th largest key, most significant byte first
+            for (int shift = 56; shift >= 0; shift -= 8) {
+                for (int i = threadIdx.x; i < 256; i += blockDim.x) s_hist[i] = 0;
+                __syncthreads();
+                const unsigned long long prefix = s_prefix;
+                for (int i = threadIdx.x; i < n; i += blockDim.x) {
+                    const unsigned long long key = head_key(__ldcg(row + i), v0 + i);
+                    if (shift == 56 || (key >> (shift + 8)) == (prefix >> (shift + 8)))
+                        atomicAdd(&s_hist[(uint32_t)(key >> shift) & 255u], 1u);
+                }
+                __syncthreads();
+                if (threadIdx.x == 0) {
+                    uint32_t want = s_want;
+                    int dgt = 255;
+                    for (; dgt > 0 && s_hist[dgt] < want; --dgt) want -= s_hist[dgt];
+                    s_prefix = prefix | ((unsigned long long)dgt << shift);
+                    s_want = want;
+                }
+                __syncthreads();
+            }
+            // the keys at or above it are exactly `take`; they fit the keep list (take <= HEAD_MAX_K)
+            const unsigned long long kth = s_prefix;
+            for (int i = threadIdx.x; i < n; i += blockDim.x) {
+                const unsigned long long key = head_key(__ldcg(row + i), v0 + i);
+                if (key >= kth) s_keep[atomicAdd(&s_fill, 1u)] = key;
+            }
+            __syncthreads();
+            for (uint32_t i = threadIdx.x; i < take; i += blockDim.x) {
+                const unsigned long long key = s_keep[i];
+                uint32_t rank = 0;
+                for (uint32_t j = 0; j < take; ++j) rank += s_keep[j] > key;
+                cand[rank] = key;
+            }
+        }
+    }
+    // ---- the block that closes the row merges its segments
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(&p.row_done[b], 1u) == HEAD_SEGMENTS - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    head_merge_row(p, b, s_keep, &s_lse);
+    if (threadIdx.x == 0) p.row_done[b] = 0;         // re-armed for the next call
 }
 
 // ------------------------------------------------------------------ host side
@@ -586,7 +630,7 @@ struct tfe_head {
     int64_t ld = 0;
     float *d_seg_max = nullptr, *d_seg_sum = nullptr, *d_lse = nullptr;
     unsigned long long *d_seg_cand = nullptr;
-    uint32_t *d_status = nullptr;
+    uint32_t *d_status = nullptr, *d_row_done = nullptr;
     int32_t seg_len = 0;
 };
 
@@ -624,11 +668,10 @@ tfe_status tfe_head_create(const void *w_pref, int32_t V, int32_t d, int32_t max
         return fail(TFE_ERR_CUDA);
     if (cudaMalloc(&h->d_status, sizeof(uint32_t)) != cudaSuccess) return fail(TFE_ERR_CUDA);
     if (cudaMemset(h->d_status, 0, sizeof(uint32_t)) != cudaSuccess) return fail(TFE_ERR_CUDA);
+    if (cudaMalloc(&h->d_row_done, nb * sizeof(uint32_t)) != cudaSuccess) return fail(TFE_ERR_CUDA);
+    if (cudaMemset(h->d_row_done, 0, nb * sizeof(uint32_t)) != cudaSuccess) return fail(TFE_ERR_CUDA);
     if (cudaFuncSetAttribute(tfe_head_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) !=
         cudaSuccess)
-        return fail(TFE_ERR_CUDA);
-    if (cudaFuncSetAttribute(tfe_head_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             h->seg_len * (int)sizeof(float)) != cudaSuccess)
         return fail(TFE_ERR_CUDA);
     *out = h;
     return TFE_OK;
@@ -647,6 +690,7 @@ void tfe_head_destroy(tfe_head *h)
     if (h->d_lse) (void)cudaFree(h->d_lse);
     if (h->d_seg_cand) (void)cudaFree(h->d_seg_cand);
     if (h->d_status) (void)cudaFree(h->d_status);
+    if (h->d_row_done) (void)cudaFree(h->d_row_done);
     (void)cudaSetDevice(prev);
     delete h;
 }
@@ -680,10 +724,8 @@ tfe_status tfe_head_topk(tfe_head *h, const void *hidden, int32_t B, int32_t K, 
     HeadSelParams s{};
     s.logits = h->d_logits; s.ld = h->ld; s.V = h->V; s.B = B; s.K = K; s.seg_len = h->seg_len;
     s.seg_max = h->d_seg_max; s.seg_sum = h->d_seg_sum; s.seg_cand = h->d_seg_cand;
-    s.out_tokens = cand_tokens; s.out_prob = cand_prob; s.out_lse = h->d_lse;
-    tfe_head_partial_kernel<<<dim3(HEAD_SEGMENTS, (unsigned)B), HEAD_SEL_THREADS, (size_t)h->seg_len * sizeof(float),
-                              stream>>>(s);
-    tfe_head_merge_kernel<<<(unsigned)B, HEAD_SEL_THREADS, 0, stream>>>(s);
+    s.out_tokens = cand_tokens; s.out_prob = cand_prob; s.out_lse = h->d_lse; s.row_done = h->d_row_done;
+    tfe_head_select_kernel<<<dim3(HEAD_SEGMENTS, (unsigned)B), HEAD_SEL_THREADS, 0, stream>>>(s);
     if (cudaGetLastError() != cudaSuccess) return TFE_ERR_CUDA;
     return TFE_OK;
 }
