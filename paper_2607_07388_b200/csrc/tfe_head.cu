@@ -41,6 +41,7 @@
 #define HEAD_SEGMENTS 8             // segments per row in the selection
 #define HEAD_SEL_THREADS 512
 #define HEAD_WAIT_LIMIT (1u << 22)  // polls of one mbarrier before a wait gives up
+#define HEAD_DYN_SMEM (227 * 1024 - 8192)   // dynamic shared memory of the GEMM: the SM's 227 KB minus its static arrays
 
 // device status bits
 #define HEAD_ST_TIMEOUT_PRODUCER 1u
@@ -173,6 +174,7 @@ struct HeadGemmParams {
     uint32_t tmem_cols;             // power of two >= 2 N
     float *logits;                  // [B][ld]
     int64_t ld;
+    float *group_max;               // [B][4 * gridDim.x]: largest logit of every (CTA, epilogue warp) per sequence
     uint32_t *status;
 };
 
@@ -184,6 +186,7 @@ tfe_head_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     __shared__ __align__(8) uint64_t s_full[HEAD_MAX_STAGES], s_empty[HEAD_MAX_STAGES], s_acc_full[2], s_acc_empty[2];
     __shared__ uint32_t s_tmem_base;
     __shared__ volatile uint32_t s_abort;
+    __shared__ float s_gmax[4][HEAD_MAX_N];            // running column maxima of the four epilogue warps
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -279,6 +282,8 @@ tfe_head_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     } else {
         // ============================ epilogue ================================
         const uint32_t quarter = (uint32_t)warp & 3u;               // tensor-memory lanes 32*quarter .. +31
+        for (int32_t c = lane; c < p.N; c += 32) s_gmax[quarter][c] = -INFINITY;
+        __syncwarp();
         for (int32_t t = 0; t < n_tiles; ++t) {
             const uint32_t acc = (uint32_t)t & 1u, acc_phase = ((uint32_t)t >> 1) & 1u;
             if (!mbar_wait(smem_u32(&s_acc_full[acc]), acc_phase, &s_abort)) {
@@ -295,16 +300,43 @@ tfe_head_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                 uint32_t v[16];
                 tmem_ld16(taddr + (uint32_t)c0, v);
                 tmem_ld_wait();
+                float f[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) f[j] = row_in_tile < valid ? __uint_as_float(v[j]) : -INFINITY;
                 if (row_in_tile < valid) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        if (c0 + j < p.B) p.logits[(int64_t)(c0 + j) * p.ld + row] = __uint_as_float(v[j]);
+                        if (c0 + j < p.B) p.logits[(int64_t)(c0 + j) * p.ld + row] = f[j];
+                }
+                // Maximum of each of the 16 columns over the warp's 32 rows: a butterfly in which
+                // every exchange halves the columns a lane is responsible for, 16 shuffles in all;
+                // lane l ends with the maximum of column c0 + (l >> 1).
+                const bool b4 = lane & 16, b3 = lane & 8, b2 = lane & 4, b1 = lane & 2;
+                float r8[8], r4[4], r2[2];
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    r8[i] = fmaxf(b4 ? f[i + 8] : f[i], __shfl_xor_sync(0xFFFFFFFFu, b4 ? f[i] : f[i + 8], 16));
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    r4[i] = fmaxf(b3 ? r8[i + 4] : r8[i], __shfl_xor_sync(0xFFFFFFFFu, b3 ? r8[i] : r8[i + 4], 8));
+#pragma unroll
+                for (int i = 0; i < 2; ++i)
+                    r2[i] = fmaxf(b2 ? r4[i + 2] : r4[i], __shfl_xor_sync(0xFFFFFFFFu, b2 ? r4[i] : r4[i + 2], 4));
+                float r1 = fmaxf(b1 ? r2[1] : r2[0], __shfl_xor_sync(0xFFFFFFFFu, b1 ? r2[0] : r2[1], 2));
+                r1 = fmaxf(r1, __shfl_xor_sync(0xFFFFFFFFu, r1, 1));
+                if ((lane & 1) == 0) {
+                    const int32_t c = c0 + (lane >> 1);
+                    s_gmax[quarter][c] = fmaxf(s_gmax[quarter][c], r1);
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty[acc]));
         }
+        __syncwarp();
+        const int32_t groups = 4 * (int32_t)gridDim.x;
+        for (int32_t c = lane; c < p.B; c += 32)
+            p.group_max[(int64_t)c * groups + 4 * blockIdx.x + quarter] = s_gmax[quarter][c];
     }
 
     tc_fence_before();
@@ -340,23 +372,24 @@ struct HeadSelParams {
     float *out_prob;                // [B][K]
     float *out_lse;                 // [B] or nullptr
     uint32_t *row_done;             // [B] segments finished per row, zero between calls
+    const float *group_max;         // [B][groups] from the GEMM's epilogue
+    int32_t groups;
 };
 
-// Selection, one block per (segment, row): the segment's softmax statistics (max, sum of
-// exp(z - max)) and its K best candidates as 64-bit keys orderable(z) << 32 | ~token -- distinct,
-// so "largest K keys" has one answer: descending logit, equal logits ascending token id -- in
+// Selection, one block per (segment, row): the segment's sum of exp(z - row maximum) and its
+// candidates for the row's K best as 64-bit keys orderable(z) << 32 | ~token -- distinct, so
+// "largest K keys" has one answer: descending logit, equal logits ascending token id -- in
 // descending order.  The block that finishes a row last merges the segments.
 //
-// One sweep over the segment gives every thread the maximum and the sum of exponentials of its
-// own elements (online softmax, one rescale per four elements).  Neighbouring
-// threads pool their maxima into 256 group maxima; the K-th largest of those bounds the K-th
-// largest element from below (they are K different elements; with fewer than K non-empty groups
-// the bound is -inf), so a second sweep (the segment is still in L2) keeps only the elements at or above it, a few more than
-// K.  Each survivor finds its rank by counting the survivors above it, and the first K land in
-// order.  More than HEAD_KEEP_CAP survivors (many equal logits) send the block to an exact radix
-// selection over all keys, eight 8-bit digits, slower but indifferent to the distribution.
+// The GEMM's epilogue left the largest logit of every (CTA, epilogue warp) group of vocabulary
+// rows.  Their maximum is the row maximum, and the K-th largest of them bounds the row's K-th
+// largest logit from below (K different elements reach it; with fewer than K groups the bound is
+// -inf).  So one sweep over the segment sums the exponentials and keeps the elements at or above
+// the bound -- about K per row, a handful per segment.  Each survivor finds its rank by counting
+// the survivors above it.  More than HEAD_KEEP_CAP survivors in a segment (many equal logits)
+// send the block to an exact radix selection over the segment's keys, eight 8-bit digits, slower
+// but indifferent to the distribution.
 #define HEAD_KEEP_CAP 2048
-#define HEAD_GROUPS (HEAD_SEL_THREADS / 2)
 
 __device__ __forceinline__ unsigned long long head_key(float z, int32_t token)
 {
@@ -372,16 +405,20 @@ __device__ __forceinline__ void head_merge_row(const HeadSelParams &p, int b, un
     const uint32_t n = (uint32_t)(HEAD_SEGMENTS * K);
     const unsigned long long *cand = p.seg_cand + (int64_t)b * HEAD_SEGMENTS * K;
     for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) s_v[i] = __ldcg(cand + i);
-    if (threadIdx.x == 0) {
-        float m = -INFINITY, t = 0.f;
-        for (int s = 0; s < HEAD_SEGMENTS; ++s)
-            if (__ldcg(p.seg_sum + b * HEAD_SEGMENTS + s) > 0.f) m = fmaxf(m, __ldcg(p.seg_max + b * HEAD_SEGMENTS + s));
-        for (int s = 0; s < HEAD_SEGMENTS; ++s) {
-            const float ss = __ldcg(p.seg_sum + b * HEAD_SEGMENTS + s);
-            if (ss > 0.f) t += ss * __expf(__ldcg(p.seg_max + b * HEAD_SEGMENTS + s) - m);
+    if (threadIdx.x < 32) {                         // the segments' statistics, one per lane
+        const bool has = threadIdx.x < HEAD_SEGMENTS;
+        const float ss = has ? __ldcg(p.seg_sum + b * HEAD_SEGMENTS + threadIdx.x) : 0.f;
+        const float sm = has ? __ldcg(p.seg_max + b * HEAD_SEGMENTS + threadIdx.x) : -INFINITY;
+        float m = ss > 0.f ? sm : -INFINITY;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+        float t = ss > 0.f ? ss * __expf(sm - m) : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+        if (threadIdx.x == 0) {
+            *s_lse = m + __logf(t);
+            if (p.out_lse) p.out_lse[b] = *s_lse;
         }
-        *s_lse = m + __logf(t);
-        if (p.out_lse) p.out_lse[b] = *s_lse;
     }
     __syncthreads();
     const float lse = *s_lse;
@@ -409,11 +446,10 @@ __global__ void __launch_bounds__(HEAD_SEL_THREADS)
 tfe_head_select_kernel(const HeadSelParams p)
 {
     __shared__ unsigned long long s_keep[HEAD_KEEP_CAP];
-    __shared__ float s_gmax[HEAD_GROUPS];
-    __shared__ float s_red[2 * HEAD_SEL_THREADS / 32];
+    __shared__ float s_red[HEAD_SEL_THREADS / 32];
     __shared__ uint32_t s_hist[256];
     __shared__ unsigned long long s_prefix;
-    __shared__ float s_theta, s_lse;
+    __shared__ float s_lse;
     __shared__ uint32_t s_want, s_fill, s_nkeep, s_last;
     const int seg = blockIdx.x, b = blockIdx.y;
     const int32_t v0 = seg * p.seg_len;
@@ -421,57 +457,42 @@ tfe_head_select_kernel(const HeadSelParams p)
     const float *row = p.logits + (int64_t)b * p.ld + v0;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int NW = HEAD_SEL_THREADS / 32;
+    const int32_t G = p.groups;
+    const float *gmax = p.group_max + (int64_t)b * G;
 
-    // ---- sweep 1: global -> shared, per-thread maximum and online sum of exponentials
-    float m = -INFINITY, sum = 0.f;
-    auto take_in = [&](float z) {
-        const float nm = fmaxf(m, z);
-        sum = sum * __expf(m - nm) + __expf(z - nm);
-        m = nm;
-    };
-    auto take_in4 = [&](const float4 a) {           // one rescale of the running sum per four elements
-        const float nm = fmaxf(fmaxf(m, fmaxf(a.x, a.y)), fmaxf(a.z, a.w));
-        sum = sum * __expf(m - nm) + ((__expf(a.x - nm) + __expf(a.y - nm)) + (__expf(a.z - nm) + __expf(a.w - nm)));
-        m = nm;
-    };
-    // 16-byte loads, several in flight per thread (the row and the segment start are 16-byte aligned)
-    const int n4 = n >> 2;
-    const float4 *row4 = reinterpret_cast<const float4 *>(row);
-    int i4 = threadIdx.x;
-    for (; i4 + 2 * (int)blockDim.x < n4; i4 += 3 * blockDim.x) {
-        const float4 a = __ldcg(row4 + i4), c = __ldcg(row4 + i4 + blockDim.x), e = __ldcg(row4 + i4 + 2 * blockDim.x);
-        take_in4(a); take_in4(c); take_in4(e);
-    }
-    for (; i4 < n4; i4 += blockDim.x) take_in4(__ldcg(row4 + i4));
-    for (int i = 4 * n4 + threadIdx.x; i < n; i += blockDim.x) take_in(__ldcg(row + i));
-
-    const float pair = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
-    if ((lane & 1) == 0) s_gmax[threadIdx.x >> 1] = pair;
+    // ---- row maximum, and the K-th largest group maximum (with multiplicity) rounded down to the
+    // upper 16 bits of its order-preserving integer image (any lower bound serves): radix selection,
+    // two 8-bit digits, most significant first
+    // (at most 2 * HEAD_SEL_THREADS groups: two per thread, loaded once)
+    const float g0v = (int)threadIdx.x < G ? __ldcg(gmax + threadIdx.x) : -INFINITY;
+    const float g1v = (int)threadIdx.x + HEAD_SEL_THREADS < G ? __ldcg(gmax + threadIdx.x + HEAD_SEL_THREADS) : -INFINITY;
+    float row_max = fmaxf(g0v, g1v);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) row_max = fmaxf(row_max, __shfl_xor_sync(0xFFFFFFFFu, row_max, o));
+    if (lane == 0) s_red[warp] = row_max;
     if (threadIdx.x == 0) { s_prefix = 0; s_fill = 0; s_nkeep = 0; }
-    float bm = pair;
-#pragma unroll
-    for (int o = 16; o > 1; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xFFFFFFFFu, bm, o));
-    if (lane == 0) s_red[warp] = bm;
     __syncthreads();
-    bm = s_red[0];
-    for (int w = 1; w < NW; ++w) bm = fmaxf(bm, s_red[w]);
-    float part = (sum > 0.f) ? sum * __expf(m - bm) : 0.f;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
-    if (lane == 0) s_red[NW + warp] = part;
-    unsigned long long *cand = p.seg_cand + ((int64_t)b * HEAD_SEGMENTS + seg) * p.K;
-    const uint32_t take = (uint32_t)min(p.K, n);
-    for (int i = take + threadIdx.x; i < p.K; i += blockDim.x) cand[i] = 0ull;
-    // ---- the take-th largest group maximum (with multiplicity): radix selection over the 256
-    // values, four 8-bit digits of the order-preserving integer image, most significant first
-    {
-        const uint32_t gkey = threadIdx.x < HEAD_GROUPS ? orderable(s_gmax[threadIdx.x]) : 0u;
-        uint32_t prefix = 0, want = take;
-        for (int shift = 24; shift >= 0 && take > 0; shift -= 8) {
+    row_max = s_red[0];
+    for (int w = 1; w < NW; ++w) row_max = fmaxf(row_max, s_red[w]);
+    __syncthreads();                                // s_red is reused for the sums
+    float theta = -INFINITY;
+    if (G >= p.K) {
+        uint32_t prefix = 0, want = (uint32_t)p.K;
+        for (int shift = 24; shift >= 16; shift -= 8) {
             if (threadIdx.x < 256) s_hist[threadIdx.x] = 0;
             __syncthreads();
-            if (threadIdx.x < HEAD_GROUPS && (shift == 24 || (gkey >> (shift + 8)) == (prefix >> (shift + 8))))
-                atomicAdd(&s_hist[(gkey >> shift) & 255u], 1u);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int g = (int)threadIdx.x + half * HEAD_SEL_THREADS;
+                const uint32_t gkey = orderable(half ? g1v : g0v);
+                const bool live = g < G && (shift == 24 || (gkey >> (shift + 8)) == (prefix >> (shift + 8)));
+                const uint32_t digit = (gkey >> shift) & 255u;
+                const uint32_t vote = __ballot_sync(0xFFFFFFFFu, live);
+                if (live) {                         // one shared-memory atomic per distinct digit of the warp
+                    const uint32_t peers = __match_any_sync(vote, digit);
+                    if (lane == __ffs(peers) - 1) atomicAdd(&s_hist[digit], __popc(peers));
+                }
+            }
             __syncthreads();
             // every warp repeats the search: lane l owns digits 255-8l .. 248-8l, largest first
             uint32_t c[8], local = 0;
@@ -497,81 +518,92 @@ tfe_head_select_kernel(const HeadSelParams p)
             want = __shfl_sync(0xFFFFFFFFu, rest, who);
             __syncthreads();
         }
-        if (threadIdx.x == 0) s_theta = from_orderable(prefix);
+        theta = from_orderable(prefix);
     }
+
+    // ---- the sweep: sum of exponentials, survivors
+    float sum = 0.f;
+    auto take_in = [&](float z, int i) {
+        sum += __expf(z - row_max);
+        if (z >= theta) {
+            const uint32_t at = atomicAdd(&s_nkeep, 1u);
+            if (at < HEAD_KEEP_CAP) s_keep[at] = head_key(z, v0 + i);
+        }
+    };
+    // 16-byte loads, several in flight per thread (the row and the segment start are 16-byte aligned)
+    const int n4 = n >> 2;
+    const float4 *row4 = reinterpret_cast<const float4 *>(row);
+    int i4 = threadIdx.x;
+    for (; i4 + 2 * (int)blockDim.x < n4; i4 += 3 * blockDim.x) {
+        const int ic = i4 + blockDim.x, ie = i4 + 2 * blockDim.x;
+        const float4 a = __ldcs(row4 + i4), c = __ldcs(row4 + ic), e = __ldcs(row4 + ie);
+        take_in(a.x, 4 * i4); take_in(a.y, 4 * i4 + 1); take_in(a.z, 4 * i4 + 2); take_in(a.w, 4 * i4 + 3);
+        take_in(c.x, 4 * ic); take_in(c.y, 4 * ic + 1); take_in(c.z, 4 * ic + 2); take_in(c.w, 4 * ic + 3);
+        take_in(e.x, 4 * ie); take_in(e.y, 4 * ie + 1); take_in(e.z, 4 * ie + 2); take_in(e.w, 4 * ie + 3);
+    }
+    for (; i4 < n4; i4 += blockDim.x) {
+        const float4 a = __ldcs(row4 + i4);
+        take_in(a.x, 4 * i4); take_in(a.y, 4 * i4 + 1); take_in(a.z, 4 * i4 + 2); take_in(a.w, 4 * i4 + 3);
+    }
+    for (int i = 4 * n4 + threadIdx.x; i < n; i += blockDim.x) take_in(__ldcs(row + i), i);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+    if (lane == 0) s_red[warp] = sum;
     __syncthreads();
+    const uint32_t n_keep = s_nkeep;
+    unsigned long long *cand = p.seg_cand + ((int64_t)b * HEAD_SEGMENTS + seg) * p.K;
     if (threadIdx.x == 0) {
         float t = 0.f;
-        for (int w = 0; w < NW; ++w) t += s_red[NW + w];
-        p.seg_max[b * HEAD_SEGMENTS + seg] = bm;
+        for (int w = 0; w < NW; ++w) t += s_red[w];
+        p.seg_max[b * HEAD_SEGMENTS + seg] = row_max;
         p.seg_sum[b * HEAD_SEGMENTS + seg] = n > 0 ? t : 0.f;
-        s_want = take;
+        s_want = (uint32_t)min(p.K, n);
     }
-    if (take > 0) {
-        // ---- sweep 2: keep what is at or above the bound
-        const float theta = s_theta;
-        auto keep = [&](float z, int i) {
-            if (z >= theta) {
-                const uint32_t at = atomicAdd(&s_nkeep, 1u);
-                if (at < HEAD_KEEP_CAP) s_keep[at] = head_key(z, v0 + i);
-            }
-        };
-        int j4 = threadIdx.x;                       // the segment again, now from L2
-        for (; j4 + 2 * (int)blockDim.x < n4; j4 += 3 * blockDim.x) {
-            const int jc = j4 + blockDim.x, je = j4 + 2 * blockDim.x;
-            const float4 a = __ldcg(row4 + j4), c = __ldcg(row4 + jc), e = __ldcg(row4 + je);
-            keep(a.x, 4 * j4); keep(a.y, 4 * j4 + 1); keep(a.z, 4 * j4 + 2); keep(a.w, 4 * j4 + 3);
-            keep(c.x, 4 * jc); keep(c.y, 4 * jc + 1); keep(c.z, 4 * jc + 2); keep(c.w, 4 * jc + 3);
-            keep(e.x, 4 * je); keep(e.y, 4 * je + 1); keep(e.z, 4 * je + 2); keep(e.w, 4 * je + 3);
+    if (n_keep <= HEAD_KEEP_CAP) {
+        const uint32_t take = min((uint32_t)p.K, n_keep);
+        for (int i = take + threadIdx.x; i < p.K; i += blockDim.x) cand[i] = 0ull;
+        for (uint32_t i = threadIdx.x; i < n_keep; i += blockDim.x) {
+            const unsigned long long key = s_keep[i];
+            uint32_t rank = 0;
+            for (uint32_t j = 0; j < n_keep; ++j) rank += s_keep[j] > key;
+            if (rank < take) cand[rank] = key;
         }
-        for (; j4 < n4; j4 += blockDim.x) {
-            const float4 a = __ldcg(row4 + j4);
-            keep(a.x, 4 * j4); keep(a.y, 4 * j4 + 1); keep(a.z, 4 * j4 + 2); keep(a.w, 4 * j4 + 3);
-        }
-        for (int i = 4 * n4 + threadIdx.x; i < n; i += blockDim.x) keep(__ldcg(row + i), i);
+    } else {
+        // ---- exact radix selection of the segment's take-th largest key, most significant byte first
+        const uint32_t take = (uint32_t)min(p.K, n);
+        for (int i = take + threadIdx.x; i < p.K; i += blockDim.x) cand[i] = 0ull;
         __syncthreads();
-        const uint32_t n_keep = s_nkeep;
-        if (n_keep <= HEAD_KEEP_CAP) {
-            for (uint32_t i = threadIdx.x; i < n_keep; i += blockDim.x) {
-                const unsigned long long key = s_keep[i];
-                uint32_t rank = 0;
-                for (uint32_t j = 0; j < n_keep; ++j) rank += s_keep[j] > key;
-                if (rank < take) cand[rank] = key;
-            }
-        } else {
-            // ---- exact radix selection of the take-th largest key, most significant byte first
-            for (int shift = 56; shift >= 0; shift -= 8) {
-                for (int i = threadIdx.x; i < 256; i += blockDim.x) s_hist[i] = 0;
-                __syncthreads();
-                const unsigned long long prefix = s_prefix;
-                for (int i = threadIdx.x; i < n; i += blockDim.x) {
-                    const unsigned long long key = head_key(__ldcg(row + i), v0 + i);
-                    if (shift == 56 || (key >> (shift + 8)) == (prefix >> (shift + 8)))
-                        atomicAdd(&s_hist[(uint32_t)(key >> shift) & 255u], 1u);
-                }
-                __syncthreads();
-                if (threadIdx.x == 0) {
-                    uint32_t want = s_want;
-                    int dgt = 255;
-                    for (; dgt > 0 && s_hist[dgt] < want; --dgt) want -= s_hist[dgt];
-                    s_prefix = prefix | ((unsigned long long)dgt << shift);
-                    s_want = want;
-                }
-                __syncthreads();
-            }
-            // the keys at or above it are exactly `take`; they fit the keep list (take <= HEAD_MAX_K)
-            const unsigned long long kth = s_prefix;
+        for (int shift = 56; shift >= 0; shift -= 8) {
+            for (int i = threadIdx.x; i < 256; i += blockDim.x) s_hist[i] = 0;
+            __syncthreads();
+            const unsigned long long prefix = s_prefix;
             for (int i = threadIdx.x; i < n; i += blockDim.x) {
                 const unsigned long long key = head_key(__ldcg(row + i), v0 + i);
-                if (key >= kth) s_keep[atomicAdd(&s_fill, 1u)] = key;
+                if (shift == 56 || (key >> (shift + 8)) == (prefix >> (shift + 8)))
+                    atomicAdd(&s_hist[(uint32_t)(key >> shift) & 255u], 1u);
             }
             __syncthreads();
-            for (uint32_t i = threadIdx.x; i < take; i += blockDim.x) {
-                const unsigned long long key = s_keep[i];
-                uint32_t rank = 0;
-                for (uint32_t j = 0; j < take; ++j) rank += s_keep[j] > key;
-                cand[rank] = key;
+            if (threadIdx.x == 0) {
+                uint32_t want = s_want;
+                int dgt = 255;
+                for (; dgt > 0 && s_hist[dgt] < want; --dgt) want -= s_hist[dgt];
+                s_prefix = prefix | ((unsigned long long)dgt << shift);
+                s_want = want;
             }
+            __syncthreads();
+        }
+        // the keys at or above it are exactly `take`; they fit the keep list (take <= HEAD_MAX_K)
+        const unsigned long long kth = s_prefix;
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            const unsigned long long key = head_key(__ldcg(row + i), v0 + i);
+            if (key >= kth) s_keep[atomicAdd(&s_fill, 1u)] = key;
+        }
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < take; i += blockDim.x) {
+            const unsigned long long key = s_keep[i];
+            uint32_t rank = 0;
+            for (uint32_t j = 0; j < take; ++j) rank += s_keep[j] > key;
+            cand[rank] = key;
         }
     }
     // ---- the block that closes the row merges its segments
@@ -631,6 +663,7 @@ struct tfe_head {
     float *d_seg_max = nullptr, *d_seg_sum = nullptr, *d_lse = nullptr;
     unsigned long long *d_seg_cand = nullptr;
     uint32_t *d_status = nullptr, *d_row_done = nullptr;
+    float *d_group_max = nullptr;
     int32_t seg_len = 0;
 };
 
@@ -650,7 +683,8 @@ tfe_status tfe_head_create(const void *w_pref, int32_t V, int32_t d, int32_t max
     if (cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess)
         return fail(TFE_ERR_CUDA);
     // contiguous row ranges of equal size (a multiple of 8) per CTA
-    const int32_t ctas = std::max(1, std::min(h->sm_count, (V + HEAD_TILE_M - 1) / HEAD_TILE_M));
+    // (the selection kernel holds at most 2 * HEAD_SEL_THREADS groups = 4 per CTA)
+    const int32_t ctas = std::max(1, std::min(std::min(h->sm_count, 2 * HEAD_SEL_THREADS / 4), (V + HEAD_TILE_M - 1) / HEAD_TILE_M));
     h->rows_per_cta = (int32_t)((((int64_t)V + ctas - 1) / ctas + 7) / 8 * 8);
     h->grid = (int32_t)(((int64_t)V + h->rows_per_cta - 1) / h->rows_per_cta);
     h->tail_rows = h->rows_per_cta % HEAD_TILE_M;
@@ -669,8 +703,9 @@ tfe_status tfe_head_create(const void *w_pref, int32_t V, int32_t d, int32_t max
     if (cudaMalloc(&h->d_status, sizeof(uint32_t)) != cudaSuccess) return fail(TFE_ERR_CUDA);
     if (cudaMemset(h->d_status, 0, sizeof(uint32_t)) != cudaSuccess) return fail(TFE_ERR_CUDA);
     if (cudaMalloc(&h->d_row_done, nb * sizeof(uint32_t)) != cudaSuccess) return fail(TFE_ERR_CUDA);
+    if (cudaMalloc(&h->d_group_max, nb * 4 * (size_t)h->grid * sizeof(float)) != cudaSuccess) return fail(TFE_ERR_CUDA);
     if (cudaMemset(h->d_row_done, 0, nb * sizeof(uint32_t)) != cudaSuccess) return fail(TFE_ERR_CUDA);
-    if (cudaFuncSetAttribute(tfe_head_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048) !=
+    if (cudaFuncSetAttribute(tfe_head_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, HEAD_DYN_SMEM) !=
         cudaSuccess)
         return fail(TFE_ERR_CUDA);
     *out = h;
@@ -691,6 +726,7 @@ void tfe_head_destroy(tfe_head *h)
     if (h->d_seg_cand) (void)cudaFree(h->d_seg_cand);
     if (h->d_status) (void)cudaFree(h->d_status);
     if (h->d_row_done) (void)cudaFree(h->d_row_done);
+    if (h->d_group_max) (void)cudaFree(h->d_group_max);
     (void)cudaSetDevice(prev);
     delete h;
 }
@@ -708,13 +744,13 @@ tfe_status tfe_head_topk(tfe_head *h, const void *hidden, int32_t B, int32_t K, 
     g.N = (B + 15) / 16 * 16;
     g.rows_per_cta = h->rows_per_cta; g.tail_rows = h->tail_rows;
     const uint32_t stage_bytes = HEAD_TILE_M * 128u + (uint32_t)g.N * 128u;
-    const uint32_t budget = 227 * 1024 - 2048 - 1024;          // minus the alignment slack
+    const uint32_t budget = HEAD_DYN_SMEM - 1024;               // minus the alignment slack
     g.stages = (int32_t)std::min<uint32_t>(HEAD_MAX_STAGES, budget / stage_bytes);
     if (g.stages < 2) return TFE_ERR_INTERNAL;
     uint32_t cols = 32;
     while (cols < 2u * (uint32_t)g.N) cols <<= 1;
     g.tmem_cols = cols;
-    g.logits = h->d_logits; g.ld = h->ld; g.status = h->d_status;
+    g.logits = h->d_logits; g.ld = h->ld; g.status = h->d_status; g.group_max = h->d_group_max;
     CUtensorMap map_h;
     if (!make_map(&map_h, hidden, (uint64_t)B, (uint64_t)h->d, (uint32_t)g.N)) return TFE_ERR_CUDA;
     const size_t smem = (size_t)g.stages * stage_bytes + 1024;
@@ -725,6 +761,7 @@ tfe_status tfe_head_topk(tfe_head *h, const void *hidden, int32_t B, int32_t K, 
     s.logits = h->d_logits; s.ld = h->ld; s.V = h->V; s.B = B; s.K = K; s.seg_len = h->seg_len;
     s.seg_max = h->d_seg_max; s.seg_sum = h->d_seg_sum; s.seg_cand = h->d_seg_cand;
     s.out_tokens = cand_tokens; s.out_prob = cand_prob; s.out_lse = h->d_lse; s.row_done = h->d_row_done;
+    s.group_max = h->d_group_max; s.groups = 4 * h->grid;
     tfe_head_select_kernel<<<dim3(HEAD_SEGMENTS, (unsigned)B), HEAD_SEL_THREADS, 0, stream>>>(s);
     if (cudaGetLastError() != cudaSuccess) return TFE_ERR_CUDA;
     return TFE_OK;
