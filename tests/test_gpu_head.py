@@ -114,3 +114,44 @@ def test_head_argument_checks():
     tfe.tfe_head_topk(hd, h, 0, 4, t, p)                               # empty batch: nothing to do
     assert tfe.tfe_head_status(hd) == 0
     tfe.tfe_head_destroy(hd)
+
+
+def test_head_feeds_prefetch_candidates(orc):
+    """The chain of Sec. 4.4 on the device: hidden states -> top-K tokens and probabilities (head)
+    -> candidate phrases and priorities (tfe_prefetch_candidates), without a host round trip.  The
+    head's outputs are checked against the oracle head, and the candidate step against the oracle fed
+    with those same tokens and probabilities."""
+    import parity_harness as H
+    from paper_2607_07388_b200.engine import EarlyExitHead
+    w = synth.config(2, n_phrases=60_000, gpu_slots=20_000, B=48)
+    tb, pr = H.pair_from_workload(w)
+    V, d, B, K = w.vocab, 128, w.B, 32
+    rng = np.random.default_rng(17)
+    # small-integer weights: fp32 logits are exact, so the head's tokens equal the oracle's
+    Wf = rng.integers(-3, 4, size=(V, d)).astype(np.float32)
+    hf = rng.integers(-2, 3, size=(B, d)).astype(np.float32)
+    # the token that follows each sequence's history in the table stream gets a row aligned with
+    # that sequence's hidden state, so it is predicted and its phrases are looked up
+    base = tb.safe_len - 3 * B - 16            # late in the stream: rare phrases, mostly outside the GPU tier
+    nxt = tb.stream[base + 2 * np.arange(B) + 2]
+    for b in range(B):
+        Wf[nxt[b]] = 3 * np.sign(hf[b])
+    W, h = synth.f32_to_bf16_bits(Wf), synth.f32_to_bf16_bits(hf)
+    head = EarlyExitHead(_bits_to_gpu(W), max_batch=B)
+    tok, prob = head.topk(_bits_to_gpu(h), K)
+    assert head.status() == 0
+    e_tok, e_prob, _ = orc.head_topk(orc.head_logits(W, h), K)
+    assert (e_tok[:, 0] == nxt).mean() > 0.5
+    np.testing.assert_array_equal(tok.cpu().numpy(), e_tok)
+    np.testing.assert_allclose(prob.cpu().numpy(), e_prob, rtol=1e-4, atol=1e-30)
+    hist = torch.from_numpy(np.stack([tb.stream[base + 2 * b:base + 2 * b + 2] for b in range(B)]).astype(np.int32)).to(DEV)
+    ph, tr, sc, sr, cnt = pr.eng.prefetch_candidates(hist, tok, prob, benefit_host=1.0, benefit_ssd=2.0, budget=256)
+    torch.cuda.synchronize()
+    eph, etr, esc, esr, total = pr.ora.prefetch_candidates(hist.cpu().numpy(), tok.cpu().numpy(), prob.cpu().numpy(),
+                                                           benefit_host=1.0, benefit_ssd=2.0, budget=256)
+    n = int(cnt[0].item())
+    assert int(cnt[1].item()) == total and n == len(eph) and total >= 5
+    np.testing.assert_array_equal(ph[:n].cpu().numpy().view(np.uint32), eph)
+    np.testing.assert_array_equal(sc[:n].cpu().numpy().view(np.uint32), esc.view(np.uint32))
+    head.close()
+    pr.close()
