@@ -95,6 +95,22 @@ tfe_status tfe_index_build(const tfe_config *cfg, const int32_t *phrase_tokens,
                            void *stream, tfe_ctx **out);
 
 /*
+ * tfe_index_build_device -- the same construction with the phrase table already on the DEVICE
+ * (phrase_tokens int32 [N][4] 16-byte aligned, phrase_len uint8 [N], init_slot int32 [N]) and
+ * every step on the GPU: key formation and input checks, two-choice cuckoo placement with
+ * 128-bit compare-and-swap / exchange on whole index slots, and a final pass in which every
+ * phrase looks itself up (which is also how equal tuples and colliding hashes are found).  The
+ * paper's index construction is its dominant offline cost (Sec. 5.3); this is that step for
+ * tables that are produced or kept on the GPU.  Results of later calls do not depend on which
+ * of the two builds made the context (only the mapping is defined, not the slot a key sits in).
+ * Synchronises `stream` (twice).  Errors as tfe_index_build; when several problems are present
+ * the one reported may differ.
+ */
+tfe_status tfe_index_build_device(const tfe_config *cfg, const int32_t *phrase_tokens,
+                                  const uint8_t *phrase_len, const int32_t *init_slot,
+                                  void *gpu_rows, void *stream, tfe_ctx **out);
+
+/*
  * tfe_cache_install -- write n fetched vectors into GPU-tier slots and make
  * their phrases GPU-resident (paper Sec. 4.3: an entry read from DRAM / SSD is
  * inserted into a faster tier when it arrives; Sec. 4.4: prefetched entries

@@ -28,7 +28,7 @@ GATE_CONST, GATE_COSINE = 0, 1
 HIDDEN_BF16, HIDDEN_F32 = 0, 1
 NO_PHRASE = 0xFFFFFFFF
 
-EXPORTS = ["tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
+EXPORTS = ["tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
            "tfe_miss_list", "tfe_miss_list_device", "tfe_destroy", "tfe_status_string",
            "tfe_last_cuda_error", "tfe_index_geometry", "tfe_phrase_key64", "tfe_home_bucket",
            "tfe_launch_geometry", "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
@@ -74,6 +74,7 @@ def lib() -> C.CDLL:
         L = C.CDLL(LIB_PATH)
         vp, i32, i64, u64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64
         L.tfe_index_build.argtypes = [C.POINTER(TfeConfig), vp, vp, vp, vp, vp, C.POINTER(vp)]
+        L.tfe_index_build_device.argtypes = L.tfe_index_build.argtypes
         L.tfe_cache_install.argtypes = [vp, i32, vp, vp, vp, vp]
         L.tfe_lookup_inject.argtypes = [vp, vp, i32, i32, i32, vp, vp, C.POINTER(TfeInjectParams), vp, vp, vp, vp]
         L.tfe_lookup_inject_host.argtypes = L.tfe_lookup_inject.argtypes
@@ -106,7 +107,7 @@ def lib() -> C.CDLL:
         L.tfe_head_buffers.argtypes = [vp, C.POINTER(vp), C.POINTER(i64), C.POINTER(vp)]
         L.tfe_head_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         L.tfe_head_geometry.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
-        for name in ("tfe_index_build", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
+        for name in ("tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
                      "tfe_miss_list", "tfe_miss_list_device", "tfe_index_geometry", "tfe_launch_geometry",
                      "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
                      "tfe_cache_policy_enable", "tfe_cache_select_victims", "tfe_cache_select_victims_device",
@@ -164,6 +165,14 @@ def tfe_index_build(cfg: TfeConfig, phrase_tokens, phrase_len, init_slot, gpu_ro
     out = C.c_void_p()
     _check(lib().tfe_index_build(C.byref(cfg), _addr(pt), _addr(pl), _addr(sl), _addr(gpu_rows),
                                  _stream(stream), C.byref(out)), "tfe_index_build")
+    return out.value
+
+
+def tfe_index_build_device(cfg: TfeConfig, phrase_tokens, phrase_len, init_slot, gpu_rows, stream=None) -> int:
+    """As tfe_index_build, with the three phrase arrays on the device (int32 [N,4], uint8 [N], int32 [N])."""
+    out = C.c_void_p()
+    _check(lib().tfe_index_build_device(C.byref(cfg), _addr(phrase_tokens), _addr(phrase_len), _addr(init_slot),
+                                        _addr(gpu_rows), _stream(stream), C.byref(out)), "tfe_index_build_device")
     return out.value
 
 

@@ -439,6 +439,115 @@ tfe_status tfe_index_build(const tfe_config *cfg, const int32_t *phrase_tokens,
     return TFE_OK;
 }
 
+tfe_status tfe_index_build_device(const tfe_config *cfg, const int32_t *phrase_tokens,
+                                  const uint8_t *phrase_len, const int32_t *init_slot, void *gpu_rows,
+                                  void *stream_, tfe_ctx **out)
+{
+    if (!out) return TFE_ERR_INVALID_ARG;
+    *out = nullptr;
+    tfe_status st = validate_config(cfg);
+    if (st != TFE_OK) return st;
+    const int64_t N = cfg->n_phrases, C = cfg->gpu_slots;
+    if (N > 0 && (!phrase_tokens || !phrase_len || !init_slot)) return TFE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(phrase_tokens) & 15u) != 0) return TFE_ERR_INVALID_ARG;
+    if (C > 0 && !gpu_rows) return TFE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(gpu_rows) & 15u) != 0) return TFE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int bits = tfe_token_bits(cfg->vocab);
+    uint32_t order_mask = 0, hashed_mask = 0;
+    for (int i = 0; i < cfg->n_orders; ++i) {
+        order_mask |= 1u << cfg->orders[i];
+        if (!tfe_order_is_packed(cfg->orders[i], bits)) hashed_mask |= 1u << cfg->orders[i];
+    }
+    const double want_slots = std::max<double>(1.0, (double)N / (double)cfg->load_factor);
+    const uint64_t n_buckets =
+        std::max<uint64_t>(1, (uint64_t)((want_slots + TFE_SLOTS_PER_BUCKET - 1) / TFE_SLOTS_PER_BUCKET));
+    if (n_buckets * TFE_SLOTS_PER_BUCKET > 0xFFFFFFFFull) return TFE_ERR_CAPACITY;
+    if ((uint64_t)N > n_buckets * TFE_SLOTS_PER_BUCKET) return TFE_ERR_CAPACITY;
+
+    tfe_ctx *c = new (std::nothrow) tfe_ctx();
+    if (!c) return TFE_ERR_INVALID_ARG;
+    c->cfg = *cfg;
+    c->tok_bits = bits;
+    c->any_hashed = hashed_mask != 0;
+    c->n_buckets = n_buckets;
+    c->row_vecs = cfg->d / 8;
+    c->gpu_rows = static_cast<uint4 *>(gpu_rows);
+    unsigned long long *d_keys = nullptr;
+    uint32_t *d_status = nullptr;
+    auto fail = [&](tfe_status s) {
+        if (d_keys) (void)cudaFree(d_keys);
+        if (d_status) (void)cudaFree(d_status);
+        tfe_destroy(c);
+        return s;
+    };
+#define CUF(call)                                                  \
+    do {                                                           \
+        if (cuda_failed((call), #call)) return fail(TFE_ERR_CUDA); \
+    } while (0)
+    CUF(cudaGetDevice(&c->device));
+    CUF(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device));
+    const size_t n_slots = (size_t)n_buckets * TFE_SLOTS_PER_BUCKET;
+    const size_t owner_entries = std::max<size_t>(4, (size_t)(C + 3) / 4 * 4);
+    CUF(cudaMalloc(&c->d_index, n_slots * sizeof(ulonglong2)));
+    CUF(cudaMalloc(&c->d_phrase_pos, std::max<size_t>(4, (size_t)N * 4)));
+    CUF(cudaMalloc(&c->d_slot_owner, owner_entries * 4));
+    CUF(cudaMalloc(&c->d_counters, TFE_CTR_WORDS * sizeof(uint32_t)));
+    CUF(cudaMalloc(&d_keys, std::max<size_t>(8, (size_t)N * 8)));
+    CUF(cudaMalloc(&d_status, sizeof(uint32_t)));
+    CUF(cudaMemsetAsync(c->d_index, 0, n_slots * sizeof(ulonglong2), stream));
+    CUF(cudaMemsetAsync(c->d_slot_owner, 0xFF, owner_entries * 4, stream));
+    CUF(cudaMemsetAsync(c->d_counters, 0, TFE_CTR_WORDS * sizeof(uint32_t), stream));
+    CUF(cudaMemsetAsync(d_status, 0, sizeof(uint32_t), stream));
+    if (c->any_hashed && N > 0) {
+        CUF(cudaMalloc(&c->d_phrase_tokens, (size_t)N * sizeof(int4)));
+        CUF(cudaMemcpyAsync(c->d_phrase_tokens, phrase_tokens, (size_t)N * sizeof(int4), cudaMemcpyDeviceToDevice, stream));
+    }
+    TfeBuildParams b{};
+    b.phrase_tokens = reinterpret_cast<const int4 *>(phrase_tokens);
+    b.phrase_len = phrase_len; b.init_slot = init_slot;
+    b.n_phrases = (uint32_t)N; b.gpu_slots = C; b.vocab = cfg->vocab; b.tok_bits = bits;
+    b.order_mask = order_mask; b.hashed_mask = hashed_mask;
+    b.max_kicks = cfg->max_kicks > 0 ? cfg->max_kicks : kDefaultMaxKicks;
+    b.keys = d_keys; b.index = c->d_index; b.n_buckets = n_buckets;
+    b.slot_owner = c->d_slot_owner; b.phrase_pos = c->d_phrase_pos; b.status = d_status;
+    uint32_t status = 0;
+    if (N > 0) {
+        const unsigned blocks = (unsigned)((N + 255) / 256);
+        tfe_build_keys_kernel<<<blocks, 256, 0, stream>>>(b);
+        // input problems end the build before anything is placed
+        CUF(cudaMemcpyAsync(&status, d_status, sizeof status, cudaMemcpyDeviceToHost, stream));
+        CUF(cudaStreamSynchronize(stream));
+        if (status & TFE_BUILD_BAD_PHRASE) return fail(TFE_ERR_INVALID_ARG);
+        if (status & TFE_BUILD_BAD_SLOT) return fail(TFE_ERR_SLOT_RANGE);
+        tfe_build_insert_kernel<<<blocks, 256, 0, stream>>>(b);
+        tfe_build_finish_kernel<<<(unsigned)((n_slots + 255) / 256), 256, 0, stream>>>(c->d_index, n_slots, c->d_phrase_pos);
+        tfe_build_verify_kernel<<<blocks, 256, 0, stream>>>(b);
+        CUF(cudaGetLastError());
+        CUF(cudaMemcpyAsync(&status, d_status, sizeof status, cudaMemcpyDeviceToHost, stream));
+    }
+    // host mirror of the residency state (tfe_cache_install checks its arguments against it)
+    c->h_slot.resize((size_t)N);
+    c->h_owner.resize((size_t)C);
+    if (N > 0) CUF(cudaMemcpyAsync(c->h_slot.data(), init_slot, (size_t)N * 4, cudaMemcpyDeviceToHost, stream));
+    if (C > 0) CUF(cudaMemcpyAsync(c->h_owner.data(), c->d_slot_owner, (size_t)C * 4, cudaMemcpyDeviceToHost, stream));
+    for (int v = 0; v < kVarCount; ++v) {
+        int occ = 0;
+        CUF(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, pick_kernel(v), TFE_BLOCK_THREADS, 0));
+        c->occ[v] = std::max(1, occ);
+    }
+    CUF(cudaStreamSynchronize(stream));
+    if (status & TFE_BUILD_DUPLICATE) return fail(TFE_ERR_DUPLICATE_PHRASE);
+    if (status & TFE_BUILD_COLLISION) return fail(TFE_ERR_KEY_COLLISION);
+    if (status & TFE_BUILD_KICKS) return fail(TFE_ERR_PROBE_LIMIT);
+    if (status & TFE_BUILD_LOST) return fail(TFE_ERR_INTERNAL);
+#undef CUF
+    (void)cudaFree(d_keys);
+    (void)cudaFree(d_status);
+    *out = c;
+    return TFE_OK;
+}
+
 tfe_status tfe_index_geometry(const tfe_ctx *c, int64_t *n_buckets, int64_t *index_bytes,
                               int64_t *metadata_bytes)
 {

@@ -1162,3 +1162,190 @@ tfe_victim_sort_kernel(const unsigned long long *list, TfeVictimState *state, ui
     }
     if (threadIdx.x == 0) state->n_out = 0;      // re-armed for the next selection
 }
+
+
+// ------------------------------------------------ index construction on the device
+//
+// The cold step of the method (the paper's index construction is its dominant offline cost):
+// N phrases -> keys -> two-choice cuckoo placement in buckets of four 16-byte slots, all on the
+// GPU.  A slot {key, value} is written and moved with 128-bit atomics, so every slot always holds
+// one whole entry and the placement needs no locks:
+//
+//   tfe_build_keys_kernel     one thread per phrase: checks its length, ids and residency, forms
+//                             the key, claims its GPU-tier slot in the owner array
+//   tfe_build_insert_kernel   one thread per phrase: compare-and-swap into a free slot of either
+//                             bucket; if both are full, exchange with a resident entry and carry
+//                             that one to its other bucket (bounded number of moves)
+//   tfe_build_finish_kernel   one thread per slot: records where each phrase ended up
+//   tfe_build_verify_kernel   one thread per phrase: looks its own key up; finding another phrase
+//                             under it means two phrases share a key -- the same tuple twice, or
+//                             (hashed orders) two tuples with one hash
+// Problems are reported as bits of a status word; the host turns them into error codes.
+#define TFE_BUILD_BAD_PHRASE 1u         // length not a configured order, id outside the vocabulary, residency < -2
+#define TFE_BUILD_BAD_SLOT 2u           // GPU-tier slot out of range or claimed twice
+#define TFE_BUILD_KICKS 4u              // an insertion ran out of moves
+#define TFE_BUILD_DUPLICATE 8u
+#define TFE_BUILD_COLLISION 16u
+#define TFE_BUILD_LOST 32u              // a phrase is not where a lookup would find it
+
+__device__ __forceinline__ ulonglong2 atomic_cas_slot(ulonglong2 *slot, ulonglong2 expect, ulonglong2 put)
+{
+    ulonglong2 old;
+    asm volatile(
+        "{\n\t.reg .b128 o, n, c;\n\t"
+        "mov.b128 c, {%2, %3};\n\t"
+        "mov.b128 n, {%4, %5};\n\t"
+        "atom.global.cas.b128 o, [%6], c, n;\n\t"
+        "mov.b128 {%0, %1}, o;\n\t}"
+        : "=l"(old.x), "=l"(old.y)
+        : "l"(expect.x), "l"(expect.y), "l"(put.x), "l"(put.y), "l"(slot)
+        : "memory");
+    return old;
+}
+
+__device__ __forceinline__ ulonglong2 atomic_exch_slot(ulonglong2 *slot, ulonglong2 put)
+{
+    ulonglong2 old;
+    asm volatile(
+        "{\n\t.reg .b128 o, n;\n\t"
+        "mov.b128 n, {%2, %3};\n\t"
+        "atom.global.exch.b128 o, [%4], n;\n\t"
+        "mov.b128 {%0, %1}, o;\n\t}"
+        : "=l"(old.x), "=l"(old.y)
+        : "l"(put.x), "l"(put.y), "l"(slot)
+        : "memory");
+    return old;
+}
+
+struct TfeBuildParams {
+    const int4 *phrase_tokens;      // [N]
+    const uint8_t *phrase_len;      // [N]
+    const int32_t *init_slot;       // [N]
+    uint32_t n_phrases;
+    int64_t gpu_slots;
+    int32_t vocab, tok_bits;
+    uint32_t order_mask;            // bit n set: n is a configured order
+    uint32_t hashed_mask;           // bit n set: order n is hashed
+    int32_t max_kicks;
+    unsigned long long *keys;       // [N] work array
+    ulonglong2 *index;
+    uint64_t n_buckets;
+    uint32_t *slot_owner;           // [C], preset to "no owner"
+    uint32_t *phrase_pos;           // [N]
+    uint32_t *status;
+};
+
+__global__ void __launch_bounds__(256)
+tfe_build_keys_kernel(const TfeBuildParams p)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= p.n_phrases) return;
+    const int n = p.phrase_len[i];
+    const int4 t = p.phrase_tokens[i];
+    const int32_t tok[4] = {t.x, t.y, t.z, t.w};
+    bool ok = n >= 1 && n <= 4 && ((p.order_mask >> n) & 1u);
+    int32_t tk[4] = {-1, -1, -1, -1};       // tk[j] = id at distance j before the phrase's last token
+    if (ok) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (j < n) {
+                const int32_t x = tok[n - 1 - j];
+                if (x < 0 || x >= p.vocab) ok = false;
+                tk[j] = x;
+            }
+    }
+    const int32_t s = p.init_slot[i];
+    if (s < -2) ok = false;
+    if (!ok) {
+        atomicOr(p.status, TFE_BUILD_BAD_PHRASE);
+        p.keys[i] = 0ull;
+        return;
+    }
+    p.keys[i] = tfe_make_key(n, tk, p.tok_bits);
+    if (s >= 0) {
+        if ((int64_t)s >= p.gpu_slots || atomicCAS(&p.slot_owner[s], 0xFFFFFFFFu, i) != 0xFFFFFFFFu)
+            atomicOr(p.status, TFE_BUILD_BAD_SLOT);
+    }
+}
+
+__global__ void __launch_bounds__(256)
+tfe_build_insert_kernel(const TfeBuildParams p)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= p.n_phrases) return;
+    ulonglong2 cur;
+    cur.x = p.keys[i];
+    if (cur.x == 0ull) return;              // refused by the checks
+    cur.y = ((unsigned long long)i << 32) | (uint32_t)p.init_slot[i];
+    const ulonglong2 empty = make_ulonglong2(0ull, 0ull);
+    uint64_t first = tfe_home_bucket_of(cur.x, p.n_buckets);
+    uint32_t rng = i * 2654435761u + 12345u;
+    for (int32_t kick = 0; kick <= p.max_kicks; ++kick) {
+        // a free slot in the bucket at hand, then in the entry's other bucket
+        const uint64_t home = tfe_home_bucket_of(cur.x, p.n_buckets);
+        const uint64_t second = tfe_second_bucket_of(cur.x, home, p.n_buckets);
+        const uint64_t other = first == home ? second : home;
+#pragma unroll
+        for (int which = 0; which < 2; ++which) {
+            ulonglong2 *bucket = p.index + (which == 0 ? first : other) * TFE_SLOTS_PER_BUCKET;
+            for (int sl = 0; sl < TFE_SLOTS_PER_BUCKET; ++sl) {
+                if (__ldcg(&bucket[sl].x) != 0ull) continue;
+                if (atomic_cas_slot(bucket + sl, empty, cur).x == 0ull) return;      // placed
+            }
+        }
+        // both full: take the place of a resident entry of the bucket at hand and carry that one
+        // to its other bucket (the walk moves on from there)
+        rng = rng * 1664525u + 1013904223u;
+        ulonglong2 *victim = p.index + first * TFE_SLOTS_PER_BUCKET + (rng >> 30);
+        const ulonglong2 out = atomic_exch_slot(victim, cur);
+        if (out.x == 0ull) return;          // cannot happen (slots are never emptied); placed either way
+        cur = out;
+        const uint64_t h2 = tfe_home_bucket_of(cur.x, p.n_buckets);
+        first = h2 == first ? tfe_second_bucket_of(cur.x, h2, p.n_buckets) : h2;
+    }
+    atomicOr(p.status, TFE_BUILD_KICKS);
+}
+
+__global__ void __launch_bounds__(256)
+tfe_build_finish_kernel(const ulonglong2 *index, uint64_t n_slots, uint32_t *phrase_pos)
+{
+    const uint64_t s = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= n_slots) return;
+    const ulonglong2 e = index[s];
+    if (e.x != 0ull) phrase_pos[(uint32_t)(e.y >> 32)] = (uint32_t)s;
+}
+
+__global__ void __launch_bounds__(256)
+tfe_build_verify_kernel(const TfeBuildParams p)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= p.n_phrases) return;
+    const unsigned long long key = p.keys[i];
+    if (key == 0ull) return;
+    const uint64_t b1 = tfe_home_bucket_of(key, p.n_buckets);
+    const uint64_t b2 = tfe_second_bucket_of(key, b1, p.n_buckets);
+    uint32_t found = 0xFFFFFFFFu;
+    bool mine = false;
+#pragma unroll
+    for (int which = 0; which < 2; ++which) {
+        const ulonglong2 *bucket = p.index + (which == 0 ? b1 : b2) * TFE_SLOTS_PER_BUCKET;
+        for (int sl = 0; sl < TFE_SLOTS_PER_BUCKET; ++sl) {
+            const ulonglong2 e = bucket[sl];
+            if (e.x != key) continue;
+            const uint32_t id = (uint32_t)(e.y >> 32);
+            if (id == i) mine = true; else found = id;
+        }
+        if (b2 == b1) break;
+    }
+    if (!mine) atomicOr(p.status, TFE_BUILD_LOST);
+    if (found != 0xFFFFFFFFu) {
+        const int n = p.phrase_len[i];
+        bool same = p.phrase_len[found] == n;
+        if (same && ((p.hashed_mask >> n) & 1u)) {
+            const int4 a = p.phrase_tokens[i], b = p.phrase_tokens[found];
+            const int32_t ta[4] = {a.x, a.y, a.z, a.w}, tb[4] = {b.x, b.y, b.z, b.w};
+            for (int j = 0; j < n; ++j) same = same && ta[j] == tb[j];
+        }
+        atomicOr(p.status, same ? TFE_BUILD_DUPLICATE : TFE_BUILD_COLLISION);
+    }
+}

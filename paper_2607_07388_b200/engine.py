@@ -25,7 +25,7 @@ class Engram:
     """GPU-resident phrase index + GPU-tier row store for one table."""
 
     def __init__(self, phrase_tokens, phrase_len, init_slot, gpu_rows: torch.Tensor, *, vocab, orders,
-                 load_factor=0.7, hidden_dtype=tfe.HIDDEN_BF16, max_kicks=0, stream=None):
+                 load_factor=0.7, hidden_dtype=tfe.HIDDEN_BF16, max_kicks=0, stream=None, device_build=False):
         assert gpu_rows.is_cuda and gpu_rows.dtype == torch.bfloat16 and gpu_rows.is_contiguous()
         self.rows = gpu_rows
         self.C, self.d = gpu_rows.shape
@@ -35,10 +35,20 @@ class Engram:
         self.cfg = tfe.make_config(d=self.d, vocab=vocab, orders=self.orders, n_phrases=len(phrase_len),
                                    gpu_slots=self.C, load_factor=load_factor, hidden_dtype=hidden_dtype,
                                    max_kicks=max_kicks)
-        self.ctx = tfe.tfe_index_build(self.cfg, phrase_tokens, phrase_len, init_slot, gpu_rows, stream)
+        self.ctx = 0
+        if device_build:        # the phrase arrays go to (or already are on) the device; the index is built there
+            dev = gpu_rows.device
+            as_dev = lambda a, dt: a.to(dev, dt).contiguous() if torch.is_tensor(a) else \
+                torch.from_numpy(np.ascontiguousarray(a)).to(dev, dt)
+            pt = as_dev(phrase_tokens, torch.int32).reshape(-1, 4)
+            pl = as_dev(phrase_len, torch.uint8)
+            sl = as_dev(init_slot, torch.int32)
+            self.ctx = tfe.tfe_index_build_device(self.cfg, pt, pl, sl, gpu_rows, stream)
+        else:
+            self.ctx = tfe.tfe_index_build(self.cfg, phrase_tokens, phrase_len, init_slot, gpu_rows, stream)
 
     def close(self):
-        if self.ctx:
+        if getattr(self, "ctx", 0):
             tfe.tfe_destroy(self.ctx)
             self.ctx = 0
 

@@ -28,14 +28,14 @@ class Pair:
     """One table, twice: ``eng`` on the GPU, ``ora`` on the CPU."""
 
     def __init__(self, pt, pl, init_slot, rows_bits, *, vocab, orders, load_factor=0.7, hidden_dtype=0,
-                 max_kicks=0):
+                 max_kicks=0, device_build=False):
         self.rows_bits = np.ascontiguousarray(rows_bits, np.uint16)
         C, d = self.rows_bits.shape
         self.d, self.C, self.orders, self.hidden_dtype = d, C, tuple(orders), hidden_dtype
         self.rows_gpu = bf16_tensor_from_bits(self.rows_bits, DEV)
         self.eng = Engram(pt, pl, init_slot, self.rows_gpu, vocab=vocab, orders=orders,
                           load_factor=load_factor, hidden_dtype=hidden_dtype,
-                          max_kicks=max_kicks)
+                          max_kicks=max_kicks, device_build=device_build)
         self.ora = orc.Oracle(pt, pl, init_slot, self.rows_bits.copy(), d=d, vocab=vocab, orders=orders,
                               gpu_slots=C)
 
