@@ -103,7 +103,9 @@ tfe_status tfe_index_build(const tfe_config *cfg, const int32_t *phrase_tokens,
  * paper's index construction is its dominant offline cost (Sec. 5.3); this is that step for
  * tables that are produced or kept on the GPU.  Results of later calls do not depend on which
  * of the two builds made the context (only the mapping is defined, not the slot a key sits in).
- * Synchronises `stream` (twice).  Errors as tfe_index_build; when several problems are present
+ * Two kernel launches, one synchronisation of `stream`; the host-side copy of the residency
+ * state that tfe_cache_install checks its arguments against is fetched on its first call.
+ * Errors as tfe_index_build; when several problems are present
  * the one reported may differ.
  */
 tfe_status tfe_index_build_device(const tfe_config *cfg, const int32_t *phrase_tokens,

@@ -91,6 +91,8 @@ struct tfe_ctx {
     unsigned long long *d_vs_list = nullptr;
     int32_t *d_vs_slots = nullptr;
 
+    bool mirror_ready = true;               // h_slot / h_owner filled (a device build fills them on first use)
+
     // host-buffer variant staging
     int32_t *d_h_tokens = nullptr;
     void *d_h_hidden = nullptr, *d_h_out = nullptr;
@@ -473,10 +475,8 @@ tfe_status tfe_index_build_device(const tfe_config *cfg, const int32_t *phrase_t
     c->n_buckets = n_buckets;
     c->row_vecs = cfg->d / 8;
     c->gpu_rows = static_cast<uint4 *>(gpu_rows);
-    unsigned long long *d_keys = nullptr;
     uint32_t *d_status = nullptr;
     auto fail = [&](tfe_status s) {
-        if (d_keys) (void)cudaFree(d_keys);
         if (d_status) (void)cudaFree(d_status);
         tfe_destroy(c);
         return s;
@@ -493,7 +493,6 @@ tfe_status tfe_index_build_device(const tfe_config *cfg, const int32_t *phrase_t
     CUF(cudaMalloc(&c->d_phrase_pos, std::max<size_t>(4, (size_t)N * 4)));
     CUF(cudaMalloc(&c->d_slot_owner, owner_entries * 4));
     CUF(cudaMalloc(&c->d_counters, TFE_CTR_WORDS * sizeof(uint32_t)));
-    CUF(cudaMalloc(&d_keys, std::max<size_t>(8, (size_t)N * 8)));
     CUF(cudaMalloc(&d_status, sizeof(uint32_t)));
     CUF(cudaMemsetAsync(c->d_index, 0, n_slots * sizeof(ulonglong2), stream));
     CUF(cudaMemsetAsync(c->d_slot_owner, 0xFF, owner_entries * 4, stream));
@@ -509,40 +508,30 @@ tfe_status tfe_index_build_device(const tfe_config *cfg, const int32_t *phrase_t
     b.n_phrases = (uint32_t)N; b.gpu_slots = C; b.vocab = cfg->vocab; b.tok_bits = bits;
     b.order_mask = order_mask; b.hashed_mask = hashed_mask;
     b.max_kicks = cfg->max_kicks > 0 ? cfg->max_kicks : kDefaultMaxKicks;
-    b.keys = d_keys; b.index = c->d_index; b.n_buckets = n_buckets;
+    b.index = c->d_index; b.n_buckets = n_buckets;
     b.slot_owner = c->d_slot_owner; b.phrase_pos = c->d_phrase_pos; b.status = d_status;
     uint32_t status = 0;
     if (N > 0) {
         const unsigned blocks = (unsigned)((N + 255) / 256);
-        tfe_build_keys_kernel<<<blocks, 256, 0, stream>>>(b);
-        // input problems end the build before anything is placed
-        CUF(cudaMemcpyAsync(&status, d_status, sizeof status, cudaMemcpyDeviceToHost, stream));
-        CUF(cudaStreamSynchronize(stream));
-        if (status & TFE_BUILD_BAD_PHRASE) return fail(TFE_ERR_INVALID_ARG);
-        if (status & TFE_BUILD_BAD_SLOT) return fail(TFE_ERR_SLOT_RANGE);
         tfe_build_insert_kernel<<<blocks, 256, 0, stream>>>(b);
-        tfe_build_finish_kernel<<<(unsigned)((n_slots + 255) / 256), 256, 0, stream>>>(c->d_index, n_slots, c->d_phrase_pos);
         tfe_build_verify_kernel<<<blocks, 256, 0, stream>>>(b);
         CUF(cudaGetLastError());
         CUF(cudaMemcpyAsync(&status, d_status, sizeof status, cudaMemcpyDeviceToHost, stream));
     }
-    // host mirror of the residency state (tfe_cache_install checks its arguments against it)
-    c->h_slot.resize((size_t)N);
-    c->h_owner.resize((size_t)C);
-    if (N > 0) CUF(cudaMemcpyAsync(c->h_slot.data(), init_slot, (size_t)N * 4, cudaMemcpyDeviceToHost, stream));
-    if (C > 0) CUF(cudaMemcpyAsync(c->h_owner.data(), c->d_slot_owner, (size_t)C * 4, cudaMemcpyDeviceToHost, stream));
+    c->mirror_ready = false;        // the host mirror of the residency state is fetched when tfe_cache_install first needs it
     for (int v = 0; v < kVarCount; ++v) {
         int occ = 0;
         CUF(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, pick_kernel(v), TFE_BLOCK_THREADS, 0));
         c->occ[v] = std::max(1, occ);
     }
     CUF(cudaStreamSynchronize(stream));
+    if (status & TFE_BUILD_BAD_PHRASE) return fail(TFE_ERR_INVALID_ARG);
+    if (status & TFE_BUILD_BAD_SLOT) return fail(TFE_ERR_SLOT_RANGE);
     if (status & TFE_BUILD_DUPLICATE) return fail(TFE_ERR_DUPLICATE_PHRASE);
     if (status & TFE_BUILD_COLLISION) return fail(TFE_ERR_KEY_COLLISION);
     if (status & TFE_BUILD_KICKS) return fail(TFE_ERR_PROBE_LIMIT);
     if (status & TFE_BUILD_LOST) return fail(TFE_ERR_INTERNAL);
 #undef CUF
-    (void)cudaFree(d_keys);
     (void)cudaFree(d_status);
     *out = c;
     return TFE_OK;
@@ -577,6 +566,35 @@ tfe_status tfe_launch_geometry(const tfe_ctx *c, int32_t *grid, int32_t *block, 
     return TFE_OK;
 }
 
+namespace {
+
+// Host mirror {phrase -> residency, slot -> owner} of a context built on the device, read back
+// from the index; synchronises the stream.
+tfe_status fetch_mirror(tfe_ctx *c, cudaStream_t stream)
+{
+    const int64_t N = c->cfg.n_phrases, C = c->cfg.gpu_slots;
+    c->h_slot.resize((size_t)N);
+    c->h_owner.resize((size_t)C);
+    int32_t *d_res = nullptr;
+    if (N > 0) {
+        CU(cudaMalloc(&d_res, (size_t)N * 4));
+        tfe_gather_residency_kernel<<<(unsigned)((N + 255) / 256), 256, 0, stream>>>(c->d_index, c->d_phrase_pos,
+                                                                                  (uint32_t)N, d_res);
+        const cudaError_t e1 = cudaMemcpyAsync(c->h_slot.data(), d_res, (size_t)N * 4, cudaMemcpyDeviceToHost, stream);
+        const cudaError_t e2 = cudaStreamSynchronize(stream);
+        (void)cudaFree(d_res);
+        if (cuda_failed(e1, "copy of the residency mirror") || cuda_failed(e2, "cudaStreamSynchronize")) return TFE_ERR_CUDA;
+    }
+    if (C > 0) {
+        CU(cudaMemcpyAsync(c->h_owner.data(), c->d_slot_owner, (size_t)C * 4, cudaMemcpyDeviceToHost, stream));
+        CU(cudaStreamSynchronize(stream));
+    }
+    c->mirror_ready = true;
+    return TFE_OK;
+}
+
+}  // namespace
+
 tfe_status tfe_cache_install(tfe_ctx *c, int32_t n, const uint32_t *phrase_ids, const void *src_rows,
                              const int32_t *dst_slots, void *stream_)
 {
@@ -586,6 +604,10 @@ tfe_status tfe_cache_install(tfe_ctx *c, int32_t n, const uint32_t *phrase_ids, 
     if ((reinterpret_cast<uintptr_t>(src_rows) & 15u) != 0) return TFE_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const int64_t N = c->cfg.n_phrases, C = c->cfg.gpu_slots;
+    if (!c->mirror_ready) {
+        const tfe_status ms = fetch_mirror(c, stream);
+        if (ms != TFE_OK) return ms;
+    }
     for (int32_t k = 0; k < n; ++k) {
         if ((int64_t)phrase_ids[k] >= N) return TFE_ERR_UNKNOWN_PHRASE;
         if (c->h_slot[phrase_ids[k]] >= 0) return TFE_ERR_ALREADY_RESIDENT;

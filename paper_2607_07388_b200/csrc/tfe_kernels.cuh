@@ -1171,15 +1171,14 @@ tfe_victim_sort_kernel(const unsigned long long *list, TfeVictimState *state, ui
 // GPU.  A slot {key, value} is written and moved with 128-bit atomics, so every slot always holds
 // one whole entry and the placement needs no locks:
 //
-//   tfe_build_keys_kernel     one thread per phrase: checks its length, ids and residency, forms
-//                             the key, claims its GPU-tier slot in the owner array
-//   tfe_build_insert_kernel   one thread per phrase: compare-and-swap into a free slot of either
-//                             bucket; if both are full, exchange with a resident entry and carry
-//                             that one to its other bucket (bounded number of moves)
-//   tfe_build_finish_kernel   one thread per slot: records where each phrase ended up
-//   tfe_build_verify_kernel   one thread per phrase: looks its own key up; finding another phrase
-//                             under it means two phrases share a key -- the same tuple twice, or
-//                             (hashed orders) two tuples with one hash
+//   tfe_build_insert_kernel   one thread per phrase: checks its length, ids and residency, forms
+//                             the key, claims its GPU-tier slot in the owner array, then
+//                             compare-and-swaps the entry into a free slot of either bucket; if
+//                             both are full it exchanges with a resident entry and carries that
+//                             one to its other bucket (bounded number of moves)
+//   tfe_build_verify_kernel   one thread per phrase: looks its own key up and records where it
+//                             sits; finding another phrase under the key means two phrases share
+//                             it -- the same tuple twice, or (hashed orders) two tuples, one hash
 // Problems are reported as bits of a status word; the host turns them into error codes.
 #define TFE_BUILD_BAD_PHRASE 1u         // length not a configured order, id outside the vocabulary, residency < -2
 #define TFE_BUILD_BAD_SLOT 2u           // GPU-tier slot out of range or claimed twice
@@ -1227,7 +1226,6 @@ struct TfeBuildParams {
     uint32_t order_mask;            // bit n set: n is a configured order
     uint32_t hashed_mask;           // bit n set: order n is hashed
     int32_t max_kicks;
-    unsigned long long *keys;       // [N] work array
     ulonglong2 *index;
     uint64_t n_buckets;
     uint32_t *slot_owner;           // [C], preset to "no owner"
@@ -1235,37 +1233,23 @@ struct TfeBuildParams {
     uint32_t *status;
 };
 
-__global__ void __launch_bounds__(256)
-tfe_build_keys_kernel(const TfeBuildParams p)
+// Key of phrase i, or 0 if its length is not a configured order or it holds an id outside the vocabulary.
+__device__ __forceinline__ unsigned long long tfe_build_key(const TfeBuildParams &p, uint32_t i)
 {
-    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= p.n_phrases) return;
     const int n = p.phrase_len[i];
+    if (n < 1 || n > 4 || !((p.order_mask >> n) & 1u)) return 0ull;
     const int4 t = p.phrase_tokens[i];
     const int32_t tok[4] = {t.x, t.y, t.z, t.w};
-    bool ok = n >= 1 && n <= 4 && ((p.order_mask >> n) & 1u);
     int32_t tk[4] = {-1, -1, -1, -1};       // tk[j] = id at distance j before the phrase's last token
-    if (ok) {
+    bool ok = true;
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (j < n) {
-                const int32_t x = tok[n - 1 - j];
-                if (x < 0 || x >= p.vocab) ok = false;
-                tk[j] = x;
-            }
-    }
-    const int32_t s = p.init_slot[i];
-    if (s < -2) ok = false;
-    if (!ok) {
-        atomicOr(p.status, TFE_BUILD_BAD_PHRASE);
-        p.keys[i] = 0ull;
-        return;
-    }
-    p.keys[i] = tfe_make_key(n, tk, p.tok_bits);
-    if (s >= 0) {
-        if ((int64_t)s >= p.gpu_slots || atomicCAS(&p.slot_owner[s], 0xFFFFFFFFu, i) != 0xFFFFFFFFu)
-            atomicOr(p.status, TFE_BUILD_BAD_SLOT);
-    }
+    for (int j = 0; j < 4; ++j)
+        if (j < n) {
+            const int32_t x = tok[n - 1 - j];
+            if (x < 0 || x >= p.vocab) ok = false;
+            tk[j] = x;
+        }
+    return ok ? tfe_make_key(n, tk, p.tok_bits) : 0ull;
 }
 
 __global__ void __launch_bounds__(256)
@@ -1274,9 +1258,19 @@ tfe_build_insert_kernel(const TfeBuildParams p)
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= p.n_phrases) return;
     ulonglong2 cur;
-    cur.x = p.keys[i];
-    if (cur.x == 0ull) return;              // refused by the checks
-    cur.y = ((unsigned long long)i << 32) | (uint32_t)p.init_slot[i];
+    cur.x = tfe_build_key(p, i);
+    const int32_t res = p.init_slot[i];
+    if (cur.x == 0ull || res < -2) {
+        atomicOr(p.status, TFE_BUILD_BAD_PHRASE);
+        return;
+    }
+    if (res >= 0) {
+        if ((int64_t)res >= p.gpu_slots || atomicCAS(&p.slot_owner[res], 0xFFFFFFFFu, i) != 0xFFFFFFFFu) {
+            atomicOr(p.status, TFE_BUILD_BAD_SLOT);
+            return;
+        }
+    }
+    cur.y = ((unsigned long long)i << 32) | (uint32_t)res;
     const ulonglong2 empty = make_ulonglong2(0ull, 0ull);
     uint64_t first = tfe_home_bucket_of(cur.x, p.n_buckets);
     uint32_t rng = i * 2654435761u + 12345u;
@@ -1307,37 +1301,29 @@ tfe_build_insert_kernel(const TfeBuildParams p)
 }
 
 __global__ void __launch_bounds__(256)
-tfe_build_finish_kernel(const ulonglong2 *index, uint64_t n_slots, uint32_t *phrase_pos)
-{
-    const uint64_t s = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (s >= n_slots) return;
-    const ulonglong2 e = index[s];
-    if (e.x != 0ull) phrase_pos[(uint32_t)(e.y >> 32)] = (uint32_t)s;
-}
-
-__global__ void __launch_bounds__(256)
 tfe_build_verify_kernel(const TfeBuildParams p)
 {
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= p.n_phrases) return;
-    const unsigned long long key = p.keys[i];
+    const unsigned long long key = tfe_build_key(p, i);
     if (key == 0ull) return;
     const uint64_t b1 = tfe_home_bucket_of(key, p.n_buckets);
     const uint64_t b2 = tfe_second_bucket_of(key, b1, p.n_buckets);
-    uint32_t found = 0xFFFFFFFFu;
-    bool mine = false;
+    uint32_t found = 0xFFFFFFFFu, mine = 0xFFFFFFFFu;
 #pragma unroll
     for (int which = 0; which < 2; ++which) {
-        const ulonglong2 *bucket = p.index + (which == 0 ? b1 : b2) * TFE_SLOTS_PER_BUCKET;
+        const uint64_t b = which == 0 ? b1 : b2;
+        const ulonglong2 *bucket = p.index + b * TFE_SLOTS_PER_BUCKET;
         for (int sl = 0; sl < TFE_SLOTS_PER_BUCKET; ++sl) {
             const ulonglong2 e = bucket[sl];
             if (e.x != key) continue;
             const uint32_t id = (uint32_t)(e.y >> 32);
-            if (id == i) mine = true; else found = id;
+            if (id == i) mine = (uint32_t)(b * TFE_SLOTS_PER_BUCKET + sl); else found = id;
         }
         if (b2 == b1) break;
     }
-    if (!mine) atomicOr(p.status, TFE_BUILD_LOST);
+    if (mine == 0xFFFFFFFFu) atomicOr(p.status, TFE_BUILD_LOST);
+    else p.phrase_pos[i] = mine;            // where the entry sits (the install kernel rewrites its value there)
     if (found != 0xFFFFFFFFu) {
         const int n = p.phrase_len[i];
         bool same = p.phrase_len[found] == n;
@@ -1348,4 +1334,13 @@ tfe_build_verify_kernel(const TfeBuildParams p)
         }
         atomicOr(p.status, same ? TFE_BUILD_DUPLICATE : TFE_BUILD_COLLISION);
     }
+}
+
+// Residency of every phrase as the index holds it (>= 0 slot, -1 host, -2 SSD): the host-side
+// mirror of a context built on the device is filled from this on its first use.
+__global__ void __launch_bounds__(256)
+tfe_gather_residency_kernel(const ulonglong2 *index, const uint32_t *phrase_pos, uint32_t n_phrases, int32_t *out)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n_phrases) out[i] = (int32_t)(uint32_t)index[phrase_pos[i]].y;
 }
