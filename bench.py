@@ -896,9 +896,10 @@ def run_sweep(a, dev, rank):
 
 TFE_CTR_BYTES = 16      # the launch-state words tfe_miss_list reads back
 NBUF_DECODE = 32        # decode shapes: this many distinct query / hidden-state sets rotate
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the lookup kernel, from the ncu capture
-# summarised under profiles/ (a 1M-phrase capture scaled is not needed: traffic does not depend on N)
-NCU_TRAFFIC = {"c3_prefill8x4096": 124_960_000}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the lookup kernel in steady state (no cache
+# flush between launches, so the write-back of the previous launch's output is included), from the ncu
+# capture summarised under profiles/; taken on a 1M-phrase table: traffic does not depend on N
+NCU_TRAFFIC = {"c3_prefill8x4096": 163_200_000}
 
 
 # ------------------------------------------------------------ reference arm
