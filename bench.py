@@ -64,6 +64,8 @@ def parse_args():
     ap.add_argument("--head-vocab", type=int, default=synth.VOCAB)
     ap.add_argument("--head-d", type=int, default=1024)
     ap.add_argument("--head-batch", type=int, default=64)
+    ap.add_argument("--variants", action="store_true",
+                    help="time the other selection policies and gates (ALL, COSINE, a lambda that is not a bf16 number)")
     ap.add_argument("--build", action="store_true",
                     help="time index construction on the GPU (tfe_index_build_device) against the host build")
     ap.add_argument("--cache-policy", action="store_true",
@@ -199,8 +201,8 @@ def oracle_step(orc, ora, tok, h, q_start):
     return ref, rounded
 
 
-def materialise_rows_for(ora, w, tok, q_start):
-    ref = ora.lookup(tok, q_start)
+def materialise_rows_for(ora, w, tok, q_start, policy=0):
+    ref = ora.lookup(tok, q_start, policy=policy)
     hit = ref.flags == 1
     slots = np.unique(ref.sel_slot[hit])
     ora._sparse.materialise(slots, ora.slot_owner[slots])
@@ -410,6 +412,8 @@ def run_ours(a):
         return run_head(a, dev, rank)
     if a.build:
         return run_build(a, dev, rank)
+    if a.variants:
+        return run_variants(a, dev, rank)
 
     w = make_workload(a)
     sampler = ClockSampler(local_rank) if rank == 0 else None
@@ -843,6 +847,59 @@ def run_build(a, dev, rank):
                              "ms": host_s * 1e3},
             "parity": {"device_vs_host_build": bool(same), "device_build_vs_oracle": oracle_ok}}))
     eng.close(); host.close()
+
+
+def run_variants(a, dev, rank):
+    """The lookup with the other policies / gates of the injection rule, on the workload's inputs."""
+    import torch
+    from paper_2607_07388_b200 import binding as tfe
+    from paper_2607_07388_b200.engine import bits_from_bf16_tensor
+    L = tfe.lib()
+    w = make_workload(a)
+    nbuf = 4 if w.shape == "prefill" else NBUF_DECODE
+    sess = Session(w, dev, nbuf, a.tune_batch)
+    stream = torch.cuda.current_stream()
+    sp = stream.cuda_stream
+    peak, peak_src = measured_peak()
+    orc, ora = oracle_for(w, sess.tb)
+    materialise_rows_for(ora, w, sess.toks_np[0], w.q_start, policy=1)       # every matched order's row
+    h0 = bits_from_bf16_tensor(sess.hs[0])
+    pairs = float(np.mean([valid_pairs(t, w.q_start, w.orders, w.vocab) for t in sess.toks_np]))
+    rows_out = []
+    for name, pol, gate, lam in (("LONGEST / CONST", 0, 0, 1.0), ("LONGEST / CONST, lambda 0.3", 0, 0, 0.3),
+                                 ("LONGEST / COSINE", 0, 1, 1.0), ("ALL / CONST", 1, 0, 1.0), ("ALL / COSINE", 1, 1, 1.0)):
+        prm = tfe.TfeInjectParams(pol, gate, lam)
+        calls = [(sess.eng.ctx, sess.toks[v].data_ptr(), w.B, w.T, w.q_start, sess.hs[v].data_ptr(),
+                  sess.outs[v].data_ptr(), C.byref(prm), None, None, None, sp) for v in range(nbuf)]
+
+        def step(i):
+            st = L.tfe_lookup_inject(*calls[i % nbuf])
+            if st:
+                raise RuntimeError(f"tfe_lookup_inject failed: {st}")
+
+        ms, _ = timed_region(step, a.steps, max(3, a.warmup), stream, 1, None, dev)
+        us = ms / a.steps * 1e3
+        # rows gathered (every GPU-resident matched order in ALL mode) and parity on buffer 0
+        n_rows, n_miss = [], []
+        for v in range(nbuf):
+            ref = ora.lookup(sess.toks_np[v], w.q_start, policy=pol)
+            n_rows.append(int((ref.flags == 1).sum())); n_miss.append(int((ref.flags >= 2).sum()))
+        step(0)
+        torch.cuda.synchronize()
+        ref = ora.lookup(sess.toks_np[0], w.q_start, policy=pol)
+        exact, _ = ora.inject(ref, h0, policy=pol, gate=gate, lam=lam)
+        got = synth.bf16_bits_to_f32(bits_from_bf16_tensor(sess.outs[0])).astype(np.float64)
+        err = float(np.abs(got - exact).max())
+        bytes_alg = w.B * w.T * 4 + pairs * 128 + 2 * w.Q * w.d * 2 + float(np.mean(n_rows)) * w.d * 2 + float(np.mean(n_miss)) * 9
+        rows_out.append({"variant": name, "us_per_call": us, "tokens_per_s": w.Q / (us * 1e-6),
+                         "rows_gathered": float(np.mean(n_rows)), "algorithmic_bytes": bytes_alg,
+                         "achieved_gbs": bytes_alg / us / 1e3, "frac_of_measured_peak": bytes_alg / us / 1e3 / peak,
+                         "out_max_abs_err": err, "within_2e-2": bool(err <= 2e-2)})
+    if rank == 0:
+        print(json.dumps({"metric": "lookup+inject tokens/s by policy and gate", "unit": "tokens/s",
+                          "config": {"workload": w.name, "Q": w.Q, "d": w.d, "launches": "direct, one per step"},
+                          "peak": peak, "peak_source": peak_src, "steps": a.steps, "variants": rows_out}))
+    sess.close()
 
 
 def run_sweep(a, dev, rank):

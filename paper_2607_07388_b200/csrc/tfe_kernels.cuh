@@ -397,12 +397,14 @@ __device__ __forceinline__ int32_t tfe_select_longest(const TfeLookupParams &p, 
 // --------------------------------------------------------------- the hot path
 //
 // One launch does everything, and every warp works on its own: it takes batches of `qb`
-// consecutive queries (qb = 1, 2, 4 or 8) in a grid-strided order and runs two phases per batch.
+// queries (1..8; query lq of batch b is b + lq * n_batches, so neighbouring positions go to
+// different warps) in a grid-strided order and runs two phases per batch.
 //
 //   Probe   one THREAD per (query, order): lane 4*ql + oi forms the key of the trailing
-//           orders[oi]-gram of the batch's query ql, fetches the whole 128-byte home bucket with
-//           four 32-byte loads and scans it in registers; a full bucket without the key sends it
-//           on to the next one.  A match of a hashed order is confirmed against the stored tuple.
+//           orders[oi]-gram of the batch's query ql, fetches both candidate buckets (64 bytes
+//           each: two-choice cuckoo hashing, a key sits in one of the two) with four 32-byte
+//           loads and scans them in registers.  A match of a hashed order is confirmed against
+//           the stored tuple.
 //           The four lanes of a query then agree on the retained phrase (LONGEST) or each keeps
 //           its own (ALL); lane 4*ql records the result.
 //   Gather  the whole warp per query: h streams to out in 16-byte vectors, GPU hits fetch their
@@ -442,10 +444,10 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
 
     const uint32_t n_warps = gridDim.x * TFE_WARPS_PER_BLOCK;
     for (uint32_t batch = blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5); batch < n_batches; batch += n_warps) {
-        const uint32_t q0 = batch * qb;
-
+        // query lq of batch b is b + lq * n_batches: the queries of a warp are spread over the call,
+        // so a run of consecutive positions that all hit is shared out among many warps
         // ================================ probe phase ================================
-        const uint32_t q = q0 + ql;
+        const uint32_t q = batch + (uint32_t)ql * n_batches;
         const bool mine = ql < (int)qb && q < p.Q;
         const unsigned long long found = tfe_probe_lane(p, q, mine, my_order, my_hashed);
         // ---- selection policy + tier walk; the 4 lanes of a query form one aligned quad
@@ -483,7 +485,7 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
 
         // ================================ gather phase ===============================
         for (uint32_t lq = 0; lq < qb; ++lq) {
-            const uint32_t gq = q0 + lq;
+            const uint32_t gq = batch + lq * n_batches;
             if (gq >= p.Q) break;
             const char *hrow = reinterpret_cast<const char *>(p.h) + (size_t)gq * hid_row_bytes;
             char *orow = reinterpret_cast<char *>(p.out) + (size_t)gq * hid_row_bytes;
@@ -517,8 +519,51 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
                 continue;
             }
             float gate = p.lambda;
+            if constexpr (COS && !ALL) {
+                // a row of at most 32 * UNROLL steps stays in registers between the dot products
+                // and the update: one trip to memory instead of two
+                if (steps <= 32 * UNROLL) {
+                    uint4 hv[UNROLL];
+                    typename TfeVec<HT>::RowRaw rv[UNROLL];
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u) {
+                        const int k = u * 32 + lane;
+                        if (k < steps) {
+                            hv[u] = ld_stream(reinterpret_cast<const uint4 *>(hrow) + k);
+                            rv[u] = ld_row_raw<HT>(rowp[0], k);
+                        }
+                    }
+                    float sa = 0.f, sb = 0.f, sc = 0.f;      // <h,m>, <h,h>, <m,m>, same order of terms as below
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u) {
+                        if (u * 32 + lane >= steps) continue;
+                        float x[VN], m[VN];
+                        unpack_hidden<HT>(hv[u], x);
+                        unpack_row<HT>(rv[u], m);
+#pragma unroll
+                        for (int e = 0; e < VN; ++e) {
+                            sa = fmaf(x[e], m[e], sa); sb = fmaf(x[e], x[e], sb); sc = fmaf(m[e], m[e], sc);
+                        }
+                    }
+                    sa = warp_sum(sa); sb = warp_sum(sb); sc = warp_sum(sc);
+                    gate = p.lambda / (1.f + __expf(-sa * rsqrtf(fmaf(sb, sc, 1e-12f))));
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u) {
+                        const int k = u * 32 + lane;
+                        if (k >= steps) continue;
+                        float x[VN], m[VN], y[VN];
+                        unpack_hidden<HT>(hv[u], x);
+                        unpack_row<HT>(rv[u], m);
+#pragma unroll
+                        for (int e = 0; e < VN; ++e) y[e] = fmaf(gate, m[e], x[e]);
+                        store_hidden<HT>(orow, k, y);
+                    }
+                    continue;
+                }
+            }
             if constexpr (COS) {
                 float sa = 0.f, sb = 0.f, sc = 0.f;      // <h,m>, <h,h>, <m,m>
+#pragma unroll 4
                 for (int k = lane; k < steps; k += 32) {
                     float x[VN], m[VN];
                     load_hidden<HT>(hrow, k, x);
@@ -567,6 +612,7 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
                     }
                 }
             } else {
+#pragma unroll 4
                 for (int k = lane; k < steps; k += 32) {
                     float x[VN], m[VN], y[VN];
                     load_hidden<HT>(hrow, k, x);

@@ -109,3 +109,24 @@ def test_index_bytes_per_entry_below_the_papers_overhead():
     assert 100 < paper_overhead < 120
     ours = 16 / 0.7 + 4 + 4 + 16        # index slot / load factor + position + owner + stored tuple
     assert ours < paper_overhead
+
+
+def test_header_is_plain_c(tmp_path):
+    """The boundary is a C ABI: the header must compile as C11 with nothing but the standard headers,
+    and a C program must link against the library by name."""
+    import subprocess
+    src = tmp_path / "use_tfe.c"
+    src.write_text('#include "tfe.h"\n'
+                   'int main(void) {\n'
+                   '    tfe_config cfg; tfe_inject_params prm; tfe_prefetch_params pf;\n'
+                   '    (void)cfg; (void)prm; (void)pf;\n'
+                   '    return tfe_status_string(TFE_OK) == 0;\n'
+                   '}\n')
+    inc = os.path.join(ROOT, "include")
+    subprocess.run(["gcc", "-std=c11", "-Wall", "-Werror", "-pedantic", "-fsyntax-only", f"-I{inc}", str(src)], check=True)
+    from paper_2607_07388_b200 import build
+    lib = build.build()
+    exe = tmp_path / "use_tfe"
+    subprocess.run(["gcc", "-std=c11", f"-I{inc}", str(src), lib, "-o", str(exe),
+                    f"-Wl,-rpath,{os.path.dirname(lib)}"], check=True)
+    assert subprocess.run([str(exe)]).returncode == 0
