@@ -120,7 +120,9 @@ def valid_pairs(tokens: np.ndarray, q_start: int, orders, vocab: int) -> int:
 
 
 def algorithmic_bytes(w, n_pairs, hits, misses, in_place=False):
-    """Bytes the method itself must move per call ('Algorithmic bytes')."""
+    """Bytes the method itself must move per call: token ids, two 64-byte buckets per valid (query, order)
+    pair, hidden states in and out (every position, or only the hits when updating in place), the rows of
+    the hits, nine bytes per miss-list entry."""
     hid = 2
     b = w.B * w.T * 4 + n_pairs * 128 + hits * w.d * 2 + misses * 9
     if in_place:

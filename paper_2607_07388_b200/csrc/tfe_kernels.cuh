@@ -418,12 +418,15 @@ __device__ __forceinline__ int32_t tfe_select_longest(const TfeLookupParams &p, 
 // several dependent DRAM round trips, and a barrier makes 8 warps wait for it (measured: 12.8 us
 // of probing before any byte streamed).  Autonomous warps wait only for their own 32 lanes while
 // the other warps of the SM keep the memory pipes busy.
+#ifndef TFE_MIN_BLOCKS_GENERAL
+#define TFE_MIN_BLOCKS_GENERAL 2     // blocks per SM the ALL / COSINE variants are compiled for
+#endif
 #ifndef TFE_MIN_BLOCKS
 #define TFE_MIN_BLOCKS 3
 #endif
 
 template <int HT, bool ALL, bool COS, bool PACKED>
-__global__ void __launch_bounds__(TFE_BLOCK_THREADS, (ALL || COS) ? 2 : TFE_MIN_BLOCKS)
+__global__ void __launch_bounds__(TFE_BLOCK_THREADS, (ALL || COS) ? TFE_MIN_BLOCKS_GENERAL : TFE_MIN_BLOCKS)
 tfe_lookup_inject_kernel(const TfeLookupParams p)
 {
     constexpr int VN = TfeVec<HT>::N;
