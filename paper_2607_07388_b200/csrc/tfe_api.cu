@@ -608,19 +608,6 @@ tfe_status tfe_cache_install(tfe_ctx *c, int32_t n, const uint32_t *phrase_ids, 
         const tfe_status ms = fetch_mirror(c, stream);
         if (ms != TFE_OK) return ms;
     }
-    for (int32_t k = 0; k < n; ++k) {
-        if ((int64_t)phrase_ids[k] >= N) return TFE_ERR_UNKNOWN_PHRASE;
-        if (c->h_slot[phrase_ids[k]] >= 0) return TFE_ERR_ALREADY_RESIDENT;
-        if (dst_slots[k] < 0 || dst_slots[k] >= C) return TFE_ERR_SLOT_RANGE;
-    }
-    {
-        std::vector<uint32_t> a(phrase_ids, phrase_ids + n);
-        std::vector<int32_t> b(dst_slots, dst_slots + n);
-        std::sort(a.begin(), a.end());
-        std::sort(b.begin(), b.end());
-        if (std::adjacent_find(a.begin(), a.end()) != a.end()) return TFE_ERR_INVALID_ARG;
-        if (std::adjacent_find(b.begin(), b.end()) != b.end()) return TFE_ERR_INVALID_ARG;
-    }
     cudaPointerAttributes attr{};
     bool src_on_device = false;
     if (cudaPointerGetAttributes(&attr, src_rows) == cudaSuccess)
@@ -638,14 +625,30 @@ tfe_status tfe_cache_install(tfe_ctx *c, int32_t n, const uint32_t *phrase_ids, 
         CU(cudaMalloc(&c->d_inst_rows, (size_t)n * c->row_vecs * sizeof(uint4)));
         c->inst_cap = n;
     }
-    CU(cudaMemcpyAsync(c->d_inst_ids, phrase_ids, (size_t)n * 4, cudaMemcpyHostToDevice, stream));
-    CU(cudaMemcpyAsync(c->d_inst_slots, dst_slots, (size_t)n * 4, cudaMemcpyHostToDevice, stream));
+    // The rows start travelling before the arguments are checked: the copy into the staging area
+    // changes nothing a caller can see, and the checks below (a few tens of microseconds for
+    // thousands of rows) run while it is under way.
     const uint4 *src = static_cast<const uint4 *>(src_rows);
     if (!src_on_device) {
         CU(cudaMemcpyAsync(c->d_inst_rows, src_rows, (size_t)n * c->row_vecs * sizeof(uint4),
                            cudaMemcpyHostToDevice, stream));
         src = c->d_inst_rows;
     }
+    for (int32_t k = 0; k < n; ++k) {
+        if ((int64_t)phrase_ids[k] >= N) return TFE_ERR_UNKNOWN_PHRASE;
+        if (c->h_slot[phrase_ids[k]] >= 0) return TFE_ERR_ALREADY_RESIDENT;
+        if (dst_slots[k] < 0 || dst_slots[k] >= C) return TFE_ERR_SLOT_RANGE;
+    }
+    {
+        std::vector<uint32_t> a(phrase_ids, phrase_ids + n);
+        std::vector<int32_t> b(dst_slots, dst_slots + n);
+        std::sort(a.begin(), a.end());
+        std::sort(b.begin(), b.end());
+        if (std::adjacent_find(a.begin(), a.end()) != a.end()) return TFE_ERR_INVALID_ARG;
+        if (std::adjacent_find(b.begin(), b.end()) != b.end()) return TFE_ERR_INVALID_ARG;
+    }
+    CU(cudaMemcpyAsync(c->d_inst_ids, phrase_ids, (size_t)n * 4, cudaMemcpyHostToDevice, stream));
+    CU(cudaMemcpyAsync(c->d_inst_slots, dst_slots, (size_t)n * 4, cudaMemcpyHostToDevice, stream));
     const unsigned blocks = (unsigned)((n + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK);
     tfe_install_kernel<<<blocks, TFE_BLOCK_THREADS, 0, stream>>>(c->d_index, c->d_phrase_pos, c->d_slot_owner,
                                                                  c->gpu_rows, c->row_vecs, n, c->d_inst_ids,
