@@ -130,3 +130,34 @@ def test_header_is_plain_c(tmp_path):
     subprocess.run(["gcc", "-std=c11", f"-I{inc}", str(src), lib, "-o", str(exe),
                     f"-Wl,-rpath,{os.path.dirname(lib)}"], check=True)
     assert subprocess.run([str(exe)]).returncode == 0
+
+
+def test_new_entry_points_refuse_bad_arguments_on_the_host(tfe):
+    """Argument errors come back before any device call (this box has no GPU)."""
+    L = tfe.lib()
+    out = C.c_void_p()
+    # early-exit head
+    for w, V, d, mb in ((None, 100, 64, 4), (0x1000, 0, 64, 4), (0x1000, 100, 32, 4), (0x1000, 100, 96, 4),
+                        (0x1000, 100, 64, 0), (0x1000, 100, 64, 257), (0x1004, 100, 64, 4)):
+        assert L.tfe_head_create(w, V, d, mb, C.byref(out)) == tfe.TFE_ERR_INVALID_ARG, (w, V, d, mb)
+        assert out.value is None
+    assert L.tfe_head_create(0x1000, 100, 64, 4, None) == tfe.TFE_ERR_INVALID_ARG
+    assert L.tfe_head_topk(None, 0x1000, 1, 1, 0x1000, 0x1000, None) == tfe.TFE_ERR_INVALID_ARG
+    flags = C.c_uint32(0)
+    assert L.tfe_head_status(None, C.byref(flags), None) == tfe.TFE_ERR_INVALID_ARG
+    assert L.tfe_head_geometry(None, None, None, None) == tfe.TFE_ERR_INVALID_ARG
+    L.tfe_head_destroy(None)                                    # a no-op
+    # retention ranking
+    cnt = C.c_int32(0)
+    assert L.tfe_cache_policy_enable(None, None) == tfe.TFE_ERR_INVALID_ARG
+    assert L.tfe_cache_select_victims(None, 4, 0, 0x1000, None, C.byref(cnt), None) == tfe.TFE_ERR_INVALID_ARG
+    assert L.tfe_cache_stats(None, None, None, None) == tfe.TFE_ERR_INVALID_ARG
+    # device build: the same configuration checks as the host build
+    pt = np.zeros((2, 4), np.int32)
+    for kw in (dict(d=12), dict(orders=(3, 2)), dict(load_factor=0.0), dict(hidden_dtype=2)):
+        cfg = tfe.make_config(**dict(dict(d=16, vocab=10, orders=(2, 3), n_phrases=2, gpu_slots=2), **kw))
+        assert L.tfe_index_build_device(C.byref(cfg), pt.ctypes.data, 0x1000, 0x1000, 0x1000, None, C.byref(out)) \
+            == tfe.TFE_ERR_INVALID_ARG, kw
+    cfg = tfe.make_config(d=16, vocab=10, orders=(2, 3), n_phrases=2, gpu_slots=2)
+    assert L.tfe_index_build_device(C.byref(cfg), None, 0x1000, 0x1000, 0x1000, None, C.byref(out)) == tfe.TFE_ERR_INVALID_ARG
+    assert L.tfe_index_build_device(C.byref(cfg), 0x1004, 0x1000, 0x1000, 0x1000, None, C.byref(out)) == tfe.TFE_ERR_INVALID_ARG
