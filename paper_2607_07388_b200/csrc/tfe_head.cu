@@ -518,7 +518,8 @@ tfe_head_select_kernel(const HeadSelParams p)
             want = __shfl_sync(0xFFFFFFFFu, rest, who);
             __syncthreads();
         }
-        theta = from_orderable(prefix);
+        // (rounding the image of -inf down lands among the NaN patterns: no bound then)
+        theta = prefix <= orderable(-INFINITY) ? -INFINITY : from_orderable(prefix);
     }
 
     // ---- the sweep: sum of exponentials, survivors

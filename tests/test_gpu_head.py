@@ -43,7 +43,7 @@ def check_topk(z64, tokens, prob, K, logit_tol, lse=None):
         kth = np.partition(z64[b], V - K)[V - K]                 # K-th largest oracle logit
         assert z64[b, t].min() >= kth - logit_tol, (b, z64[b, t].min(), kth)
         rest = np.ones(V, bool); rest[t] = False
-        assert z64[b, rest].max() <= z64[b, t].min() + logit_tol
+        assert K == V or z64[b, rest].max() <= z64[b, t].min() + logit_tol
         p64 = np.exp(z64[b, t] - lse64[b])
         np.testing.assert_allclose(prob[b], p64, rtol=2e-3, atol=1e-9)
         assert (np.diff(prob[b]) <= 1e-7 * prob[b][:-1] + 1e-12).all()      # descending
@@ -155,3 +155,35 @@ def test_head_feeds_prefetch_candidates(orc):
     np.testing.assert_array_equal(sc[:n].cpu().numpy().view(np.uint32), esc.view(np.uint32))
     head.close()
     pr.close()
+
+
+@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("TFE_RANDOM_CASES", "24"))))
+def test_head_random_shapes(orc, seed):
+    """Seeded random vocabulary size / width / batch / K, including sizes that leave short last tiles,
+    batches that are not multiples of 16 and K up to the limit."""
+    from paper_2607_07388_b200.engine import EarlyExitHead
+    rng = np.random.default_rng([4404, seed])
+    d = int(rng.choice([64, 128, 192, 320, 512, 1024]))
+    B = int(rng.choice([1, 2, 15, 16, 17, 48, 64, 100, 128, 200, 256]))
+    V = int(rng.integers(8, max(9, min(80_000, 200_000_000 // (d * B)))))
+    K = int(rng.integers(1, min(128, V) + 1))
+    exact_inputs = bool(rng.random() < 0.4)
+    if exact_inputs:                        # small integers: fp32 sums are exact, ties are frequent
+        W = synth.f32_to_bf16_bits(rng.integers(-2, 3, size=(V, d)).astype(np.float32))
+        h = synth.f32_to_bf16_bits(rng.integers(-2, 3, size=(B, d)).astype(np.float32))
+    else:
+        W, h = _inputs(seed, V, d, B)
+    head = EarlyExitHead(_bits_to_gpu(W), max_batch=B)
+    tok, prob = head.topk(_bits_to_gpu(h), K)
+    assert head.status() == 0
+    z64 = orc.head_logits(W, h)
+    if exact_inputs:
+        np.testing.assert_array_equal(head.logits(B).cpu().numpy().astype(np.float64), z64)
+        e_tok, e_prob, _ = orc.head_topk(z64, K)
+        np.testing.assert_array_equal(tok.cpu().numpy(), e_tok)
+        np.testing.assert_allclose(prob.cpu().numpy(), e_prob, rtol=1e-4, atol=1e-30)
+    else:
+        tol = 4e-6 * d * max(np.abs(z64).max(), 1e-6)
+        np.testing.assert_allclose(head.logits(B).cpu().numpy(), z64, rtol=0, atol=tol)
+        check_topk(z64, tok.cpu().numpy(), prob.cpu().numpy(), K, logit_tol=2 * tol, lse=head.lse(B).cpu().numpy())
+    head.close()
