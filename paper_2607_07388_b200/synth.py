@@ -96,6 +96,8 @@ def build_table(seed: int, n_phrases: int, orders, s: float, vocab: int = VOCAB)
     perm_table = np.random.default_rng([seed, 2]).permutation(vocab)
     cdf = zipf_cdf(vocab, s)
     orders = sorted(int(o) for o in orders)
+    if n_phrases > sum(min(vocab ** n, 2 ** 62) for n in orders):
+        raise ValueError(f"{n_phrases} distinct phrases of orders {orders} do not exist over {vocab} token ids")
     L = max(64, int(n_phrases * 0.55) + 16)
     while True:
         S = zipf_tokens(np.random.default_rng([seed, 1]), L, cdf, perm_table)

@@ -110,3 +110,36 @@ def test_victims_more_than_slots_and_host_pipeline_epoch(H):
     slots = _compare_victims(pr, 4096, 0)
     assert len(slots) == 1500 and len(set(slots.tolist())) == 1500
     pr.close()
+
+
+@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("TFE_RANDOM_CASES", "10"))))
+def test_policy_random_histories(H, seed):
+    """Seeded random interleavings of lookups (either policy), victim selections (any n, any half-life)
+    and installs into the selected victims: bookkeeping and ranking follow the oracle at every step."""
+    rng = np.random.default_rng([808, seed])
+    n_phrases = int(rng.integers(200, 20_000))
+    gpu_slots = max(8, int(n_phrases * rng.uniform(0.1, 0.9)))
+    w = synth.config(1, B=int(rng.integers(1, 6)), T=int(rng.integers(40, 300)), n_phrases=n_phrases, gpu_slots=gpu_slots,
+                     residency="hot_host_ssd", reserve_free=int(gpu_slots * rng.uniform(0.0, 0.3)), p=0.5,
+                     orders=(2, 3) if rng.random() < 0.5 else (2, 3, 4), d=16)
+    tb, pr = H.pair_from_workload(w, device_build=bool(rng.random() < 0.5))
+    pr.eng.cache_policy_enable()
+    h = synth.make_hidden_np(w)
+    for step in range(int(rng.integers(3, 9))):
+        tok = synth.make_queries(w, tb, variant=int(rng.integers(0, 3)))
+        policy = int(rng.random() < 0.4)
+        _, ref, _ = pr.run_and_compare(tok, h, policy=policy, lam=1.0)
+        pr.ora.touch(ref)
+        _compare_state(pr)
+        n = int(rng.choice([1, 5, 64, 1000, 4096]))
+        hl = int(rng.choice([0, 1, 2, 5]))
+        slots = _compare_victims(pr, n, hl)
+        if rng.random() < 0.7:
+            want = np.unique(pr.ora.lookup(tok, policy=policy).miss_phrase).astype(np.uint32)
+            k = int(min(len(want), len(slots), rng.integers(1, 200)))
+            if k:
+                src = synth.phrase_rows_np(w, want[:k])
+                assert pr.ora.cache_install(want[:k], src, slots[:k].copy()) == 0
+                pr.eng.cache_install(want[:k], src, slots[:k].copy())
+                _compare_state(pr)
+    pr.close()

@@ -99,3 +99,36 @@ def test_prefetch_budget_cut_with_many_candidates(H):
     assert total > 4096 and n == 4096
     n, total = _compare(pr, hist, cand, prob, None, 1000, 1.0, 3.0)
     pr.close()
+
+
+@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("TFE_RANDOM_CASES", "16"))))
+def test_prefetch_random_configurations(H, seed):
+    """Seeded random orders, vocabulary, batch, top-K, history length, budget, benefits and usefulness."""
+    rng = np.random.default_rng([515, seed])
+    orders = tuple(o for o in (1, 2, 3, 4) if rng.random() < 0.6) or (2,)
+    vocab = int(rng.choice([300, 4096, synth.VOCAB]))
+    n_phrases = int(rng.integers(500, 60_000))
+    n_phrases = min(n_phrases, sum(min(vocab ** n, 10 ** 6) for n in orders) // 4)      # what the tuple space allows
+    w = synth.config(2, n_phrases=max(n_phrases, 16), gpu_slots=max(4, int(n_phrases * rng.uniform(0.05, 0.8))),
+                     residency=str(rng.choice(["hot_host", "hot_host_ssd"])), orders=orders, d=16, rows="gaussian",
+                     vocab=vocab)
+    tb, pr = H.pair_from_workload(w, max_kicks=100_000)
+    B, K = int(rng.integers(1, 300)), int(rng.integers(1, 129))
+    if max(orders) == 1:                     # single tokens are the phrases: no history at all
+        hist = np.zeros((B, 0), np.int32)
+        cand = rng.choice(tb.stream[:tb.safe_len], size=(B, K)).astype(np.int32)
+        cand[:, ::3] = rng.integers(0, vocab, size=cand[:, ::3].shape)
+        prob = rng.random((B, K)).astype(np.float32)
+    else:
+        hist, cand, prob = _inputs(w, tb, B, K, seed, planted=float(rng.uniform(0.2, 1.0)))
+    if rng.random() < 0.3 and hist.shape[1] > 1:
+        hist = np.ascontiguousarray(hist[:, 1:])                # a history shorter than the longest order needs
+    if rng.random() < 0.3:
+        prob[:] = np.float32(0.25)                               # ties everywhere
+    use = None if rng.random() < 0.4 else rng.choice([0.0, 0.5, 1.0, 2.0], size=w.n_phrases).astype(np.float32)
+    budget = int(rng.choice([0, 1, 13, 256, 4096]))
+    c_host, c_ssd = float(rng.choice([0.0, 1.0, 1.5])), float(rng.choice([0.0, 2.0, 3.0]))
+    if hist.shape[1] == 0:
+        hist = np.zeros((B, 0), np.int32)
+    _compare(pr, hist, cand, prob, use, budget, c_host, c_ssd)
+    pr.close()
