@@ -362,3 +362,44 @@ def test_host_buffer_entry_point_in_pieces(H):
         np.testing.assert_array_equal(mt, ref.miss_tier)
     pr.run_and_compare(tok, h, lam=1.0)
     pr.close()
+
+
+@pytest.mark.parametrize("seed", range(min(30, int(__import__("os").environ.get("TFE_RANDOM_CASES", "4")))))
+def test_host_buffer_pieces_random_shapes(H, seed):
+    """Host-buffer calls large enough to go in pieces, with seeded random shapes: piece boundaries
+    fall anywhere in the sequences, pieces may hold no hit or no miss at all."""
+    from paper_2607_07388_b200 import binding as tfe
+    rng = np.random.default_rng([909, seed])
+    d = int(rng.choice([512, 1024, 2048, 4104]))
+    Q_target = int(rng.integers(16 << 20, 72 << 20)) // (2 * d) + 1
+    shape = "prefill" if rng.random() < 0.6 else "decode"
+    orders = (2, 3) if rng.random() < 0.5 else (2, 3, 4)
+    if shape == "prefill":
+        B = int(rng.integers(1, 9)); T = Q_target // B + 1
+    else:
+        B = Q_target; T = max(orders)
+    w = synth.config(1, shape=shape, B=B, T=T, d=d, orders=orders, n_phrases=40_000, gpu_slots=15_000,
+                     residency=str(rng.choice(["hot_host", "hot_host_ssd"])), p=float(rng.uniform(0.05, 0.5)))
+    assert w.Q * w.d * 2 >= 16 << 20
+    tb, pr = H.pair_from_workload(w)
+    tok = synth.make_queries(w, tb)
+    h = synth.make_hidden_np(w)
+    out = np.empty_like(h)
+    sp = np.empty(w.Q, np.uint32); ss = np.empty(w.Q, np.int32); fl = np.empty(w.Q, np.uint8)
+    lam = float(rng.choice([1.0, 0.5, 0.3]))
+    tfe.tfe_lookup_inject_host(pr.eng.ctx, tok, w.B, w.T, w.q_start, h, out, lam=lam, sel_phrase=sp, sel_slot=ss, flags=fl)
+    mq, mp, mt, cnt = pr.eng.miss_list()
+    ref = pr.ora.lookup(tok, w.q_start)
+    np.testing.assert_array_equal(sp, ref.sel_phrase)
+    np.testing.assert_array_equal(ss, ref.sel_slot)
+    np.testing.assert_array_equal(fl, ref.flags)
+    assert cnt == len(ref.miss_q)
+    np.testing.assert_array_equal(mq, ref.miss_q)
+    np.testing.assert_array_equal(mp, ref.miss_phrase)
+    np.testing.assert_array_equal(mt, ref.miss_tier)
+    exact, rounded = pr.ora.inject(ref, h, lam=lam)
+    if lam != 0.3:
+        np.testing.assert_array_equal(out, rounded)
+    else:
+        assert np.abs(synth.bf16_bits_to_f32(out).astype(np.float64) - exact).max() <= 2e-2
+    pr.close()
