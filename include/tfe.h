@@ -15,7 +15,10 @@
  * pointer is marked HOST or DEVICE.  "stream" is a cudaStream_t passed as
  * void* (NULL = the legacy default stream).  All device work of one context
  * must be issued in stream order (one stream, or streams the caller orders);
- * two calls on the same context that overlap on the GPU race.
+ * two calls on the same context that overlap on the GPU race.  A context (and
+ * a head) is also not safe for concurrent calls from several host threads:
+ * each entry point updates host-side state of its object without locking.
+ * Different contexts are independent.
  *
  * No entry point throws, aborts or traps.  Argument errors are found on the
  * host before anything is launched and leave the context unchanged.
@@ -43,7 +46,7 @@ typedef enum {
     TFE_ERR_MISS_OVERFLOW = 8,      /* caller's miss buffers are smaller than the miss count    */
     TFE_ERR_PROBE_LIMIT = 9,        /* index build could not place a key within max_kicks moves   */
     TFE_ERR_CUDA = 10,              /* a CUDA runtime call failed; see tfe_last_cuda_error()    */
-    TFE_ERR_INTERNAL = 11           /* reserved: the device reported an inconsistent state        */
+    TFE_ERR_INTERNAL = 11           /* the device reported an inconsistent state or a bounded wait ran out */
 } tfe_status;
 
 /* Table geometry, fixed at build time. */
