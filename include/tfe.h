@@ -247,7 +247,9 @@ tfe_status tfe_miss_list_device(tfe_ctx *ctx, const uint32_t **q_idx, const uint
  * tfe_cache_install sets {freq, last} = {1, epoch} for the slots it fills.  The epoch is a device
  * counter of completed lookups (a replayed launch advances it like a fresh one).  Calling it
  * again clears the counters and the epoch.  Allocates 12 bytes per GPU-tier slot; waits for the
- * device.  Errors: INVALID_ARG, CUDA.
+ * device.  Launches recorded earlier (a captured CUDA graph) keep the arguments they were
+ * recorded with and do no bookkeeping; record them again after enabling.
+ * Errors: INVALID_ARG, CUDA.
  */
 tfe_status tfe_cache_policy_enable(tfe_ctx *ctx, void *stream);
 
