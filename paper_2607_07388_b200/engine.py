@@ -137,7 +137,10 @@ class EarlyExitHead:
             self.handle = 0
 
     def __del__(self):
-        self.close()
+        try:
+            self.close()
+        except Exception:       # interpreter shutdown: the binding may be gone already
+            pass
 
     def topk(self, hidden: torch.Tensor, K: int, stream=None):
         """(tokens int32 [B, K], prob float32 [B, K]) on the device."""
