@@ -1,5 +1,7 @@
 """GPU-tier retention ranking (frequency / recency bookkeeping in the lookup kernels, victim
 selection) against the oracle's state machine, through the C ABI."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -112,7 +114,7 @@ def test_victims_more_than_slots_and_host_pipeline_epoch(H):
     pr.close()
 
 
-@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("TFE_RANDOM_CASES", "10"))))
+@pytest.mark.parametrize("seed", range(int(os.environ.get("TFE_RANDOM_CASES", "10"))))
 def test_policy_random_histories(H, seed):
     """Seeded random interleavings of lookups (either policy), victim selections (any n, any half-life)
     and installs into the selected victims: bookkeeping and ranking follow the oracle at every step."""

@@ -1,4 +1,6 @@
 """Early-exit prefetch head (tcgen05 GEMM + softmax + top-K) against the fp64 oracle, through the C ABI."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -157,7 +159,7 @@ def test_head_feeds_prefetch_candidates(orc):
     pr.close()
 
 
-@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("TFE_RANDOM_CASES", "24"))))
+@pytest.mark.parametrize("seed", range(int(os.environ.get("TFE_RANDOM_CASES", "24"))))
 def test_head_random_shapes(orc, seed):
     """Seeded random vocabulary size / width / batch / K, including sizes that leave short last tiles,
     batches that are not multiples of 16 and K up to the limit."""

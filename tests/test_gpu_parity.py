@@ -2,6 +2,8 @@
 the same seeded inputs.  Integer outputs (phrase ids, slots, flags, miss lists)
 must be bit-exact; hidden states within 2e-2 (bf16) / 1e-5 (fp32) of the exact
 value.  Every call goes through the C ABI."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -364,7 +366,7 @@ def test_host_buffer_entry_point_in_pieces(H):
     pr.close()
 
 
-@pytest.mark.parametrize("seed", range(min(30, int(__import__("os").environ.get("TFE_RANDOM_CASES", "4")))))
+@pytest.mark.parametrize("seed", range(min(30, int(os.environ.get("TFE_RANDOM_CASES", "4")))))
 def test_host_buffer_pieces_random_shapes(H, seed):
     """Host-buffer calls large enough to go in pieces, with seeded random shapes: piece boundaries
     fall anywhere in the sequences, pieces may hold no hit or no miss at all."""

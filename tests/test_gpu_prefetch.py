@@ -1,6 +1,8 @@
 """GPU parity of tfe_prefetch_candidates (candidate expansion + priority, paper Sec. 4.4) against
 the CPU oracle: phrase ids, tiers, sources and counts bit-exact; priorities bit-exact too, because
 both sides form the product p*r*c in single precision in the same order and the ranking hangs on it."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -101,7 +103,7 @@ def test_prefetch_budget_cut_with_many_candidates(H):
     pr.close()
 
 
-@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("TFE_RANDOM_CASES", "16"))))
+@pytest.mark.parametrize("seed", range(int(os.environ.get("TFE_RANDOM_CASES", "16"))))
 def test_prefetch_random_configurations(H, seed):
     """Seeded random orders, vocabulary, batch, top-K, history length, budget, benefits and usefulness."""
     rng = np.random.default_rng([515, seed])
