@@ -29,7 +29,7 @@ def _compare_victims(pr, n, half_life):
     e_slots, e_keys = pr.ora.cache_victims(n, half_life)
     np.testing.assert_array_equal(slots, e_slots)
     np.testing.assert_array_equal(keys, e_keys)
-    return slots
+    return e_slots          # the oracle's own (equal) values: nothing the GPU computed feeds the oracle
 
 
 @pytest.mark.parametrize("policy", [0, 1])

@@ -54,14 +54,17 @@ def test_prefetch_loop_turns_predicted_misses_into_hits():
         assert (e_tok[:, 0] == nxt).mean() > 0.9
         # 3. candidate phrases of the predicted tokens, by priority
         hist = torch.from_numpy(np.ascontiguousarray(tok[:, 1:])).to(DEV)               # the last two tokens
-        ph, tr, sc, sr, cnt = pr.eng.prefetch_candidates(hist, t_tok, t_prob, benefit_host=1.0, benefit_ssd=2.0, budget=64)
+        ph, tr, sc, sr, cnt = pr.eng.prefetch_candidates(hist, t_tok, t_prob, benefit_host=1.0, benefit_ssd=2.0, budget=4096)
         torch.cuda.synchronize()
-        eph, etr, esc, esr, total = pr.ora.prefetch_candidates(tok[:, 1:], t_tok.cpu().numpy(), t_prob.cpu().numpy(),
-                                                               benefit_host=1.0, benefit_ssd=2.0, budget=64)
+        # the oracle's chain runs on the oracle head's own outputs (nothing the GPU computed goes into it)
+        eph, etr, esc, esr, total = pr.ora.prefetch_candidates(tok[:, 1:], e_tok, e_prob.astype(np.float32),
+                                                               benefit_host=1.0, benefit_ssd=2.0, budget=4096)
         n = int(cnt[0].item())
-        assert n == len(eph) and int(cnt[1].item()) == total
-        np.testing.assert_array_equal(ph[:n].cpu().numpy().view(np.uint32), eph)
-        np.testing.assert_array_equal(sc[:n].cpu().numpy().view(np.uint32), esc.view(np.uint32))
+        assert n == len(eph) and int(cnt[1].item()) == total and total <= 4096
+        got = sorted(zip(sr[:n].cpu().numpy().view(np.uint32).tolist(), ph[:n].cpu().numpy().view(np.uint32).tolist(),
+                         tr[:n].cpu().numpy().tolist()))
+        assert got == sorted(zip(esr.tolist(), eph.tolist(), etr.tolist()))
+        np.testing.assert_allclose(np.sort(sc[:n].cpu().numpy()), np.sort(esc), rtol=1e-4)
         # 4. fetch: the distinct candidate phrases, best first; victims from the retention ranking
         ids = np.array(list(dict.fromkeys(eph.tolist())), np.uint32)
         if len(ids):

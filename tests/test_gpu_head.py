@@ -147,14 +147,24 @@ def test_head_feeds_prefetch_candidates(orc):
     np.testing.assert_array_equal(tok.cpu().numpy(), e_tok)
     np.testing.assert_allclose(prob.cpu().numpy(), e_prob, rtol=1e-4, atol=1e-30)
     hist = torch.from_numpy(np.stack([tb.stream[base + 2 * b:base + 2 * b + 2] for b in range(B)]).astype(np.int32)).to(DEV)
-    ph, tr, sc, sr, cnt = pr.eng.prefetch_candidates(hist, tok, prob, benefit_host=1.0, benefit_ssd=2.0, budget=256)
+    ph, tr, sc, sr, cnt = pr.eng.prefetch_candidates(hist, tok, prob, benefit_host=1.0, benefit_ssd=2.0, budget=4096)
     torch.cuda.synchronize()
-    eph, etr, esc, esr, total = pr.ora.prefetch_candidates(hist.cpu().numpy(), tok.cpu().numpy(), prob.cpu().numpy(),
-                                                           benefit_host=1.0, benefit_ssd=2.0, budget=256)
+    # the oracle's chain runs on the oracle head's own outputs (nothing the GPU computed goes into it)
+    eph, etr, esc, esr, total = pr.ora.prefetch_candidates(hist.cpu().numpy(), e_tok, e_prob.astype(np.float32),
+                                                           benefit_host=1.0, benefit_ssd=2.0, budget=4096)
     n = int(cnt[0].item())
-    assert int(cnt[1].item()) == total and n == len(eph) and total >= 5
-    np.testing.assert_array_equal(ph[:n].cpu().numpy().view(np.uint32), eph)
-    np.testing.assert_array_equal(sc[:n].cpu().numpy().view(np.uint32), esc.view(np.uint32))
+    assert int(cnt[1].item()) == total and n == len(eph) and 5 <= total <= 4096
+    # the same candidates (phrase, tier, source); priorities agree to fp32 rounding of the probabilities,
+    # so the two orders may differ only among candidates whose priorities are that close
+    got = sorted(zip(sr[:n].cpu().numpy().view(np.uint32).tolist(), ph[:n].cpu().numpy().view(np.uint32).tolist(),
+                     tr[:n].cpu().numpy().tolist()))
+    want = sorted(zip(esr.tolist(), eph.tolist(), etr.tolist()))
+    assert got == want
+    g_sc = sc[:n].cpu().numpy()
+    assert (np.diff(g_sc) <= 0).all()
+    by_key = {(s_, p_): v for s_, p_, v in zip(esr.tolist(), eph.tolist(), esc.tolist())}
+    for s_, p_, v in zip(sr[:n].cpu().numpy().view(np.uint32).tolist(), ph[:n].cpu().numpy().view(np.uint32).tolist(), g_sc.tolist()):
+        assert abs(v - by_key[(s_, p_)]) <= 1e-4 * abs(by_key[(s_, p_)]) + 1e-30
     head.close()
     pr.close()
 
