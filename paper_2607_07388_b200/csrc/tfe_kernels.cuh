@@ -419,14 +419,14 @@ __device__ __forceinline__ int32_t tfe_select_longest(const TfeLookupParams &p, 
 // of probing before any byte streamed).  Autonomous warps wait only for their own 32 lanes while
 // the other warps of the SM keep the memory pipes busy.
 #ifndef TFE_MIN_BLOCKS_GENERAL
-#define TFE_MIN_BLOCKS_GENERAL 2     // blocks per SM the ALL / COSINE variants are compiled for
+#define TFE_MIN_BLOCKS_GENERAL 2     // blocks per SM the COSINE variants are compiled for (the others: TFE_MIN_BLOCKS)
 #endif
 #ifndef TFE_MIN_BLOCKS
 #define TFE_MIN_BLOCKS 3
 #endif
 
 template <int HT, bool ALL, bool COS, bool PACKED>
-__global__ void __launch_bounds__(TFE_BLOCK_THREADS, (ALL || COS) ? TFE_MIN_BLOCKS_GENERAL : TFE_MIN_BLOCKS)
+__global__ void __launch_bounds__(TFE_BLOCK_THREADS, COS ? TFE_MIN_BLOCKS_GENERAL : TFE_MIN_BLOCKS)
 tfe_lookup_inject_kernel(const TfeLookupParams p)
 {
     constexpr int VN = TfeVec<HT>::N;
@@ -566,7 +566,7 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
             }
             if constexpr (COS) {
                 float sa = 0.f, sb = 0.f, sc = 0.f;      // <h,m>, <h,h>, <m,m>
-#pragma unroll 4
+#pragma unroll (COS ? 2 : 1)
                 for (int k = lane; k < steps; k += 32) {
                     float x[VN], m[VN];
                     load_hidden<HT>(hrow, k, x);
@@ -615,7 +615,7 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
                     }
                 }
             } else {
-#pragma unroll 4
+#pragma unroll (COS ? 2 : 1)
                 for (int k = lane; k < steps; k += 32) {
                     float x[VN], m[VN], y[VN];
                     load_hidden<HT>(hrow, k, x);
