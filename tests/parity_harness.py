@@ -6,7 +6,6 @@ import numpy as np
 import torch
 
 from oracle import tfe_oracle as orc
-from paper_2607_07388_b200 import binding as tfe
 from paper_2607_07388_b200 import synth
 from paper_2607_07388_b200.engine import Engram, bf16_tensor_from_bits, bits_from_bf16_tensor
 
