@@ -99,3 +99,18 @@ def test_config4_install_then_lookup(H):
     got = H.bits_from_bf16_tensor(bp.rows_gpu[torch.from_numpy(pick).to(H.DEV)])
     np.testing.assert_array_equal(got, want)
     bp.close()
+
+
+def test_millions_of_positions_narrow_rows(H):
+    """The largest calls: millions of query positions in one launch (32-bit position arithmetic, the
+    division by the sequence length, a miss list of hundreds of thousands of entries), rows of 8
+    elements so that the inputs stay small.  Prefill: 3 long sequences; decode: 2^21 sequences."""
+    for shape, B, T in (("prefill", 3, 1_400_003), ("decode", 1 << 21, 3)):
+        w = synth.Workload("wide", 31, shape, B, T, (2, 3), 60_000, 20_000, d=8, p=0.3, residency="hot_host_ssd",
+                           rows="gaussian")
+        tb, pr = H.pair_from_workload(w)
+        tok = synth.make_queries(w, tb)
+        h = synth.make_hidden_np(w)
+        _, ref, info = pr.run_and_compare(tok, h, q_start=w.q_start, lam=1.0)
+        assert info["n_hit"] > 50_000 and info["n_miss"] > 50_000
+        pr.close()
