@@ -411,6 +411,49 @@ int32_t orc_cache_install(int64_t N, int64_t C, int32_t d,
     return 0;
 }
 
+/* The same insertion for a caller that cannot check its batch beforehand -- a prefetch loop that
+ * stays on the device hands over whatever the candidate step produced [Sec. 4.4: candidates are
+ * fetched and inserted while the model computes].  Entries that cannot be applied are skipped
+ * instead of refusing the batch.  Whether entry k is applied is judged against the state BEFORE
+ * the call:
+ *   candidate[k]: ids[k] is a phrase, it was not GPU-resident, dst[k] is a slot, and no earlier
+ *                 entry of the batch names the same phrase;
+ *   applied[k]:   candidate[k], and no earlier candidate of the batch names the same slot.
+ * The applied entries then take effect in order, exactly as above.  Returns their number;
+ * applied (uint8 [n]) receives the flags. */
+int32_t orc_cache_install_lenient(int64_t N, int64_t C, int32_t d,
+                                  int32_t *slot_state, int64_t *slot_owner, uint16_t *rows,
+                                  int32_t n, const uint32_t *ids, const uint16_t *src, const int32_t *dst,
+                                  uint8_t *applied)
+{
+    uint8_t *cand = (uint8_t *)malloc((size_t)(n > 0 ? n : 1));
+    for (int32_t k = 0; k < n; ++k) {
+        int ok = (int64_t)ids[k] < N && slot_state[ids[k]] < 0 && dst[k] >= 0 && (int64_t)dst[k] < C;
+        for (int32_t l = 0; ok && l < k; ++l)
+            if (ids[l] == ids[k]) ok = 0;
+        cand[k] = (uint8_t)ok;
+    }
+    int32_t count = 0;
+    for (int32_t k = 0; k < n; ++k) {
+        int ok = cand[k];
+        for (int32_t l = 0; ok && l < k; ++l)
+            if (cand[l] && dst[l] == dst[k]) ok = 0;
+        applied[k] = (uint8_t)ok;
+        count += ok;
+    }
+    for (int32_t k = 0; k < n; ++k) {
+        if (!applied[k]) continue;
+        int64_t prev = slot_owner[dst[k]];
+        if (prev >= 0) slot_state[prev] = -1;
+        if (rows && src)
+            memcpy(rows + (int64_t)dst[k] * d, src + (int64_t)k * d, sizeof(uint16_t) * (size_t)d);
+        slot_state[ids[k]] = dst[k];
+        slot_owner[dst[k]] = (int64_t)ids[k];
+    }
+    free(cand);
+    return count;
+}
+
 /* ------------------------------------------------ GPU-tier retention ranking */
 
 /* The paper ranks cached entries by signals -- access frequency and recency first among them --

@@ -59,6 +59,7 @@ def lib() -> C.CDLL:
         _lib.orc_sort_phrases.restype = C.c_int64
         _lib.orc_select.restype = C.c_int64
         _lib.orc_cache_install.restype = C.c_int32
+        _lib.orc_cache_install_lenient.restype = C.c_int32
         _lib.orc_prefetch_candidates.restype = C.c_int64
         _lib.orc_cache_victims.restype = C.c_int64
         _lib.orc_retention_key.restype = C.c_uint32
@@ -194,6 +195,22 @@ class Oracle:
             lib().orc_cache_installed(C.c_int32(len(ids)), _p(dst), C.c_uint32(self.epoch), _p(self.freq),
                                       _p(self.last))
         return rc
+
+    def cache_install_lenient(self, ids, src_rows, dst_slots):
+        """Skips what cannot be applied; returns (applied uint8 [n], count)."""
+        ids = _c(ids, np.uint32)
+        dst = _c(dst_slots, np.int32)
+        src = None if src_rows is None else _c(src_rows, np.uint16)
+        applied = np.zeros(max(len(ids), 1), np.uint8)
+        cnt = int(lib().orc_cache_install_lenient(
+            C.c_int64(self.N), C.c_int64(self.C), C.c_int32(self.d), _p(self.slot_state), _p(self.slot_owner),
+            _p(self.rows), C.c_int32(len(ids)), _p(ids), _p(src), _p(dst), _p(applied)))
+        applied = applied[:len(ids)]
+        if cnt:
+            done = _c(dst[applied == 1], np.int32)
+            lib().orc_cache_installed(C.c_int32(len(done)), _p(done), C.c_uint32(self.epoch), _p(self.freq),
+                                      _p(self.last))
+        return applied, cnt
 
     # -- GPU-tier retention ranking ---------------------------------------------
     def touch(self, res: LookupResult) -> None:

@@ -713,3 +713,91 @@ def test_head_invariants(oracle_mod):
     for b in range(3):
         pos = {int(v): i for i, v in enumerate(t3[b])}
         assert pos[400] == pos[10] + 1
+
+
+# ---------------------------------------------------------------- lenient installation
+
+def test_lenient_install_hand_worked(oracle_mod):
+    # 8 phrases (i // 50, i % 50), 5 slots; phrases 0, 1, 2 start in slots 0, 1, 2; slots 3, 4 are free
+    owners = np.array([0, 1, 2, -1, -1, -1, -2, -1], np.int32)
+    pt = np.full((8, 4), -1, np.int32); pt[:, 0] = 0; pt[:, 1] = np.arange(8)
+    o = oracle_mod.Oracle(pt, np.full(8, 2, np.uint8), owners, np.zeros((5, 16), np.uint16), d=16, vocab=64,
+                          orders=(2,), gpu_slots=5)
+    ids = np.array([3, 9, 1, 4, 3, 5, 6, 7, 7], np.uint32)
+    dst = np.array([3, 4, 4, 3, 4, 7, 1, -1, 0], np.int32)
+    src = (np.arange(9)[:, None] + 1).astype(np.uint16) * np.ones((1, 16), np.uint16)
+    applied, cnt = o.cache_install_lenient(ids, src, dst)
+    # 0: phrase 3 -> free slot 3: applied.          1: id 9 is no phrase.            2: phrase 1 is resident.
+    # 3: phrase 4 -> slot 3, taken by entry 0.      4: phrase 3 again.               5: slot 7 does not exist.
+    # 6: phrase 6 (SSD) -> slot 1, evicts phrase 1. 7: slot -1 does not exist.       8: phrase 7 again (entry 7 came first).
+    np.testing.assert_array_equal(applied, [1, 0, 0, 0, 0, 0, 1, 0, 0])
+    assert cnt == 2
+    np.testing.assert_array_equal(o.slot_state, [0, -1, 2, 3, -1, -1, 1, -1])
+    np.testing.assert_array_equal(o.slot_owner, [0, 6, 2, 3, -1])
+    assert (o.rows[3] == 1).all() and (o.rows[1] == 7).all() and (o.rows[0] == 0).all()
+
+
+def test_lenient_install_equals_strict_install_on_clean_batches(oracle_mod):
+    rng = np.random.default_rng(12)
+    for trial in range(20):
+        N, C = 300, 120
+        owners = np.full(N, -1, np.int32)
+        res = rng.choice(N, 80, replace=False)
+        owners[res] = rng.permutation(C)[:80]
+        pt = np.full((N, 4), -1, np.int32); pt[:, 0] = np.arange(N) // 20; pt[:, 1] = np.arange(N) % 20
+        mk = lambda: oracle_mod.Oracle(pt, np.full(N, 2, np.uint8), owners, np.zeros((C, 8), np.uint16), d=8, vocab=32,
+                                       orders=(2,), gpu_slots=C)
+        a, b = mk(), mk()
+        n = int(rng.integers(1, 60))
+        ids = rng.choice(np.nonzero(owners < 0)[0], n, replace=False).astype(np.uint32)
+        dst = rng.choice(C, n, replace=False).astype(np.int32)
+        src = rng.integers(1, 60000, size=(n, 8)).astype(np.uint16)
+        assert a.cache_install(ids, src, dst) == 0
+        applied, cnt = b.cache_install_lenient(ids, src, dst)
+        assert cnt == n and applied.all()
+        np.testing.assert_array_equal(a.slot_state, b.slot_state)
+        np.testing.assert_array_equal(a.slot_owner, b.slot_owner)
+        np.testing.assert_array_equal(a.rows, b.rows)
+
+
+def test_lenient_install_against_independent_restatement(oracle_mod):
+    rng = np.random.default_rng(13)
+    for trial in range(30):
+        N, C = 200, 64
+        owners = np.full(N, -1, np.int32)
+        res = rng.choice(N, 40, replace=False)
+        owners[res] = rng.permutation(C)[:40]
+        owners[rng.choice(np.nonzero(owners < 0)[0], 30, replace=False)] = -2
+        pt = np.full((N, 4), -1, np.int32); pt[:, 0] = np.arange(N) // 20; pt[:, 1] = np.arange(N) % 20
+        o = oracle_mod.Oracle(pt, np.full(N, 2, np.uint8), owners, np.zeros((C, 4), np.uint16), d=4, vocab=32,
+                              orders=(2,), gpu_slots=C)
+        n = int(rng.integers(1, 150))
+        ids = rng.integers(0, N + 20, size=n).astype(np.uint32)
+        dst = rng.integers(-3, C + 5, size=n).astype(np.int32)
+        src = (np.arange(n)[:, None] + 1).astype(np.uint16) * np.ones((1, 4), np.uint16)
+        # restatement with dictionaries and sets
+        state = {i: int(owners[i]) for i in range(N)}
+        owner = {int(owners[i]): i for i in range(N) if owners[i] >= 0}
+        rows = {}
+        seen_ids, seen_slots, expect = set(), set(), []
+        for k in range(n):
+            i, s_ = int(ids[k]), int(dst[k])
+            cand = i < N and owners[i] < 0 and 0 <= s_ < C and i not in seen_ids
+            seen_ids.add(i)
+            ok = cand and s_ not in seen_slots
+            if cand:
+                seen_slots.add(s_)
+            expect.append(int(ok))
+        for k in range(n):
+            if expect[k]:
+                i, s_ = int(ids[k]), int(dst[k])
+                if s_ in owner:
+                    state[owner[s_]] = -1
+                state[i] = s_; owner[s_] = i; rows[s_] = k + 1
+        applied, cnt = o.cache_install_lenient(ids, src, dst)
+        np.testing.assert_array_equal(applied, expect)
+        assert cnt == sum(expect)
+        np.testing.assert_array_equal(o.slot_state, [state[i] for i in range(N)])
+        np.testing.assert_array_equal(o.slot_owner, [owner.get(s_, -1) for s_ in range(C)])
+        for s_, v in rows.items():
+            assert (o.rows[s_] == v).all()
