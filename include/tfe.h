@@ -135,6 +135,30 @@ tfe_status tfe_cache_install(tfe_ctx *ctx, int32_t n, const uint32_t *phrase_ids
                              const void *src_rows, const int32_t *dst_slots, void *stream);
 
 /*
+ * tfe_cache_install_device -- the same insertion with the whole batch on the DEVICE and no check
+ * by the host: what a prefetch loop that stays on the GPU produces (candidate phrases from
+ * tfe_prefetch_candidates, destination slots from tfe_cache_select_victims_device, rows staged in
+ * device memory).  Entries that cannot be applied are skipped instead of refusing the batch.
+ * Judged against the state before the call, entry k is a candidate if phrase_ids[k] is a phrase,
+ * that phrase is not GPU-resident, dst_slots[k] is a slot and no earlier entry names the same
+ * phrase; it is applied if in addition no earlier candidate names the same slot.  Applied
+ * entries take effect as in tfe_cache_install.
+ *
+ *   n              0..4096
+ *   phrase_ids     DEVICE uint32 [n];  src_rows DEVICE [n][d] bf16, 16-byte aligned;
+ *   dst_slots      DEVICE int32 [n]
+ *   applied        DEVICE uint8 [n], receives 1 / 0 per entry, or NULL
+ *   applied_count  DEVICE uint32, receives the number applied, or NULL
+ * Asynchronous on `stream`, three kernel launches, never synchronises; the first call allocates
+ * 4 bytes per phrase and per slot.  The host-side residency copy that tfe_cache_install checks
+ * against is refreshed (one synchronisation) on that function's next call.
+ * Errors: INVALID_ARG, CUDA.
+ */
+tfe_status tfe_cache_install_device(tfe_ctx *ctx, int32_t n, const uint32_t *phrase_ids,
+                                    const void *src_rows, const int32_t *dst_slots, uint8_t *applied,
+                                    uint32_t *applied_count, void *stream);
+
+/*
  * tfe_lookup_inject -- the hot path, one kernel launch (paper Sec. 2.2: key
  * from token n-grams, lookup m_t = M(q_t), aggregation m_t = sum alpha_i v_i,
  * injection h'_t = h_t + g_t * m_t; Sec. 4.2: longest-match selection;
@@ -262,11 +286,13 @@ tfe_status tfe_cache_policy_enable(tfe_ctx *ctx, void *stream);
  * use, then by slot.  half_life -> large gives least-frequently-used order, equal frequencies
  * give least-recently-used order.
  *
- *   n        0..4096;  slots HOST int32 [n];  keys HOST uint32 [n] or NULL;
+ *   n        0..4096;  slots HOST int32 [n], or NULL;  keys HOST uint32 [n] or NULL;
  *   count    HOST: entries written = min(n, gpu_slots).
- * Eight kernel launches on `stream`, then synchronises it (the slots feed tfe_cache_install,
- * which takes host arrays).  tfe_cache_select_victims_device returns the DEVICE copies of the
- * most recent selection (owned by the context, valid until the next one).
+ * Eight kernel launches on `stream`; with host `slots` the results are copied there and the
+ * stream is synchronised (they feed tfe_cache_install, which takes host arrays); with slots =
+ * NULL nothing is copied and nothing synchronises.  tfe_cache_select_victims_device returns the
+ * DEVICE copies of the most recent selection (owned by the context, valid until the next one;
+ * they feed tfe_cache_install_device).
  * Errors: INVALID_ARG (also: policy not enabled), CUDA.
  */
 tfe_status tfe_cache_select_victims(tfe_ctx *ctx, int32_t n, int32_t half_life, int32_t *slots,

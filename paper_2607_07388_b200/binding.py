@@ -28,7 +28,7 @@ GATE_CONST, GATE_COSINE = 0, 1
 HIDDEN_BF16, HIDDEN_F32 = 0, 1
 NO_PHRASE = 0xFFFFFFFF
 
-EXPORTS = ["tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
+EXPORTS = ["tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tfe_cache_install_device", "tfe_lookup_inject", "tfe_lookup_inject_host",
            "tfe_miss_list", "tfe_miss_list_device", "tfe_destroy", "tfe_status_string",
            "tfe_last_cuda_error", "tfe_index_geometry", "tfe_phrase_key64", "tfe_home_bucket",
            "tfe_launch_geometry", "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
@@ -76,6 +76,7 @@ def lib() -> C.CDLL:
         L.tfe_index_build.argtypes = [C.POINTER(TfeConfig), vp, vp, vp, vp, vp, C.POINTER(vp)]
         L.tfe_index_build_device.argtypes = L.tfe_index_build.argtypes
         L.tfe_cache_install.argtypes = [vp, i32, vp, vp, vp, vp]
+        L.tfe_cache_install_device.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
         L.tfe_lookup_inject.argtypes = [vp, vp, i32, i32, i32, vp, vp, C.POINTER(TfeInjectParams), vp, vp, vp, vp]
         L.tfe_lookup_inject_host.argtypes = L.tfe_lookup_inject.argtypes
         L.tfe_lookup_inject_noalloc.argtypes = [vp, vp, i32, i32, i32, vp, vp, C.POINTER(TfeInjectParams), vp, vp, vp,
@@ -107,7 +108,7 @@ def lib() -> C.CDLL:
         L.tfe_head_buffers.argtypes = [vp, C.POINTER(vp), C.POINTER(i64), C.POINTER(vp)]
         L.tfe_head_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         L.tfe_head_geometry.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
-        for name in ("tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tfe_lookup_inject", "tfe_lookup_inject_host",
+        for name in ("tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tfe_cache_install_device", "tfe_lookup_inject", "tfe_lookup_inject_host",
                      "tfe_miss_list", "tfe_miss_list_device", "tfe_index_geometry", "tfe_launch_geometry",
                      "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
                      "tfe_cache_policy_enable", "tfe_cache_select_victims", "tfe_cache_select_victims_device",
@@ -236,6 +237,15 @@ def tfe_prefetch_candidates(ctx: int, history, B, H, cand_tokens, cand_prob, K, 
 
 
 VICTIMS_MAX = 4096
+INSTALL_DEVICE_MAX = 4096
+
+
+def tfe_cache_install_device(ctx: int, n: int, phrase_ids, src_rows, dst_slots, applied=None, applied_count=None,
+                             stream=None) -> None:
+    """All arrays on the device; entries that cannot be applied are skipped."""
+    _check(lib().tfe_cache_install_device(ctx, int(n), _addr(phrase_ids), _addr(src_rows), _addr(dst_slots),
+                                          _addr(applied), _addr(applied_count), _stream(stream)),
+           "tfe_cache_install_device")
 
 
 def tfe_cache_policy_enable(ctx: int, stream=None) -> None:
@@ -249,6 +259,14 @@ def tfe_cache_select_victims(ctx: int, n: int, half_life: int = 0, stream=None):
     _check(lib().tfe_cache_select_victims(ctx, int(n), int(half_life), _addr(slots), _addr(keys), C.byref(cnt),
                                           _stream(stream)), "tfe_cache_select_victims")
     return slots[:cnt.value], keys[:cnt.value]
+
+
+def tfe_cache_select_victims_async(ctx: int, n: int, half_life: int = 0, stream=None) -> int:
+    """Selection left on the device (see tfe_cache_select_victims_device); returns min(n, gpu_slots)."""
+    cnt = C.c_int32(0)
+    _check(lib().tfe_cache_select_victims(ctx, int(n), int(half_life), None, None, C.byref(cnt), _stream(stream)),
+           "tfe_cache_select_victims")
+    return cnt.value
 
 
 def tfe_cache_select_victims_device(ctx: int):

@@ -93,6 +93,10 @@ struct tfe_ctx {
 
     bool mirror_ready = true;               // h_slot / h_owner filled (a device build fills them on first use)
 
+    // tfe_cache_install_device: stamps per phrase and per slot, the call counter, the applied count
+    uint32_t *d_phrase_stamp = nullptr, *d_slot_stamp = nullptr, *d_inst_count = nullptr;
+    uint32_t inst_call_no = 0;
+
     // host-buffer variant staging
     int32_t *d_h_tokens = nullptr;
     void *d_h_hidden = nullptr, *d_h_out = nullptr;
@@ -309,6 +313,7 @@ void tfe_destroy(tfe_ctx *c)
     free_dev(c->d_h_tokens); free_dev(c->d_h_hidden); free_dev(c->d_h_out);
     free_dev(c->d_h_phrase); free_dev(c->d_h_slot); free_dev(c->d_h_flag);
     free_dev(c->d_pf_keys); free_dev(c->d_pf_phrase); free_dev(c->d_pf_tier); free_dev(c->d_pf_counter);
+    free_dev(c->d_phrase_stamp); free_dev(c->d_slot_stamp); free_dev(c->d_inst_count);
     free_dev(c->d_slot_stats); free_dev(c->d_epoch); free_dev(c->d_slot_key); free_dev(c->d_vs_hist);
     free_dev(c->d_vs_keys); free_dev(c->d_vs_state); free_dev(c->d_vs_list); free_dev(c->d_vs_slots);
     if (c->hb_in) (void)cudaStreamDestroy(c->hb_in);
@@ -663,6 +668,52 @@ tfe_status tfe_cache_install(tfe_ctx *c, int32_t n, const uint32_t *phrase_ids, 
     return TFE_OK;
 }
 
+tfe_status tfe_cache_install_device(tfe_ctx *c, int32_t n, const uint32_t *phrase_ids, const void *src_rows,
+                                    const int32_t *dst_slots, uint8_t *applied, uint32_t *applied_count,
+                                    void *stream_)
+{
+    if (!c || n < 0 || n > TFE_INSTALL_DEVICE_MAX) return TFE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (n == 0) {
+        if (applied_count) CU(cudaMemsetAsync(applied_count, 0, sizeof(uint32_t), stream));
+        return TFE_OK;
+    }
+    if (!phrase_ids || !src_rows || !dst_slots) return TFE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(src_rows) & 15u) != 0) return TFE_ERR_INVALID_ARG;
+    const int64_t N = c->cfg.n_phrases, C = c->cfg.gpu_slots;
+    if (!c->d_phrase_stamp) {       // first use: the stamp arrays (4 bytes per phrase and per slot)
+        CU(cudaDeviceSynchronize());
+        CU(cudaMalloc(&c->d_phrase_stamp, std::max<size_t>(4, (size_t)N * 4)));
+        CU(cudaMalloc(&c->d_slot_stamp, std::max<size_t>(4, (size_t)C * 4)));
+        CU(cudaMalloc(&c->d_inst_count, sizeof(uint32_t)));
+        c->inst_call_no = 0;
+    }
+    if (c->inst_call_no == 0 || c->inst_call_no >= (1u << 20) - 1) {     // fresh stamps (also when the counter wraps)
+        CU(cudaMemsetAsync(c->d_phrase_stamp, 0, std::max<size_t>(4, (size_t)N * 4), stream));
+        CU(cudaMemsetAsync(c->d_slot_stamp, 0, std::max<size_t>(4, (size_t)C * 4), stream));
+        c->inst_call_no = 0;
+    }
+    ++c->inst_call_no;
+    TfeInstallDeviceParams p{};
+    p.index = c->d_index; p.phrase_pos = c->d_phrase_pos; p.slot_owner = c->d_slot_owner;
+    p.rows = c->gpu_rows; p.row_vecs = c->row_vecs; p.n = n;
+    p.n_phrases = (uint32_t)N; p.gpu_slots = C;
+    p.ids = phrase_ids; p.src = static_cast<const uint4 *>(src_rows); p.dst_slots = dst_slots;
+    p.phrase_stamp = c->d_phrase_stamp; p.slot_stamp = c->d_slot_stamp;
+    p.tag = c->inst_call_no << 12;
+    p.applied = applied; p.count = applied_count ? applied_count : c->d_inst_count;
+    p.slot_stats = c->d_slot_stats; p.epoch = c->d_epoch;
+    CU(cudaMemsetAsync(p.count, 0, sizeof(uint32_t), stream));
+    const unsigned blocks = (unsigned)((n + 255) / 256);
+    tfe_install_claim_kernel<0><<<blocks, 256, 0, stream>>>(p);
+    tfe_install_claim_kernel<1><<<blocks, 256, 0, stream>>>(p);
+    tfe_install_device_kernel<<<(unsigned)((n + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK), TFE_BLOCK_THREADS, 0,
+                                stream>>>(p);
+    CU(cudaGetLastError());
+    c->mirror_ready = false;        // the host copy of the residency state is stale now; fetched again when needed
+    return TFE_OK;
+}
+
 // Bytes of hidden state per piece of the host-buffer variant's copy / compute pipeline: the
 // largest piece, and the smallest (the last ones).
 #ifndef TFE_HOST_CHUNK_BYTES
@@ -959,7 +1010,7 @@ tfe_status tfe_cache_policy_enable(tfe_ctx *c, void *stream_)
 tfe_status tfe_cache_select_victims(tfe_ctx *c, int32_t n, int32_t half_life, int32_t *slots, uint32_t *keys,
                                     int32_t *count, void *stream_)
 {
-    if (!c || n < 0 || n > TFE_VICTIMS_MAX || !count || (n > 0 && !slots)) return TFE_ERR_INVALID_ARG;
+    if (!c || n < 0 || n > TFE_VICTIMS_MAX || !count) return TFE_ERR_INVALID_ARG;
     if (!c->d_slot_stats) return TFE_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const int64_t C = c->cfg.gpu_slots;
@@ -982,6 +1033,7 @@ tfe_status tfe_cache_select_victims(tfe_ctx *c, int32_t n, int32_t half_life, in
     tfe_victim_sort_kernel<<<1, 1024, 0, stream>>>(c->d_vs_list, c->d_vs_state, (uint32_t)take, c->d_vs_slots,
                                                    c->d_vs_keys);
     CU(cudaGetLastError());
+    if (!slots) return TFE_OK;      // results stay on the device (tfe_cache_select_victims_device); no synchronisation
     CU(cudaMemcpyAsync(slots, c->d_vs_slots, (size_t)take * 4, cudaMemcpyDeviceToHost, stream));
     if (keys) CU(cudaMemcpyAsync(keys, c->d_vs_keys, (size_t)take * 4, cudaMemcpyDeviceToHost, stream));
     CU(cudaStreamSynchronize(stream));

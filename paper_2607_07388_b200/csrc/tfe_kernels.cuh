@@ -836,6 +836,97 @@ tfe_install_kernel(ulonglong2 *index, const uint32_t *phrase_pos, uint32_t *slot
     for (int i = lane; i < row_vecs; i += 32) o[i] = ld_stream(s + i);
 }
 
+// ---------------------------------------------- cache install from the device
+//
+// The same insertion for a batch that lives on the device and was never checked by the host (the
+// output of the candidate step and of the victim selection): entries that cannot be applied are
+// skipped.  Judged against the state before the call, entry k is a candidate if its id is a
+// phrase, the phrase is not GPU-resident, its slot exists and no earlier entry names the same
+// phrase; it is applied if, in addition, no earlier candidate names the same slot.  "Earlier" is
+// settled with one atomicMax per entry on a stamp per phrase and per slot: a stamp is
+// (call number << 12) | (4095 - k), so the current call beats every older stamp and, within the
+// call, the smallest k wins; nothing has to be cleared between calls.
+//
+//   tfe_install_claim_kernel<0>  every entry stamps its phrase
+//   tfe_install_claim_kernel<1>  every candidate stamps its slot
+//   tfe_install_device_kernel    one warp per entry: the winners install (as tfe_install_kernel)
+#define TFE_INSTALL_DEVICE_MAX 4096
+
+struct TfeInstallDeviceParams {
+    ulonglong2 *index;
+    const uint32_t *phrase_pos;
+    uint32_t *slot_owner;
+    uint4 *rows;
+    int32_t row_vecs;
+    int32_t n;
+    uint32_t n_phrases;
+    int64_t gpu_slots;
+    const uint32_t *ids;            // [n]
+    const uint4 *src;               // [n][row_vecs]
+    const int32_t *dst_slots;       // [n]
+    uint32_t *phrase_stamp;         // [n_phrases]
+    uint32_t *slot_stamp;           // [gpu_slots]
+    uint32_t tag;                   // call number << 12
+    uint8_t *applied;               // [n] or nullptr
+    uint32_t *count;                // entries applied (cleared by the host side before the launches)
+    uint2 *slot_stats;
+    const uint32_t *epoch;
+};
+
+__device__ __forceinline__ bool tfe_install_candidate(const TfeInstallDeviceParams &p, int k)
+{
+    const uint32_t id = p.ids[k];
+    const int32_t dst = p.dst_slots[k];
+    if (id >= p.n_phrases || dst < 0 || (int64_t)dst >= p.gpu_slots) return false;
+    if ((int32_t)(uint32_t)p.index[p.phrase_pos[id]].y >= 0) return false;          // resident before the call
+    return __ldcg(p.phrase_stamp + id) == (p.tag | (uint32_t)(TFE_INSTALL_DEVICE_MAX - 1 - k));
+}
+
+template <int STAGE>
+__global__ void __launch_bounds__(256)
+tfe_install_claim_kernel(const TfeInstallDeviceParams p)
+{
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= p.n) return;
+    const uint32_t stamp = p.tag | (uint32_t)(TFE_INSTALL_DEVICE_MAX - 1 - k);
+    if (STAGE == 0) {
+        const uint32_t id = p.ids[k];
+        if (id < p.n_phrases) atomicMax(p.phrase_stamp + id, stamp);
+    } else {
+        if (tfe_install_candidate(p, k)) atomicMax(p.slot_stamp + p.dst_slots[k], stamp);
+    }
+}
+
+__global__ void __launch_bounds__(TFE_BLOCK_THREADS)
+tfe_install_device_kernel(const TfeInstallDeviceParams p)
+{
+    const int lane = threadIdx.x & 31;
+    const int k = blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5);
+    if (k >= p.n) return;
+    bool apply = false;
+    if (lane == 0) {
+        apply = tfe_install_candidate(p, k) &&
+                __ldcg(p.slot_stamp + p.dst_slots[k]) == (p.tag | (uint32_t)(TFE_INSTALL_DEVICE_MAX - 1 - k));
+        if (p.applied) p.applied[k] = apply ? 1 : 0;
+        if (apply) atomicAdd(p.count, 1u);
+    }
+    apply = __shfl_sync(0xFFFFFFFFu, apply, 0);
+    if (!apply) return;
+    const uint32_t id = p.ids[k];
+    const int32_t dst = p.dst_slots[k];
+    if (lane == 0) {
+        const uint32_t prev = p.slot_owner[dst];
+        if (prev != 0xFFFFFFFFu)
+            p.index[p.phrase_pos[prev]].y = ((unsigned long long)prev << 32) | 0xFFFFFFFFull;   // -1: host tier
+        p.index[p.phrase_pos[id]].y = ((unsigned long long)id << 32) | (uint32_t)dst;
+        p.slot_owner[dst] = id;
+        if (p.slot_stats != nullptr) p.slot_stats[dst] = make_uint2(1u, *p.epoch);
+    }
+    const uint4 *s = p.src + (size_t)k * p.row_vecs;
+    uint4 *o = p.rows + (size_t)dst * p.row_vecs;
+    for (int i = lane; i < p.row_vecs; i += 32) o[i] = ld_stream(s + i);
+}
+
 // ------------------------------------------- prefetch candidates + priority
 //
 // Early-exit guided prefetching after the top-K tokens are known: every predicted next token is

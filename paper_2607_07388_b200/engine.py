@@ -102,6 +102,14 @@ class Engram:
     def cache_install(self, phrase_ids, src_rows, dst_slots, stream=None):
         tfe.tfe_cache_install(self.ctx, phrase_ids, src_rows, dst_slots, stream)
 
+    def cache_install_device(self, phrase_ids: torch.Tensor, src_rows: torch.Tensor, dst_slots: torch.Tensor, stream=None):
+        """Device tensors in, (applied uint8 [n], count int32 [1]) device tensors out; nothing synchronises."""
+        n = int(phrase_ids.shape[0])
+        applied = torch.empty(max(n, 1), dtype=torch.uint8, device=phrase_ids.device)
+        count = torch.zeros(1, dtype=torch.int32, device=phrase_ids.device)
+        tfe.tfe_cache_install_device(self.ctx, n, phrase_ids, src_rows, dst_slots, applied, count, stream)
+        return applied[:n], count
+
     def cache_policy_enable(self, stream=None):
         tfe.tfe_cache_policy_enable(self.ctx, stream)
 
