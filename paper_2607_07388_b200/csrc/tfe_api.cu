@@ -837,7 +837,15 @@ tfe_status lookup_inject_range(tfe_ctx *c, const int32_t *tokens, int32_t B, int
     p.counters = c->d_counters;
     p.slot_stats = c->d_slot_stats; p.epoch = c->d_epoch;
 
-    pick_kernel(variant)<<<(unsigned)grid, TFE_BLOCK_THREADS, 0, stream>>>(p);
+    // Programmatic stream serialisation: the launch may be set up while the kernel before it on the
+    // stream drains; the kernel itself waits for that kernel's completion before its first global access.
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(TFE_BLOCK_THREADS); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    CU(cudaLaunchKernelEx(&cfg, pick_kernel(variant), p));
     CU(cudaGetLastError());
     c->last_entries = Q * cols;
     c->last_grid = (int)grid;

@@ -30,6 +30,16 @@
 // (mul = floor(2^shr / d) + 1, shr = 31 + ceil(log2 d); the host computes both).
 struct TfeFastDiv { uint32_t mul, shr; };
 
+// Programmatic dependent launch: a lookup launched with the stream-serialisation attribute may be set up
+// while the kernel before it on the stream is still draining; it must not touch global memory before
+// this point, where it waits until that kernel has completed and its writes are visible.  No early
+// trigger is issued for the kernel after it (measured: successors that become resident early and sit
+// waiting cost more than the hidden launch latency gains).  Without the attribute this is a no-op.
+__device__ __forceinline__ void tfe_grid_dependency_sync()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 struct TfeLookupParams {
     const int32_t *tokens;
     int32_t B, T, q_start, Tq;
@@ -445,6 +455,7 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
     const uint32_t n_batches = (p.Q + qb - 1) / qb;
     uint32_t my_miss = 0;                        // per thread here; summed per warp below
 
+    tfe_grid_dependency_sync();
     const uint32_t n_warps = gridDim.x * TFE_WARPS_PER_BLOCK;
     for (uint32_t batch = blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5); batch < n_batches; batch += n_warps) {
         // query lq of batch b is b + lq * n_batches: the queries of a warp are spread over the call,
@@ -665,6 +676,7 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
     const uint32_t q_lo = RANGED ? p.q_lo : 0u, q_hi = RANGED ? p.q_hi : p.Q;
     const uint32_t n_batches = (q_hi - q_lo + qb - 1) / qb;
     const uint32_t n_warps = gridDim.x * TFE_WARPS_PER_BLOCK;
+    tfe_grid_dependency_sync();
     const uint32_t epoch = p.slot_stats != nullptr ? __ldcg(p.epoch) : 0u;
     uint32_t my_miss = 0;
 
