@@ -21,6 +21,7 @@
  *   - prefetch candidates from predicted tokens + priority     [Sec. 4.4, candidate set Q_t, score s = p r c]
  *   - retention ranking of GPU-tier slots (frequency, recency) [Sec. 4.3, cache policy signals]
  *   - early-exit prefetch head: softmax(W_pref h), top-K        [Sec. 4.4, p_early and T_early equations]
+ *   - n-gram extraction with a frequency threshold              [Sec. 4.2, construction pipeline; Sec. 5.3]
  *
  * Parity pins: every function here is pinned by tests that do not call it to
  * produce their expected values (hand-made cases, closed forms, a library
@@ -662,4 +663,91 @@ void orc_head_topk(int32_t V, int32_t B, int32_t K, const double *z, int32_t *to
         if (lse) lse[b] = top + log(sum);
         free(r);
     }
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * N-gram extraction with a frequency threshold [Sec. 4.2 construction pipeline: candidate phrases
+ * are multi-token expressions such as bigrams and trigrams, selected by a frequency threshold;
+ * Sec. 5.3: this tokenizer-level n-gram extraction is the dominant offline cost].
+ *
+ * corpus   tokens int32 [L]; an id outside [0, vocab) separates documents: no window contains one.
+ * window   for a configured order n and an end position t >= n - 1 whose n ids x_{t-n+1} .. x_t are
+ *          all valid, that tuple occurs once at t.
+ * count(tuple) = number of its occurrences, first(tuple) = its smallest end position.
+ *
+ * Result: the tuples with count >= min_count, in ascending (first, n) order -- the order in which a
+ * reader of the corpus meets them.  Returns how many there are; writes the first `cap` of them
+ * (out_tokens [cap][4] padded with -1, out_len, out_count).  distinct[oi] = number of different
+ * tuples of order orders[oi].  hist (length hist_bins, may be NULL): hist[c] = number of different
+ * tuples, all orders together, that occur exactly c times, the last bin collecting every c >=
+ * hist_bins - 1.
+ *
+ * Method: the definition.  Every window becomes a record; records are sorted by (n, tuple, t), so that
+ * the occurrences of one tuple are adjacent and its first one leads; the survivors are sorted by
+ * (first, n). */
+typedef struct { int32_t n, tok[ORC_MAX_ORDERS]; int64_t t; uint32_t count; } orc_window;
+
+static int window_cmp(const void *pa, const void *pb)
+{
+    const orc_window *a = (const orc_window *)pa, *b = (const orc_window *)pb;
+    if (a->n != b->n) return a->n < b->n ? -1 : 1;
+    for (int j = 0; j < ORC_MAX_ORDERS; ++j)
+        if (a->tok[j] != b->tok[j]) return a->tok[j] < b->tok[j] ? -1 : 1;
+    return a->t < b->t ? -1 : (a->t > b->t ? 1 : 0);
+}
+
+static int first_cmp(const void *pa, const void *pb)
+{
+    const orc_window *a = (const orc_window *)pa, *b = (const orc_window *)pb;
+    if (a->t != b->t) return a->t < b->t ? -1 : 1;
+    return a->n < b->n ? -1 : (a->n > b->n ? 1 : 0);
+}
+
+int64_t orc_mine_ngrams(int64_t L, const int32_t *tokens, int32_t vocab, int32_t n_orders, const int32_t *orders,
+                        uint32_t min_count, int64_t cap, int32_t *out_tokens, uint8_t *out_len, uint32_t *out_count,
+                        int64_t *distinct, int32_t hist_bins, int64_t *hist)
+{
+    orc_window *w = (orc_window *)malloc((size_t)(L * n_orders + 1) * sizeof *w);
+    int64_t n_w = 0;
+    for (int64_t t = 0; t < L; ++t)
+        for (int32_t oi = 0; oi < n_orders; ++oi) {
+            const int32_t n = orders[oi];
+            if (t < n - 1) continue;
+            int valid = 1;
+            for (int32_t j = 0; j < n; ++j) {
+                const int32_t x = tokens[t - n + 1 + j];
+                if (x < 0 || x >= vocab) valid = 0;
+            }
+            if (!valid) continue;
+            w[n_w].n = n;
+            for (int32_t j = 0; j < ORC_MAX_ORDERS; ++j) w[n_w].tok[j] = j < n ? tokens[t - n + 1 + j] : -1;
+            w[n_w].t = t;
+            w[n_w].count = 0;
+            ++n_w;
+        }
+    qsort(w, (size_t)n_w, sizeof *w, window_cmp);
+    for (int32_t oi = 0; oi < n_orders; ++oi) distinct[oi] = 0;
+    if (hist) for (int32_t c = 0; c < hist_bins; ++c) hist[c] = 0;
+    int64_t n_keep = 0;                         /* survivors are moved to the front of w */
+    for (int64_t i = 0; i < n_w;) {
+        int64_t j = i + 1;
+        while (j < n_w && w[j].n == w[i].n && memcmp(w[j].tok, w[i].tok, sizeof w[i].tok) == 0) ++j;
+        const int64_t count = j - i;            /* w[i] is the first occurrence: smallest t of the run */
+        for (int32_t oi = 0; oi < n_orders; ++oi) if (orders[oi] == w[i].n) ++distinct[oi];
+        if (hist) ++hist[count < hist_bins - 1 ? count : hist_bins - 1];
+        if (count >= (int64_t)min_count) {
+            w[n_keep] = w[i];
+            w[n_keep].count = (uint32_t)count;
+            ++n_keep;
+        }
+        i = j;
+    }
+    qsort(w, (size_t)n_keep, sizeof *w, first_cmp);
+    for (int64_t i = 0; i < n_keep && i < cap; ++i) {
+        for (int32_t j = 0; j < ORC_MAX_ORDERS; ++j) out_tokens[i * ORC_MAX_ORDERS + j] = w[i].tok[j];
+        out_len[i] = (uint8_t)w[i].n;
+        out_count[i] = w[i].count;
+    }
+    free(w);
+    return n_keep;
 }

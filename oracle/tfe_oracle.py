@@ -270,3 +270,23 @@ def head_topk(z, K):
     tokens, prob, lse = np.empty((B, K), np.int32), np.empty((B, K), np.float64), np.empty(B, np.float64)
     lib().orc_head_topk(C.c_int32(V), C.c_int32(B), C.c_int32(K), _p(z), _p(tokens), _p(prob), _p(lse))
     return tokens, prob, lse
+
+
+# -- n-gram extraction with a frequency threshold (independent of any phrase table) ---------------
+def mine_ngrams(tokens, vocab, orders, min_count=1, cap=None, hist_bins=1024):
+    """(phrase_tokens int32 [n, 4], phrase_len uint8 [n], count uint32 [n], n_found, distinct int64
+    [n_orders], hist int64 [hist_bins]); n = min(n_found, cap), ascending (first occurrence, order)."""
+    tokens = _c(tokens, np.int32).reshape(-1)
+    orders = _c(orders, np.int32)
+    L = len(tokens)
+    cap = L * len(orders) if cap is None else int(cap)
+    pt = np.full((max(cap, 1), 4), -1, np.int32)
+    pl, pc = np.zeros(max(cap, 1), np.uint8), np.zeros(max(cap, 1), np.uint32)
+    distinct, hist = np.zeros(len(orders), np.int64), np.zeros(hist_bins, np.int64)
+    f = lib().orc_mine_ngrams
+    f.restype = C.c_int64
+    n_found = f(C.c_int64(L), _p(tokens), C.c_int32(vocab), C.c_int32(len(orders)), _p(orders),
+                C.c_uint32(min_count), C.c_int64(cap), _p(pt), _p(pl), _p(pc), _p(distinct),
+                C.c_int32(hist_bins), _p(hist))
+    n = int(min(n_found, cap))
+    return pt[:n].copy(), pl[:n].copy(), pc[:n].copy(), int(n_found), distinct, hist

@@ -801,3 +801,79 @@ def test_lenient_install_against_independent_restatement(oracle_mod):
         np.testing.assert_array_equal(o.slot_owner, [owner.get(s_, -1) for s_ in range(C)])
         for s_, v in rows.items():
             assert (o.rows[s_] == v).all()
+
+
+# ---------------------------------------------------------------------------------------------
+# n-gram extraction with a frequency threshold (Sec. 4.2 construction pipeline, Sec. 5.3)
+# ---------------------------------------------------------------------------------------------
+def test_mine_ngrams_hand_worked(oracle_mod):
+    """Corpus 5 7 5 7 9 | 5 7 with one separator, orders 2 and 3, worked by hand: (5,7) ends at 1, 3 and 7;
+    the windows ending at 5, 6 (and, for order 3, 7) contain the separator."""
+    tok = np.array([5, 7, 5, 7, 9, -1, 5, 7], np.int32)
+    pt, pl, pc, n_found, distinct, hist = oracle_mod.mine_ngrams(tok, 10, (2, 3), min_count=1, hist_bins=8)
+    assert n_found == 6 and distinct.tolist() == [3, 3]
+    assert pt.tolist() == [[5, 7, -1, -1], [7, 5, -1, -1], [5, 7, 5, -1], [7, 5, 7, -1], [7, 9, -1, -1], [5, 7, 9, -1]]
+    assert pl.tolist() == [2, 2, 3, 3, 2, 3] and pc.tolist() == [3, 1, 1, 1, 1, 1]
+    assert hist.tolist() == [0, 5, 0, 1, 0, 0, 0, 0]
+    pt, pl, pc, n_found, _, _ = oracle_mod.mine_ngrams(tok, 10, (2, 3), min_count=2)
+    assert n_found == 1 and pt.tolist() == [[5, 7, -1, -1]] and pc.tolist() == [3]
+    pt, pl, pc, n_found, _, _ = oracle_mod.mine_ngrams(tok, 10, (2, 3), min_count=1, cap=2)
+    assert n_found == 6 and pt.tolist() == [[5, 7, -1, -1], [7, 5, -1, -1]]
+    # an id at or above the vocabulary size separates like a negative one; the last histogram bin collects
+    pt, _, pc, n_found, distinct, hist = oracle_mod.mine_ngrams(np.array([5, 7, 5, 7, 9, 10, 5, 7], np.int32), 10, (2,), hist_bins=3)
+    assert n_found == 3 and pc.tolist() == [3, 1, 1] and hist.tolist() == [0, 2, 1]
+
+
+def test_mine_ngrams_closed_forms(oracle_mod):
+    # one token repeated: a single tuple per order, L - n + 1 times, first met at n - 1
+    L = 37
+    pt, pl, pc, n_found, distinct, _ = oracle_mod.mine_ngrams(np.full(L, 3, np.int32), 8, (1, 2, 3, 4))
+    assert n_found == 4 and pl.tolist() == [1, 2, 3, 4] and pc.tolist() == [L, L - 1, L - 2, L - 3]
+    assert distinct.tolist() == [1, 1, 1, 1]
+    # a corpus of period P over P different tokens: P tuples per order, the L - n + 1 windows shared out evenly
+    P, L = 7, 100
+    tok = (np.arange(L) % P).astype(np.int32)
+    for n in (2, 3, 4):
+        pt, pl, pc, n_found, distinct, _ = oracle_mod.mine_ngrams(tok, P, (n,))
+        assert n_found == P == distinct[0] and int(pc.sum()) == L - n + 1
+        assert set(pc.tolist()) <= {(L - n + 1) // P, (L - n + 1) // P + 1}
+        assert pt[:, 0].tolist() == list(range(P))              # met in corpus order
+        assert all(pt[i, j] == (i + j) % P for i in range(P) for j in range(n))
+    # every token different: every window is its own tuple, nothing survives a threshold of 2
+    tok = np.random.default_rng(5).permutation(500).astype(np.int32)
+    pt, pl, pc, n_found, distinct, hist = oracle_mod.mine_ngrams(tok, 500, (2, 3))
+    assert n_found == 499 + 498 and distinct.tolist() == [499, 498] and hist[1] == n_found
+    assert oracle_mod.mine_ngrams(tok, 500, (2, 3), min_count=2)[3] == 0
+    # shorter than the order / empty
+    assert oracle_mod.mine_ngrams(np.array([1, 2], np.int32), 5, (3, 4))[3] == 0
+    assert oracle_mod.mine_ngrams(np.zeros(0, np.int32), 5, (2,))[3] == 0
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_mine_ngrams_against_library_unique(oracle_mod, seed):
+    """The counts are numpy.unique's over the sliding windows; the order is that of first occurrence."""
+    rng = np.random.default_rng([88, seed])
+    vocab = int(rng.integers(3, 40))
+    L = int(rng.integers(50, 3000))
+    tok = rng.integers(0, vocab, size=L).astype(np.int32)
+    tok[rng.random(L) < 0.05] = rng.choice([-1, vocab, vocab + 7])
+    orders = [o for o in (1, 2, 3, 4) if rng.random() < 0.7] or [2]
+    min_count = int(rng.integers(1, 4))
+    pt, pl, pc, n_found, distinct, hist = oracle_mod.mine_ngrams(tok, vocab, orders, min_count=min_count, hist_bins=16)
+    expect, exp_hist = {}, np.zeros(16, np.int64)
+    for oi, n in enumerate(orders):
+        win = np.lib.stride_tricks.sliding_window_view(tok, n)                 # window i ends at i + n - 1
+        ok = ((win >= 0) & (win < vocab)).all(axis=1)
+        uniq, first_idx, counts = np.unique(win[ok], axis=0, return_index=True, return_counts=True)
+        ends = np.flatnonzero(ok)[first_idx] + n - 1
+        assert distinct[oi] == len(uniq)
+        np.add.at(exp_hist, np.minimum(counts, 15), 1)
+        for u, e, c in zip(uniq, ends, counts):
+            if c >= min_count:
+                expect[(int(e), n)] = (tuple(int(x) for x in u), int(c))
+    np.testing.assert_array_equal(hist, exp_hist)
+    assert n_found == len(expect)
+    for i, key in enumerate(sorted(expect)):
+        tup, c = expect[key]
+        assert pl[i] == key[1] and pc[i] == c
+        assert tuple(pt[i, :key[1]].tolist()) == tup and (pt[i, key[1]:] == -1).all()
