@@ -408,6 +408,42 @@ tfe_status tfe_head_status(tfe_head *head, uint32_t *device_flags, void *stream)
 /* Launch geometry: CTAs, vocabulary rows per CTA, rows of each CTA's short last tile. */
 tfe_status tfe_head_geometry(const tfe_head *head, int32_t *grid, int32_t *rows_per_cta, int32_t *tail_rows);
 
+/*
+ * N-gram extraction with a frequency threshold (paper Sec. 4.2, construction pipeline: candidate
+ * phrases such as bigrams and trigrams are selected by a frequency threshold; Sec. 5.3: this
+ * tokenizer-level n-gram extraction dominates the offline cost of building a table).  Independent of
+ * any context; its output is the phrase table that tfe_index_build_device takes.
+ *
+ *   tokens         DEVICE int32 [L], the tokenised corpus; an id outside [0, vocab) separates documents:
+ *                  no window contains one.  0 <= L <= TFE_MINE_MAX_TOKENS.
+ *   orders         HOST int32 [n_orders], strictly ascending, each in 1..4.
+ *   window         for an order n and an end position t >= n - 1 whose n ids x_{t-n+1} .. x_t are all
+ *                  valid, that tuple occurs once at t.  count(tuple) = number of occurrences,
+ *                  first(tuple) = its smallest end position.
+ *   result         the tuples with count >= min_count (0 means 1) in ascending (first, n) order:
+ *                  phrase_tokens DEVICE int32 [cap][4] (16-byte aligned; unused trailing ids -1),
+ *                  phrase_len DEVICE uint8 [cap], phrase_count DEVICE uint32 [cap]; may be NULL if cap = 0.
+ *   n_found        HOST: how many tuples qualify; min(n_found, cap) entries were written (the first ones
+ *                  in that order) -- n_found > cap is not an error, the caller raises min_count or cap.
+ *   distinct       HOST int64 [n_orders] or NULL: different tuples per order.
+ *   hist           HOST int64 [TFE_MINE_HIST_BINS] or NULL: hist[c] = different tuples, all orders together,
+ *                  that occur exactly c times; the last bin collects every c >= TFE_MINE_HIST_BINS - 1.
+ *                  sum_{c >= m} hist[c] is n_found for min_count = m, so one call tells which threshold
+ *                  yields a table of a wanted size.
+ *
+ * Allocates and frees its own workspace (tfe_mine_workspace_bytes; about 24..48 bytes per token for the
+ * counting table plus 4 bytes per token and order), launches on `stream` and synchronises it.  Exact for
+ * every vocabulary: orders whose ids do not fit one 64-bit key side by side are keyed through the exact
+ * names of their halves.  Errors: TFE_ERR_INVALID_ARG, TFE_ERR_CUDA (workspace does not fit),
+ * TFE_ERR_INTERNAL (a bounded probe ran out).
+ */
+#define TFE_MINE_HIST_BINS 1024
+#define TFE_MINE_MAX_TOKENS (1ll << 30)
+tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int32_t n_orders, const int32_t *orders,
+                           uint32_t min_count, int64_t cap, int32_t *phrase_tokens, uint8_t *phrase_len,
+                           uint32_t *phrase_count, int64_t *n_found, int64_t *distinct, int64_t *hist, void *stream);
+int64_t tfe_mine_workspace_bytes(int64_t L, int32_t n_orders);   /* -1 for invalid arguments */
+
 #ifdef __cplusplus
 }
 #endif

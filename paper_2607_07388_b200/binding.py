@@ -34,7 +34,7 @@ EXPORTS = ["tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tf
            "tfe_launch_geometry", "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
            "tfe_cache_policy_enable", "tfe_cache_select_victims", "tfe_cache_select_victims_device",
            "tfe_cache_stats", "tfe_head_create", "tfe_head_destroy", "tfe_head_topk", "tfe_head_buffers",
-           "tfe_head_status", "tfe_head_geometry"]
+           "tfe_head_status", "tfe_head_geometry", "tfe_mine_ngrams", "tfe_mine_workspace_bytes"]
 
 
 class TfeConfig(C.Structure):
@@ -108,12 +108,15 @@ def lib() -> C.CDLL:
         L.tfe_head_buffers.argtypes = [vp, C.POINTER(vp), C.POINTER(i64), C.POINTER(vp)]
         L.tfe_head_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         L.tfe_head_geometry.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
+        L.tfe_mine_ngrams.argtypes = [vp, i64, i32, i32, vp, C.c_uint32, i64, vp, vp, vp, C.POINTER(i64), vp, vp, vp]
+        L.tfe_mine_workspace_bytes.argtypes = [i64, i32]
+        L.tfe_mine_workspace_bytes.restype = i64
         for name in ("tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tfe_cache_install_device", "tfe_lookup_inject", "tfe_lookup_inject_host",
                      "tfe_miss_list", "tfe_miss_list_device", "tfe_index_geometry", "tfe_launch_geometry",
                      "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
                      "tfe_cache_policy_enable", "tfe_cache_select_victims", "tfe_cache_select_victims_device",
                      "tfe_cache_stats", "tfe_head_create", "tfe_head_topk", "tfe_head_buffers", "tfe_head_status",
-                     "tfe_head_geometry"):
+                     "tfe_head_geometry", "tfe_mine_ngrams"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -377,3 +380,24 @@ def tfe_head_geometry(head: int):
     g, r, t = C.c_int32(0), C.c_int32(0), C.c_int32(0)
     _check(lib().tfe_head_geometry(head, C.byref(g), C.byref(r), C.byref(t)), "tfe_head_geometry")
     return g.value, r.value, t.value
+
+
+MINE_HIST_BINS = 1024
+MINE_MAX_TOKENS = 1 << 30
+
+
+def tfe_mine_workspace_bytes(L: int, n_orders: int) -> int:
+    return int(lib().tfe_mine_workspace_bytes(int(L), int(n_orders)))
+
+
+def tfe_mine_ngrams(tokens, L: int, vocab: int, orders, min_count: int, cap: int, phrase_tokens=None, phrase_len=None,
+                    phrase_count=None, want_hist: bool = True, stream=None):
+    """tokens and the three outputs on the device; returns (n_found, distinct int64 [n_orders], hist int64 [1024] or None)."""
+    o = np.ascontiguousarray(orders, np.int32)
+    found = C.c_int64(0)
+    distinct = np.zeros(len(o), np.int64)
+    hist = np.zeros(MINE_HIST_BINS, np.int64) if want_hist else None
+    _check(lib().tfe_mine_ngrams(_addr(tokens), int(L), int(vocab), len(o), _addr(o), int(min_count), int(cap),
+                                 _addr(phrase_tokens), _addr(phrase_len), _addr(phrase_count), C.byref(found),
+                                 _addr(distinct), _addr(hist), _stream(stream)), "tfe_mine_ngrams")
+    return found.value, distinct, hist

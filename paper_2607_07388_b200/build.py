@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtfe.so")
-SOURCES = [os.path.join(CSRC, "tfe_api.cu"), os.path.join(CSRC, "tfe_head.cu")]
+SOURCES = [os.path.join(CSRC, "tfe_api.cu"), os.path.join(CSRC, "tfe_head.cu"), os.path.join(CSRC, "tfe_mine.cu")]
 DEPS = SOURCES + [os.path.join(CSRC, "tfe_kernels.cuh"), os.path.join(CSRC, "tfe_key.cuh"),
                   os.path.join(os.path.dirname(HERE), "include", "tfe.h")]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",

@@ -1,0 +1,377 @@
+// N-gram extraction with a frequency threshold (paper Sec. 4.2, construction pipeline: candidate phrases
+// such as bigrams and trigrams selected by a frequency threshold; Sec. 5.3: this tokenizer-level n-gram
+// extraction is the dominant offline cost of building a table).
+//
+// Input: a tokenised corpus on the device, int32 [L]; an id outside [0, vocab) separates documents.  For
+// every configured order n and end position t whose n ids are valid, the tuple x_{t-n+1..t} occurs once.
+// Output: every tuple that occurs at least min_count times, with its count, in ascending (end position of
+// its first occurrence, n) order -- the phrase table that tfe_index_build_device takes.
+//
+// No sort: counting is a hash-table pass, the order comes from the corpus itself.
+//
+//   tfe_mine_count_kernel   one thread per end position.  The window's exact 64-bit key (ids packed side
+//                           by side; an order too wide for 64 bits is keyed by the table slots of its two
+//                           halves, which are exact names of those bigrams) is inserted into an
+//                           open-addressing table of 16-byte slots {key, count, first} by a 64-bit
+//                           compare-and-swap on the key; equal keys inside a warp are combined first
+//                           (match.any), then one atomicAdd on the count and one atomicMin on the first
+//                           end position.  The slot index is remembered per position.
+//   tfe_mine_mark_kernel    one thread per end position: the position that IS the first occurrence of its
+//                           tuple speaks for the tuple -- counts it as distinct, adds it to the histogram of
+//                           counts and, if the count reaches the threshold, leaves the count in the
+//                           per-position array (0 everywhere else).  The table is then reused by the next
+//                           order.
+//   tfe_mine_block_sums / tfe_mine_scan / tfe_mine_emit
+//                           ordered compaction over (position, order): per-block totals, their exclusive
+//                           scan, and the writes of tuple, length and count at the scanned offsets.
+//
+// All loops over table slots are bounded by the table's size; a probe that runs out sets an error word.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdint>
+#include <cstring>
+#include <vector>
+
+#include "../../include/tfe.h"
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kPosPerThread = 4;                       // emit / block-sum kernels
+constexpr int kPosPerBlock = kThreads * kPosPerThread;
+constexpr uint64_t kEmpty = 0xFFFFFFFFFFFFFFFFull;
+constexpr uint32_t kNoSlot = 0xFFFFFFFFu;
+
+struct MineSlot { unsigned long long key; uint32_t count_m1; uint32_t first; };   // memset 0xFF = empty, count 0
+static_assert(sizeof(MineSlot) == 16, "slot layout");
+
+struct MineTotals {
+    unsigned long long distinct;       // tuples of the order being marked
+    unsigned long long found;          // written by the scan: entries that qualify, all orders
+    uint32_t error;                    // a probe ran the whole table without finding a place
+    uint32_t pad;
+    unsigned long long hist[TFE_MINE_HIST_BINS];
+};
+
+__device__ __forceinline__ uint64_t mix64(uint64_t x)
+{
+    x ^= x >> 30; x *= 0xBF58476D1CE4E5B9ull;
+    x ^= x >> 27; x *= 0x94D049BB133111EBull;
+    x ^= x >> 31;
+    return x;
+}
+
+// mode 0: ids packed side by side (n * tok_bits <= 63).  mode 1 (n = 4 only): the slots of the bigrams
+// ending at t - 2 and at t in the bigram table of this corpus, 31 bits each.
+__global__ void __launch_bounds__(kThreads)
+tfe_mine_count_kernel(const int32_t *__restrict__ tokens, uint32_t L, int32_t vocab, int n, int tok_bits, int mode,
+                      const uint32_t *__restrict__ pair_slot, MineSlot *table, uint32_t mask,
+                      uint32_t *__restrict__ slot_of, MineTotals *totals)
+{
+    const uint32_t t = blockIdx.x * (uint32_t)kThreads + threadIdx.x;
+    const int lane = threadIdx.x & 31;
+    bool valid = t < L && t + 1 >= (uint32_t)n;
+    unsigned long long key = 0;
+    if (valid) {
+        if (mode == 0) {
+            for (int j = 0; j < n; ++j) {
+                const int32_t x = __ldg(tokens + t - (n - 1) + j);
+                if ((uint32_t)x >= (uint32_t)vocab) valid = false;
+                key = (key << tok_bits) | (uint32_t)x;
+            }
+        } else {
+            const uint32_t a = __ldg(pair_slot + t - 2), b = __ldg(pair_slot + t);
+            valid = a != kNoSlot && b != kNoSlot;
+            key = ((unsigned long long)a << 31) | b;
+        }
+    }
+    uint32_t slot = kNoSlot;
+    const unsigned act = __ballot_sync(0xFFFFFFFFu, valid);
+    if (valid) {
+        const unsigned grp = __match_any_sync(act, key);
+        const int leader = __ffs(grp) - 1;                 // lowest lane: the smallest t of the group
+        if (lane == leader) {
+            uint32_t s = (uint32_t)mix64(key) & mask;
+            for (uint32_t probes = 0; probes <= mask; ++probes, s = (s + 1) & mask) {
+                unsigned long long k = *reinterpret_cast<volatile unsigned long long *>(&table[s].key);
+                if (k == kEmpty) k = atomicCAS(&table[s].key, kEmpty, key);
+                if (k == kEmpty || k == key) { slot = s; break; }
+            }
+            if (slot != kNoSlot) {
+                atomicAdd(&table[slot].count_m1, (uint32_t)__popc(grp));
+                atomicMin(&table[slot].first, t);
+            } else {
+                atomicExch(&totals->error, 1u);
+            }
+        }
+        slot = __shfl_sync(grp, slot, leader);
+    }
+    if (t < L) slot_of[t] = slot;
+}
+
+// val[t] = count of the tuple ending at t if t is its first occurrence and count >= min_count, else 0.
+__global__ void __launch_bounds__(kThreads)
+tfe_mine_mark_kernel(const uint32_t *__restrict__ slot_of, uint32_t L, const MineSlot *__restrict__ table,
+                     uint32_t min_count, uint32_t *__restrict__ val, MineTotals *totals)
+{
+    __shared__ uint32_t s_hist[TFE_MINE_HIST_BINS];
+    __shared__ uint32_t s_distinct;
+    for (int i = threadIdx.x; i < TFE_MINE_HIST_BINS; i += kThreads) s_hist[i] = 0;
+    if (threadIdx.x == 0) s_distinct = 0;
+    __syncthreads();
+    const uint32_t t = blockIdx.x * (uint32_t)kThreads + threadIdx.x;
+    if (t < L) {
+        const uint32_t s = __ldg(slot_of + t);
+        uint32_t v = 0;
+        if (s != kNoSlot) {
+            const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(table + s));     // {key lo, key hi, count - 1, first}
+            if (raw.w == t) {
+                const uint32_t count = raw.z + 1u;
+                atomicAdd(&s_distinct, 1u);
+                atomicAdd(&s_hist[min(count, (uint32_t)TFE_MINE_HIST_BINS - 1u)], 1u);
+                if (count >= min_count) v = count;
+            }
+        }
+        val[t] = v;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < TFE_MINE_HIST_BINS; i += kThreads)
+        if (s_hist[i]) atomicAdd(&totals->hist[i], (unsigned long long)s_hist[i]);
+    if (threadIdx.x == 0 && s_distinct) atomicAdd(&totals->distinct, (unsigned long long)s_distinct);
+}
+
+struct MineVals { const uint32_t *val[4]; int n[4]; int n_orders; };
+
+__global__ void __launch_bounds__(kThreads)
+tfe_mine_block_sums_kernel(MineVals v, uint32_t L, uint32_t *__restrict__ block_sums)
+{
+    __shared__ uint32_t s_sum;
+    if (threadIdx.x == 0) s_sum = 0;
+    __syncthreads();
+    uint32_t mine = 0;
+    const uint32_t base = blockIdx.x * (uint32_t)kPosPerBlock;
+    for (int j = 0; j < kPosPerThread; ++j) {
+        const uint32_t t = base + j * kThreads + threadIdx.x;
+        if (t < L) {
+#pragma unroll
+            for (int oi = 0; oi < 4; ++oi)
+                if (oi < v.n_orders) mine += __ldg(v.val[oi] + t) != 0u;
+        }
+    }
+    mine = __reduce_add_sync(0xFFFFFFFFu, mine);
+    if ((threadIdx.x & 31) == 0 && mine) atomicAdd(&s_sum, mine);
+    __syncthreads();
+    if (threadIdx.x == 0) block_sums[blockIdx.x] = s_sum;
+}
+
+// Exclusive scan of the block totals, one block, running carry; the grand total goes to totals->found.
+__global__ void __launch_bounds__(1024)
+tfe_mine_scan_kernel(const uint32_t *__restrict__ block_sums, uint32_t n_blocks, unsigned long long *__restrict__ block_offs,
+                     MineTotals *totals)
+{
+    __shared__ unsigned long long s_warp[32];
+    __shared__ unsigned long long s_carry;
+    if (threadIdx.x == 0) s_carry = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (uint32_t base = 0; base < n_blocks; base += 1024) {
+        const uint32_t i = base + threadIdx.x;
+        const unsigned long long x = i < n_blocks ? block_sums[i] : 0ull;
+        unsigned long long incl = x;
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+            if (lane >= d) incl += y;
+        }
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            unsigned long long w = s_warp[lane], wi = w;
+            for (int d = 1; d < 32; d <<= 1) {
+                const unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, wi, d);
+                if (lane >= d) wi += y;
+            }
+            s_warp[lane] = wi - w;                     // exclusive over warps
+        }
+        __syncthreads();
+        const unsigned long long carry = s_carry;
+        if (i < n_blocks) block_offs[i] = carry + s_warp[warp] + incl - x;
+        __syncthreads();
+        if (threadIdx.x == 1023) s_carry = carry + s_warp[warp] + incl;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) totals->found = s_carry;
+}
+
+// Entry e = (t, oi) in ascending (t, oi) order.  A thread owns kPosPerThread CONSECUTIVE positions here
+// (unlike the block-sum kernel, whose per-block totals do not depend on the assignment).
+__global__ void __launch_bounds__(kThreads)
+tfe_mine_emit_kernel(MineVals v, const int32_t *__restrict__ tokens, uint32_t L,
+                     const unsigned long long *__restrict__ block_offs, unsigned long long cap,
+                     int32_t *__restrict__ out_tokens, uint8_t *__restrict__ out_len, uint32_t *__restrict__ out_count)
+{
+    __shared__ uint32_t s_warp[kThreads / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t t0 = blockIdx.x * (uint32_t)kPosPerBlock + threadIdx.x * kPosPerThread;
+    uint32_t cnt[kPosPerThread][4];
+    uint32_t mine = 0;
+#pragma unroll
+    for (int j = 0; j < kPosPerThread; ++j)
+#pragma unroll
+        for (int oi = 0; oi < 4; ++oi) {
+            cnt[j][oi] = (oi < v.n_orders && t0 + j < L) ? __ldg(v.val[oi] + t0 + j) : 0u;
+            mine += cnt[j][oi] != 0u;
+        }
+    uint32_t incl = mine;
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= d) incl += y;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    uint32_t before = 0;
+    for (int w = 0; w < warp; ++w) before += s_warp[w];
+    unsigned long long pos = block_offs[blockIdx.x] + before + incl - mine;
+    if (mine == 0) return;
+#pragma unroll
+    for (int j = 0; j < kPosPerThread; ++j)
+#pragma unroll
+        for (int oi = 0; oi < 4; ++oi) {
+            if (cnt[j][oi] == 0u) continue;
+            if (pos < cap) {
+                const int n = v.n[oi];
+                const uint32_t t = t0 + j;
+                int4 tup;
+                tup.x = n > 0 ? __ldg(tokens + t - (n - 1)) : -1;
+                tup.y = n > 1 ? __ldg(tokens + t - (n - 1) + 1) : -1;
+                tup.z = n > 2 ? __ldg(tokens + t - (n - 1) + 2) : -1;
+                tup.w = n > 3 ? __ldg(tokens + t - (n - 1) + 3) : -1;
+                reinterpret_cast<int4 *>(out_tokens)[pos] = tup;
+                out_len[pos] = (uint8_t)n;
+                out_count[pos] = cnt[j][oi];
+            }
+            ++pos;
+        }
+}
+
+int bits_for(uint32_t max_value)
+{
+    int b = 1;
+    while (b < 32 && (max_value >> b) != 0) ++b;
+    return b;
+}
+
+uint64_t table_slots_for(int64_t L)
+{
+    uint64_t want = (uint64_t)std::max<int64_t>(1024, L + L / 2), cap = 1024;
+    while (cap < want) cap <<= 1;
+    return cap;
+}
+
+struct Workspace {
+    std::vector<void *> ptrs;
+    ~Workspace() { for (void *p : ptrs) cudaFree(p); }
+    template <class T> bool alloc(T **p, size_t n)
+    {
+        void *q = nullptr;
+        if (cudaMalloc(&q, std::max<size_t>(n, 1) * sizeof(T)) != cudaSuccess) { (void)cudaGetLastError(); return false; }
+        ptrs.push_back(q);
+        *p = static_cast<T *>(q);
+        return true;
+    }
+};
+
+}  // namespace
+
+extern "C" {
+
+int64_t tfe_mine_workspace_bytes(int64_t L, int32_t n_orders)
+{
+    if (L < 0 || n_orders < 1 || n_orders > 4) return -1;
+    const int64_t n_blocks = (L + kPosPerBlock - 1) / kPosPerBlock;
+    return (int64_t)table_slots_for(L) * (int64_t)sizeof(MineSlot) + (int64_t)(n_orders + 2) * L * 4 + n_blocks * 12
+           + (int64_t)sizeof(MineTotals);
+}
+
+tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int32_t n_orders, const int32_t *orders,
+                           uint32_t min_count, int64_t cap, int32_t *phrase_tokens, uint8_t *phrase_len,
+                           uint32_t *phrase_count, int64_t *n_found, int64_t *distinct, int64_t *hist, void *stream_)
+{
+    if (L < 0 || L > TFE_MINE_MAX_TOKENS || vocab < 1 || n_orders < 1 || n_orders > 4 || !orders || cap < 0 || !n_found)
+        return TFE_ERR_INVALID_ARG;
+    for (int i = 0; i < n_orders; ++i)
+        if (orders[i] < 1 || orders[i] > 4 || (i > 0 && orders[i] <= orders[i - 1])) return TFE_ERR_INVALID_ARG;
+    if (L > 0 && !tokens) return TFE_ERR_INVALID_ARG;
+    if (cap > 0 && (!phrase_tokens || !phrase_len || !phrase_count)) return TFE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(phrase_tokens) & 15u) != 0) return TFE_ERR_INVALID_ARG;
+    *n_found = 0;
+    if (distinct) for (int i = 0; i < n_orders; ++i) distinct[i] = 0;
+    if (hist) for (int i = 0; i < TFE_MINE_HIST_BINS; ++i) hist[i] = 0;
+    if (L == 0) return TFE_OK;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+#define MCU(call) do { if ((call) != cudaSuccess) { (void)cudaGetLastError(); return TFE_ERR_CUDA; } } while (0)
+
+    const int tok_bits = bits_for((uint32_t)(vocab - 1));
+    const bool composite4 = orders[n_orders - 1] == 4 && 4 * tok_bits > 63;
+    const uint64_t slots = table_slots_for(L);
+    const uint32_t mask = (uint32_t)(slots - 1);
+    const uint32_t n_pos_blocks = (uint32_t)((L + kThreads - 1) / kThreads);
+    const uint32_t n_blocks = (uint32_t)((L + kPosPerBlock - 1) / kPosPerBlock);
+
+    Workspace ws;
+    MineSlot *table = nullptr;
+    uint32_t *slot_of = nullptr, *pair_slot = nullptr, *block_sums = nullptr, *val[4] = {nullptr, nullptr, nullptr, nullptr};
+    unsigned long long *block_offs = nullptr;
+    MineTotals *totals = nullptr;
+    bool ok = ws.alloc(&table, slots) && ws.alloc(&slot_of, (size_t)L) && ws.alloc(&block_sums, n_blocks)
+              && ws.alloc(&block_offs, n_blocks) && ws.alloc(&totals, 1);
+    if (ok && composite4) ok = ws.alloc(&pair_slot, (size_t)L);
+    for (int i = 0; ok && i < n_orders; ++i) ok = ws.alloc(&val[i], (size_t)L);
+    if (!ok) return TFE_ERR_CUDA;
+    MCU(cudaMemsetAsync(totals, 0, sizeof(MineTotals), stream));
+
+    // bigrams first when the 4-grams are keyed by them, even if order 2 itself is not asked for
+    std::vector<int> passes;
+    if (composite4 && orders[0] != 2 && !(n_orders > 1 && orders[1] == 2)) passes.push_back(-2);
+    for (int i = 0; i < n_orders; ++i) passes.push_back(i);
+    std::stable_sort(passes.begin(), passes.end(), [&](int a, int b) {
+        return (a < 0 ? 2 : orders[a]) < (b < 0 ? 2 : orders[b]);
+    });
+    for (int pass : passes) {
+        const int n = pass < 0 ? 2 : orders[pass];
+        const bool keep_pairs = composite4 && n == 2;
+        const int mode = (composite4 && n == 4) ? 1 : 0;
+        uint32_t *where = keep_pairs ? pair_slot : slot_of;
+        MCU(cudaMemsetAsync(table, 0xFF, slots * sizeof(MineSlot), stream));
+        tfe_mine_count_kernel<<<n_pos_blocks, kThreads, 0, stream>>>(tokens, (uint32_t)L, vocab, n, tok_bits, mode, pair_slot,
+                                                                    table, mask, where, totals);
+        MCU(cudaGetLastError());
+        if (pass < 0) continue;
+        MCU(cudaMemsetAsync(&totals->distinct, 0, sizeof(unsigned long long), stream));
+        tfe_mine_mark_kernel<<<n_pos_blocks, kThreads, 0, stream>>>(where, (uint32_t)L, table, std::max(min_count, 1u),
+                                                                   val[pass], totals);
+        MCU(cudaGetLastError());
+        unsigned long long d = 0;
+        MCU(cudaMemcpyAsync(&d, &totals->distinct, sizeof d, cudaMemcpyDeviceToHost, stream));
+        MCU(cudaStreamSynchronize(stream));
+        if (distinct) distinct[pass] = (int64_t)d;
+    }
+    MineVals mv{};
+    mv.n_orders = n_orders;
+    for (int i = 0; i < n_orders; ++i) { mv.val[i] = val[i]; mv.n[i] = orders[i]; }
+    tfe_mine_block_sums_kernel<<<n_blocks, kThreads, 0, stream>>>(mv, (uint32_t)L, block_sums);
+    tfe_mine_scan_kernel<<<1, 1024, 0, stream>>>(block_sums, n_blocks, block_offs, totals);
+    tfe_mine_emit_kernel<<<n_blocks, kThreads, 0, stream>>>(mv, tokens, (uint32_t)L, block_offs, (unsigned long long)cap,
+                                                          phrase_tokens, phrase_len, phrase_count);
+    MCU(cudaGetLastError());
+    MineTotals host_totals;
+    MCU(cudaMemcpyAsync(&host_totals, totals, sizeof host_totals, cudaMemcpyDeviceToHost, stream));
+    MCU(cudaStreamSynchronize(stream));
+#undef MCU
+    if (host_totals.error) return TFE_ERR_INTERNAL;
+    *n_found = (int64_t)host_totals.found;
+    if (hist) for (int i = 0; i < TFE_MINE_HIST_BINS; ++i) hist[i] = (int64_t)host_totals.hist[i];
+    return TFE_OK;
+}
+
+}  // extern "C"

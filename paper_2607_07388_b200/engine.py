@@ -182,3 +182,29 @@ class _DevicePointer:
 def _device_view(ptr: int, shape, typestr: str, device) -> torch.Tensor:
     """A tensor over library-owned device memory (no copy, no ownership)."""
     return torch.as_tensor(_DevicePointer(ptr, shape, typestr), device=device)
+
+
+class MinedPhrases:
+    """Result of mine_ngrams: device tensors cut to the entries written, plus the host-side totals."""
+
+    def __init__(self, tokens, length, count, n_found, distinct, hist):
+        self.phrase_tokens, self.phrase_len, self.count = tokens, length, count
+        self.n_found, self.distinct, self.hist = n_found, distinct, hist
+
+    def __len__(self):
+        return self.phrase_len.numel()
+
+
+def mine_ngrams(corpus: torch.Tensor, *, vocab: int, orders, min_count: int = 2, cap: int, want_hist: bool = True,
+                stream=None) -> MinedPhrases:
+    """Every n-gram of `corpus` (device int32 [L]) that occurs at least `min_count` times, in order of first
+    occurrence; `count` holds uint32 values in an int32 tensor.  The result feeds Engram(device_build=True)."""
+    assert corpus.is_cuda and corpus.dtype == torch.int32 and corpus.is_contiguous()
+    dev = corpus.device
+    pt = torch.empty((max(cap, 1), 4), dtype=torch.int32, device=dev)
+    pl = torch.empty(max(cap, 1), dtype=torch.uint8, device=dev)
+    pc = torch.empty(max(cap, 1), dtype=torch.int32, device=dev)
+    n_found, distinct, hist = tfe.tfe_mine_ngrams(corpus, corpus.numel(), vocab, orders, min_count, cap, pt, pl, pc,
+                                                  want_hist=want_hist, stream=stream)
+    n = min(n_found, cap)
+    return MinedPhrases(pt[:n], pl[:n], pc[:n], n_found, distinct, hist)

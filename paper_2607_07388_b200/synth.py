@@ -440,3 +440,37 @@ def head_hidden_np(B: int, d: int, variant: int = 0) -> np.ndarray:
 def head_hidden_torch(B: int, d: int, device, variant: int = 0):
     import torch
     return procedural_bf16_torch(torch.arange(B, device=device) + variant * 100_003, d, HEAD_H_TAG, HEAD_H_SHIFT)
+
+
+# ------------------------------------------------------------------ corpus for n-gram extraction
+
+
+def make_corpus(seed: int, L: int, vocab: int = VOCAB, *, s: float = 1.1, n_expr: int = 0, expr_rate: float = 0.3,
+                expr_s: float = 1.05, doc_len: int = 512, chunk: int = 1 << 24) -> np.ndarray:
+    """A tokenised corpus int32 [L] for the construction pipeline: Zipf-distributed ids (exponent ``s``, ranks
+    mapped through a seeded permutation of the whole vocabulary, so ids need all their bits), with
+    multi-token expressions (``n_expr`` of them, 2..4 ids each, Zipf-distributed popularity) written over
+    the filler at about ``expr_rate`` of the positions, cut into documents of geometric length (mean
+    ``doc_len``) by -1 separators.  Generated in chunks, reproducible for any chunk-independent prefix."""
+    rng = np.random.default_rng([seed, 424242])
+    perm = rng.permutation(vocab)
+    cdf = zipf_cdf(vocab, s)
+    n_expr = int(n_expr) if n_expr else max(16, L // 64)
+    expr_len = rng.integers(2, 5, size=n_expr)
+    expr_tok = zipf_tokens(rng, 4 * n_expr, cdf, perm).reshape(n_expr, 4)
+    ecdf = zipf_cdf(n_expr, expr_s)
+    out = np.empty(L, np.int32)
+    for lo in range(0, L, chunk):
+        n = min(chunk, L - lo)
+        crng = np.random.default_rng([seed, 424243, lo // chunk])
+        tok = zipf_tokens(crng, n, cdf, perm)
+        n_starts = int(n * expr_rate / 3)
+        starts = crng.integers(0, max(1, n - 4), size=n_starts)
+        which = np.minimum(np.searchsorted(ecdf, crng.random(n_starts), side="right"), n_expr - 1)
+        for j in range(4):
+            sel = expr_len[which] > j
+            tok[starts[sel] + j] = expr_tok[which[sel], j]
+        n_docs = max(1, n // max(2, doc_len))
+        tok[crng.integers(0, n, size=n_docs)] = -1
+        out[lo:lo + n] = tok
+    return out
