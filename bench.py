@@ -68,6 +68,9 @@ def parse_args():
                     help="time the other selection policies and gates (ALL, COSINE, a lambda that is not a bf16 number)")
     ap.add_argument("--build", action="store_true",
                     help="time index construction on the GPU (tfe_index_build_device) against the host build")
+    ap.add_argument("--mine", action="store_true", help="n-gram extraction with a frequency threshold over a synthetic corpus")
+    ap.add_argument("--mine-tokens", type=int, default=1 << 26)
+    ap.add_argument("--mine-min-count", type=int, default=3)
     ap.add_argument("--cache-policy", action="store_true",
                     help="time the retention bookkeeping in the lookup and tfe_cache_select_victims on the workload")
     ap.add_argument("--sweep", action="store_true", help="c5: tokens x row width x hit rate sweep")
@@ -414,6 +417,8 @@ def run_ours(a):
         return run_head(a, dev, rank)
     if a.build:
         return run_build(a, dev, rank)
+    if a.mine:
+        return run_mine(a, dev, rank)
     if a.variants:
         return run_variants(a, dev, rank)
 
@@ -892,6 +897,90 @@ def run_build(a, dev, rank):
                              "ms": host_s * 1e3},
             "parity": {"device_vs_host_build": bool(same), "device_build_vs_oracle": oracle_ok}}))
     eng.close(); host.close()
+
+
+def run_mine(a, dev, rank):
+    """Construction pipeline, first stage: every 2-, 3- and 4-gram of a corpus that occurs min_count times or more."""
+    import torch
+    from paper_2607_07388_b200 import binding as tfe
+    from paper_2607_07388_b200.engine import mine_ngrams
+    from oracle import tfe_oracle as orc
+    orc.build()
+    L, orders, m = a.mine_tokens, (2, 3, 4), a.mine_min_count
+    t0 = time.perf_counter()
+    corpus_np = synth.make_corpus(21, L)
+    gen_s = time.perf_counter() - t0
+    corpus = torch.from_numpy(corpus_np).to(dev)
+    first = mine_ngrams(corpus, vocab=synth.VOCAB, orders=orders, min_count=m, cap=0)          # warm-up; sizes the output
+    cap = first.n_found
+    reps = max(3, min(10, a.steps))
+    stream = torch.cuda.current_stream()
+    ws = torch.empty(tfe.tfe_mine_workspace_bytes(L, len(orders)), dtype=torch.uint8, device=dev)
+
+    def timed(workspace):
+        wall, evms = [], []
+        for _ in range(reps):
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0 = time.perf_counter()
+            e0.record(stream)
+            res = mine_ngrams(corpus, vocab=synth.VOCAB, orders=orders, min_count=m, cap=cap, want_hist=True, workspace=workspace)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            wall.append(time.perf_counter() - t0)
+            evms.append(e0.elapsed_time(e1))
+        return res, float(np.median(wall)), float(np.median(evms))
+
+    _, sec_alloc, _ = timed(None)
+    got, sec, ev_ms = timed(ws)
+    # parity 1: a prefix of the corpus, every output against the oracle
+    n_pre = min(L, 1 << 20)
+    t0 = time.perf_counter()
+    e_pt, e_pl, e_pc, e_found, e_distinct, e_hist = orc.mine_ngrams(corpus_np[:n_pre], synth.VOCAB, orders, min_count=m, cap=n_pre * 3)
+    cpu_s = time.perf_counter() - t0
+    pre = mine_ngrams(corpus[:n_pre].contiguous(), vocab=synth.VOCAB, orders=orders, min_count=m, cap=n_pre * 3)
+    prefix_ok = bool(pre.n_found == e_found and np.array_equal(pre.distinct, e_distinct) and np.array_equal(pre.hist, e_hist)
+                     and np.array_equal(pre.phrase_tokens.cpu().numpy(), e_pt) and np.array_equal(pre.phrase_len.cpu().numpy(), e_pl)
+                     and np.array_equal(pre.count.cpu().numpy().view(np.uint32), e_pc))
+    # parity 2, full size: sampled entries counted one by one by the oracle's scan; properties of the whole result
+    g_pt, g_pl, g_pc = got.phrase_tokens.cpu().numpy(), got.phrase_len.cpu().numpy(), got.count.cpu().numpy().view(np.uint32)
+    rng = np.random.default_rng(5)
+    sample = rng.choice(len(g_pl), size=min(24, len(g_pl)), replace=False) if len(g_pl) else []
+    sample_ok, prev_first = True, None
+    firsts = {}
+    for i in sorted(int(x) for x in sample):
+        n = int(g_pl[i])
+        c, f = orc.count_tuple(corpus_np, g_pt[i, :n])
+        sample_ok &= (c == int(g_pc[i])) and (g_pt[i, n:] == -1).all()
+        firsts[i] = (f, n)
+    keys = [firsts[i] for i in sorted(firsts)]
+    sample_ok &= keys == sorted(keys)                                        # entries are in (first, n) order
+    tail = np.cumsum(got.hist[::-1])[::-1]
+    props_ok = bool(got.n_found == cap == tail[m] and int(g_pc.min()) >= m and got.distinct.sum() == tail[1]
+                    and len(np.unique(np.concatenate([g_pt, g_pl[:, None].astype(np.int32)], axis=1), axis=0)) == len(g_pl))
+    slots = 1024
+    while slots < L + L // 2:
+        slots *= 2
+    per_order = slots * 16 + L * (4 + 64 + 4) + L * (4 + 32 + 4)      # table clear; count: ids, slot read-modify-write, slot index; mark
+    bytes_alg = len(orders) * per_order + 2 * len(orders) * 4 * L + cap * 21
+    peak, peak_src = measured_peak()
+    if rank == 0:
+        print(json.dumps({
+            "metric": "n-gram extraction tokens/s", "value": L / sec, "unit": "tokens/s", "ms_per_call": sec * 1e3,
+            "ms_per_call_device_events": ev_ms, "ms_per_call_allocating_its_workspace": sec_alloc * 1e3, "steps": reps,
+            "config": {"workload": f"corpus of {L} ids, vocabulary {synth.VOCAB}, orders 2-4, min_count {m}",
+                       "windows": int(3 * L), "distinct": [int(x) for x in got.distinct], "phrases_out": int(cap),
+                       "table_slots": slots, "workspace_bytes": tfe.tfe_mine_workspace_bytes(L, len(orders)),
+                       "corpus_generation_s": gen_s,
+                       "call": "tfe_mine_ngrams with the caller's workspace: 3 x (clear, count, mark), ordered compaction, synchronise (wall clock)"},
+            "roofline": {"bound": "hbm", "achieved": bytes_alg / sec / 1e9, "peak": peak, "unit": "GB/s",
+                         "frac": bytes_alg / sec / 1e9 / peak, "traffic": None, "peak_source": peak_src,
+                         "algorithmic_bytes_per_call": bytes_alg,
+                         "note": "random 32-byte sectors of the counting table dominate: 64 B per window in the count pass, 32 B in the mark pass"},
+            "cpu_baseline": {"value": n_pre / cpu_s, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+                             "sample": f"the first {n_pre} ids of the corpus (sort-based definition, single thread)"},
+            "parity": {"prefix_all_outputs": prefix_ok, "full_size_sampled_counts_and_order": bool(sample_ok),
+                       "full_size_properties": props_ok}}))
 
 
 def run_variants(a, dev, rank):

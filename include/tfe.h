@@ -431,17 +431,22 @@ tfe_status tfe_head_geometry(const tfe_head *head, int32_t *grid, int32_t *rows_
  *                  sum_{c >= m} hist[c] is n_found for min_count = m, so one call tells which threshold
  *                  yields a table of a wanted size.
  *
- * Allocates and frees its own workspace (tfe_mine_workspace_bytes; about 24..48 bytes per token for the
- * counting table plus 4 bytes per token and order), launches on `stream` and synchronises it.  Exact for
- * every vocabulary: orders whose ids do not fit one 64-bit key side by side are keyed through the exact
- * names of their halves.  Errors: TFE_ERR_INVALID_ARG, TFE_ERR_CUDA (workspace does not fit),
+ *   workspace      DEVICE scratch of workspace_bytes >= tfe_mine_workspace_bytes(L, n_orders) (about 24..48
+ *                  bytes per token for the counting table plus 4 bytes per token and order; smaller:
+ *                  TFE_ERR_CAPACITY), contents undefined before and after; or NULL with workspace_bytes = 0:
+ *                  the call allocates and frees it (several milliseconds per call at 10^8 tokens).
+ *
+ * Launches on `stream` and synchronises it.  Exact for every vocabulary: orders whose ids do not fit one
+ * 64-bit key side by side are keyed through the exact names of their halves.  Errors:
+ * TFE_ERR_INVALID_ARG, TFE_ERR_CAPACITY, TFE_ERR_CUDA (the workspace could not be allocated),
  * TFE_ERR_INTERNAL (a bounded probe ran out).
  */
 #define TFE_MINE_HIST_BINS 1024
 #define TFE_MINE_MAX_TOKENS (1ll << 30)
 tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int32_t n_orders, const int32_t *orders,
                            uint32_t min_count, int64_t cap, int32_t *phrase_tokens, uint8_t *phrase_len,
-                           uint32_t *phrase_count, int64_t *n_found, int64_t *distinct, int64_t *hist, void *stream);
+                           uint32_t *phrase_count, int64_t *n_found, int64_t *distinct, int64_t *hist,
+                           void *workspace, int64_t workspace_bytes, void *stream);
 int64_t tfe_mine_workspace_bytes(int64_t L, int32_t n_orders);   /* -1 for invalid arguments */
 
 #ifdef __cplusplus

@@ -751,3 +751,22 @@ int64_t orc_mine_ngrams(int64_t L, const int32_t *tokens, int32_t vocab, int32_t
     free(w);
     return n_keep;
 }
+
+/* orc_count_tuple: occurrences of ONE tuple of n ids in the corpus, by the definition above (a scan over
+ * all end positions); *first receives the smallest end position, -1 if there is none.  For spot checks
+ * on corpora that orc_mine_ngrams would take too long to sort. */
+int64_t orc_count_tuple(int64_t L, const int32_t *tokens, int32_t n, const int32_t *tuple, int64_t *first)
+{
+    int64_t count = 0;
+    *first = -1;
+    for (int64_t t = n - 1; t < L; ++t) {
+        int same = 1;
+        for (int32_t j = 0; j < n; ++j)
+            if (tokens[t - n + 1 + j] != tuple[j]) same = 0;
+        if (same) {
+            if (count == 0) *first = t;
+            ++count;
+        }
+    }
+    return count;
+}

@@ -290,3 +290,14 @@ def mine_ngrams(tokens, vocab, orders, min_count=1, cap=None, hist_bins=1024):
                 C.c_int32(hist_bins), _p(hist))
     n = int(min(n_found, cap))
     return pt[:n].copy(), pl[:n].copy(), pc[:n].copy(), int(n_found), distinct, hist
+
+
+def count_tuple(tokens, tup):
+    """(count, first end position or -1) of one tuple of valid ids in the corpus."""
+    tokens = _c(tokens, np.int32).reshape(-1)
+    tup = _c(tup, np.int32)
+    first = C.c_int64(-1)
+    f = lib().orc_count_tuple
+    f.restype = C.c_int64
+    n = f(C.c_int64(len(tokens)), _p(tokens), C.c_int32(len(tup)), _p(tup), C.byref(first))
+    return int(n), int(first.value)

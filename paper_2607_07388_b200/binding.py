@@ -108,7 +108,7 @@ def lib() -> C.CDLL:
         L.tfe_head_buffers.argtypes = [vp, C.POINTER(vp), C.POINTER(i64), C.POINTER(vp)]
         L.tfe_head_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         L.tfe_head_geometry.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
-        L.tfe_mine_ngrams.argtypes = [vp, i64, i32, i32, vp, C.c_uint32, i64, vp, vp, vp, C.POINTER(i64), vp, vp, vp]
+        L.tfe_mine_ngrams.argtypes = [vp, i64, i32, i32, vp, C.c_uint32, i64, vp, vp, vp, C.POINTER(i64), vp, vp, vp, i64, vp]
         L.tfe_mine_workspace_bytes.argtypes = [i64, i32]
         L.tfe_mine_workspace_bytes.restype = i64
         for name in ("tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tfe_cache_install_device", "tfe_lookup_inject", "tfe_lookup_inject_host",
@@ -391,7 +391,7 @@ def tfe_mine_workspace_bytes(L: int, n_orders: int) -> int:
 
 
 def tfe_mine_ngrams(tokens, L: int, vocab: int, orders, min_count: int, cap: int, phrase_tokens=None, phrase_len=None,
-                    phrase_count=None, want_hist: bool = True, stream=None):
+                    phrase_count=None, want_hist: bool = True, workspace=None, workspace_bytes: int = 0, stream=None):
     """tokens and the three outputs on the device; returns (n_found, distinct int64 [n_orders], hist int64 [1024] or None)."""
     o = np.ascontiguousarray(orders, np.int32)
     found = C.c_int64(0)
@@ -399,5 +399,6 @@ def tfe_mine_ngrams(tokens, L: int, vocab: int, orders, min_count: int, cap: int
     hist = np.zeros(MINE_HIST_BINS, np.int64) if want_hist else None
     _check(lib().tfe_mine_ngrams(_addr(tokens), int(L), int(vocab), len(o), _addr(o), int(min_count), int(cap),
                                  _addr(phrase_tokens), _addr(phrase_len), _addr(phrase_count), C.byref(found),
-                                 _addr(distinct), _addr(hist), _stream(stream)), "tfe_mine_ngrams")
+                                 _addr(distinct), _addr(hist), _addr(workspace), int(workspace_bytes), _stream(stream)),
+           "tfe_mine_ngrams")
     return found.value, distinct, hist

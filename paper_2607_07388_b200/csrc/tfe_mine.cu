@@ -47,7 +47,7 @@ struct MineSlot { unsigned long long key; uint32_t count_m1; uint32_t first; }; 
 static_assert(sizeof(MineSlot) == 16, "slot layout");
 
 struct MineTotals {
-    unsigned long long distinct;       // tuples of the order being marked
+    unsigned long long distinct[4];    // tuples per configured order
     unsigned long long found;          // written by the scan: entries that qualify, all orders
     uint32_t error;                    // a probe ran the whole table without finding a place
     uint32_t pad;
@@ -67,7 +67,7 @@ __device__ __forceinline__ uint64_t mix64(uint64_t x)
 __global__ void __launch_bounds__(kThreads)
 tfe_mine_count_kernel(const int32_t *__restrict__ tokens, uint32_t L, int32_t vocab, int n, int tok_bits, int mode,
                       const uint32_t *__restrict__ pair_slot, MineSlot *table, uint32_t mask,
-                      uint32_t *__restrict__ slot_of, MineTotals *totals)
+                      uint32_t *__restrict__ all_slots, uint32_t *__restrict__ cand_slot, MineTotals *totals)
 {
     const uint32_t t = blockIdx.x * (uint32_t)kThreads + threadIdx.x;
     const int lane = threadIdx.x & 31;
@@ -87,33 +87,46 @@ tfe_mine_count_kernel(const int32_t *__restrict__ tokens, uint32_t L, int32_t vo
         }
     }
     uint32_t slot = kNoSlot;
+    bool may_be_first = false;                             // only such positions are looked at by the mark pass
     const unsigned act = __ballot_sync(0xFFFFFFFFu, valid);
     if (valid) {
         const unsigned grp = __match_any_sync(act, key);
         const int leader = __ffs(grp) - 1;                 // lowest lane: the smallest t of the group
         if (lane == leader) {
             uint32_t s = (uint32_t)mix64(key) & mask;
+            uint32_t seen_first = 0xFFFFFFFFu;
             for (uint32_t probes = 0; probes <= mask; ++probes, s = (s + 1) & mask) {
-                unsigned long long k = *reinterpret_cast<volatile unsigned long long *>(&table[s].key);
-                if (k == kEmpty) k = atomicCAS(&table[s].key, kEmpty, key);
+                // one 16-byte look at the slot: the key and, if it is ours already, the first position so far
+                const uint4 raw = __ldcv(reinterpret_cast<const uint4 *>(table + s));
+                unsigned long long k = ((unsigned long long)raw.y << 32) | raw.x;
+                seen_first = raw.w;
+                // (a key whose low word is all ones could be imitated by a half-written slot: ask again, atomically)
+                if (k == kEmpty || (k == key && raw.x == 0xFFFFFFFFu)) {
+                    k = atomicCAS(&table[s].key, kEmpty, key);
+                    seen_first = 0xFFFFFFFFu;
+                }
                 if (k == kEmpty || k == key) { slot = s; break; }
             }
             if (slot != kNoSlot) {
                 atomicAdd(&table[slot].count_m1, (uint32_t)__popc(grp));
-                atomicMin(&table[slot].first, t);
+                // `first` only ever decreases: a value already below t needs no update, and t cannot be the first
+                if (seen_first > t) { atomicMin(&table[slot].first, t); may_be_first = true; }
             } else {
                 atomicExch(&totals->error, 1u);
             }
         }
         slot = __shfl_sync(grp, slot, leader);
     }
-    if (t < L) slot_of[t] = slot;
+    if (t < L) {
+        if (all_slots) all_slots[t] = slot;
+        if (cand_slot) cand_slot[t] = may_be_first ? slot : kNoSlot;
+    }
 }
 
 // val[t] = count of the tuple ending at t if t is its first occurrence and count >= min_count, else 0.
 __global__ void __launch_bounds__(kThreads)
 tfe_mine_mark_kernel(const uint32_t *__restrict__ slot_of, uint32_t L, const MineSlot *__restrict__ table,
-                     uint32_t min_count, uint32_t *__restrict__ val, MineTotals *totals)
+                     uint32_t min_count, uint32_t *__restrict__ val, MineTotals *totals, int order_index)
 {
     __shared__ uint32_t s_hist[TFE_MINE_HIST_BINS];
     __shared__ uint32_t s_distinct;
@@ -138,7 +151,7 @@ tfe_mine_mark_kernel(const uint32_t *__restrict__ slot_of, uint32_t L, const Min
     __syncthreads();
     for (int i = threadIdx.x; i < TFE_MINE_HIST_BINS; i += kThreads)
         if (s_hist[i]) atomicAdd(&totals->hist[i], (unsigned long long)s_hist[i]);
-    if (threadIdx.x == 0 && s_distinct) atomicAdd(&totals->distinct, (unsigned long long)s_distinct);
+    if (threadIdx.x == 0 && s_distinct) atomicAdd(&totals->distinct[order_index], (unsigned long long)s_distinct);
 }
 
 struct MineVals { const uint32_t *val[4]; int n[4]; int n_orders; };
@@ -268,18 +281,28 @@ uint64_t table_slots_for(int64_t L)
     return cap;
 }
 
-struct Workspace {
-    std::vector<void *> ptrs;
-    ~Workspace() { for (void *p : ptrs) cudaFree(p); }
-    template <class T> bool alloc(T **p, size_t n)
+// Carves the arrays out of one buffer (the caller's, or one allocated here and freed on return).
+struct Carver {
+    char *base = nullptr, *cur = nullptr, *end = nullptr;
+    void *owned = nullptr;
+    ~Carver() { if (owned) cudaFree(owned); }
+    template <class T> T *take(size_t n)
     {
-        void *q = nullptr;
-        if (cudaMalloc(&q, std::max<size_t>(n, 1) * sizeof(T)) != cudaSuccess) { (void)cudaGetLastError(); return false; }
-        ptrs.push_back(q);
-        *p = static_cast<T *>(q);
-        return true;
+        const size_t bytes = (std::max<size_t>(n, 1) * sizeof(T) + 255) & ~(size_t)255;
+        if (cur + bytes > end) return nullptr;
+        T *p = reinterpret_cast<T *>(cur);
+        cur += bytes;
+        return p;
     }
 };
+
+int64_t workspace_bytes_for(int64_t L, int32_t n_orders)
+{
+    const int64_t n_blocks = (L + kPosPerBlock - 1) / kPosPerBlock;
+    const int64_t pad = 256;
+    return (int64_t)table_slots_for(L) * (int64_t)sizeof(MineSlot) + pad + (int64_t)(n_orders + 2) * (L * 4 + pad)
+           + n_blocks * 12 + 2 * pad + (int64_t)sizeof(MineTotals) + pad + 256;
+}
 
 }  // namespace
 
@@ -287,15 +310,14 @@ extern "C" {
 
 int64_t tfe_mine_workspace_bytes(int64_t L, int32_t n_orders)
 {
-    if (L < 0 || n_orders < 1 || n_orders > 4) return -1;
-    const int64_t n_blocks = (L + kPosPerBlock - 1) / kPosPerBlock;
-    return (int64_t)table_slots_for(L) * (int64_t)sizeof(MineSlot) + (int64_t)(n_orders + 2) * L * 4 + n_blocks * 12
-           + (int64_t)sizeof(MineTotals);
+    if (L < 0 || L > TFE_MINE_MAX_TOKENS || n_orders < 1 || n_orders > 4) return -1;
+    return workspace_bytes_for(L, n_orders);
 }
 
 tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int32_t n_orders, const int32_t *orders,
                            uint32_t min_count, int64_t cap, int32_t *phrase_tokens, uint8_t *phrase_len,
-                           uint32_t *phrase_count, int64_t *n_found, int64_t *distinct, int64_t *hist, void *stream_)
+                           uint32_t *phrase_count, int64_t *n_found, int64_t *distinct, int64_t *hist,
+                           void *workspace, int64_t workspace_bytes, void *stream_)
 {
     if (L < 0 || L > TFE_MINE_MAX_TOKENS || vocab < 1 || n_orders < 1 || n_orders > 4 || !orders || cap < 0 || !n_found)
         return TFE_ERR_INVALID_ARG;
@@ -304,6 +326,8 @@ tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int3
     if (L > 0 && !tokens) return TFE_ERR_INVALID_ARG;
     if (cap > 0 && (!phrase_tokens || !phrase_len || !phrase_count)) return TFE_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(phrase_tokens) & 15u) != 0) return TFE_ERR_INVALID_ARG;
+    if (workspace_bytes < 0 || (workspace_bytes > 0 && !workspace)) return TFE_ERR_INVALID_ARG;
+    if (workspace && workspace_bytes < workspace_bytes_for(L, n_orders)) return TFE_ERR_CAPACITY;
     *n_found = 0;
     if (distinct) for (int i = 0; i < n_orders; ++i) distinct[i] = 0;
     if (hist) for (int i = 0; i < TFE_MINE_HIST_BINS; ++i) hist[i] = 0;
@@ -318,16 +342,27 @@ tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int3
     const uint32_t n_pos_blocks = (uint32_t)((L + kThreads - 1) / kThreads);
     const uint32_t n_blocks = (uint32_t)((L + kPosPerBlock - 1) / kPosPerBlock);
 
-    Workspace ws;
-    MineSlot *table = nullptr;
-    uint32_t *slot_of = nullptr, *pair_slot = nullptr, *block_sums = nullptr, *val[4] = {nullptr, nullptr, nullptr, nullptr};
-    unsigned long long *block_offs = nullptr;
-    MineTotals *totals = nullptr;
-    bool ok = ws.alloc(&table, slots) && ws.alloc(&slot_of, (size_t)L) && ws.alloc(&block_sums, n_blocks)
-              && ws.alloc(&block_offs, n_blocks) && ws.alloc(&totals, 1);
-    if (ok && composite4) ok = ws.alloc(&pair_slot, (size_t)L);
-    for (int i = 0; ok && i < n_orders; ++i) ok = ws.alloc(&val[i], (size_t)L);
-    if (!ok) return TFE_ERR_CUDA;
+    Carver ws;
+    if (workspace) {
+        ws.base = reinterpret_cast<char *>((reinterpret_cast<uintptr_t>(workspace) + 255) & ~(uintptr_t)255);
+        ws.end = static_cast<char *>(workspace) + workspace_bytes;
+    } else {
+        const int64_t bytes = workspace_bytes_for(L, n_orders);
+        MCU(cudaMalloc(&ws.owned, (size_t)bytes));
+        ws.base = static_cast<char *>(ws.owned);
+        ws.end = ws.base + bytes;
+    }
+    ws.cur = ws.base;
+    MineSlot *table = ws.take<MineSlot>(slots);
+    uint32_t *cand_slot = ws.take<uint32_t>((size_t)L);
+    uint32_t *pair_slot = composite4 ? ws.take<uint32_t>((size_t)L) : nullptr;
+    uint32_t *block_sums = ws.take<uint32_t>(n_blocks);
+    unsigned long long *block_offs = ws.take<unsigned long long>(n_blocks);
+    MineTotals *totals = ws.take<MineTotals>(1);
+    uint32_t *val[4] = {nullptr, nullptr, nullptr, nullptr};
+    bool ok = table && cand_slot && (pair_slot || !composite4) && block_sums && block_offs && totals;
+    for (int i = 0; ok && i < n_orders; ++i) ok = (val[i] = ws.take<uint32_t>((size_t)L)) != nullptr;
+    if (!ok) return TFE_ERR_INTERNAL;
     MCU(cudaMemsetAsync(totals, 0, sizeof(MineTotals), stream));
 
     // bigrams first when the 4-grams are keyed by them, even if order 2 itself is not asked for
@@ -341,20 +376,15 @@ tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int3
         const int n = pass < 0 ? 2 : orders[pass];
         const bool keep_pairs = composite4 && n == 2;
         const int mode = (composite4 && n == 4) ? 1 : 0;
-        uint32_t *where = keep_pairs ? pair_slot : slot_of;
         MCU(cudaMemsetAsync(table, 0xFF, slots * sizeof(MineSlot), stream));
         tfe_mine_count_kernel<<<n_pos_blocks, kThreads, 0, stream>>>(tokens, (uint32_t)L, vocab, n, tok_bits, mode, pair_slot,
-                                                                    table, mask, where, totals);
+                                                                    table, mask, keep_pairs ? pair_slot : nullptr,
+                                                                    pass < 0 ? nullptr : cand_slot, totals);
         MCU(cudaGetLastError());
         if (pass < 0) continue;
-        MCU(cudaMemsetAsync(&totals->distinct, 0, sizeof(unsigned long long), stream));
-        tfe_mine_mark_kernel<<<n_pos_blocks, kThreads, 0, stream>>>(where, (uint32_t)L, table, std::max(min_count, 1u),
-                                                                   val[pass], totals);
+        tfe_mine_mark_kernel<<<n_pos_blocks, kThreads, 0, stream>>>(cand_slot, (uint32_t)L, table, std::max(min_count, 1u),
+                                                                   val[pass], totals, pass);
         MCU(cudaGetLastError());
-        unsigned long long d = 0;
-        MCU(cudaMemcpyAsync(&d, &totals->distinct, sizeof d, cudaMemcpyDeviceToHost, stream));
-        MCU(cudaStreamSynchronize(stream));
-        if (distinct) distinct[pass] = (int64_t)d;
     }
     MineVals mv{};
     mv.n_orders = n_orders;
@@ -370,6 +400,7 @@ tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int3
 #undef MCU
     if (host_totals.error) return TFE_ERR_INTERNAL;
     *n_found = (int64_t)host_totals.found;
+    if (distinct) for (int i = 0; i < n_orders; ++i) distinct[i] = (int64_t)host_totals.distinct[i];
     if (hist) for (int i = 0; i < TFE_MINE_HIST_BINS; ++i) hist[i] = (int64_t)host_totals.hist[i];
     return TFE_OK;
 }

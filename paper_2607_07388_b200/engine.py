@@ -196,15 +196,19 @@ class MinedPhrases:
 
 
 def mine_ngrams(corpus: torch.Tensor, *, vocab: int, orders, min_count: int = 2, cap: int, want_hist: bool = True,
-                stream=None) -> MinedPhrases:
+                workspace: torch.Tensor | None = None, stream=None) -> MinedPhrases:
     """Every n-gram of `corpus` (device int32 [L]) that occurs at least `min_count` times, in order of first
-    occurrence; `count` holds uint32 values in an int32 tensor.  The result feeds Engram(device_build=True)."""
+    occurrence; `count` holds uint32 values in an int32 tensor.  The result feeds Engram(device_build=True).
+    `workspace`: a device uint8 tensor of tfe_mine_workspace_bytes(L, n_orders) bytes kept by the caller across
+    calls (None: the library allocates and frees its own)."""
     assert corpus.is_cuda and corpus.dtype == torch.int32 and corpus.is_contiguous()
     dev = corpus.device
     pt = torch.empty((max(cap, 1), 4), dtype=torch.int32, device=dev)
     pl = torch.empty(max(cap, 1), dtype=torch.uint8, device=dev)
     pc = torch.empty(max(cap, 1), dtype=torch.int32, device=dev)
     n_found, distinct, hist = tfe.tfe_mine_ngrams(corpus, corpus.numel(), vocab, orders, min_count, cap, pt, pl, pc,
-                                                  want_hist=want_hist, stream=stream)
+                                                  want_hist=want_hist, workspace=workspace,
+                                                  workspace_bytes=0 if workspace is None else workspace.numel(),
+                                                  stream=stream)
     n = min(n_found, cap)
     return MinedPhrases(pt[:n], pl[:n], pc[:n], n_found, distinct, hist)

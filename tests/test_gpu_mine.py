@@ -131,3 +131,25 @@ def test_mine_workspace_and_argument_checks():
         tfe.tfe_mine_ngrams(tok, 16, 0, (2,), 1, 0)
     with pytest.raises(tfe.TfeError):
         tfe.tfe_mine_ngrams(tok, 16, 10, (2,), 1, 4)             # cap > 0 without output arrays
+    small = torch.empty(1000, dtype=torch.uint8, device=DEV)
+    with pytest.raises(tfe.TfeError) as e:
+        tfe.tfe_mine_ngrams(tok, 16, 10, (2,), 1, 0, workspace=small, workspace_bytes=small.numel())
+    assert e.value.status == tfe.TFE_ERR_CAPACITY
+
+
+def test_mine_with_callers_workspace(orc):
+    """The same results from a workspace the caller keeps (left dirty between calls, and deliberately misaligned)."""
+    from paper_2607_07388_b200 import binding as tfe
+    from paper_2607_07388_b200.engine import mine_ngrams
+    L = 50_000
+    buf = torch.full((tfe.tfe_mine_workspace_bytes(L, 3) + 1,), 0x5A, dtype=torch.uint8, device=DEV)
+    for seed in range(3):
+        tok = synth.make_corpus(30 + seed, L)
+        e_pt, e_pl, e_pc, e_found, e_distinct, e_hist = orc.mine_ngrams(tok, synth.VOCAB, (2, 3, 4), min_count=2, cap=L)
+        got = mine_ngrams(torch.from_numpy(tok).to(DEV), vocab=synth.VOCAB, orders=(2, 3, 4), min_count=2, cap=L,
+                          workspace=buf[1:])
+        assert got.n_found == e_found
+        np.testing.assert_array_equal(got.distinct, e_distinct)
+        np.testing.assert_array_equal(got.hist, e_hist)
+        np.testing.assert_array_equal(got.phrase_tokens.cpu().numpy(), e_pt)
+        np.testing.assert_array_equal(got.count.cpu().numpy().view(np.uint32), e_pc)

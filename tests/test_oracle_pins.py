@@ -877,3 +877,19 @@ def test_mine_ngrams_against_library_unique(oracle_mod, seed):
         tup, c = expect[key]
         assert pl[i] == key[1] and pc[i] == c
         assert tuple(pt[i, :key[1]].tolist()) == tup and (pt[i, key[1]:] == -1).all()
+
+
+def test_count_tuple_by_hand_and_against_the_extraction(oracle_mod):
+    tok = np.array([5, 7, 5, 7, 9, -1, 5, 7], np.int32)
+    assert oracle_mod.count_tuple(tok, (5, 7)) == (3, 1)
+    assert oracle_mod.count_tuple(tok, (7, 9)) == (1, 4)
+    assert oracle_mod.count_tuple(tok, (9, 5)) == (0, -1)
+    assert oracle_mod.count_tuple(tok, (5, 7, 9)) == (1, 4)
+    rng = np.random.default_rng(17)
+    tok = rng.integers(0, 6, size=4000).astype(np.int32)
+    pt, pl, pc, n_found, _, _ = oracle_mod.mine_ngrams(tok, 6, (2, 3, 4))
+    for i in rng.choice(n_found, size=40, replace=False):
+        n = int(pl[i])
+        win = np.lib.stride_tricks.sliding_window_view(tok, n)
+        hits = np.flatnonzero((win == pt[i, :n]).all(axis=1))
+        assert oracle_mod.count_tuple(tok, pt[i, :n]) == (len(hits), int(hits[0]) + n - 1) == (int(pc[i]), int(hits[0]) + n - 1)
