@@ -9,13 +9,14 @@
 //
 // No sort: counting is a hash-table pass, the order comes from the corpus itself.
 //
-//   tfe_mine_count_kernel   one thread per end position.  The window's exact 64-bit key (ids packed side
+//   tfe_mine_count_kernel   two end positions per thread.  The window's exact 64-bit key (ids packed side
 //                           by side; an order too wide for 64 bits is keyed by the table slots of its two
 //                           halves, which are exact names of those bigrams) is inserted into an
 //                           open-addressing table of 16-byte slots {key, count, first} by a 64-bit
-//                           compare-and-swap on the key; equal keys inside a warp are combined first
-//                           (match.any), then one atomicAdd on the count and one atomicMin on the first
-//                           end position.  The slot index is remembered per position.
+//                           compare-and-swap on the key; equal keys are combined first inside a warp
+//                           (match.any) and inside the block (shared-memory table), then one atomicAdd on
+//                           the count and, only where it can lower it, one atomicMin on the first end
+//                           position.  The slot index is remembered for the positions that may be first.
 //   tfe_mine_mark_kernel    one thread per end position: the position that IS the first occurrence of its
 //                           tuple speaks for the tuple -- counts it as distinct, adds it to the histogram of
 //                           counts and, if the count reaches the threshold, leaves the count in the
@@ -62,64 +63,144 @@ __device__ __forceinline__ uint64_t mix64(uint64_t x)
     return x;
 }
 
+// Whole-slot compare-and-swap: {key, count - 1, first} <- put if the slot is still all ones; returns what was there.
+__device__ __forceinline__ uint4 cas_empty_slot(MineSlot *slot, unsigned long long key, uint32_t count_m1, uint32_t first)
+{
+    unsigned long long old_lo, old_hi;
+    const unsigned long long put_hi = ((unsigned long long)first << 32) | count_m1;
+    asm volatile(
+        "{\n\t.reg .b128 o, n, c;\n\t"
+        "mov.b128 c, {%2, %3};\n\t"
+        "mov.b128 n, {%4, %5};\n\t"
+        "atom.global.cas.b128 o, [%6], c, n;\n\t"
+        "mov.b128 {%0, %1}, o;\n\t}"
+        : "=l"(old_lo), "=l"(old_hi)
+        : "l"(kEmpty), "l"(kEmpty), "l"(key), "l"(put_hi), "l"(slot)
+        : "memory");
+    return make_uint4((uint32_t)old_lo, (uint32_t)(old_lo >> 32), (uint32_t)old_hi, (uint32_t)(old_hi >> 32));
+}
+
 // mode 0: ids packed side by side (n * tok_bits <= 63).  mode 1 (n = 4 only): the slots of the bigrams
 // ending at t - 2 and at t in the bigram table of this corpus, 31 bits each.
+//
+// A block takes kCountSpan consecutive end positions.  Equal keys are combined first inside a warp
+// (match.any) and then inside the block, in a small shared-memory table {key, count, smallest t}: a frequent
+// tuple then costs the global table one update per block instead of one per warp, which is what the hot
+// slots of a Zipf-distributed corpus need.  Every distinct key of the block is then looked up / inserted in the
+// global table once (the first probes of a thread's entries are issued together), and the positions read
+// their slot back from shared memory.
+constexpr int kCountWin = 2;                               // end positions per thread
+constexpr int kCountSpan = kThreads * kCountWin;           // end positions per block
+constexpr int kCountEntries = 2 * kCountSpan;              // shared-memory entries: at most half full
+constexpr int kEntriesPerThread = kCountEntries / kThreads;
+
 __global__ void __launch_bounds__(kThreads)
 tfe_mine_count_kernel(const int32_t *__restrict__ tokens, uint32_t L, int32_t vocab, int n, int tok_bits, int mode,
                       const uint32_t *__restrict__ pair_slot, MineSlot *table, uint32_t mask,
                       uint32_t *__restrict__ all_slots, uint32_t *__restrict__ cand_slot, MineTotals *totals)
 {
-    const uint32_t t = blockIdx.x * (uint32_t)kThreads + threadIdx.x;
+    __shared__ unsigned long long s_key[kCountEntries];
+    __shared__ uint32_t s_cnt[kCountEntries];              // occurrences in this block; afterwards: 1 if s_min may be the first
+    __shared__ uint32_t s_min[kCountEntries];              // smallest end position in this block
+    __shared__ uint32_t s_slot[kCountEntries];             // slot in the global table
+    for (int e = threadIdx.x; e < kCountEntries; e += kThreads) { s_key[e] = kEmpty; s_cnt[e] = 0; s_min[e] = 0xFFFFFFFFu; }
+    __syncthreads();
+
     const int lane = threadIdx.x & 31;
-    bool valid = t < L && t + 1 >= (uint32_t)n;
-    unsigned long long key = 0;
-    if (valid) {
-        if (mode == 0) {
-            for (int j = 0; j < n; ++j) {
-                const int32_t x = __ldg(tokens + t - (n - 1) + j);
-                if ((uint32_t)x >= (uint32_t)vocab) valid = false;
-                key = (key << tok_bits) | (uint32_t)x;
-            }
-        } else {
-            const uint32_t a = __ldg(pair_slot + t - 2), b = __ldg(pair_slot + t);
-            valid = a != kNoSlot && b != kNoSlot;
-            key = ((unsigned long long)a << 31) | b;
-        }
-    }
-    uint32_t slot = kNoSlot;
-    bool may_be_first = false;                             // only such positions are looked at by the mark pass
-    const unsigned act = __ballot_sync(0xFFFFFFFFu, valid);
-    if (valid) {
-        const unsigned grp = __match_any_sync(act, key);
-        const int leader = __ffs(grp) - 1;                 // lowest lane: the smallest t of the group
-        if (lane == leader) {
-            uint32_t s = (uint32_t)mix64(key) & mask;
-            uint32_t seen_first = 0xFFFFFFFFu;
-            for (uint32_t probes = 0; probes <= mask; ++probes, s = (s + 1) & mask) {
-                // one 16-byte look at the slot: the key and, if it is ours already, the first position so far
-                const uint4 raw = __ldcv(reinterpret_cast<const uint4 *>(table + s));
-                unsigned long long k = ((unsigned long long)raw.y << 32) | raw.x;
-                seen_first = raw.w;
-                // (a key whose low word is all ones could be imitated by a half-written slot: ask again, atomically)
-                if (k == kEmpty || (k == key && raw.x == 0xFFFFFFFFu)) {
-                    k = atomicCAS(&table[s].key, kEmpty, key);
-                    seen_first = 0xFFFFFFFFu;
+    const uint32_t base = blockIdx.x * (uint32_t)kCountSpan;
+    int entry[kCountWin];
+#pragma unroll
+    for (int w = 0; w < kCountWin; ++w) {
+        const uint32_t t = base + w * kThreads + threadIdx.x;
+        bool valid = t < L && t + 1 >= (uint32_t)n;
+        unsigned long long key = 0;
+        if (valid) {
+            if (mode == 0) {
+                for (int j = 0; j < n; ++j) {
+                    const int32_t x = __ldg(tokens + t - (n - 1) + j);
+                    if ((uint32_t)x >= (uint32_t)vocab) valid = false;
+                    key = (key << tok_bits) | (uint32_t)x;
                 }
-                if (k == kEmpty || k == key) { slot = s; break; }
-            }
-            if (slot != kNoSlot) {
-                atomicAdd(&table[slot].count_m1, (uint32_t)__popc(grp));
-                // `first` only ever decreases: a value already below t needs no update, and t cannot be the first
-                if (seen_first > t) { atomicMin(&table[slot].first, t); may_be_first = true; }
             } else {
-                atomicExch(&totals->error, 1u);
+                const uint32_t a = __ldg(pair_slot + t - 2), b = __ldg(pair_slot + t);
+                valid = a != kNoSlot && b != kNoSlot;
+                key = ((unsigned long long)a << 31) | b;
             }
         }
-        slot = __shfl_sync(grp, slot, leader);
+        entry[w] = -1;
+        const unsigned act = __ballot_sync(0xFFFFFFFFu, valid);
+        if (valid) {
+            const unsigned grp = __match_any_sync(act, key);
+            const int leader = __ffs(grp) - 1;             // lowest lane: the smallest t of the group
+            int e = -1;
+            if (lane == leader) {
+                e = (int)((mix64(key) >> 40) & (kCountEntries - 1));
+                for (int probes = 0; probes < kCountEntries; ++probes, e = (e + 1) & (kCountEntries - 1)) {
+                    const unsigned long long k = atomicCAS(&s_key[e], kEmpty, key);
+                    if (k == kEmpty || k == key) break;
+                }
+                atomicAdd(&s_cnt[e], (uint32_t)__popc(grp));
+                atomicMin(&s_min[e], t);
+            }
+            entry[w] = __shfl_sync(grp, e, leader);
+        }
     }
-    if (t < L) {
+    __syncthreads();
+
+    // every distinct key of the block, once, against the global table
+    unsigned long long keys[kEntriesPerThread];
+    uint32_t start[kEntriesPerThread];
+    uint4 raw0[kEntriesPerThread];
+#pragma unroll
+    for (int i = 0; i < kEntriesPerThread; ++i) {
+        keys[i] = s_key[threadIdx.x + i * kThreads];
+        start[i] = (uint32_t)mix64(keys[i]) & mask;
+        if (keys[i] != kEmpty) raw0[i] = __ldcv(reinterpret_cast<const uint4 *>(table + start[i]));
+    }
+#pragma unroll
+    for (int i = 0; i < kEntriesPerThread; ++i) {
+        if (keys[i] == kEmpty) continue;
+        const int e = threadIdx.x + i * kThreads;
+        const unsigned long long key = keys[i];
+        const uint32_t t = s_min[e];
+        uint32_t slot = kNoSlot, s = start[i];
+        uint4 raw = raw0[i];
+        bool may_be_first = false;                         // only such positions are looked at by the mark pass
+        for (uint32_t probes = 0; probes <= mask; ++probes) {
+            // one 16-byte look at the slot: the key and, if it is ours already, the first position so far
+            unsigned long long k = ((unsigned long long)raw.y << 32) | raw.x;
+            // an empty slot takes the whole entry in one 16-byte compare-and-swap; if another block was
+            // faster, the swap returns that block's entry.  (A key whose low word is all ones could be
+            // imitated by a half-written slot: the swap then only serves to read the slot atomically.)
+            if (k == kEmpty || (k == key && raw.x == 0xFFFFFFFFu)) {
+                raw = cas_empty_slot(table + s, key, s_cnt[e] - 1u, t);
+                k = ((unsigned long long)raw.y << 32) | raw.x;
+                if (k == kEmpty) { slot = s; may_be_first = true; break; }
+            }
+            if (k == key) {
+                slot = s;
+                atomicAdd(&table[s].count_m1, s_cnt[e]);
+                // `first` only ever decreases: a value already below t needs no update, and t cannot be the first
+                if (raw.w > t) { atomicMin(&table[s].first, t); may_be_first = true; }
+                break;
+            }
+            s = (s + 1) & mask;
+            raw = __ldcv(reinterpret_cast<const uint4 *>(table + s));
+        }
+        if (slot == kNoSlot) atomicExch(&totals->error, 1u);
+        s_slot[e] = slot;
+        s_cnt[e] = may_be_first ? 1u : 0u;
+    }
+    __syncthreads();
+
+#pragma unroll
+    for (int w = 0; w < kCountWin; ++w) {
+        const uint32_t t = base + w * kThreads + threadIdx.x;
+        if (t >= L) continue;
+        const int e = entry[w];
+        const uint32_t slot = e >= 0 ? s_slot[e] : kNoSlot;
         if (all_slots) all_slots[t] = slot;
-        if (cand_slot) cand_slot[t] = may_be_first ? slot : kNoSlot;
+        if (cand_slot) cand_slot[t] = (e >= 0 && s_cnt[e] != 0u && s_min[e] == t) ? slot : kNoSlot;
     }
 }
 
@@ -341,6 +422,7 @@ tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int3
     const uint32_t mask = (uint32_t)(slots - 1);
     const uint32_t n_pos_blocks = (uint32_t)((L + kThreads - 1) / kThreads);
     const uint32_t n_blocks = (uint32_t)((L + kPosPerBlock - 1) / kPosPerBlock);
+    const uint32_t n_count_blocks = (uint32_t)((L + kCountSpan - 1) / kCountSpan);
 
     Carver ws;
     if (workspace) {
@@ -377,7 +459,7 @@ tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int3
         const bool keep_pairs = composite4 && n == 2;
         const int mode = (composite4 && n == 4) ? 1 : 0;
         MCU(cudaMemsetAsync(table, 0xFF, slots * sizeof(MineSlot), stream));
-        tfe_mine_count_kernel<<<n_pos_blocks, kThreads, 0, stream>>>(tokens, (uint32_t)L, vocab, n, tok_bits, mode, pair_slot,
+        tfe_mine_count_kernel<<<n_count_blocks, kThreads, 0, stream>>>(tokens, (uint32_t)L, vocab, n, tok_bits, mode, pair_slot,
                                                                     table, mask, keep_pairs ? pair_slot : nullptr,
                                                                     pass < 0 ? nullptr : cand_slot, totals);
         MCU(cudaGetLastError());
