@@ -161,3 +161,24 @@ def test_new_entry_points_refuse_bad_arguments_on_the_host(tfe):
     cfg = tfe.make_config(d=16, vocab=10, orders=(2, 3), n_phrases=2, gpu_slots=2)
     assert L.tfe_index_build_device(C.byref(cfg), None, 0x1000, 0x1000, 0x1000, None, C.byref(out)) == tfe.TFE_ERR_INVALID_ARG
     assert L.tfe_index_build_device(C.byref(cfg), 0x1004, 0x1000, 0x1000, 0x1000, None, C.byref(out)) == tfe.TFE_ERR_INVALID_ARG
+    # device-side installation
+    assert L.tfe_cache_install_device(None, 4, 0x1000, 0x1000, 0x1000, None, None, None) == tfe.TFE_ERR_INVALID_ARG
+    # n-gram extraction: every refusal below happens before the first device call
+    found = C.c_int64(7)
+    orders = np.array([2, 3], np.int32)
+    bad = np.array([3, 2], np.int32)
+    mine = lambda tok, Ln, vocab, n_o, o, cap, pt_, ws, wsb: L.tfe_mine_ngrams(
+        tok, Ln, vocab, n_o, o, 1, cap, pt_, 0x1000, 0x1000, C.byref(found), None, None, ws, wsb, None)
+    assert mine(0x1000, -1, 10, 2, orders.ctypes.data, 0, None, None, 0) == tfe.TFE_ERR_INVALID_ARG
+    assert mine(0x1000, (1 << 30) + 1, 10, 2, orders.ctypes.data, 0, None, None, 0) == tfe.TFE_ERR_INVALID_ARG
+    assert mine(0x1000, 16, 0, 2, orders.ctypes.data, 0, None, None, 0) == tfe.TFE_ERR_INVALID_ARG
+    assert mine(0x1000, 16, 10, 2, bad.ctypes.data, 0, None, None, 0) == tfe.TFE_ERR_INVALID_ARG
+    assert mine(0x1000, 16, 10, 5, orders.ctypes.data, 0, None, None, 0) == tfe.TFE_ERR_INVALID_ARG
+    assert mine(None, 16, 10, 2, orders.ctypes.data, 0, None, None, 0) == tfe.TFE_ERR_INVALID_ARG
+    assert mine(0x1000, 16, 10, 2, orders.ctypes.data, 4, None, None, 0) == tfe.TFE_ERR_INVALID_ARG         # cap without outputs
+    assert mine(0x1000, 16, 10, 2, orders.ctypes.data, 4, 0x1004, None, 0) == tfe.TFE_ERR_INVALID_ARG       # misaligned tuples
+    assert mine(0x1000, 16, 10, 2, orders.ctypes.data, 0, None, None, 64) == tfe.TFE_ERR_INVALID_ARG        # size without buffer
+    assert mine(0x1000, 16, 10, 2, orders.ctypes.data, 0, None, 0x1000, 64) == tfe.TFE_ERR_CAPACITY         # workspace too small
+    assert mine(None, 0, 10, 2, orders.ctypes.data, 0, None, None, 0) == tfe.TFE_OK and found.value == 0   # empty corpus: no device call
+    assert L.tfe_mine_workspace_bytes(-1, 2) == -1 and L.tfe_mine_workspace_bytes(16, 0) == -1
+    assert L.tfe_mine_workspace_bytes(1 << 20, 3) >= (1 << 21) * 16 + 5 * 4 * (1 << 20)
