@@ -32,6 +32,20 @@ bool cuda_failed(cudaError_t e, const char *what)
         if (cuda_failed((call), #call)) return TFE_ERR_CUDA;           \
     } while (0)
 
+// Launch with programmatic stream serialisation: the launch is set up while the kernel before it on the
+// stream drains.  Only for kernels that call tfe_grid_dependency_sync() before their first global access.
+template <class... KArgs, class... Args>
+cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 0; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 constexpr uint32_t kNoOwner = 0xFFFFFFFFu;
 constexpr int kDefaultMaxKicks = 2000;
 constexpr int kVarSlots = 16;
@@ -705,11 +719,10 @@ tfe_status tfe_cache_install_device(tfe_ctx *c, int32_t n, const uint32_t *phras
     p.slot_stats = c->d_slot_stats; p.epoch = c->d_epoch;
     CU(cudaMemsetAsync(p.count, 0, sizeof(uint32_t), stream));
     const unsigned blocks = (unsigned)((n + 255) / 256);
-    tfe_install_claim_kernel<0><<<blocks, 256, 0, stream>>>(p);
-    tfe_install_claim_kernel<1><<<blocks, 256, 0, stream>>>(p);
-    tfe_install_device_kernel<<<(unsigned)((n + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK), TFE_BLOCK_THREADS, 0,
-                                stream>>>(p);
-    CU(cudaGetLastError());
+    CU(launch_overlapped(tfe_install_claim_kernel<0>, dim3(blocks), dim3(256), stream, p));
+    CU(launch_overlapped(tfe_install_claim_kernel<1>, dim3(blocks), dim3(256), stream, p));
+    CU(launch_overlapped(tfe_install_device_kernel, dim3((unsigned)((n + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK)),
+                         dim3(TFE_BLOCK_THREADS), stream, p));
     c->mirror_ready = false;        // the host copy of the residency state is stale now; fetched again when needed
     return TFE_OK;
 }
@@ -1029,17 +1042,17 @@ tfe_status tfe_cache_select_victims(tfe_ctx *c, int32_t n, int32_t half_life, in
     const unsigned grid = (unsigned)std::max<int64_t>(
         1, std::min<int64_t>((int64_t)c->sm_count * 4, (C + 4 * TFE_VICTIM_THREADS - 1) / (4 * TFE_VICTIM_THREADS)));
     static const int kShift[6] = {53, 42, 31, 20, 9, 0}, kBits[6] = {11, 11, 11, 11, 11, 9};
-    tfe_victim_pass_kernel<true><<<grid, TFE_VICTIM_THREADS, 0, stream>>>(c->d_slot_stats, c->d_slot_owner, c->d_epoch, half_life,
-                                                            c->d_slot_key, (uint32_t)C, (uint32_t)take, kShift[0],
-                                                            kBits[0], c->d_vs_hist, c->d_vs_state);
+    CU(launch_overlapped(tfe_victim_pass_kernel<true>, dim3(grid), dim3(TFE_VICTIM_THREADS), stream, c->d_slot_stats,
+                         c->d_slot_owner, c->d_epoch, half_life, c->d_slot_key, (uint32_t)C, (uint32_t)take, kShift[0],
+                         kBits[0], c->d_vs_hist, c->d_vs_state));
     for (int i = 1; i < 6; ++i)
-        tfe_victim_pass_kernel<false><<<grid, TFE_VICTIM_THREADS, 0, stream>>>(c->d_slot_stats, c->d_slot_owner, c->d_epoch, half_life,
-                                                                 c->d_slot_key, (uint32_t)C, 0u, kShift[i], kBits[i],
-                                                                 c->d_vs_hist, c->d_vs_state);
-    tfe_victim_collect_kernel<<<grid, TFE_VICTIM_THREADS, 0, stream>>>(c->d_slot_key, (uint32_t)C, c->d_vs_state, c->d_vs_list,
-                                                        TFE_VICTIMS_MAX);
-    tfe_victim_sort_kernel<<<1, 1024, 0, stream>>>(c->d_vs_list, c->d_vs_state, (uint32_t)take, c->d_vs_slots,
-                                                   c->d_vs_keys);
+        CU(launch_overlapped(tfe_victim_pass_kernel<false>, dim3(grid), dim3(TFE_VICTIM_THREADS), stream, c->d_slot_stats,
+                             c->d_slot_owner, c->d_epoch, half_life, c->d_slot_key, (uint32_t)C, 0u, kShift[i], kBits[i],
+                             c->d_vs_hist, c->d_vs_state));
+    CU(launch_overlapped(tfe_victim_collect_kernel, dim3(grid), dim3(TFE_VICTIM_THREADS), stream, c->d_slot_key, (uint32_t)C,
+                         c->d_vs_state, c->d_vs_list, (uint32_t)TFE_VICTIMS_MAX));
+    CU(launch_overlapped(tfe_victim_sort_kernel, dim3(1), dim3(1024), stream, c->d_vs_list, c->d_vs_state, (uint32_t)take,
+                         c->d_vs_slots, c->d_vs_keys));
     CU(cudaGetLastError());
     if (!slots) return TFE_OK;      // results stay on the device (tfe_cache_select_victims_device); no synchronisation
     CU(cudaMemcpyAsync(slots, c->d_vs_slots, (size_t)take * 4, cudaMemcpyDeviceToHost, stream));
@@ -1112,12 +1125,10 @@ tfe_status tfe_prefetch_candidates(tfe_ctx *c, const int32_t *history, int32_t B
     p.tok_bits = c->tok_bits; p.vocab = c->cfg.vocab;
     p.benefit_host = prm->benefit_host; p.benefit_ssd = prm->benefit_ssd;
     p.keys = c->d_pf_keys; p.entry_phrase = c->d_pf_phrase; p.entry_tier = c->d_pf_tier; p.counter = c->d_pf_counter;
-    tfe_prefetch_probe_kernel<<<(unsigned)((E + 255) / 256), 256, 0, stream>>>(p);
-    CU(cudaGetLastError());
-    tfe_prefetch_select_kernel<<<1, 1024, 0, stream>>>(c->d_pf_keys, c->d_pf_phrase, c->d_pf_tier, c->d_pf_counter,
-                                                       (uint32_t)prm->budget, p.div_orders, (uint32_t)c->cfg.n_orders,
-                                                       out_phrase, out_tier, out_score, out_src, out_count);
-    CU(cudaGetLastError());
+    CU(launch_overlapped(tfe_prefetch_probe_kernel, dim3((unsigned)((E + 255) / 256)), dim3(256), stream, p));
+    CU(launch_overlapped(tfe_prefetch_select_kernel, dim3(1), dim3(1024), stream, c->d_pf_keys, c->d_pf_phrase, c->d_pf_tier,
+                         c->d_pf_counter, (uint32_t)prm->budget, p.div_orders, (uint32_t)c->cfg.n_orders, out_phrase,
+                         out_tier, out_score, out_src, out_count));
     return TFE_OK;
 }
 

@@ -898,6 +898,7 @@ template <int STAGE>
 __global__ void __launch_bounds__(256)
 tfe_install_claim_kernel(const TfeInstallDeviceParams p)
 {
+    tfe_grid_dependency_sync();
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= p.n) return;
     const uint32_t stamp = p.tag | (uint32_t)(TFE_INSTALL_DEVICE_MAX - 1 - k);
@@ -912,6 +913,7 @@ tfe_install_claim_kernel(const TfeInstallDeviceParams p)
 __global__ void __launch_bounds__(TFE_BLOCK_THREADS)
 tfe_install_device_kernel(const TfeInstallDeviceParams p)
 {
+    tfe_grid_dependency_sync();
     const int lane = threadIdx.x & 31;
     const int k = blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5);
     if (k >= p.n) return;
@@ -977,6 +979,7 @@ struct TfePrefetchParams {
 
 __global__ void __launch_bounds__(256) tfe_prefetch_probe_kernel(const TfePrefetchParams p)
 {
+    tfe_grid_dependency_sync();
     const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;
     const int lane = threadIdx.x & 31;
     unsigned long long key64 = 0;
@@ -1050,6 +1053,7 @@ tfe_prefetch_select_kernel(const unsigned long long *keys, const uint32_t *entry
     __shared__ uint32_t s_fill;
     __shared__ unsigned long long s_prefix;
     __shared__ uint32_t s_want;
+    tfe_grid_dependency_sync();
     const uint32_t n = *(volatile uint32_t *)counter;
     const uint32_t take = min(n, budget);
     // ---- threshold: the take-th largest key, by most-significant-digit-first radix selection
@@ -1172,6 +1176,7 @@ tfe_victim_pass_kernel(const uint2 *slot_stats, const uint32_t *slot_owner, cons
     __shared__ uint32_t s_last;
     for (int i = threadIdx.x; i < TFE_VICTIM_BINS; i += blockDim.x) s_hist[i] = 0;
     __syncthreads();
+    tfe_grid_dependency_sync();                 // the pass before this one decides the prefix
     const unsigned long long prefix = FIRST ? 0ull : state->prefix;
     const uint32_t now = FIRST ? *epoch : 0u;
     const int above = shift + bits;             // bits above this digit are decided
@@ -1271,6 +1276,7 @@ __global__ void __launch_bounds__(TFE_VICTIM_THREADS)
 tfe_victim_collect_kernel(const uint32_t *slot_key, uint32_t C, TfeVictimState *state, unsigned long long *list,
                           uint32_t cap)
 {
+    tfe_grid_dependency_sync();
     const unsigned long long limit = state->prefix;
     const uint32_t n_quads = (C + 3u) >> 2;
     for (uint32_t g = blockIdx.x * blockDim.x + threadIdx.x; g < n_quads; g += gridDim.x * blockDim.x) {
@@ -1295,6 +1301,7 @@ tfe_victim_sort_kernel(const unsigned long long *list, TfeVictimState *state, ui
     __shared__ unsigned long long s_v[TFE_VICTIMS_MAX];
     uint32_t pow2 = 1;
     while (pow2 < n) pow2 <<= 1;
+    tfe_grid_dependency_sync();
     for (uint32_t i = threadIdx.x; i < pow2; i += blockDim.x) s_v[i] = i < n ? list[i] : ~0ull;
     __syncthreads();
     for (uint32_t k = 2; k <= pow2; k <<= 1)
