@@ -1294,31 +1294,66 @@ tfe_victim_collect_kernel(const uint32_t *slot_key, uint32_t C, TfeVictimState *
     }
 }
 
+// One block sorts the selected composites (at most TFE_VICTIMS_MAX = 4,096) ascending: a bitonic network
+// with four consecutive elements per thread.  Compare-exchange distances 1 and 2 stay inside a thread,
+// distances 4..64 are warp shuffles, only distances >= 128 go through shared memory (15 of the 78 steps at
+// 4,096 elements).
 __global__ void __launch_bounds__(1024)
 tfe_victim_sort_kernel(const unsigned long long *list, TfeVictimState *state, uint32_t n, int32_t *out_slots,
                        uint32_t *out_keys)
 {
+    static_assert(TFE_VICTIMS_MAX == 4 * 1024, "four elements per thread of a 1,024-thread block");
     __shared__ unsigned long long s_v[TFE_VICTIMS_MAX];
     uint32_t pow2 = 1;
     while (pow2 < n) pow2 <<= 1;
     tfe_grid_dependency_sync();
-    for (uint32_t i = threadIdx.x; i < pow2; i += blockDim.x) s_v[i] = i < n ? list[i] : ~0ull;
-    __syncthreads();
-    for (uint32_t k = 2; k <= pow2; k <<= 1)
-        for (uint32_t j = k >> 1; j > 0; j >>= 1) {
-            for (uint32_t t = threadIdx.x; t < pow2 / 2; t += blockDim.x) {
-                const uint32_t i = ((t & ~(j - 1)) << 1) | (t & (j - 1));      // the pair's lower index
-                const uint32_t l = i | j;
-                const unsigned long long a = s_v[i], b = s_v[l];
-                const bool up = (i & k) == 0;
-                if ((a > b) == up) { s_v[i] = b; s_v[l] = a; }
-            }
+    const uint32_t base = 4u * threadIdx.x;
+    unsigned long long v[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) v[e] = base + e < n ? list[base + e] : ~0ull;      // padding sorts to the end
+    for (uint32_t k = 2; k <= pow2; k <<= 1) {
+        uint32_t j = k >> 1;
+        if (j >= 128) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) s_v[base + e] = v[e];
             __syncthreads();
+            for (; j >= 128; j >>= 1) {
+                for (uint32_t t = threadIdx.x; t < TFE_VICTIMS_MAX / 2; t += blockDim.x) {
+                    const uint32_t i = ((t & ~(j - 1)) << 1) | (t & (j - 1));      // the pair's lower index
+                    const uint32_t l = i | j;
+                    const unsigned long long a = s_v[i], b = s_v[l];
+                    const bool up = (i & k) == 0;
+                    if ((a > b) == up) { s_v[i] = b; s_v[l] = a; }
+                }
+                __syncthreads();
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) v[e] = s_v[base + e];
         }
-    for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) {
-        out_slots[i] = (int32_t)(uint32_t)s_v[i];
-        out_keys[i] = (uint32_t)(s_v[i] >> 32);
+        for (; j >= 4; j >>= 1) {                   // partner element in another lane of this warp
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, v[e], (int)(j >> 2));
+                const uint32_t i = base + e;
+                const bool up = (i & k) == 0, lower = (i & j) == 0;
+                v[e] = (lower == up) ? (other < v[e] ? other : v[e]) : (other > v[e] ? other : v[e]);
+            }
+        }
+        // partner element in this thread: distance 2 (from k = 4 on), then distance 1
+        auto exchange = [&](unsigned long long &a, unsigned long long &b, uint32_t i) {
+            const bool up = (i & k) == 0;
+            if ((a > b) == up) { const unsigned long long t = a; a = b; b = t; }
+        };
+        if (k >= 4) { exchange(v[0], v[2], base); exchange(v[1], v[3], base + 1); }
+        exchange(v[0], v[1], base);
+        exchange(v[2], v[3], base + 2);
     }
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+        if (base + e < n) {
+            out_slots[base + e] = (int32_t)(uint32_t)v[e];
+            out_keys[base + e] = (uint32_t)(v[e] >> 32);
+        }
     if (threadIdx.x == 0) state->n_out = 0;      // re-armed for the next selection
 }
 

@@ -82,3 +82,34 @@ def test_prefetch_loop_turns_predicted_misses_into_hits():
     assert hits_with > hits_without + B, (hits_with, hits_without)
     head.close()
     pr.close()
+
+
+def test_launch_overlap_respects_the_producer_on_the_stream():
+    """The lookup is launched so that its set-up overlaps the kernel before it on the stream; it must still see
+    everything that kernel wrote.  Producer -> lookup -> lookup chains with no host synchronisation in between:
+    hidden states and ids written by torch kernels immediately before, and a lookup in place on the output of
+    the previous one (the residual stream through two injection layers)."""
+    import parity_harness as H
+    w = synth.config(1, B=8, T=256, n_phrases=30_000, gpu_slots=30_000, d=512, p=0.5)
+    tb, pr = H.pair_from_workload(w)
+    rng = np.random.default_rng(77)
+    for rep in range(20):
+        tok = synth.make_queries(w, tb, variant=rep)
+        h_np = synth.gaussian_bf16([77, rep], (w.Q, w.d), 1.0)
+        # producers: ids arrive shifted and are fixed up on the device; h is the sum of two halves
+        tok_shift = torch.from_numpy(tok + 5).to(H.DEV)
+        h_full = H.bf16_tensor_from_bits(h_np, H.DEV)
+        half = (h_full.float() * 0.5).to(torch.bfloat16)                      # exact: a power of two
+        big = torch.empty(1 << 22, device=H.DEV)                              # keeps the stream busy before the producers
+        torch.cuda.synchronize()
+        big.normal_()
+        tok_dev = tok_shift - 5                                               # producer kernel 1
+        h_dev = half + half                                                   # producer kernel 2, directly before the lookup
+        out1 = pr.eng.lookup_inject(tok_dev, h_dev, lam=1.0).out              # layer 1, out of place
+        out2 = pr.eng.lookup_inject(tok_dev, out1, out1, lam=0.5).out         # layer 2, in place on layer 1's output
+        torch.cuda.synchronize()
+        ref = pr.ora.lookup(tok)
+        _, r1 = pr.ora.inject(ref, h_np, lam=1.0)
+        _, r2 = pr.ora.inject(ref, r1, lam=0.5)
+        np.testing.assert_array_equal(H.bits_from_bf16_tensor(out2), r2)
+    pr.close()
