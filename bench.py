@@ -718,7 +718,9 @@ def run_cache_policy(a, dev, rank):
     sel_ms, _ = timed_region(select, reps, 3, stream, 1, None, dev)
     us = sel_ms / reps * 1e3
     peak, peak_src = measured_peak()
-    bytes_alg = w.gpu_slots * 40 + n_vic * 24
+    # per slot: {freq, last} 8 + owner 4 read and key 4 written (first pass), the key re-read by two more digit
+    # passes, the tie count and the collect (4 x 4)
+    bytes_alg = w.gpu_slots * 32 + n_vic * 24
 
     # the device-side loop: selection left on the device, then installation of a batch that lives on the
     # device into those slots; every call a fresh batch of phrases that are not resident
@@ -766,7 +768,7 @@ def run_cache_policy(a, dev, rank):
             "metric": "victim selection slots/s", "value": w.gpu_slots / (us * 1e-6), "unit": "slots/s",
             "us_per_call": us, "steps": reps,
             "config": {"workload": w.name, "gpu_slots": w.gpu_slots, "n_victims": n_vic, "half_life": half_life,
-                       "call": "tfe_cache_select_victims: 8 launches + copy of the slots to the host + synchronise"},
+                       "call": "tfe_cache_select_victims: 6 launches + copy of the slots to the host + synchronise"},
             "roofline": {"bound": "hbm", "achieved": bytes_alg / us / 1e3, "peak": peak, "unit": "GB/s",
                          "frac": bytes_alg / us / 1e3 / peak, "traffic": None, "peak_source": peak_src,
                          "algorithmic_bytes_per_call": bytes_alg},

@@ -288,7 +288,7 @@ tfe_status tfe_cache_policy_enable(tfe_ctx *ctx, void *stream);
  *
  *   n        0..4096;  slots HOST int32 [n], or NULL;  keys HOST uint32 [n] or NULL;
  *   count    HOST: entries written = min(n, gpu_slots).
- * Eight kernel launches on `stream`; with host `slots` the results are copied there and the
+ * Six kernel launches on `stream`; with host `slots` the results are copied there and the
  * stream is synchronised (they feed tfe_cache_install, which takes host arrays); with slots =
  * NULL nothing is copied and nothing synchronises.  tfe_cache_select_victims_device returns the
  * DEVICE copies of the most recent selection (owned by the context, valid until the next one;

@@ -1041,14 +1041,18 @@ tfe_status tfe_cache_select_victims(tfe_ctx *c, int32_t n, int32_t half_life, in
     CU(cudaMemsetAsync(c->d_vs_state, 0, sizeof(TfeVictimState), stream));
     const unsigned grid = (unsigned)std::max<int64_t>(
         1, std::min<int64_t>((int64_t)c->sm_count * 4, (C + 4 * TFE_VICTIM_THREADS - 1) / (4 * TFE_VICTIM_THREADS)));
-    static const int kShift[6] = {53, 42, 31, 20, 9, 0}, kBits[6] = {11, 11, 11, 11, 11, 9};
+    static const int kShift[3] = {53, 42, 32}, kBits[3] = {11, 11, 10};      // the key's 32 bits
     CU(launch_overlapped(tfe_victim_pass_kernel<true>, dim3(grid), dim3(TFE_VICTIM_THREADS), stream, c->d_slot_stats,
                          c->d_slot_owner, c->d_epoch, half_life, c->d_slot_key, (uint32_t)C, (uint32_t)take, kShift[0],
                          kBits[0], c->d_vs_hist, c->d_vs_state));
-    for (int i = 1; i < 6; ++i)
+    for (int i = 1; i < 3; ++i)
         CU(launch_overlapped(tfe_victim_pass_kernel<false>, dim3(grid), dim3(TFE_VICTIM_THREADS), stream, c->d_slot_stats,
                              c->d_slot_owner, c->d_epoch, half_life, c->d_slot_key, (uint32_t)C, 0u, kShift[i], kBits[i],
                              c->d_vs_hist, c->d_vs_state));
+    static_assert(TFE_VICTIM_BINS >= 4 * 256, "the histogram array doubles as one counter per block");
+    if (grid > TFE_VICTIM_BINS) return TFE_ERR_INTERNAL;
+    CU(launch_overlapped(tfe_victim_tie_kernel, dim3(grid), dim3(TFE_VICTIM_THREADS), stream, c->d_slot_key, (uint32_t)C,
+                         c->d_vs_hist, c->d_vs_state));
     CU(launch_overlapped(tfe_victim_collect_kernel, dim3(grid), dim3(TFE_VICTIM_THREADS), stream, c->d_slot_key, (uint32_t)C,
                          c->d_vs_state, c->d_vs_list, (uint32_t)TFE_VICTIMS_MAX));
     CU(launch_overlapped(tfe_victim_sort_kernel, dim3(1), dim3(1024), stream, c->d_vs_list, c->d_vs_state, (uint32_t)take,

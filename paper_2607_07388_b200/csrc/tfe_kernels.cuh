@@ -1137,10 +1137,12 @@ tfe_prefetch_select_kernel(const unsigned long long *keys, const uint32_t *entry
 // and the victims are the n slots of smallest (key, slot).  (key << 32 | slot) is a distinct
 // 64-bit number per slot, so this is a selection of the n smallest of C distinct numbers:
 //
-//   tfe_victim_pass_kernel   x6, most significant digit first (11,11,11,11,11,9 bits): histogram of
-//                            the digit over the slots that agree with the digits chosen so far; the
-//                            block that finishes last picks the digit holding the n-th smallest
+//   tfe_victim_pass_kernel   x3 over the key's 32 bits, most significant digit first (11,11,10 bits):
+//                            histogram of the digit over the slots that agree with the digits chosen so
+//                            far; the block that finishes last picks the digit holding the n-th smallest
 //                            and re-arms the histogram.  The first pass computes and stores the keys.
+//   tfe_victim_tie_kernel    the slot half of the n-th smallest: a count of the slots that hold exactly
+//                            its key, in slot (= memory) order, instead of three more digit passes
 //   tfe_victim_collect_kernel  appends every number <= the n-th smallest to a list (any order)
 //   tfe_victim_sort_kernel     one block: bitonic sort of the list, writes slots and keys
 #define TFE_VICTIMS_MAX 4096
@@ -1270,6 +1272,102 @@ tfe_victim_pass_kernel(const uint2 *slot_stats, const uint32_t *slot_owner, cons
         state->k_rem = k;
         state->ticket = 0;
     }
+}
+
+// After the three passes over the key's 32 bits the wanted number is known to be the k_rem-th smallest
+// SLOT among those holding exactly that key.  Slot order is memory order, so no further digit passes are
+// needed: every block counts the ties of one contiguous range of slots; the block that finishes last
+// scans the per-block counts, finds the range that holds the k_rem-th tie, walks that range once more and
+// completes state->prefix with the slot.  `tie_count` is the (zeroed) histogram array, left zeroed again.
+__global__ void __launch_bounds__(TFE_VICTIM_THREADS)
+tfe_victim_tie_kernel(const uint32_t *slot_key, uint32_t C, uint32_t *tie_count, TfeVictimState *state)
+{
+    __shared__ uint32_t s_warp[TFE_VICTIM_THREADS / 32];
+    __shared__ uint32_t s_last, s_block, s_rank;
+    tfe_grid_dependency_sync();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned long long prefix = state->prefix;
+    const uint32_t key_star = (uint32_t)(prefix >> 32);
+    const uint32_t n_quads = (C + 3u) >> 2;
+    const uint32_t per_block = (n_quads + gridDim.x - 1) / gridDim.x;
+    auto ties_of = [&](uint32_t g) -> uint32_t {            // slots of quad g that hold the key
+        const uint4 k4 = __ldcg(reinterpret_cast<const uint4 *>(slot_key) + g);
+        return (uint32_t)(k4.x == key_star && 4 * g < C) + (uint32_t)(k4.y == key_star && 4 * g + 1 < C) +
+               (uint32_t)(k4.z == key_star && 4 * g + 2 < C) + (uint32_t)(k4.w == key_star && 4 * g + 3 < C);
+    };
+    {
+        const uint32_t q0 = min(n_quads, blockIdx.x * per_block), q1 = min(n_quads, q0 + per_block);
+        uint32_t mine = 0;
+        for (uint32_t g = q0 + threadIdx.x; g < q1; g += blockDim.x) mine += ties_of(g);
+        mine = __reduce_add_sync(0xFFFFFFFFu, mine);
+        if (lane == 0) s_warp[warp] = mine;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t total = 0;
+            for (int w = 0; w < TFE_VICTIM_THREADS / 32; ++w) total += s_warp[w];
+            tie_count[blockIdx.x] = total;
+            __threadfence();
+            s_last = atomicAdd(&state->ticket, 1u) == gridDim.x - 1;
+        }
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+    }
+    // ---- last block: which range holds the k_rem-th tie
+    if (warp == 0) {
+        const uint32_t want = state->k_rem;
+        uint32_t running = 0;
+        bool found = false;
+        for (uint32_t base = 0; base < gridDim.x; base += 32) {
+            const uint32_t i = base + lane;
+            const uint32_t c = i < gridDim.x ? __ldcg(tie_count + i) : 0u;
+            if (i < gridDim.x) tie_count[i] = 0;
+            uint32_t incl = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            const uint32_t reach = __ballot_sync(0xFFFFFFFFu, running + incl >= want);
+            if (!found && reach != 0u) {
+                found = true;
+                if (lane == __ffs(reach) - 1) { s_block = i; s_rank = want - (running + incl - c); }
+            }
+            running += __shfl_sync(0xFFFFFFFFu, incl, 31);
+        }
+        if (!found && lane == 0) { s_block = 0; s_rank = 0; }       // cannot happen: k_rem <= number of ties
+    }
+    __syncthreads();
+    // ---- walk that range: a contiguous piece per thread, counts, scan, then the piece that holds the tie
+    const uint32_t q0 = min(n_quads, s_block * per_block), q1 = min(n_quads, q0 + per_block);
+    const uint32_t per_thread = (q1 - q0 + blockDim.x - 1) / blockDim.x;
+    const uint32_t t0 = min(q1, q0 + threadIdx.x * per_thread), t1 = min(q1, t0 + per_thread);
+    uint32_t mine = 0;
+    for (uint32_t g = t0; g < t1; ++g) mine += ties_of(g);
+    uint32_t incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    __syncthreads();
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    uint32_t before = incl - mine;
+    for (int w = 0; w < warp; ++w) before += s_warp[w];
+    const uint32_t want = s_rank;
+    if (want > before && want <= before + mine) {          // exactly one thread
+        uint32_t left = want - before;
+        for (uint32_t g = t0; g < t1 && left; ++g) {
+            const uint4 k4 = __ldcg(reinterpret_cast<const uint4 *>(slot_key) + g);
+            const uint32_t key[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (left && key[j] == key_star && 4 * g + j < C && --left == 0)
+                    state->prefix = (prefix & 0xFFFFFFFF00000000ull) | (4 * g + j);
+        }
+    }
+    if (threadIdx.x == 0) state->ticket = 0;
 }
 
 __global__ void __launch_bounds__(TFE_VICTIM_THREADS)
