@@ -149,9 +149,12 @@ tfe_status tfe_cache_install(tfe_ctx *ctx, int32_t n, const uint32_t *phrase_ids
  *   dst_slots      DEVICE int32 [n]
  *   applied        DEVICE uint8 [n], receives 1 / 0 per entry, or NULL
  *   applied_count  DEVICE uint32, receives the number applied, or NULL
- * Asynchronous on `stream`, three kernel launches, never synchronises; the first call allocates
- * 4 bytes per phrase and per slot.  The host-side residency copy that tfe_cache_install checks
- * against is refreshed (one synchronisation) on that function's next call.
+ * Asynchronous on `stream`, four kernel launches, never synchronises.  The first call on a context
+ * allocates 4 bytes per phrase and per slot (with a device synchronisation: make it outside a stream
+ * capture); every later call keeps no state on the host and may be captured into a CUDA graph and
+ * replayed with new contents in the same buffers.  Once this function has been used, the host-side
+ * residency copy that tfe_cache_install checks against is re-read from the device (one
+ * synchronisation) on every call of that function.
  * Errors: INVALID_ARG, CUDA.
  */
 tfe_status tfe_cache_install_device(tfe_ctx *ctx, int32_t n, const uint32_t *phrase_ids,

@@ -106,10 +106,11 @@ struct tfe_ctx {
     int32_t *d_vs_slots = nullptr;
 
     bool mirror_ready = true;               // h_slot / h_owner filled (a device build fills them on first use)
+    bool device_installs = false;           // tfe_cache_install_device was used: replays of a captured call change the
+                                            // residency without the host seeing it, so the mirror is never trusted again
 
     // tfe_cache_install_device: stamps per phrase and per slot, the call counter, the applied count
     uint32_t *d_phrase_stamp = nullptr, *d_slot_stamp = nullptr, *d_inst_count = nullptr;
-    uint32_t inst_call_no = 0;
 
     // host-buffer variant staging
     int32_t *d_h_tokens = nullptr;
@@ -608,7 +609,7 @@ tfe_status fetch_mirror(tfe_ctx *c, cudaStream_t stream)
         CU(cudaMemcpyAsync(c->h_owner.data(), c->d_slot_owner, (size_t)C * 4, cudaMemcpyDeviceToHost, stream));
         CU(cudaStreamSynchronize(stream));
     }
-    c->mirror_ready = true;
+    c->mirror_ready = !c->device_installs;
     return TFE_OK;
 }
 
@@ -700,21 +701,16 @@ tfe_status tfe_cache_install_device(tfe_ctx *c, int32_t n, const uint32_t *phras
         CU(cudaMalloc(&c->d_phrase_stamp, std::max<size_t>(4, (size_t)N * 4)));
         CU(cudaMalloc(&c->d_slot_stamp, std::max<size_t>(4, (size_t)C * 4)));
         CU(cudaMalloc(&c->d_inst_count, sizeof(uint32_t)));
-        c->inst_call_no = 0;
-    }
-    if (c->inst_call_no == 0 || c->inst_call_no >= (1u << 20) - 1) {     // fresh stamps (also when the counter wraps)
+        // zero once; every call leaves them zeroed again
         CU(cudaMemsetAsync(c->d_phrase_stamp, 0, std::max<size_t>(4, (size_t)N * 4), stream));
         CU(cudaMemsetAsync(c->d_slot_stamp, 0, std::max<size_t>(4, (size_t)C * 4), stream));
-        c->inst_call_no = 0;
     }
-    ++c->inst_call_no;
     TfeInstallDeviceParams p{};
     p.index = c->d_index; p.phrase_pos = c->d_phrase_pos; p.slot_owner = c->d_slot_owner;
     p.rows = c->gpu_rows; p.row_vecs = c->row_vecs; p.n = n;
     p.n_phrases = (uint32_t)N; p.gpu_slots = C;
     p.ids = phrase_ids; p.src = static_cast<const uint4 *>(src_rows); p.dst_slots = dst_slots;
     p.phrase_stamp = c->d_phrase_stamp; p.slot_stamp = c->d_slot_stamp;
-    p.tag = c->inst_call_no << 12;
     p.applied = applied; p.count = applied_count ? applied_count : c->d_inst_count;
     p.slot_stats = c->d_slot_stats; p.epoch = c->d_epoch;
     CU(cudaMemsetAsync(p.count, 0, sizeof(uint32_t), stream));
@@ -723,7 +719,9 @@ tfe_status tfe_cache_install_device(tfe_ctx *c, int32_t n, const uint32_t *phras
     CU(launch_overlapped(tfe_install_claim_kernel<1>, dim3(blocks), dim3(256), stream, p));
     CU(launch_overlapped(tfe_install_device_kernel, dim3((unsigned)((n + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK)),
                          dim3(TFE_BLOCK_THREADS), stream, p));
+    CU(launch_overlapped(tfe_install_clear_kernel, dim3(blocks), dim3(256), stream, p));
     c->mirror_ready = false;        // the host copy of the residency state is stale now; fetched again when needed
+    c->device_installs = true;
     return TFE_OK;
 }
 

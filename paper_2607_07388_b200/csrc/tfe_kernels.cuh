@@ -855,13 +855,14 @@ tfe_install_kernel(ulonglong2 *index, const uint32_t *phrase_pos, uint32_t *slot
 // skipped.  Judged against the state before the call, entry k is a candidate if its id is a
 // phrase, the phrase is not GPU-resident, its slot exists and no earlier entry names the same
 // phrase; it is applied if, in addition, no earlier candidate names the same slot.  "Earlier" is
-// settled with one atomicMax per entry on a stamp per phrase and per slot: a stamp is
-// (call number << 12) | (4095 - k), so the current call beats every older stamp and, within the
-// call, the smallest k wins; nothing has to be cleared between calls.
+// settled with one atomicMax per entry on a stamp per phrase and per slot: the stamp of entry k is
+// 4096 - k, so the smallest k wins; the stamps are zero between calls (the last kernel puts back the
+// ones this call touched), so the call keeps no state on the host and can be replayed from a graph.
 //
 //   tfe_install_claim_kernel<0>  every entry stamps its phrase
 //   tfe_install_claim_kernel<1>  every candidate stamps its slot
 //   tfe_install_device_kernel    one warp per entry: the winners install (as tfe_install_kernel)
+//   tfe_install_clear_kernel     the stamps this call wrote go back to zero
 #define TFE_INSTALL_DEVICE_MAX 4096
 
 struct TfeInstallDeviceParams {
@@ -878,7 +879,6 @@ struct TfeInstallDeviceParams {
     const int32_t *dst_slots;       // [n]
     uint32_t *phrase_stamp;         // [n_phrases]
     uint32_t *slot_stamp;           // [gpu_slots]
-    uint32_t tag;                   // call number << 12
     uint8_t *applied;               // [n] or nullptr
     uint32_t *count;                // entries applied (cleared by the host side before the launches)
     uint2 *slot_stats;
@@ -891,7 +891,7 @@ __device__ __forceinline__ bool tfe_install_candidate(const TfeInstallDevicePara
     const int32_t dst = p.dst_slots[k];
     if (id >= p.n_phrases || dst < 0 || (int64_t)dst >= p.gpu_slots) return false;
     if ((int32_t)(uint32_t)p.index[p.phrase_pos[id]].y >= 0) return false;          // resident before the call
-    return __ldcg(p.phrase_stamp + id) == (p.tag | (uint32_t)(TFE_INSTALL_DEVICE_MAX - 1 - k));
+    return __ldcg(p.phrase_stamp + id) == (uint32_t)(TFE_INSTALL_DEVICE_MAX - k);
 }
 
 template <int STAGE>
@@ -901,13 +901,25 @@ tfe_install_claim_kernel(const TfeInstallDeviceParams p)
     tfe_grid_dependency_sync();
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
     if (k >= p.n) return;
-    const uint32_t stamp = p.tag | (uint32_t)(TFE_INSTALL_DEVICE_MAX - 1 - k);
+    const uint32_t stamp = (uint32_t)(TFE_INSTALL_DEVICE_MAX - k);         // 1..4096: never the cleared value
     if (STAGE == 0) {
         const uint32_t id = p.ids[k];
         if (id < p.n_phrases) atomicMax(p.phrase_stamp + id, stamp);
     } else {
         if (tfe_install_candidate(p, k)) atomicMax(p.slot_stamp + p.dst_slots[k], stamp);
     }
+}
+
+__global__ void __launch_bounds__(256)
+tfe_install_clear_kernel(const TfeInstallDeviceParams p)
+{
+    tfe_grid_dependency_sync();
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= p.n) return;
+    const uint32_t id = p.ids[k];
+    const int32_t dst = p.dst_slots[k];
+    if (id < p.n_phrases) p.phrase_stamp[id] = 0;
+    if (dst >= 0 && (int64_t)dst < p.gpu_slots) p.slot_stamp[dst] = 0;
 }
 
 __global__ void __launch_bounds__(TFE_BLOCK_THREADS)
@@ -920,7 +932,7 @@ tfe_install_device_kernel(const TfeInstallDeviceParams p)
     bool apply = false;
     if (lane == 0) {
         apply = tfe_install_candidate(p, k) &&
-                __ldcg(p.slot_stamp + p.dst_slots[k]) == (p.tag | (uint32_t)(TFE_INSTALL_DEVICE_MAX - 1 - k));
+                __ldcg(p.slot_stamp + p.dst_slots[k]) == (uint32_t)(TFE_INSTALL_DEVICE_MAX - k);
         if (p.applied) p.applied[k] = apply ? 1 : 0;
         if (apply) atomicAdd(p.count, 1u);
     }

@@ -178,3 +178,56 @@ def test_prefetch_loop_without_a_host_round_trip(H):
     pr.run_and_compare(tok, hid, q_start=2, lam=1.0)
     head.close()
     pr.close()
+
+
+def test_device_install_replayed_from_a_graph(H):
+    """Victim selection + device-side installation captured once and replayed with new batches written into the
+    same buffers: the call keeps no state on the host, so every replay must act like a fresh call."""
+    from paper_2607_07388_b200 import binding as tfe
+    from paper_2607_07388_b200.engine import bf16_tensor_from_bits, _device_view
+    w = synth.config(1, B=3, T=128, n_phrases=6_000, gpu_slots=1_500, d=64, residency="hot_host_ssd", p=0.5)
+    tb, pr = H.pair_from_workload(w)
+    pr.eng.cache_policy_enable()
+    n = 64
+    ids_buf = torch.zeros(n, dtype=torch.int32, device=DEV)
+    src_buf = torch.zeros((n, w.d), dtype=torch.bfloat16, device=DEV)
+    applied = torch.zeros(n, dtype=torch.uint8, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int32, device=DEV)
+    # first calls outside the capture (allocations), checked like any other
+    tfe.tfe_cache_select_victims_async(pr.eng.ctx, n, 2)
+    slots_ptr, _ = tfe.tfe_cache_select_victims_device(pr.eng.ctx)
+    slots_dev = _device_view(slots_ptr, (n,), "<i4", DEV)
+    pr.eng.cache_install_device(ids_buf.fill_(-1), src_buf, slots_dev)             # nothing valid: applies nothing
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            tfe.tfe_cache_select_victims_async(pr.eng.ctx, n, 2, stream=side)
+            tfe.tfe_cache_install_device(pr.eng.ctx, n, ids_buf, src_buf, slots_dev, applied, cnt, stream=side)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(8)
+    h = synth.make_hidden_np(w)
+    total = 0
+    for step in range(6):
+        tok = synth.make_queries(w, tb, variant=step)
+        _, ref, _ = pr.run_and_compare(tok, h, lam=1.0)
+        pr.ora.touch(ref)
+        # a batch with repeats of earlier steps' ids (now resident), invalid ids and fresh misses
+        pool = np.concatenate([ref.miss_phrase.astype(np.int64), rng.integers(0, w.n_phrases + 20, size=n)])
+        ids = rng.choice(pool, size=n).astype(np.uint32)
+        src = synth.phrase_rows_np(w, np.minimum(ids.astype(np.int64), w.n_phrases - 1))
+        ids_buf.copy_(torch.from_numpy(ids.view(np.int32)))
+        src_buf.copy_(bf16_tensor_from_bits(src, DEV))
+        graph.replay()
+        torch.cuda.synchronize()
+        e_slots, _ = pr.ora.cache_victims(n, 2)
+        e_applied, e_cnt = pr.ora.cache_install_lenient(ids, src, e_slots)
+        np.testing.assert_array_equal(slots_dev.cpu().numpy(), e_slots)
+        np.testing.assert_array_equal(applied.cpu().numpy(), e_applied)
+        assert int(cnt.item()) == e_cnt
+        total += e_cnt
+        pr.run_and_compare(tok, h, lam=1.0)
+        pr.ora.touch(pr.ora.lookup(tok))
+    assert total > 30
+    pr.close()
