@@ -68,6 +68,8 @@ def parse_args():
                     help="time the other selection policies and gates (ALL, COSINE, a lambda that is not a bf16 number)")
     ap.add_argument("--build", action="store_true",
                     help="time index construction on the GPU (tfe_index_build_device) against the host build")
+    ap.add_argument("--loop", action="store_true",
+                    help="decode shapes: lookup -> early-exit head -> candidates -> victims -> installation, all on the device")
     ap.add_argument("--mine", action="store_true", help="n-gram extraction with a frequency threshold over a synthetic corpus")
     ap.add_argument("--mine-tokens", type=int, default=1 << 26)
     ap.add_argument("--mine-min-count", type=int, default=3)
@@ -419,6 +421,8 @@ def run_ours(a):
         return run_build(a, dev, rank)
     if a.mine:
         return run_mine(a, dev, rank)
+    if a.loop:
+        return run_loop(a, dev, rank)
     if a.variants:
         return run_variants(a, dev, rank)
 
@@ -899,6 +903,115 @@ def run_build(a, dev, rank):
                              "ms": host_s * 1e3},
             "parity": {"device_vs_host_build": bool(same), "device_build_vs_oracle": oracle_ok}}))
     eng.close(); host.close()
+
+
+def run_loop(a, dev, rank):
+    """One decode step of the whole inference-side path (Sec. 4.4: lookup and injection for the current token,
+    early-exit prediction of the next ones, candidate expansion, and -- here also -- the choice of the slots to
+    overwrite and the installation), every stage taking the previous stage's device output, replayed from a
+    CUDA graph.  The rows of the candidates come from a pool staged on the device: the DRAM / SSD read that
+    would deliver them is outside this library."""
+    import torch
+    from paper_2607_07388_b200 import binding as tfe
+    from paper_2607_07388_b200.engine import EarlyExitHead, _device_view
+    L = tfe.lib()
+    w = make_workload(a)
+    assert w.shape == "decode", "--loop needs a decode workload (c2, c4, c5)"
+    nbuf, K, budget, half_life = 8, a.top_k, 4096, 2
+    sess = Session(w, dev, nbuf, a.tune_batch)
+    eng = sess.eng
+    eng.cache_policy_enable()
+    B, d = w.B, w.d
+    head = EarlyExitHead(synth.head_weights_torch(a.head_vocab, d, dev), max_batch=B)
+    pool_n = 1 << 18
+    pool = torch.empty((pool_n, d), dtype=torch.bfloat16, device=dev)
+    synth.fill_rows_torch(pool, torch.arange(pool_n, dtype=torch.int64, device=dev))
+    H = w.T - 1
+    hist = [t[:, 1:].contiguous() for t in sess.toks]
+    t_tok = torch.empty((B, K), dtype=torch.int32, device=dev)
+    t_prob = torch.empty((B, K), dtype=torch.float32, device=dev)
+    ph = torch.empty(budget, dtype=torch.int32, device=dev)
+    tr = torch.empty(budget, dtype=torch.uint8, device=dev)
+    sc = torch.empty(budget, dtype=torch.float32, device=dev)
+    sr = torch.empty(budget, dtype=torch.int32, device=dev)
+    cnt = torch.zeros(2, dtype=torch.int32, device=dev)
+    applied = torch.empty(budget, dtype=torch.uint8, device=dev)
+    n_applied = torch.zeros(1, dtype=torch.int32, device=dev)
+    installed_total = torch.zeros(1, dtype=torch.int64, device=dev)
+    tfe.tfe_cache_select_victims_async(eng.ctx, budget, half_life)
+    slots_ptr, _ = tfe.tfe_cache_select_victims_device(eng.ctx)
+    slots_dev = _device_view(slots_ptr, (budget,), "<i4", dev)
+    src = torch.empty((budget, d), dtype=torch.bfloat16, device=dev)
+
+    def stage_lookup(v, st):
+        calls = sess.lookup_calls(st.cuda_stream)
+        if L.tfe_lookup_inject(*calls[v]):
+            raise RuntimeError("tfe_lookup_inject failed")
+
+    def stage_head(v, st):
+        tfe.tfe_head_topk(head.handle, sess.outs[v], B, K, t_tok, t_prob, st)
+
+    def stage_candidates(v, st):
+        ph.fill_(-1)                                             # unwritten entries are no phrases
+        tfe.tfe_prefetch_candidates(eng.ctx, hist[v], B, H, t_tok, t_prob, K, out_phrase=ph, out_tier=tr, out_score=sc,
+                                    out_src=sr, out_count=cnt, budget=budget, stream=st)
+
+    def stage_victims(v, st):
+        tfe.tfe_cache_select_victims_async(eng.ctx, budget, half_life, st)
+
+    def stage_install(v, st):
+        torch.index_select(pool, 0, torch.remainder(ph.clamp(min=0), pool_n).long(), out=src)    # stands in for the fetch
+        tfe.tfe_cache_install_device(eng.ctx, budget, ph, src, slots_dev, applied, n_applied, st)
+        installed_total.add_(n_applied.long())
+
+    stages = [("lookup_inject", stage_lookup), ("head_topk", stage_head), ("prefetch_candidates", stage_candidates),
+              ("select_victims", stage_victims), ("gather + install_device", stage_install)]
+    cur = torch.cuda.current_stream()
+    for v in range(2):                                           # first calls allocate
+        for _, f in stages:
+            f(v, cur)
+    torch.cuda.synchronize()
+
+    def timed_graph(fs, reps):
+        side = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for v in range(nbuf):
+                    for f in fs:
+                        f(v, side)
+            torch.cuda.synchronize()
+            for _ in range(3):
+                g.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(side)
+            for _ in range(reps):
+                g.replay()
+            e1.record(side)
+            torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (reps * nbuf)
+
+    reps = max(5, min(50, a.steps // nbuf))
+    installed_total.zero_()
+    us_step = timed_graph([f for _, f in stages], reps)
+    n_inst = int(installed_total.item())
+    per_stage = {name: timed_graph([f], reps) for name, f in stages}
+    status = head.status()
+    if rank == 0:
+        print(json.dumps({
+            "metric": "decode steps/s, whole inference-side path on the device", "value": 1e6 / us_step, "unit": "steps/s",
+            "us_per_step": us_step, "tokens_per_s": B * 1e6 / us_step, "steps": reps * nbuf,
+            "config": {"workload": w.name, "B": B, "d": d, "top_k": K, "budget": budget, "head_vocab": a.head_vocab,
+                       "gpu_slots": w.gpu_slots, "n_phrases": w.n_phrases,
+                       "launch": f"CUDA graph of {nbuf} steps, replayed; no host synchronisation inside a step",
+                       "rows": "candidate rows gathered from a pool staged on the device (the DRAM / SSD read is outside the library)"},
+            "us_per_stage_alone": per_stage, "sum_of_stages_us": sum(per_stage.values()),
+            "installed_per_step": n_inst / ((reps + 3) * nbuf), "head_status": status,
+            "parity": "the chain is checked against the oracle in tests/test_gpu_install_device.py (not in this mode: "
+                      "fp64 logits over the whole vocabulary take seconds per step on the host)"}))
+    head.close()
+    sess.close()
 
 
 def run_mine(a, dev, rank):
