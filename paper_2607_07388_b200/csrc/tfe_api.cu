@@ -1048,7 +1048,7 @@ tfe_status tfe_cache_select_victims(tfe_ctx *c, int32_t n, int32_t half_life, in
                              c->d_slot_owner, c->d_epoch, half_life, c->d_slot_key, (uint32_t)C, 0u, kShift[i], kBits[i],
                              c->d_vs_hist, c->d_vs_state));
     static_assert(TFE_VICTIM_BINS >= 4 * 256, "the histogram array doubles as one counter per block");
-    if (grid > TFE_VICTIM_BINS) return TFE_ERR_INTERNAL;
+    if (grid > 2 * TFE_VICTIM_THREADS) return TFE_ERR_INTERNAL;      // two range counts per thread of the closing block
     CU(launch_overlapped(tfe_victim_tie_kernel, dim3(grid), dim3(TFE_VICTIM_THREADS), stream, c->d_slot_key, (uint32_t)C,
                          c->d_vs_hist, c->d_vs_state));
     CU(launch_overlapped(tfe_victim_collect_kernel, dim3(grid), dim3(TFE_VICTIM_THREADS), stream, c->d_slot_key, (uint32_t)C,

@@ -1325,29 +1325,45 @@ tfe_victim_tie_kernel(const uint32_t *slot_key, uint32_t C, uint32_t *tie_count,
         if (!s_last) return;
         __threadfence();
     }
-    // ---- last block: which range holds the k_rem-th tie
-    if (warp == 0) {
+    // ---- last block: which range holds the k_rem-th tie.  The per-block counts (at most two per thread,
+    // loaded together) are scanned in block order: first all threads' first element, then the second ones.
+    {
         const uint32_t want = state->k_rem;
-        uint32_t running = 0;
-        bool found = false;
-        for (uint32_t base = 0; base < gridDim.x; base += 32) {
-            const uint32_t i = base + lane;
-            const uint32_t c = i < gridDim.x ? __ldcg(tie_count + i) : 0u;
+        uint32_t c[2], incl[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t i = h * TFE_VICTIM_THREADS + threadIdx.x;
+            c[h] = i < gridDim.x ? __ldcg(tie_count + i) : 0u;
             if (i < gridDim.x) tie_count[i] = 0;
-            uint32_t incl = c;
+        }
+        uint32_t carry = 0;                                   // total of the first half, for the second
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t v = c[h];
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                if (lane >= o) incl += v;
+                const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, v, o);
+                if (lane >= o) v += u;
             }
-            const uint32_t reach = __ballot_sync(0xFFFFFFFFu, running + incl >= want);
-            if (!found && reach != 0u) {
-                found = true;
-                if (lane == __ffs(reach) - 1) { s_block = i; s_rank = want - (running + incl - c); }
+            __syncthreads();
+            if (lane == 31) s_warp[warp] = v;
+            __syncthreads();
+            uint32_t before = carry, total = 0;
+            for (int w = 0; w < TFE_VICTIM_THREADS / 32; ++w) {
+                if (w < warp) before += s_warp[w];
+                total += s_warp[w];
             }
-            running += __shfl_sync(0xFFFFFFFFu, incl, 31);
+            incl[h] = before + v;
+            carry += total;
         }
-        if (!found && lane == 0) { s_block = 0; s_rank = 0; }       // cannot happen: k_rem <= number of ties
+        if (threadIdx.x == 0) { s_block = 0; s_rank = 0; }      // overwritten below: k_rem <= number of ties
+        __syncthreads();
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+            if (incl[h] >= want && incl[h] - c[h] < want) {      // exactly one element
+                s_block = h * TFE_VICTIM_THREADS + threadIdx.x;
+                s_rank = want - (incl[h] - c[h]);
+            }
     }
     __syncthreads();
     // ---- walk that range: a contiguous piece per thread, counts, scan, then the piece that holds the tie
