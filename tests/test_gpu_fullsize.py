@@ -114,3 +114,44 @@ def test_millions_of_positions_narrow_rows(H):
         _, ref, info = pr.run_and_compare(tok, h, q_start=w.q_start, lam=1.0)
         assert info["n_hit"] > 50_000 and info["n_miss"] > 50_000
         pr.close()
+
+
+def test_mine_tens_of_millions_of_ids(H):
+    """n-gram extraction at a benchmark-sized corpus (2^25 ids, 100 M windows), with the caller's workspace as
+    bench.py times it: the oracle recounts sampled tuples one by one by a scan over the whole corpus, checks
+    their order, a prefix of the corpus is compared on every output, and the properties that tie the outputs
+    together hold."""
+    from oracle import tfe_oracle as orc
+    from paper_2607_07388_b200 import binding as tfe
+    from paper_2607_07388_b200.engine import mine_ngrams
+    L, orders, m = 1 << 25, (2, 3, 4), 3
+    corpus_np = synth.make_corpus(21, L)
+    corpus = torch.from_numpy(corpus_np).to(H.DEV)
+    ws = torch.empty(tfe.tfe_mine_workspace_bytes(L, len(orders)), dtype=torch.uint8, device=H.DEV)
+    sizing = mine_ngrams(corpus, vocab=synth.VOCAB, orders=orders, min_count=m, cap=0, workspace=ws)
+    got = mine_ngrams(corpus, vocab=synth.VOCAB, orders=orders, min_count=m, cap=sizing.n_found, workspace=ws)
+    assert got.n_found == sizing.n_found == len(got) > 1_000_000
+    np.testing.assert_array_equal(got.hist, sizing.hist)
+    g_pt, g_pl = got.phrase_tokens.cpu().numpy(), got.phrase_len.cpu().numpy()
+    g_pc = got.count.cpu().numpy().view(np.uint32)
+    tail = np.cumsum(got.hist[::-1])[::-1]
+    assert got.n_found == tail[m] and got.distinct.sum() == tail[1] and int(g_pc.min()) >= m
+    n_windows = sum(int(((np.lib.stride_tricks.sliding_window_view(corpus_np, n) >= 0).all(axis=1)).sum()) for n in orders)
+    assert n_windows >= int((got.hist[:-1] * np.arange(len(got.hist) - 1)).sum())          # the last bin holds larger counts
+    rng = np.random.default_rng(3)
+    firsts = []
+    for i in np.sort(rng.choice(len(g_pl), size=16, replace=False)):
+        n = int(g_pl[i])
+        count, first = orc.count_tuple(corpus_np, g_pt[i, :n])
+        assert count == int(g_pc[i]) and (g_pt[i, n:] == -1).all()
+        firsts.append((first, n))
+    assert firsts == sorted(firsts)
+    n_pre = 1 << 19
+    e_pt, e_pl, e_pc, e_found, e_distinct, e_hist = orc.mine_ngrams(corpus_np[:n_pre], synth.VOCAB, orders, min_count=m, cap=n_pre)
+    pre = mine_ngrams(corpus[:n_pre].contiguous(), vocab=synth.VOCAB, orders=orders, min_count=m, cap=n_pre, workspace=ws)
+    assert pre.n_found == e_found
+    np.testing.assert_array_equal(pre.distinct, e_distinct)
+    np.testing.assert_array_equal(pre.hist, e_hist)
+    np.testing.assert_array_equal(pre.phrase_tokens.cpu().numpy(), e_pt)
+    np.testing.assert_array_equal(pre.phrase_len.cpu().numpy(), e_pl)
+    np.testing.assert_array_equal(pre.count.cpu().numpy().view(np.uint32), e_pc)
