@@ -46,6 +46,7 @@
  *   sel_slot      slot for a GPU hit, -1 / -2 for a miss, -3 for absent.
  *   sel_phrase    phrase id, 0xFFFFFFFF for absent.
  */
+#define _GNU_SOURCE     /* qsort_r */
 #include <math.h>
 #include <stdint.h>
 #include <stdlib.h>
