@@ -73,6 +73,8 @@ def parse_args():
     ap.add_argument("--mine", action="store_true", help="n-gram extraction with a frequency threshold over a synthetic corpus")
     ap.add_argument("--mine-tokens", type=int, default=1 << 26)
     ap.add_argument("--mine-min-count", type=int, default=3)
+    ap.add_argument("--mine-build", action="store_true",
+                    help="--mine: also build the index from the mined table on the device and look the corpus up in it")
     ap.add_argument("--cache-policy", action="store_true",
                     help="time the retention bookkeeping in the lookup and tfe_cache_select_victims on the workload")
     ap.add_argument("--sweep", action="store_true", help="c5: tokens x row width x hit rate sweep")
@@ -1071,8 +1073,58 @@ def run_mine(a, dev, rank):
     keys = [firsts[i] for i in sorted(firsts)]
     sample_ok &= keys == sorted(keys)                                        # entries are in (first, n) order
     tail = np.cumsum(got.hist[::-1])[::-1]
-    props_ok = bool(got.n_found == cap == tail[m] and int(g_pc.min()) >= m and got.distinct.sum() == tail[1]
-                    and len(np.unique(np.concatenate([g_pt, g_pl[:, None].astype(np.int32)], axis=1), axis=0)) == len(g_pl))
+    props_ok = bool(got.n_found == cap == tail[max(m, 1)] and int(g_pc.min()) >= m and got.distinct.sum() == tail[1])
+    if len(g_pl) <= 20_000_000:          # no tuple twice (larger results: the index build refuses duplicates)
+        props_ok &= len(np.unique(np.concatenate([g_pt, g_pl[:, None].astype(np.int32)], axis=1), axis=0)) == len(g_pl)
+    built = None
+    if a.mine_build:
+        # corpus -> table -> index -> lookups without leaving the device.  The first C phrases (the ones met
+        # first) live in the GPU tier, the rest is tagged host; rows are not read by this check.
+        from paper_2607_07388_b200.engine import Engram
+        N, C_slots, d_rows = len(got), int(min(len(got), 1 << 20)), 16
+        init_slot = torch.full((N,), -1, dtype=torch.int32, device=dev)
+        init_slot[:C_slots] = torch.arange(C_slots, dtype=torch.int32, device=dev)
+        rows = torch.zeros((C_slots, d_rows), dtype=torch.bfloat16, device=dev)
+        times = []
+        for _ in range(3):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            eng = Engram(got.phrase_tokens, got.phrase_len, init_slot, rows, vocab=synth.VOCAB, orders=orders, device_build=True)
+            torch.cuda.synchronize()
+            times.append(time.perf_counter() - t0)
+            if len(times) < 3:
+                eng.close()
+        build_s = float(np.median(times))
+        # every position of a stretch of the corpus: the retained phrase must be the longest window that ends
+        # there, occurs min_count times and contains no separator -- checked against the mined table itself
+        Bq, Tq = 256, 4096
+        tok = corpus[:Bq * Tq].view(Bq, Tq).contiguous()
+        hid = torch.zeros((Bq * Tq, d_rows), dtype=torch.bfloat16, device=dev)
+        r = eng.lookup_inject(tok, hid, torch.empty_like(hid))
+        sel = r.sel_phrase.view(Bq, Tq).long()
+        found = r.flags.view(Bq, Tq) != 0
+        safe = torch.where(found, sel, torch.zeros_like(sel))
+        ln = got.phrase_len.long()[safe]                                    # length of the retained phrase
+        tup = got.phrase_tokens[safe]                                       # [Bq, Tq, 4]
+        ok = torch.ones_like(found)
+        tpos = torch.arange(Tq, device=dev).view(1, Tq)
+        for j in range(4):                                                  # tuple element j sits at t - (len - 1) + j
+            src_t = tpos - (ln - 1) + j
+            inside = found & (j < ln)
+            ok &= ~inside | ((src_t >= 0) & (torch.gather(tok, 1, src_t.clamp(min=0, max=Tq - 1)) == tup[..., j]))
+        n_found_pos = int(found.sum().item())
+        tuples_ok = bool(ok.all().item())
+        if m <= 1:          # every separator-free window is a phrase: a 4-gram wherever four valid ids end
+            valid = (tok >= 0)
+            four = valid & torch.roll(valid, 1, 1) & torch.roll(valid, 2, 1) & torch.roll(valid, 3, 1)
+            four[:, :3] = False
+            longest_ok = bool(((ln == 4) & found)[four].all().item())
+        else:
+            longest_ok = None
+        built = {"n_phrases": N, "gpu_slots": C_slots, "build_ms": build_s * 1e3, "phrases_per_s": N / build_s,
+                 "lookup_positions": Bq * Tq, "positions_with_a_phrase": n_found_pos,
+                 "retained_tuple_equals_the_corpus_window": tuples_ok, "four_gram_wherever_four_ids_end": longest_ok}
+        eng.close()
     slots = 1024
     while slots < L + L // 2:
         slots *= 2
@@ -1094,6 +1146,7 @@ def run_mine(a, dev, rank):
                          "note": "random 32-byte sectors of the counting table dominate: 64 B per window in the count pass, 32 B in the mark pass"},
             "cpu_baseline": {"value": n_pre / cpu_s, "unit": "tokens/s", "cores": 1, "kind": "oracle",
                              "sample": f"the first {n_pre} ids of the corpus (sort-based definition, single thread)"},
+            "index_from_the_mined_table": built,
             "parity": {"prefix_all_outputs": prefix_ok, "full_size_sampled_counts_and_order": bool(sample_ok),
                        "full_size_properties": props_ok}}))
 
