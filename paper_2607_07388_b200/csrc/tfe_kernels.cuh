@@ -137,10 +137,15 @@ __device__ __forceinline__ bool tuple_matches(const int4 st, const int32_t (&tk)
     }
 }
 
+// The index is what every call probes again; its lines ask to stay in L2 (evict-last), the hidden states that
+// stream through ask to leave first (ld.global.cs / st.global.cs above).
 __device__ __forceinline__ ulonglong4 ld_bucket32(const ulonglong4 *p)    // 32 bytes = two index slots
 {
     ulonglong4 v;
-    asm volatile("ld.global.nc.v4.u64 {%0,%1,%2,%3}, [%4];" : "=l"(v.x), "=l"(v.y), "=l"(v.z), "=l"(v.w) : "l"(p));
+    unsigned long long policy;
+    asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
+    asm volatile("ld.global.nc.L2::cache_hint.v4.u64 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=l"(v.x), "=l"(v.y), "=l"(v.z), "=l"(v.w) : "l"(p), "l"(policy));
     return v;
 }
 
