@@ -1298,7 +1298,7 @@ NBUF_DECODE = 32        # decode shapes: this many distinct query / hidden-state
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the lookup kernel in steady state (no cache
 # flush between launches, so the write-back of the previous launch's output is included), from the ncu
 # capture summarised under profiles/; taken on a 1M-phrase table: traffic does not depend on N
-NCU_TRAFFIC = {"c3_prefill8x4096": 163_200_000}
+NCU_TRAFFIC = {"c3_prefill8x4096": 162_400_000}
 
 
 # ------------------------------------------------------------ reference arm
