@@ -771,3 +771,38 @@ int64_t orc_count_tuple(int64_t L, const int32_t *tokens, int32_t n, const int32
     }
     return count;
 }
+
+/* ------------------------------------------------------------------------------------------------
+ * Initial residency from corpus counts [Sec. 4.3: the GPU tier is reserved for the most frequently
+ * accessed entries, DRAM holds warm entries, SSD absorbs the long tail].
+ *
+ * The G = min(gpu_slots, N) phrases of largest count start in the GPU tier; among equal counts the
+ * smaller id goes first.  GPU-tier slots are handed out in id order: the chosen phrase with the k-th
+ * smallest id gets slot k.  Of the others, a count >= host_min_count means host DRAM (-1), a smaller
+ * one SSD (-2).  tiers[0..2] receive the number of phrases per tier (GPU, host, SSD). */
+typedef struct { uint32_t count; int64_t id; } orc_ranked;
+
+static int ranked_cmp(const void *pa, const void *pb)
+{
+    const orc_ranked *a = (const orc_ranked *)pa, *b = (const orc_ranked *)pb;
+    if (a->count != b->count) return a->count > b->count ? -1 : 1;
+    return a->id < b->id ? -1 : (a->id > b->id ? 1 : 0);
+}
+
+void orc_assign_residency(int64_t N, const uint32_t *count, int64_t gpu_slots, uint32_t host_min_count,
+                          int32_t *init_slot, int64_t *tiers)
+{
+    orc_ranked *r = (orc_ranked *)malloc((size_t)(N + 1) * sizeof *r);
+    for (int64_t i = 0; i < N; ++i) { r[i].count = count[i]; r[i].id = i; }
+    qsort(r, (size_t)N, sizeof *r, ranked_cmp);
+    const int64_t G = gpu_slots < N ? gpu_slots : N;
+    tiers[0] = tiers[1] = tiers[2] = 0;
+    for (int64_t i = 0; i < N; ++i) init_slot[i] = count[i] >= host_min_count ? -1 : -2;
+    for (int64_t k = 0; k < G; ++k) init_slot[r[k].id] = 0;           /* chosen; numbered below */
+    int32_t next = 0;
+    for (int64_t i = 0; i < N; ++i) {
+        if (init_slot[i] == 0) init_slot[i] = next++;
+        ++tiers[init_slot[i] >= 0 ? 0 : (init_slot[i] == -1 ? 1 : 2)];
+    }
+    free(r);
+}

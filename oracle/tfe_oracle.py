@@ -301,3 +301,13 @@ def count_tuple(tokens, tup):
     f.restype = C.c_int64
     n = f(C.c_int64(len(tokens)), _p(tokens), C.c_int32(len(tup)), _p(tup), C.byref(first))
     return int(n), int(first.value)
+
+
+def assign_residency(count, gpu_slots, host_min_count=2):
+    """(init_slot int32 [N], (n_gpu, n_host, n_ssd)): the gpu_slots most frequent phrases in the GPU tier."""
+    count = _c(count, np.uint32)
+    N = len(count)
+    init_slot, tiers = np.empty(max(N, 1), np.int32), np.zeros(3, np.int64)
+    lib().orc_assign_residency(C.c_int64(N), _p(count), C.c_int64(gpu_slots), C.c_uint32(host_min_count),
+                               _p(init_slot), _p(tiers))
+    return init_slot[:N].copy(), tuple(int(x) for x in tiers)

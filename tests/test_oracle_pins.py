@@ -893,3 +893,37 @@ def test_count_tuple_by_hand_and_against_the_extraction(oracle_mod):
         win = np.lib.stride_tricks.sliding_window_view(tok, n)
         hits = np.flatnonzero((win == pt[i, :n]).all(axis=1))
         assert oracle_mod.count_tuple(tok, pt[i, :n]) == (len(hits), int(hits[0]) + n - 1) == (int(pc[i]), int(hits[0]) + n - 1)
+
+
+# ---------------------------------------------------------------------------------------------
+# initial residency from corpus counts (Sec. 4.3: hottest entries in the GPU tier)
+# ---------------------------------------------------------------------------------------------
+def test_assign_residency_hand_worked_and_closed_forms(oracle_mod):
+    #            id: 0  1  2  3  4  5  6
+    count = np.array([5, 9, 5, 1, 9, 2, 5], np.uint32)
+    # three slots: the two 9s, then the first of the 5s (id 0); slots in id order: id 0 -> 0, id 1 -> 1, id 4 -> 2
+    slot, tiers = oracle_mod.assign_residency(count, 3, host_min_count=2)
+    assert slot.tolist() == [0, 1, -1, -2, 2, -1, -1] and tiers == (3, 3, 1)
+    slot, tiers = oracle_mod.assign_residency(count, 4, host_min_count=6)
+    assert slot.tolist() == [0, 1, 2, -2, 3, -2, -2] and tiers == (4, 0, 3)
+    # no slots / more slots than phrases / all counts equal: the first ids
+    assert oracle_mod.assign_residency(count, 0, 1)[0].tolist() == [-1] * 7
+    assert oracle_mod.assign_residency(count, 100, 1)[0].tolist() == list(range(7))
+    assert oracle_mod.assign_residency(np.full(6, 4, np.uint32), 2, 5)[0].tolist() == [0, 1, -2, -2, -2, -2]
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_assign_residency_against_library_sort(oracle_mod, seed):
+    rng = np.random.default_rng([55, seed])
+    N = int(rng.integers(1, 5000))
+    count = rng.integers(1, int(rng.choice([3, 20, 100000])), size=N).astype(np.uint32)
+    G = int(rng.integers(0, N + 5))
+    hm = int(rng.integers(0, 6))
+    slot, tiers = oracle_mod.assign_residency(count, G, hm)
+    order = np.lexsort((np.arange(N), -count.astype(np.int64)))              # count descending, then id
+    chosen = np.zeros(N, bool)
+    chosen[order[:min(G, N)]] = True
+    expect = np.where(count >= hm, -1, -2).astype(np.int32)
+    expect[chosen] = np.arange(int(chosen.sum()), dtype=np.int32)
+    np.testing.assert_array_equal(slot, expect)
+    assert tiers == (int(chosen.sum()), int((expect == -1).sum()), int((expect == -2).sum()))
