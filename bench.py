@@ -1078,12 +1078,20 @@ def run_mine(a, dev, rank):
         props_ok &= len(np.unique(np.concatenate([g_pt, g_pl[:, None].astype(np.int32)], axis=1), axis=0)) == len(g_pl)
     built = None
     if a.mine_build:
-        # corpus -> table -> index -> lookups without leaving the device.  The first C phrases (the ones met
-        # first) live in the GPU tier, the rest is tagged host; rows are not read by this check.
+        # corpus -> table -> residency -> index -> lookups without leaving the device; rows are not read by this check
         from paper_2607_07388_b200.engine import Engram
         N, C_slots, d_rows = len(got), int(min(len(got), 1 << 20)), 16
-        init_slot = torch.full((N,), -1, dtype=torch.int32, device=dev)
-        init_slot[:C_slots] = torch.arange(C_slots, dtype=torch.int32, device=dev)
+        rt = []
+        init_slot = torch.empty(N, dtype=torch.int32, device=dev)
+        for _ in range(5):                       # the C most frequent phrases start in the GPU tier
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            tiers = tfe.tfe_assign_residency(got.count, N, C_slots, 3, init_slot)
+            torch.cuda.synchronize()
+            rt.append(time.perf_counter() - t0)
+        resid_ms = float(np.median(rt)) * 1e3
+        chosen_min = int(got.count[init_slot >= 0].view(torch.int32).min().item()) if C_slots else 0
+        rest_max = int(got.count[init_slot < 0].max().item()) if C_slots < N else 0
         rows = torch.zeros((C_slots, d_rows), dtype=torch.bfloat16, device=dev)
         times = []
         for _ in range(3):
@@ -1121,7 +1129,9 @@ def run_mine(a, dev, rank):
             longest_ok = bool(((ln == 4) & found)[four].all().item())
         else:
             longest_ok = None
-        built = {"n_phrases": N, "gpu_slots": C_slots, "build_ms": build_s * 1e3, "phrases_per_s": N / build_s,
+        built = {"n_phrases": N, "gpu_slots": C_slots, "residency_ms": resid_ms, "tiers_gpu_host_ssd": list(tiers),
+                 "smallest_count_in_gpu_tier": chosen_min, "largest_count_outside": rest_max,
+                 "build_ms": build_s * 1e3, "phrases_per_s": N / build_s,
                  "lookup_positions": Bq * Tq, "positions_with_a_phrase": n_found_pos,
                  "retained_tuple_equals_the_corpus_window": tuples_ok, "four_gram_wherever_four_ids_end": longest_ok}
         eng.close()

@@ -452,6 +452,24 @@ tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int3
                            void *workspace, int64_t workspace_bytes, void *stream);
 int64_t tfe_mine_workspace_bytes(int64_t L, int32_t n_orders);   /* -1 for invalid arguments */
 
+/*
+ * Initial residency from corpus counts (paper Sec. 4.3: the GPU tier is reserved for the most frequently
+ * accessed entries, DRAM holds warm entries, SSD absorbs the long tail).  Turns the counts that
+ * tfe_mine_ngrams returns into the init_slot array that tfe_index_build_device takes.
+ *
+ *   count           DEVICE uint32 [N];  init_slot DEVICE int32 [N] (output);  0 <= N, gpu_slots < 2^31
+ *   rule            the G = min(gpu_slots, N) phrases of largest count start in the GPU tier, among equal
+ *                   counts the smaller id first; GPU-tier slots are handed out in id order (the chosen
+ *                   phrase with the k-th smallest id gets slot k).  Of the others, count >= host_min_count
+ *                   means host DRAM (-1), a smaller count SSD (-2).
+ *   tiers           HOST int64 [3] or NULL: phrases per tier (GPU, host, SSD).
+ *
+ * Allocates a few bytes per 1,024 phrases, launches on `stream`, synchronises it.
+ * Errors: TFE_ERR_INVALID_ARG, TFE_ERR_CUDA, TFE_ERR_INTERNAL (the selection's totals do not add up).
+ */
+tfe_status tfe_assign_residency(const uint32_t *count, int64_t N, int64_t gpu_slots, uint32_t host_min_count,
+                                int32_t *init_slot, int64_t *tiers, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,6 +22,7 @@
  *   - retention ranking of GPU-tier slots (frequency, recency) [Sec. 4.3, cache policy signals]
  *   - early-exit prefetch head: softmax(W_pref h), top-K        [Sec. 4.4, p_early and T_early equations]
  *   - n-gram extraction with a frequency threshold              [Sec. 4.2, construction pipeline; Sec. 5.3]
+ *   - initial residency from corpus counts                      [Sec. 4.3, tiers by access frequency]
  *
  * Parity pins: every function here is pinned by tests that do not call it to
  * produce their expected values (hand-made cases, closed forms, a library

@@ -34,7 +34,7 @@ EXPORTS = ["tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tf
            "tfe_launch_geometry", "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
            "tfe_cache_policy_enable", "tfe_cache_select_victims", "tfe_cache_select_victims_device",
            "tfe_cache_stats", "tfe_head_create", "tfe_head_destroy", "tfe_head_topk", "tfe_head_buffers",
-           "tfe_head_status", "tfe_head_geometry", "tfe_mine_ngrams", "tfe_mine_workspace_bytes"]
+           "tfe_head_status", "tfe_head_geometry", "tfe_mine_ngrams", "tfe_mine_workspace_bytes", "tfe_assign_residency"]
 
 
 class TfeConfig(C.Structure):
@@ -110,13 +110,14 @@ def lib() -> C.CDLL:
         L.tfe_head_geometry.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
         L.tfe_mine_ngrams.argtypes = [vp, i64, i32, i32, vp, C.c_uint32, i64, vp, vp, vp, C.POINTER(i64), vp, vp, vp, i64, vp]
         L.tfe_mine_workspace_bytes.argtypes = [i64, i32]
+        L.tfe_assign_residency.argtypes = [vp, i64, i64, C.c_uint32, vp, vp, vp]
         L.tfe_mine_workspace_bytes.restype = i64
         for name in ("tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tfe_cache_install_device", "tfe_lookup_inject", "tfe_lookup_inject_host",
                      "tfe_miss_list", "tfe_miss_list_device", "tfe_index_geometry", "tfe_launch_geometry",
                      "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
                      "tfe_cache_policy_enable", "tfe_cache_select_victims", "tfe_cache_select_victims_device",
                      "tfe_cache_stats", "tfe_head_create", "tfe_head_topk", "tfe_head_buffers", "tfe_head_status",
-                     "tfe_head_geometry", "tfe_mine_ngrams"):
+                     "tfe_head_geometry", "tfe_mine_ngrams", "tfe_assign_residency"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -402,3 +403,11 @@ def tfe_mine_ngrams(tokens, L: int, vocab: int, orders, min_count: int, cap: int
                                  _addr(distinct), _addr(hist), _addr(workspace), int(workspace_bytes), _stream(stream)),
            "tfe_mine_ngrams")
     return found.value, distinct, hist
+
+
+def tfe_assign_residency(count, N: int, gpu_slots: int, host_min_count: int, init_slot, stream=None):
+    """count and init_slot on the device; returns (n_gpu, n_host, n_ssd)."""
+    tiers = np.zeros(3, np.int64)
+    _check(lib().tfe_assign_residency(_addr(count), int(N), int(gpu_slots), int(host_min_count), _addr(init_slot),
+                                      _addr(tiers), _stream(stream)), "tfe_assign_residency")
+    return tuple(int(x) for x in tiers)

@@ -262,7 +262,7 @@ tfe_mine_block_sums_kernel(MineVals v, uint32_t L, uint32_t *__restrict__ block_
 // Exclusive scan of the block totals, one block, running carry; the grand total goes to totals->found.
 __global__ void __launch_bounds__(1024)
 tfe_mine_scan_kernel(const uint32_t *__restrict__ block_sums, uint32_t n_blocks, unsigned long long *__restrict__ block_offs,
-                     MineTotals *totals)
+                     unsigned long long *total_out)
 {
     __shared__ unsigned long long s_warp[32];
     __shared__ unsigned long long s_carry;
@@ -294,7 +294,7 @@ tfe_mine_scan_kernel(const uint32_t *__restrict__ block_sums, uint32_t n_blocks,
         if (threadIdx.x == 1023) s_carry = carry + s_warp[warp] + incl;
         __syncthreads();
     }
-    if (threadIdx.x == 0) totals->found = s_carry;
+    if (threadIdx.x == 0) *total_out = s_carry;
 }
 
 // Entry e = (t, oi) in ascending (t, oi) order.  A thread owns kPosPerThread CONSECUTIVE positions here
@@ -346,6 +346,158 @@ tfe_mine_emit_kernel(MineVals v, const int32_t *__restrict__ tokens, uint32_t L,
             }
             ++pos;
         }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Initial residency from the counts (paper Sec. 4.3: the GPU tier holds the most frequently accessed entries,
+// DRAM the warm ones, SSD the long tail).  The G phrases of largest count are chosen, among equal counts the
+// smaller id first; GPU-tier slots are handed out in id order.  key = ~count turns "largest count" into
+// "smallest key": three histogram passes (11, 11, 10 bits) find the G-th smallest key and its rank r among the
+// phrases that share it; ids are memory order, so the r ties that are in are the first r in memory: per-block
+// counts of smaller keys and of ties, their scans, and one pass that numbers the chosen phrases.
+constexpr int kResidBins = 2048;
+
+struct ResidState {
+    uint32_t hist[kResidBins];
+    uint32_t prefix;                // digits of the wanted key chosen so far, in place
+    uint32_t k_rem;                 // rank (1-based) of the wanted key among those that share the prefix
+    uint32_t ticket;                // blocks done in the current pass
+    uint32_t pad;
+    unsigned long long total_gt, total_tie, n_host;
+};
+
+__global__ void __launch_bounds__(kThreads)
+tfe_resid_pass_kernel(const uint32_t *__restrict__ count, uint32_t N, int shift, int bits, uint32_t k_first, int first,
+                      ResidState *st)
+{
+    __shared__ uint32_t s_hist[kResidBins];
+    __shared__ uint32_t s_part[kThreads];
+    __shared__ uint32_t s_last;
+    for (int i = threadIdx.x; i < kResidBins; i += kThreads) s_hist[i] = 0;
+    __syncthreads();
+    const uint32_t prefix = first ? 0u : st->prefix;
+    const int above = shift + bits;
+    const uint32_t mask = (1u << bits) - 1u;
+    const uint32_t n_round = (N + 31u) & ~31u;
+    for (uint32_t i = blockIdx.x * kThreads + threadIdx.x; i < n_round; i += gridDim.x * kThreads) {
+        const uint32_t key = i < N ? ~__ldg(count + i) : 0u;
+        const bool live = i < N && (above >= 32 || (key >> above) == (prefix >> above));
+        const uint32_t digit = (key >> shift) & mask;
+        const uint32_t vote = __ballot_sync(0xFFFFFFFFu, live);
+        if (live) {
+            const uint32_t peers = __match_any_sync(vote, digit);
+            if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&s_hist[digit], __popc(peers));
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kResidBins; i += kThreads)
+        if (s_hist[i]) atomicAdd(&st->hist[i], s_hist[i]);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(&st->ticket, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    // ---- last block: the digit whose bin holds the wanted rank; the histogram is left zeroed
+    constexpr int PER = kResidBins / kThreads;
+    uint32_t mine[PER], sum = 0;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+        mine[j] = __ldcg(st->hist + threadIdx.x * PER + j);
+        st->hist[threadIdx.x * PER + j] = 0;
+        sum += mine[j];
+    }
+    s_part[threadIdx.x] = sum;
+    __syncthreads();
+    uint32_t before = 0;
+    for (int t = 0; t < (int)threadIdx.x; ++t) before += s_part[t];
+    const uint32_t want = first ? k_first : st->k_rem;
+    if (want > before && want <= before + sum) {            // exactly one thread
+        uint32_t k = want - before;
+        int j = 0;
+        for (; j < PER - 1 && mine[j] < k; ++j) k -= mine[j];
+        st->prefix = prefix | ((uint32_t)(threadIdx.x * PER + j) << shift);
+        st->k_rem = k;
+    }
+    if (threadIdx.x == 0) st->ticket = 0;
+}
+
+__global__ void __launch_bounds__(kThreads)
+tfe_resid_count_kernel(const uint32_t *__restrict__ count, uint32_t N, const ResidState *st,
+                       uint32_t *__restrict__ block_gt, uint32_t *__restrict__ block_tie)
+{
+    __shared__ uint32_t s_gt, s_tie;
+    if (threadIdx.x == 0) { s_gt = 0; s_tie = 0; }
+    __syncthreads();
+    const uint32_t key_star = st->prefix;
+    uint32_t gt = 0, tie = 0;
+    const uint32_t base = blockIdx.x * (uint32_t)kPosPerBlock;
+    for (int j = 0; j < kPosPerThread; ++j) {
+        const uint32_t i = base + j * kThreads + threadIdx.x;
+        if (i < N) {
+            const uint32_t key = ~__ldg(count + i);
+            gt += key < key_star;
+            tie += key == key_star;
+        }
+    }
+    gt = __reduce_add_sync(0xFFFFFFFFu, gt);
+    tie = __reduce_add_sync(0xFFFFFFFFu, tie);
+    if ((threadIdx.x & 31) == 0) { if (gt) atomicAdd(&s_gt, gt); if (tie) atomicAdd(&s_tie, tie); }
+    __syncthreads();
+    if (threadIdx.x == 0) { block_gt[blockIdx.x] = s_gt; block_tie[blockIdx.x] = s_tie; }
+}
+
+// A thread owns kPosPerThread consecutive ids.  chosen = smaller key, or a tie whose rank among all ties (in id
+// order) is below r; its slot is the number of chosen phrases before it.
+__global__ void __launch_bounds__(kThreads)
+tfe_resid_assign_kernel(const uint32_t *__restrict__ count, uint32_t N, ResidState *st, int any_chosen,
+                        const unsigned long long *__restrict__ gt_offs, const unsigned long long *__restrict__ tie_offs,
+                        uint32_t host_min_count, int32_t *__restrict__ init_slot)
+{
+    __shared__ uint32_t s_gt[kThreads / 32], s_tie[kThreads / 32], s_host;
+    if (threadIdx.x == 0) s_host = 0;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t key_star = st->prefix;
+    const unsigned long long r = any_chosen ? st->k_rem : 0ull;
+    const uint32_t i0 = blockIdx.x * (uint32_t)kPosPerBlock + threadIdx.x * kPosPerThread;
+    uint32_t c[kPosPerThread];
+    uint32_t gt = 0, tie = 0;
+#pragma unroll
+    for (int j = 0; j < kPosPerThread; ++j) {
+        c[j] = i0 + j < N ? __ldg(count + i0 + j) : 0u;
+        if (i0 + j < N && any_chosen) { gt += ~c[j] < key_star; tie += ~c[j] == key_star; }
+    }
+    uint32_t gi = gt, ti = tie;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t a = __shfl_up_sync(0xFFFFFFFFu, gi, o), b = __shfl_up_sync(0xFFFFFFFFu, ti, o);
+        if (lane >= o) { gi += a; ti += b; }
+    }
+    if (lane == 31) { s_gt[warp] = gi; s_tie[warp] = ti; }
+    __syncthreads();
+    unsigned long long gt_before = gt_offs[blockIdx.x] + gi - gt, tie_before = tie_offs[blockIdx.x] + ti - tie;
+    for (int w = 0; w < warp; ++w) { gt_before += s_gt[w]; tie_before += s_tie[w]; }
+    uint32_t host = 0;
+#pragma unroll
+    for (int j = 0; j < kPosPerThread; ++j) {
+        if (i0 + j >= N) break;
+        const uint32_t key = ~c[j];
+        const bool is_gt = any_chosen && key < key_star, is_tie = any_chosen && key == key_star;
+        int32_t out;
+        if (is_gt || (is_tie && tie_before < r)) {
+            out = (int32_t)(gt_before + (tie_before < r ? tie_before : r));
+        } else {
+            out = c[j] >= host_min_count ? -1 : -2;
+            host += out == -1;
+        }
+        init_slot[i0 + j] = out;
+        gt_before += is_gt;
+        tie_before += is_tie;
+    }
+    host = __reduce_add_sync(0xFFFFFFFFu, host);
+    if (lane == 0 && host) atomicAdd(&s_host, host);
+    __syncthreads();
+    if (threadIdx.x == 0 && s_host) atomicAdd(&st->n_host, (unsigned long long)s_host);
 }
 
 int bits_for(uint32_t max_value)
@@ -472,7 +624,7 @@ tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int3
     mv.n_orders = n_orders;
     for (int i = 0; i < n_orders; ++i) { mv.val[i] = val[i]; mv.n[i] = orders[i]; }
     tfe_mine_block_sums_kernel<<<n_blocks, kThreads, 0, stream>>>(mv, (uint32_t)L, block_sums);
-    tfe_mine_scan_kernel<<<1, 1024, 0, stream>>>(block_sums, n_blocks, block_offs, totals);
+    tfe_mine_scan_kernel<<<1, 1024, 0, stream>>>(block_sums, n_blocks, block_offs, &totals->found);
     tfe_mine_emit_kernel<<<n_blocks, kThreads, 0, stream>>>(mv, tokens, (uint32_t)L, block_offs, (unsigned long long)cap,
                                                           phrase_tokens, phrase_len, phrase_count);
     MCU(cudaGetLastError());
@@ -484,6 +636,56 @@ tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int3
     *n_found = (int64_t)host_totals.found;
     if (distinct) for (int i = 0; i < n_orders; ++i) distinct[i] = (int64_t)host_totals.distinct[i];
     if (hist) for (int i = 0; i < TFE_MINE_HIST_BINS; ++i) hist[i] = (int64_t)host_totals.hist[i];
+    return TFE_OK;
+}
+
+tfe_status tfe_assign_residency(const uint32_t *count, int64_t N, int64_t gpu_slots, uint32_t host_min_count,
+                                int32_t *init_slot, int64_t *tiers, void *stream_)
+{
+    if (N < 0 || N > 0x7FFFFFFFll || gpu_slots < 0 || gpu_slots > 0x7FFFFFFFll) return TFE_ERR_INVALID_ARG;
+    if (N > 0 && (!count || !init_slot)) return TFE_ERR_INVALID_ARG;
+    const int64_t G = std::min(gpu_slots, N);
+    if (tiers) { tiers[0] = G; tiers[1] = 0; tiers[2] = 0; }
+    if (N == 0) return TFE_OK;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+#define RCU(call) do { if ((call) != cudaSuccess) { (void)cudaGetLastError(); return TFE_ERR_CUDA; } } while (0)
+    const uint32_t n_blocks = (uint32_t)((N + kPosPerBlock - 1) / kPosPerBlock);
+    Carver ws;
+    const size_t bytes = sizeof(ResidState) + 256 + 2 * ((size_t)n_blocks * 4 + 256) + 2 * ((size_t)n_blocks * 8 + 256) + 256;
+    RCU(cudaMalloc(&ws.owned, bytes));
+    ws.base = ws.cur = static_cast<char *>(ws.owned);
+    ws.end = ws.base + bytes;
+    ResidState *st = ws.take<ResidState>(1);
+    uint32_t *block_gt = ws.take<uint32_t>(n_blocks), *block_tie = ws.take<uint32_t>(n_blocks);
+    unsigned long long *gt_offs = ws.take<unsigned long long>(n_blocks), *tie_offs = ws.take<unsigned long long>(n_blocks);
+    if (!st || !block_gt || !block_tie || !gt_offs || !tie_offs) return TFE_ERR_INTERNAL;
+    RCU(cudaMemsetAsync(st, 0, sizeof(ResidState), stream));
+    int dev = 0, sms = 0;
+    RCU(cudaGetDevice(&dev));
+    RCU(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>((int64_t)sms * 8, (N + kThreads - 1) / kThreads));
+    if (G > 0) {
+        static const int kShift[3] = {21, 10, 0}, kBits[3] = {11, 11, 10};
+        for (int i = 0; i < 3; ++i)
+            tfe_resid_pass_kernel<<<grid, kThreads, 0, stream>>>(count, (uint32_t)N, kShift[i], kBits[i], (uint32_t)G, i == 0, st);
+        tfe_resid_count_kernel<<<n_blocks, kThreads, 0, stream>>>(count, (uint32_t)N, st, block_gt, block_tie);
+        tfe_mine_scan_kernel<<<1, 1024, 0, stream>>>(block_gt, n_blocks, gt_offs, &st->total_gt);
+        tfe_mine_scan_kernel<<<1, 1024, 0, stream>>>(block_tie, n_blocks, tie_offs, &st->total_tie);
+    } else {
+        RCU(cudaMemsetAsync(gt_offs, 0, (size_t)n_blocks * 8, stream));
+        RCU(cudaMemsetAsync(tie_offs, 0, (size_t)n_blocks * 8, stream));
+    }
+    tfe_resid_assign_kernel<<<n_blocks, kThreads, 0, stream>>>(count, (uint32_t)N, st, G > 0 ? 1 : 0, gt_offs, tie_offs,
+                                                             host_min_count, init_slot);
+    RCU(cudaGetLastError());
+    ResidState host_state;
+    RCU(cudaMemcpyAsync(&host_state, st, sizeof host_state, cudaMemcpyDeviceToHost, stream));
+    RCU(cudaStreamSynchronize(stream));
+#undef RCU
+    // the selection must account for exactly G phrases: every smaller key plus r of the ties
+    if (G > 0 && (host_state.total_gt + host_state.k_rem != (unsigned long long)G || host_state.k_rem > host_state.total_tie))
+        return TFE_ERR_INTERNAL;
+    if (tiers) { tiers[1] = (int64_t)host_state.n_host; tiers[2] = N - G - (int64_t)host_state.n_host; }
     return TFE_OK;
 }
 

@@ -212,3 +212,12 @@ def mine_ngrams(corpus: torch.Tensor, *, vocab: int, orders, min_count: int = 2,
                                                   stream=stream)
     n = min(n_found, cap)
     return MinedPhrases(pt[:n], pl[:n], pc[:n], n_found, distinct, hist)
+
+
+def assign_residency(count: torch.Tensor, gpu_slots: int, host_min_count: int = 2, stream=None):
+    """(init_slot int32 [N] on the device, (n_gpu, n_host, n_ssd)): the gpu_slots most frequent phrases start in
+    the GPU tier (equal counts: smaller id first; slots in id order), the rest is tagged host or SSD by count."""
+    assert count.is_cuda and count.dtype == torch.int32 and count.is_contiguous()
+    init_slot = torch.empty(max(count.numel(), 1), dtype=torch.int32, device=count.device)
+    tiers = tfe.tfe_assign_residency(count, count.numel(), gpu_slots, host_min_count, init_slot, stream)
+    return init_slot[:count.numel()], tiers

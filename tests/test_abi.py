@@ -182,3 +182,11 @@ def test_new_entry_points_refuse_bad_arguments_on_the_host(tfe):
     assert mine(None, 0, 10, 2, orders.ctypes.data, 0, None, None, 0) == tfe.TFE_OK and found.value == 0   # empty corpus: no device call
     assert L.tfe_mine_workspace_bytes(-1, 2) == -1 and L.tfe_mine_workspace_bytes(16, 0) == -1
     assert L.tfe_mine_workspace_bytes(1 << 20, 3) >= (1 << 21) * 16 + 5 * 4 * (1 << 20)
+    # initial residency: refusals before any device call; N = 0 touches nothing
+    tiers = np.zeros(3, np.int64)
+    assert L.tfe_assign_residency(0x1000, -1, 4, 2, 0x1000, tiers.ctypes.data, None) == tfe.TFE_ERR_INVALID_ARG
+    assert L.tfe_assign_residency(0x1000, 1 << 31, 4, 2, 0x1000, tiers.ctypes.data, None) == tfe.TFE_ERR_INVALID_ARG
+    assert L.tfe_assign_residency(0x1000, 8, -1, 2, 0x1000, tiers.ctypes.data, None) == tfe.TFE_ERR_INVALID_ARG
+    assert L.tfe_assign_residency(None, 8, 4, 2, 0x1000, tiers.ctypes.data, None) == tfe.TFE_ERR_INVALID_ARG
+    assert L.tfe_assign_residency(0x1000, 8, 4, 2, None, tiers.ctypes.data, None) == tfe.TFE_ERR_INVALID_ARG
+    assert L.tfe_assign_residency(None, 0, 4, 2, None, tiers.ctypes.data, None) == tfe.TFE_OK and tiers.tolist() == [0, 0, 0]

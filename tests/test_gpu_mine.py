@@ -153,3 +153,60 @@ def test_mine_with_callers_workspace(orc):
         np.testing.assert_array_equal(got.hist, e_hist)
         np.testing.assert_array_equal(got.phrase_tokens.cpu().numpy(), e_pt)
         np.testing.assert_array_equal(got.count.cpu().numpy().view(np.uint32), e_pc)
+
+
+# ------------------------------------------------------------------ initial residency from the counts
+def _assign_both(orc, count, G, hm):
+    from paper_2607_07388_b200.engine import assign_residency
+    e_slot, e_tiers = orc.assign_residency(count, G, hm)
+    g_slot, g_tiers = assign_residency(torch.from_numpy(count.view(np.int32).copy()).to(DEV), G, hm)
+    assert g_tiers == e_tiers
+    np.testing.assert_array_equal(g_slot.cpu().numpy()[:len(count)], e_slot)
+    return e_slot
+
+
+@pytest.mark.parametrize("seed", range(int(os.environ.get("TFE_RANDOM_CASES", "24"))))
+def test_assign_residency_random(orc, seed):
+    rng = np.random.default_rng([6, seed])
+    N = int(rng.choice([1, 2, 31, 1023, 1024, 1025, 5000, 70_000, 300_000]))
+    kind = seed % 4
+    if kind == 0:
+        count = rng.integers(1, 4, size=N)                       # almost everything ties
+    elif kind == 1:
+        count = rng.zipf(1.5, size=N)                            # heavy tail
+    elif kind == 2:
+        count = rng.integers(0, 2**32, size=N, dtype=np.uint64)  # all 32 bits in use
+    else:
+        count = np.full(N, 7)                                    # one value
+    count = np.minimum(count, 2**32 - 1).astype(np.uint32)
+    for G in sorted({0, 1, N // 3, N - 1 if N > 1 else 1, N, N + 9}):
+        _assign_both(orc, count, int(G), int(rng.integers(0, 5)))
+
+
+def test_corpus_to_lookups_with_residency_from_counts(orc):
+    """corpus -> phrase table -> residency from the counts -> index -> lookups, every step on the device, against
+    the same chain run by the oracle on its own outputs."""
+    import parity_harness as H
+    from paper_2607_07388_b200.engine import Engram, assign_residency, bf16_tensor_from_bits, mine_ngrams
+    L, orders, d = 200_000, (2, 3, 4), 32
+    corpus = synth.make_corpus(41, L)
+    got = mine_ngrams(torch.from_numpy(corpus).to(DEV), vocab=synth.VOCAB, orders=orders, min_count=2, cap=L)
+    e_pt, e_pl, e_pc, e_found, _, _ = orc.mine_ngrams(corpus, synth.VOCAB, orders, min_count=2, cap=L)
+    N = e_found
+    C = N // 4
+    e_slot, e_tiers = orc.assign_residency(e_pc, C, host_min_count=3)
+    g_slot, g_tiers = assign_residency(got.count, C, host_min_count=3)
+    assert g_tiers == e_tiers and e_tiers[0] == C and e_tiers[1] > 0 and e_tiers[2] > 0
+    np.testing.assert_array_equal(g_slot.cpu().numpy(), e_slot)
+    rows = synth.gaussian_bf16([41, 5], (C, d), 1 / 32)
+    eng = Engram(got.phrase_tokens, got.phrase_len, g_slot, bf16_tensor_from_bits(rows, DEV), vocab=synth.VOCAB,
+                 orders=orders, device_build=True)
+    pr = H.Pair.__new__(H.Pair)
+    pr.rows_bits, pr.d, pr.C, pr.orders, pr.hidden_dtype, pr.eng = rows, d, C, orders, 0, eng
+    pr.ora = orc.Oracle(e_pt, e_pl, e_slot, rows.copy(), d=d, vocab=synth.VOCAB, orders=orders, gpu_slots=C)
+    tok = corpus[50_000:50_000 + 4 * 512].reshape(4, 512).copy()
+    h = synth.gaussian_bf16([41, 6], (4 * 512, d), 1.0)
+    _, ref, info = pr.run_and_compare(tok, h, lam=1.0)
+    assert info["n_hit"] > 300 and info["n_miss"] > 100
+    assert set(np.unique(ref.miss_tier).tolist()) == {2, 3}                   # host and SSD entries both met
+    pr.close()
