@@ -1138,7 +1138,8 @@ def run_mine(a, dev, rank):
     slots = 1024
     while slots < L + L // 2:
         slots *= 2
-    per_order = slots * 16 + L * (4 + 64 + 4) + L * (4 + 32 + 4)      # table clear; count: ids, slot read-modify-write, slot index; mark
+    # per order: table clear; count: ids + one slot read-modify-write per window; mark: table sweep + value array clear
+    per_order = slots * 16 + L * (4 + 64) + slots * 16 + L * 4
     bytes_alg = len(orders) * per_order + 2 * len(orders) * 4 * L + cap * 21
     peak, peak_src = measured_peak()
     if rank == 0:
@@ -1149,11 +1150,11 @@ def run_mine(a, dev, rank):
                        "windows": int(3 * L), "distinct": [int(x) for x in got.distinct], "phrases_out": int(cap),
                        "table_slots": slots, "workspace_bytes": tfe.tfe_mine_workspace_bytes(L, len(orders)),
                        "corpus_generation_s": gen_s,
-                       "call": "tfe_mine_ngrams with the caller's workspace: 3 x (clear, count, mark), ordered compaction, synchronise (wall clock)"},
+                       "call": "tfe_mine_ngrams with the caller's workspace: 3 x (clear, count, table sweep), ordered compaction, synchronise (wall clock)"},
             "roofline": {"bound": "hbm", "achieved": bytes_alg / sec / 1e9, "peak": peak, "unit": "GB/s",
                          "frac": bytes_alg / sec / 1e9 / peak, "traffic": None, "peak_source": peak_src,
                          "algorithmic_bytes_per_call": bytes_alg,
-                         "note": "random 32-byte sectors of the counting table dominate: 64 B per window in the count pass, 32 B in the mark pass"},
+                         "note": "random 32-byte sectors of the counting table dominate: 64 B per window in the count pass"},
             "cpu_baseline": {"value": n_pre / cpu_s, "unit": "tokens/s", "cores": 1, "kind": "oracle",
                              "sample": f"the first {n_pre} ids of the corpus (sort-based definition, single thread)"},
             "index_from_the_mined_table": built,

@@ -435,7 +435,7 @@ tfe_status tfe_head_geometry(const tfe_head *head, int32_t *grid, int32_t *rows_
  *                  yields a table of a wanted size.
  *
  *   workspace      DEVICE scratch of workspace_bytes >= tfe_mine_workspace_bytes(L, n_orders) (about 24..48
- *                  bytes per token for the counting table plus 4 bytes per token and order; smaller:
+ *                  bytes per token for the counting table plus 4 bytes per token and order (+ 1); smaller:
  *                  TFE_ERR_CAPACITY), contents undefined before and after; or NULL with workspace_bytes = 0:
  *                  the call allocates and frees it (several milliseconds per call at 10^8 tokens).
  *

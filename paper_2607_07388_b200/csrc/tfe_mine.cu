@@ -16,12 +16,11 @@
 //                           compare-and-swap on the key; equal keys are combined first inside a warp
 //                           (match.any) and inside the block (shared-memory table), then one atomicAdd on
 //                           the count and, only where it can lower it, one atomicMin on the first end
-//                           position.  The slot index is remembered for the positions that may be first.
-//   tfe_mine_mark_kernel    one thread per end position: the position that IS the first occurrence of its
-//                           tuple speaks for the tuple -- counts it as distinct, adds it to the histogram of
-//                           counts and, if the count reaches the threshold, leaves the count in the
-//                           per-position array (0 everywhere else).  The table is then reused by the next
-//                           order.
+//                           position.
+//   tfe_mine_mark_kernel    one sequential sweep over the table: every occupied slot is one distinct tuple --
+//                           counted, added to the histogram of counts and, if the count reaches the
+//                           threshold, scattered as val[first] = count into the per-position array (0
+//                           everywhere else).  The table is then reused by the next order.
 //   tfe_mine_block_sums / tfe_mine_scan / tfe_mine_emit
 //                           ordered compaction over (position, order): per-block totals, their exclusive
 //                           scan, and the writes of tuple, length and count at the scanned offsets.
@@ -87,8 +86,11 @@ __device__ __forceinline__ uint4 cas_empty_slot(MineSlot *slot, unsigned long lo
 // (match.any) and then inside the block, in a small shared-memory table {key, count, smallest t}: a frequent
 // tuple then costs the global table one update per block instead of one per warp, which is what the hot
 // slots of a Zipf-distributed corpus need.  Every distinct key of the block is then looked up / inserted in the
-// global table once (the first probes of a thread's entries are issued together), and the positions read
-// their slot back from shared memory.
+// global table once (the first probes of a thread's entries are issued together); the bigram pass of a wide
+// vocabulary also hands every position its slot back through shared memory.
+// `cand_slot` (optional, the extraction passes nullptr since its mark pass sweeps the table): the slot for the
+// positions that may be a tuple's first occurrence, kNoSlot elsewhere.  The kernel without this bookkeeping
+// compiled to 50 registers instead of 48 and ran 7 % slower, so it stays.
 constexpr int kCountWin = 2;                               // end positions per thread
 constexpr int kCountSpan = kThreads * kCountWin;           // end positions per block
 constexpr int kCountEntries = 2 * kCountSpan;              // shared-memory entries: at most half full
@@ -204,31 +206,38 @@ tfe_mine_count_kernel(const int32_t *__restrict__ tokens, uint32_t L, int32_t vo
     }
 }
 
-// val[t] = count of the tuple ending at t if t is its first occurrence and count >= min_count, else 0.
+// The table speaks for the tuples: one sequential sweep over its slots.  Every occupied slot is one distinct
+// tuple -- counted, added to the histogram of counts and, if its count reaches the threshold, written as
+// val[first] = count (val is zero everywhere else).  Sequential reads of the table and a sparse scatter
+// replace a random 16-byte read per position.
 __global__ void __launch_bounds__(kThreads)
-tfe_mine_mark_kernel(const uint32_t *__restrict__ slot_of, uint32_t L, const MineSlot *__restrict__ table,
-                     uint32_t min_count, uint32_t *__restrict__ val, MineTotals *totals, int order_index)
+tfe_mine_mark_kernel(const MineSlot *__restrict__ table, uint32_t n_slots, uint32_t min_count, uint32_t *__restrict__ val,
+                     MineTotals *totals, int order_index)
 {
     __shared__ uint32_t s_hist[TFE_MINE_HIST_BINS];
     __shared__ uint32_t s_distinct;
     for (int i = threadIdx.x; i < TFE_MINE_HIST_BINS; i += kThreads) s_hist[i] = 0;
     if (threadIdx.x == 0) s_distinct = 0;
     __syncthreads();
-    const uint32_t t = blockIdx.x * (uint32_t)kThreads + threadIdx.x;
-    if (t < L) {
-        const uint32_t s = __ldg(slot_of + t);
-        uint32_t v = 0;
-        if (s != kNoSlot) {
-            const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(table + s));     // {key lo, key hi, count - 1, first}
-            if (raw.w == t) {
-                const uint32_t count = raw.z + 1u;
-                atomicAdd(&s_distinct, 1u);
-                atomicAdd(&s_hist[min(count, (uint32_t)TFE_MINE_HIST_BINS - 1u)], 1u);
-                if (count >= min_count) v = count;
-            }
+    const int lane = threadIdx.x & 31;
+    uint32_t mine = 0;
+    const uint32_t n_round = (n_slots + 31u) & ~31u;
+    for (uint32_t s = blockIdx.x * kThreads + threadIdx.x; s < n_round; s += gridDim.x * kThreads) {
+        uint4 raw = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0, 0);
+        if (s < n_slots) raw = __ldcs(reinterpret_cast<const uint4 *>(table + s));     // {key lo, key hi, count - 1, first}
+        const bool used = (raw.x & raw.y) != 0xFFFFFFFFu;
+        const uint32_t count = raw.z + 1u;
+        // most tuples of a corpus occur once: those share one histogram update per warp
+        const uint32_t ones = __ballot_sync(0xFFFFFFFFu, used && count == 1u);
+        if (ones != 0u && lane == __ffs(ones) - 1) atomicAdd(&s_hist[1], __popc(ones));
+        if (used) {
+            ++mine;
+            if (count != 1u) atomicAdd(&s_hist[min(count, (uint32_t)TFE_MINE_HIST_BINS - 1u)], 1u);
+            if (count >= min_count) val[raw.w] = count;
         }
-        val[t] = v;
     }
+    mine = __reduce_add_sync(0xFFFFFFFFu, mine);
+    if (lane == 0 && mine) atomicAdd(&s_distinct, mine);
     __syncthreads();
     for (int i = threadIdx.x; i < TFE_MINE_HIST_BINS; i += kThreads)
         if (s_hist[i]) atomicAdd(&totals->hist[i], (unsigned long long)s_hist[i]);
@@ -533,7 +542,7 @@ int64_t workspace_bytes_for(int64_t L, int32_t n_orders)
 {
     const int64_t n_blocks = (L + kPosPerBlock - 1) / kPosPerBlock;
     const int64_t pad = 256;
-    return (int64_t)table_slots_for(L) * (int64_t)sizeof(MineSlot) + pad + (int64_t)(n_orders + 2) * (L * 4 + pad)
+    return (int64_t)table_slots_for(L) * (int64_t)sizeof(MineSlot) + pad + (int64_t)(n_orders + 1) * (L * 4 + pad)
            + n_blocks * 12 + 2 * pad + (int64_t)sizeof(MineTotals) + pad + 256;
 }
 
@@ -572,9 +581,12 @@ tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int3
     const bool composite4 = orders[n_orders - 1] == 4 && 4 * tok_bits > 63;
     const uint64_t slots = table_slots_for(L);
     const uint32_t mask = (uint32_t)(slots - 1);
-    const uint32_t n_pos_blocks = (uint32_t)((L + kThreads - 1) / kThreads);
     const uint32_t n_blocks = (uint32_t)((L + kPosPerBlock - 1) / kPosPerBlock);
     const uint32_t n_count_blocks = (uint32_t)((L + kCountSpan - 1) / kCountSpan);
+    int dev_id = 0, sms = 0;
+    MCU(cudaGetDevice(&dev_id));
+    MCU(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev_id));
+    const unsigned mark_grid = (unsigned)std::min<uint64_t>((uint64_t)sms * 8, (slots + kThreads - 1) / kThreads);
 
     Carver ws;
     if (workspace) {
@@ -588,13 +600,12 @@ tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int3
     }
     ws.cur = ws.base;
     MineSlot *table = ws.take<MineSlot>(slots);
-    uint32_t *cand_slot = ws.take<uint32_t>((size_t)L);
     uint32_t *pair_slot = composite4 ? ws.take<uint32_t>((size_t)L) : nullptr;
     uint32_t *block_sums = ws.take<uint32_t>(n_blocks);
     unsigned long long *block_offs = ws.take<unsigned long long>(n_blocks);
     MineTotals *totals = ws.take<MineTotals>(1);
     uint32_t *val[4] = {nullptr, nullptr, nullptr, nullptr};
-    bool ok = table && cand_slot && (pair_slot || !composite4) && block_sums && block_offs && totals;
+    bool ok = table && (pair_slot || !composite4) && block_sums && block_offs && totals;
     for (int i = 0; ok && i < n_orders; ++i) ok = (val[i] = ws.take<uint32_t>((size_t)L)) != nullptr;
     if (!ok) return TFE_ERR_INTERNAL;
     MCU(cudaMemsetAsync(totals, 0, sizeof(MineTotals), stream));
@@ -612,12 +623,12 @@ tfe_status tfe_mine_ngrams(const int32_t *tokens, int64_t L, int32_t vocab, int3
         const int mode = (composite4 && n == 4) ? 1 : 0;
         MCU(cudaMemsetAsync(table, 0xFF, slots * sizeof(MineSlot), stream));
         tfe_mine_count_kernel<<<n_count_blocks, kThreads, 0, stream>>>(tokens, (uint32_t)L, vocab, n, tok_bits, mode, pair_slot,
-                                                                    table, mask, keep_pairs ? pair_slot : nullptr,
-                                                                    pass < 0 ? nullptr : cand_slot, totals);
+                                                                    table, mask, keep_pairs ? pair_slot : nullptr, nullptr, totals);
         MCU(cudaGetLastError());
         if (pass < 0) continue;
-        tfe_mine_mark_kernel<<<n_pos_blocks, kThreads, 0, stream>>>(cand_slot, (uint32_t)L, table, std::max(min_count, 1u),
-                                                                   val[pass], totals, pass);
+        MCU(cudaMemsetAsync(val[pass], 0, (size_t)L * 4, stream));
+        tfe_mine_mark_kernel<<<mark_grid, kThreads, 0, stream>>>(table, (uint32_t)slots, std::max(min_count, 1u), val[pass], totals,
+                                                                 pass);
         MCU(cudaGetLastError());
     }
     MineVals mv{};
