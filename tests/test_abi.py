@@ -181,7 +181,7 @@ def test_new_entry_points_refuse_bad_arguments_on_the_host(tfe):
     assert mine(0x1000, 16, 10, 2, orders.ctypes.data, 0, None, 0x1000, 64) == tfe.TFE_ERR_CAPACITY         # workspace too small
     assert mine(None, 0, 10, 2, orders.ctypes.data, 0, None, None, 0) == tfe.TFE_OK and found.value == 0   # empty corpus: no device call
     assert L.tfe_mine_workspace_bytes(-1, 2) == -1 and L.tfe_mine_workspace_bytes(16, 0) == -1
-    assert L.tfe_mine_workspace_bytes(1 << 20, 3) >= (1 << 21) * 16 + 5 * 4 * (1 << 20)
+    assert L.tfe_mine_workspace_bytes(1 << 20, 3) >= (1 << 21) * 16 + 4 * 4 * (1 << 20)     # table + one array per order + bigram slots
     # initial residency: refusals before any device call; N = 0 touches nothing
     tiers = np.zeros(3, np.int64)
     assert L.tfe_assign_residency(0x1000, -1, 4, 2, 0x1000, tiers.ctypes.data, None) == tfe.TFE_ERR_INVALID_ARG
