@@ -71,8 +71,7 @@ struct tfe_ctx {
     std::vector<uint32_t> h_owner;
 
     int64_t ent_cap = 0;                    // capacity (entries) of the five buffers below
-    uint32_t *d_scr_phrase = nullptr;
-    uint8_t *d_scr_flag = nullptr;
+    unsigned long long *d_scr_rec = nullptr;        // one result record per (query, order column) of the last lookup
     uint32_t *d_miss_q = nullptr, *d_miss_phrase = nullptr;
     uint8_t *d_miss_tier = nullptr;
     uint32_t *d_counters = nullptr;         // TFE_CTR_WORDS words of launch state
@@ -155,19 +154,27 @@ lookup_kernel_t pick_kernel(int variant)
 // rounds of qb = ceil(Q / (warps*r)) queries gives the busiest warp r*qb queries; among the splits
 // within 8 % of the least such load the largest batch wins (fewer probe phases per warp).  Small
 // calls: one query per warp, the lowest latency.
-int pick_batch(int64_t Q, int64_t warps)
+int pick_batch(int64_t Q, int64_t warps, int max_qb = 8)
 {
     if (Q <= warps) return 1;
     int64_t load[9];
     int64_t best = INT64_MAX;
-    for (int qb = 1; qb <= 8; ++qb) {
+    for (int qb = 1; qb <= max_qb; ++qb) {
         const int64_t r = (Q + warps * qb - 1) / (warps * qb);      // rounds needed with this batch size
         load[qb] = r * qb;
         best = std::min(best, load[qb]);
     }
-    for (int qb = 8; qb >= 1; --qb)
+    for (int qb = max_qb; qb >= 1; --qb)
         if (load[qb] * 100 <= best * 108) return qb;
     return 1;
+}
+
+// Most queries a warp batch of a variant holds: the LONGEST / CONST kernels give a query two lanes per order
+// (at least four), the general kernels four.
+int max_batch(const tfe_ctx *c, int variant)
+{
+    if (variant < kVarLongest) return 8;
+    return std::min(8, 32 / std::max(4, 2 * c->cfg.n_orders));
 }
 
 TfeFastDiv make_fastdiv(uint32_t d)
@@ -255,13 +262,13 @@ tfe_status ensure_entries(tfe_ctx *c, int64_t entries)
     if (entries <= c->ent_cap) return TFE_OK;
     int64_t cap = std::max<int64_t>(entries, 1024);
     CU(cudaDeviceSynchronize());
-    free_dev(c->d_scr_phrase); free_dev(c->d_scr_flag);
+    free_dev(c->d_scr_rec);
     free_dev(c->d_miss_q); free_dev(c->d_miss_phrase); free_dev(c->d_miss_tier);
-    c->d_scr_phrase = nullptr; c->d_scr_flag = nullptr;
+    c->d_scr_rec = nullptr;
     c->d_miss_q = c->d_miss_phrase = nullptr; c->d_miss_tier = nullptr;
     c->ent_cap = 0;
-    CU(cudaMalloc(&c->d_scr_phrase, cap * 4));
-    CU(cudaMalloc(&c->d_scr_flag, cap));
+    CU(cudaMalloc(&c->d_scr_rec, cap * 8));
+    CU(cudaMemset(c->d_scr_rec, 0, cap * 8));      // tag 0: no call's record
     CU(cudaMalloc(&c->d_miss_q, cap * 4));
     CU(cudaMalloc(&c->d_miss_phrase, cap * 4));
     CU(cudaMalloc(&c->d_miss_tier, cap));
@@ -321,7 +328,7 @@ void tfe_destroy(tfe_ctx *c)
     (void)cudaSetDevice(c->device);
     (void)cudaDeviceSynchronize();
     free_dev(c->d_index); free_dev(c->d_phrase_tokens); free_dev(c->d_phrase_pos);
-    free_dev(c->d_slot_owner); free_dev(c->d_scr_phrase); free_dev(c->d_scr_flag);
+    free_dev(c->d_slot_owner); free_dev(c->d_scr_rec);
     free_dev(c->d_miss_q); free_dev(c->d_miss_phrase); free_dev(c->d_miss_tier);
     free_dev(c->d_counters);
     free_dev(c->d_inst_ids); free_dev(c->d_inst_slots); free_dev(c->d_inst_rows);
@@ -828,7 +835,7 @@ tfe_status lookup_inject_range(tfe_ctx *c, const int32_t *tokens, int32_t B, int
     if (ranged) variant += kVarRanged;
     const int64_t Qr = q_hi - q_lo;
     const int64_t resident = (int64_t)c->sm_count * c->occ[variant];
-    const int64_t qb = c->qb_override ? c->qb_override : pick_batch(Qr, resident * TFE_WARPS_PER_BLOCK);
+    const int64_t qb = c->qb_override ? std::min(c->qb_override, max_batch(c, variant)) : pick_batch(Qr, resident * TFE_WARPS_PER_BLOCK, max_batch(c, variant));
     const int64_t n_batches = (Qr + qb - 1) / qb;
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(resident, (n_batches + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK));
     TfeLookupParams p{};
@@ -843,7 +850,7 @@ tfe_status lookup_inject_range(tfe_ctx *c, const int32_t *tokens, int32_t B, int
     p.tok_bits = c->tok_bits; p.vocab = c->cfg.vocab; p.lambda = prm->lambda;
     p.lambda_bf16x2 = (lam_bits >> 16) | (lam_bits & 0xFFFF0000u);
     p.sel_phrase = sel_phrase; p.sel_slot = sel_slot; p.flags = flags;
-    p.scr_phrase = c->d_scr_phrase; p.scr_flag = c->d_scr_flag;
+    p.scr_rec = c->d_scr_rec;
     p.miss_q = c->d_miss_q; p.miss_phrase = c->d_miss_phrase; p.miss_tier = c->d_miss_tier;
     p.counters = c->d_counters;
     p.slot_stats = c->d_slot_stats; p.epoch = c->d_epoch;
@@ -979,6 +986,7 @@ tfe_status tfe_miss_list(tfe_ctx *c, uint32_t *q_idx, uint32_t *phrase_id, uint8
     uint32_t words[TFE_CTR_WORDS] = {0};
     CU(cudaMemcpyAsync(words, c->d_counters, sizeof words, cudaMemcpyDeviceToHost, stream));
     CU(cudaStreamSynchronize(stream));
+    if (words[TFE_CTR_STATUS] & TFE_DEV_RECORD_TIMEOUT) return TFE_ERR_INTERNAL;      // the closing block gave up waiting
     const int64_t n = words[TFE_CTR_TOTAL];
     *count = n;
     const int64_t take = std::min(n, cap);
@@ -1153,7 +1161,7 @@ tfe_status tfe_prefetch_candidates(tfe_ctx *c, const int32_t *history, int32_t B
 // The first call on each device asks once and remembers the answer.
 #define TFE_NOALLOC_MAX_ENTRIES 262144
 #define TFE_NOALLOC_COUNTER_BYTES 256
-#define TFE_NOALLOC_BYTES (TFE_NOALLOC_COUNTER_BYTES + TFE_NOALLOC_MAX_ENTRIES * 4 + TFE_NOALLOC_MAX_ENTRIES)
+#define TFE_NOALLOC_BYTES (TFE_NOALLOC_COUNTER_BYTES + TFE_NOALLOC_MAX_ENTRIES * 8)
 static __device__ __align__(256) unsigned char g_tfe_noalloc_scratch[TFE_NOALLOC_BYTES];
 
 namespace {
@@ -1186,15 +1194,18 @@ extern "C" tfe_status tfe_lookup_inject_noalloc(tfe_ctx *c, const int32_t *token
     }
     unsigned char *const scratch = g_noalloc_ptr[dev];
     uint32_t *const counters = reinterpret_cast<uint32_t *>(scratch);
-    // the area is shared by every call and keeps what the last one left: start the counters from zero
-    CU(cudaMemsetAsync(counters, 0, TFE_CTR_WORDS * sizeof(uint32_t), stream));
+    if (Q != 0) {                              // a refused call leaves the shared area as it was
+        if (!tokens || !h || !out) return TFE_ERR_INVALID_ARG;
+        if (((reinterpret_cast<uintptr_t>(h) | reinterpret_cast<uintptr_t>(out)) & 15u) != 0)
+            return TFE_ERR_INVALID_ARG;
+    }
+    // the area is shared by every call and keeps what the last one left: the launch state starts from zero (the
+    // count of closed calls behind it, which tags the records, carries on)
+    CU(cudaMemsetAsync(counters, 0, TFE_CTR_SEQ * sizeof(uint32_t), stream));
     if (Q == 0) {
         CU(cudaMemsetAsync(miss_count, 0, sizeof(uint32_t), stream));
         return TFE_OK;
     }
-    if (!tokens || !h || !out) return TFE_ERR_INVALID_ARG;
-    if (((reinterpret_cast<uintptr_t>(h) | reinterpret_cast<uintptr_t>(out)) & 15u) != 0)
-        return TFE_ERR_INVALID_ARG;
 
     const bool all = prm->policy == TFE_POLICY_ALL, cos = prm->gate == TFE_GATE_COSINE;
     uint32_t lam_bits;
@@ -1204,7 +1215,7 @@ extern "C" tfe_status tfe_lookup_inject_noalloc(tfe_ctx *c, const int32_t *token
     const int variant = (all || cos) ? ht * 4 + (all ? 2 : 0) + (cos ? 1 : 0)
                                      : (ht == 1 ? kVarLongestF32 : (lam_is_bf16 ? kVarLongestPacked : kVarLongest));
     const int64_t resident = (int64_t)c->sm_count * c->occ[variant];
-    const int64_t qb = c->qb_override ? c->qb_override : pick_batch(Q, resident * TFE_WARPS_PER_BLOCK);
+    const int64_t qb = c->qb_override ? std::min(c->qb_override, max_batch(c, variant)) : pick_batch(Q, resident * TFE_WARPS_PER_BLOCK, max_batch(c, variant));
     const int64_t n_batches = (Q + qb - 1) / qb;
     const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(resident, (n_batches + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK));
     TfeLookupParams p{};
@@ -1219,8 +1230,7 @@ extern "C" tfe_status tfe_lookup_inject_noalloc(tfe_ctx *c, const int32_t *token
     p.tok_bits = c->tok_bits; p.vocab = c->cfg.vocab; p.lambda = prm->lambda;
     p.lambda_bf16x2 = (lam_bits >> 16) | (lam_bits & 0xFFFF0000u);
     p.sel_phrase = sel_phrase; p.sel_slot = sel_slot; p.flags = flags;
-    p.scr_phrase = reinterpret_cast<uint32_t *>(scratch + TFE_NOALLOC_COUNTER_BYTES);
-    p.scr_flag = scratch + TFE_NOALLOC_COUNTER_BYTES + (size_t)TFE_NOALLOC_MAX_ENTRIES * 4;
+    p.scr_rec = reinterpret_cast<unsigned long long *>(scratch + TFE_NOALLOC_COUNTER_BYTES);
     p.miss_q = miss_q; p.miss_phrase = miss_phrase; p.miss_tier = miss_tier;
     p.counters = counters;
     pick_kernel(variant)<<<(unsigned)grid, TFE_BLOCK_THREADS, 0, stream>>>(p);

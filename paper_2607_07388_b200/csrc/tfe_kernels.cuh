@@ -25,6 +25,7 @@
 // device status bits (counters[TFE_CTR_STATUS])
 #define TFE_DEV_PROBE_LIMIT 2u
 #define TFE_DEV_DUP_KEY 4u
+#define TFE_DEV_RECORD_TIMEOUT 8u      // the block that closes a call gave up waiting for a block's report or a record
 
 // Division by a divisor fixed per call: q = (n * mul) >> shr, exact for every n < 2^31
 // (mul = floor(2^shr / d) + 1, shr = 31 + ceil(log2 d); the host computes both).
@@ -64,8 +65,7 @@ struct TfeLookupParams {
     uint32_t *sel_phrase;           // optional outputs
     int32_t *sel_slot;
     uint8_t *flags;
-    uint32_t *scr_phrase;           // context scratch, [Q*cols]
-    uint8_t *scr_flag;
+    unsigned long long *scr_rec;    // context scratch, [Q*cols] result records (tfe_make_record)
     uint32_t *miss_q, *miss_phrase; // context miss list, [Q*cols]
     uint8_t *miss_tier;
     uint32_t *counters;             // TFE_CTR_* words
@@ -77,7 +77,24 @@ struct TfeLookupParams {
 // atomic updates).  Blocks of a lookup add their miss counts to RUNNING and tick DONE when they finish; the block that finishes last compacts the miss list,
 // moves RUNNING to TOTAL and zeroes RUNNING / DONE for the next launch.  Because nothing of this
 // lives in kernel parameters, a launch can be replayed unchanged.
-enum { TFE_CTR_DONE = 0, TFE_CTR_RUNNING = 1, TFE_CTR_TOTAL = 2, TFE_CTR_STATUS = 3, TFE_CTR_WORDS = 4 };
+// SEQ numbers the calls that have been closed on these counters: a call's records carry SEQ + 1 (its "tag"),
+// which is how the block that builds the miss list tells a record of this call from what an earlier call left
+// in the same place.
+enum { TFE_CTR_DONE = 0, TFE_CTR_RUNNING = 1, TFE_CTR_TOTAL = 2, TFE_CTR_STATUS = 3, TFE_CTR_SEQ = 4, TFE_CTR_WORDS = 8 };
+
+// One result record per (query, order column): tag (30 bits) | flag (2 bits) | phrase id (32 bits), written with
+// a single 8-byte store, so whoever reads it sees all of it or an older record.
+#define TFE_TAG_MASK 0x3FFFFFFFu
+__device__ __forceinline__ uint32_t tfe_call_tag(const uint32_t *counters)
+{
+    const uint32_t tag = (__ldcg(counters + TFE_CTR_SEQ) + 1u) & TFE_TAG_MASK;
+    return tag ? tag : 1u;           // 0 is what fresh (zeroed) scratch memory holds: never a call's tag
+}
+__device__ __forceinline__ unsigned long long tfe_make_record(uint32_t tag, uint32_t flag, uint32_t phrase)
+{
+    return ((unsigned long long)((tag << 2) | flag) << 32) | phrase;
+}
+#define TFE_SPIN_LIMIT (1u << 22)
 
 // -------------------------------------------------------------- small helpers
 
@@ -236,56 +253,36 @@ __device__ __forceinline__ void load_memory(const uint4 *const (&rowp)[ALL ? 4 :
     }
 }
 
-// End of a lookup block.  Every thread has recorded flag bytes (and phrase ids of misses) in the
-// context scratch arrays; `my_miss` is warp-uniform.  Blocks add their miss counts to RUNNING and
-// tick DONE (one 64-bit atomic); the block that finishes last turns the flag bytes into the ordered miss list
-// (ascending entry index = ascending (q, order)), publishes TOTAL and re-arms the counters.
-__device__ __forceinline__ void tfe_finish_block(const TfeLookupParams &p, uint32_t my_miss, int cols,
-                                                 bool finalize = true)
+// The ordered miss list of a call, built by one whole block: ascending entry index = ascending (q, order).
+// `total` is the number of misses the blocks reported.  Every record is checked for this call's tag and read
+// again (bounded) while it still shows an older one: the LONGEST / CONST kernels report without a fence, so a
+// report can be seen before the records it covers.  The block then publishes TOTAL, closes the call (SEQ) and
+// re-arms the launch state.
+__device__ __forceinline__ void tfe_compact_misses(const TfeLookupParams &p, uint32_t total, int cols, uint32_t tag)
 {
-    __shared__ uint32_t s_miss, s_last, s_total, s_scan;
+    __shared__ uint32_t s_scan;
     __shared__ uint32_t s_warp[32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n_warps_blk = (blockDim.x + 31) >> 5;
-    if (threadIdx.x == 0) s_miss = 0;
+    if (threadIdx.x == 0) s_scan = 0;
     __syncthreads();
-    // ---- hand the block's miss count in; the block that finishes last builds the list
-    __threadfence();                       // this thread's flag / phrase records, device-wide
-    if (lane == 0 && my_miss) atomicAdd(&s_miss, my_miss);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        // one atomic carries both: blocks done (low word) and misses so far (high word)
-        const unsigned long long before = atomicAdd(
-            reinterpret_cast<unsigned long long *>(&p.counters[TFE_CTR_DONE]), ((unsigned long long)s_miss << 32) | 1ull);
-        s_last = (uint32_t)before == gridDim.x - 1;
-        s_total = (uint32_t)(before >> 32) + s_miss;
-        s_scan = 0;
-    }
-    __syncthreads();
-    if (!s_last) return;
-    if (!finalize) {        // a partial launch of a call issued in pieces: misses keep accumulating
-        if (threadIdx.x == 0) p.counters[TFE_CTR_DONE] = 0;
-        return;
-    }
-    __threadfence();
-    const uint32_t total = s_total;
     if (total != 0) {
-        // order-stable compaction: every thread takes 16 consecutive flag bytes per round
+        // order-stable compaction: every thread takes 4 consecutive records per round
         const uint32_t n_ent = p.Q * (uint32_t)cols;
-        const uint32_t per_round = blockDim.x * 16;
+        const uint32_t per_round = blockDim.x * 4;
         for (uint32_t e0 = 0; e0 < n_ent; e0 += per_round) {
-            const uint32_t mine = e0 + threadIdx.x * 16;
-            uint32_t w[4] = {0, 0, 0, 0};
-            if (mine + 16 <= n_ent) {
-                const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(p.scr_flag + mine));
-                w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-            } else if (mine < n_ent) {
-                for (uint32_t k = 0; mine + k < n_ent; ++k)
-                    w[k >> 2] |= (uint32_t)__ldcg(p.scr_flag + mine + k) << (8 * (k & 3));
-            }
-            uint32_t cnt = 0;                    // flags 2 and 3 have bit 1 set
+            const uint32_t mine = e0 + threadIdx.x * 4;
+            unsigned long long rec[4] = {0, 0, 0, 0};
+            uint32_t cnt = 0;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) cnt += __popc(w[k] & 0x02020202u);
+            for (int k = 0; k < 4; ++k) {
+                if (mine + k >= n_ent) continue;
+                const unsigned long long *src = p.scr_rec + mine + k;
+                rec[k] = __ldcg(src);
+                for (uint32_t spin = 0; (uint32_t)(rec[k] >> 34) != tag && spin < TFE_SPIN_LIMIT; ++spin) rec[k] = __ldcg(src);
+                if ((uint32_t)(rec[k] >> 34) != tag) { atomicOr(&p.counters[TFE_CTR_STATUS], TFE_DEV_RECORD_TIMEOUT); rec[k] = 0; }
+                cnt += (uint32_t)(rec[k] >> 33) & 1u;            // flags 2 and 3 have bit 1 set
+            }
             uint32_t incl = cnt;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -298,12 +295,11 @@ __device__ __forceinline__ void tfe_finish_block(const TfeLookupParams &p, uint3
             for (int k = 0; k < warp; ++k) off += s_warp[k];
             if (cnt) {
 #pragma unroll
-                for (int k = 0; k < 16; ++k) {
-                    const uint32_t flag = (w[k >> 2] >> (8 * (k & 3))) & 0xFFu;
+                for (int k = 0; k < 4; ++k) {
+                    const uint32_t flag = (uint32_t)(rec[k] >> 32) & 3u;
                     if (flag >= 2) {
-                        const uint32_t e = mine + k;
-                        p.miss_q[off] = e / (uint32_t)cols;
-                        p.miss_phrase[off] = __ldcg(p.scr_phrase + e);
+                        p.miss_q[off] = (mine + k) / (uint32_t)cols;
+                        p.miss_phrase[off] = (uint32_t)rec[k];
                         p.miss_tier[off] = (uint8_t)flag;
                         ++off;
                     }
@@ -322,8 +318,76 @@ __device__ __forceinline__ void tfe_finish_block(const TfeLookupParams &p, uint3
         p.counters[TFE_CTR_TOTAL] = total;
         p.counters[TFE_CTR_DONE] = 0;
         p.counters[TFE_CTR_RUNNING] = 0;
+        p.counters[TFE_CTR_SEQ] = tag;
         if (p.slot_stats != nullptr) *p.epoch = *p.epoch + 1;     // every block has read it by now
     }
+}
+
+// End of a lookup block of the general kernel.  Every thread has written its result records; `my_miss` is
+// warp-uniform.  Blocks add their miss counts to RUNNING and tick DONE (one 64-bit atomic); the block that
+// finishes last builds the miss list.
+__device__ __forceinline__ void tfe_finish_block(const TfeLookupParams &p, uint32_t my_miss, int cols, uint32_t tag)
+{
+    __shared__ uint32_t s_miss, s_last, s_total;
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) s_miss = 0;
+    __syncthreads();
+    // ---- hand the block's miss count in; the block that finishes last builds the list
+    __threadfence();                       // this thread's records, device-wide
+    if (lane == 0 && my_miss) atomicAdd(&s_miss, my_miss);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        // one atomic carries both: blocks done (low word) and misses so far (high word)
+        const unsigned long long before = atomicAdd(
+            reinterpret_cast<unsigned long long *>(&p.counters[TFE_CTR_DONE]), ((unsigned long long)s_miss << 32) | 1ull);
+        s_last = (uint32_t)before == gridDim.x - 1;
+        s_total = (uint32_t)(before >> 32) + s_miss;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    tfe_compact_misses(p, s_total, cols, tag);
+}
+
+// The LONGEST / CONST kernels take this hand-over off the end of the launch, where a fence and an atomic
+// round trip in every block sit between the last byte of one launch and the first of the next (0.85 us of the
+// 32 us the 32,768-position prefill call takes).  What the miss list needs is complete once a warp's last probe
+// is on record, well before its last row has streamed, so:
+//   * every WARP reports then (tfe_warp_probing_done): a shared-memory atomic, and from the warp that completes
+//     its block one reduction on DONE / RUNNING that nobody waits for.  No fence: records carry the call's tag
+//     and the reader checks it;
+//   * the launch's last block (tfe_closing_block_epilogue, after its own rows) waits until DONE shows every
+//     block -- all of them reported microseconds ago, unless the launch is tiny -- and builds the list.
+// Every other block leaves with its last store.  The wait is bounded; the blocks of a launch are resident
+// together (the grid never exceeds what the device holds), and a closing block that gives up says so in STATUS.
+struct TfeProbeTick { unsigned long long warps_and_misses; };      // low word: warps reported, high word: their misses
+
+__device__ __forceinline__ void tfe_warp_probing_done(const TfeLookupParams &p, TfeProbeTick *tick, uint32_t warp_miss)
+{
+    if ((threadIdx.x & 31) != 0) return;
+    const uint32_t n_warps_blk = (blockDim.x + 31) >> 5;
+    const unsigned long long before = atomicAdd(&tick->warps_and_misses, ((unsigned long long)warp_miss << 32) | 1ull);
+    if ((uint32_t)before != n_warps_blk - 1) return;
+    const unsigned long long block_miss = (before >> 32) + warp_miss;
+    unsigned long long *dst = reinterpret_cast<unsigned long long *>(&p.counters[TFE_CTR_DONE]);
+    asm volatile("red.global.add.u64 [%0], %1;" :: "l"(dst), "l"((block_miss << 32) | 1ull) : "memory");
+}
+
+__device__ __forceinline__ void tfe_closing_block_epilogue(const TfeLookupParams &p, int cols, uint32_t tag, bool finalize)
+{
+    if (blockIdx.x != gridDim.x - 1) return;
+    __shared__ uint32_t s_total;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const volatile unsigned long long *src = reinterpret_cast<const volatile unsigned long long *>(&p.counters[TFE_CTR_DONE]);
+        unsigned long long v = *src;
+        for (uint32_t spin = 0; (uint32_t)v != gridDim.x && spin < TFE_SPIN_LIMIT; ++spin) v = *src;
+        if ((uint32_t)v != gridDim.x) atomicOr(&p.counters[TFE_CTR_STATUS], TFE_DEV_RECORD_TIMEOUT);
+        s_total = (uint32_t)(v >> 32);
+        if (!finalize) p.counters[TFE_CTR_DONE] = 0;      // a partial launch of a call issued in pieces: misses keep accumulating
+    }
+    __syncthreads();
+    if (finalize) tfe_compact_misses(p, s_total, cols, tag);
 }
 
 // A GPU-tier slot served an injection in the lookup of epoch `epoch`.
@@ -384,7 +448,7 @@ __device__ __forceinline__ unsigned long long tfe_probe_lane(const TfeLookupPara
 // retained, its tier decides hit / miss, lane 4*ql records the result.  Returns (on that lane) the
 // GPU-tier slot to add, or -1.
 __device__ __forceinline__ int32_t tfe_select_longest(const TfeLookupParams &p, unsigned long long found, uint32_t q,
-                                                      bool mine, int lane, uint32_t &my_miss)
+                                                      bool mine, int lane, uint32_t &my_miss, uint32_t tag)
 {
     const uint32_t quad_found = (__ballot_sync(0xFFFFFFFFu, found != TFE_NONE64) >> (lane & ~3)) & 0xFu;
     const int top = quad_found ? 31 - __clz(quad_found) : 0;                   // greatest order that matched
@@ -400,8 +464,37 @@ __device__ __forceinline__ int32_t tfe_select_longest(const TfeLookupParams &p, 
             flag = st_ >= 0 ? 1 : (st_ == -1 ? 2 : 3);
         }
         if (flag == 1) my_slot = st_;
-        p.scr_flag[q] = (uint8_t)flag;
-        if (flag >= 2) { p.scr_phrase[q] = phrase; ++my_miss; }
+        p.scr_rec[q] = tfe_make_record(tag, flag, phrase);
+        if (flag >= 2) ++my_miss;
+        if (p.flags) p.flags[q] = (uint8_t)flag;
+        if (p.sel_phrase) p.sel_phrase[q] = phrase;
+        if (p.sel_slot) p.sel_slot[q] = st_;
+    }
+    return my_slot;
+}
+
+// The same for a query probed by the lanes base .. base + popc(group_mask) - 1 (two per order: both lanes of a
+// pair hold the pair's result); the query's first lane records.
+__device__ __forceinline__ int32_t tfe_select_longest_group(const TfeLookupParams &p, unsigned long long found, uint32_t q,
+                                                            bool mine, int base, uint32_t group_mask, bool first_lane,
+                                                            uint32_t &my_miss, uint32_t tag)
+{
+    const uint32_t group_found = (__ballot_sync(0xFFFFFFFFu, found != TFE_NONE64) >> base) & group_mask;
+    const int top = group_found ? 31 - __clz(group_found) : 0;                 // a lane of the greatest order that matched
+    const unsigned long long sel = __shfl_sync(0xFFFFFFFFu, found, base + top);
+    int32_t my_slot = -1;
+    if (first_lane && mine) {
+        uint32_t phrase = 0xFFFFFFFFu;
+        int32_t st_ = -3;
+        uint32_t flag = 0;
+        if (group_found) {
+            phrase = (uint32_t)(sel >> 32);
+            st_ = (int32_t)(uint32_t)sel;
+            flag = st_ >= 0 ? 1 : (st_ == -1 ? 2 : 3);
+        }
+        if (flag == 1) my_slot = st_;
+        p.scr_rec[q] = tfe_make_record(tag, flag, phrase);
+        if (flag >= 2) ++my_miss;
         if (p.flags) p.flags[q] = (uint8_t)flag;
         if (p.sel_phrase) p.sel_phrase[q] = phrase;
         if (p.sel_slot) p.sel_slot[q] = st_;
@@ -461,6 +554,7 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
     uint32_t my_miss = 0;                        // per thread here; summed per warp below
 
     tfe_grid_dependency_sync();
+    const uint32_t tag = tfe_call_tag(p.counters);
     const uint32_t n_warps = gridDim.x * TFE_WARPS_PER_BLOCK;
     for (uint32_t batch = blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5); batch < n_batches; batch += n_warps) {
         // query lq of batch b is b + lq * n_batches: the queries of a warp are spread over the call,
@@ -474,7 +568,7 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
         int32_t my_slot = -1;                    // GPU-tier slot this lane contributes, or -1
         float my_alpha = 0.f;
         if constexpr (!ALL) {
-            my_slot = tfe_select_longest(p, found, q, mine, lane, my_miss);
+            my_slot = tfe_select_longest(p, found, q, mine, lane, my_miss, tag);
         } else {
             const uint32_t quad_found = (__ballot_sync(0xFFFFFFFFu, found != TFE_NONE64) >> (lane & ~3)) & 0xFu;
             int n_sum = 0;                       // sum of the matched orders of this query
@@ -492,8 +586,8 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
                 }
                 if (flag == 1) { my_slot = st_; my_alpha = (float)my_order / (float)n_sum; }
                 const size_t k = (size_t)q * cols + oi;
-                p.scr_flag[k] = (uint8_t)flag;
-                if (flag >= 2) { p.scr_phrase[k] = phrase; ++my_miss; }
+                p.scr_rec[k] = tfe_make_record(tag, flag, phrase);
+                if (flag >= 2) ++my_miss;
                 if (p.flags) p.flags[k] = (uint8_t)flag;
                 if (p.sel_phrase) p.sel_phrase[k] = phrase;
                 if (p.sel_slot) p.sel_slot[k] = st_;
@@ -645,14 +739,19 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
     }
 
     my_miss = __reduce_add_sync(0xFFFFFFFFu, my_miss);
-    tfe_finish_block(p, my_miss, cols);
+    tfe_finish_block(p, my_miss, cols, tag);
 }
 
 // ------------------------------------- the hot path, LONGEST / CONST version
 //
 // The same batches, the same two phases and bit-identical results as the general kernel above
-// for the policy the benchmark grades, with the probe's three dependent steps (token ids ->
-// buckets -> stored tuple) cut down to one exposed step per batch:
+// for the policy the benchmark grades.  A probe is shared by a PAIR of lanes: each loads one 32-byte half
+// of both candidate buckets (two loads in flight per lane, 16 registers instead of 32 -- this is what
+// keeps the kernel from spilling inside its 80 registers -- and the two halves of a bucket are one line,
+// so the load unit handles half as many lines per probe), the pair then agrees by one exchange.  A query
+// takes 2 * n_orders lanes (at least 4: the four ids an n-gram can need are fetched one per lane), so a
+// batch holds up to 8 / 5 / 4 queries with <= 2 / 3 / 4 orders.  The probe's three dependent steps (token
+// ids -> buckets -> stored tuple) are cut down to one exposed step per batch:
 //   * the token ids of the NEXT batch are requested while the current batch streams (one id per
 //     lane, shared inside the quad by shuffles), so a batch starts with its ids in registers;
 //   * the stored tuple of a hashed-order match is requested but not waited for: selection runs on
@@ -673,28 +772,34 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
     const int steps = p.d / VN;                  // 16-byte steps of h per row
     const size_t hid_row_bytes = (size_t)p.d * (HT == 0 ? 2 : 4);
     const bool in_place = p.out == p.h;
-    const int ql = lane >> 2, oi = lane & 3;
+    const int lpq = max(4, 2 * p.n_orders);      // lanes per query
+    const int ql = lane / lpq, role = lane - ql * lpq, base = ql * lpq;
+    const int oi = role >> 1, half = role & 1;   // order column and bucket half of this lane's probe
     const int my_order = oi < p.n_orders ? p.orders[oi] : 0;
     const bool my_hashed = my_order > 0 && !tfe_order_is_packed(my_order, p.tok_bits);
-    const uint32_t qb = p.qb;
+    const uint32_t qb = p.qb;                    // <= 32 / lpq
     // RANGED: the call is issued in several launches, each over a query range [q_lo, q_hi)
     const uint32_t q_lo = RANGED ? p.q_lo : 0u, q_hi = RANGED ? p.q_hi : p.Q;
     const uint32_t n_batches = (q_hi - q_lo + qb - 1) / qb;
     const uint32_t n_warps = gridDim.x * TFE_WARPS_PER_BLOCK;
+    __shared__ TfeProbeTick s_tick;
+    if (threadIdx.x == 0) s_tick.warps_and_misses = 0ull;
+    __syncthreads();
     tfe_grid_dependency_sync();
+    const uint32_t tag = tfe_call_tag(p.counters);
     const uint32_t epoch = p.slot_stats != nullptr ? __ldcg(p.epoch) : 0u;
     uint32_t my_miss = 0;
 
-    // the id `oi` places before query ql of a batch, or -1 (no such position / padding id)
+    // the id `role` places before query ql of a batch (roles 0..3), or -1 (no such position / padding id)
     // Query lq of batch b is q_lo + b + lq * n_batches: a warp's queries are spread over the whole call, so
     // a run of consecutive positions that all hit (phrases overlap) is shared out among many warps
     // instead of making one warp fetch a row for every query of its batch.
     auto fetch_token = [&](uint32_t batch) -> int32_t {
         const uint32_t q = q_lo + batch + (uint32_t)ql * n_batches;
         int32_t v = -1;
-        if (batch < n_batches && ql < (int)qb && q < q_hi) {
+        if (batch < n_batches && ql < (int)qb && q < q_hi && role < 4) {
             const uint32_t b = tfe_div(q, p.div_tq);
-            const int32_t t = p.q_start + (int32_t)(q - b * (uint32_t)p.Tq) - oi;
+            const int32_t t = p.q_start + (int32_t)(q - b * (uint32_t)p.Tq) - role;
             if (t >= 0) {
                 v = __ldg(p.tokens + (size_t)b * p.T + t);
                 if ((uint32_t)v >= (uint32_t)p.vocab) v = -1;
@@ -702,16 +807,18 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
         }
         return v;
     };
-    // slot of the retained phrase if it is GPU-resident (valid on the quad's first lane), else -1
+    // slot of the retained phrase if it is GPU-resident (valid on the query's first lane), else -1
+    const uint32_t group_mask = (1u << lpq) - 1u;
     auto choose = [&](unsigned long long f) -> int32_t {
-        const uint32_t quad_found = (__ballot_sync(0xFFFFFFFFu, f != TFE_NONE64) >> (lane & ~3)) & 0xFu;
-        const int top = quad_found ? 31 - __clz(quad_found) : 0;
-        const unsigned long long sel = __shfl_sync(0xFFFFFFFFu, f, (lane & ~3) + top);
+        const uint32_t group_found = (__ballot_sync(0xFFFFFFFFu, f != TFE_NONE64) >> base) & group_mask;
+        const int top = group_found ? 31 - __clz(group_found) : 0;      // a lane of the greatest order that matched
+        const unsigned long long sel = __shfl_sync(0xFFFFFFFFu, f, base + top);
         const int32_t st_ = (int32_t)(uint32_t)sel;
-        return (oi == 0 && quad_found && st_ >= 0) ? st_ : -1;
+        return (role == 0 && group_found && st_ >= 0) ? st_ : -1;
     };
 
     uint32_t batch = blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5);
+    if (batch >= n_batches) tfe_warp_probing_done(p, &s_tick, 0u);     // a warp without queries
     int32_t tok = fetch_token(batch);
     for (; batch < n_batches; batch += n_warps) {
         const uint32_t q = q_lo + batch + (uint32_t)ql * n_batches;
@@ -720,7 +827,7 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
         // ================================ probe phase ================================
         int32_t tk[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) tk[j] = __shfl_sync(0xFFFFFFFFu, tok, (lane & ~3) + j);
+        for (int j = 0; j < 4; ++j) tk[j] = __shfl_sync(0xFFFFFFFFu, tok, base + j);
         tok = fetch_token(batch + n_warps);      // lands while this batch is processed
         bool ok = mine && my_order > 0;
 #pragma unroll
@@ -734,17 +841,20 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
             const uint64_t b2 = tfe_second_bucket_of(key, b1, p.n_buckets);
             const ulonglong4 *p1 = reinterpret_cast<const ulonglong4 *>(p.index + b1 * TFE_SLOTS_PER_BUCKET);
             const ulonglong4 *p2 = reinterpret_cast<const ulonglong4 *>(p.index + b2 * TFE_SLOTS_PER_BUCKET);
-            ulonglong4 w[4];                     // 2 buckets x 4 slots of {key, value}, all four loads in flight
-            w[0] = ld_bucket32(p1); w[1] = ld_bucket32(p1 + 1);
-            w[2] = ld_bucket32(p2); w[3] = ld_bucket32(p2 + 1);
+            ulonglong4 w[2];                     // this lane's half (2 slots of {key, value}) of both buckets, both loads in flight
+            w[0] = ld_bucket32(p1 + half); w[1] = ld_bucket32(p2 + half);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
+            for (int k = 0; k < 2; ++k) {
                 if (w[k].x == key) found = w[k].y;
                 if (w[k].z == key) found = w[k].w;
             }
-            if (my_hashed && found != TFE_NONE64) tuple = __ldg(p.phrase_tokens + (uint32_t)(found >> 32));
         }
         __syncwarp();
+        {   // the pair agrees: the key sits in at most one slot, "none" is the largest value
+            const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, found, 1);
+            found = other < found ? other : found;
+        }
+        if (my_hashed && found != TFE_NONE64) tuple = __ldg(p.phrase_tokens + (uint32_t)(found >> 32));
         const int32_t guess = choose(found);     // selection on key matches, tuples not yet compared
 
         // ---- loads of the batch's first row, issued on the guess
@@ -769,14 +879,16 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
 
         // ---- the tuples have arrived by now: final selection, tier walk, record
         if (my_hashed && found != TFE_NONE64 && !tuple_matches(tuple, tk, my_order)) found = TFE_NONE64;
-        const int32_t my_slot = tfe_select_longest(p, found, q, mine, lane, my_miss);
+        const int32_t my_slot = tfe_select_longest_group(p, found, q, mine, base, group_mask, role == 0, my_miss, tag);
         const bool redo_first = __shfl_sync(0xFFFFFFFFu, my_slot, 0) != guess0;
+        if (batch + n_warps >= n_batches)        // this warp's last probe is on record: report (its rows are still to stream)
+            tfe_warp_probing_done(p, &s_tick, __reduce_add_sync(0xFFFFFFFFu, my_miss));
 
         // ================================ gather phase ===============================
         for (uint32_t lq = 0; lq < qb; ++lq) {
             const uint32_t gq = q_lo + batch + lq * n_batches;
             if (gq >= q_hi) break;
-            const int32_t sl = __shfl_sync(0xFFFFFFFFu, my_slot, 4 * lq);
+            const int32_t sl = __shfl_sync(0xFFFFFFFFu, my_slot, lpq * (int)lq);
             if (lq > 0 || redo_first) issue_first(lq, sl);
             if (sl < 0 && in_place) continue;    // nothing to add and nothing to copy
             const char *hrow = reinterpret_cast<const char *>(p.h) + (size_t)gq * hid_row_bytes;
@@ -822,8 +934,7 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
         if (p.slot_stats != nullptr && my_slot >= 0) tfe_touch_slot(p.slot_stats, my_slot, epoch);
     }
 
-    my_miss = __reduce_add_sync(0xFFFFFFFFu, my_miss);
-    tfe_finish_block(p, my_miss, 1, !RANGED || p.finalize != 0);
+    tfe_closing_block_epilogue(p, 1, tag, !RANGED || p.finalize != 0);
 }
 
 // ------------------------------------------------------------- cache install

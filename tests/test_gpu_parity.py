@@ -225,7 +225,8 @@ def test_large_calls_all_batch_sizes(H, d, hidden, lam, orders):
         pr.run_and_compare(tok, h, lam=lam, in_place=True)
         pr.run_and_compare(tok, h[: w.B * (w.T - 2000)], lam=lam, q_start=2000, want_sel=False)
         pr.run_and_compare(tok, h, lam=lam, policy=1, gate=1)
-    assert {1, 3, 5, 8} <= seen
+    cap = min(8, 32 // max(4, 2 * len(orders)))      # a query takes two lanes per order (at least four) of the warp
+    assert {min(q, cap) for q in (1, 3, 5, 8)} <= seen
     pr.close()
 
 
