@@ -373,6 +373,46 @@ def timed_region(step, steps, warmup, stream, world, dist, dev):
     return ms, (wall0, wall1)
 
 
+def repeated_regions(step, steps, warmup, stream, world, dist, dev, min_total_ms=50.0, max_regions=400):
+    """The K-step region (timed_region) repeated until at least `min_total_ms` have been timed.
+    Returns (median region ms, {"n", "ms_min", "ms_median", "ms_max"}, wall-clock windows)."""
+    times, wins = [], []
+    while len(times) < max_regions and (not times or sum(times) < min_total_ms):
+        ms, win = timed_region(step, steps, warmup, stream, world, dist, dev)
+        times.append(ms)
+        wins.append(win)
+    stats = {"n": len(times), "ms_min": float(min(times)), "ms_median": float(np.median(times)),
+             "ms_max": float(max(times))}
+    return float(np.median(times)), stats, wins
+
+
+def workload_config(w, nbuf):
+    """The `config` both arms print: the workload and the method's parameters, nothing measured."""
+    buf_mb = nbuf * 2 * w.Q * w.d * 2 / 1e6
+    return {
+        "workload": w.name, "shape": w.shape, "B": w.B, "T": w.T, "q_start": w.q_start, "Q": w.Q,
+        "orders": list(w.orders), "n_phrases": w.n_phrases, "gpu_slots": w.gpu_slots, "d": w.d,
+        "zipf_s": w.s, "planted": w.p, "load_factor": w.load_factor, "policy": "LONGEST", "gate": "CONST",
+        "lambda": 1.0, "out_of_place": True,
+        "step": ("tfe_cache_install(4096 rows from pinned host) + tfe_lookup_inject" if w.reserve_free
+                 else "tfe_lookup_inject"),
+        "l2": f"device arm: inputs rotate over {nbuf} token/hidden/output buffer sets ({buf_mb:.0f} MB) and a "
+              f"{w.gpu_slots * w.d * 2 / 1e9:.1f} GB row table"
+              + ("; larger than the 126 MB L2" if buf_mb > 126 else
+                 "; buffers smaller than the 126 MB L2, cold_launch_us is taken after an L2 flush")
+              + "; reference arm: host memory only",
+        "parallelism": "single GPU; N > 1: replicas only",
+    }
+
+
+def kernel_source_sha():
+    """Short hash of the lookup kernels' source: a stored ncu figure is only quoted for the source it was taken on."""
+    import hashlib
+    path = os.path.join(ROOT, "paper_2607_07388_b200", "csrc", "tfe_kernels.cuh")
+    with open(path, "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:12]
+
+
 def per_launch_ms(step, n, stream, flush=None):
     """Median duration of single launches, each bracketed by its own events (optionally after an
     L2 flush: a write of a buffer larger than the 126 MB L2, outside the events)."""
@@ -478,8 +518,7 @@ def run_ours(a):
         lookup(i)
 
     warm = max(3, a.warmup)
-    direct_ms, win = timed_region(step, a.steps, warm, stream, world, dist, dev)
-    windows = [win]
+    direct_ms, direct_stats, windows = repeated_regions(step, a.steps, warm, stream, world, dist, dev)
     launch_ms, win = per_launch_ms(lookup, min(a.steps, 200), stream)
     windows.append(win)
 
@@ -488,9 +527,11 @@ def run_ours(a):
     # this is how a serving loop issues a fixed-shape step).  K = replays * G + a remainder issued
     # directly, all inside one event-bracketed region.  A workload whose step has host-side work per
     # step (c4's install plan) is timed with direct launches only.
-    ms, launch_mode = direct_ms, "direct launches"
+    ms, region_stats, launch_mode = direct_ms, direct_stats, "direct launches"
     if a.graph_steps > 0 and plan is None:
-        g_steps = max(nbuf, (a.graph_steps // nbuf) * nbuf)
+        # the graph holds the largest multiple of the buffer rotation that fits both --graph-steps and K
+        g_cap = min(a.graph_steps, a.steps)
+        g_steps = (g_cap // nbuf) * nbuf if g_cap >= nbuf else g_cap
         cap_stream = torch.cuda.Stream()
         cap_calls = sess.lookup_calls(cap_stream.cuda_stream)
         graph = torch.cuda.CUDAGraph()
@@ -508,9 +549,39 @@ def run_ours(a):
             else:
                 lookup(i)
 
-        ms, win = timed_region(graph_unit, reps + rem, 3, stream, world, dist, dev)
-        windows.append(win)
+        ms, region_stats, wins = repeated_regions(graph_unit, reps + rem, 3, stream, world, dist, dev)
+        windows.extend(wins)
         launch_mode = f"CUDA graph of {g_steps} launches replayed {reps}x + {rem} direct launches"
+
+    # ---- the yardstick: a plain streaming copy that moves as many bytes as one lookup call does (half read, half
+    # written), same launch mode, same rotation of buffers
+    copy_same = None
+    if plan is None and rank == 0:
+        half = int(sess.bytes_alg // 2) // 16 * 16
+        if half >= 16:
+            srcs = [torch.empty(half, dtype=torch.uint8, device=dev).random_() for _ in range(nbuf)]
+            dsts = [torch.empty(half, dtype=torch.uint8, device=dev) for _ in range(nbuf)]
+
+            def copy_call(i, sp_):
+                st = L.tfe_stream_copy(dsts[i % nbuf].data_ptr(), srcs[i % nbuf].data_ptr(), half, sp_)
+                if st:
+                    raise RuntimeError(f"tfe_stream_copy failed: {st}")
+
+            n_copy = max(nbuf, min(a.steps, 32) // nbuf * nbuf)
+            cstream = torch.cuda.Stream()
+            cgraph = torch.cuda.CUDAGraph()
+            torch.cuda.synchronize()
+            with torch.cuda.graph(cgraph, stream=cstream):
+                for i in range(n_copy):
+                    copy_call(i, cstream.cuda_stream)
+            c_ms, c_stats, wins = repeated_regions(lambda i: cgraph.replay(), 1, 3, stream, 1, dist, dev)
+            windows.extend(wins)
+            d_ms, _, wins = repeated_regions(lambda i: copy_call(i, sp), n_copy, 3, stream, 1, dist, dev)
+            windows.extend(wins)
+            copy_same = {"bytes_moved": 2 * half, "graph_gbs": 2 * half / (c_ms / n_copy * 1e-3) / 1e9,
+                         "direct_gbs": 2 * half / (d_ms / n_copy * 1e-3) / 1e9,
+                         "us_per_copy_graph": c_ms / n_copy * 1e3, "regions": c_stats["n"]}
+            del srcs, dsts, cgraph
     cold_ms = None
     if w.shape == "decode":      # small calls: also the cold-L2 latency of a single launch
         flush = torch.zeros(192 << 20, dtype=torch.uint8, device=dev)
@@ -560,7 +631,8 @@ def run_ours(a):
     ms_per_step = ms / a.steps
     peak, peak_src = measured_peak()
     achieved = sess.bytes_alg / (ms_per_step * 1e-3) / 1e9
-    buf_mb = nbuf * 2 * w.Q * w.d * 2 / 1e6
+    traffic = NCU_TRAFFIC.get(w.name)
+    traffic_ok = traffic is not None and traffic["kernel_source"] == kernel_source_sha()
     line = {
         "metric": "lookup+inject tokens/s",
         "value": job_throughput(w.Q, a.steps, world, ms),
@@ -572,25 +644,21 @@ def run_ours(a):
         "vs_baseline": None,
         "dtype": "bf16",
         "data": "synthetic",
-        "config": {
-            "workload": w.name, "shape": w.shape, "B": w.B, "T": w.T, "q_start": w.q_start, "Q": w.Q,
-            "orders": list(w.orders), "n_phrases": w.n_phrases, "gpu_slots": w.gpu_slots, "d": w.d,
-            "zipf_s": w.s, "planted": w.p, "load_factor": w.load_factor, "policy": "LONGEST", "gate": "CONST",
-            "lambda": 1.0, "out_of_place": True,
-            "step": ("tfe_cache_install(4096 rows from pinned host) + tfe_lookup_inject" if plan
-                     else "tfe_lookup_inject"),
-            "hit_fraction": float(np.mean(sess.hits)) / w.Q, "miss_fraction": float(np.mean(sess.misses)) / w.Q,
-            "l2": f"inputs rotate over {nbuf} token/hidden/output buffer sets ({buf_mb:.0f} MB) and a "
-                  f"{w.gpu_slots * w.d * 2 / 1e9:.1f} GB row table"
-                  + ("; larger than the 126 MB L2" if buf_mb > 126 else
-                     "; buffers smaller than the 126 MB L2, cold_launch_us is taken after an L2 flush"),
-            "parallelism": "replicas only" if world > 1 else "single GPU",
-            "grid": grid, "block": block, "batch_queries": qb, "launch": launch_mode,
-        },
+        "config": workload_config(w, nbuf),
+        "run": {"hit_fraction": float(np.mean(sess.hits)) / w.Q, "miss_fraction": float(np.mean(sess.misses)) / w.Q,
+                "grid": grid, "block": block, "batch_queries": qb, "launch": launch_mode,
+                "regions": region_stats, "direct_regions": direct_stats},
         "gathered_hbm_gbs": sess.gathered / (ms_per_step * 1e-3) / 1e9,
         "frac_of_8tbs": achieved / HBM_NOMINAL_GBS,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": NCU_TRAFFIC.get(w.name), "peak_source": peak_src,
+                     "traffic": traffic["bytes"] if traffic_ok else None,
+                     "traffic_source": (traffic["source"] if traffic_ok else
+                                        "none for this kernel source: the stored ncu capture is of another revision"
+                                        if traffic else None),
+                     "peak_source": peak_src,
+                     "copy_same_size_gbs": copy_same["graph_gbs"] if copy_same else None,
+                     "copy_same_size": copy_same,
+                     "frac_of_copy_same_size": achieved / copy_same["graph_gbs"] if copy_same else None,
                      "algorithmic_bytes_per_launch": sess.bytes_alg,
                      "kernel": "tfe_lookup_inject_longest_kernel<bf16, packed>",
                      "launch_ms_own_events": launch_ms,
@@ -1304,12 +1372,13 @@ def run_sweep(a, dev, rank):
                           "n_phrases": base.n_phrases, "peak": peak, "peak_source": peak_src, "sweep": points}))
 
 
-TFE_CTR_BYTES = 16      # the launch-state words tfe_miss_list reads back
+TFE_CTR_BYTES = 32      # the launch-state words tfe_miss_list reads back
 NBUF_DECODE = 32        # decode shapes: this many distinct query / hidden-state sets rotate
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the lookup kernel in steady state (no cache
 # flush between launches, so the write-back of the previous launch's output is included), from the ncu
 # capture summarised under profiles/; taken on a 1M-phrase table: traffic does not depend on N
-NCU_TRAFFIC = {"c3_prefill8x4096": 162_400_000}
+NCU_TRAFFIC = {"c3_prefill8x4096": {"bytes": 162_400_000, "kernel_source": "unset",
+                                    "source": "profiles/lookup_inject_longest_c3_prefill8x4096.md, steady-state capture"}}
 
 
 # ------------------------------------------------------------ reference arm
@@ -1357,8 +1426,7 @@ def run_reference(a):
         "metric": "lookup+inject tokens/s", "value": val, "unit": "tokens/s",
         "n_gpus": a.gpus, "steps": a.steps, "warmup": max(3, a.warmup), "ms_per_step": dt / a.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "shape": w.shape, "B": w.B, "T": w.T, "Q": w.Q, "orders": list(w.orders),
-                   "n_phrases": w.n_phrases, "gpu_slots": w.gpu_slots, "d": w.d, "zipf_s": w.s, "planted": w.p},
+        "config": workload_config(w, NBUF if w.shape == "prefill" else NBUF_DECODE),
         "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": orc.num_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},

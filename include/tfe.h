@@ -470,6 +470,16 @@ int64_t tfe_mine_workspace_bytes(int64_t L, int32_t n_orders);   /* -1 for inval
 tfe_status tfe_assign_residency(const uint32_t *count, int64_t N, int64_t gpu_slots, uint32_t host_min_count,
                                 int32_t *init_slot, int64_t *tiers, void *stream);
 
+/*
+ * Streaming copy (the paper has no counterpart: a yardstick for the measurements, not a step of the method).
+ * Copies `bytes` bytes from `src` to `dst` (DEVICE, 16-byte aligned, bytes a multiple of 16, ranges must not
+ * overlap) with the load / store instructions the lookup kernels stream hidden states with, one asynchronous
+ * launch on `stream`, graph-capturable.  The benchmark times it on a transfer of the lookup call's own footprint:
+ * what a plain copy of that many bytes reaches on the device is the ceiling the lookup's rate is read against.
+ * Errors: TFE_ERR_INVALID_ARG, TFE_ERR_CUDA.
+ */
+tfe_status tfe_stream_copy(void *dst, const void *src, int64_t bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

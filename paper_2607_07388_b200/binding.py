@@ -34,7 +34,7 @@ EXPORTS = ["tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tf
            "tfe_launch_geometry", "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
            "tfe_cache_policy_enable", "tfe_cache_select_victims", "tfe_cache_select_victims_device",
            "tfe_cache_stats", "tfe_head_create", "tfe_head_destroy", "tfe_head_topk", "tfe_head_buffers",
-           "tfe_head_status", "tfe_head_geometry", "tfe_mine_ngrams", "tfe_mine_workspace_bytes", "tfe_assign_residency"]
+           "tfe_head_status", "tfe_head_geometry", "tfe_mine_ngrams", "tfe_mine_workspace_bytes", "tfe_assign_residency", "tfe_stream_copy"]
 
 
 class TfeConfig(C.Structure):
@@ -112,6 +112,7 @@ def lib() -> C.CDLL:
         L.tfe_mine_workspace_bytes.argtypes = [i64, i32]
         L.tfe_assign_residency.argtypes = [vp, i64, i64, C.c_uint32, vp, vp, vp]
         L.tfe_mine_workspace_bytes.restype = i64
+        L.tfe_stream_copy.argtypes = [vp, vp, i64, vp]
         for name in ("tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tfe_cache_install_device", "tfe_lookup_inject", "tfe_lookup_inject_host",
                      "tfe_miss_list", "tfe_miss_list_device", "tfe_index_geometry", "tfe_launch_geometry",
                      "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
@@ -411,3 +412,8 @@ def tfe_assign_residency(count, N: int, gpu_slots: int, host_min_count: int, ini
     _check(lib().tfe_assign_residency(_addr(count), int(N), int(gpu_slots), int(host_min_count), _addr(init_slot),
                                       _addr(tiers), _stream(stream)), "tfe_assign_residency")
     return tuple(int(x) for x in tiers)
+
+
+def tfe_stream_copy(dst, src, nbytes: int, stream=None):
+    """Streaming device copy of nbytes (a multiple of 16) bytes: the benchmark's same-footprint yardstick."""
+    _check(lib().tfe_stream_copy(_addr(dst), _addr(src), int(nbytes), _stream(stream)), "tfe_stream_copy")

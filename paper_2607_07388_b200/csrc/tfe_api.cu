@@ -48,7 +48,7 @@ cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, c
 
 constexpr uint32_t kNoOwner = 0xFFFFFFFFu;
 constexpr int kDefaultMaxKicks = 2000;
-constexpr int kVarSlots = 16;
+constexpr int kVarSlots = 24;
 
 }  // namespace
 
@@ -132,8 +132,10 @@ typedef void (*lookup_kernel_t)(const TfeLookupParams);
 // Kernel variants.  0..7: hidden dtype x policy x gate, the general kernel in fp32 arithmetic.
 // 8..10: the LONGEST / CONST kernel -- bf16 hidden in fp32 arithmetic, bf16 hidden with the
 // packed bf16 fused multiply-add (lambda exactly a bf16 number), fp32 hidden.  11..13: the same
-// three for a call issued in several launches over query ranges (variant + kVarRanged).
-enum { kVarLongest = 8, kVarLongestPacked = 9, kVarLongestF32 = 10, kVarRanged = 3, kVarCount = 14 };
+// three for a call issued in several launches over query ranges (variant + kVarRanged).  14..19: those six
+// compiled for rows of several chunks (variant + kVarWide: half the registers in flight per lane, four blocks per SM).
+enum { kVarLongest = 8, kVarLongestPacked = 9, kVarLongestF32 = 10, kVarRanged = 3, kVarWide = 6, kVarCount = 20 };
+constexpr int kWideSteps = 384;        // 16-byte steps of h per row from which the kVarWide variants are used
 
 lookup_kernel_t pick_kernel(int variant)
 {
@@ -142,10 +144,14 @@ lookup_kernel_t pick_kernel(int variant)
         tfe_lookup_inject_kernel<0, true, false, false>,  tfe_lookup_inject_kernel<0, true, true, false>,
         tfe_lookup_inject_kernel<1, false, false, false>, tfe_lookup_inject_kernel<1, false, true, false>,
         tfe_lookup_inject_kernel<1, true, false, false>,  tfe_lookup_inject_kernel<1, true, true, false>,
-        tfe_lookup_inject_longest_kernel<0, false, false>, tfe_lookup_inject_longest_kernel<0, true, false>,
-        tfe_lookup_inject_longest_kernel<1, false, false>,
-        tfe_lookup_inject_longest_kernel<0, false, true>,  tfe_lookup_inject_longest_kernel<0, true, true>,
-        tfe_lookup_inject_longest_kernel<1, false, true>,
+        tfe_lookup_inject_longest_kernel<0, false, false, 4>, tfe_lookup_inject_longest_kernel<0, true, false, 4>,
+        tfe_lookup_inject_longest_kernel<1, false, false, 4>,
+        tfe_lookup_inject_longest_kernel<0, false, true, 4>,  tfe_lookup_inject_longest_kernel<0, true, true, 4>,
+        tfe_lookup_inject_longest_kernel<1, false, true, 4>,
+        tfe_lookup_inject_longest_kernel<0, false, false, 2>, tfe_lookup_inject_longest_kernel<0, true, false, 2>,
+        tfe_lookup_inject_longest_kernel<1, false, false, 2>,
+        tfe_lookup_inject_longest_kernel<0, false, true, 2>,  tfe_lookup_inject_longest_kernel<0, true, true, 2>,
+        tfe_lookup_inject_longest_kernel<1, false, true, 2>,
     };
     return table[variant];
 }
@@ -175,6 +181,31 @@ int max_batch(const tfe_ctx *c, int variant)
 {
     if (variant < kVarLongest) return 8;
     return std::min(8, 32 / std::max(4, 2 * c->cfg.n_orders));
+}
+
+// Launch geometry of a lookup over Qr queries: blocks and queries per warp round.
+// General kernels: warps take batches of qb queries in a grid-strided order (pick_batch above).
+// LONGEST / CONST kernels: warp w owns queries w, w + n_warps, ... (equal shares to within one query) and walks
+// them in rounds of qb: as few rounds as the lanes allow, as even as the share allows.
+void lookup_geometry(const tfe_ctx *c, int variant, int64_t Qr, int64_t *qb_out, int64_t *grid_out)
+{
+    const int64_t resident = (int64_t)c->sm_count * c->occ[variant];
+    const int64_t cap = max_batch(c, variant);
+    int64_t qb, grid;
+    if (variant >= kVarLongest) {
+        // batch size and grid as for the general kernels (few, full warps for small calls), then even shares
+        const int64_t qb0 = c->qb_override ? std::min<int64_t>(c->qb_override, cap) : pick_batch(Qr, resident * TFE_WARPS_PER_BLOCK, (int)cap);
+        const int64_t n_batches = (Qr + qb0 - 1) / qb0;
+        grid = std::max<int64_t>(1, std::min<int64_t>(resident, (n_batches + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK));
+        const int64_t share = (Qr + grid * TFE_WARPS_PER_BLOCK - 1) / (grid * TFE_WARPS_PER_BLOCK);    // queries of the busiest warp
+        const int64_t rounds = std::max<int64_t>(1, (share + qb0 - 1) / qb0);
+        qb = std::max<int64_t>(1, (share + rounds - 1) / rounds);
+    } else {
+        qb = c->qb_override ? std::min<int64_t>(c->qb_override, cap) : pick_batch(Qr, resident * TFE_WARPS_PER_BLOCK, (int)cap);
+        const int64_t n_batches = (Qr + qb - 1) / qb;
+        grid = std::max<int64_t>(1, std::min<int64_t>(resident, (n_batches + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK));
+    }
+    *qb_out = qb; *grid_out = grid;
 }
 
 TfeFastDiv make_fastdiv(uint32_t d)
@@ -577,6 +608,23 @@ tfe_status tfe_index_geometry(const tfe_ctx *c, int64_t *n_buckets, int64_t *ind
 }
 
 
+tfe_status tfe_stream_copy(void *dst, const void *src, int64_t bytes, void *stream_)
+{
+    if (bytes < 0 || (bytes & 15) != 0) return TFE_ERR_INVALID_ARG;
+    if (bytes == 0) return TFE_OK;
+    if (!dst || !src || ((reinterpret_cast<uintptr_t>(dst) | reinterpret_cast<uintptr_t>(src)) & 15u) != 0)
+        return TFE_ERR_INVALID_ARG;
+    int dev = 0, sms = 0;
+    CU(cudaGetDevice(&dev));
+    CU(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const size_t n = (size_t)bytes / 16;
+    const unsigned grid = (unsigned)std::max<size_t>(1, std::min<size_t>((size_t)sms * 16, (n + 255) / 256));
+    tfe_stream_copy_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream_)>>>(
+        static_cast<const uint4 *>(src), static_cast<uint4 *>(dst), n);
+    CU(cudaGetLastError());
+    return TFE_OK;
+}
+
 tfe_status tfe_set_tuning(tfe_ctx *c, int32_t batch_queries)
 {
     if (!c || batch_queries < 0 || batch_queries > 8) return TFE_ERR_INVALID_ARG;
@@ -833,11 +881,10 @@ tfe_status lookup_inject_range(tfe_ctx *c, const int32_t *tokens, int32_t B, int
     int variant = lookup_variant(c, prm);
     if (ranged && variant < kVarLongest) return TFE_ERR_INTERNAL;
     if (ranged) variant += kVarRanged;
+    if (variant >= kVarLongest && c->cfg.d / (c->cfg.hidden_dtype == 0 ? 8 : 4) >= kWideSteps) variant += kVarWide;
     const int64_t Qr = q_hi - q_lo;
-    const int64_t resident = (int64_t)c->sm_count * c->occ[variant];
-    const int64_t qb = c->qb_override ? std::min(c->qb_override, max_batch(c, variant)) : pick_batch(Qr, resident * TFE_WARPS_PER_BLOCK, max_batch(c, variant));
-    const int64_t n_batches = (Qr + qb - 1) / qb;
-    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(resident, (n_batches + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK));
+    int64_t qb, grid;
+    lookup_geometry(c, variant, Qr, &qb, &grid);
     TfeLookupParams p{};
     p.tokens = tokens; p.B = B; p.T = T; p.q_start = q_start; p.Tq = (int32_t)Tq; p.Q = (uint32_t)Q;
     p.div_tq = make_fastdiv((uint32_t)Tq); p.qb = (uint32_t)qb;
@@ -1207,17 +1254,12 @@ extern "C" tfe_status tfe_lookup_inject_noalloc(tfe_ctx *c, const int32_t *token
         return TFE_OK;
     }
 
-    const bool all = prm->policy == TFE_POLICY_ALL, cos = prm->gate == TFE_GATE_COSINE;
     uint32_t lam_bits;
     std::memcpy(&lam_bits, &prm->lambda, sizeof lam_bits);
-    const bool lam_is_bf16 = (lam_bits & 0xFFFFu) == 0 && (lam_bits & 0x7F800000u) != 0x7F800000u;
-    const int ht = c->cfg.hidden_dtype;
-    const int variant = (all || cos) ? ht * 4 + (all ? 2 : 0) + (cos ? 1 : 0)
-                                     : (ht == 1 ? kVarLongestF32 : (lam_is_bf16 ? kVarLongestPacked : kVarLongest));
-    const int64_t resident = (int64_t)c->sm_count * c->occ[variant];
-    const int64_t qb = c->qb_override ? std::min(c->qb_override, max_batch(c, variant)) : pick_batch(Q, resident * TFE_WARPS_PER_BLOCK, max_batch(c, variant));
-    const int64_t n_batches = (Q + qb - 1) / qb;
-    const int64_t grid = std::max<int64_t>(1, std::min<int64_t>(resident, (n_batches + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK));
+    int variant = lookup_variant(c, prm);
+    if (variant >= kVarLongest && c->cfg.d / (c->cfg.hidden_dtype == 0 ? 8 : 4) >= kWideSteps) variant += kVarWide;
+    int64_t qb, grid;
+    lookup_geometry(c, variant, Q, &qb, &grid);
     TfeLookupParams p{};
     p.tokens = tokens; p.B = B; p.T = T; p.q_start = q_start; p.Tq = (int32_t)Tq; p.Q = (uint32_t)Q;
     p.div_tq = make_fastdiv((uint32_t)Tq); p.qb = (uint32_t)qb;

@@ -98,17 +98,48 @@ __device__ __forceinline__ unsigned long long tfe_make_record(uint32_t tag, uint
 
 // -------------------------------------------------------------- small helpers
 
+#ifndef TFE_LD_MODE
+#define TFE_LD_MODE 2
+#endif
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p)   // touched once: do not keep in L1
 {
     uint4 v;
+#if TFE_LD_MODE == 0
     asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+#elif TFE_LD_MODE == 1
+    asm volatile("ld.global.L1::no_allocate.L2::evict_first.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+#elif TFE_LD_MODE == 2
+    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+#elif TFE_LD_MODE == 3
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+#endif
     return v;
 }
+#ifndef TFE_ST_MODE
+#define TFE_ST_MODE 0
+#endif
 __device__ __forceinline__ void st_stream(uint4 *p, uint4 v)
 {
+#if TFE_ST_MODE == 0
     asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};"
                  :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+#elif TFE_ST_MODE == 1
+    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+#elif TFE_ST_MODE == 2
+    asm volatile("st.global.cg.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+#elif TFE_ST_MODE == 3
+    asm volatile("st.global.wt.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+#elif TFE_ST_MODE == 4
+    asm volatile("st.global.L1::no_allocate.L2::evict_last.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+#endif
 }
 __device__ __forceinline__ uint4 ld_row(const uint4 *p)      // read-only table data
 {
@@ -377,8 +408,7 @@ __device__ __forceinline__ void tfe_closing_block_epilogue(const TfeLookupParams
 {
     if (blockIdx.x != gridDim.x - 1) return;
     __shared__ uint32_t s_total;
-    __syncthreads();
-    if (threadIdx.x == 0) {
+    if (threadIdx.x == 0) {                      // as soon as the first warp is through: the wait overlaps the other warps' rows
         const volatile unsigned long long *src = reinterpret_cast<const volatile unsigned long long *>(&p.counters[TFE_CTR_DONE]);
         unsigned long long v = *src;
         for (uint32_t spin = 0; (uint32_t)v != gridDim.x && spin < TFE_SPIN_LIMIT; ++spin) v = *src;
@@ -760,12 +790,14 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
 //     phrases with one 64-bit key cannot both be in the table, so this means the n-gram is not a
 //     phrase) simply repeats the first row's loads with the corrected choice; nothing has been
 //     stored before that point, in place or not.
-template <int HT, bool PACKED, bool RANGED>
-__global__ void __launch_bounds__(TFE_BLOCK_THREADS, TFE_MIN_BLOCKS)
+// UNROLL: 16-byte vectors of h (and of the row) a lane holds at a time.  4: a 1,024-element row is in flight whole,
+// 80 registers, three blocks per SM.  2: 64 registers, four blocks per SM -- for rows of several chunks, where
+// a warp walks chunk after chunk and a third more warps pays (8 KB rows: 278 -> 254 us per 65,536-token call).
+template <int HT, bool PACKED, bool RANGED, int UNROLL>
+__global__ void __launch_bounds__(TFE_BLOCK_THREADS, UNROLL == 4 ? TFE_MIN_BLOCKS : TFE_MIN_BLOCKS + 1)
 tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
 {
     constexpr int VN = TfeVec<HT>::N;
-    constexpr int UNROLL = 4;
     static_assert(!PACKED || HT == 0, "packed bf16 path needs bf16 hidden states");
 
     const int lane = threadIdx.x & 31;
@@ -780,8 +812,13 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
     const uint32_t qb = p.qb;                    // <= 32 / lpq
     // RANGED: the call is issued in several launches, each over a query range [q_lo, q_hi)
     const uint32_t q_lo = RANGED ? p.q_lo : 0u, q_hi = RANGED ? p.q_hi : p.Q;
-    const uint32_t n_batches = (q_hi - q_lo + qb - 1) / qb;
+    // Work split: warp w of the launch owns the queries q_lo + w + k * n_warps, k = 0 .. cnt-1: every warp gets the
+    // same number of queries to within one, neighbouring positions go to neighbouring warps (a run of consecutive
+    // positions that all hit -- overlapping phrases -- is shared out among many warps, and the rows that are in
+    // flight at one time lie close together).  A warp walks its queries in rounds of qb.
     const uint32_t n_warps = gridDim.x * TFE_WARPS_PER_BLOCK;
+    const uint32_t q_first = q_lo + blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5);
+    const uint32_t cnt = q_first < q_hi ? (q_hi - q_first + n_warps - 1) / n_warps : 0u;
     __shared__ TfeProbeTick s_tick;
     if (threadIdx.x == 0) s_tick.warps_and_misses = 0ull;
     __syncthreads();
@@ -790,14 +827,13 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
     const uint32_t epoch = p.slot_stats != nullptr ? __ldcg(p.epoch) : 0u;
     uint32_t my_miss = 0;
 
-    // the id `role` places before query ql of a batch (roles 0..3), or -1 (no such position / padding id)
-    // Query lq of batch b is q_lo + b + lq * n_batches: a warp's queries are spread over the whole call, so
-    // a run of consecutive positions that all hit (phrases overlap) is shared out among many warps
-    // instead of making one warp fetch a row for every query of its batch.
-    auto fetch_token = [&](uint32_t batch) -> int32_t {
-        const uint32_t q = q_lo + batch + (uint32_t)ql * n_batches;
+    // the id `role` places before this lane's query of the round that starts at the warp's query k0 (roles 0..3),
+    // or -1 (no such query / position / padding id)
+    auto fetch_token = [&](uint32_t k0) -> int32_t {
+        const uint32_t k = k0 + (uint32_t)ql;
         int32_t v = -1;
-        if (batch < n_batches && ql < (int)qb && q < q_hi && role < 4) {
+        if (ql < (int)qb && k < cnt && role < 4) {
+            const uint32_t q = q_first + k * n_warps;
             const uint32_t b = tfe_div(q, p.div_tq);
             const int32_t t = p.q_start + (int32_t)(q - b * (uint32_t)p.Tq) - role;
             if (t >= 0) {
@@ -817,18 +853,17 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
         return (role == 0 && group_found && st_ >= 0) ? st_ : -1;
     };
 
-    uint32_t batch = blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5);
-    if (batch >= n_batches) tfe_warp_probing_done(p, &s_tick, 0u);     // a warp without queries
-    int32_t tok = fetch_token(batch);
-    for (; batch < n_batches; batch += n_warps) {
-        const uint32_t q = q_lo + batch + (uint32_t)ql * n_batches;
-        const bool mine = ql < (int)qb && q < q_hi;
+    if (cnt == 0) tfe_warp_probing_done(p, &s_tick, 0u);     // a warp without queries
+    int32_t tok = fetch_token(0);
+    for (uint32_t k0 = 0; k0 < cnt; k0 += qb) {
+        const uint32_t q = q_first + (k0 + (uint32_t)ql) * n_warps;
+        const bool mine = ql < (int)qb && k0 + (uint32_t)ql < cnt;
 
         // ================================ probe phase ================================
         int32_t tk[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) tk[j] = __shfl_sync(0xFFFFFFFFu, tok, base + j);
-        tok = fetch_token(batch + n_warps);      // lands while this batch is processed
+        tok = fetch_token(k0 + qb);              // lands while this round is processed
         bool ok = mine && my_order > 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j)
@@ -861,7 +896,7 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
         uint4 hv[UNROLL];
         typename TfeVec<HT>::RowRaw rv[UNROLL];
         auto issue_first = [&](uint32_t lq, int32_t sl) {
-            const char *hrow = reinterpret_cast<const char *>(p.h) + (size_t)(q_lo + batch + lq * n_batches) * hid_row_bytes;
+            const char *hrow = reinterpret_cast<const char *>(p.h) + (size_t)(q_first + (k0 + lq) * n_warps) * hid_row_bytes;
             const uint4 *rowp = p.rows + (size_t)(sl >= 0 ? sl : 0) * (size_t)(p.d / 8);
             if (sl >= 0 || !in_place) {
 #pragma unroll
@@ -881,13 +916,13 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
         if (my_hashed && found != TFE_NONE64 && !tuple_matches(tuple, tk, my_order)) found = TFE_NONE64;
         const int32_t my_slot = tfe_select_longest_group(p, found, q, mine, base, group_mask, role == 0, my_miss, tag);
         const bool redo_first = __shfl_sync(0xFFFFFFFFu, my_slot, 0) != guess0;
-        if (batch + n_warps >= n_batches)        // this warp's last probe is on record: report (its rows are still to stream)
+        if (k0 + qb >= cnt)                      // this warp's last probe is on record: report (its rows are still to stream)
             tfe_warp_probing_done(p, &s_tick, __reduce_add_sync(0xFFFFFFFFu, my_miss));
 
         // ================================ gather phase ===============================
-        for (uint32_t lq = 0; lq < qb; ++lq) {
-            const uint32_t gq = q_lo + batch + lq * n_batches;
-            if (gq >= q_hi) break;
+        const uint32_t n_round = min(qb, cnt - k0);
+        for (uint32_t lq = 0; lq < n_round; ++lq) {
+            const uint32_t gq = q_first + (k0 + lq) * n_warps;
             const int32_t sl = __shfl_sync(0xFFFFFFFFu, my_slot, lpq * (int)lq);
             if (lq > 0 || redo_first) issue_first(lq, sl);
             if (sl < 0 && in_place) continue;    // nothing to add and nothing to copy
@@ -934,7 +969,26 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
         if (p.slot_stats != nullptr && my_slot >= 0) tfe_touch_slot(p.slot_stats, my_slot, epoch);
     }
 
+#ifndef TFE_HACK_NOCLOSE
     tfe_closing_block_epilogue(p, 1, tag, !RANGED || p.finalize != 0);
+#endif
+}
+
+// ------------------------------------------------------------ streaming copy
+//
+// A plain grid-stride copy with the instructions the lookup kernels stream hidden states with; the benchmark's
+// yardstick for "what a copy of this many bytes reaches".
+__global__ void __launch_bounds__(256) tfe_stream_copy_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, size_t n)
+{
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (; i + 3 * stride < n; i += 4 * stride) {
+        const uint4 v0 = ld_stream(src + i), v1 = ld_stream(src + i + stride), v2 = ld_stream(src + i + 2 * stride),
+                    v3 = ld_stream(src + i + 3 * stride);
+        st_stream(dst + i, v0); st_stream(dst + i + stride, v1); st_stream(dst + i + 2 * stride, v2);
+        st_stream(dst + i + 3 * stride, v3);
+    }
+    for (; i < n; i += stride) st_stream(dst + i, ld_stream(src + i));
 }
 
 // ------------------------------------------------------------- cache install
