@@ -115,9 +115,15 @@ class Pair:
                 mag = np.maximum(np.maximum(np.abs(a), np.abs(b)), 2.0 ** -126)
                 ulp = np.ldexp(1.0, np.floor(np.log2(mag)).astype(np.int64) - 7)
                 assert (np.abs(a - b) <= ulp).all(), float((np.abs(a - b) / ulp).max())
-            # aggregation / cosine gate run in fp32 on the GPU and fp64 in the oracle: the absolute
-            # tolerance above is the contract; most elements still round to the same bf16
-            assert n_diff <= max(2, out.size // 20), n_diff
+            # Side check beside the contract (the absolute tolerance above): how many elements round to another
+            # bf16 number than the oracle's single rounding of the exact value.  Two sources: fp32 aggregation /
+            # gate arithmetic against fp64 (a relative error near 1e-6 moves a result across a bf16 rounding
+            # boundary, 2^-9 relative, about once in 10^4 elements), and the fp32-then-bf16 double rounding
+            # of h + lambda*m for a lambda that is no bf16 number (procedural rows are small integers times a
+            # power of two, so exact ties are common).  Over 881 such cases of 300 random configurations per
+            # test the most seen was 0.85 % of the injected elements; 1 % is the budget.
+            n_injected = int(touched.sum()) * out.shape[1]
+            assert n_diff <= max(2, n_injected // 100), (n_diff, n_injected)
         return got, ref, dict(max_abs_err=float(err), n_bits_differ=n_diff, n_hit=int(touched.sum()),
                               n_miss=int(cnt))
 
@@ -134,13 +140,13 @@ class BigPair:
     looked up lazily by the oracle through a sparsely committed host mapping, so nothing the size
     of the table ever sits in host memory."""
 
-    def __init__(self, w: synth.Workload, table=None):
+    def __init__(self, w: synth.Workload, table=None, device_build=False):
         self.w = w
         self.tb = table if table is not None else synth.make_table(w)
         self.rows_gpu = torch.empty((w.gpu_slots, w.d), dtype=torch.bfloat16, device=DEV)
         synth.fill_rows_torch(self.rows_gpu, torch.from_numpy(synth.slot_owner_of(self.tb)).to(DEV))
         self.eng = Engram(self.tb.phrase_tokens, self.tb.phrase_len, self.tb.init_slot, self.rows_gpu,
-                          vocab=w.vocab, orders=w.orders, load_factor=w.load_factor)
+                          vocab=w.vocab, orders=w.orders, load_factor=w.load_factor, device_build=device_build)
         self.sparse = synth.SparseRows(w.gpu_slots, w.d)
         self.ora = orc.Oracle(self.tb.phrase_tokens, self.tb.phrase_len, self.tb.init_slot, self.sparse.array,
                               d=w.d, vocab=w.vocab, orders=w.orders, gpu_slots=w.gpu_slots)

@@ -101,6 +101,78 @@ def test_config4_install_then_lookup(H):
     bp.close()
 
 
+def test_config5_full_table_65536_tokens(H):
+    """The sweep's table at its stated size (8,000,000 phrases, all GPU-resident) and its two heaviest points:
+    65,536 tokens per call at 90 % hits with 2 KB and with 8 KB rows (16 GB and 66 GB of rows on the device; the
+    8 KB rows run the kernel's wide-row variant).  Integer outputs and the miss list on every query, hidden
+    states on 4,096 seeded rows."""
+    base = synth.config(5)
+    assert base.n_phrases == 8_000_000 and base.gpu_slots == 8_000_000
+    table = synth.make_table(base)
+    for d in (1024, 4096):
+        w = synth.config(5, d=d, B=65536, p=0.9)
+        bp = H.BigPair(w, table=table, device_build=(d == 4096))
+        info = bp.check(synth.make_queries(w, table), sample_rows=4096)
+        assert info["Q"] == 65536 and abs(info["n_hit"] / 65536 - 0.9) < 0.03
+        hit_slots = info["ref"].sel_slot[info["ref"].flags == 1]
+        assert int(hit_slots.max()) * d * 2 > (1 << 33)          # row offsets beyond 8 GB are reached
+        bp.close()
+        del bp
+        torch.cuda.empty_cache()
+
+
+def test_config4_full_size_install_then_lookup(H):
+    """Config 4 at its stated size: 32,000,000 phrases, 16,777,216 GPU-tier slots (34 GB of rows), the last
+    262,144 slots free at the start, the rest of the table tagged host / SSD.  Three steps of decode batch
+    256: two install 4,096 fetched rows from pinned host memory into free slots (the first batch takes the
+    highest slots, its first phrase the very last one), the third overwrites occupied slots and so demotes
+    their owners.  Every lookup is checked against the oracle on all outputs."""
+    w = synth.config(4)
+    assert w.n_phrases == 32_000_000 and w.gpu_slots == 16_777_216 and w.reserve_free == 262_144
+    bp = H.BigPair(w)
+    ora, eng = bp.ora, bp.eng
+    rng = np.random.default_rng(45)
+    free = np.nonzero(ora.slot_owner < 0)[0].astype(np.int32)
+    assert len(free) == w.reserve_free and free[-1] == w.gpu_slots - 1
+    n_install, top = 4096, w.gpu_slots - 1
+    saw_far_slot = False
+    for step in range(3):
+        tok = synth.make_queries(w, bp.tb, variant=step)
+        before = ora.lookup(tok, w.q_start)
+        take = np.unique(before.miss_phrase)
+        take = take[: max(1, len(take) // 2)]
+        pool = np.nonzero(ora.slot_state < 0)[0]
+        extra = rng.choice(pool, 2 * n_install, replace=False).astype(np.uint32)
+        ids = np.concatenate([take, np.setdiff1d(extra, take)])[:n_install].astype(np.uint32)
+        if step == 0:
+            dst = free[::-1][:n_install].copy()              # highest free slots first: ids[0] goes into the top slot
+        elif step == 1:
+            dst = free[:n_install].copy()
+        else:                                                # occupied slots: their owners fall back to the host tier
+            occ = np.nonzero(ora.slot_owner >= 0)[0]
+            dst = rng.choice(occ, n_install, replace=False).astype(np.int32)
+            demoted = ora.slot_owner[dst].copy()
+        pinned = torch.from_numpy(synth.phrase_rows_np(w, ids).view(np.int16)).pin_memory()
+        eng.cache_install(ids, pinned, dst)
+        assert ora.cache_install(ids, None, dst) == 0
+        info = bp.check(tok, variant=step)
+        after = info["ref"]
+        assert info["Q"] == 256 and not np.isin(after.miss_phrase, take).any()
+        assert info["n_hit"] >= (before.flags == 1).sum() + 1
+        if step == 0:                                        # the phrase in the top slot is a hit at the last row of the table
+            assert (after.sel_slot[after.sel_phrase == ids[0]] == top).all() and (after.sel_phrase == ids[0]).any()
+        if step == 2:
+            assert (ora.slot_state[demoted] == -1).all()
+        saw_far_slot |= bool((after.sel_slot[after.flags == 1] >= (1 << 23)).any())
+    assert saw_far_slot                                      # rows beyond 16 GB into the table were gathered
+    pick = np.sort(rng.choice(np.nonzero(ora.slot_owner >= 0)[0], 2048, replace=False))
+    pick[-1] = top
+    want = synth.procedural_bf16_np(ora.slot_owner[pick], w.d, synth.ROW_TAG, synth.ROW_SHIFT)
+    got = H.bits_from_bf16_tensor(bp.rows_gpu[torch.from_numpy(pick).to(H.DEV)])
+    np.testing.assert_array_equal(got, want)
+    bp.close()
+
+
 def test_millions_of_positions_narrow_rows(H):
     """The largest calls: millions of query positions in one launch (32-bit position arithmetic, the
     division by the sequence length, a miss list of hundreds of thousands of entries), rows of 8
