@@ -77,8 +77,8 @@ typedef struct {
 
 /*
  * tfe_index_build -- build the exact-match phrase index and the per-phrase
- * metadata (paper Sec. 4.2: two-level index "token prefix -> phrase id ->
- * memory address", metadata = length, vector address, storage tier).
+ * metadata (paper Sec. 4.2: an index in two levels, from token prefixes to phrase ids and from
+ * phrase ids to memory addresses; per phrase its length, the address of its vector, its tier).
  *
  *   cfg            HOST.
  *   phrase_tokens  HOST int32 [N][4]; phrase i is the first phrase_len[i] entries, the rest -1.
@@ -233,8 +233,8 @@ tfe_status tfe_miss_list(tfe_ctx *ctx, uint32_t *q_idx, uint32_t *phrase_id, uin
  * a larger call arrives.  A runtime that has given all free device memory to its own pool, or a
  * latency-critical loop that cannot tolerate the device-wide synchronisation an allocation or a
  * free brings, calls this instead: it allocates and frees nothing, on the host or on the device.
- * Its scratch is a fixed area inside the loaded library image (about 1.3 MB, present on every GPU
- * that loads the library until the process ends), which bounds the call:
+ * Its scratch is a fixed area inside the loaded library image (2 MiB: one 8-byte result record per
+ * entry; present on every GPU that loads the library until the process ends), which bounds the call:
  *
  *     Q * (policy == ALL ? n_orders : 1)  <=  262,144      otherwise TFE_ERR_CAPACITY.
  *
@@ -247,9 +247,11 @@ tfe_status tfe_miss_list(tfe_ctx *ctx, uint32_t *q_idx, uint32_t *phrase_id, uin
  *
  * The context's device must be the current device.  The first call on a device looks up the
  * address of the scratch area (cudaGetSymbolAddress); make that first call outside any stream
- * capture.  All calls on one device share the area, whatever their context: a call clears what
- * must start at zero and the stream orders it, but two calls that overlap on the GPU (different
- * streams, no dependency) race.  Results are those of tfe_lookup_inject.
+ * capture.  All calls on one device share the area, whatever their context, and it keeps what the
+ * last call left: a call puts the launch state back to zero on its stream (a call refused for its
+ * arguments touches nothing), and records carry the number of the call that wrote them, so a record
+ * left by an earlier call is never taken for one of this call.  Two calls that overlap on the GPU
+ * (different streams, no dependency) race.  Results are those of tfe_lookup_inject.
  * Errors: INVALID_ARG, CAPACITY, CUDA.
  */
 tfe_status tfe_lookup_inject_noalloc(tfe_ctx *ctx, const int32_t *tokens, int32_t B, int32_t T,
@@ -264,9 +266,9 @@ tfe_status tfe_miss_list_device(tfe_ctx *ctx, const uint32_t **q_idx, const uint
                                 const uint8_t **tier, const uint32_t **count);
 
 /*
- * GPU-tier retention ranking (paper Sec. 4.3: "TF-Engram can rank memory entries using access
- * frequency, recency, ..." -- the signals are the paper's, it gives no formula; the ranking below
- * is this library's reading).
+ * GPU-tier retention ranking (paper Sec. 4.3 names the signals an implementation may rank entries by --
+ * access frequency and recency among them -- and gives no formula; the ranking below is this
+ * library's reading).
  *
  * tfe_cache_policy_enable -- starts the bookkeeping: from now on every lookup of this context
  * (tfe_lookup_inject, tfe_lookup_inject_host; not tfe_lookup_inject_noalloc) adds 1 to `freq` and
@@ -317,12 +319,11 @@ typedef struct {
 
 /*
  * tfe_prefetch_candidates -- candidate phrase expansion and priority for early-exit guided
- * prefetching (paper Sec. 4.4: the top-K predicted tokens "are combined with the recent token
- * history to infer possible future phrases", mapped through the token-to-phrase index to the
- * candidate set Q_t; each candidate gets the priority s_i = p_i * r_i * c_i and "high-priority
- * candidates are prefetched first, while low-priority candidates are dropped when the I/O budget
- * or queue capacity is exhausted").  The early-exit head itself (projection + top-K) is not part
- * of this library: its top-K tokens and probabilities are inputs.
+ * prefetching (paper Sec. 4.4: each predicted token is put behind the sequence's recent history, the
+ * n-grams that result are looked up in the token-to-phrase index and give the candidate set Q_t;
+ * a candidate's priority is s_i = p_i * r_i * c_i, and the budget goes to the highest priorities,
+ * the rest is dropped).  The top-K tokens and their probabilities are inputs: they come from the
+ * early-exit head, tfe_head_topk below, or from anywhere else.
  *
  *   history      DEVICE int32 [B][H]: the last H tokens of every sequence (H >= n_max - 1 to let
  *                every order contribute; an order n with n - 1 > H contributes nothing).
@@ -354,11 +355,11 @@ const char *tfe_last_cuda_error(void);
 
 /*
  * Introspection used by tests and the benchmark (HOST only, no device work).
- *   tfe_index_geometry  buckets of 8 slots, bytes of the device index, bytes of per-phrase metadata.
+ *   tfe_index_geometry  buckets (of 4 slots of 16 bytes), bytes of the device index, bytes of per-phrase metadata.
  *   tfe_phrase_key64    the 64-bit index key of a token tuple (0 if n or a token is invalid) and
  *                       whether that order is packed injectively (exact) or hashed + verified.
  *   tfe_home_bucket     the first bucket probed for a key.
- *   tfe_launch_geometry grid size, block size and queries per warp batch of the last lookup.
+ *   tfe_launch_geometry grid size, block size and queries per warp round of the last lookup.
  */
 tfe_status tfe_index_geometry(const tfe_ctx *ctx, int64_t *n_buckets, int64_t *index_bytes,
                               int64_t *metadata_bytes);

@@ -17,7 +17,7 @@
  *   - aggregation  m_t = sum_i alpha_i e_i                    [Sec. 2.2 aggregation eq.; Sec. 4.2 e_phi eq.]
  *   - gated residual injection  h'_t = h_t + g_t * m_t        [Sec. 2.2 injection eq.]
  *   - list of matched-but-not-GPU-resident phrases            [Sec. 4.3, staged / asynchronous reads]
- *   - insertion of fetched entries into the GPU tier          [Sec. 4.3, "inserts the entry into a faster tier"]
+ *   - insertion of fetched entries into the GPU tier          [Sec. 4.3, promotion of a fetched entry into a faster tier]
  *   - prefetch candidates from predicted tokens + priority     [Sec. 4.4, candidate set Q_t, score s = p r c]
  *   - retention ranking of GPU-tier slots (frequency, recency) [Sec. 4.3, cache policy signals]
  *   - early-exit prefetch head: softmax(W_pref h), top-K        [Sec. 4.4, p_early and T_early equations]
@@ -27,8 +27,8 @@
  * Parity pins: every function here is pinned by tests that do not call it to
  * produce their expected values (hand-made cases, closed forms, a library
  * conversion routine, brute force) EXCEPT the COSINE gate away from its
- * special cases (m = h, m = -h, m orthogonal to h, m = 0): the paper only says
- * the gate "may be a scalar, a vector, or a learned function", so the formula
+ * special cases (m = h, m = -h, m orthogonal to h, m = 0): the paper leaves the
+ * form of the gate open (Sec. 2.2), so the formula
  * g = lambda * sigmoid(cos(h, m)) is this build's own reading --
  * COSINE gate: parity unpinned.
  * The same holds for the retention ranking: the paper lists its signals and no formula, so the
@@ -312,7 +312,7 @@ static double hidden_at(const void *h, int32_t hidden_dtype, int64_t idx)
  *        ALL:     sum over the matched phrases that are GPU-resident of
  *                 alpha_i * row_i, alpha_i = n_i / (sum of n_j over ALL matched
  *                 phrases of this query, resident or not)  [Sec. 4.2 e_phi eq.;
- *                 alpha "determined by phrase length"].
+ *                 weights by phrase length, one of the choices Sec. 4.2 allows].
  *   g_t  CONST:   lambda.
  *        COSINE:  lambda * sigmoid( <h,m> / sqrt(<h,h><m,m> + 1e-12) ).
  *

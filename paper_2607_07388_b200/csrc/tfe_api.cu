@@ -936,14 +936,16 @@ tfe_status tfe_lookup_inject_host(tfe_ctx *c, const int32_t *tokens, int32_t B, 
     if (!tokens || !h || !out) return TFE_ERR_INVALID_ARG;
     const size_t hid_bytes = (size_t)Q * c->cfg.d * (c->cfg.hidden_dtype == 0 ? 2 : 4);
     if (n_tok > c->hb_tok_cap || Q > c->hb_q_cap || ent > c->hb_ent_cap) {
+        // every dimension keeps the larger of what it had and what this call needs, so calls of alternating
+        // shapes settle after one regrow each
+        const int64_t tok_cap = std::max(n_tok, c->hb_tok_cap), q_cap = std::max(Q, c->hb_q_cap);
+        const int64_t e_cap = std::max<int64_t>(std::max(ent, c->hb_ent_cap), q_cap * c->cfg.n_orders);
         CU(cudaDeviceSynchronize());
         free_dev(c->d_h_tokens); free_dev(c->d_h_hidden); free_dev(c->d_h_out);
         free_dev(c->d_h_phrase); free_dev(c->d_h_slot); free_dev(c->d_h_flag);
         c->d_h_tokens = nullptr; c->d_h_hidden = c->d_h_out = nullptr;
         c->d_h_phrase = nullptr; c->d_h_slot = nullptr; c->d_h_flag = nullptr;
         c->hb_tok_cap = c->hb_q_cap = c->hb_ent_cap = 0;
-        const int64_t tok_cap = std::max(n_tok, c->hb_tok_cap), q_cap = std::max(Q, c->hb_q_cap);
-        const int64_t e_cap = std::max<int64_t>(ent, q_cap * c->cfg.n_orders);
         const size_t row_bytes = (size_t)c->cfg.d * (c->cfg.hidden_dtype == 0 ? 2 : 4);
         CU(cudaMalloc(&c->d_h_tokens, (size_t)tok_cap * 4));
         CU(cudaMalloc(&c->d_h_hidden, (size_t)q_cap * row_bytes));

@@ -1,8 +1,8 @@
 // Phrase-key formation and bucket hashing, shared by the host-side index build
 // and the device kernels of the library (never by the CPU oracle).
 //
-// A phrase key is derived from the token ids of an n-gram (paper Sec. 2.2: the
-// key "may be derived from ... token n-grams").  The memory must be exact -- one
+// A phrase key is derived from the token ids of an n-gram (paper Sec. 2.2 names token
+// n-grams as a source of keys).  The memory must be exact -- one
 // logical entry per phrase, no shared slots (Sec. 3.1) -- so a key identifies a
 // token tuple, not a hash class:
 //   * an order n with n * bits_per_token <= 61 is PACKED: the ids are laid side
