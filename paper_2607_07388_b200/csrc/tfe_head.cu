@@ -14,14 +14,20 @@
 //                            memory, two accumulators so that a tile's epilogue overlaps the next
 //                            tile's MMAs), warps 2-5 read finished accumulators with tcgen05.ld and
 //                            store fp32 logits [B][V].  All mbarrier waits are bounded.
-//   tfe_head_select_kernel   grid (segments, B): softmax statistics (max, sum of exponentials) and
-//                            the K largest logits of one segment of one row, in order; the block
-//                            that finishes a row last merges the segments' candidates (descending
-//                            logit, equal logits ascending token id) and turns the best K into
-//                            probabilities exp(z - logsumexp).
+//                            The epilogue also leaves, per sequence, what the selection needs so that
+//                            it never reads the logits back: the largest logit of every group of 32
+//                            vocabulary rows (one warp's rows of one tile), and per (CTA, epilogue
+//                            warp) a running maximum with the sum of exp(z - maximum) over the
+//                            warp's rows (online softmax).
+//   tfe_head_select_kernel   one block per sequence: logsumexp from the per-warp partial sums; the
+//                            K-th largest of the 32-row group maxima is a lower bound of the K-th
+//                            largest logit, and every logit at or above it lies in a group whose
+//                            maximum is at or above it: about K groups of 32 logits are read back
+//                            (8 KB of the 600 KB row), ranked (descending logit, equal logits
+//                            ascending token id) and the best K become probabilities exp(z - logsumexp).
 //
-// The logits make a round trip through global memory (B*V*4 bytes, 39 MB for B = 64); they are
-// written and re-read within microseconds and stay in the 126 MB L2 for the batch sizes of decode.
+// The fp32 logits [B][V] are still written (they are an output: tfe_head_buffers), but only the
+// candidate groups are read again.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -35,13 +41,16 @@
 #define HEAD_TILE_K 64              // bf16 elements per stage along d: one 128-byte swizzle row
 #define HEAD_UMMA_K 16              // bf16 elements per tcgen05.mma
 #define HEAD_MAX_N 256              // batch columns (MMA N)
-#define HEAD_THREADS 192            // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+#ifndef HEAD_EPI_PER_QUARTER
+#define HEAD_EPI_PER_QUARTER 2      // epilogue warps per tensor-memory lane quarter
+#endif
+#define HEAD_EPI_STRIDE (16 * HEAD_EPI_PER_QUARTER)
+#define HEAD_THREADS (64 + 128 * HEAD_EPI_PER_QUARTER)   // warp 0 TMA, warp 1 MMA, the rest epilogue
 #define HEAD_MAX_STAGES 8
 #define HEAD_MAX_K 128              // top-K limit
-#define HEAD_SEGMENTS 8             // segments per row in the selection
 #define HEAD_SEL_THREADS 512
 #define HEAD_WAIT_LIMIT (1u << 22)  // polls of one mbarrier before a wait gives up
-#define HEAD_DYN_SMEM (227 * 1024 - 8192)   // dynamic shared memory of the GEMM: the SM's 227 KB minus its static arrays
+#define HEAD_DYN_SMEM (227 * 1024 - 12288)  // dynamic shared memory of the GEMM: the SM's 227 KB minus its static arrays
 
 // device status bits
 #define HEAD_ST_TIMEOUT_PRODUCER 1u
@@ -163,6 +172,17 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(uint32_t M, uint32_t N)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 
+// fp32 -> uint32 whose unsigned order is the float order (NaN sorts above +inf; not produced here)
+__device__ __forceinline__ uint32_t orderable(float x)
+{
+    const uint32_t u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float from_orderable(uint32_t k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
+}
+
 // ------------------------------------------------------------------ GEMM
 
 struct HeadGemmParams {
@@ -174,7 +194,11 @@ struct HeadGemmParams {
     uint32_t tmem_cols;             // power of two >= 2 N
     float *logits;                  // [B][ld]
     int64_t ld;
-    float *group_max;               // [B][4 * gridDim.x]: largest logit of every (CTA, epilogue warp) per sequence
+    float *group_max;               // [B][4 * gridDim.x]: running maximum of every (CTA, epilogue warp) per sequence
+    float *group_sum;               // [B][4 * gridDim.x]: sum of exp(z - that maximum) over the warp's rows
+    float *fine_max;                // [B][n_fine]: largest logit of every (CTA, tile, epilogue warp): 32 vocabulary rows
+    int32_t n_fine;                 // gridDim.x * tiles_per_cta * 4
+    int32_t tiles_per_cta;
     uint32_t *status;
 };
 
@@ -187,6 +211,7 @@ tfe_head_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     __shared__ uint32_t s_tmem_base;
     __shared__ volatile uint32_t s_abort;
     __shared__ float s_gmax[4][HEAD_MAX_N];            // running column maxima of the four epilogue warps
+    __shared__ float s_gsum[4][HEAD_MAX_N];            // sums of exp(z - running maximum) over the warps' rows
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -202,7 +227,7 @@ tfe_head_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(smem_u32(&s_full[s]), 1); mbar_init(smem_u32(&s_empty[s]), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&s_acc_full[a]), 1); mbar_init(smem_u32(&s_acc_empty[a]), 4); }
+        for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&s_acc_full[a]), 1); mbar_init(smem_u32(&s_acc_empty[a]), 4 * HEAD_EPI_PER_QUARTER); }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -287,9 +312,18 @@ tfe_head_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
         }
     } else {
         // ============================ epilogue ================================
+        // Two warps share a tensor-memory lane quarter (a warp may only read the lanes 32 * (warp % 4) .. +31) and
+        // split its columns: the 16-column chunks alternate between them.
         const uint32_t quarter = (uint32_t)warp & 3u;               // tensor-memory lanes 32*quarter .. +31
-        for (int32_t c = lane; c < p.N; c += 32) s_gmax[quarter][c] = -INFINITY;
+        const int32_t c_first = 16 * ((warp - 2) >> 2);             // this warp's chunks: c_first, c_first + HEAD_EPI_STRIDE, ...
+        for (int32_t c0 = c_first; c0 < p.N; c0 += HEAD_EPI_STRIDE)
+            if (lane < 16) { s_gmax[quarter][c0 + lane] = -INFINITY; s_gsum[quarter][c0 + lane] = 0.f; }
         __syncwarp();
+        // 32-row groups of tiles this CTA does not have (the last CTA's range may end early): no logit
+        for (int32_t t = n_tiles; t < p.tiles_per_cta; ++t)
+            for (int32_t c0 = c_first; c0 < p.N; c0 += HEAD_EPI_STRIDE)
+                if (lane < 16 && c0 + lane < p.B)
+                    p.fine_max[(int64_t)(c0 + lane) * p.n_fine + ((int64_t)blockIdx.x * p.tiles_per_cta + t) * 4 + quarter] = -INFINITY;
         for (int32_t t = 0; t < n_tiles; ++t) {
             const uint32_t acc = (uint32_t)t & 1u, acc_phase = ((uint32_t)t >> 1) & 1u;
             if (!mbar_wait(smem_u32(&s_acc_full[acc]), acc_phase, &s_abort)) {
@@ -302,7 +336,7 @@ tfe_head_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
             const int32_t row_in_tile = (int32_t)(quarter * 32u) + lane;
             const int64_t row = r0 + (int64_t)t * HEAD_TILE_M + row_in_tile;
             const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + acc * (uint32_t)p.N;
-            for (int32_t c0 = 0; c0 < p.N; c0 += 16) {
+            for (int32_t c0 = c_first; c0 < p.N; c0 += HEAD_EPI_STRIDE) {
                 uint32_t v[16];
                 tmem_ld16(taddr + (uint32_t)c0, v);
                 tmem_ld_wait();
@@ -314,25 +348,35 @@ tfe_head_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                     for (int j = 0; j < 16; ++j)
                         if (c0 + j < p.B) p.logits[(int64_t)(c0 + j) * p.ld + row] = f[j];
                 }
-                // Maximum of each of the 16 columns over the warp's 32 rows: a butterfly in which
-                // every exchange halves the columns a lane is responsible for, 16 shuffles in all;
-                // lane l ends with the maximum of column c0 + (l >> 1).
-                const bool b4 = lane & 16, b3 = lane & 8, b2 = lane & 4, b1 = lane & 2;
-                float r8[8], r4[4], r2[2];
+                // Per column: the maximum over the warp's 32 rows (one warp reduction on the order-preserving integer
+                // image of the logit), then the sum of exp(z - maximum) as a 24-bit fixed-point integer sum (the warp
+                // reduction has no floating-point addition; a term is at most 1, 32 of them stay below 2^30).  Every
+                // lane ends with both for all 16 columns: no shuffles to route, nothing through shared memory.
+                float gm[16];
+                uint32_t gs[16];
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    r8[i] = fmaxf(b4 ? f[i + 8] : f[i], __shfl_xor_sync(0xFFFFFFFFu, b4 ? f[i] : f[i + 8], 16));
+                for (int j = 0; j < 16; ++j) gm[j] = from_orderable(__reduce_max_sync(0xFFFFFFFFu, orderable(f[j])));
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    r4[i] = fmaxf(b3 ? r8[i + 4] : r8[i], __shfl_xor_sync(0xFFFFFFFFu, b3 ? r8[i] : r8[i + 4], 8));
+                for (int j = 0; j < 16; ++j) {
+                    const float ev = row_in_tile < valid ? __expf(f[j] - gm[j]) : 0.f;
+                    gs[j] = __reduce_add_sync(0xFFFFFFFFu, __float2uint_rn(ev * 16777216.f));
+                }
+                // lane j folds column c0 + j into the warp's running (maximum, sum) pair: online softmax
+                float my_m = -INFINITY;
+                uint32_t my_s = 0;
 #pragma unroll
-                for (int i = 0; i < 2; ++i)
-                    r2[i] = fmaxf(b2 ? r4[i + 2] : r4[i], __shfl_xor_sync(0xFFFFFFFFu, b2 ? r4[i] : r4[i + 2], 4));
-                float r1 = fmaxf(b1 ? r2[1] : r2[0], __shfl_xor_sync(0xFFFFFFFFu, b1 ? r2[0] : r2[1], 2));
-                r1 = fmaxf(r1, __shfl_xor_sync(0xFFFFFFFFu, r1, 1));
-                if ((lane & 1) == 0) {
-                    const int32_t c = c0 + (lane >> 1);
-                    s_gmax[quarter][c] = fmaxf(s_gmax[quarter][c], r1);
+                for (int j = 0; j < 16; ++j)
+                    if (lane == j) { my_m = gm[j]; my_s = gs[j]; }
+                if (lane < 16) {
+                    const int32_t c = c0 + lane;
+                    if (c < p.B)
+                        p.fine_max[(int64_t)c * p.n_fine + ((int64_t)blockIdx.x * p.tiles_per_cta + t) * 4 + quarter] = my_m;
+                    if (my_m > -INFINITY) {
+                        const float old_ref = s_gmax[quarter][c], new_ref = fmaxf(old_ref, my_m);
+                        const float kept = old_ref == -INFINITY ? 0.f : s_gsum[quarter][c] * __expf(old_ref - new_ref);
+                        s_gsum[quarter][c] = kept + (float)my_s * (1.f / 16777216.f) * __expf(my_m - new_ref);
+                        s_gmax[quarter][c] = new_ref;
+                    }
                 }
             }
             tc_fence_before();
@@ -341,8 +385,13 @@ tfe_head_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
         }
         __syncwarp();
         const int32_t groups = 4 * (int32_t)gridDim.x;
-        for (int32_t c = lane; c < p.B; c += 32)
-            p.group_max[(int64_t)c * groups + 4 * blockIdx.x + quarter] = s_gmax[quarter][c];
+        for (int32_t c0 = c_first; c0 < p.N; c0 += HEAD_EPI_STRIDE) {
+            const int32_t c = c0 + lane;
+            if (lane < 16 && c < p.B) {
+                p.group_max[(int64_t)c * groups + 4 * blockIdx.x + quarter] = s_gmax[quarter][c];
+                p.group_sum[(int64_t)c * groups + 4 * blockIdx.x + quarter] = s_gsum[quarter][c];
+            }
+        }
     }
 
     tc_fence_before();
@@ -356,126 +405,70 @@ tfe_head_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
 
 // ------------------------------------------------------------------ selection
 
-// fp32 -> uint32 whose unsigned order is the float order (NaN sorts above +inf; not produced here)
-__device__ __forceinline__ uint32_t orderable(float x)
-{
-    const uint32_t u = __float_as_uint(x);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-__device__ __forceinline__ float from_orderable(uint32_t k)
-{
-    return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
-}
-
 struct HeadSelParams {
     const float *logits;
     int64_t ld;
     int32_t V, B, K;
-    int32_t seg_len;                // multiple of 4
-    float *seg_max, *seg_sum;       // [B][HEAD_SEGMENTS]
-    unsigned long long *seg_cand;   // [B][HEAD_SEGMENTS][K]: orderable(z) << 32 | ~token, 0 = none
     int32_t *out_tokens;            // [B][K]
     float *out_prob;                // [B][K]
     float *out_lse;                 // [B] or nullptr
-    uint32_t *row_done;             // [B] segments finished per row, zero between calls
-    const float *group_max;         // [B][groups] from the GEMM's epilogue
+    const float *group_max;         // [B][groups] from the GEMM's epilogue: running maxima ...
+    const float *group_sum;         // ... and sums of exp(z - maximum) of every (CTA, epilogue warp)
     int32_t groups;
+    const float *fine_max;          // [B][n_fine]: largest logit of every 32-row group
+    int32_t n_fine, tiles_per_cta, rows_per_cta;
 };
 
-// Selection, one block per (segment, row): the segment's sum of exp(z - row maximum) and its
-// candidates for the row's K best as 64-bit keys orderable(z) << 32 | ~token -- distinct, so
-// "largest K keys" has one answer: descending logit, equal logits ascending token id -- in
-// descending order.  The block that finishes a row last merges the segments.
+// Selection, one block per sequence.  Keys are orderable(z) << 32 | ~token -- distinct, so "largest K keys" has
+// one answer: descending logit, equal logits ascending token id.
 //
-// The GEMM's epilogue left the largest logit of every (CTA, epilogue warp) group of vocabulary
-// rows.  Their maximum is the row maximum, and the K-th largest of them bounds the row's K-th
-// largest logit from below (K different elements reach it; with fewer than K groups the bound is
-// -inf).  So one sweep over the segment sums the exponentials and keeps the elements at or above
-// the bound -- about K per row, a handful per segment.  Each survivor finds its rank by counting
-// the survivors above it.  More than HEAD_KEEP_CAP survivors in a segment (many equal logits)
-// send the block to an exact radix selection over the segment's keys, eight 8-bit digits, slower
-// but indifferent to the distribution.
+// The GEMM's epilogue left the largest logit of every group of 32 vocabulary rows.  The K-th largest of them
+// (with multiplicity) bounds the row's K-th largest logit from below (K different logits reach it), and a logit
+// at or above the bound sits in a group whose maximum is at or above it: only those groups -- K of them, more
+// with equal maxima -- are read back, the logits at or above the bound are kept, each survivor finds its rank
+// by counting the survivors above it.  More than HEAD_KEEP_CAP survivors (many equal logits) send the block to
+// an exact radix selection over the whole row, eight 8-bit digits, slower but indifferent to the distribution.
+// The softmax denominator comes from the epilogue's per-warp (maximum, sum) pairs; no logit is read for it.
 #define HEAD_KEEP_CAP 2048
+#define HEAD_MAX_FINE 6144
 
 __device__ __forceinline__ unsigned long long head_key(float z, int32_t token)
 {
     return ((unsigned long long)orderable(z) << 32) | (uint32_t)~(uint32_t)token;
 }
 
-// Merge of one row: every segment's list is in descending order, so a candidate's place in the
-// merged order is the number of keys above it in every list (binary searches); the first K are
-// written out with their probabilities exp(z - logsumexp).  s_v: HEAD_SEGMENTS * K keys.
-__device__ __forceinline__ void head_merge_row(const HeadSelParams &p, int b, unsigned long long *s_v, float *s_lse)
-{
-    const int K = p.K;
-    const uint32_t n = (uint32_t)(HEAD_SEGMENTS * K);
-    const unsigned long long *cand = p.seg_cand + (int64_t)b * HEAD_SEGMENTS * K;
-    for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) s_v[i] = __ldcg(cand + i);
-    if (threadIdx.x < 32) {                         // the segments' statistics, one per lane
-        const bool has = threadIdx.x < HEAD_SEGMENTS;
-        const float ss = has ? __ldcg(p.seg_sum + b * HEAD_SEGMENTS + threadIdx.x) : 0.f;
-        const float sm = has ? __ldcg(p.seg_max + b * HEAD_SEGMENTS + threadIdx.x) : -INFINITY;
-        float m = ss > 0.f ? sm : -INFINITY;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-        float t = ss > 0.f ? ss * __expf(sm - m) : 0.f;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
-        if (threadIdx.x == 0) {
-            *s_lse = m + __logf(t);
-            if (p.out_lse) p.out_lse[b] = *s_lse;
-        }
-    }
-    __syncthreads();
-    const float lse = *s_lse;
-    for (uint32_t i = threadIdx.x; i < n; i += blockDim.x) {
-        const unsigned long long key = s_v[i];
-        if (key == 0ull) continue;
-        uint32_t rank = 0;
-        for (int s = 0; s < HEAD_SEGMENTS && rank < (uint32_t)K; ++s) {
-            const unsigned long long *list = s_v + s * K;
-            int lo = 0, hi = K;                     // first position whose key is not above `key`
-            while (lo < hi) {
-                const int mid = (lo + hi) >> 1;
-                if (list[mid] > key) lo = mid + 1; else hi = mid;
-            }
-            rank += (uint32_t)lo;
-        }
-        if (rank < (uint32_t)K) {
-            p.out_tokens[(int64_t)b * K + rank] = (int32_t)~(uint32_t)key;
-            p.out_prob[(int64_t)b * K + rank] = __expf(from_orderable((uint32_t)(key >> 32)) - lse);
-        }
-    }
-}
-
+#ifdef HEAD_TIMELINE
+__device__ long long g_head_tl[16];
+#define HSTAMP(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) g_head_tl[i] = clock64(); } while (0)
+#else
+#define HSTAMP(i) do { } while (0)
+#endif
 __global__ void __launch_bounds__(HEAD_SEL_THREADS)
 tfe_head_select_kernel(const HeadSelParams p)
 {
     __shared__ unsigned long long s_keep[HEAD_KEEP_CAP];
+    __shared__ uint32_t s_fine[HEAD_MAX_FINE];
     __shared__ float s_red[HEAD_SEL_THREADS / 32];
     __shared__ uint32_t s_hist[256];
     __shared__ unsigned long long s_prefix;
-    __shared__ float s_lse;
-    __shared__ uint32_t s_want, s_fill, s_nkeep, s_last;
-    const int seg = blockIdx.x, b = blockIdx.y;
-    const int32_t v0 = seg * p.seg_len;
-    const int32_t n = max(0, min(p.seg_len, p.V - v0));
-    const float *row = p.logits + (int64_t)b * p.ld + v0;
+    __shared__ uint32_t s_want, s_fill, s_nkeep;
+    const int b = blockIdx.x;
+    const float *row = p.logits + (int64_t)b * p.ld;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int NW = HEAD_SEL_THREADS / 32;
     const int32_t G = p.groups;
-    const float *gmax = p.group_max + (int64_t)b * G;
 
-    // ---- row maximum, and the K-th largest group maximum (with multiplicity) rounded down to the
-    // upper 16 bits of its order-preserving integer image (any lower bound serves): radix selection,
-    // two 8-bit digits, most significant first
-    // (at most 2 * HEAD_SEL_THREADS groups: two per thread, loaded once)
     // launched with programmatic stream serialisation: the blocks may be resident before the GEMM has
     // finished; nothing of its output is read before this point
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const float g0v = (int)threadIdx.x < G ? __ldcg(gmax + threadIdx.x) : -INFINITY;
-    const float g1v = (int)threadIdx.x + HEAD_SEL_THREADS < G ? __ldcg(gmax + threadIdx.x + HEAD_SEL_THREADS) : -INFINITY;
-    float row_max = fmaxf(g0v, g1v);
+    HSTAMP(0);
+
+    // ---- logsumexp from the epilogue's partial sums (at most 2 * HEAD_SEL_THREADS groups: two per thread)
+    const float *gmax = p.group_max + (int64_t)b * G, *gsum = p.group_sum + (int64_t)b * G;
+    const bool h0 = (int)threadIdx.x < G, h1 = (int)threadIdx.x + HEAD_SEL_THREADS < G;
+    const float m0 = h0 ? __ldcg(gmax + threadIdx.x) : -INFINITY, m1 = h1 ? __ldcg(gmax + threadIdx.x + HEAD_SEL_THREADS) : -INFINITY;
+    const float t0 = h0 ? __ldcg(gsum + threadIdx.x) : 0.f, t1 = h1 ? __ldcg(gsum + threadIdx.x + HEAD_SEL_THREADS) : 0.f;
+    float row_max = fmaxf(m0, m1);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) row_max = fmaxf(row_max, __shfl_xor_sync(0xFFFFFFFFu, row_max, o));
     if (lane == 0) s_red[warp] = row_max;
@@ -484,7 +477,21 @@ tfe_head_select_kernel(const HeadSelParams p)
     row_max = s_red[0];
     for (int w = 1; w < NW; ++w) row_max = fmaxf(row_max, s_red[w]);
     __syncthreads();                                // s_red is reused for the sums
-    float theta = -INFINITY;
+    float sum = (t0 > 0.f ? t0 * __expf(m0 - row_max) : 0.f) + (t1 > 0.f ? t1 * __expf(m1 - row_max) : 0.f);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+    if (lane == 0) s_red[warp] = sum;
+    __syncthreads();
+    float total = 0.f;
+    for (int w = 0; w < NW; ++w) total += s_red[w];
+    const float lse = row_max + __logf(total);
+    if (threadIdx.x == 0 && p.out_lse) p.out_lse[b] = lse;
+
+    HSTAMP(1);
+    // ---- a lower bound of the row's K-th largest logit: the K-th largest (with multiplicity) of the per-(CTA,
+    // epilogue warp) maxima, rounded down to the upper 16 bits of its integer image (any lower bound serves):
+    // radix selection, two 8-bit digits, most significant first.  With fewer than K such groups: no bound.
+    uint32_t theta_key = 0;                         // below every image
     if (G >= p.K) {
         uint32_t prefix = 0, want = (uint32_t)p.K;
         for (int shift = 24; shift >= 16; shift -= 8) {
@@ -492,9 +499,8 @@ tfe_head_select_kernel(const HeadSelParams p)
             __syncthreads();
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                const int g = (int)threadIdx.x + half * HEAD_SEL_THREADS;
-                const uint32_t gkey = orderable(half ? g1v : g0v);
-                const bool live = g < G && (shift == 24 || (gkey >> (shift + 8)) == (prefix >> (shift + 8)));
+                const uint32_t gkey = orderable(half ? m1 : m0);
+                const bool live = (half ? h1 : h0) && (shift == 24 || (gkey >> (shift + 8)) == (prefix >> (shift + 8)));
                 const uint32_t digit = (gkey >> shift) & 255u;
                 const uint32_t vote = __ballot_sync(0xFFFFFFFFu, live);
                 if (live) {                         // one shared-memory atomic per distinct digit of the warp
@@ -527,68 +533,85 @@ tfe_head_select_kernel(const HeadSelParams p)
             want = __shfl_sync(0xFFFFFFFFu, rest, who);
             __syncthreads();
         }
-        // (rounding the image of -inf down lands among the NaN patterns: no bound then)
-        theta = prefix <= orderable(-INFINITY) ? -INFINITY : from_orderable(prefix);
+        theta_key = prefix;
     }
+    HSTAMP(2);
 
-    // ---- the sweep: sum of exponentials, survivors
-    float sum = 0.f;
-    auto take_in = [&](float z, int i) {
-        sum += __expf(z - row_max);
-        if (z >= theta) {
-            const uint32_t at = atomicAdd(&s_nkeep, 1u);
-            if (at < HEAD_KEEP_CAP) s_keep[at] = head_key(z, v0 + i);
-        }
-    };
-    // 16-byte loads, several in flight per thread (the row and the segment start are 16-byte aligned)
-    const int n4 = n >> 2;
-    const float4 *row4 = reinterpret_cast<const float4 *>(row);
-    int i4 = threadIdx.x;
-    for (; i4 + 2 * (int)blockDim.x < n4; i4 += 3 * blockDim.x) {
-        const int ic = i4 + blockDim.x, ie = i4 + 2 * blockDim.x;
-        const float4 a = __ldcs(row4 + i4), c = __ldcs(row4 + ic), e = __ldcs(row4 + ie);
-        take_in(a.x, 4 * i4); take_in(a.y, 4 * i4 + 1); take_in(a.z, 4 * i4 + 2); take_in(a.w, 4 * i4 + 3);
-        take_in(c.x, 4 * ic); take_in(c.y, 4 * ic + 1); take_in(c.z, 4 * ic + 2); take_in(c.w, 4 * ic + 3);
-        take_in(e.x, 4 * ie); take_in(e.y, 4 * ie + 1); take_in(e.z, 4 * ie + 2); take_in(e.w, 4 * ie + 3);
-    }
-    for (; i4 < n4; i4 += blockDim.x) {
-        const float4 a = __ldcs(row4 + i4);
-        take_in(a.x, 4 * i4); take_in(a.y, 4 * i4 + 1); take_in(a.z, 4 * i4 + 2); take_in(a.w, 4 * i4 + 3);
-    }
-    for (int i = 4 * n4 + threadIdx.x; i < n; i += blockDim.x) take_in(__ldcs(row + i), i);
+    // ---- the 32-row groups that can hold a logit at or above the bound (their maximum reaches it): a list
+    const int32_t F = p.n_fine;
+    const float *fmax_row = p.fine_max + (int64_t)b * F;
+    {
+        constexpr int PER = HEAD_MAX_FINE / HEAD_SEL_THREADS;       // all of a thread's loads in flight together
+        float fm[PER];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
-    if (lane == 0) s_red[warp] = sum;
-    __syncthreads();
-    const uint32_t n_keep = s_nkeep;
-    unsigned long long *cand = p.seg_cand + ((int64_t)b * HEAD_SEGMENTS + seg) * p.K;
-    if (threadIdx.x == 0) {
-        float t = 0.f;
-        for (int w = 0; w < NW; ++w) t += s_red[w];
-        p.seg_max[b * HEAD_SEGMENTS + seg] = row_max;
-        p.seg_sum[b * HEAD_SEGMENTS + seg] = n > 0 ? t : 0.f;
-        s_want = (uint32_t)min(p.K, n);
+        for (int u = 0; u < PER; ++u) {
+            const int32_t g = (int32_t)threadIdx.x + u * HEAD_SEL_THREADS;
+            fm[u] = g < F ? __ldcg(fmax_row + g) : -INFINITY;
+        }
+#pragma unroll
+        for (int u = 0; u < PER; ++u) {
+            const int32_t g = (int32_t)threadIdx.x + u * HEAD_SEL_THREADS;
+            if (g < F && orderable(fm[u]) >= theta_key) {
+                const uint32_t at = atomicAdd(&s_fill, 1u);
+                if (at < HEAD_MAX_FINE) s_fine[at] = (uint32_t)g;
+            }
+        }
     }
+    __syncthreads();
+    HSTAMP(3);
+    // ---- read them back, one warp per group, one row per lane, four groups in flight per warp
+    const uint32_t n_list = min(s_fill, (uint32_t)HEAD_MAX_FINE);
+    for (uint32_t i0 = warp; i0 < n_list; i0 += 4 * NW) {
+        float z[4];
+        int64_t vv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t i = i0 + (uint32_t)u * NW;
+            vv[u] = -1;
+            z[u] = 0.f;
+            if (i < n_list) {
+                const int32_t g = (int32_t)s_fine[i];
+                const int32_t cta = g / (4 * p.tiles_per_cta), rest = g - cta * 4 * p.tiles_per_cta;
+                const int32_t in_cta = (rest >> 2) * HEAD_TILE_M + (rest & 3) * 32 + lane;
+                const int64_t v = (int64_t)cta * p.rows_per_cta + in_cta;
+                if (in_cta < p.rows_per_cta && v < p.V) { vv[u] = v; z[u] = __ldcg(row + v); }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (vv[u] >= 0 && orderable(z[u]) >= theta_key) {
+                const uint32_t at = atomicAdd(&s_nkeep, 1u);
+                if (at < HEAD_KEEP_CAP) s_keep[at] = head_key(z[u], (int32_t)vv[u]);
+            }
+    }
+    __syncthreads();
+    HSTAMP(4);
+    const uint32_t n_keep = s_nkeep;
+#ifdef HEAD_TIMELINE
+    if (blockIdx.x == 0 && threadIdx.x == 0) g_head_tl[8] = n_keep;
+#endif
+    const uint32_t take = (uint32_t)min(p.K, p.V);
+    if (threadIdx.x == 0) s_want = take;
     if (n_keep <= HEAD_KEEP_CAP) {
-        const uint32_t take = min((uint32_t)p.K, n_keep);
-        for (int i = take + threadIdx.x; i < p.K; i += blockDim.x) cand[i] = 0ull;
+        // (fewer survivors than K cannot happen: K logits reach the bound)
         for (uint32_t i = threadIdx.x; i < n_keep; i += blockDim.x) {
             const unsigned long long key = s_keep[i];
             uint32_t rank = 0;
             for (uint32_t j = 0; j < n_keep; ++j) rank += s_keep[j] > key;
-            if (rank < take) cand[rank] = key;
+            if (rank < take) {
+                p.out_tokens[(int64_t)b * p.K + rank] = (int32_t)~(uint32_t)key;
+                p.out_prob[(int64_t)b * p.K + rank] = __expf(from_orderable((uint32_t)(key >> 32)) - lse);
+            }
         }
     } else {
-        // ---- exact radix selection of the segment's take-th largest key, most significant byte first
-        const uint32_t take = (uint32_t)min(p.K, n);
-        for (int i = take + threadIdx.x; i < p.K; i += blockDim.x) cand[i] = 0ull;
+        // ---- exact radix selection of the row's take-th largest key, most significant byte first
         __syncthreads();
         for (int shift = 56; shift >= 0; shift -= 8) {
             for (int i = threadIdx.x; i < 256; i += blockDim.x) s_hist[i] = 0;
             __syncthreads();
             const unsigned long long prefix = s_prefix;
-            for (int i = threadIdx.x; i < n; i += blockDim.x) {
-                const unsigned long long key = head_key(__ldcg(row + i), v0 + i);
+            for (int i = threadIdx.x; i < p.V; i += blockDim.x) {
+                const unsigned long long key = head_key(__ldcg(row + i), i);
                 if (shift == 56 || (key >> (shift + 8)) == (prefix >> (shift + 8)))
                     atomicAdd(&s_hist[(uint32_t)(key >> shift) & 255u], 1u);
             }
@@ -604,8 +627,10 @@ tfe_head_select_kernel(const HeadSelParams p)
         }
         // the keys at or above it are exactly `take`; they fit the keep list (take <= HEAD_MAX_K)
         const unsigned long long kth = s_prefix;
-        for (int i = threadIdx.x; i < n; i += blockDim.x) {
-            const unsigned long long key = head_key(__ldcg(row + i), v0 + i);
+        if (threadIdx.x == 0) s_fill = 0;           // (it counted the group list above)
+        __syncthreads();
+        for (int i = threadIdx.x; i < p.V; i += blockDim.x) {
+            const unsigned long long key = head_key(__ldcg(row + i), i);
             if (key >= kth) s_keep[atomicAdd(&s_fill, 1u)] = key;
         }
         __syncthreads();
@@ -613,18 +638,11 @@ tfe_head_select_kernel(const HeadSelParams p)
             const unsigned long long key = s_keep[i];
             uint32_t rank = 0;
             for (uint32_t j = 0; j < take; ++j) rank += s_keep[j] > key;
-            cand[rank] = key;
+            p.out_tokens[(int64_t)b * p.K + rank] = (int32_t)~(uint32_t)key;
+            p.out_prob[(int64_t)b * p.K + rank] = __expf(from_orderable((uint32_t)(key >> 32)) - lse);
         }
     }
-    // ---- the block that closes the row merges its segments
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_last = atomicAdd(&p.row_done[b], 1u) == HEAD_SEGMENTS - 1;
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    head_merge_row(p, b, s_keep, &s_lse);
-    if (threadIdx.x == 0) p.row_done[b] = 0;         // re-armed for the next call
+    HSTAMP(5);
 }
 
 // ------------------------------------------------------------------ host side
@@ -670,11 +688,10 @@ struct tfe_head {
     CUtensorMap map_w, map_w_tail;
     float *d_logits = nullptr;
     int64_t ld = 0;
-    float *d_seg_max = nullptr, *d_seg_sum = nullptr, *d_lse = nullptr;
-    unsigned long long *d_seg_cand = nullptr;
-    uint32_t *d_status = nullptr, *d_row_done = nullptr;
-    float *d_group_max = nullptr;
-    int32_t seg_len = 0;
+    float *d_lse = nullptr;
+    uint32_t *d_status = nullptr;
+    float *d_group_max = nullptr, *d_group_sum = nullptr, *d_fine_max = nullptr;
+    int32_t tiles_per_cta = 0, n_fine = 0;
 };
 
 extern "C" {
@@ -702,19 +719,17 @@ tfe_status tfe_head_create(const void *w_pref, int32_t V, int32_t d, int32_t max
     if (!make_map(&h->map_w_tail, w_pref, (uint64_t)V, (uint64_t)d, h->tail_rows ? (uint32_t)h->tail_rows : 8u))
         return fail(TFE_ERR_CUDA);
     h->ld = ((int64_t)V + 3) / 4 * 4;
-    h->seg_len = (int32_t)((((int64_t)V + HEAD_SEGMENTS - 1) / HEAD_SEGMENTS + 3) / 4 * 4);
+    h->tiles_per_cta = (h->rows_per_cta + HEAD_TILE_M - 1) / HEAD_TILE_M;
+    h->n_fine = h->grid * h->tiles_per_cta * 4;
+    if (h->n_fine > HEAD_MAX_FINE) return fail(TFE_ERR_INVALID_ARG);      // a vocabulary beyond 148 x 14 tiles of 128 rows
     const size_t nb = (size_t)max_batch;
     if (cudaMalloc(&h->d_logits, nb * (size_t)h->ld * sizeof(float)) != cudaSuccess) return fail(TFE_ERR_CUDA);
-    if (cudaMalloc(&h->d_seg_max, nb * HEAD_SEGMENTS * sizeof(float)) != cudaSuccess) return fail(TFE_ERR_CUDA);
-    if (cudaMalloc(&h->d_seg_sum, nb * HEAD_SEGMENTS * sizeof(float)) != cudaSuccess) return fail(TFE_ERR_CUDA);
     if (cudaMalloc(&h->d_lse, nb * sizeof(float)) != cudaSuccess) return fail(TFE_ERR_CUDA);
-    if (cudaMalloc(&h->d_seg_cand, nb * HEAD_SEGMENTS * HEAD_MAX_K * sizeof(unsigned long long)) != cudaSuccess)
-        return fail(TFE_ERR_CUDA);
     if (cudaMalloc(&h->d_status, sizeof(uint32_t)) != cudaSuccess) return fail(TFE_ERR_CUDA);
     if (cudaMemset(h->d_status, 0, sizeof(uint32_t)) != cudaSuccess) return fail(TFE_ERR_CUDA);
-    if (cudaMalloc(&h->d_row_done, nb * sizeof(uint32_t)) != cudaSuccess) return fail(TFE_ERR_CUDA);
     if (cudaMalloc(&h->d_group_max, nb * 4 * (size_t)h->grid * sizeof(float)) != cudaSuccess) return fail(TFE_ERR_CUDA);
-    if (cudaMemset(h->d_row_done, 0, nb * sizeof(uint32_t)) != cudaSuccess) return fail(TFE_ERR_CUDA);
+    if (cudaMalloc(&h->d_group_sum, nb * 4 * (size_t)h->grid * sizeof(float)) != cudaSuccess) return fail(TFE_ERR_CUDA);
+    if (cudaMalloc(&h->d_fine_max, nb * (size_t)h->n_fine * sizeof(float)) != cudaSuccess) return fail(TFE_ERR_CUDA);
     if (cudaFuncSetAttribute(tfe_head_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, HEAD_DYN_SMEM) !=
         cudaSuccess)
         return fail(TFE_ERR_CUDA);
@@ -730,13 +745,11 @@ void tfe_head_destroy(tfe_head *h)
     (void)cudaSetDevice(h->device);
     (void)cudaDeviceSynchronize();
     if (h->d_logits) (void)cudaFree(h->d_logits);
-    if (h->d_seg_max) (void)cudaFree(h->d_seg_max);
-    if (h->d_seg_sum) (void)cudaFree(h->d_seg_sum);
     if (h->d_lse) (void)cudaFree(h->d_lse);
-    if (h->d_seg_cand) (void)cudaFree(h->d_seg_cand);
     if (h->d_status) (void)cudaFree(h->d_status);
-    if (h->d_row_done) (void)cudaFree(h->d_row_done);
     if (h->d_group_max) (void)cudaFree(h->d_group_max);
+    if (h->d_group_sum) (void)cudaFree(h->d_group_sum);
+    if (h->d_fine_max) (void)cudaFree(h->d_fine_max);
     (void)cudaSetDevice(prev);
     delete h;
 }
@@ -761,6 +774,7 @@ tfe_status tfe_head_topk(tfe_head *h, const void *hidden, int32_t B, int32_t K, 
     while (cols < 2u * (uint32_t)g.N) cols <<= 1;
     g.tmem_cols = cols;
     g.logits = h->d_logits; g.ld = h->ld; g.status = h->d_status; g.group_max = h->d_group_max;
+    g.group_sum = h->d_group_sum; g.fine_max = h->d_fine_max; g.n_fine = h->n_fine; g.tiles_per_cta = h->tiles_per_cta;
     CUtensorMap map_h;
     if (!make_map(&map_h, hidden, (uint64_t)B, (uint64_t)h->d, (uint32_t)g.N)) return TFE_ERR_CUDA;
     const size_t smem = (size_t)g.stages * stage_bytes + 1024;
@@ -776,11 +790,11 @@ tfe_status tfe_head_topk(tfe_head *h, const void *hidden, int32_t B, int32_t K, 
     }
 
     HeadSelParams s{};
-    s.logits = h->d_logits; s.ld = h->ld; s.V = h->V; s.B = B; s.K = K; s.seg_len = h->seg_len;
-    s.seg_max = h->d_seg_max; s.seg_sum = h->d_seg_sum; s.seg_cand = h->d_seg_cand;
-    s.out_tokens = cand_tokens; s.out_prob = cand_prob; s.out_lse = h->d_lse; s.row_done = h->d_row_done;
-    s.group_max = h->d_group_max; s.groups = 4 * h->grid;
-    cfg.gridDim = dim3(HEAD_SEGMENTS, (unsigned)B); cfg.blockDim = dim3(HEAD_SEL_THREADS); cfg.dynamicSmemBytes = 0;
+    s.logits = h->d_logits; s.ld = h->ld; s.V = h->V; s.B = B; s.K = K;
+    s.out_tokens = cand_tokens; s.out_prob = cand_prob; s.out_lse = h->d_lse;
+    s.group_max = h->d_group_max; s.group_sum = h->d_group_sum; s.groups = 4 * h->grid;
+    s.fine_max = h->d_fine_max; s.n_fine = h->n_fine; s.tiles_per_cta = h->tiles_per_cta; s.rows_per_cta = h->rows_per_cta;
+    cfg.gridDim = dim3((unsigned)B); cfg.blockDim = dim3(HEAD_SEL_THREADS); cfg.dynamicSmemBytes = 0;
     if (cudaLaunchKernelEx(&cfg, tfe_head_select_kernel, s) != cudaSuccess) { (void)cudaGetLastError(); return TFE_ERR_CUDA; }
     return TFE_OK;
 }
@@ -814,3 +828,10 @@ tfe_status tfe_head_geometry(const tfe_head *h, int32_t *grid, int32_t *rows_per
 }
 
 }  // extern "C"
+
+#ifdef HEAD_TIMELINE
+extern "C" int tfe_head_debug_timeline(long long *host16)
+{
+    return (int)cudaMemcpyFromSymbol(host16, g_head_tl, sizeof(long long) * 16);
+}
+#endif

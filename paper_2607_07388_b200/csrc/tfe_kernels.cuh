@@ -98,48 +98,17 @@ __device__ __forceinline__ unsigned long long tfe_make_record(uint32_t tag, uint
 
 // -------------------------------------------------------------- small helpers
 
-#ifndef TFE_LD_MODE
-#define TFE_LD_MODE 2
-#endif
-__device__ __forceinline__ uint4 ld_stream(const uint4 *p)   // touched once: do not keep in L1
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p)   // touched once: cached in L2 only
 {
     uint4 v;
-#if TFE_LD_MODE == 0
-    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-#elif TFE_LD_MODE == 1
-    asm volatile("ld.global.L1::no_allocate.L2::evict_first.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-#elif TFE_LD_MODE == 2
     asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-#elif TFE_LD_MODE == 3
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-#endif
     return v;
 }
-#ifndef TFE_ST_MODE
-#define TFE_ST_MODE 0
-#endif
 __device__ __forceinline__ void st_stream(uint4 *p, uint4 v)
 {
-#if TFE_ST_MODE == 0
     asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};"
                  :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-#elif TFE_ST_MODE == 1
-    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};"
-                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-#elif TFE_ST_MODE == 2
-    asm volatile("st.global.cg.v4.u32 [%0], {%1,%2,%3,%4};"
-                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-#elif TFE_ST_MODE == 3
-    asm volatile("st.global.wt.v4.u32 [%0], {%1,%2,%3,%4};"
-                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-#elif TFE_ST_MODE == 4
-    asm volatile("st.global.L1::no_allocate.L2::evict_last.v4.u32 [%0], {%1,%2,%3,%4};"
-                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-#endif
 }
 __device__ __forceinline__ uint4 ld_row(const uint4 *p)      // read-only table data
 {
@@ -969,9 +938,7 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
         if (p.slot_stats != nullptr && my_slot >= 0) tfe_touch_slot(p.slot_stats, my_slot, epoch);
     }
 
-#ifndef TFE_HACK_NOCLOSE
     tfe_closing_block_epilogue(p, 1, tag, !RANGED || p.finalize != 0);
-#endif
 }
 
 // ------------------------------------------------------------ streaming copy
