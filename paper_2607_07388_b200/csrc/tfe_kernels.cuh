@@ -255,7 +255,7 @@ __device__ __forceinline__ void load_memory(const uint4 *const (&rowp)[ALL ? 4 :
 
 // The ordered miss list of a call, built by one whole block: ascending entry index = ascending (q, order).
 // `total` is the number of misses the blocks reported.  Every record is checked for this call's tag and read
-// again (bounded) while it still shows an older one: the LONGEST / CONST kernels report without a fence, so a
+// again (bounded) while it still shows an older one: the lookup kernels report without a fence, so a
 // report can be seen before the records it covers.  The block then publishes TOTAL, closes the call (SEQ) and
 // re-arms the launch state.
 __device__ __forceinline__ void tfe_compact_misses(const TfeLookupParams &p, uint32_t total, int cols, uint32_t tag)
@@ -323,36 +323,10 @@ __device__ __forceinline__ void tfe_compact_misses(const TfeLookupParams &p, uin
     }
 }
 
-// End of a lookup block of the general kernel.  Every thread has written its result records; `my_miss` is
-// warp-uniform.  Blocks add their miss counts to RUNNING and tick DONE (one 64-bit atomic); the block that
-// finishes last builds the miss list.
-__device__ __forceinline__ void tfe_finish_block(const TfeLookupParams &p, uint32_t my_miss, int cols, uint32_t tag)
-{
-    __shared__ uint32_t s_miss, s_last, s_total;
-    const int lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) s_miss = 0;
-    __syncthreads();
-    // ---- hand the block's miss count in; the block that finishes last builds the list
-    __threadfence();                       // this thread's records, device-wide
-    if (lane == 0 && my_miss) atomicAdd(&s_miss, my_miss);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        // one atomic carries both: blocks done (low word) and misses so far (high word)
-        const unsigned long long before = atomicAdd(
-            reinterpret_cast<unsigned long long *>(&p.counters[TFE_CTR_DONE]), ((unsigned long long)s_miss << 32) | 1ull);
-        s_last = (uint32_t)before == gridDim.x - 1;
-        s_total = (uint32_t)(before >> 32) + s_miss;
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    tfe_compact_misses(p, s_total, cols, tag);
-}
-
-// The LONGEST / CONST kernels take this hand-over off the end of the launch, where a fence and an atomic
-// round trip in every block sit between the last byte of one launch and the first of the next (0.85 us of the
-// 32 us the 32,768-position prefill call takes).  What the miss list needs is complete once a warp's last probe
-// is on record, well before its last row has streamed, so:
+// The hand-over from the blocks of a lookup to the one that builds the miss list is kept off the end of the
+// launch, where a fence and an atomic round trip in every block would sit between the last byte of one launch
+// and the first of the next (a decode call of 64 positions: 7.1 -> 5.1 us).  What the miss list needs is
+// complete once a warp's last probe is on record, well before its last row has streamed, so:
 //   * every WARP reports then (tfe_warp_probing_done): a shared-memory atomic, and from the warp that completes
 //     its block one reduction on DONE / RUNNING that nobody waits for.  No fence: records carry the call's tag
 //     and the reader checks it;
@@ -552,9 +526,17 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
     const uint32_t n_batches = (p.Q + qb - 1) / qb;
     uint32_t my_miss = 0;                        // per thread here; summed per warp below
 
+    __shared__ TfeProbeTick s_tick;
+    if (threadIdx.x == 0) s_tick.warps_and_misses = 0ull;
+    __syncthreads();
     tfe_grid_dependency_sync();
     const uint32_t tag = tfe_call_tag(p.counters);
     const uint32_t n_warps = gridDim.x * TFE_WARPS_PER_BLOCK;
+    // ALL / CONST reports after its rows instead of after its last probe: with the report inside the
+    // batch loop that instantiation measured 58.4 us on the 32,768-token prefill, 49.4 us this way
+    // (the gated ones gained from the early report: LONGEST 35.4 -> 34.4 us, ALL decode 8.1 -> 6.5 us)
+    constexpr bool LATE_TICK = ALL && !COS;
+    if (!LATE_TICK && blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5) >= n_batches) tfe_warp_probing_done(p, &s_tick, 0u);     // a warp without queries
     for (uint32_t batch = blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5); batch < n_batches; batch += n_warps) {
         // query lq of batch b is b + lq * n_batches: the queries of a warp are spread over the call,
         // so a run of consecutive positions that all hit is shared out among many warps
@@ -594,6 +576,8 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
         }
 
         if (p.slot_stats != nullptr && my_slot >= 0) tfe_touch_slot(p.slot_stats, my_slot, __ldcg(p.epoch));
+        if (!LATE_TICK && batch + n_warps >= n_batches)        // this warp's last probe is on record: report (its rows are still to stream)
+            tfe_warp_probing_done(p, &s_tick, __reduce_add_sync(0xFFFFFFFFu, my_miss));
 
         // ================================ gather phase ===============================
         for (uint32_t lq = 0; lq < qb; ++lq) {
@@ -737,8 +721,8 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
         }
     }
 
-    my_miss = __reduce_add_sync(0xFFFFFFFFu, my_miss);
-    tfe_finish_block(p, my_miss, cols, tag);
+    if (LATE_TICK) tfe_warp_probing_done(p, &s_tick, __reduce_add_sync(0xFFFFFFFFu, my_miss));
+    tfe_closing_block_epilogue(p, cols, tag, true);
 }
 
 // ------------------------------------- the hot path, LONGEST / CONST version
