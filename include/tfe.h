@@ -291,18 +291,33 @@ tfe_status tfe_cache_policy_enable(tfe_ctx *ctx, void *stream);
  * use, then by slot.  half_life -> large gives least-frequently-used order, equal frequencies
  * give least-recently-used order.
  *
- *   n        0..4096;  slots HOST int32 [n], or NULL;  keys HOST uint32 [n] or NULL;
+ *   n        0..4096;  half_life at most 2^26 - 1;  slots HOST int32 [n], or NULL;  keys HOST uint32 [n] or NULL;
  *   count    HOST: entries written = min(n, gpu_slots).
- * Six kernel launches on `stream`; with host `slots` the results are copied there and the
- * stream is synchronised (they feed tfe_cache_install, which takes host arrays); with slots =
- * NULL nothing is copied and nothing synchronises.  tfe_cache_select_victims_device returns the
- * DEVICE copies of the most recent selection (owned by the context, valid until the next one;
- * they feed tfe_cache_install_device).
- * Errors: INVALID_ARG (also: policy not enabled), CUDA.
+ * One cooperative kernel launch on `stream` (one block per SM; its blocks wait for one another at
+ * four or more step boundaries, every wait bounded) after a 64 KiB clear of its work space.  The
+ * per-slot bookkeeping is read once; a threshold taken from a sample of the slots keeps the work
+ * after that pass to a candidate list, and the result does not depend on the sample: a threshold
+ * that turns out too low or too high only makes the call walk the table again.  With host `slots`
+ * the results are copied there and the stream is synchronised (they feed tfe_cache_install, which
+ * takes host arrays); with slots = NULL nothing is copied and nothing synchronises.
+ * tfe_cache_select_victims_device returns the DEVICE copies of the most recent selection (owned
+ * by the context, valid until the next one; they feed tfe_cache_install_device).
+ * Errors: INVALID_ARG (also: policy not enabled), CUDA, INTERNAL (host `slots` only: a wait inside
+ * the kernel ran out or its counts contradicted one another; the outputs are not valid).
  */
 tfe_status tfe_cache_select_victims(tfe_ctx *ctx, int32_t n, int32_t half_life, int32_t *slots,
                                     uint32_t *keys, int32_t *count, void *stream);
 tfe_status tfe_cache_select_victims_device(tfe_ctx *ctx, const int32_t **slots, const uint32_t **keys);
+
+/*
+ * tfe_cache_select_tuning -- sizes of the selection's internal steps, for tests and tuning; the
+ * result of tfe_cache_select_victims does not depend on them.  list_cap: entries of the candidate
+ * list (1..1048576), final_cap: numbers the last step ranks (..8192; at least n + 1 is used; a table
+ * with more slots than either is sampled for a threshold), n_samples: slots sampled
+ * (..2048).  0 or less: the default.  Takes effect with the next selection.
+ * Errors: INVALID_ARG.
+ */
+tfe_status tfe_cache_select_tuning(tfe_ctx *ctx, int32_t list_cap, int32_t final_cap, int32_t n_samples);
 
 /*
  * tfe_cache_stats -- copies the bookkeeping to the host: freq_last HOST uint32 [gpu_slots][2]

@@ -34,7 +34,8 @@ EXPORTS = ["tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tf
            "tfe_launch_geometry", "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
            "tfe_cache_policy_enable", "tfe_cache_select_victims", "tfe_cache_select_victims_device",
            "tfe_cache_stats", "tfe_head_create", "tfe_head_destroy", "tfe_head_topk", "tfe_head_buffers",
-           "tfe_head_status", "tfe_head_geometry", "tfe_mine_ngrams", "tfe_mine_workspace_bytes", "tfe_assign_residency", "tfe_stream_copy"]
+           "tfe_head_status", "tfe_head_geometry", "tfe_mine_ngrams", "tfe_mine_workspace_bytes", "tfe_assign_residency", "tfe_stream_copy",
+           "tfe_cache_select_tuning"]
 
 
 class TfeConfig(C.Structure):
@@ -113,12 +114,13 @@ def lib() -> C.CDLL:
         L.tfe_assign_residency.argtypes = [vp, i64, i64, C.c_uint32, vp, vp, vp]
         L.tfe_mine_workspace_bytes.restype = i64
         L.tfe_stream_copy.argtypes = [vp, vp, i64, vp]
+        L.tfe_cache_select_tuning.argtypes = [vp, i32, i32, i32]
         for name in ("tfe_index_build", "tfe_index_build_device", "tfe_cache_install", "tfe_cache_install_device", "tfe_lookup_inject", "tfe_lookup_inject_host",
                      "tfe_miss_list", "tfe_miss_list_device", "tfe_index_geometry", "tfe_launch_geometry",
                      "tfe_set_tuning", "tfe_lookup_inject_noalloc", "tfe_prefetch_candidates",
                      "tfe_cache_policy_enable", "tfe_cache_select_victims", "tfe_cache_select_victims_device",
                      "tfe_cache_stats", "tfe_head_create", "tfe_head_topk", "tfe_head_buffers", "tfe_head_status",
-                     "tfe_head_geometry", "tfe_mine_ngrams", "tfe_assign_residency"):
+                     "tfe_head_geometry", "tfe_mine_ngrams", "tfe_assign_residency", "tfe_cache_select_tuning"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -264,6 +266,10 @@ def tfe_cache_select_victims(ctx: int, n: int, half_life: int = 0, stream=None):
     _check(lib().tfe_cache_select_victims(ctx, int(n), int(half_life), _addr(slots), _addr(keys), C.byref(cnt),
                                           _stream(stream)), "tfe_cache_select_victims")
     return slots[:cnt.value], keys[:cnt.value]
+
+
+def tfe_cache_select_tuning(ctx: int, list_cap: int = 0, final_cap: int = 0, n_samples: int = 0) -> None:
+    _check(lib().tfe_cache_select_tuning(ctx, int(list_cap), int(final_cap), int(n_samples)), "tfe_cache_select_tuning")
 
 
 def tfe_cache_select_victims_async(ctx: int, n: int, half_life: int = 0, stream=None) -> int:

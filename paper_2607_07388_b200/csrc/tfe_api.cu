@@ -6,6 +6,7 @@
 // used to validate arguments before anything is launched.
 #include <algorithm>
 #include <climits>
+#include <cmath>
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
@@ -99,10 +100,12 @@ struct tfe_ctx {
     // the victim selection's work space
     uint2 *d_slot_stats = nullptr;
     uint32_t *d_epoch = nullptr;
-    uint32_t *d_slot_key = nullptr, *d_vs_hist = nullptr, *d_vs_keys = nullptr;
+    uint32_t *d_vs_keys = nullptr;
     TfeVictimState *d_vs_state = nullptr;
-    unsigned long long *d_vs_list = nullptr;
+    unsigned long long *d_vs_list = nullptr, *d_vs_fin = nullptr;
     int32_t *d_vs_slots = nullptr;
+    int vs_grid_max = 0;                    // blocks of the selection kernel the device holds at once
+    int32_t vs_list_cap = 0, vs_final_cap = 0, vs_samples = 0;     // 0: the defaults (tfe_cache_select_tuning)
 
     bool mirror_ready = true;               // h_slot / h_owner filled (a device build fills them on first use)
     bool device_installs = false;           // tfe_cache_install_device was used: replays of a captured call change the
@@ -367,7 +370,7 @@ void tfe_destroy(tfe_ctx *c)
     free_dev(c->d_h_phrase); free_dev(c->d_h_slot); free_dev(c->d_h_flag);
     free_dev(c->d_pf_keys); free_dev(c->d_pf_phrase); free_dev(c->d_pf_tier); free_dev(c->d_pf_counter);
     free_dev(c->d_phrase_stamp); free_dev(c->d_slot_stamp); free_dev(c->d_inst_count);
-    free_dev(c->d_slot_stats); free_dev(c->d_epoch); free_dev(c->d_slot_key); free_dev(c->d_vs_hist);
+    free_dev(c->d_slot_stats); free_dev(c->d_epoch); free_dev(c->d_vs_fin);
     free_dev(c->d_vs_keys); free_dev(c->d_vs_state); free_dev(c->d_vs_list); free_dev(c->d_vs_slots);
     if (c->hb_in) (void)cudaStreamDestroy(c->hb_in);
     if (c->hb_out) (void)cudaStreamDestroy(c->hb_out);
@@ -1069,54 +1072,91 @@ tfe_status tfe_cache_policy_enable(tfe_ctx *c, void *stream_)
         uint2 *stats = nullptr;
         CU(cudaMalloc(&stats, C * sizeof(uint2)));
         CU(cudaMalloc(&c->d_epoch, sizeof(uint32_t)));
-        CU(cudaMalloc(&c->d_slot_key, C * sizeof(uint32_t)));
-        CU(cudaMalloc(&c->d_vs_hist, TFE_VICTIM_BINS * sizeof(uint32_t)));
         CU(cudaMalloc(&c->d_vs_state, sizeof(TfeVictimState)));
-        CU(cudaMalloc(&c->d_vs_list, TFE_VICTIMS_MAX * sizeof(unsigned long long)));
+        CU(cudaMalloc(&c->d_vs_list, (size_t)TFE_VS_LIST_CAP * sizeof(unsigned long long)));
+        CU(cudaMalloc(&c->d_vs_fin, (size_t)TFE_VS_FINAL_CAP * sizeof(unsigned long long)));
+        CU(cudaFuncSetAttribute(tfe_victim_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TFE_VS_DYN_SMEM));
+        CU(cudaFuncSetAttribute(tfe_victim_select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TFE_VS_DYN_SMEM));
+        int per_sm = 0, per_sm_plain = 0;
+        CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tfe_victim_select_kernel<true>, TFE_VS_THREADS, TFE_VS_DYN_SMEM));
+        CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm_plain, tfe_victim_select_kernel<false>, TFE_VS_THREADS, TFE_VS_DYN_SMEM));
+        if (per_sm < 1 || per_sm_plain < 1) return TFE_ERR_INTERNAL;
+        c->vs_grid_max = c->sm_count;       // one block per SM: the blocks of the launch wait for one another
         CU(cudaMalloc(&c->d_vs_slots, TFE_VICTIMS_MAX * sizeof(int32_t)));
         CU(cudaMalloc(&c->d_vs_keys, TFE_VICTIMS_MAX * sizeof(uint32_t)));
         c->d_slot_stats = stats;
     }
-    CU(cudaMemsetAsync(c->d_slot_stats, 0, C * sizeof(uint2), stream));
+    tfe_policy_reset_kernel<<<(unsigned)std::min<size_t>(4096, (C + 255) / 256), 256, 0, stream>>>(c->d_slot_stats, c->d_slot_owner,
+                                                                                                    (uint32_t)C);
+    CU(cudaGetLastError());
     CU(cudaMemsetAsync(c->d_epoch, 0, sizeof(uint32_t), stream));
-    CU(cudaMemsetAsync(c->d_vs_hist, 0, TFE_VICTIM_BINS * sizeof(uint32_t), stream));
     return TFE_OK;
 }
 
 tfe_status tfe_cache_select_victims(tfe_ctx *c, int32_t n, int32_t half_life, int32_t *slots, uint32_t *keys,
                                     int32_t *count, void *stream_)
 {
-    if (!c || n < 0 || n > TFE_VICTIMS_MAX || !count) return TFE_ERR_INVALID_ARG;
+    if (!c || n < 0 || n > TFE_VICTIMS_MAX || !count || half_life > TFE_HALF_LIFE_MAX) return TFE_ERR_INVALID_ARG;
     if (!c->d_slot_stats) return TFE_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const int64_t C = c->cfg.gpu_slots;
     const int32_t take = (int32_t)std::min<int64_t>(n, C);
     *count = take;
     if (take == 0) return TFE_OK;
+    TfeVictimParams p{};
+    p.slot_stats = c->d_slot_stats; p.epoch = c->d_epoch;
+    p.div_half_life = make_fastdiv(half_life > 0 ? (uint32_t)half_life : 1u);
+    p.age_cap = half_life > 0 ? 32u * (uint32_t)half_life : 0u;
+    p.C = (uint32_t)C; p.take = (uint32_t)take;
+    p.list_cap = (uint32_t)(c->vs_list_cap > 0 ? c->vs_list_cap : TFE_VS_LIST_CAP);
+    p.final_cap = (uint32_t)std::max<int32_t>(take + 1, c->vs_final_cap > 0 ? c->vs_final_cap : TFE_VS_FINAL_DEFAULT);
+    p.range_cap = c->vs_final_cap > 0 ? (uint32_t)std::max(1, std::min(c->vs_final_cap / 2, TFE_VS_FINAL_CAP - TFE_VICTIMS_MAX))
+                                      : (uint32_t)TFE_VS_RANGE_DEFAULT;
+    if (C > (int64_t)std::min(p.list_cap, p.final_cap)) {     // else: the whole table goes to the final step
+        // a threshold from S sampled slots: the take-th smallest number has rank ~ Poisson(mu) among them,
+        // mu = take * S / C; the rank used is six standard deviations and a margin above that
+        // (S by default: about three samples expected below the take-th smallest -- more only make the merge longer)
+        int64_t S = TFE_VS_SAMPLES;
+        while (S > 64 && (double)take * (double)(S / 2) / (double)C >= 3.0) S /= 2;
+        if (c->vs_samples > 0) S = c->vs_samples;
+        S = std::min<int64_t>(C, S);
+        const double mu = (double)take * (double)S / (double)C;
+        p.n_samples = (uint32_t)S;
+        p.sample_stretch = (uint32_t)(C / S); p.sample_longer = (uint32_t)(C % S);
+        p.sample_rank = (uint32_t)std::min<double>((double)S, std::ceil(mu + 6.0 * std::sqrt(mu) + 6.0));
+    }
+    p.list = c->d_vs_list; p.fin = c->d_vs_fin; p.st = c->d_vs_state;
+    p.out_slots = c->d_vs_slots; p.out_keys = c->d_vs_keys;
     CU(cudaMemsetAsync(c->d_vs_state, 0, sizeof(TfeVictimState), stream));
-    const unsigned grid = (unsigned)std::max<int64_t>(
-        1, std::min<int64_t>((int64_t)c->sm_count * 4, (C + 4 * TFE_VICTIM_THREADS - 1) / (4 * TFE_VICTIM_THREADS)));
-    static const int kShift[3] = {53, 42, 32}, kBits[3] = {11, 11, 10};      // the key's 32 bits
-    CU(launch_overlapped(tfe_victim_pass_kernel<true>, dim3(grid), dim3(TFE_VICTIM_THREADS), stream, c->d_slot_stats,
-                         c->d_slot_owner, c->d_epoch, half_life, c->d_slot_key, (uint32_t)C, (uint32_t)take, kShift[0],
-                         kBits[0], c->d_vs_hist, c->d_vs_state));
-    for (int i = 1; i < 3; ++i)
-        CU(launch_overlapped(tfe_victim_pass_kernel<false>, dim3(grid), dim3(TFE_VICTIM_THREADS), stream, c->d_slot_stats,
-                             c->d_slot_owner, c->d_epoch, half_life, c->d_slot_key, (uint32_t)C, 0u, kShift[i], kBits[i],
-                             c->d_vs_hist, c->d_vs_state));
-    static_assert(TFE_VICTIM_BINS >= 4 * 256, "the histogram array doubles as one counter per block");
-    if (grid > 2 * TFE_VICTIM_THREADS) return TFE_ERR_INTERNAL;      // two range counts per thread of the closing block
-    CU(launch_overlapped(tfe_victim_tie_kernel, dim3(grid), dim3(TFE_VICTIM_THREADS), stream, c->d_slot_key, (uint32_t)C,
-                         c->d_vs_hist, c->d_vs_state));
-    CU(launch_overlapped(tfe_victim_collect_kernel, dim3(grid), dim3(TFE_VICTIM_THREADS), stream, c->d_slot_key, (uint32_t)C,
-                         c->d_vs_state, c->d_vs_list, (uint32_t)TFE_VICTIMS_MAX));
-    CU(launch_overlapped(tfe_victim_sort_kernel, dim3(1), dim3(1024), stream, c->d_vs_list, c->d_vs_state, (uint32_t)take,
-                         c->d_vs_slots, c->d_vs_keys));
+    {
+        const int64_t n_quads = (C + 3) / 4;
+        cudaLaunchConfig_t cfg{};
+        // a small table keeps at least 32 blocks: the final step's cost is shared by the blocks, whatever the table's size
+        cfg.gridDim = dim3((unsigned)std::max<int64_t>(std::min(32, c->vs_grid_max), std::min<int64_t>(c->vs_grid_max, (n_quads + TFE_VS_THREADS - 1) / TFE_VS_THREADS)));
+        if (take > 512) cfg.gridDim = dim3((unsigned)c->vs_grid_max);
+        cfg.blockDim = dim3(TFE_VS_THREADS); cfg.dynamicSmemBytes = TFE_VS_DYN_SMEM; cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeCooperative;      // the blocks wait for one another: resident together
+        attr[0].val.cooperative = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        CU(cudaLaunchKernelEx(&cfg, half_life > 0 ? tfe_victim_select_kernel<true> : tfe_victim_select_kernel<false>, p));
+    }
     CU(cudaGetLastError());
     if (!slots) return TFE_OK;      // results stay on the device (tfe_cache_select_victims_device); no synchronisation
     CU(cudaMemcpyAsync(slots, c->d_vs_slots, (size_t)take * 4, cudaMemcpyDeviceToHost, stream));
     if (keys) CU(cudaMemcpyAsync(keys, c->d_vs_keys, (size_t)take * 4, cudaMemcpyDeviceToHost, stream));
+    uint32_t dev_status = 0;
+    CU(cudaMemcpyAsync(&dev_status, &c->d_vs_state->status, sizeof(uint32_t), cudaMemcpyDeviceToHost, stream));
     CU(cudaStreamSynchronize(stream));
+    return dev_status ? TFE_ERR_INTERNAL : TFE_OK;
+}
+
+tfe_status tfe_cache_select_tuning(tfe_ctx *c, int32_t list_cap, int32_t final_cap, int32_t n_samples)
+{
+    if (!c || list_cap > TFE_VS_LIST_CAP || final_cap > TFE_VS_FINAL_CAP || n_samples > TFE_VS_SAMPLES) return TFE_ERR_INVALID_ARG;
+    c->vs_list_cap = std::max(0, list_cap);
+    c->vs_final_cap = std::max(0, final_cap);
+    c->vs_samples = std::max(0, n_samples);
     return TFE_OK;
 }
 
@@ -1137,6 +1177,9 @@ tfe_status tfe_cache_stats(tfe_ctx *c, uint32_t *freq_last, uint32_t *epoch, voi
                            stream));
     if (epoch) CU(cudaMemcpyAsync(epoch, c->d_epoch, sizeof(uint32_t), cudaMemcpyDeviceToHost, stream));
     CU(cudaStreamSynchronize(stream));
+    if (freq_last)                          // the device marks a slot without owner in its freq word; it has served nothing
+        for (int64_t i = 0; i < c->cfg.gpu_slots; ++i)
+            if (freq_last[2 * i] == TFE_FREE_SLOT_FREQ) freq_last[2 * i] = 0u;
     return TFE_OK;
 }
 

@@ -1268,340 +1268,555 @@ tfe_prefetch_select_kernel(const unsigned long long *keys, const uint32_t *entry
 //     age = now - last,  decayed = freq >> min(31, age / half_life)   (half_life <= 0: no decay)
 //     key = min(decayed, 65535) << 16 | (65535 - min(age, 65535)),    0 for a slot without owner
 // and the victims are the n slots of smallest (key, slot).  (key << 32 | slot) is a distinct
-// 64-bit number per slot, so this is a selection of the n smallest of C distinct numbers:
+// 64-bit number per slot, so this is a selection of the n smallest of C distinct numbers, and it is
+// ONE cooperative launch (tfe_victim_select_kernel, one block per SM) that reads the 8 bytes of
+// bookkeeping per slot once (a slot without owner is marked in its freq word):
 //
-//   tfe_victim_pass_kernel   x3 over the key's 32 bits, most significant digit first (11,11,10 bits):
-//                            histogram of the digit over the slots that agree with the digits chosen so
-//                            far; the block that finishes last picks the digit holding the n-th smallest
-//                            and re-arms the histogram.  The first pass computes and stores the keys.
-//   tfe_victim_tie_kernel    the slot half of the n-th smallest: a count of the slots that hold exactly
-//                            its key, in slot (= memory) order, instead of three more digit passes
-//   tfe_victim_collect_kernel  appends every number <= the n-th smallest to a list (any order)
-//   tfe_victim_sort_kernel     one block: bitonic sort of the list, writes slots and keys
+//   threshold   block 0 draws up to 2,048 slots, one from each of as many equal stretches of the table, and
+//               publishes a threshold T that r or more of their numbers do not exceed; r sits six standard
+//               deviations above the expected rank of the n-th smallest in the sample, so that n or more of
+//               all numbers are <= T, but not many more (c4: ~90,000 of 16.8 M).  A table that fits the final
+//               step whole skips this (T = max).
+//   scan        the one pass over {freq, last}: every number <= T goes to a candidate list (collected per
+//               block in shared memory, handed over with one atomic per 1,024) and is counted by its distance
+//               below T on a logarithmic scale, 128 steps per octave.
+//   narrow      from those counts: the piece of the scale that holds the n-th smallest, and how many numbers
+//               lie beyond it.  Mostly the piece holds few enough to go on; else
+//   refine      a histogram of the candidates over 2,048 equal parts of the piece, the part that holds the
+//               n-th smallest becomes the new piece; repeated while it is too full.
+//   final       everything up to the piece's upper end is gathered (n plus at most a few thousand numbers),
+//               every block copies the set to shared memory and its warps place one number each by counting
+//               the smaller ones; ranks below n are the result, already sorted.
+//
+// The result never depends on the sample: if fewer than n numbers turn out to be <= T, or more than the
+// list holds, the later steps walk the table itself instead of the list (slower, same answer).
+// Blocks wait for one another at the step boundaries (a counter in global memory, release / acquire); the
+// launch is cooperative, so they are resident together, and every wait is bounded.
 #define TFE_VICTIMS_MAX 4096
-#define TFE_VICTIM_BINS 2048
+#define TFE_VS_THREADS 1024
+#define TFE_VS_BINS 2048
+#define TFE_VS_LIST_CAP (1024 * 1024)    // candidate list entries (8 MiB): the sampled threshold admits ~7 * C / 2,048 or more
+#define TFE_VS_FINAL_CAP 8192            // most numbers the final step ranks; also the shared-memory buffer's entries
+#define TFE_VS_FINAL_DEFAULT 5120        // refine until this many are left to rank ...
+#define TFE_VS_RANGE_DEFAULT 2048        // ... or this many above the ones that are certain
+#define TFE_VS_SAMPLES 2048
+#define TFE_VS_MAX_REFINE 8              // a refine step shrinks hi - lo at least 1,024-fold: 7 cover 64 bits
+#define TFE_VS_DYN_SMEM (TFE_VS_FINAL_CAP * 8)
+#define TFE_VS_NEAR_MANT 7                                   // bits of T - number kept below its leading one
+#define TFE_VS_NEAR_BINS ((64 - TFE_VS_NEAR_MANT + 1) << TFE_VS_NEAR_MANT)      // 7,424
+
+#define TFE_VS_ERR_BARRIER 1u            // a wait at a step boundary ran out
+#define TFE_VS_ERR_INTERNAL 2u           // counts that contradict one another
 
 struct TfeVictimState {
-    unsigned long long prefix;      // digits chosen so far, in place
-    uint32_t k_rem;                 // rank (1-based) of the wanted number among those sharing the prefix
-    uint32_t ticket;                // blocks done in the current pass
-    uint32_t n_out;                 // entries appended by the collect kernel
+    uint32_t arrived;               // blocks through the step boundaries so far
+    uint32_t n_cand;                // numbers <= T seen by the scan (entries beyond the list's capacity are dropped)
+    uint32_t n_final;               // numbers gathered for the final step
+    uint32_t status;                // TFE_VS_ERR_*
+    uint32_t threshold_ready;       // block 0 has published `threshold`
     uint32_t pad;
+    unsigned long long threshold;
+    uint32_t near[TFE_VS_NEAR_BINS];   // candidates by tfe_vs_near_bin(T - number)
+    uint32_t hist[TFE_VS_MAX_REFINE][TFE_VS_BINS];
 };
 
-__device__ __forceinline__ uint32_t tfe_retention_key(uint2 st, uint32_t owner, uint32_t now, int32_t half_life)
+struct TfeVictimParams {
+    const uint2 *slot_stats;        // [C4] {freq, last}; freq = TFE_FREE_SLOT_FREQ marks a slot without owner
+    const uint32_t *epoch;
+    TfeFastDiv div_half_life;       // for half_life > 0 ...
+    uint32_t age_cap;               // ... with 32 * half_life
+    uint32_t C, take;
+    uint32_t n_samples, sample_rank;    // 0 samples: no threshold
+    uint32_t sample_stretch, sample_longer;     // C / n_samples, C % n_samples
+    uint32_t list_cap, final_cap, range_cap;    // refine until <= final_cap numbers are left to rank, or <= range_cap above the certain ones
+    unsigned long long *list;       // [list_cap]
+    unsigned long long *fin;        // [TFE_VS_FINAL_CAP]
+    TfeVictimState *st;
+    int32_t *out_slots;             // [take]
+    uint32_t *out_keys;             // [take]
+};
+
+// A slot without owner carries freq = TFE_FREE_SLOT_FREQ in its bookkeeping (written when the policy is enabled;
+// a slot only ever goes from free to owned, and the installation overwrites the mark), so the ranking reads the
+// 8 bytes of {freq, last} per slot and nothing else.
+#define TFE_FREE_SLOT_FREQ 0xFFFFFFFFu
+#define TFE_HALF_LIFE_MAX ((1 << 26) - 1)       // 32 * half_life stays below 2^31
+
+__global__ void __launch_bounds__(256) tfe_policy_reset_kernel(uint2 *slot_stats, const uint32_t *slot_owner, uint32_t C)
 {
-    if (owner == 0xFFFFFFFFu) return 0u;
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < C; i += gridDim.x * blockDim.x)
+        slot_stats[i] = make_uint2(slot_owner[i] == 0xFFFFFFFFu ? TFE_FREE_SLOT_FREQ : 0u, 0u);
+}
+
+// DECAY: half_life > 0.  age_cap = 32 * half_life (below 2^31, which the fast division needs): the quotient
+// saturates at 31 from there on.
+template <bool DECAY>
+__device__ __forceinline__ uint32_t tfe_retention_key(uint2 st, uint32_t now, TfeFastDiv div, uint32_t age_cap)
+{
     const uint32_t age = now - st.y;
-    const uint32_t shift = half_life > 0 ? min(31u, age / (uint32_t)half_life) : 0u;
-    return (min(st.x >> shift, 65535u) << 16) | (65535u - min(age, 65535u));
+    uint32_t decayed = st.x;
+    if (DECAY) decayed >>= min(31u, tfe_div(min(age, age_cap), div));
+    const uint32_t key = (min(decayed, 65535u) << 16) | (65535u - min(age, 65535u));
+    return st.x == TFE_FREE_SLOT_FREQ ? 0u : key;
 }
 
-#define TFE_VICTIM_THREADS 512
+#define TFE_VS_NONE 0xFFFFFFFFFFFFFFFFull       // never a slot's number: slots are below 2^31
 
-// slot_stats, slot_owner and slot_key hold a multiple of 4 entries (the tail is padding).
-template <bool FIRST>
-__global__ void __launch_bounds__(TFE_VICTIM_THREADS)
-tfe_victim_pass_kernel(const uint2 *slot_stats, const uint32_t *slot_owner, const uint32_t *epoch, int32_t half_life,
-                       uint32_t *slot_key, uint32_t C, uint32_t n_first, int shift, int bits, uint32_t *hist,
-                       TfeVictimState *state)
+// Distance d = T - number of a candidate on a logarithmic scale with 128 steps per octave: d itself below 128,
+// else the position of its leading one and the seven bits after it.  Grows with d; bin b >= 128 covers
+// [m << s, ((m + 1) << s) - 1] with m = 128 + (b & 127), s = (b >> 7) - 1.
+__device__ __forceinline__ uint32_t tfe_vs_near_bin(unsigned long long d)
 {
-    __shared__ uint32_t s_hist[TFE_VICTIM_BINS];
-    __shared__ uint32_t s_part[256];
-    __shared__ uint32_t s_last;
-    for (int i = threadIdx.x; i < TFE_VICTIM_BINS; i += blockDim.x) s_hist[i] = 0;
-    __syncthreads();
-    tfe_grid_dependency_sync();                 // the pass before this one decides the prefix
-    const unsigned long long prefix = FIRST ? 0ull : state->prefix;
-    const uint32_t now = FIRST ? *epoch : 0u;
-    const int above = shift + bits;             // bits above this digit are decided
-    const uint32_t mask = (1u << bits) - 1u;
-    const uint32_t n_quads = (C + 3u) >> 2;
-    const uint32_t n_round = (n_quads + 31u) & ~31u;    // whole warps stay together for the match
-    const uint32_t stride = gridDim.x * blockDim.x;
-    uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
-    uint4 nxt = make_uint4(0, 0, 0, 0);         // the keys one iteration ahead (later passes)
-    if (!FIRST && g < n_quads) nxt = reinterpret_cast<const uint4 *>(slot_key)[g];
-    for (; g < n_round; g += stride) {
-        uint32_t key[4] = {0, 0, 0, 0};
-        if (FIRST) {
-            if (g < n_quads) {
-                const uint4 a = __ldcs(reinterpret_cast<const uint4 *>(slot_stats) + 2 * g);
-                const uint4 b = __ldcs(reinterpret_cast<const uint4 *>(slot_stats) + 2 * g + 1);
-                const uint4 o = __ldcs(reinterpret_cast<const uint4 *>(slot_owner) + g);
-                key[0] = tfe_retention_key(make_uint2(a.x, a.y), o.x, now, half_life);
-                key[1] = tfe_retention_key(make_uint2(a.z, a.w), o.y, now, half_life);
-                key[2] = tfe_retention_key(make_uint2(b.x, b.y), o.z, now, half_life);
-                key[3] = tfe_retention_key(make_uint2(b.z, b.w), o.w, now, half_life);
-                reinterpret_cast<uint4 *>(slot_key)[g] = make_uint4(key[0], key[1], key[2], key[3]);
-            }
-        } else {
-            key[0] = nxt.x; key[1] = nxt.y; key[2] = nxt.z; key[3] = nxt.w;
-            if (g + stride < n_quads) nxt = reinterpret_cast<const uint4 *>(slot_key)[g + stride];
-        }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const uint32_t s0 = 4 * g + j;
-            const unsigned long long comp = ((unsigned long long)key[j] << 32) | s0;
-            const bool live = s0 < C && g < n_quads && (above >= 64 || (comp >> above) == (prefix >> above));
-            const uint32_t digit = (uint32_t)(comp >> shift) & mask;
-            // one shared-memory atomic per distinct digit of the warp
-            const uint32_t vote = __ballot_sync(0xFFFFFFFFu, live);
-            if (live) {
-                const uint32_t peers = __match_any_sync(vote, digit);
-                if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&s_hist[digit], __popc(peers));
-            }
-        }
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < TFE_VICTIM_BINS; i += blockDim.x)
-        if (s_hist[i]) atomicAdd(&hist[i], s_hist[i]);
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_last = atomicAdd(&state->ticket, 1u) == gridDim.x - 1;
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    // ---- last block: the digit whose bin holds the k_rem-th smallest
-    constexpr int PER = TFE_VICTIM_BINS / 256;
-    uint32_t mine[PER], sum = 0;
-    if (threadIdx.x < 256) {
-#pragma unroll
-        for (int j = 0; j < PER; ++j) {
-            mine[j] = __ldcg(hist + threadIdx.x * PER + j);
-            hist[threadIdx.x * PER + j] = 0;
-            sum += mine[j];
-        }
-        s_part[threadIdx.x] = sum;
-    }
-    __syncthreads();
-    // inclusive scan of the 256 partial sums by the first 8 warps, then the thread whose range
-    // holds the k-th smallest announces itself
-    const uint32_t k_want = FIRST ? n_first : state->k_rem;
-    uint32_t incl = 0;
-    if (threadIdx.x < 256) {
-        incl = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-            if ((threadIdx.x & 31) >= o) incl += v;
-        }
-        if ((threadIdx.x & 31) == 31) s_hist[threadIdx.x >> 5] = incl;      // warp totals
-    }
-    __syncthreads();
-    if (threadIdx.x < 256) {
-        for (int wq = 0; wq < (int)(threadIdx.x >> 5); ++wq) incl += s_hist[wq];
-        if (incl >= k_want && incl - sum < k_want) {
-            s_part[0] = threadIdx.x;                // owning thread (exactly one)
-            s_hist[8] = k_want - (incl - sum);      // rank within its bins
-        }
-    }
-    __syncthreads();
-    if (threadIdx.x < 256 && threadIdx.x == s_part[0]) {
-        uint32_t k = s_hist[8];
-        int j = 0;
-        for (; j < PER - 1 && mine[j] < k; ++j) k -= mine[j];
-        state->prefix = prefix | ((unsigned long long)(threadIdx.x * PER + j) << shift);
-        state->k_rem = k;
-        state->ticket = 0;
-    }
+    if (d < (1ull << TFE_VS_NEAR_MANT)) return (uint32_t)d;
+    const int s = (63 - __clzll((long long)d)) - TFE_VS_NEAR_MANT;
+    return ((uint32_t)(s + 1) << TFE_VS_NEAR_MANT) | ((uint32_t)(d >> s) & ((1u << TFE_VS_NEAR_MANT) - 1u));
+}
+__device__ __forceinline__ void tfe_vs_near_range(uint32_t b, unsigned long long &d_min, unsigned long long &d_max)
+{
+    if (b < (1u << TFE_VS_NEAR_MANT)) { d_min = d_max = b; return; }
+    const int s = (int)(b >> TFE_VS_NEAR_MANT) - 1;
+    const unsigned long long m = (1ull << TFE_VS_NEAR_MANT) | (b & ((1u << TFE_VS_NEAR_MANT) - 1u));
+    d_min = m << s;
+    d_max = d_min + ((1ull << s) - 1ull);
 }
 
-// After the three passes over the key's 32 bits the wanted number is known to be the k_rem-th smallest
-// SLOT among those holding exactly that key.  Slot order is memory order, so no further digit passes are
-// needed: every block counts the ties of one contiguous range of slots; the block that finishes last
-// scans the per-block counts, finds the range that holds the k_rem-th tie, walks that range once more and
-// completes state->prefix with the slot.  `tie_count` is the (zeroed) histogram array, left zeroed again.
-__global__ void __launch_bounds__(TFE_VICTIM_THREADS)
-tfe_victim_tie_kernel(const uint32_t *slot_key, uint32_t C, uint32_t *tie_count, TfeVictimState *state)
+// Blocks of the launch meet: the b-th boundary is passed when b * gridDim.x arrivals are on record.
+// False when the wait ran out or another block has reported an error (the caller returns at once).
+__device__ __forceinline__ bool tfe_vs_boundary(TfeVictimState *st, uint32_t &boundary)
 {
-    __shared__ uint32_t s_warp[TFE_VICTIM_THREADS / 32];
-    __shared__ uint32_t s_last, s_block, s_rank;
-    tfe_grid_dependency_sync();
+    __shared__ uint32_t s_ok;
+    ++boundary;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        // release: the block's writes (ordered before this thread by the barrier above) are visible to whoever
+        // acquires the count
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" :: "l"(&st->arrived) : "memory");
+        const uint32_t want = boundary * gridDim.x;
+        const volatile uint32_t *status = &st->status;
+        uint32_t spin = 0, seen = 0;
+        bool ok = true;
+        for (;;) {
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(&st->arrived) : "memory");
+            if (seen >= want) break;
+            if (*status != 0u || ++spin > TFE_SPIN_LIMIT) { ok = false; break; }
+        }
+        if (!ok) atomicOr(&st->status, TFE_VS_ERR_BARRIER);
+        s_ok = ok;
+    }
+    __syncthreads();
+    return s_ok != 0u;
+}
+
+// Numbers found by the threads of a block, collected in shared memory and handed to a global list with one
+// atomic per 1,024 of them; a warp that finds many at once (a dense stretch) reserves in the global list directly.
+struct TfeVsAppender {
+    unsigned long long *buf;        // shared memory, `cap` entries, all TFE_VS_NONE before the first append
+    uint32_t *s_count;              // shared memory, entries reserved in buf (may run past cap)
+    uint32_t cap;
+    uint32_t *g_count;
+    unsigned long long *g_list;
+    uint32_t g_cap;
+};
+
+__device__ __forceinline__ void tfe_vs_append(const TfeVsAppender &a, uint32_t vote, bool have, unsigned long long v)
+{                                                       // whole warp; vote = ballot of `have`, not zero
+    const int lane = threadIdx.x & 31, leader = __ffs(vote) - 1;
+    const uint32_t n = __popc(vote), rank = __popc(vote & ((1u << lane) - 1u));
+    uint32_t base = 0;
+    if (n < 16u) {
+        if (lane == leader) base = atomicAdd(a.s_count, n);
+        base = __shfl_sync(0xFFFFFFFFu, base, leader);
+        if (base + n <= a.cap) {
+            if (have) a.buf[base + rank] = v;
+            return;
+        }
+    }
+    if (lane == leader) base = atomicAdd(a.g_count, n);
+    base = __shfl_sync(0xFFFFFFFFu, base, leader);
+    if (have && base + rank < a.g_cap) a.g_list[base + rank] = v;
+}
+
+// Whole block; leaves buf cleared and the count at zero.  s_warp: 33 words of shared memory.
+__device__ __forceinline__ void tfe_vs_flush(const TfeVsAppender &a, uint32_t *s_warp)
+{
+    __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const unsigned long long prefix = state->prefix;
-    const uint32_t key_star = (uint32_t)(prefix >> 32);
-    const uint32_t n_quads = (C + 3u) >> 2;
-    const uint32_t per_block = (n_quads + gridDim.x - 1) / gridDim.x;
-    auto ties_of = [&](uint32_t g) -> uint32_t {            // slots of quad g that hold the key
-        const uint4 k4 = __ldcg(reinterpret_cast<const uint4 *>(slot_key) + g);
-        return (uint32_t)(k4.x == key_star && 4 * g < C) + (uint32_t)(k4.y == key_star && 4 * g + 1 < C) +
-               (uint32_t)(k4.z == key_star && 4 * g + 2 < C) + (uint32_t)(k4.w == key_star && 4 * g + 3 < C);
-    };
-    {
-        const uint32_t q0 = min(n_quads, blockIdx.x * per_block), q1 = min(n_quads, q0 + per_block);
-        uint32_t mine = 0;
-        for (uint32_t g = q0 + threadIdx.x; g < q1; g += blockDim.x) mine += ties_of(g);
-        mine = __reduce_add_sync(0xFFFFFFFFu, mine);
-        if (lane == 0) s_warp[warp] = mine;
+    const uint32_t n_s = min(*a.s_count, a.cap);
+    __syncthreads();
+    for (uint32_t c0 = 0; c0 < n_s; c0 += blockDim.x) {
+        const uint32_t i = c0 + threadIdx.x;
+        const unsigned long long v = i < n_s ? a.buf[i] : TFE_VS_NONE;
+        const bool ok = v != TFE_VS_NONE;
+        const uint32_t vote = __ballot_sync(0xFFFFFFFFu, ok);
+        if (lane == 0) s_warp[warp] = __popc(vote);
         __syncthreads();
         if (threadIdx.x == 0) {
             uint32_t total = 0;
-            for (int w = 0; w < TFE_VICTIM_THREADS / 32; ++w) total += s_warp[w];
-            tie_count[blockIdx.x] = total;
-            __threadfence();
-            s_last = atomicAdd(&state->ticket, 1u) == gridDim.x - 1;
+            for (uint32_t w = 0; w < (blockDim.x >> 5); ++w) { const uint32_t c = s_warp[w]; s_warp[w] = total; total += c; }
+            s_warp[32] = total ? atomicAdd(a.g_count, total) : 0u;
         }
         __syncthreads();
-        if (!s_last) return;
-        __threadfence();
+        const uint32_t pos = s_warp[32] + s_warp[warp] + __popc(vote & ((1u << lane) - 1u));
+        if (ok && pos < a.g_cap) a.g_list[pos] = v;
+        __syncthreads();
     }
-    // ---- last block: which range holds the k_rem-th tie.  The per-block counts (at most two per thread,
-    // loaded together) are scanned in block order: first all threads' first element, then the second ones.
+    for (uint32_t i = threadIdx.x; i < a.cap; i += blockDim.x) a.buf[i] = TFE_VS_NONE;
+    if (threadIdx.x == 0) *a.s_count = 0;
+    __syncthreads();
+}
+
+// A walk over the bookkeeping of the whole table: four quads of slots (128 bytes) per thread and trip; quad g of a
+// trip belongs to thread (g mod threads of the grid), so that a stretch of the table is spread over all blocks.
+template <bool DECAY>
+struct TfeVsTableWalk {
+    static constexpr int U = 4;
+    const TfeVictimParams &p;
+    uint32_t now, n_quads, n_round, stride;
+    __device__ __forceinline__ TfeVsTableWalk(const TfeVictimParams &p_, uint32_t now_) : p(p_), now(now_)
     {
-        const uint32_t want = state->k_rem;
-        uint32_t c[2], incl[2];
+        n_quads = (p.C + 3u) >> 2;
+        n_round = (n_quads + 31u) & ~31u;              // whole warps stay together
+        stride = gridDim.x * blockDim.x;
+    }
+    // number of slot j of a quad whose bookkeeping is {a, b}
+    __device__ __forceinline__ unsigned long long number(const uint4 &a, const uint4 &b, uint32_t quad, int j) const
+    {
+        const uint2 st = j == 0 ? make_uint2(a.x, a.y) : j == 1 ? make_uint2(a.z, a.w) : j == 2 ? make_uint2(b.x, b.y) : make_uint2(b.z, b.w);
+        return ((unsigned long long)tfe_retention_key<DECAY>(st, now, p.div_half_life, p.age_cap) << 32) | (4u * quad + j);
+    }
+    // f(number, wanted) for the slots of a trip in which some lane of the warp holds a number <= limit (wanted: this
+    // one is) -- called by whole warps.  Most trips have none: one vote per sixteen slots, and the numbers are worked
+    // out a second time in the trips that have.
+    template <class F>
+    __device__ __forceinline__ void for_each_up_to(unsigned long long limit, F f) const
+    {
+        for (uint32_t g = blockIdx.x * blockDim.x + threadIdx.x; g < n_round; g += U * stride) {
+            uint4 a[U], b[U];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const uint32_t i = h * TFE_VICTIM_THREADS + threadIdx.x;
-            c[h] = i < gridDim.x ? __ldcg(tie_count + i) : 0u;
-            if (i < gridDim.x) tie_count[i] = 0;
+            for (int u = 0; u < U; ++u) {
+                const uint32_t gq = g + u * stride;
+                a[u] = b[u] = make_uint4(0, 0, 0, 0);
+                if (gq < n_quads) {
+                    a[u] = __ldcs(reinterpret_cast<const uint4 *>(p.slot_stats) + 2 * (size_t)gq);
+                    b[u] = __ldcs(reinterpret_cast<const uint4 *>(p.slot_stats) + 2 * (size_t)gq + 1);
+                }
+            }
+            bool any = false;
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const unsigned long long v = number(a[u], b[u], g + u * stride, j);
+                    any |= (uint32_t)v < p.C && v <= limit;
+                }
+            if (!__any_sync(0xFFFFFFFFu, any)) continue;
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const unsigned long long v = number(a[u], b[u], g + u * stride, j);
+                    f(v, (uint32_t)v < p.C && v <= limit);
+                }
         }
-        uint32_t carry = 0;                                   // total of the first half, for the second
+    }
+};
+
+// f(number, valid) for the first n entries of the candidate list, whole warps together.
+template <class F>
+__device__ __forceinline__ void tfe_vs_for_each_listed(const unsigned long long *list, uint32_t n, F f)
+{
+    const uint32_t n_round = (n + 31u) & ~31u;
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n_round; i += gridDim.x * blockDim.x) {
+        const bool in = i < n;
+        f(in ? __ldcg(list + i) : 0ull, in);
+    }
+}
+
+// 64 numbers of a warp, two per lane (v0: position `lane`, v1: position `lane + 32`), sorted ascending by position
+// with a bitonic network over shuffles.
+__device__ __forceinline__ void tfe_vs_warp_sort64(unsigned long long &v0, unsigned long long &v1, int lane)
+{
+#pragma unroll
+    for (int k = 2; k <= 64; k <<= 1) {
+#pragma unroll
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            if (j == 32) {                               // positions lane and lane + 32 (k = 64: ascending)
+                if (v0 > v1) { const unsigned long long t = v0; v0 = v1; v1 = t; }
+            } else {
+                const unsigned long long o0 = __shfl_xor_sync(0xFFFFFFFFu, v0, j), o1 = __shfl_xor_sync(0xFFFFFFFFu, v1, j);
+                const bool lower = (lane & j) == 0;
+                const bool up0 = (lane & k) == 0, up1 = ((lane + 32) & k) == 0;
+                v0 = (lower == up0) ? (o0 < v0 ? o0 : v0) : (o0 > v0 ? o0 : v0);
+                v1 = (lower == up1) ? (o1 < v1 ? o1 : v1) : (o1 > v1 ? o1 : v1);
+            }
+        }
+    }
+}
+
+// A number that r or more of the block's 2 * blockDim.x numbers do not exceed (two per thread, all distinct
+// except TFE_VS_NONE, of which there are fewer than 2 * blockDim.x - r + 1), and few more than r: every warp
+// sorts its 64 and leaves them in `lists`, the first warp then merges the 32 lists up to the r-th smallest.
+// s_out: one number.
+__device__ __forceinline__ unsigned long long tfe_vs_block_rth(unsigned long long v0, unsigned long long v1, uint32_t r,
+                                                                unsigned long long *lists, unsigned long long *s_out)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t n_lists = blockDim.x >> 5;
+    // a small r: the r-th smallest of the warps' minima stands in for it.  Those are r distinct numbers of the
+    // block, so it is never below the r-th smallest of all, which is all a threshold has to guarantee.
+    const bool minima_only = r <= n_lists && r <= 32u;
+    uint32_t list_len = 64;
+    if (minima_only) {
+        const unsigned long long m = v0 < v1 ? v0 : v1;
+        const uint32_t m_hi = __reduce_min_sync(0xFFFFFFFFu, (uint32_t)(m >> 32));
+        const uint32_t m_lo = __reduce_min_sync(0xFFFFFFFFu, (uint32_t)(m >> 32) == m_hi ? (uint32_t)m : 0xFFFFFFFFu);
+        if (lane == 0) lists[warp * 64] = ((unsigned long long)m_hi << 32) | m_lo;
+        list_len = 1;
+    } else {
+        tfe_vs_warp_sort64(v0, v1, lane);
+        lists[warp * 64 + lane] = v0;
+        lists[warp * 64 + lane + 32] = v1;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t head = 0;
+        unsigned long long cur = (uint32_t)lane < n_lists ? lists[lane * 64] : TFE_VS_NONE;
+        unsigned long long picked = TFE_VS_NONE;
+        for (uint32_t it = 0; it < r; ++it) {            // r times: the smallest head leaves its list
+            const uint32_t m_hi = __reduce_min_sync(0xFFFFFFFFu, (uint32_t)(cur >> 32));
+            const uint32_t m_lo = __reduce_min_sync(0xFFFFFFFFu, (uint32_t)(cur >> 32) == m_hi ? (uint32_t)cur : 0xFFFFFFFFu);
+            picked = ((unsigned long long)m_hi << 32) | m_lo;
+            if (cur == picked && picked != TFE_VS_NONE) {
+                ++head;
+                cur = head < list_len ? lists[lane * 64 + head] : TFE_VS_NONE;
+            }
+        }
+        if (lane == 0) *s_out = picked;
+    }
+    __syncthreads();
+    return *s_out;
+}
+
+template <bool DECAY>
+__global__ void __launch_bounds__(TFE_VS_THREADS, 1) tfe_victim_select_kernel(const TfeVictimParams p)
+{
+    extern __shared__ unsigned long long s_buf[];          // TFE_VS_FINAL_CAP numbers: samples, then collected candidates, then the final set
+    __shared__ uint32_t s_hist[TFE_VS_BINS];
+    __shared__ uint32_t s_warp[33];
+    __shared__ uint32_t s_count;
+    __shared__ uint32_t s_pick[4];
+    __shared__ uint32_t s_near[TFE_VS_NEAR_BINS];
+    __shared__ unsigned long long s_T;
+    static_assert(TFE_VS_SAMPLES == 2 * TFE_VS_THREADS, "two samples per thread");
+    static_assert(TFE_VS_BINS == 2 * TFE_VS_THREADS, "two pieces of the histogram per thread");
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    TfeVictimState *st = p.st;
+    uint32_t boundary = 0;
+    tfe_grid_dependency_sync();
+    const uint32_t now = *p.epoch;
+    const TfeVsTableWalk<DECAY> walk(p, now);
+
+    // ---- threshold from a sample, worked out by block 0 for all (148 blocks drawing the same 2,048 slots took
+    // 7.5 us, most of it queueing for the same lines of L2): sample i is drawn from the i-th of n_samples equal
+    // stretches of the table, so the samples are distinct slots
+    unsigned long long T = TFE_VS_NONE;
+    if (p.n_samples > 0u && blockIdx.x == 0) {
+        unsigned long long v[2];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            uint32_t v = c[h];
+            // sample number of this thread's h-th value: consecutive stretches of the table go to different warps
+            // (a table whose keys all tie is ordered by slot; its smallest samples must not share a warp)
+            const uint32_t i = (uint32_t)lane * 64u + 32u * h + (uint32_t)warp;
+            v[h] = TFE_VS_NONE;
+            if (i < p.n_samples) {
+                // stretch i: C / n_samples slots, one more in the first C % n_samples stretches
+                const uint32_t len = p.sample_stretch + (i < p.sample_longer ? 1u : 0u);
+                const uint32_t s0 = i * p.sample_stretch + min(i, p.sample_longer) +
+                                    (uint32_t)tfe_mulhi64(tfe_mix64((unsigned long long)i * 0x9E3779B97F4A7C15ull + 1ull), (unsigned long long)len);
+                v[h] = ((unsigned long long)tfe_retention_key<DECAY>(p.slot_stats[s0], now, p.div_half_life, p.age_cap) << 32) | s0;
+            }
+        }
+        T = tfe_vs_block_rth(v[0], v[1], p.sample_rank, s_buf, &s_T);
+        if (threadIdx.x == 0) {
+            st->threshold = T;
+            __threadfence();
+            *(volatile uint32_t *)&st->threshold_ready = 1u;
+        }
+    }
+    for (uint32_t i = threadIdx.x; i < TFE_VS_FINAL_CAP; i += blockDim.x) s_buf[i] = TFE_VS_NONE;
+    for (uint32_t i = threadIdx.x; i < TFE_VS_NEAR_BINS; i += blockDim.x) s_near[i] = 0;
+    if (threadIdx.x == 0) s_count = 0;
+    if (p.n_samples > 0u && blockIdx.x != 0) {             // bounded wait for block 0's threshold
+        if (threadIdx.x == 0) {
+            const volatile uint32_t *ready = &st->threshold_ready, *status = &st->status;
+            uint32_t spin = 0;
+            while (*ready == 0u && *status == 0u && ++spin <= TFE_SPIN_LIMIT) __nanosleep(40);
+            if (*ready == 0u) atomicOr(&st->status, TFE_VS_ERR_BARRIER);
+            __threadfence();
+            s_T = *(volatile unsigned long long *)&st->threshold;
+        }
+        __syncthreads();
+        T = s_T;
+        if (*(volatile uint32_t *)&st->status != 0u) return;
+    }
+    __syncthreads();
+
+    // ---- scan: candidates (<= T) to the list, smallest and largest number of all
+    {
+        TfeVsAppender app{s_buf, &s_count, TFE_VS_FINAL_CAP, &st->n_cand, p.list, p.list_cap};
+        walk.for_each_up_to(T, [&](unsigned long long v, bool cand) {
+            const uint32_t vote = __ballot_sync(0xFFFFFFFFu, cand);
+            if (vote == 0u) return;
+            tfe_vs_append(app, vote, cand, v);
+            if (cand) {                                   // how far below T, on a logarithmic scale
+                const uint32_t b = tfe_vs_near_bin(T - v);
+                int same;
+                __match_all_sync(vote, b, &same);
+                if (!same) atomicAdd(&s_near[b], 1u);
+                else if (lane == __ffs(vote) - 1) atomicAdd(&s_near[b], (uint32_t)__popc(vote));
+            }
+        });
+        tfe_vs_flush(app, s_warp);                       // synchronises the block
+        for (uint32_t i = threadIdx.x; i < TFE_VS_NEAR_BINS; i += blockDim.x)
+            if (s_near[i]) atomicAdd(&st->near[i], s_near[i]);
+    }
+    if (!tfe_vs_boundary(st, boundary)) return;
+
+    // ---- the range [lo, hi] that holds the take-th smallest, `cnt` numbers in it, `k` = its rank inside
+    const uint32_t n_cand = __ldcg(&st->n_cand);
+    const bool listed = n_cand >= p.take && n_cand <= p.list_cap;      // else: walk the table
+    unsigned long long lo = 0ull, hi = 0xFFFFFFFF00000000ull | (p.C - 1u);     // every number lies in [lo, hi]
+    uint32_t cnt = p.C, k = p.take;
+    if (n_cand >= p.take) {
+        // the candidates counted by their distance below T, on a logarithmic scale: the piece that holds the
+        // take-th smallest (a few numbers far below the rest do not stretch the range the refine steps divide)
+        // (with 128 steps per octave the piece mostly holds few enough numbers to go straight to the final step)
+        constexpr int PER = (TFE_VS_NEAR_BINS + TFE_VS_THREADS - 1) / TFE_VS_THREADS;      // consecutive bins per thread
+        uint32_t c[PER], mine = 0;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const uint32_t i = threadIdx.x * PER + j;
+            c[j] = i < TFE_VS_NEAR_BINS ? __ldcg(&st->near[i]) : 0u;
+            mine += c[j];
+        }
+        // numbers beyond this thread's bins (farther below T): a suffix sum over the block
+        uint32_t incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t u = __shfl_down_sync(0xFFFFFFFFu, incl, o);
+            if (lane + o < 32) incl += u;
+        }
+        if (threadIdx.x == 0) s_pick[0] = 0xFFFFFFFFu;
+        if (lane == 0) s_warp[warp] = incl;
+        __syncthreads();
+        uint32_t beyond = incl - mine;
+        for (int w = warp + 1; w < (int)(blockDim.x >> 5); ++w) beyond += s_warp[w];
+        if (beyond < p.take && beyond + mine >= p.take) {      // exactly one thread: the take-th smallest is in its bins
+            int j = PER - 1;
+            for (; j > 0 && beyond + c[j] < p.take; --j) beyond += c[j];
+            s_pick[0] = threadIdx.x * PER + j; s_pick[1] = beyond; s_pick[2] = c[j];
+        }
+        __syncthreads();
+        if (s_pick[0] == 0xFFFFFFFFu) {                  // the bins do not add up to n_cand
+            if (threadIdx.x == 0) atomicOr(&st->status, TFE_VS_ERR_INTERNAL);
+            return;
+        }
+        unsigned long long d_min, d_max;
+        tfe_vs_near_range(s_pick[0], d_min, d_max);
+        const unsigned long long piece_lo = T >= d_max ? T - d_max : 0ull, piece_hi = T - d_min;
+        lo = piece_lo > lo ? piece_lo : lo;
+        hi = piece_hi < hi ? piece_hi : hi;
+        k = p.take - s_pick[1];
+        cnt = s_pick[2];
+        __syncthreads();
+    }
+    // refine while the set to rank would be large (its cost grows with the square) and the range still splits
+    for (int it = 0; (p.take - k) + cnt > p.final_cap && cnt > p.range_cap && hi > lo; ++it) {
+        if (it >= TFE_VS_MAX_REFINE) {
+            if (threadIdx.x == 0) atomicOr(&st->status, TFE_VS_ERR_INTERNAL);
+            return;
+        }
+        const unsigned long long span = hi - lo;
+        const int sh = span < (unsigned long long)TFE_VS_BINS ? 0 : (64 - __clzll((long long)span)) - 11;
+        for (uint32_t i = threadIdx.x; i < TFE_VS_BINS; i += blockDim.x) s_hist[i] = 0;
+        __syncthreads();
+        auto count = [&](unsigned long long v, bool valid) {
+            if (valid && v >= lo && v <= hi) atomicAdd(&s_hist[(uint32_t)((v - lo) >> sh)], 1u);
+        };
+        if (listed) tfe_vs_for_each_listed(p.list, n_cand, count);
+        else walk.for_each_up_to(hi, count);
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < TFE_VS_BINS; i += blockDim.x)
+            if (s_hist[i]) atomicAdd(&st->hist[it][i], s_hist[i]);
+        if (!tfe_vs_boundary(st, boundary)) return;
+        // the piece that holds the k-th smallest of the range: every block works it out for itself
+        {
+            const uint32_t h0 = __ldcg(&st->hist[it][2 * threadIdx.x]), h1 = __ldcg(&st->hist[it][2 * threadIdx.x + 1]);
+            const uint32_t sum = h0 + h1;
+            uint32_t incl = sum;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, v, o);
-                if (lane >= o) v += u;
+                const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += u;
+            }
+            if (threadIdx.x == 0) s_pick[0] = 0xFFFFFFFFu;
+            if (lane == 31) s_warp[warp] = incl;
+            __syncthreads();
+            for (int w = 0; w < warp; ++w) incl += s_warp[w];
+            if (incl >= k && incl - sum < k) {           // exactly one thread
+                const uint32_t before = incl - sum;
+                const bool second = k - before > h0;
+                s_pick[0] = 2 * threadIdx.x + (second ? 1u : 0u);
+                s_pick[1] = before + (second ? h0 : 0u);
+                s_pick[2] = second ? h1 : h0;
             }
             __syncthreads();
-            if (lane == 31) s_warp[warp] = v;
+            if (s_pick[0] == 0xFFFFFFFFu) {              // the histogram holds fewer than k numbers
+                if (threadIdx.x == 0) atomicOr(&st->status, TFE_VS_ERR_INTERNAL);
+                return;
+            }
+            const unsigned long long piece_lo = lo + ((unsigned long long)s_pick[0] << sh);
+            const unsigned long long piece_hi = piece_lo + ((1ull << sh) - 1ull);
+            lo = piece_lo;
+            hi = piece_hi < hi ? piece_hi : hi;
+            k -= s_pick[1];
+            cnt = s_pick[2];
             __syncthreads();
-            uint32_t before = carry, total = 0;
-            for (int w = 0; w < TFE_VICTIM_THREADS / 32; ++w) {
-                if (w < warp) before += s_warp[w];
-                total += s_warp[w];
-            }
-            incl[h] = before + v;
-            carry += total;
-        }
-        if (threadIdx.x == 0) { s_block = 0; s_rank = 0; }      // overwritten below: k_rem <= number of ties
-        __syncthreads();
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-            if (incl[h] >= want && incl[h] - c[h] < want) {      // exactly one element
-                s_block = h * TFE_VICTIM_THREADS + threadIdx.x;
-                s_rank = want - (incl[h] - c[h]);
-            }
-    }
-    __syncthreads();
-    // ---- walk that range: a contiguous piece per thread, counts, scan, then the piece that holds the tie
-    const uint32_t q0 = min(n_quads, s_block * per_block), q1 = min(n_quads, q0 + per_block);
-    const uint32_t per_thread = (q1 - q0 + blockDim.x - 1) / blockDim.x;
-    const uint32_t t0 = min(q1, q0 + threadIdx.x * per_thread), t1 = min(q1, t0 + per_thread);
-    uint32_t mine = 0;
-    for (uint32_t g = t0; g < t1; ++g) mine += ties_of(g);
-    uint32_t incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    __syncthreads();
-    if (lane == 31) s_warp[warp] = incl;
-    __syncthreads();
-    uint32_t before = incl - mine;
-    for (int w = 0; w < warp; ++w) before += s_warp[w];
-    const uint32_t want = s_rank;
-    if (want > before && want <= before + mine) {          // exactly one thread
-        uint32_t left = want - before;
-        for (uint32_t g = t0; g < t1 && left; ++g) {
-            const uint4 k4 = __ldcg(reinterpret_cast<const uint4 *>(slot_key) + g);
-            const uint32_t key[4] = {k4.x, k4.y, k4.z, k4.w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (left && key[j] == key_star && 4 * g + j < C && --left == 0)
-                    state->prefix = (prefix & 0xFFFFFFFF00000000ull) | (4 * g + j);
         }
     }
-    if (threadIdx.x == 0) state->ticket = 0;
-}
 
-__global__ void __launch_bounds__(TFE_VICTIM_THREADS)
-tfe_victim_collect_kernel(const uint32_t *slot_key, uint32_t C, TfeVictimState *state, unsigned long long *list,
-                          uint32_t cap)
-{
-    tfe_grid_dependency_sync();
-    const unsigned long long limit = state->prefix;
-    const uint32_t n_quads = (C + 3u) >> 2;
-    for (uint32_t g = blockIdx.x * blockDim.x + threadIdx.x; g < n_quads; g += gridDim.x * blockDim.x) {
-        const uint4 k4 = reinterpret_cast<const uint4 *>(slot_key)[g];
-        const uint32_t key[4] = {k4.x, k4.y, k4.z, k4.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const uint32_t s0 = 4 * g + j;
-            const unsigned long long comp = ((unsigned long long)key[j] << 32) | s0;
-            if (s0 < C && comp <= limit) {
-                const uint32_t at = atomicAdd(&state->n_out, 1u);
-                if (at < cap) list[at] = comp;
-            }
-        }
-    }
-}
-
-// One block sorts the selected composites (at most TFE_VICTIMS_MAX = 4,096) ascending: a bitonic network
-// with four consecutive elements per thread.  Compare-exchange distances 1 and 2 stay inside a thread,
-// distances 4..64 are warp shuffles, only distances >= 128 go through shared memory (15 of the 78 steps at
-// 4,096 elements).
-__global__ void __launch_bounds__(1024)
-tfe_victim_sort_kernel(const unsigned long long *list, TfeVictimState *state, uint32_t n, int32_t *out_slots,
-                       uint32_t *out_keys)
-{
-    static_assert(TFE_VICTIMS_MAX == 4 * 1024, "four elements per thread of a 1,024-thread block");
-    __shared__ unsigned long long s_v[TFE_VICTIMS_MAX];
-    uint32_t pow2 = 1;
-    while (pow2 < n) pow2 <<= 1;
-    tfe_grid_dependency_sync();
-    const uint32_t base = 4u * threadIdx.x;
-    unsigned long long v[4];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) v[e] = base + e < n ? list[base + e] : ~0ull;      // padding sorts to the end
-    for (uint32_t k = 2; k <= pow2; k <<= 1) {
-        uint32_t j = k >> 1;
-        if (j >= 128) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) s_v[base + e] = v[e];
-            __syncthreads();
-            for (; j >= 128; j >>= 1) {
-                for (uint32_t t = threadIdx.x; t < TFE_VICTIMS_MAX / 2; t += blockDim.x) {
-                    const uint32_t i = ((t & ~(j - 1)) << 1) | (t & (j - 1));      // the pair's lower index
-                    const uint32_t l = i | j;
-                    const unsigned long long a = s_v[i], b = s_v[l];
-                    const bool up = (i & k) == 0;
-                    if ((a > b) == up) { s_v[i] = b; s_v[l] = a; }
-                }
-                __syncthreads();
-            }
-#pragma unroll
-            for (int e = 0; e < 4; ++e) v[e] = s_v[base + e];
-        }
-        for (; j >= 4; j >>= 1) {                   // partner element in another lane of this warp
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, v[e], (int)(j >> 2));
-                const uint32_t i = base + e;
-                const bool up = (i & k) == 0, lower = (i & j) == 0;
-                v[e] = (lower == up) ? (other < v[e] ? other : v[e]) : (other > v[e] ? other : v[e]);
-            }
-        }
-        // partner element in this thread: distance 2 (from k = 4 on), then distance 1
-        auto exchange = [&](unsigned long long &a, unsigned long long &b, uint32_t i) {
-            const bool up = (i & k) == 0;
-            if ((a > b) == up) { const unsigned long long t = a; a = b; b = t; }
+    // ---- final: gather everything <= hi, rank it
+    {
+        TfeVsAppender app{s_buf, &s_count, TFE_VS_FINAL_CAP, &st->n_final, p.fin, (uint32_t)TFE_VS_FINAL_CAP};
+        auto gather = [&](unsigned long long v, bool valid) {
+            const bool have = valid && v <= hi;
+            const uint32_t vote = __ballot_sync(0xFFFFFFFFu, have);
+            if (vote) tfe_vs_append(app, vote, have, v);
         };
-        if (k >= 4) { exchange(v[0], v[2], base); exchange(v[1], v[3], base + 1); }
-        exchange(v[0], v[1], base);
-        exchange(v[2], v[3], base + 2);
+        if (listed) tfe_vs_for_each_listed(p.list, n_cand, gather);
+        else walk.for_each_up_to(hi, gather);
+        tfe_vs_flush(app, s_warp);
     }
-#pragma unroll
-    for (int e = 0; e < 4; ++e)
-        if (base + e < n) {
-            out_slots[base + e] = (int32_t)(uint32_t)v[e];
-            out_keys[base + e] = (uint32_t)(v[e] >> 32);
+    if (!tfe_vs_boundary(st, boundary)) return;
+    const uint32_t n_final = __ldcg(&st->n_final);
+    if (n_final != (p.take - k) + cnt || n_final > (uint32_t)TFE_VS_FINAL_CAP) {
+        if (threadIdx.x == 0) atomicOr(&st->status, TFE_VS_ERR_INTERNAL);
+        return;
+    }
+    for (uint32_t i = threadIdx.x; i < n_final; i += blockDim.x) s_buf[i] = __ldcg(p.fin + i);
+    __syncthreads();
+    // one number per warp and trip, dealt to the blocks first so that a small set still uses every SM
+    for (uint32_t e = warp * gridDim.x + blockIdx.x; e < n_final; e += gridDim.x * (blockDim.x >> 5)) {
+        const unsigned long long x = s_buf[e];
+        uint32_t below = 0;
+#pragma unroll 8
+        for (uint32_t i = lane; i < n_final; i += 32) below += s_buf[i] < x;
+        below = __reduce_add_sync(0xFFFFFFFFu, below);
+        if (lane == 0 && below < p.take) {
+            p.out_slots[below] = (int32_t)(uint32_t)x;
+            p.out_keys[below] = (uint32_t)(x >> 32);
         }
-    if (threadIdx.x == 0) state->n_out = 0;      // re-armed for the next selection
+    }
 }
 
 

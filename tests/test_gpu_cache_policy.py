@@ -69,6 +69,34 @@ def test_bookkeeping_and_victims_follow_the_oracle(H, policy):
     pr.close()
 
 
+# (list_cap, final_cap, n_samples): every path of the selection on one history -- the whole table in the list;
+# a sampled threshold with and without refine steps; a list that overflows (the table is walked again); a
+# threshold from a single sample (mostly too low: the table is walked again); the defaults
+_TUNINGS = [(0, 0, 0), (16384, 4500, 0), (1024, 0, 256), (1024, 4200, 64), (64, 0, 2048), (8192, 4500, 1), (300, 4100, 7),
+            (2000, 1, 2048)]
+
+
+@pytest.mark.parametrize("ties", [False, True])
+def test_selection_result_is_independent_of_its_internal_sizes(H, ties):
+    from paper_2607_07388_b200 import binding as tfe
+    w = synth.config(1, B=6, T=300, n_phrases=40_000, gpu_slots=13_001, residency="hot_host", p=0.7,
+                     reserve_free=0 if ties else 700)
+    tb, pr = H.pair_from_workload(w)
+    pr.eng.cache_policy_enable()
+    h = synth.make_hidden_np(w)
+    for step in range(0 if ties else 6):       # ties: nothing looked up, every key equal, the slot decides
+        tok = synth.make_queries(w, tb, variant=step % 3)
+        g, ref, _ = pr.run_and_compare(tok, h, lam=1.0)
+        pr.ora.touch(ref)
+    with pytest.raises(tfe.TfeError):
+        tfe.tfe_cache_select_tuning(pr.eng.ctx, 1_048_577, 0, 0)
+    for list_cap, final_cap, n_samples in _TUNINGS:
+        tfe.tfe_cache_select_tuning(pr.eng.ctx, list_cap, final_cap, n_samples)
+        for n, hl in ((1, 0), (33, 1), (700, 2), (701, 0), (4096, 3), (4095, 0)):
+            _compare_victims(pr, n, hl)
+    pr.close()
+
+
 def test_policy_off_and_argument_checks(H):
     from paper_2607_07388_b200 import binding as tfe
     w = synth.config(1)
@@ -118,6 +146,7 @@ def test_victims_more_than_slots_and_host_pipeline_epoch(H):
 def test_policy_random_histories(H, seed):
     """Seeded random interleavings of lookups (either policy), victim selections (any n, any half-life)
     and installs into the selected victims: bookkeeping and ranking follow the oracle at every step."""
+    from paper_2607_07388_b200 import binding as tfe
     rng = np.random.default_rng([808, seed])
     n_phrases = int(rng.integers(200, 20_000))
     gpu_slots = max(8, int(n_phrases * rng.uniform(0.1, 0.9)))
@@ -135,6 +164,9 @@ def test_policy_random_histories(H, seed):
         _compare_state(pr)
         n = int(rng.choice([1, 5, 64, 1000, 4096]))
         hl = int(rng.choice([0, 1, 2, 5]))
+        # the sizes of the selection's internal steps never change its result
+        tfe.tfe_cache_select_tuning(pr.eng.ctx, int(rng.choice([0, 16, 200, 3000])), int(rng.choice([0, 2, 700, 4500])),
+                                    int(rng.choice([0, 1, 9, 300, 2048])))
         slots = _compare_victims(pr, n, hl)
         if rng.random() < 0.7:
             want = np.unique(pr.ora.lookup(tok, policy=policy).miss_phrase).astype(np.uint32)
