@@ -294,7 +294,7 @@ tfe_status tfe_cache_policy_enable(tfe_ctx *ctx, void *stream);
  *   n        0..4096;  half_life at most 2^26 - 1;  slots HOST int32 [n], or NULL;  keys HOST uint32 [n] or NULL;
  *   count    HOST: entries written = min(n, gpu_slots).
  * One cooperative kernel launch on `stream` (one block per SM; its blocks wait for one another at
- * four or more step boundaries, every wait bounded) after a 64 KiB clear of its work space.  The
+ * two or more step boundaries, every wait bounded).  The
  * per-slot bookkeeping is read once; a threshold taken from a sample of the slots keeps the work
  * after that pass to a candidate list, and the result does not depend on the sample: a threshold
  * that turns out too low or too high only makes the call walk the table again.  With host `slots`
@@ -302,8 +302,10 @@ tfe_status tfe_cache_policy_enable(tfe_ctx *ctx, void *stream);
  * takes host arrays); with slots = NULL nothing is copied and nothing synchronises.
  * tfe_cache_select_victims_device returns the DEVICE copies of the most recent selection (owned
  * by the context, valid until the next one; they feed tfe_cache_install_device).
- * Errors: INVALID_ARG (also: policy not enabled), CUDA, INTERNAL (host `slots` only: a wait inside
- * the kernel ran out or its counts contradicted one another; the outputs are not valid).
+ * One selection at a time per context (the work space is the context's).
+ * Errors: INVALID_ARG (also: policy not enabled, half_life too large), CUDA, INTERNAL (a wait inside the
+ * kernel ran out or its counts contradicted one another; the outputs are not valid.  Reported by the
+ * form with host `slots`, which also clears the condition; until then later selections do nothing).
  */
 tfe_status tfe_cache_select_victims(tfe_ctx *ctx, int32_t n, int32_t half_life, int32_t *slots,
                                     uint32_t *keys, int32_t *count, void *stream);

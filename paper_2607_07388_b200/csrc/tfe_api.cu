@@ -1090,6 +1090,7 @@ tfe_status tfe_cache_policy_enable(tfe_ctx *c, void *stream_)
                                                                                                     (uint32_t)C);
     CU(cudaGetLastError());
     CU(cudaMemsetAsync(c->d_epoch, 0, sizeof(uint32_t), stream));
+    CU(cudaMemsetAsync(c->d_vs_state, 0, sizeof(TfeVictimState), stream));
     return TFE_OK;
 }
 
@@ -1127,7 +1128,6 @@ tfe_status tfe_cache_select_victims(tfe_ctx *c, int32_t n, int32_t half_life, in
     }
     p.list = c->d_vs_list; p.fin = c->d_vs_fin; p.st = c->d_vs_state;
     p.out_slots = c->d_vs_slots; p.out_keys = c->d_vs_keys;
-    CU(cudaMemsetAsync(c->d_vs_state, 0, sizeof(TfeVictimState), stream));
     {
         const int64_t n_quads = (C + 3) / 4;
         cudaLaunchConfig_t cfg{};
@@ -1148,7 +1148,12 @@ tfe_status tfe_cache_select_victims(tfe_ctx *c, int32_t n, int32_t half_life, in
     uint32_t dev_status = 0;
     CU(cudaMemcpyAsync(&dev_status, &c->d_vs_state->status, sizeof(uint32_t), cudaMemcpyDeviceToHost, stream));
     CU(cudaStreamSynchronize(stream));
-    return dev_status ? TFE_ERR_INTERNAL : TFE_OK;
+    if (dev_status) {                       // the launch gave up and left its work space as it was
+        CU(cudaMemsetAsync(c->d_vs_state, 0, sizeof(TfeVictimState), stream));
+        CU(cudaStreamSynchronize(stream));
+        return TFE_ERR_INTERNAL;
+    }
+    return TFE_OK;
 }
 
 tfe_status tfe_cache_select_tuning(tfe_ctx *c, int32_t list_cap, int32_t final_cap, int32_t n_samples)

@@ -1308,13 +1308,15 @@ tfe_prefetch_select_kernel(const unsigned long long *keys, const uint32_t *entry
 #define TFE_VS_ERR_BARRIER 1u            // a wait at a step boundary ran out
 #define TFE_VS_ERR_INTERNAL 2u           // counts that contradict one another
 
+// All zero before a launch.  A launch that completes leaves it so (its blocks clear what they used once nobody
+// reads it any more); one that gave up leaves `status` set and the rest as it was: the host clears it.
 struct TfeVictimState {
     uint32_t arrived;               // blocks through the step boundaries so far
     uint32_t n_cand;                // numbers <= T seen by the scan (entries beyond the list's capacity are dropped)
     uint32_t n_final;               // numbers gathered for the final step
     uint32_t status;                // TFE_VS_ERR_*
     uint32_t threshold_ready;       // block 0 has published `threshold`
-    uint32_t pad;
+    uint32_t left;                  // blocks that have finished; the last one clears the counters for the next launch
     unsigned long long threshold;
     uint32_t near[TFE_VS_NEAR_BINS];   // candidates by tfe_vs_near_bin(T - number)
     uint32_t hist[TFE_VS_MAX_REFINE][TFE_VS_BINS];
@@ -1613,6 +1615,7 @@ __global__ void __launch_bounds__(TFE_VS_THREADS, 1) tfe_victim_select_kernel(co
     TfeVictimState *st = p.st;
     uint32_t boundary = 0;
     tfe_grid_dependency_sync();
+    if (*(volatile uint32_t *)&st->status != 0u) return;     // an earlier launch gave up: nothing runs until the host has cleared the state
     const uint32_t now = *p.epoch;
     const TfeVsTableWalk<DECAY> walk(p, now);
 
@@ -1731,11 +1734,13 @@ __global__ void __launch_bounds__(TFE_VS_THREADS, 1) tfe_victim_select_kernel(co
         __syncthreads();
     }
     // refine while the set to rank would be large (its cost grows with the square) and the range still splits
+    int n_refined = 0;
     for (int it = 0; (p.take - k) + cnt > p.final_cap && cnt > p.range_cap && hi > lo; ++it) {
         if (it >= TFE_VS_MAX_REFINE) {
             if (threadIdx.x == 0) atomicOr(&st->status, TFE_VS_ERR_INTERNAL);
             return;
         }
+        n_refined = it + 1;
         const unsigned long long span = hi - lo;
         const int sh = span < (unsigned long long)TFE_VS_BINS ? 0 : (64 - __clzll((long long)span)) - 11;
         for (uint32_t i = threadIdx.x; i < TFE_VS_BINS; i += blockDim.x) s_hist[i] = 0;
@@ -1815,6 +1820,18 @@ __global__ void __launch_bounds__(TFE_VS_THREADS, 1) tfe_victim_select_kernel(co
         if (lane == 0 && below < p.take) {
             p.out_slots[below] = (int32_t)(uint32_t)x;
             p.out_keys[below] = (uint32_t)(x >> 32);
+        }
+    }
+    // ---- ready for the next launch: every block is past its last read of the counts by distance and of the
+    // histograms (they were read before the boundary above); the counters go when the last block leaves
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < TFE_VS_NEAR_BINS; i += gridDim.x * blockDim.x) st->near[i] = 0u;
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < (uint32_t)n_refined * TFE_VS_BINS; i += gridDim.x * blockDim.x)
+        (&st->hist[0][0])[i] = 0u;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(&st->left, 1u) == gridDim.x - 1u) {
+            st->arrived = 0u; st->n_cand = 0u; st->n_final = 0u; st->threshold_ready = 0u; st->left = 0u;
         }
     }
 }
