@@ -10,6 +10,7 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -62,6 +63,7 @@ struct tfe_ctx {
     uint64_t n_buckets = 0;
     int row_vecs = 0;                       // 16-byte vectors per GPU-tier row
 
+    void *d_arena = nullptr;                // device build: index, positions, owners, counters (and tuples) are one allocation
     ulonglong2 *d_index = nullptr;
     int4 *d_phrase_tokens = nullptr;        // only when an order is hashed
     uint32_t *d_phrase_pos = nullptr;
@@ -223,6 +225,31 @@ TfeFastDiv make_fastdiv(uint32_t d)
 
 void free_dev(void *p) { if (p) (void)cudaFree(p); }
 
+// Resident blocks per SM of every lookup variant, asked of the runtime once per device and process.
+cudaError_t lookup_occupancy(int device, int (&occ)[kVarSlots])
+{
+    constexpr int kMaxDevices = 64;
+    static int cache[kMaxDevices][kVarSlots];
+    static bool have[kMaxDevices];
+    static std::mutex guard;
+    std::lock_guard<std::mutex> lock(guard);
+    const bool cached = device >= 0 && device < kMaxDevices;
+    if (!cached || !have[device]) {
+        int fresh[kVarSlots] = {};
+        for (int v = 0; v < kVarCount; ++v) {
+            int o = 0;
+            const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, pick_kernel(v), TFE_BLOCK_THREADS, 0);
+            if (e != cudaSuccess) return e;
+            fresh[v] = std::max(1, o);
+        }
+        if (!cached) { for (int v = 0; v < kVarSlots; ++v) occ[v] = fresh[v]; return cudaSuccess; }
+        for (int v = 0; v < kVarSlots; ++v) cache[device][v] = fresh[v];
+        have[device] = true;
+    }
+    for (int v = 0; v < kVarSlots; ++v) occ[v] = cache[device][v];
+    return cudaSuccess;
+}
+
 tfe_status validate_config(const tfe_config *c)
 {
     if (!c) return TFE_ERR_INVALID_ARG;
@@ -361,10 +388,14 @@ void tfe_destroy(tfe_ctx *c)
     (void)cudaGetDevice(&prev);
     (void)cudaSetDevice(c->device);
     (void)cudaDeviceSynchronize();
-    free_dev(c->d_index); free_dev(c->d_phrase_tokens); free_dev(c->d_phrase_pos);
-    free_dev(c->d_slot_owner); free_dev(c->d_scr_rec);
+    if (c->d_arena) {
+        free_dev(c->d_arena);
+    } else {
+        free_dev(c->d_index); free_dev(c->d_phrase_tokens); free_dev(c->d_phrase_pos);
+        free_dev(c->d_slot_owner); free_dev(c->d_counters);
+    }
+    free_dev(c->d_scr_rec);
     free_dev(c->d_miss_q); free_dev(c->d_miss_phrase); free_dev(c->d_miss_tier);
-    free_dev(c->d_counters);
     free_dev(c->d_inst_ids); free_dev(c->d_inst_slots); free_dev(c->d_inst_rows);
     free_dev(c->d_h_tokens); free_dev(c->d_h_hidden); free_dev(c->d_h_out);
     free_dev(c->d_h_phrase); free_dev(c->d_h_slot); free_dev(c->d_h_flag);
@@ -488,11 +519,7 @@ tfe_status tfe_index_build(const tfe_config *cfg, const int32_t *phrase_tokens,
         CUF(cudaMemcpyAsync(c->d_phrase_tokens, phrase_tokens, (size_t)N * sizeof(int4),
                             cudaMemcpyHostToDevice, stream));
     }
-    for (int v = 0; v < kVarCount; ++v) {
-        int occ = 0;
-        CUF(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, pick_kernel(v), TFE_BLOCK_THREADS, 0));
-        c->occ[v] = std::max(1, occ);
-    }
+    CUF(lookup_occupancy(c->device, c->occ));
     CUF(cudaStreamSynchronize(stream));
     if (rc != TFE_OK) return fail(rc);
     CUF(cudaMemsetAsync(c->d_counters, 0, TFE_CTR_WORDS * sizeof(uint32_t), stream));
@@ -538,7 +565,6 @@ tfe_status tfe_index_build_device(const tfe_config *cfg, const int32_t *phrase_t
     c->gpu_rows = static_cast<uint4 *>(gpu_rows);
     uint32_t *d_status = nullptr;
     auto fail = [&](tfe_status s) {
-        if (d_status) (void)cudaFree(d_status);
         tfe_destroy(c);
         return s;
     };
@@ -550,19 +576,27 @@ tfe_status tfe_index_build_device(const tfe_config *cfg, const int32_t *phrase_t
     CUF(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device));
     const size_t n_slots = (size_t)n_buckets * TFE_SLOTS_PER_BUCKET;
     const size_t owner_entries = std::max<size_t>(4, (size_t)(C + 3) / 4 * 4);
-    CUF(cudaMalloc(&c->d_index, n_slots * sizeof(ulonglong2)));
-    CUF(cudaMalloc(&c->d_phrase_pos, std::max<size_t>(4, (size_t)N * 4)));
-    CUF(cudaMalloc(&c->d_slot_owner, owner_entries * 4));
-    CUF(cudaMalloc(&c->d_counters, TFE_CTR_WORDS * sizeof(uint32_t)));
-    CUF(cudaMalloc(&d_status, sizeof(uint32_t)));
+    {
+        // one allocation for everything the build fills (several cost most of a millisecond each at these sizes)
+        auto round = [](size_t b) { return (b + 255) & ~(size_t)255; };
+        const size_t b_index = round(n_slots * sizeof(ulonglong2)), b_pos = round(std::max<size_t>(4, (size_t)N * 4));
+        const size_t b_owner = round(owner_entries * 4), b_ctr = round((TFE_CTR_WORDS + 1) * sizeof(uint32_t));
+        const size_t b_tok = c->any_hashed && N > 0 ? round((size_t)N * sizeof(int4)) : 0;
+        CUF(cudaMalloc(&c->d_arena, b_index + b_pos + b_owner + b_ctr + b_tok));
+        char *at = static_cast<char *>(c->d_arena);
+        c->d_index = reinterpret_cast<ulonglong2 *>(at); at += b_index;
+        c->d_phrase_pos = reinterpret_cast<uint32_t *>(at); at += b_pos;
+        c->d_slot_owner = reinterpret_cast<uint32_t *>(at); at += b_owner;
+        c->d_counters = reinterpret_cast<uint32_t *>(at);
+        d_status = c->d_counters + TFE_CTR_WORDS; at += b_ctr;
+        if (b_tok) c->d_phrase_tokens = reinterpret_cast<int4 *>(at);
+    }
     CUF(cudaMemsetAsync(c->d_index, 0, n_slots * sizeof(ulonglong2), stream));
     CUF(cudaMemsetAsync(c->d_slot_owner, 0xFF, owner_entries * 4, stream));
     CUF(cudaMemsetAsync(c->d_counters, 0, TFE_CTR_WORDS * sizeof(uint32_t), stream));
     CUF(cudaMemsetAsync(d_status, 0, sizeof(uint32_t), stream));
-    if (c->any_hashed && N > 0) {
-        CUF(cudaMalloc(&c->d_phrase_tokens, (size_t)N * sizeof(int4)));
+    if (c->d_phrase_tokens)
         CUF(cudaMemcpyAsync(c->d_phrase_tokens, phrase_tokens, (size_t)N * sizeof(int4), cudaMemcpyDeviceToDevice, stream));
-    }
     TfeBuildParams b{};
     b.phrase_tokens = reinterpret_cast<const int4 *>(phrase_tokens);
     b.phrase_len = phrase_len; b.init_slot = init_slot;
@@ -580,11 +614,7 @@ tfe_status tfe_index_build_device(const tfe_config *cfg, const int32_t *phrase_t
         CUF(cudaMemcpyAsync(&status, d_status, sizeof status, cudaMemcpyDeviceToHost, stream));
     }
     c->mirror_ready = false;        // the host mirror of the residency state is fetched when tfe_cache_install first needs it
-    for (int v = 0; v < kVarCount; ++v) {
-        int occ = 0;
-        CUF(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, pick_kernel(v), TFE_BLOCK_THREADS, 0));
-        c->occ[v] = std::max(1, occ);
-    }
+    CUF(lookup_occupancy(c->device, c->occ));
     CUF(cudaStreamSynchronize(stream));
     if (status & TFE_BUILD_BAD_PHRASE) return fail(TFE_ERR_INVALID_ARG);
     if (status & TFE_BUILD_BAD_SLOT) return fail(TFE_ERR_SLOT_RANGE);
@@ -593,7 +623,6 @@ tfe_status tfe_index_build_device(const tfe_config *cfg, const int32_t *phrase_t
     if (status & TFE_BUILD_KICKS) return fail(TFE_ERR_PROBE_LIMIT);
     if (status & TFE_BUILD_LOST) return fail(TFE_ERR_INTERNAL);
 #undef CUF
-    (void)cudaFree(d_status);
     *out = c;
     return TFE_OK;
 }

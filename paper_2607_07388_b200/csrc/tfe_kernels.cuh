@@ -500,14 +500,14 @@ __device__ __forceinline__ int32_t tfe_select_longest_group(const TfeLookupParam
 // of probing before any byte streamed).  Autonomous warps wait only for their own 32 lanes while
 // the other warps of the SM keep the memory pipes busy.
 #ifndef TFE_MIN_BLOCKS_GENERAL
-#define TFE_MIN_BLOCKS_GENERAL 2     // blocks per SM the COSINE variants are compiled for (the others: TFE_MIN_BLOCKS)
+#define TFE_MIN_BLOCKS_GENERAL 2     // blocks per SM the COSINE and the ALL variants are compiled for (the others: TFE_MIN_BLOCKS)
 #endif
 #ifndef TFE_MIN_BLOCKS
 #define TFE_MIN_BLOCKS 3
 #endif
 
 template <int HT, bool ALL, bool COS, bool PACKED>
-__global__ void __launch_bounds__(TFE_BLOCK_THREADS, COS ? TFE_MIN_BLOCKS_GENERAL : TFE_MIN_BLOCKS)
+__global__ void __launch_bounds__(TFE_BLOCK_THREADS, (COS || ALL) ? TFE_MIN_BLOCKS_GENERAL : TFE_MIN_BLOCKS)
 tfe_lookup_inject_kernel(const TfeLookupParams p)
 {
     constexpr int VN = TfeVec<HT>::N;
@@ -653,6 +653,69 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
 #pragma unroll
                         for (int e = 0; e < VN; ++e) y[e] = fmaf(gate, m[e], x[e]);
                         store_hidden<HT>(orow, k, y);
+                    }
+                    continue;
+                }
+            }
+            if constexpr (ALL) {
+                // every row of the query in flight together, the weighted sum m kept in registers: the rows are
+                // read once (the gated form needs the whole of m before its update, so it takes this path only
+                // when one trip covers the row)
+                constexpr int UA = UNROLL;
+                if (!COS || steps <= 32 * UA) {
+                    for (int s0 = 0; s0 < steps; s0 += 32 * UA) {
+                        uint4 hv[UA];
+                        float m[UA][VN];
+#pragma unroll
+                        for (int u = 0; u < UA; ++u) {
+                            const int k = s0 + u * 32 + lane;
+                            if (k < steps) hv[u] = ld_stream(reinterpret_cast<const uint4 *>(hrow) + k);
+#pragma unroll
+                            for (int e = 0; e < VN; ++e) m[u][e] = 0.f;
+                        }
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            if (rowp[g] == nullptr) continue;
+                            typename TfeVec<HT>::RowRaw rv[UA];
+#pragma unroll
+                            for (int u = 0; u < UA; ++u) {
+                                const int k = s0 + u * 32 + lane;
+                                if (k < steps) rv[u] = ld_row_raw<HT>(rowp[g], k);
+                            }
+#pragma unroll
+                            for (int u = 0; u < UA; ++u) {
+                                if (s0 + u * 32 + lane >= steps) continue;
+                                float r[VN];
+                                unpack_row<HT>(rv[u], r);
+#pragma unroll
+                                for (int e = 0; e < VN; ++e) m[u][e] = fmaf(alpha[g], r[e], m[u][e]);
+                            }
+                        }
+                        if constexpr (COS) {
+                            float sa = 0.f, sb = 0.f, sc = 0.f;      // <h,m>, <h,h>, <m,m>, same order of terms as below
+#pragma unroll
+                            for (int u = 0; u < UA; ++u) {
+                                if (s0 + u * 32 + lane >= steps) continue;
+                                float x[VN];
+                                unpack_hidden<HT>(hv[u], x);
+#pragma unroll
+                                for (int e = 0; e < VN; ++e) {
+                                    sa = fmaf(x[e], m[u][e], sa); sb = fmaf(x[e], x[e], sb); sc = fmaf(m[u][e], m[u][e], sc);
+                                }
+                            }
+                            sa = warp_sum(sa); sb = warp_sum(sb); sc = warp_sum(sc);
+                            gate = p.lambda / (1.f + __expf(-sa * rsqrtf(fmaf(sb, sc, 1e-12f))));
+                        }
+#pragma unroll
+                        for (int u = 0; u < UA; ++u) {
+                            const int k = s0 + u * 32 + lane;
+                            if (k >= steps) continue;
+                            float x[VN], y[VN];
+                            unpack_hidden<HT>(hv[u], x);
+#pragma unroll
+                            for (int e = 0; e < VN; ++e) y[e] = fmaf(gate, m[u][e], x[e]);
+                            store_hidden<HT>(orow, k, y);
+                        }
                     }
                     continue;
                 }
