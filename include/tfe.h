@@ -398,10 +398,13 @@ tfe_status tfe_set_tuning(tfe_ctx *ctx, int32_t batch_queries);
  * probabilities, which are the inputs of tfe_prefetch_candidates.  The only dense contraction of
  * the method; it runs on the tensor cores.  A head is independent of any phrase index.
  *
- * tfe_head_create -- w_pref DEVICE bf16 [V][d] row-major, 16-byte aligned, CALLER-OWNED and read
- * in place by every call (it must outlive the head); d a multiple of 64; max_batch 1..256.
- * Allocates the logits buffer (max_batch * V * 4 bytes) and small work areas on the current
- * device.  Errors: INVALID_ARG, CUDA.
+ * tfe_head_create -- w_pref DEVICE bf16 [V][d] row-major, 16-byte aligned, CALLER-OWNED; it is
+ * copied into the head in the order the GEMM reads it (pieces of 128 rows x 64 columns, 16
+ * contiguous KB each) and may be released when the call returns (the call waits for the device);
+ * d a multiple of 64; max_batch 1..256.  Allocates that copy (V * d * 2 bytes, rounded up to
+ * whole 128-row tiles per CTA: 349 MB for V = 151,936, d = 1,024), the logits buffer
+ * (max_batch * V * 4 bytes) and small work areas on the current device.
+ * Errors: INVALID_ARG, CUDA.
  */
 typedef struct tfe_head tfe_head;
 tfe_status tfe_head_create(const void *w_pref, int32_t V, int32_t d, int32_t max_batch, tfe_head **out);

@@ -251,9 +251,8 @@ tfe_head_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             for (int32_t t = 0; t < n_tiles && ok; ++t) {
-                const int32_t row0 = (int32_t)r0 + t * HEAD_TILE_M;
                 const int32_t valid = min(HEAD_TILE_M, n_rows - t * HEAD_TILE_M);
-                // a short last tile is fetched with the short box, so no row of the next CTA is read
+                // a short last tile is fetched with the short box: only its rows are read
                 const bool use_tail = valid < HEAD_TILE_M && valid == p.tail_rows;
                 const uint32_t w_bytes = use_tail ? (uint32_t)p.tail_rows * 128u : HEAD_TILE_M * 128u;
                 for (int32_t kb = 0; kb < num_kb; ++kb) {
@@ -266,7 +265,9 @@ tfe_head_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
                     const uint32_t bar = smem_u32(&s_full[stage]);
                     const uint32_t dst = smem_base + stage * stage_bytes;
                     mbar_expect_tx(bar, w_bytes + (uint32_t)p.N * 128u);
-                    tma_load_2d(dst, use_tail ? &map_w_tail : &map_w, bar, kb * HEAD_TILE_K, row0, hint_stream);
+                    // W_pref was re-laid at creation: the 128 x 64 piece of (CTA, tile, k-slice) is 16 contiguous KB
+                    const int32_t piece = ((int32_t)blockIdx.x * p.tiles_per_cta + t) * num_kb + kb;
+                    tma_load_2d(dst, use_tail ? &map_w_tail : &map_w, bar, 0, piece * HEAD_TILE_M, hint_stream);
                     tma_load_2d(dst + HEAD_TILE_M * 128u, &map_h, bar, kb * HEAD_TILE_K, 0, hint_keep);
                     if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
                 }
@@ -664,6 +665,29 @@ encode_tiled_fn get_encode_tiled()
     return fn;
 }
 
+// W_pref [V][d] row-major -> pieces of 128 rows x 64 columns (16 KB each, rows 128 bytes apart), in the order the
+// GEMM's CTAs read them: piece ((cta * tiles_per_cta + tile) * d / 64 + k-slice).  A tile's k-slice is then one
+// contiguous 16 KB read instead of 128 reads of 128 bytes 2 * d bytes apart.  Rows a tile does not have are zero.
+__global__ void __launch_bounds__(256)
+tfe_head_retile_kernel(const uint4 *__restrict__ w, uint4 *__restrict__ tiled, int32_t V, int32_t d, int32_t rows_per_cta,
+                       int32_t tiles_per_cta, int64_t n_pieces)
+{
+    const int32_t num_kb = d / HEAD_TILE_K;
+    const int64_t n_vec = n_pieces * HEAD_TILE_M * 8;               // 16-byte vectors: 8 per 128-byte row of a piece
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t vec = (int32_t)(i & 7), r = (int32_t)((i >> 3) & (HEAD_TILE_M - 1));
+        const int64_t piece = i >> 10;
+        const int32_t kb = (int32_t)(piece % num_kb);
+        const int64_t tile = piece / num_kb;
+        const int32_t t = (int32_t)(tile % tiles_per_cta);
+        const int64_t cta = tile / tiles_per_cta;
+        const int64_t in_cta = (int64_t)t * HEAD_TILE_M + r, row = cta * rows_per_cta + in_cta;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (in_cta < rows_per_cta && row < V) v = w[row * (d / 8) + kb * 8 + vec];
+        tiled[i] = v;
+    }
+}
+
 // bf16 matrix [rows][cols] row-major, box = 64 columns x box_rows rows, 128-byte swizzle
 bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows)
 {
@@ -681,7 +705,7 @@ bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, 
 }  // namespace
 
 struct tfe_head {
-    const void *w = nullptr;
+    void *d_w_tiled = nullptr;              // W_pref in the GEMM's reading order (tfe_head_retile_kernel)
     int32_t V = 0, d = 0, max_batch = 0;
     int device = 0, sm_count = 0;
     int32_t rows_per_cta = 0, tail_rows = 0, grid = 0;
@@ -705,7 +729,7 @@ tfe_status tfe_head_create(const void *w_pref, int32_t V, int32_t d, int32_t max
     if ((reinterpret_cast<uintptr_t>(w_pref) & 15u) != 0) return TFE_ERR_INVALID_ARG;
     tfe_head *h = new tfe_head();
     auto fail = [&](tfe_status st) { tfe_head_destroy(h); return st; };
-    h->w = w_pref; h->V = V; h->d = d; h->max_batch = max_batch;
+    h->V = V; h->d = d; h->max_batch = max_batch;
     if (cudaGetDevice(&h->device) != cudaSuccess) return fail(TFE_ERR_CUDA);
     if (cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess)
         return fail(TFE_ERR_CUDA);
@@ -715,11 +739,20 @@ tfe_status tfe_head_create(const void *w_pref, int32_t V, int32_t d, int32_t max
     h->rows_per_cta = (int32_t)((((int64_t)V + ctas - 1) / ctas + 7) / 8 * 8);
     h->grid = (int32_t)(((int64_t)V + h->rows_per_cta - 1) / h->rows_per_cta);
     h->tail_rows = h->rows_per_cta % HEAD_TILE_M;
-    if (!make_map(&h->map_w, w_pref, (uint64_t)V, (uint64_t)d, HEAD_TILE_M)) return fail(TFE_ERR_CUDA);
-    if (!make_map(&h->map_w_tail, w_pref, (uint64_t)V, (uint64_t)d, h->tail_rows ? (uint32_t)h->tail_rows : 8u))
-        return fail(TFE_ERR_CUDA);
     h->ld = ((int64_t)V + 3) / 4 * 4;
     h->tiles_per_cta = (h->rows_per_cta + HEAD_TILE_M - 1) / HEAD_TILE_M;
+    {
+        const int64_t n_pieces = (int64_t)h->grid * h->tiles_per_cta * (d / HEAD_TILE_K);
+        if (n_pieces * HEAD_TILE_M > 0x7FFFFFFFll) return fail(TFE_ERR_INVALID_ARG);      // TMA coordinates are 32-bit
+        if (cudaMalloc(&h->d_w_tiled, (size_t)n_pieces * HEAD_TILE_M * 128) != cudaSuccess) return fail(TFE_ERR_CUDA);
+        tfe_head_retile_kernel<<<h->sm_count * 8, 256>>>(static_cast<const uint4 *>(w_pref), static_cast<uint4 *>(h->d_w_tiled), V, d,
+                                                        h->rows_per_cta, h->tiles_per_cta, n_pieces);
+        if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return fail(TFE_ERR_CUDA);
+        const uint64_t rows = (uint64_t)n_pieces * HEAD_TILE_M;
+        if (!make_map(&h->map_w, h->d_w_tiled, rows, HEAD_TILE_K, HEAD_TILE_M)) return fail(TFE_ERR_CUDA);
+        if (!make_map(&h->map_w_tail, h->d_w_tiled, rows, HEAD_TILE_K, h->tail_rows ? (uint32_t)h->tail_rows : 8u))
+            return fail(TFE_ERR_CUDA);
+    }
     h->n_fine = h->grid * h->tiles_per_cta * 4;
     if (h->n_fine > HEAD_MAX_FINE) return fail(TFE_ERR_INVALID_ARG);      // a vocabulary beyond 148 x 14 tiles of 128 rows
     const size_t nb = (size_t)max_batch;
@@ -744,6 +777,7 @@ void tfe_head_destroy(tfe_head *h)
     (void)cudaGetDevice(&prev);
     (void)cudaSetDevice(h->device);
     (void)cudaDeviceSynchronize();
+    if (h->d_w_tiled) (void)cudaFree(h->d_w_tiled);
     if (h->d_logits) (void)cudaFree(h->d_logits);
     if (h->d_lse) (void)cudaFree(h->d_lse);
     if (h->d_status) (void)cudaFree(h->d_status);
