@@ -1014,7 +1014,8 @@ def run_loop(a, dev, rank):
     cnt = torch.zeros(2, dtype=torch.int32, device=dev)
     applied = torch.empty(budget, dtype=torch.uint8, device=dev)
     n_applied = torch.zeros(1, dtype=torch.int32, device=dev)
-    installed_total = torch.zeros(1, dtype=torch.int64, device=dev)
+    installed_total = torch.zeros(1, dtype=torch.int32, device=dev)
+    pool_idx = torch.empty(budget, dtype=torch.int32, device=dev)
     tfe.tfe_cache_select_victims_async(eng.ctx, budget, half_life)
     slots_ptr, _ = tfe.tfe_cache_select_victims_device(eng.ctx)
     slots_dev = _device_view(slots_ptr, (budget,), "<i4", dev)
@@ -1029,7 +1030,6 @@ def run_loop(a, dev, rank):
         tfe.tfe_head_topk(head.handle, sess.outs[v], B, K, t_tok, t_prob, st)
 
     def stage_candidates(v, st):
-        ph.fill_(-1)                                             # unwritten entries are no phrases
         tfe.tfe_prefetch_candidates(eng.ctx, hist[v], B, H, t_tok, t_prob, K, out_phrase=ph, out_tier=tr, out_score=sc,
                                     out_src=sr, out_count=cnt, budget=budget, stream=st)
 
@@ -1037,9 +1037,10 @@ def run_loop(a, dev, rank):
         tfe.tfe_cache_select_victims_async(eng.ctx, budget, half_life, st)
 
     def stage_install(v, st):
-        torch.index_select(pool, 0, torch.remainder(ph.clamp(min=0), pool_n).long(), out=src)    # stands in for the fetch
+        torch.bitwise_and(ph, pool_n - 1, out=pool_idx)          # any row for "no phrase": the installation skips it
+        torch.index_select(pool, 0, pool_idx, out=src)           # stands in for the fetch
         tfe.tfe_cache_install_device(eng.ctx, budget, ph, src, slots_dev, applied, n_applied, st)
-        installed_total.add_(n_applied.long())
+        installed_total.add_(n_applied)
 
     stages = [("lookup_inject", stage_lookup), ("head_topk", stage_head), ("prefetch_candidates", stage_candidates),
               ("select_victims", stage_victims), ("gather + install_device", stage_install)]

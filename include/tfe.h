@@ -149,7 +149,7 @@ tfe_status tfe_cache_install(tfe_ctx *ctx, int32_t n, const uint32_t *phrase_ids
  *   dst_slots      DEVICE int32 [n]
  *   applied        DEVICE uint8 [n], receives 1 / 0 per entry, or NULL
  *   applied_count  DEVICE uint32, receives the number applied, or NULL
- * Asynchronous on `stream`, four kernel launches, never synchronises.  The first call on a context
+ * Asynchronous on `stream`, two kernel launches, never synchronises.  The first call on a context
  * allocates 4 bytes per phrase and per slot (with a device synchronisation: make it outside a stream
  * capture); every later call keeps no state on the host and may be captured into a CUDA graph and
  * replayed with new contents in the same buffers.  Once this function has been used, the host-side
@@ -352,7 +352,9 @@ typedef struct {
  * s = (p * r) * c in fp32, dropped if s <= 0.  Outputs (DEVICE, `budget` entries each): phrase id,
  * tier (TFE_FLAG_HOST_MISS / TFE_FLAG_SSD_MISS), s, and source b*K + k of the `budget` best, in
  * descending s, equal s in ascending (b, k, order); duplicates of one phrase are kept.
- * out_count DEVICE uint32 [2]: entries written, candidates found before the cut.
+ * out_count DEVICE uint32 [2]: entries written, candidates found before the cut.  The phrase ids
+ * beyond the entries written are set to TFE_NO_PHRASE (the other arrays are left as they were), so
+ * the whole array can be handed to tfe_cache_install_device, which skips ids that are no phrase.
  * Asynchronous on `stream`, two kernel launches; a first call with more entries than any before
  * grows context buffers.  Errors: INVALID_ARG, CUDA.
  */

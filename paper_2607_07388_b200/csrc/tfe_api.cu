@@ -115,6 +115,7 @@ struct tfe_ctx {
 
     // tfe_cache_install_device: stamps per phrase and per slot, the call counter, the applied count
     uint32_t *d_phrase_stamp = nullptr, *d_slot_stamp = nullptr, *d_inst_count = nullptr;
+    uint8_t *d_inst_flags = nullptr;        // which entries of the device-side installation in flight are applied
 
     // host-buffer variant staging
     int32_t *d_h_tokens = nullptr;
@@ -400,7 +401,7 @@ void tfe_destroy(tfe_ctx *c)
     free_dev(c->d_h_tokens); free_dev(c->d_h_hidden); free_dev(c->d_h_out);
     free_dev(c->d_h_phrase); free_dev(c->d_h_slot); free_dev(c->d_h_flag);
     free_dev(c->d_pf_keys); free_dev(c->d_pf_phrase); free_dev(c->d_pf_tier); free_dev(c->d_pf_counter);
-    free_dev(c->d_phrase_stamp); free_dev(c->d_slot_stamp); free_dev(c->d_inst_count);
+    free_dev(c->d_phrase_stamp); free_dev(c->d_slot_stamp); free_dev(c->d_inst_count); free_dev(c->d_inst_flags);
     free_dev(c->d_slot_stats); free_dev(c->d_epoch); free_dev(c->d_vs_fin);
     free_dev(c->d_vs_keys); free_dev(c->d_vs_state); free_dev(c->d_vs_list); free_dev(c->d_vs_slots);
     if (c->hb_in) (void)cudaStreamDestroy(c->hb_in);
@@ -788,6 +789,7 @@ tfe_status tfe_cache_install_device(tfe_ctx *c, int32_t n, const uint32_t *phras
         CU(cudaMalloc(&c->d_phrase_stamp, std::max<size_t>(4, (size_t)N * 4)));
         CU(cudaMalloc(&c->d_slot_stamp, std::max<size_t>(4, (size_t)C * 4)));
         CU(cudaMalloc(&c->d_inst_count, sizeof(uint32_t)));
+        CU(cudaMalloc(&c->d_inst_flags, TFE_INSTALL_DEVICE_MAX));
         // zero once; every call leaves them zeroed again
         CU(cudaMemsetAsync(c->d_phrase_stamp, 0, std::max<size_t>(4, (size_t)N * 4), stream));
         CU(cudaMemsetAsync(c->d_slot_stamp, 0, std::max<size_t>(4, (size_t)C * 4), stream));
@@ -800,13 +802,10 @@ tfe_status tfe_cache_install_device(tfe_ctx *c, int32_t n, const uint32_t *phras
     p.phrase_stamp = c->d_phrase_stamp; p.slot_stamp = c->d_slot_stamp;
     p.applied = applied; p.count = applied_count ? applied_count : c->d_inst_count;
     p.slot_stats = c->d_slot_stats; p.epoch = c->d_epoch;
-    CU(cudaMemsetAsync(p.count, 0, sizeof(uint32_t), stream));
-    const unsigned blocks = (unsigned)((n + 255) / 256);
-    CU(launch_overlapped(tfe_install_claim_kernel<0>, dim3(blocks), dim3(256), stream, p));
-    CU(launch_overlapped(tfe_install_claim_kernel<1>, dim3(blocks), dim3(256), stream, p));
+    p.flags = c->d_inst_flags;
+    CU(launch_overlapped(tfe_install_claim_kernel, dim3(1), dim3(TFE_INSTALL_CLAIM_THREADS), stream, p));
     CU(launch_overlapped(tfe_install_device_kernel, dim3((unsigned)((n + TFE_WARPS_PER_BLOCK - 1) / TFE_WARPS_PER_BLOCK)),
                          dim3(TFE_BLOCK_THREADS), stream, p));
-    CU(launch_overlapped(tfe_install_clear_kernel, dim3(blocks), dim3(256), stream, p));
     c->mirror_ready = false;        // the host copy of the residency state is stale now; fetched again when needed
     c->device_installs = true;
     return TFE_OK;

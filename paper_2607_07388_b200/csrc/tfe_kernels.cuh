@@ -1043,10 +1043,11 @@ tfe_install_kernel(ulonglong2 *index, const uint32_t *phrase_pos, uint32_t *slot
 // 4096 - k, so the smallest k wins; the stamps are zero between calls (the last kernel puts back the
 // ones this call touched), so the call keeps no state on the host and can be replayed from a graph.
 //
-//   tfe_install_claim_kernel<0>  every entry stamps its phrase
-//   tfe_install_claim_kernel<1>  every candidate stamps its slot
+//   tfe_install_claim_kernel     ONE block (a batch is at most 4,096 entries, four per thread), four steps with a
+//                                block barrier between them: every entry stamps its phrase; every candidate stamps
+//                                its slot; every entry learns whether it won both (flag, count); the stamps this
+//                                call wrote go back to zero
 //   tfe_install_device_kernel    one warp per entry: the winners install (as tfe_install_kernel)
-//   tfe_install_clear_kernel     the stamps this call wrote go back to zero
 #define TFE_INSTALL_DEVICE_MAX 4096
 
 struct TfeInstallDeviceParams {
@@ -1064,46 +1065,71 @@ struct TfeInstallDeviceParams {
     uint32_t *phrase_stamp;         // [n_phrases]
     uint32_t *slot_stamp;           // [gpu_slots]
     uint8_t *applied;               // [n] or nullptr
-    uint32_t *count;                // entries applied (cleared by the host side before the launches)
+    uint8_t *flags;                 // [TFE_INSTALL_DEVICE_MAX] the same, owned by the context: claim kernel -> install kernel
+    uint32_t *count;                // entries applied (written by the claim kernel)
     uint2 *slot_stats;
     const uint32_t *epoch;
 };
 
-__device__ __forceinline__ bool tfe_install_candidate(const TfeInstallDeviceParams &p, int k)
-{
-    const uint32_t id = p.ids[k];
-    const int32_t dst = p.dst_slots[k];
-    if (id >= p.n_phrases || dst < 0 || (int64_t)dst >= p.gpu_slots) return false;
-    if ((int32_t)(uint32_t)p.index[p.phrase_pos[id]].y >= 0) return false;          // resident before the call
-    return __ldcg(p.phrase_stamp + id) == (uint32_t)(TFE_INSTALL_DEVICE_MAX - k);
-}
+#define TFE_INSTALL_CLAIM_THREADS 1024
 
-template <int STAGE>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(TFE_INSTALL_CLAIM_THREADS)
 tfe_install_claim_kernel(const TfeInstallDeviceParams p)
 {
+    constexpr int PER = TFE_INSTALL_DEVICE_MAX / TFE_INSTALL_CLAIM_THREADS;
+    __shared__ uint32_t s_warp[TFE_INSTALL_CLAIM_THREADS / 32];
     tfe_grid_dependency_sync();
-    const int k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= p.n) return;
-    const uint32_t stamp = (uint32_t)(TFE_INSTALL_DEVICE_MAX - k);         // 1..4096: never the cleared value
-    if (STAGE == 0) {
-        const uint32_t id = p.ids[k];
-        if (id < p.n_phrases) atomicMax(p.phrase_stamp + id, stamp);
-    } else {
-        if (tfe_install_candidate(p, k)) atomicMax(p.slot_stamp + p.dst_slots[k], stamp);
+    uint32_t id[PER];
+    int32_t dst[PER];
+    bool valid[PER], cand[PER];
+    // ---- every entry stamps its phrase: 4096 - k, so the smallest k wins (never the cleared value 0)
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+        const int k = j * TFE_INSTALL_CLAIM_THREADS + threadIdx.x;
+        valid[j] = false; id[j] = 0; dst[j] = -1;
+        if (k < p.n) {
+            id[j] = p.ids[k];
+            dst[j] = p.dst_slots[k];
+            valid[j] = id[j] < p.n_phrases;
+            if (valid[j]) atomicMax(p.phrase_stamp + id[j], (uint32_t)(TFE_INSTALL_DEVICE_MAX - k));
+        }
     }
-}
-
-__global__ void __launch_bounds__(256)
-tfe_install_clear_kernel(const TfeInstallDeviceParams p)
-{
-    tfe_grid_dependency_sync();
-    const int k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= p.n) return;
-    const uint32_t id = p.ids[k];
-    const int32_t dst = p.dst_slots[k];
-    if (id < p.n_phrases) p.phrase_stamp[id] = 0;
-    if (dst >= 0 && (int64_t)dst < p.gpu_slots) p.slot_stamp[dst] = 0;
+    __syncthreads();
+    // ---- every candidate stamps its slot
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+        const int k = j * TFE_INSTALL_CLAIM_THREADS + threadIdx.x;
+        cand[j] = valid[j] && dst[j] >= 0 && (int64_t)dst[j] < p.gpu_slots &&
+                  (int32_t)(uint32_t)p.index[p.phrase_pos[id[j]]].y < 0 &&                  // not resident before the call
+                  __ldcg(p.phrase_stamp + id[j]) == (uint32_t)(TFE_INSTALL_DEVICE_MAX - k);
+        if (cand[j]) atomicMax(p.slot_stamp + dst[j], (uint32_t)(TFE_INSTALL_DEVICE_MAX - k));
+    }
+    __syncthreads();
+    // ---- who won both
+    uint32_t mine = 0;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+        const int k = j * TFE_INSTALL_CLAIM_THREADS + threadIdx.x;
+        if (k >= p.n) continue;
+        const bool apply = cand[j] && __ldcg(p.slot_stamp + dst[j]) == (uint32_t)(TFE_INSTALL_DEVICE_MAX - k);
+        p.flags[k] = apply ? 1 : 0;
+        if (p.applied) p.applied[k] = apply ? 1 : 0;
+        mine += apply;
+    }
+    mine = __reduce_add_sync(0xFFFFFFFFu, mine);
+    if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = mine;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t total = 0;
+        for (int w = 0; w < TFE_INSTALL_CLAIM_THREADS / 32; ++w) total += s_warp[w];
+        *p.count = total;
+    }
+    // ---- the stamps go back to zero (every thread is past its last look at them)
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+        if (valid[j]) p.phrase_stamp[id[j]] = 0;
+        if (dst[j] >= 0 && (int64_t)dst[j] < p.gpu_slots) p.slot_stamp[dst[j]] = 0;
+    }
 }
 
 __global__ void __launch_bounds__(TFE_BLOCK_THREADS)
@@ -1113,15 +1139,7 @@ tfe_install_device_kernel(const TfeInstallDeviceParams p)
     const int lane = threadIdx.x & 31;
     const int k = blockIdx.x * TFE_WARPS_PER_BLOCK + (threadIdx.x >> 5);
     if (k >= p.n) return;
-    bool apply = false;
-    if (lane == 0) {
-        apply = tfe_install_candidate(p, k) &&
-                __ldcg(p.slot_stamp + p.dst_slots[k]) == (uint32_t)(TFE_INSTALL_DEVICE_MAX - k);
-        if (p.applied) p.applied[k] = apply ? 1 : 0;
-        if (apply) atomicAdd(p.count, 1u);
-    }
-    apply = __shfl_sync(0xFFFFFFFFu, apply, 0);
-    if (!apply) return;
+    if (__ldcg(p.flags + k) == 0) return;
     const uint32_t id = p.ids[k];
     const int32_t dst = p.dst_slots[k];
     if (lane == 0) {
@@ -1311,6 +1329,8 @@ tfe_prefetch_select_kernel(const unsigned long long *keys, const uint32_t *entry
         out_score[i] = __uint_as_float((uint32_t)(k >> 32));
         out_src[i] = tfe_div(idx, div_orders);
     }
+    // the rest of the budget names no phrase, so that the arrays can go to tfe_cache_install_device whole
+    for (uint32_t i = take + threadIdx.x; i < budget; i += blockDim.x) out_phrase[i] = 0xFFFFFFFFu;
     __syncthreads();
     if (threadIdx.x == 0) {
         out_count[0] = take;

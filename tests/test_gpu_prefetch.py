@@ -61,6 +61,7 @@ def _compare(pr, hist, cand, prob, use, budget, c_host, c_ssd):
     n = int(cnt[0].item())
     assert int(cnt[1].item()) == total and n == len(eph)
     np.testing.assert_array_equal(ph[:n].cpu().numpy().view(np.uint32), eph)
+    assert (ph[n:budget].cpu().numpy().view(np.uint32) == 0xFFFFFFFF).all()      # the unused part of the budget: no phrase
     np.testing.assert_array_equal(tr[:n].cpu().numpy(), etr)
     np.testing.assert_array_equal(sr[:n].cpu().numpy().view(np.uint32), esr)
     np.testing.assert_array_equal(sc[:n].cpu().numpy().view(np.uint32), esc.view(np.uint32))
