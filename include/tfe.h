@@ -417,7 +417,7 @@ void       tfe_head_destroy(tfe_head *head);
  * K <= V.  Outputs DEVICE: cand_tokens int32 [B][K], cand_prob float [B][K], per sequence in
  * descending probability, equal logits in ascending token id.  Logits are bf16 products
  * accumulated in fp32 (tensor cores); selection and softmax in fp32.  Asynchronous on `stream`,
- * three kernel launches, never synchronises.  Errors: INVALID_ARG, CUDA, INTERNAL.
+ * two kernel launches, never synchronises.  Errors: INVALID_ARG, CUDA, INTERNAL.
  */
 tfe_status tfe_head_topk(tfe_head *head, const void *hidden, int32_t B, int32_t K, int32_t *cand_tokens,
                          float *cand_prob, void *stream);
