@@ -1086,6 +1086,7 @@ def run_loop(a, dev, rank):
                        "rows": "candidate rows gathered from a pool staged on the device (the DRAM / SSD read is outside the library)"},
             "us_per_stage_alone": per_stage, "sum_of_stages_us": sum(per_stage.values()),
             "installed_per_step": n_inst / ((reps + 3) * nbuf), "head_status": status,
+            "candidates_last_step": {"written": int(cnt[0].item()), "found": int(cnt[1].item())},
             "parity": "the chain is checked against the oracle in tests/test_gpu_install_device.py (not in this mode: "
                       "fp64 logits over the whole vocabulary take seconds per step on the host)"}))
     head.close()
