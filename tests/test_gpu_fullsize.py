@@ -170,6 +170,39 @@ def test_config4_full_size_install_then_lookup(H):
     want = synth.procedural_bf16_np(ora.slot_owner[pick], w.d, synth.ROW_TAG, synth.ROW_SHIFT)
     got = H.bits_from_bf16_tensor(bp.rows_gpu[torch.from_numpy(pick).to(H.DEV)])
     np.testing.assert_array_equal(got, want)
+
+    # ---- retention ranking over all 16,777,216 slots (sampled threshold, one pass, exact result): bookkeeping of
+    # three lookups, victims for several (n, half-life), an installation into the victims, victims again
+    eng.cache_policy_enable()
+    ora.freq[:] = 0; ora.last[:] = 0; ora.epoch = 0          # what enabling does on the device
+    for step in range(3):
+        info = bp.check(synth.make_queries(w, bp.tb, variant=step), variant=step)
+        ora.touch(info["ref"])
+    freq, last, epoch = eng.cache_stats()
+    assert epoch == ora.epoch == 3
+    np.testing.assert_array_equal(freq, ora.freq)
+    np.testing.assert_array_equal(last, ora.last)
+
+    def victims(n, hl):
+        slots, keys = eng.cache_select_victims(n, hl)
+        e_slots, e_keys = ora.cache_victims(n, hl)
+        np.testing.assert_array_equal(slots, e_slots)
+        np.testing.assert_array_equal(keys, e_keys)
+        return e_slots
+
+    for n, hl in ((4096, 2), (1, 0), (513, 1), (4095, 0)):
+        victims(n, hl)
+    dst = victims(4096, 2).copy()
+    assert (ora.slot_owner[dst] < 0).all()                   # 262,144 - 8,192 slots are still free: they go first
+    pool = np.nonzero(ora.slot_state < 0)[0]
+    ids = rng.choice(pool, 4096, replace=False).astype(np.uint32)
+    pinned = torch.from_numpy(synth.phrase_rows_np(w, ids).view(np.int16)).pin_memory()
+    eng.cache_install(ids, pinned, dst)
+    assert ora.cache_install(ids, None, dst) == 0
+    info = bp.check(synth.make_queries(w, bp.tb, variant=1), variant=1)
+    ora.touch(info["ref"])
+    nxt = victims(4096, 2)
+    assert not np.isin(nxt, dst).any()                       # freshly installed rows are not the next victims
     bp.close()
 
 
