@@ -140,7 +140,13 @@ typedef void (*lookup_kernel_t)(const TfeLookupParams);
 // packed bf16 fused multiply-add (lambda exactly a bf16 number), fp32 hidden.  11..13: the same
 // three for a call issued in several launches over query ranges (variant + kVarRanged).  14..19: those six
 // compiled for rows of several chunks (variant + kVarWide: half the registers in flight per lane, four blocks per SM).
-enum { kVarLongest = 8, kVarLongestPacked = 9, kVarLongestF32 = 10, kVarRanged = 3, kVarWide = 6, kVarCount = 20 };
+// 20, 21: LONGEST / COSINE on rows one trip covers (bf16 / fp32 hidden): the LONGEST kernel with the gate.
+enum { kVarLongest = 8, kVarLongestPacked = 9, kVarLongestF32 = 10, kVarRanged = 3, kVarWide = 6, kVarLongestCos = 20, kVarCount = 22 };
+constexpr int kCosSteps = 128;         // 16-byte steps of h per row up to which kVarLongestCos applies ...
+constexpr int64_t kCosMinQueries = 2048;   // ... and the call size from which
+
+// The variants that can run a call in pieces and have a wide-row form.
+inline bool is_longest_const(int variant) { return variant >= kVarLongest && variant < kVarLongestCos; }
 constexpr int kWideSteps = 384;        // 16-byte steps of h per row from which the kVarWide variants are used
 
 lookup_kernel_t pick_kernel(int variant)
@@ -158,6 +164,7 @@ lookup_kernel_t pick_kernel(int variant)
         tfe_lookup_inject_longest_kernel<1, false, false, 2>,
         tfe_lookup_inject_longest_kernel<0, false, true, 2>,  tfe_lookup_inject_longest_kernel<0, true, true, 2>,
         tfe_lookup_inject_longest_kernel<1, false, true, 2>,
+        tfe_lookup_inject_longest_kernel<0, false, false, 4, true>, tfe_lookup_inject_longest_kernel<1, false, false, 4, true>,
     };
     return table[variant];
 }
@@ -823,13 +830,15 @@ tfe_status tfe_cache_install_device(tfe_ctx *c, int32_t n, const uint32_t *phras
 namespace {
 
 // Variant of the lookup kernel a call runs: the LONGEST / CONST kernels where they apply.
-int lookup_variant(const tfe_ctx *c, const tfe_inject_params *prm)
+int lookup_variant(const tfe_ctx *c, const tfe_inject_params *prm, int64_t Q)
 {
     const bool all = prm->policy == TFE_POLICY_ALL, cos = prm->gate == TFE_GATE_COSINE;
     uint32_t lam_bits;
     std::memcpy(&lam_bits, &prm->lambda, sizeof lam_bits);
     const bool lam_is_bf16 = (lam_bits & 0xFFFFu) == 0 && (lam_bits & 0x7F800000u) != 0x7F800000u;
     const int ht = c->cfg.hidden_dtype;
+    // (a decode-sized call is a little quicker in the general kernel: 5.1 against 5.4 us at 64 positions)
+    if (!all && cos && c->cfg.d / (ht == 0 ? 8 : 4) <= kCosSteps && Q >= kCosMinQueries) return kVarLongestCos + ht;
     return (all || cos) ? ht * 4 + (all ? 2 : 0) + (cos ? 1 : 0)
                         : (ht == 1 ? kVarLongestF32 : (lam_is_bf16 ? kVarLongestPacked : kVarLongest));
 }
@@ -909,10 +918,10 @@ tfe_status lookup_inject_range(tfe_ctx *c, const int32_t *tokens, int32_t B, int
     uint32_t lam_bits;
     std::memcpy(&lam_bits, &prm->lambda, sizeof lam_bits);
     const bool ranged = q_lo != 0 || q_hi != Q || !finalize;
-    int variant = lookup_variant(c, prm);
-    if (ranged && variant < kVarLongest) return TFE_ERR_INTERNAL;
+    int variant = lookup_variant(c, prm, Q);
+    if (ranged && !is_longest_const(variant)) return TFE_ERR_INTERNAL;
     if (ranged) variant += kVarRanged;
-    if (variant >= kVarLongest && c->cfg.d / (c->cfg.hidden_dtype == 0 ? 8 : 4) >= kWideSteps) variant += kVarWide;
+    if (is_longest_const(variant) && c->cfg.d / (c->cfg.hidden_dtype == 0 ? 8 : 4) >= kWideSteps) variant += kVarWide;
     const int64_t Qr = q_hi - q_lo;
     int64_t qb, grid;
     lookup_geometry(c, variant, Qr, &qb, &grid);
@@ -987,14 +996,14 @@ tfe_status tfe_lookup_inject_host(tfe_ctx *c, const int32_t *tokens, int32_t B, 
         c->hb_tok_cap = tok_cap; c->hb_q_cap = q_cap; c->hb_ent_cap = e_cap;
     }
     const size_t row_bytes = (size_t)c->cfg.d * (c->cfg.hidden_dtype == 0 ? 2 : 4);
-    const int variant = lookup_variant(c, prm);
+    const int variant = lookup_variant(c, prm, Q);
     // The LONGEST / CONST kernels can run a call in pieces, so the hidden states go through a
     // three-stage pipeline: piece k's kernel runs while piece k+1 comes in and piece k-1 goes
     // back.  Other variants take one launch between the copies.
     int64_t cut[tfe_ctx::kPipeMaxChunks + 1];
     int n_chunks = 1;
     cut[0] = 0; cut[1] = Q;
-    if (variant >= kVarLongest && hid_bytes >= 2 * (size_t)TFE_HOST_CHUNK_BYTES)
+    if (is_longest_const(variant) && hid_bytes >= 2 * (size_t)TFE_HOST_CHUNK_BYTES)
         n_chunks = plan_pieces(Q, (int64_t)row_bytes, cut);
     if (n_chunks == 1) {
         CU(cudaMemcpyAsync(c->d_h_tokens, tokens, (size_t)n_tok * 4, cudaMemcpyHostToDevice, stream));
@@ -1334,8 +1343,8 @@ extern "C" tfe_status tfe_lookup_inject_noalloc(tfe_ctx *c, const int32_t *token
 
     uint32_t lam_bits;
     std::memcpy(&lam_bits, &prm->lambda, sizeof lam_bits);
-    int variant = lookup_variant(c, prm);
-    if (variant >= kVarLongest && c->cfg.d / (c->cfg.hidden_dtype == 0 ? 8 : 4) >= kWideSteps) variant += kVarWide;
+    int variant = lookup_variant(c, prm, Q);
+    if (is_longest_const(variant) && c->cfg.d / (c->cfg.hidden_dtype == 0 ? 8 : 4) >= kWideSteps) variant += kVarWide;
     int64_t qb, grid;
     lookup_geometry(c, variant, Q, &qb, &grid);
     TfeLookupParams p{};

@@ -809,10 +809,14 @@ tfe_lookup_inject_kernel(const TfeLookupParams p)
 // UNROLL: 16-byte vectors of h (and of the row) a lane holds at a time.  4: a 1,024-element row is in flight whole,
 // 80 registers, three blocks per SM.  2: 64 registers, four blocks per SM -- for rows of several chunks, where
 // a warp walks chunk after chunk and a third more warps pays (8 KB rows: 278 -> 254 us per 65,536-token call).
-template <int HT, bool PACKED, bool RANGED, int UNROLL>
+template <int HT, bool PACKED, bool RANGED, int UNROLL, bool COS = false>
 __global__ void __launch_bounds__(TFE_BLOCK_THREADS, UNROLL == 4 ? TFE_MIN_BLOCKS : TFE_MIN_BLOCKS + 1)
 tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
 {
+    // COS: the gate lambda * sigmoid(cos(h, m)) instead of lambda.  The host uses it only for rows one trip covers
+    // (at most 32 * UNROLL steps), so the row and the hidden state are in registers when the three dot products
+    // are formed, and only without the packed arithmetic and without ranges.
+    static_assert(!COS || (!PACKED && !RANGED && UNROLL == 4), "the gated form is one instantiation per hidden type");
     constexpr int VN = TfeVec<HT>::N;
     static_assert(!PACKED || HT == 0, "packed bf16 path needs bf16 hidden states");
 
@@ -956,6 +960,25 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
                         }
                     }
                 }
+                float gate = p.lambda;
+                if constexpr (COS) {
+                    if (sl >= 0) {
+                        float sa = 0.f, sb = 0.f, sc = 0.f;      // <h,m>, <h,h>, <m,m>: the general kernel's order of terms
+#pragma unroll
+                        for (int u = 0; u < UNROLL; ++u) {
+                            if (u * 32 + lane >= steps) continue;
+                            float x[VN], m[VN];
+                            unpack_hidden<HT>(hv[u], x);
+                            unpack_row<HT>(rv[u], m);
+#pragma unroll
+                            for (int e = 0; e < VN; ++e) {
+                                sa = fmaf(x[e], m[e], sa); sb = fmaf(x[e], x[e], sb); sc = fmaf(m[e], m[e], sc);
+                            }
+                        }
+                        sa = warp_sum(sa); sb = warp_sum(sb); sc = warp_sum(sc);
+                        gate = p.lambda / (1.f + __expf(-sa * rsqrtf(fmaf(sb, sc, 1e-12f))));
+                    }
+                }
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u) {
                     const int k = s0 + u * 32 + lane;
@@ -975,7 +998,7 @@ tfe_lookup_inject_longest_kernel(const TfeLookupParams p)
                         unpack_hidden<HT>(hv[u], x);
                         unpack_row<HT>(rv[u], m);
 #pragma unroll
-                        for (int e = 0; e < VN; ++e) y[e] = fmaf(p.lambda, m[e], x[e]);
+                        for (int e = 0; e < VN; ++e) y[e] = fmaf(gate, m[e], x[e]);
                         store_hidden<HT>(orow, k, y);
                     }
                 }

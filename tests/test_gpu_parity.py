@@ -204,6 +204,7 @@ def test_overfull_index_is_refused(H):
     (2048, 0, 0.5, (2, 3)),         # two chunks per row
     (2560, 1, 0.3, (2, 3, 4)),      # fp32 hidden states, five chunks per row
     (64, 0, 2.0, (2, 3)),           # short rows
+    (512, 1, 0.7, (2, 3)),          # fp32 hidden states, one trip per row
 ])
 def test_large_calls_all_batch_sizes(H, d, hidden, lam, orders):
     from paper_2607_07388_b200 import binding as tfe
@@ -225,6 +226,8 @@ def test_large_calls_all_batch_sizes(H, d, hidden, lam, orders):
         pr.run_and_compare(tok, h, lam=lam, in_place=True)
         pr.run_and_compare(tok, h[: w.B * (w.T - 2000)], lam=lam, q_start=2000, want_sel=False)
         pr.run_and_compare(tok, h, lam=lam, policy=1, gate=1)
+        pr.run_and_compare(tok, h, lam=lam, gate=1)           # large and narrow enough for the gated LONGEST kernel
+        pr.run_and_compare(tok, h, lam=lam, policy=1)
     cap = min(8, 32 // max(4, 2 * len(orders)))      # a query takes two lanes per order (at least four) of the warp
     assert {min(q, cap) for q in (1, 3, 5, 8)} <= seen
     pr.close()
