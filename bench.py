@@ -1391,9 +1391,9 @@ NBUF_DECODE = 32        # decode shapes: this many distinct query / hidden-state
 # N).  Reads are all there (109.1 MB: ids, buckets, hidden states, rows); of the 67.1 MB of `out` only what the
 # L2 wrote back inside the kernel's window is counted (20.5 MB), the rest leaves the L2 after the kernel has
 # ended (under ncu, between the serialised launches; in the timed region, during the next launch).
-NCU_TRAFFIC = {"c3_prefill8x4096": {"bytes": 130_200_000, "kernel_source": "8b6f32905a70",
+NCU_TRAFFIC = {"c3_prefill8x4096": {"bytes": 129_400_000, "kernel_source": "14a5d0411d8e",
                                     "source": "profiles/lookup_inject_longest_c3_prefill8x4096.md, capture without cache "
-                                              "flushes (109.2 MB read + 21.1 MB written inside the kernel's window; the "
+                                              "flushes (109.1 MB read + 20.2 MB written inside the kernel's window; the "
                                               "other 46.6 MB of the output are written back after it)"}}
 
 
