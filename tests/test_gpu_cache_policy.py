@@ -106,6 +106,10 @@ def test_policy_off_and_argument_checks(H):
     pr.eng.cache_policy_enable()
     with pytest.raises(tfe.TfeError):
         pr.eng.cache_select_victims(tfe.VICTIMS_MAX + 1)
+    with pytest.raises(tfe.TfeError):
+        pr.eng.cache_select_victims(4, half_life=1 << 26)      # 32 half-lives must stay below 2^31 epochs
+    slots, keys = pr.eng.cache_select_victims(3, half_life=(1 << 26) - 1)
+    np.testing.assert_array_equal(slots, np.arange(3))
     slots, keys = pr.eng.cache_select_victims(0)
     assert len(slots) == 0
     # nothing looked up yet: every owned slot has freq 0, age 0 -> key 65535, ascending slot order
