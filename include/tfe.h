@@ -275,8 +275,8 @@ tfe_status tfe_miss_list_device(tfe_ctx *ctx, const uint32_t **q_idx, const uint
  * stores the call's epoch in `last` for every GPU-tier slot it injects from, and every
  * tfe_cache_install sets {freq, last} = {1, epoch} for the slots it fills.  The epoch is a device
  * counter of completed lookups (a replayed launch advances it like a fresh one).  Calling it
- * again clears the counters and the epoch.  Allocates 12 bytes per GPU-tier slot; waits for the
- * device.  Launches recorded earlier (a captured CUDA graph) keep the arguments they were
+ * again clears the counters and the epoch.  Allocates 8 bytes per GPU-tier slot and 8.2 MiB of work
+ * space for the selection on the first call; waits for the device then.  Launches recorded earlier (a captured CUDA graph) keep the arguments they were
  * recorded with and do no bookkeeping; record them again after enabling.
  * Errors: INVALID_ARG, CUDA.
  */
